@@ -1,0 +1,186 @@
+"""FP64 oracle of the encoder, predictor, loss, gradient and optimiser.
+
+TEST INFRASTRUCTURE ONLY -- see oracle/__init__.py.  Dense algebra is numpy matmul in
+float64; aggregation and samplers come from oracle/sparse.py.  The backward pass is
+written out by hand from the chain rule (no autograd).
+"""
+from __future__ import annotations
+
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+from . import sparse
+
+
+def split_params(arch: str, dims: Sequence[int], params: np.ndarray):
+    """Views into the flat parameter vector.  Per layer k (input F_k, output F_{k+1}):
+    gcn : W [F_k, F_{k+1}] row-major, then b [F_{k+1}]
+    sage: W_self [F_k, F_{k+1}], W_neigh [F_k, F_{k+1}], then b [F_{k+1}]."""
+    out, o = [], 0
+    for k in range(len(dims) - 1):
+        fi, fo = dims[k], dims[k + 1]
+        layer = {}
+        if arch == "sage":
+            layer["W_self"] = params[o:o + fi * fo].reshape(fi, fo); o += fi * fo
+            layer["W_neigh"] = params[o:o + fi * fo].reshape(fi, fo); o += fi * fo
+        else:
+            layer["W"] = params[o:o + fi * fo].reshape(fi, fo); o += fi * fo
+        layer["b"] = params[o:o + fo]; o += fo
+        out.append(layer)
+    assert o == params.shape[0], "parameter vector has the wrong length"
+    return out
+
+
+def _block_as_global_csr(n: int, frontier: np.ndarray, ptr: np.ndarray, cols: np.ndarray):
+    counts = np.zeros(n, dtype=np.int64)
+    counts[frontier] = np.diff(ptr)
+    rowptr = np.zeros(n + 1, dtype=np.int64)
+    np.cumsum(counts, out=rowptr[1:])
+    return rowptr, cols
+
+
+def _layer_graphs(g, n_layers: int, blocks):
+    """Per layer l = 1..K: (rowptr, col, w, active_rows or None).
+    Full-graph training uses the loaded graph at every layer.  With a sampled computational
+    graph, layer l works on hop h = K - l + 1: rows F_{h-1} aggregate their sampled neighbours."""
+    if blocks is None:
+        return [(g.rowptr, g.col, g.w, None)] * n_layers
+    frontiers, blks = blocks
+    out = []
+    for l in range(1, n_layers + 1):
+        h = n_layers - l + 1
+        ptr, cols = blks[h - 1]
+        rp, cc = _block_as_global_csr(g.n, frontiers[h - 1], ptr, cols)
+        out.append((rp, cc, None, frontiers[h - 1]))
+    return out
+
+
+def forward(g, X: np.ndarray, params: np.ndarray, arch: str, dims: Sequence[int], blocks=None):
+    """K-layer encoder (Eq. 1).  Layer k: A = AGG(H^(k-1)) [gcn] or [H^(k-1) | mean] [sage];
+    Z = A W + b; H^(k) = ReLU(Z) for k < K and Z for k = K.  Returns the per-layer cache."""
+    K = len(dims) - 1
+    P = split_params(arch, dims, np.asarray(params, dtype=np.float64))
+    H = np.asarray(X, dtype=np.float64)
+    cache = {"H": [H], "M": [], "Z": [], "graphs": _layer_graphs(g, K, blocks)}
+    mode = "gcn" if arch == "gcn" else "mean"
+    for k in range(K):
+        rp, cc, w, act = cache["graphs"][k]
+        M = sparse.aggregate(mode, g.n, rp, cc, w if arch == "gcn" else None, H)
+        if arch == "gcn":
+            Z = M @ P[k]["W"] + P[k]["b"]
+        else:
+            Z = H @ P[k]["W_self"] + M @ P[k]["W_neigh"] + P[k]["b"]
+        Hn = np.maximum(Z, 0.0) if k < K - 1 else Z
+        if act is not None:  # rows outside the frontier are not part of the computational graph
+            keep = np.zeros(g.n, dtype=bool)
+            keep[act] = True
+            Z = np.where(keep[:, None], Z, 0.0)
+            Hn = np.where(keep[:, None], Hn, 0.0)
+        cache["M"].append(M)
+        cache["Z"].append(Z)
+        cache["H"].append(Hn)
+        H = Hn
+    return cache
+
+
+def bce_with_logits(s: np.ndarray, y: np.ndarray):
+    """Per-edge binary cross-entropy of label y and probability sigmoid(s), in the
+    overflow-free form  max(s,0) - s*y + log(1 + exp(-|s|)), and d/ds = sigmoid(s) - y."""
+    ell = np.maximum(s, 0.0) - s * y + np.log1p(np.exp(-np.abs(s)))
+    sig = np.where(s >= 0, 1.0 / (1.0 + np.exp(-np.abs(s))), np.exp(-np.abs(s)) / (1.0 + np.exp(-np.abs(s))))
+    return ell, sig - y
+
+
+def train_step(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst, blocks=None):
+    """One training step of Algorithm 1 for one worker: scores of Eq. 2 (dot product) for
+    positives (label 1) and negatives (label 0), loss L = (1/N) sum ell with N = |P| + |N|,
+    and the gradient with respect to every parameter in the flat layout."""
+    K = len(dims) - 1
+    P = split_params(arch, dims, np.asarray(params, dtype=np.float64))
+    cache = forward(g, X, params, arch, dims, blocks)
+    HK = cache["H"][K]
+    src = np.concatenate([pos_src, neg_src]).astype(np.int32)
+    dst = np.concatenate([pos_dst, neg_dst]).astype(np.int32)
+    y = np.concatenate([np.ones(len(pos_src)), np.zeros(len(neg_src))])
+    s = np.einsum("ij,ij->i", HK[src], HK[dst])
+    ell, dls = bce_with_logits(s, y)
+    N = s.shape[0]
+    loss = ell.sum() / N
+    gs = dls / N
+    dH = sparse.edge_grad(HK, src, dst, gs)
+    dHK = dH
+
+    grads = np.zeros(params.shape[0], dtype=np.float64)
+    G = split_params(arch, dims, grads)
+    mode = "gcn" if arch == "gcn" else "mean"
+    for k in range(K - 1, -1, -1):
+        rp, cc, w, act = cache["graphs"][k]
+        dZ = dH if k == K - 1 else dH * (cache["Z"][k] > 0.0)
+        if act is not None:
+            keep = np.zeros(g.n, dtype=bool)
+            keep[act] = True
+            dZ = np.where(keep[:, None], dZ, 0.0)
+        Hprev, M = cache["H"][k], cache["M"][k]
+        G[k]["b"][:] = dZ.sum(axis=0)
+        if arch == "gcn":
+            G[k]["W"][:] = M.T @ dZ
+            dM = dZ @ P[k]["W"].T
+            dH = sparse.aggregate_backward(mode, g.n, rp, cc, w, dM) if k > 0 else None
+        else:
+            G[k]["W_self"][:] = Hprev.T @ dZ
+            G[k]["W_neigh"][:] = M.T @ dZ
+            if k > 0:
+                dH = dZ @ P[k]["W_self"].T + sparse.aggregate_backward(mode, g.n, rp, cc, None, dZ @ P[k]["W_neigh"].T)
+    return {"loss": loss, "grads": grads, "scores": s, "g": gs, "dHK": dHK,
+            "cache": cache, "src": src, "dst": dst}
+
+
+def input_gradient(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst):
+    """dL/dX (not needed for training; used by the finite-difference pin of the backward
+    pass through the first layer's aggregation)."""
+    K = len(dims) - 1
+    P = split_params(arch, dims, np.asarray(params, dtype=np.float64))
+    cache = forward(g, X, params, arch, dims)
+    HK = cache["H"][K]
+    src = np.concatenate([pos_src, neg_src]).astype(np.int32)
+    dst = np.concatenate([pos_dst, neg_dst]).astype(np.int32)
+    y = np.concatenate([np.ones(len(pos_src)), np.zeros(len(neg_src))])
+    s = np.einsum("ij,ij->i", HK[src], HK[dst])
+    _, dls = bce_with_logits(s, y)
+    dH = sparse.edge_grad(HK, src, dst, dls / s.shape[0])
+    mode = "gcn" if arch == "gcn" else "mean"
+    for k in range(K - 1, -1, -1):
+        dZ = dH if k == K - 1 else dH * (cache["Z"][k] > 0.0)
+        if arch == "gcn":
+            dH = sparse.aggregate_backward(mode, g.n, g.rowptr, g.col, g.w, dZ @ P[k]["W"].T)
+        else:
+            dH = dZ @ P[k]["W_self"].T + sparse.aggregate_backward(mode, g.n, g.rowptr, g.col, None,
+                                                                   dZ @ P[k]["W_neigh"].T)
+    return dH
+
+
+def score(g, X, params, arch, dims, src, dst, blocks=None) -> np.ndarray:
+    """Edge scores s_(u,v) = <h_u^(K), h_v^(K)> (Eq. 2, dot-product predictor)."""
+    HK = forward(g, X, params, arch, dims, blocks)["H"][len(dims) - 1]
+    return np.einsum("ij,ij->i", HK[np.asarray(src)], HK[np.asarray(dst)])
+
+
+def average_gradients(grads_per_worker: List[np.ndarray]) -> np.ndarray:
+    """Gradient synchronisation of Algorithm 1: (1/p) * sum over the p workers."""
+    acc = np.zeros_like(np.asarray(grads_per_worker[0], dtype=np.float64))
+    for gi in grads_per_worker:
+        acc = acc + np.asarray(gi, dtype=np.float64)
+    return acc / len(grads_per_worker)
+
+
+def adam_step(params, m, v, grads, t: int, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8):
+    """Adam (the optimiser of the paper's experiments, lr 1e-3) with bias correction,
+    no weight decay.  t counts from 1.  Returns new (params, m, v) in float64."""
+    params = np.asarray(params, dtype=np.float64)
+    g = np.asarray(grads, dtype=np.float64)
+    m = beta1 * np.asarray(m, dtype=np.float64) + (1.0 - beta1) * g
+    v = beta2 * np.asarray(v, dtype=np.float64) + (1.0 - beta2) * g * g
+    mhat = m / (1.0 - beta1 ** t)
+    vhat = v / (1.0 - beta2 ** t)
+    return params - lr * mhat / (np.sqrt(vhat) + eps), m, v

@@ -1,0 +1,442 @@
+"""Pins for the CPU oracle: closed forms, dense brute force, finite differences, published
+known-answer vectors and invariants.  None of these re-use the oracle's own formulas."""
+import math
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import model as omodel
+from oracle import sparse as osparse
+import workloads as wl
+from helpers import (dense_adjacency, dense_forward, dense_gcn_operator, dense_loss,
+                     dense_mean_operator, rel_l2)
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ------------------------------------------------------------------ Philox
+def np_philox(c0, c1, c2, c3, k0, k1):
+    """Independent vectorised Philox4x32-10 on uint64 lanes (from the published definition)."""
+    c0, c1, c2, c3 = (np.asarray(x, dtype=np.uint64) for x in (c0, c1, c2, c3))
+    k0, k1 = np.uint64(k0), np.uint64(k1)
+    mask = np.uint64(0xFFFFFFFF)
+    for _ in range(10):
+        p0 = np.uint64(0xD2511F53) * c0
+        p1 = np.uint64(0xCD9E8D57) * c2
+        c0, c1, c2, c3 = ((p1 >> np.uint64(32)) ^ c1 ^ k0) & mask, p1 & mask, \
+                         ((p0 >> np.uint64(32)) ^ c3 ^ k1) & mask, p0 & mask
+        k0 = (k0 + np.uint64(0x9E3779B9)) & mask
+        k1 = (k1 + np.uint64(0xBB67AE85)) & mask
+    return c0, c1, c2, c3
+
+
+def test_philox_known_answers():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "philox4x32_10_kat.txt")) if l.strip() and l[0] != "#"]
+    assert len(rows) == 3
+    for r in rows:
+        v = [int(x, 16) for x in r]
+        out = oracle.philox4x32_10(v[0:4], v[4:6])
+        assert out.tolist() == v[6:10]
+
+
+def test_philox_constants_closed_form():
+    # Weyl increments are the fractional parts of the golden ratio and sqrt(3), scaled by 2^32
+    assert int((math.sqrt(5.0) - 1.0) / 2.0 * 2 ** 32) == 0x9E3779B9
+    assert int((math.sqrt(3.0) - 1.0) * 2 ** 32) == 0xBB67AE85
+    a = oracle.philox4x32_10([5, 6, 7, 8], [9, 10])
+    b = [int(x[()]) for x in np_philox(5, 6, 7, 8, 9, 10)]
+    assert a.tolist() == b
+
+
+# ------------------------------------------------------------------ structure
+def test_csc_transpose_bruteforce_and_involution():
+    g = wl.citation_directed(60, 400, 2.2, seed=11)
+    colptr, rowidx, perm = oracle.csc_transpose(g.n, g.rowptr, g.col)
+    A = dense_adjacency(g)
+    # brute force: transposed row c lists the v with A[v, c] != 0 ascending
+    exp_rows = [np.nonzero(A[:, c])[0] for c in range(g.n)]
+    assert colptr.tolist() == np.concatenate([[0], np.cumsum([len(r) for r in exp_rows])]).tolist()
+    assert rowidx.tolist() == np.concatenate(exp_rows).tolist()
+    assert sorted(perm.tolist()) == list(range(g.nnz))
+    rows = np.repeat(np.arange(g.n), np.diff(g.rowptr))
+    assert np.array_equal(rows[perm], rowidx) and np.array_equal(g.col[perm], np.repeat(np.arange(g.n), np.diff(colptr)))
+    # transpose of the transpose is the original
+    rp2, ci2, _ = oracle.csc_transpose(g.n, colptr, rowidx)
+    assert np.array_equal(rp2, g.rowptr) and np.array_equal(ci2, g.col)
+    # degrees
+    assert np.array_equal(np.diff(colptr), (A != 0).sum(axis=0))
+
+
+def test_csc_transpose_rejects_bad_input():
+    with pytest.raises(ValueError):
+        oracle.csc_transpose(3, np.array([0, 1, 2, 3]), np.array([0, 5, 1]))
+    with pytest.raises(ValueError):
+        oracle.csc_transpose(3, np.array([0, 2, 1, 3]), np.array([0, 1, 1]))
+
+
+# ------------------------------------------------------------------ aggregation
+@pytest.mark.parametrize("weighted", [False, True])
+def test_gcn_aggregate_dense_bruteforce(weighted):
+    g = wl.coauthor_weighted(50, 160, seed=5) if weighted else wl.erdos_renyi(50, 150, seed=5)
+    H = np.random.default_rng(0).standard_normal((g.n, 7))
+    S = dense_gcn_operator(g)
+    M = oracle.aggregate("gcn", g.n, g.rowptr, g.col, g.w, H)
+    assert np.allclose(M, S @ H, rtol=1e-12, atol=1e-13)
+    # invariants of the renormalised adjacency: symmetric, and sqrt(d~) is a fixed vector
+    dt = oracle.gcn_degree(g.n, g.rowptr, g.w)
+    assert np.allclose(dt, 1 + dense_adjacency(g).sum(axis=1))
+    assert np.allclose(S, S.T)
+    fixed = oracle.aggregate("gcn", g.n, g.rowptr, g.col, g.w, np.sqrt(dt)[:, None])
+    assert np.allclose(fixed[:, 0], np.sqrt(dt), rtol=1e-12)
+    # backward is multiplication by the transposed operator
+    dM = np.random.default_rng(1).standard_normal((g.n, 5))
+    assert np.allclose(oracle.aggregate_backward("gcn", g.n, g.rowptr, g.col, g.w, dM), S.T @ dM, atol=1e-13)
+
+
+def test_mean_aggregate_dense_bruteforce_directed():
+    g = wl.citation_directed(70, 200, 2.2, seed=3)
+    H = np.random.default_rng(0).standard_normal((g.n, 6))
+    S = dense_mean_operator(g)
+    M = oracle.aggregate("mean", g.n, g.rowptr, g.col, None, H)
+    assert np.allclose(M, S @ H, atol=1e-13)
+    deg = np.diff(g.rowptr)
+    assert (deg == 0).any(), "want an isolated row in this case"
+    assert np.all(M[deg == 0] == 0)
+    # rows of the mean operator sum to one: constants are preserved where deg > 0
+    ones = oracle.aggregate("mean", g.n, g.rowptr, g.col, None, np.full((g.n, 2), 3.5))
+    assert np.allclose(ones[deg > 0], 3.5)
+    dM = np.random.default_rng(1).standard_normal((g.n, 4))
+    assert np.allclose(oracle.aggregate_backward("mean", g.n, g.rowptr, g.col, None, dM), S.T @ dM, atol=1e-13)
+
+
+def test_empty_graph_reduces_to_mlp():
+    n, dims = 9, [4, 5, 3]
+    g = wl.Graph(n=n, rowptr=np.zeros(n + 1, dtype=np.int64), col=np.zeros(0, dtype=np.int32))
+    X = wl.node_features(n, 4, 0)
+    for arch in ("gcn", "sage"):
+        p = wl.glorot_params(arch, dims, 1, bias_scale=0.3)
+        HK = oracle.forward(g, X, p, arch, dims)["H"][2]
+        P = oracle.split_params(arch, dims, p.astype(np.float64))
+        W1 = P[0]["W"] if arch == "gcn" else P[0]["W_self"]
+        W2 = P[1]["W"] if arch == "gcn" else P[1]["W_self"]
+        ref = np.maximum(X.astype(np.float64) @ W1 + P[0]["b"], 0) @ W2 + P[1]["b"]
+        assert np.allclose(HK, ref, atol=1e-13)
+
+
+# ------------------------------------------------------------------ encoder forward
+@pytest.mark.parametrize("arch,dims", [("gcn", [6, 8, 5]), ("sage", [6, 8, 5]), ("gcn", [6, 7, 7, 4]), ("sage", [5, 6, 6, 3])])
+def test_forward_dense_bruteforce(arch, dims):
+    g = wl.coauthor_weighted(48, 140, seed=2) if arch == "gcn" else wl.citation_directed(48, 300, 2.2, seed=2)
+    X = wl.node_features(g.n, dims[0], 1)
+    p = wl.glorot_params(arch, dims, 3, bias_scale=0.2)
+    HK = oracle.forward(g, X, p, arch, dims)["H"][len(dims) - 1]
+    ref, _ = dense_forward(g, X, p, arch, dims)
+    assert np.allclose(HK, ref, rtol=1e-11, atol=1e-12)
+
+
+# ------------------------------------------------------------------ loss
+def test_loss_closed_forms():
+    g = wl.erdos_renyi(40, 100, seed=1)
+    dims = [4, 6, 5]
+    X = wl.node_features(g.n, 4, 0)
+    u, v = wl.undirected_edge_list(g)
+    ns, nd, _ = oracle.sample_negatives(g.n, g.rowptr, g.col, u, seed=1, step=0)
+    zero = np.zeros(wl.model_dims_param_count("gcn", dims), dtype=np.float32)
+    out = oracle.train_step(g, X, zero, "gcn", dims, u, v, ns, nd)
+    N = 2 * len(u)
+    assert abs(out["loss"] - math.log(2.0)) < 1e-15
+    assert np.allclose(out["g"][: len(u)], -0.5 / N) and np.allclose(out["g"][len(u):], 0.5 / N)
+    # symmetry of the undirected score
+    p = wl.glorot_params("gcn", dims, 3, 0.1)
+    assert np.allclose(oracle.score(g, X, p, "gcn", dims, u, v), oracle.score(g, X, p, "gcn", dims, v, u), rtol=1e-14)
+
+
+def test_bce_stability_against_extended_precision():
+    from decimal import Decimal, getcontext
+    getcontext().prec = 60
+    s = np.array([-800.0, -40.0, -3.0, -1e-9, 0.0, 1e-9, 2.5, 37.0, 745.0])
+    for y in (0.0, 1.0):
+        ell, d = oracle.bce_with_logits(s, np.full_like(s, y))
+        for si, li, di in zip(s, ell, d):
+            sig = Decimal(1) / (Decimal(1) + (-Decimal(float(si))).exp())
+            ref = -(sig.ln()) if y == 1.0 else -((Decimal(1) - sig).ln()) if sig != 1 else None
+            if y == 0.0:  # -log(1 - sigma(s)) = log(1 + e^s)
+                ref = (Decimal(1) + Decimal(float(si)).exp()).ln()
+            assert abs(float(ref) - li) <= 1e-14 * max(1.0, abs(float(ref)))
+            assert abs(float(sig) - y - di) <= 1e-15
+
+
+# ------------------------------------------------------------------ backward
+@pytest.mark.parametrize("arch,dims", [("gcn", [3, 4, 3]), ("sage", [3, 4, 3]), ("gcn", [3, 4, 4, 2]), ("sage", [3, 3, 4, 2])])
+def test_backward_finite_differences(arch, dims):
+    g = wl.coauthor_weighted(24, 60, seed=4) if arch == "gcn" else wl.citation_directed(24, 110, 2.2, seed=4)
+    X = wl.node_features(g.n, dims[0], 2)
+    p = wl.glorot_params(arch, dims, 5, bias_scale=0.3).astype(np.float64)
+    rng = np.random.default_rng(0)
+    src = rng.integers(0, g.n, 40).astype(np.int32)
+    dst = rng.integers(0, g.n, 40).astype(np.int32)
+    dst[:3] = src[:3]  # self pairs exercise the u == v branch
+    nsrc, ndst = src[:20], rng.integers(0, g.n, 20).astype(np.int32)
+    y = np.concatenate([np.ones(40), np.zeros(20)])
+    out = oracle.train_step(g, X, p, arch, dims, src, dst, nsrc, ndst)
+    s_all, d_all = np.concatenate([src, nsrc]), np.concatenate([dst, ndst])
+    assert abs(out["loss"] - dense_loss(g, X, p, arch, dims, s_all, d_all, y)) < 1e-13
+    h = 1e-6
+    fd = np.zeros_like(p)
+    for i in range(p.shape[0]):
+        pp, pm = p.copy(), p.copy()
+        pp[i] += h
+        pm[i] -= h
+        fd[i] = (dense_loss(g, X, pp, arch, dims, s_all, d_all, y) - dense_loss(g, X, pm, arch, dims, s_all, d_all, y)) / (2 * h)
+    assert rel_l2(out["grads"], fd) < 1e-7
+    assert np.max(np.abs(out["grads"] - fd)) < 1e-8
+    # gradient with respect to the input features (goes through every aggregation backward)
+    dX = omodel.input_gradient(g, X, p, arch, dims, src, dst, nsrc, ndst)
+    Xd = X.astype(np.float64)
+    for (r, c) in [(0, 0), (5, 1), (g.n - 1, 2), (11, 0)]:
+        xp, xm = Xd.copy(), Xd.copy()
+        xp[r, c] += h
+        xm[r, c] -= h
+        num = (dense_loss(g, xp, p, arch, dims, s_all, d_all, y) - dense_loss(g, xm, p, arch, dims, s_all, d_all, y)) / (2 * h)
+        assert abs(num - dX[r, c]) < 1e-8
+
+
+def test_gradient_averaging_identical_workers():
+    g = wl.erdos_renyi(30, 80, seed=9)
+    dims = [4, 5, 4]
+    X = wl.node_features(g.n, 4, 1)
+    p = wl.glorot_params("sage", dims, 1, 0.1)
+    u, v = wl.undirected_edge_list(g)
+    ns, nd, _ = oracle.sample_negatives(g.n, g.rowptr, g.col, u, seed=3, step=0)
+    g1 = oracle.train_step(g, X, p, "sage", dims, u, v, ns, nd)["grads"]
+    assert np.allclose(oracle.average_gradients([g1] * 8), g1, rtol=1e-15)
+    assert np.allclose(oracle.average_gradients([g1, 3 * g1]), 2 * g1, rtol=1e-15)
+
+
+# ------------------------------------------------------------------ Adam
+def test_adam_closed_forms():
+    rng = np.random.default_rng(0)
+    p0, g1, g2 = rng.standard_normal(50), rng.standard_normal(50), rng.standard_normal(50)
+    lr, eps = 1e-3, 1e-8
+    p1, m1, v1 = oracle.adam_step(p0, np.zeros(50), np.zeros(50), g1, t=1, lr=lr, eps=eps)
+    # first step: bias correction gives m^ = g, v^ = g^2
+    assert np.allclose(p1, p0 - lr * g1 / (np.abs(g1) + eps), rtol=1e-12, atol=1e-15)
+    p2, m2, v2 = oracle.adam_step(p1, m1, v1, g2, t=2, lr=lr, eps=eps)
+    mh = (0.9 * 0.1 * g1 + 0.1 * g2) / (1 - 0.81)
+    vh = (0.999 * 0.001 * g1 ** 2 + 0.001 * g2 ** 2) / (1 - 0.999 ** 2)
+    assert np.allclose(p2, p1 - lr * mh / (np.sqrt(vh) + eps), rtol=1e-12, atol=1e-15)
+
+
+# ------------------------------------------------------------------ negative sampler
+def test_negative_sampler_properties():
+    g = wl.chung_lu(3000, 12.0, 2.1, seed=7)
+    u, v = wl.undirected_edge_list(g)
+    ns, nd, exhausted = oracle.sample_negatives(g.n, g.rowptr, g.col, u, seed=42, step=3, k=2)
+    assert exhausted == 0
+    assert np.array_equal(ns, np.repeat(u, 2))  # per-source: the source is kept
+    A = set(zip(np.repeat(np.arange(g.n), np.diff(g.rowptr)).tolist(), g.col.tolist()))
+    assert all(a != b and (b, a) not in A for a, b in zip(ns.tolist(), nd.tolist()))
+    # batch-split invariance: the draw depends on the global edge index only
+    lo = 1000
+    ns2, nd2, _ = oracle.sample_negatives(g.n, g.rowptr, g.col, u[lo:lo + 500], seed=42, step=3, k=2, edge_index_base=lo)
+    assert np.array_equal(nd2, nd[2 * lo: 2 * (lo + 500)])
+    # different step or seed -> different draws
+    assert not np.array_equal(nd, oracle.sample_negatives(g.n, g.rowptr, g.col, u, seed=42, step=4, k=2)[1])
+    assert not np.array_equal(nd, oracle.sample_negatives(g.n, g.rowptr, g.col, u, seed=43, step=3, k=2)[1])
+
+
+def test_negative_sampler_matches_independent_philox_and_is_uniform():
+    g = wl.erdos_renyi(500, 1500, seed=1)
+    B = 40000
+    src = np.zeros(B, dtype=np.int32)
+    seed, step = (7 << 32) | 12345, 9
+    _, nd, _ = oracle.sample_negatives(g.n, g.rowptr, g.col, src, seed=seed, step=step, k=1, reject_edges=False)
+    j = np.arange(B, dtype=np.uint64)
+    x = np_philox(j & np.uint64(0xFFFFFFFF), j >> np.uint64(32), np.full(B, step, dtype=np.uint64),
+                  np.full(B, 1, dtype=np.uint64), seed & 0xFFFFFFFF, seed >> 32)[0]
+    assert np.array_equal(nd.astype(np.uint64), (x * np.uint64(g.n)) >> np.uint64(32))
+    counts = np.bincount(nd, minlength=g.n)
+    chi2 = ((counts - B / g.n) ** 2 / (B / g.n)).sum()
+    assert chi2 < 499 + 5 * math.sqrt(2 * 499)  # 5 sigma of chi-square with n-1 degrees of freedom
+
+
+def test_negative_sampler_candidates_and_global_pairs():
+    g = wl.erdos_renyi(400, 1200, seed=2)
+    cand = np.arange(0, 400, 4, dtype=np.int32)  # a "partition"
+    u, _ = wl.undirected_edge_list(g)
+    _, nd, _ = oracle.sample_negatives(g.n, g.rowptr, g.col, u, seed=5, step=0, cand=cand)
+    assert np.isin(nd, cand).all()
+    ns, nd, _ = oracle.sample_negatives(g.n, g.rowptr, g.col, u, seed=5, step=0, mode="global_pair", cand=cand)
+    assert np.isin(nd, cand).all() and np.isin(ns, cand).all() and (ns != nd).all()
+    assert len(np.unique(ns)) > 50
+    # exhausted attempts are reported: a complete graph has no valid per-source negative
+    n = 6
+    full = wl.csr_from_edges(n, *np.array([(a, b) for a in range(n) for b in range(n) if a != b]).T)
+    _, _, ex = oracle.sample_negatives(n, full.rowptr, full.col, np.arange(n, dtype=np.int32), seed=1, step=0, max_attempts=4)
+    assert ex == n
+
+
+# ------------------------------------------------------------------ neighbour sampler
+def test_neighbor_sampler_properties_and_uniformity():
+    g = wl.citation_directed(2000, 40000, 2.2, seed=8)
+    frontier = np.unique(np.random.default_rng(0).integers(0, g.n, 600)).astype(np.int32)
+    ptr, cols = oracle.sample_neighbors(g.rowptr, g.col, frontier, fanout=5, seed=3, step=1, hop=2)
+    deg = np.diff(g.rowptr)[frontier]
+    assert np.array_equal(np.diff(ptr), np.minimum(deg, 5))
+    for i, v in enumerate(frontier):
+        row = g.col[g.rowptr[v]:g.rowptr[v + 1]]
+        pick = cols[ptr[i]:ptr[i + 1]]
+        assert np.all(np.diff(pick) > 0) and np.isin(pick, row).all()
+    # uniform over the C(5,2) = 10 subsets of a 5-neighbour row, over many steps
+    star = wl.csr_from_edges(6, np.zeros(5, dtype=np.int64), np.arange(1, 6))
+    seen = {}
+    T = 20000
+    for step in range(T):
+        _, c = oracle.sample_neighbors(star.rowptr, star.col, np.array([0], dtype=np.int32), 2, seed=11, step=step, hop=1)
+        seen[tuple(c.tolist())] = seen.get(tuple(c.tolist()), 0) + 1
+    assert len(seen) == 10
+    chi2 = sum((c - T / 10) ** 2 / (T / 10) for c in seen.values())
+    assert chi2 < 9 + 5 * math.sqrt(18)
+
+
+def test_blocks_and_sampled_forward_bruteforce():
+    g = wl.citation_directed(120, 1500, 2.2, seed=6)
+    dims = [4, 5, 5, 3]
+    X = wl.node_features(g.n, 4, 0)
+    p = wl.glorot_params("sage", dims, 2, 0.2)
+    seeds = np.array([3, 17, 17, 40, 99], dtype=np.int32)
+    fr, blks = oracle.build_blocks(g.n, g.rowptr, g.col, seeds, [3, 2, 2], seed=5, step=0)
+    assert fr[0].tolist() == [3, 17, 40, 99]
+    for h in range(3):
+        assert np.all(np.diff(fr[h + 1]) > 0) and np.isin(fr[h], fr[h + 1]).all() and np.isin(blks[h][1], fr[h + 1]).all()
+    HK = oracle.forward(g, X, p, "sage", dims, blocks=(fr, blks))["H"][3]
+    # brute force: per layer a dense mean operator made from that hop's sampled rows
+    H = X.astype(np.float64)
+    P = oracle.split_params("sage", dims, p.astype(np.float64))
+    for l in range(1, 4):
+        h = 3 - l + 1
+        ptr, cols = blks[h - 1]
+        S = np.zeros((g.n, g.n))
+        for i, v in enumerate(fr[h - 1]):
+            nb = cols[ptr[i]:ptr[i + 1]]
+            if len(nb):
+                S[v, nb] = 1.0 / len(nb)
+        Z = H @ P[l - 1]["W_self"] + (S @ H) @ P[l - 1]["W_neigh"] + P[l - 1]["b"]
+        Hn = np.maximum(Z, 0) if l < 3 else Z
+        keep = np.zeros(g.n, dtype=bool)
+        keep[fr[h - 1]] = True
+        H = np.where(keep[:, None], Hn, 0.0)
+    assert np.allclose(HK, H, atol=1e-13)
+    assert np.all(HK[np.setdiff1d(np.arange(g.n), fr[0])] == 0)
+
+
+# ------------------------------------------------------------------ sparsifier (Algorithm 1, Theorems 1-2)
+def test_sparsifier_probabilities_and_weights():
+    g = wl.chung_lu(400, 10.0, 2.1, seed=3)
+    deg = np.diff(g.rowptr).astype(np.float64)
+    u, v = wl.undirected_edge_list(g)
+    npr = (deg > 0).sum()
+    pe = (1 / deg[u] + 1 / deg[v]) / npr
+    assert abs(pe.sum() - 1.0) < 1e-12  # the degree-based probabilities are normalised by n'
+    alpha = 0.2
+    L = int(alpha * len(u))
+    rows = np.repeat(np.arange(g.n), np.diff(g.rowptr))
+    upper = g.col > rows
+    acc = np.zeros(len(u))
+    hits = np.zeros(len(u))
+    T = 300
+    for s in range(T):
+        w = oracle.sparsify(g.n, g.rowptr, g.col, alpha, seed=s)
+        wu = w[upper]
+        # symmetric output, every kept weight is a positive multiple of 1 / (L p_e)
+        colptr, rowidx, perm = oracle.csc_transpose(g.n, g.rowptr, g.col)
+        assert np.array_equal(w[perm], w)
+        mult = wu * L * pe
+        assert np.allclose(mult, np.round(mult), atol=1e-9)
+        assert int(np.round(mult).sum()) == L  # exactly L draws
+        assert (wu > 0).sum() <= L
+        acc += wu
+        hits += np.round(mult)
+    # E[w~_e] = 1 (Theorem 1 weights): check the average over edges and over seeds
+    assert abs(acc.mean() / T - 1.0) < 0.02
+    # empirical draw frequencies follow p_e (chi-square over edges pooled in 20 probability bins)
+    order = np.argsort(pe)
+    bins = np.array_split(order, 20)
+    obs = np.array([hits[b].sum() for b in bins])
+    exp = np.array([pe[b].sum() for b in bins]) * T * L
+    chi2 = ((obs - exp) ** 2 / exp).sum()
+    assert chi2 < 19 + 5 * math.sqrt(38)
+    # removed fraction for alpha = 0.2 is "about 80 %" (Section IV): distinct kept edges in (0.15, 0.2] |E|
+    kept = (oracle.sparsify(g.n, g.rowptr, g.col, alpha, seed=1)[upper] > 0).mean()
+    expected_kept = (1 - (1 - pe) ** L).sum() / len(u)
+    assert 0.14 < kept <= 0.2 and abs(kept - expected_kept) < 0.02
+
+
+def test_effective_resistance_bounds_on_tiny_graph():
+    # Theorem 2: (1/2)(1/d_u + 1/d_v) <= r_(u,v) <= (1/gamma)(1/d_u + 1/d_v), r from Eq. 3
+    g = wl.erdos_renyi(40, 160, seed=2)
+    A = dense_adjacency(g)
+    d = A.sum(axis=1)
+    assert (d > 0).all()
+    Lp = np.linalg.pinv(np.diag(d) - A)
+    Lsym = np.eye(g.n) - A / np.sqrt(np.outer(d, d))
+    gamma = np.sort(np.linalg.eigvalsh(Lsym))[1]
+    u, v = wl.undirected_edge_list(g)
+    r = Lp[u, u] + Lp[v, v] - 2 * Lp[u, v]
+    approx = 1 / d[u] + 1 / d[v]
+    assert np.all(r >= 0.5 * approx - 1e-12) and np.all(r <= approx / gamma + 1e-12)
+
+
+def test_sparsified_graph_csr():
+    g = wl.erdos_renyi(200, 900, seed=4)
+    rp, cc, w = oracle.sparsified_graph(g.n, g.rowptr, g.col, 0.2, seed=0)
+    assert rp[-1] == len(cc) == len(w) and (w > 0).all()
+    for v in range(g.n):
+        assert np.all(np.diff(cc[rp[v]:rp[v + 1]]) > 0)
+        assert np.isin(cc[rp[v]:rp[v + 1]], g.col[g.rowptr[v]:g.rowptr[v + 1]]).all()
+
+
+def test_sampled_step_backward_finite_differences():
+    g = wl.citation_directed(60, 700, 2.2, seed=6)
+    dims = [3, 4, 3]
+    X = wl.node_features(g.n, 3, 0).astype(np.float64)
+    p = wl.glorot_params("sage", dims, 2, 0.2).astype(np.float64)
+    src = np.array([1, 5, 9, 30], dtype=np.int32)
+    dst = np.array([2, 7, 9, 41], dtype=np.int32)
+    nsrc, ndst = src.copy(), np.array([50, 3, 22, 8], dtype=np.int32)
+    seeds = np.concatenate([src, dst, ndst])
+    fr, blks = oracle.build_blocks(g.n, g.rowptr, g.col, seeds, [3, 2], seed=1, step=7)
+    out = oracle.train_step(g, X, p, "sage", dims, src, dst, nsrc, ndst, blocks=(fr, blks))
+    ops = []
+    for l in range(1, 3):
+        h = 2 - l + 1
+        ptr, cols = blks[h - 1]
+        S = np.zeros((g.n, g.n))
+        for i, v in enumerate(fr[h - 1]):
+            nb = cols[ptr[i]:ptr[i + 1]]
+            if len(nb):
+                S[v, nb] = 1.0 / len(nb)
+        ops.append(S)
+    s_all, d_all = np.concatenate([src, nsrc]), np.concatenate([dst, ndst])
+    y = np.concatenate([np.ones(4), np.zeros(4)])
+
+    def bf_loss(pp):
+        P = oracle.split_params("sage", dims, pp)
+        H1 = np.maximum(X @ P[0]["W_self"] + (ops[0] @ X) @ P[0]["W_neigh"] + P[0]["b"], 0)
+        keep = np.zeros(g.n, dtype=bool)
+        keep[fr[1]] = True
+        H1 = np.where(keep[:, None], H1, 0.0)
+        H2 = H1 @ P[1]["W_self"] + (ops[1] @ H1) @ P[1]["W_neigh"] + P[1]["b"]
+        s = (H2[s_all] * H2[d_all]).sum(axis=1)
+        return float(np.mean(y * np.logaddexp(0, -s) + (1 - y) * np.logaddexp(0, s)))
+
+    assert abs(bf_loss(p) - out["loss"]) < 1e-13
+    fd = np.zeros_like(p)
+    for i in range(p.shape[0]):
+        pp, pm = p.copy(), p.copy()
+        pp[i] += 1e-6
+        pm[i] -= 1e-6
+        fd[i] = (bf_loss(pp) - bf_loss(pm)) / 2e-6
+    assert rel_l2(out["grads"], fd) < 1e-7
