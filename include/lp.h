@@ -1,0 +1,235 @@
+/*
+ * lp.h -- C ABI of the B200 link-prediction GNN training step.
+ *
+ * One context trains on one graph on one GPU.  The step is the body of the per-batch loop
+ * of Algorithm 1 for one worker: sample negatives, run the K-layer encoder (Eq. 1), score
+ * every positive and negative edge with the dot product (Eq. 2), take the mean binary
+ * cross-entropy over N = |P| + |N| edges, back-propagate, and update the weights.
+ *
+ * General rules
+ *   - Every function returns an lp_status; nothing throws, aborts or traps.  After a
+ *     failure lp_last_error(ctx) holds a one-line description.
+ *   - Unless stated otherwise, array arguments are DEVICE pointers owned by the caller
+ *     (in practice torch tensors); the library reads or writes them on the context's
+ *     stream and never frees them.  The library owns only its internal workspace
+ *     (transposed graph, activations, sampled blocks), allocated with cudaMalloc at
+ *     lp_load_graph / lp_set_model and released by lp_destroy.
+ *   - All work is enqueued on the stream given to lp_create.  Calls that return a value
+ *     to the host (or take host buffers) synchronise that stream; the others do not.
+ *   - Graph convention: CSR rows are destination nodes v; the columns of row v are the
+ *     in-neighbours u in N(v) whose embeddings v aggregates (Eq. 1), strictly ascending
+ *     (no duplicates).  A positive sample (u, v) is an entry u in row v (Section II-B).
+ *   - Parameters, gradients and Adam moments are flat float32 vectors.  Layer k
+ *     (k = 0..K-1, input width dims[k], output width dims[k+1]) occupies, in order:
+ *        GCN       : W      [dims[k], dims[k+1]] row-major, b [dims[k+1]]
+ *        SAGE-mean : W_self [dims[k], dims[k+1]], W_neigh [dims[k], dims[k+1]], b [dims[k+1]]
+ */
+#ifndef LP_H_
+#define LP_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lp_ctx lp_ctx; /* opaque */
+
+typedef enum {
+    LP_OK = 0,
+    LP_EINVAL = -1,       /* bad argument (null pointer, size, malformed CSR, id out of range) */
+    LP_ESTATE = -2,       /* call out of order (e.g. train step before lp_set_model)          */
+    LP_ENOMEM = -3,       /* device or host allocation failed                                 */
+    LP_ECUDA = -4,        /* a CUDA call or kernel reported an error                          */
+    LP_EUNSUPPORTED = -5, /* valid request that this build does not implement                 */
+    LP_ETIMEOUT = -6      /* a bounded device-side wait expired; the context stays usable     */
+} lp_status;
+
+typedef enum { LP_GCN = 0, LP_SAGE_MEAN = 1 } lp_arch;
+typedef enum { LP_FP32 = 0, LP_BF16 = 1 } lp_prec;
+typedef enum { LP_NEG_PER_SOURCE = 0, LP_NEG_GLOBAL_PAIR = 1 } lp_neg_mode;
+
+#define LP_MAX_LAYERS 4
+
+/* Model description (Section IV hyperparameters: 2-3 layers, hidden width 256, per-hop
+ * fanouts).  dims = {input, hidden.., output}; every width must be a multiple of 8 (FP32)
+ * or of 64 (BF16 tensor-core path).  fanout[h] is the number of in-neighbours sampled at hop
+ * h+1 (hop 1 feeds the LAST layer); all zeros = full-graph training (every node aggregates
+ * its full neighbour list).  Sampling is supported for LP_SAGE_MEAN only. */
+typedef struct {
+    int32_t arch;                    /* lp_arch */
+    int32_t n_layers;                /* K, 1..LP_MAX_LAYERS */
+    int32_t dims[LP_MAX_LAYERS + 1];
+    int32_t prec;                    /* lp_prec: storage of activations and GEMM operand type */
+    int32_t fanout[LP_MAX_LAYERS];
+    int32_t reject_edges;            /* negatives: redraw self pairs and true edges */
+    int32_t max_attempts;            /* draws per negative when reject_edges (1..255) */
+} lp_model_desc;
+
+typedef struct {
+    int64_t negatives_exhausted;     /* negatives kept although every attempt was rejected (last lp_sample_negatives) */
+    int64_t block_nodes[LP_MAX_LAYERS + 1]; /* frontier sizes |F_0|..|F_K| of the last sampled step */
+    int64_t block_edges[LP_MAX_LAYERS];     /* sampled entries per hop of the last sampled step */
+    int64_t workspace_bytes;         /* device memory owned by the context */
+    int64_t kernel_launches;         /* kernels launched by this context since lp_create */
+} lp_stats;
+
+/* ---- life cycle ------------------------------------------------------------------- */
+
+/* Create a context on CUDA device `device`; `cuda_stream` is a cudaStream_t (NULL = the
+ * legacy default stream).  *out receives the context (NULL on failure). */
+lp_status lp_create(lp_ctx **out, int32_t device, void *cuda_stream);
+
+/* Release everything the context owns.  NULL is accepted. */
+void lp_destroy(lp_ctx *ctx);
+
+/* Last error text of this context (or of lp_create when ctx is NULL).  Never NULL. */
+const char *lp_last_error(const lp_ctx *ctx);
+
+/* ---- graph G = (V, E, X), Section II-A --------------------------------------------- */
+
+/* Load the graph the worker trains on and its node features.
+ *   n, nnz      : nodes and stored directed entries (nnz < 2^31)
+ *   rowptr[n+1] : int64, rowptr[0] = 0, non-decreasing, rowptr[n] = nnz
+ *   col[nnz]    : int32 in [0, n), strictly ascending inside a row
+ *   w[nnz]      : float32 edge weights or NULL (= all 1).  GCN uses them in A~ = A + I;
+ *                 SAGE-mean ignores them (unweighted mean over the stored neighbours)
+ *   X[n, f]     : float32 row-major, row v = x_v
+ *   ptrs_on_device : 0 = the four arrays are HOST memory, 1 = DEVICE memory
+ * The arrays are copied (the caller may free them afterwards).  The call validates the CSR
+ * (LP_EINVAL on any violation), builds the transposed structure used by the backward pass
+ * (entries of a transposed row ordered by original row), the degree normalisations
+ * (GCN: d~_v = 1 + sum_u w_vu; SAGE: 1/|N(v)|) and a BF16 copy of X.  Synchronises. */
+lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const int64_t *rowptr, const int32_t *col,
+                        const float *w, const float *X, int32_t f, int32_t ptrs_on_device);
+
+/* Transposed structure built by lp_load_graph, for bit-exact checks (device outputs):
+ * colptr[n+1] int64, rowidx[nnz] int32, perm[nnz] int64 (perm[t] = index of the original
+ * entry that transposed entry t came from).  Any of the three may be NULL. */
+lp_status lp_get_structure(lp_ctx *ctx, int64_t *colptr, int32_t *rowidx, int64_t *perm);
+
+/* ---- model -------------------------------------------------------------------------- */
+
+/* Fix the encoder (Eq. 1) and allocate the activation workspace.  `max_batch` bounds the
+ * number of positives per later call and `max_k` the negatives per positive. */
+lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *desc, int64_t max_batch, int32_t max_k);
+
+/* Length of the flat parameter vector of the model set by lp_set_model. */
+lp_status lp_param_count(const lp_ctx *ctx, int64_t *n_params);
+
+/* ---- negative sampling, Sections II-B and III ---------------------------------------- */
+
+/* Candidate set for negative endpoints: the worker's own partition V^i (local negatives)
+ * or NULL / n_cand = 0 for the entire node set (global negatives).  cand is a DEVICE array
+ * of node ids; it is copied. */
+lp_status lp_set_candidates(lp_ctx *ctx, const int32_t *cand, int64_t n_cand);
+
+/* Draw k negatives per positive with Philox4x32-10.  For the positive with global index
+ * j = edge_index_base + position, negative kk and attempt a the 32 random bits are word 0
+ * of philox(counter = (lo32(j), hi32(j), lo32(step), tag | kk<<8 | a<<16), key = (lo32(seed),
+ * hi32(seed))), tag = 1 for destinations and 2 for sources, and the endpoint is
+ * cand[floor(bits * |cand| / 2^32)].  LP_NEG_PER_SOURCE keeps the positive's source and
+ * draws the destination; LP_NEG_GLOBAL_PAIR draws both (neg_src required).  With
+ * reject_edges (model description) a self pair or an edge of the loaded graph is redrawn,
+ * at most max_attempts draws; the last draw is kept and counted in lp_stats.
+ *   pos_src[B]     : device, sources of the positives (ignored in global-pair mode)
+ *   neg_src[B*k]   : device output or NULL (per-source mode: pos_src repeated k times)
+ *   neg_dst[B*k]   : device output, negative kk of positive j at index j*k + kk
+ * Does not synchronise. */
+lp_status lp_sample_negatives(lp_ctx *ctx, uint64_t seed, uint64_t step, int32_t k, int32_t mode,
+                              const int32_t *pos_src, int64_t B, int64_t edge_index_base,
+                              int32_t *neg_src, int32_t *neg_dst);
+
+/* ---- training step, Algorithm 1 (per-batch body) -------------------------------------- */
+
+/* Forward, loss and gradient for one batch.
+ *   params[n_params]  : device float32, current weights W
+ *   pos_src/pos_dst[B]: device int32, positives (label 1)
+ *   neg_src[B*k]      : device int32 or NULL (= source of positive j for its k negatives)
+ *   neg_dst[B*k]      : device int32, negatives (label 0); k may be 0
+ *   seed, step        : Philox key / step counter of the neighbour sampler (used only when
+ *                       the model has non-zero fanouts)
+ *   loss              : device float32 scalar, L = (1/N) sum_e ell(s_e, y_e), N = B(1+k)
+ *   grads[n_params]   : device float32, dL/dW; overwritten, or added to when accumulate != 0
+ *                       (gradient accumulation over emulated workers)
+ * Node ids are checked on the device: an id outside [0, n) is clamped into range (so no
+ * access ever leaves the arrays), the results of that call are then meaningless, and the
+ * next synchronising call (lp_get_stats, lp_train_step_host) returns LP_EINVAL once.
+ * Does not synchronise. */
+lp_status lp_train_step(lp_ctx *ctx, const float *params, const int32_t *pos_src, const int32_t *pos_dst, int64_t B,
+                        const int32_t *neg_src, const int32_t *neg_dst, int32_t k, uint64_t seed, uint64_t step,
+                        float *loss, float *grads, int32_t accumulate);
+
+/* The same step for callers whose data lives in HOST memory: copies the B positives to the
+ * device, draws k per-source negatives (as lp_sample_negatives with edge_index_base),
+ * runs lp_train_step, optionally applies lp_adam_step to the DEVICE parameter vector
+ * (when adam_m/adam_v are non-NULL device arrays; hyper-parameters lr 1e-3, betas 0.9 /
+ * 0.999, eps 1e-8, step count adam_t), and copies the loss (and, if grads_host is not NULL,
+ * the gradient) back.  pos_src_host, pos_dst_host, loss_host, grads_host are HOST pointers;
+ * params, adam_m, adam_v are DEVICE pointers.  Synchronises. */
+lp_status lp_train_step_host(lp_ctx *ctx, float *params, const int32_t *pos_src_host, const int32_t *pos_dst_host,
+                             int64_t B, int32_t k, uint64_t seed, uint64_t step, int64_t edge_index_base,
+                             float *adam_m, float *adam_v, int64_t adam_t, float *loss_host, float *grads_host);
+
+/* Gradient synchronisation and update (Algorithm 1: average over p workers, then update;
+ * Section IV: Adam, lr 1e-3).  g = grad_scale * grads (grad_scale = 1/p);
+ * m = b1 m + (1-b1) g;  v = b2 v + (1-b2) g^2;
+ * params -= lr * (m / (1 - b1^t)) / (sqrt(v / (1 - b2^t)) + eps).   t counts from 1.
+ * With adam_m == NULL the plain rule W <- W - lr * g of Algorithm 1 is applied.
+ * All arrays are device float32 [n_params].  Does not synchronise. */
+lp_status lp_adam_step(lp_ctx *ctx, float *params, float *adam_m, float *adam_v, const float *grads, float grad_scale,
+                       float lr, float beta1, float beta2, float eps, int64_t t);
+
+/* ---- inference, Eq. 2 ------------------------------------------------------------------- */
+
+/* scores[E] = <h_u^(K), h_v^(K)> for the E pairs (src, dst) after a full forward pass with
+ * `params` (sampled models draw neighbours with seed/step as in lp_train_step).  Device
+ * arrays.  Does not synchronise. */
+lp_status lp_score(lp_ctx *ctx, const float *params, const int32_t *src, const int32_t *dst, int64_t E,
+                   uint64_t seed, uint64_t step, float *scores);
+
+/* ---- inspection (parity checks) ---------------------------------------------------------- */
+
+/* Embeddings H^(layer) of the last forward pass as float32, layer in 1..K.  For full-graph
+ * models `out` is [n, dims[layer]].  For sampled models `out` is [|F_{K-layer}|, dims[layer]],
+ * row i belonging to node frontier[i] of that frontier (see lp_get_block).  Device output. */
+lp_status lp_get_embeddings(lp_ctx *ctx, int32_t layer, float *out);
+
+/* Gradient of the loss with respect to H^(K) from the last lp_train_step, float32, same row
+ * indexing as lp_get_embeddings(K).  Device output. */
+lp_status lp_get_output_gradient(lp_ctx *ctx, float *out);
+
+/* Sampled computational graph of the last step (Section II-B), hop in 1..K:
+ *   frontier[|F_hop|]      : int32 global ids of F_hop, ascending (pass hop = 0 for the seeds F_0)
+ *   blk_ptr[|F_{hop-1}|+1] : int64 offsets per destination of F_{hop-1}
+ *   blk_col[entries]       : int32 sampled in-neighbours as GLOBAL ids, ascending per row
+ * Sizes come from lp_get_stats.  Any pointer may be NULL.  Device outputs. */
+lp_status lp_get_block(lp_ctx *ctx, int32_t hop, int32_t *frontier, int64_t *blk_ptr, int32_t *blk_col);
+
+/* Counters.  Synchronises the stream.  Returns LP_EINVAL (once) when an earlier step was
+ * given a node id outside [0, n). */
+lp_status lp_get_stats(lp_ctx *ctx, lp_stats *out);
+
+/* ---- single operators (used by the parity tests and the roofline benchmark) -------------- */
+
+/* AGG of Eq. 1 on the loaded graph, float32 in / float32 out (bf16 = 0) or BF16 in / BF16 out
+ * given as raw 16-bit words (bf16 = 1):
+ *   transpose = 0 : M[v] = AGG over N(v)        transpose = 1 : the adjoint, dH = AGG^T dM
+ *   arch LP_GCN: renormalised adjacency with self-loops; LP_SAGE_MEAN: mean over N(v).
+ * H and M are [n, F] row-major device arrays; F a multiple of 8, F <= 512. */
+lp_status lp_op_aggregate(lp_ctx *ctx, int32_t arch, int32_t transpose, int32_t bf16, const void *H, int32_t F, void *M);
+
+/* Dense transform C[M, N] = A[M, K] * B + bias, optional ReLU; B is [K, N] row-major
+ * (trans_b = 0) or [N, K] row-major (trans_b = 1).  prec LP_FP32: float32 everywhere;
+ * LP_BF16: A, B, C are BF16 words, bias float32, FP32 accumulation on the tensor cores. */
+lp_status lp_op_linear(lp_ctx *ctx, int32_t prec, int64_t M, int32_t N, int32_t K, const void *A, const void *B,
+                       int32_t trans_b, const float *bias, int32_t relu, void *C);
+
+/* Weight gradient dW[K, N] = A[M, K]^T * dZ[M, N] (float32 output, fixed reduction order). */
+lp_status lp_op_weight_grad(lp_ctx *ctx, int32_t prec, int64_t M, int32_t N, int32_t K, const void *A, const void *dZ,
+                            float *dW);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LP_H_ */

@@ -1,0 +1,259 @@
+"""Thin ctypes binding of the C ABI in include/lp.h.
+
+Argument marshalling only: every step of the path runs inside liblp_b200.so.  torch is used
+for device memory and streams.  There is no CPU fall-back: if the library is missing or no
+B200 is present, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "liblp_b200.so")
+
+LP_OK = 0
+LP_GCN, LP_SAGE_MEAN = 0, 1
+LP_FP32, LP_BF16 = 0, 1
+LP_NEG_PER_SOURCE, LP_NEG_GLOBAL_PAIR = 0, 1
+LP_MAX_LAYERS = 4
+
+STATUS_NAMES = {0: "LP_OK", -1: "LP_EINVAL", -2: "LP_ESTATE", -3: "LP_ENOMEM", -4: "LP_ECUDA",
+                -5: "LP_EUNSUPPORTED", -6: "LP_ETIMEOUT"}
+
+EXPORTS = [
+    "lp_create", "lp_destroy", "lp_last_error", "lp_load_graph", "lp_get_structure", "lp_set_model",
+    "lp_param_count", "lp_set_candidates", "lp_sample_negatives", "lp_train_step", "lp_train_step_host",
+    "lp_adam_step", "lp_score", "lp_get_embeddings", "lp_get_output_gradient", "lp_get_block",
+    "lp_get_stats", "lp_op_aggregate", "lp_op_linear", "lp_op_weight_grad",
+]
+
+
+class LpError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {message}")
+        self.status = status
+
+
+class ModelDesc(C.Structure):
+    _fields_ = [("arch", C.c_int32), ("n_layers", C.c_int32), ("dims", C.c_int32 * (LP_MAX_LAYERS + 1)),
+                ("prec", C.c_int32), ("fanout", C.c_int32 * LP_MAX_LAYERS), ("reject_edges", C.c_int32),
+                ("max_attempts", C.c_int32)]
+
+
+class Stats(C.Structure):
+    _fields_ = [("negatives_exhausted", C.c_int64), ("block_nodes", C.c_int64 * (LP_MAX_LAYERS + 1)),
+                ("block_edges", C.c_int64 * LP_MAX_LAYERS), ("workspace_bytes", C.c_int64),
+                ("kernel_launches", C.c_int64)]
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """dlopen the in-tree library (raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise FileNotFoundError(f"{_LIB_PATH} is missing: build it with paper_2506_20818_b200.build.build()")
+        lib = C.CDLL(_LIB_PATH)
+        lib.lp_last_error.restype = C.c_char_p
+        lib.lp_last_error.argtypes = [C.c_void_p]
+        lib.lp_destroy.restype = None
+        lib.lp_destroy.argtypes = [C.c_void_p]
+        for name in EXPORTS:
+            if name not in ("lp_last_error", "lp_destroy"):
+                getattr(lib, name).restype = C.c_int
+        _lib = lib
+    return _lib
+
+
+def _ptr(t):
+    """Device (or host) address of a torch tensor / numpy array, or None."""
+    if t is None:
+        return None
+    if hasattr(t, "data_ptr"):
+        assert t.is_contiguous()
+        return C.c_void_p(t.data_ptr())
+    assert t.flags["C_CONTIGUOUS"]
+    return C.c_void_p(t.ctypes.data)
+
+
+class Context:
+    """One lp_ctx: one graph, one model, one CUDA stream."""
+
+    def __init__(self, device: int = 0, stream=None):
+        import torch
+
+        self._torch = torch
+        self.lib = load_library()
+        self.device = device
+        self.stream = stream if stream is not None else torch.cuda.current_stream(device)
+        h = C.c_void_p()
+        st = self.lib.lp_create(C.byref(h), C.c_int32(device), C.c_void_p(self.stream.cuda_stream))
+        if st != LP_OK:
+            raise LpError(st, self.lib.lp_last_error(None).decode())
+        self.h = h
+        self.n = self.nnz = self.f = 0
+        self.n_params = 0
+        self.desc: Optional[ModelDesc] = None
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.lib.lp_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _ck(self, st: int):
+        if st != LP_OK:
+            raise LpError(st, self.lib.lp_last_error(self.h).decode())
+
+    # ---- graph
+    def load_graph(self, n, rowptr, col, w, X, on_device: bool = False):
+        """rowptr int64 [n+1], col int32 [nnz], w float32 [nnz] or None, X float32 [n, f]
+        (numpy / CPU tensors, or CUDA tensors with on_device=True)."""
+        nnz = int(col.shape[0])
+        f = int(X.shape[1])
+        self._ck(self.lib.lp_load_graph(self.h, C.c_int64(n), C.c_int64(nnz), _ptr(rowptr), _ptr(col), _ptr(w), _ptr(X),
+                                        C.c_int32(f), C.c_int32(1 if on_device else 0)))
+        self.n, self.nnz, self.f = int(n), nnz, f
+
+    def get_structure(self):
+        t = self._torch
+        dev = f"cuda:{self.device}"
+        colptr = t.empty(self.n + 1, dtype=t.int64, device=dev)
+        rowidx = t.empty(max(self.nnz, 1), dtype=t.int32, device=dev)
+        perm = t.empty(max(self.nnz, 1), dtype=t.int64, device=dev)
+        self._ck(self.lib.lp_get_structure(self.h, _ptr(colptr), _ptr(rowidx), _ptr(perm)))
+        return colptr, rowidx[: self.nnz], perm[: self.nnz]
+
+    # ---- model
+    def set_model(self, arch: str, dims: Sequence[int], prec: str = "fp32", fanout: Optional[Sequence[int]] = None,
+                  reject_edges: bool = True, max_attempts: int = 8, max_batch: int = 65536, max_k: int = 1):
+        d = ModelDesc()
+        d.arch = LP_GCN if arch == "gcn" else LP_SAGE_MEAN
+        d.n_layers = len(dims) - 1
+        for i, v in enumerate(dims):
+            d.dims[i] = int(v)
+        d.prec = LP_BF16 if prec == "bf16" else LP_FP32
+        for i, v in enumerate(fanout or []):
+            d.fanout[i] = int(v)
+        d.reject_edges = int(bool(reject_edges))
+        d.max_attempts = int(max_attempts)
+        self._ck(self.lib.lp_set_model(self.h, C.byref(d), C.c_int64(max_batch), C.c_int32(max_k)))
+        np_ = C.c_int64()
+        self._ck(self.lib.lp_param_count(self.h, C.byref(np_)))
+        self.n_params = int(np_.value)
+        self.desc = d
+        self.dims = list(dims)
+        self.K = len(dims) - 1
+        return self.n_params
+
+    # ---- sampling
+    def set_candidates(self, cand):
+        self._ck(self.lib.lp_set_candidates(self.h, _ptr(cand), C.c_int64(0 if cand is None else cand.numel())))
+
+    def sample_negatives(self, seed: int, step: int, k: int, pos_src, mode: int = LP_NEG_PER_SOURCE, edge_index_base: int = 0,
+                         want_src: bool = False):
+        t = self._torch
+        B = int(pos_src.numel())
+        neg_dst = t.empty(B * k, dtype=t.int32, device=pos_src.device)
+        neg_src = t.empty(B * k, dtype=t.int32, device=pos_src.device) if (want_src or mode == LP_NEG_GLOBAL_PAIR) else None
+        self._ck(self.lib.lp_sample_negatives(self.h, C.c_uint64(seed), C.c_uint64(step), C.c_int32(k), C.c_int32(mode), _ptr(pos_src),
+                                              C.c_int64(B), C.c_int64(edge_index_base), _ptr(neg_src), _ptr(neg_dst)))
+        return neg_src, neg_dst
+
+    # ---- step
+    def train_step(self, params, pos_src, pos_dst, neg_src, neg_dst, k: int, loss, grads, seed: int = 0, step: int = 0,
+                   accumulate: bool = False):
+        self._ck(self.lib.lp_train_step(self.h, _ptr(params), _ptr(pos_src), _ptr(pos_dst), C.c_int64(pos_src.numel()), _ptr(neg_src),
+                                        _ptr(neg_dst), C.c_int32(k), C.c_uint64(seed), C.c_uint64(step), _ptr(loss), _ptr(grads),
+                                        C.c_int32(int(accumulate))))
+
+    def train_step_host(self, params, pos_src_host, pos_dst_host, k: int, seed: int, step: int, edge_index_base: int = 0,
+                        adam_m=None, adam_v=None, adam_t: int = 1, loss_host=None, grads_host=None):
+        self._ck(self.lib.lp_train_step_host(self.h, _ptr(params), _ptr(pos_src_host), _ptr(pos_dst_host), C.c_int64(pos_src_host.shape[0]),
+                                             C.c_int32(k), C.c_uint64(seed), C.c_uint64(step), C.c_int64(edge_index_base), _ptr(adam_m),
+                                             _ptr(adam_v), C.c_int64(adam_t), _ptr(loss_host), _ptr(grads_host)))
+
+    def adam_step(self, params, m, v, grads, t: int, grad_scale: float = 1.0, lr: float = 1e-3, beta1: float = 0.9, beta2: float = 0.999,
+                  eps: float = 1e-8):
+        self._ck(self.lib.lp_adam_step(self.h, _ptr(params), _ptr(m), _ptr(v), _ptr(grads), C.c_float(grad_scale), C.c_float(lr),
+                                       C.c_float(beta1), C.c_float(beta2), C.c_float(eps), C.c_int64(t)))
+
+    def score(self, params, src, dst, seed: int = 0, step: int = 0):
+        t = self._torch
+        out = t.empty(src.numel(), dtype=t.float32, device=src.device)
+        self._ck(self.lib.lp_score(self.h, _ptr(params), _ptr(src), _ptr(dst), C.c_int64(src.numel()), C.c_uint64(seed), C.c_uint64(step),
+                                   _ptr(out)))
+        return out
+
+    # ---- inspection
+    def stats(self) -> Stats:
+        s = Stats()
+        self._ck(self.lib.lp_get_stats(self.h, C.byref(s)))
+        return s
+
+    def embeddings(self, layer: int, rows: Optional[int] = None):
+        t = self._torch
+        rows = self.n if rows is None else rows
+        out = t.empty((rows, self.dims[layer]), dtype=t.float32, device=f"cuda:{self.device}")
+        self._ck(self.lib.lp_get_embeddings(self.h, C.c_int32(layer), _ptr(out)))
+        return out
+
+    def output_gradient(self, rows: Optional[int] = None):
+        t = self._torch
+        rows = self.n if rows is None else rows
+        out = t.empty((rows, self.dims[-1]), dtype=t.float32, device=f"cuda:{self.device}")
+        self._ck(self.lib.lp_get_output_gradient(self.h, _ptr(out)))
+        return out
+
+    def block(self, hop: int):
+        """(frontier F_hop or None for the outermost hop, blk_ptr, blk_col) of the last sampled step."""
+        t = self._torch
+        dev = f"cuda:{self.device}"
+        s = self.stats()
+        frontier = None
+        if hop < self.K:
+            frontier = t.empty(int(s.block_nodes[hop]), dtype=t.int32, device=dev)
+        ptr = col = None
+        if hop >= 1:
+            ptr = t.empty(int(s.block_nodes[hop - 1]) + 1, dtype=t.int64, device=dev)
+            col = t.empty(max(int(s.block_edges[hop - 1]), 1), dtype=t.int32, device=dev)
+        self._ck(self.lib.lp_get_block(self.h, C.c_int32(hop), _ptr(frontier), _ptr(ptr), _ptr(col)))
+        if col is not None:
+            col = col[: int(s.block_edges[hop - 1])]
+        return frontier, ptr, col
+
+    # ---- single operators
+    def op_aggregate(self, arch: str, H, transpose: bool = False):
+        t = self._torch
+        M = t.empty_like(H)
+        self._ck(self.lib.lp_op_aggregate(self.h, C.c_int32(LP_GCN if arch == "gcn" else LP_SAGE_MEAN), C.c_int32(int(transpose)),
+                                          C.c_int32(int(H.dtype == t.bfloat16)), _ptr(H), C.c_int32(H.shape[1]), _ptr(M)))
+        return M
+
+    def op_linear(self, A, B, bias=None, relu: bool = False, trans_b: bool = False):
+        t = self._torch
+        M, K = A.shape
+        N = B.shape[0] if trans_b else B.shape[1]
+        Cout = t.empty((M, N), dtype=A.dtype, device=A.device)
+        prec = LP_BF16 if A.dtype == t.bfloat16 else LP_FP32
+        self._ck(self.lib.lp_op_linear(self.h, C.c_int32(prec), C.c_int64(M), C.c_int32(N), C.c_int32(K), _ptr(A), _ptr(B),
+                                       C.c_int32(int(trans_b)), _ptr(bias), C.c_int32(int(relu)), _ptr(Cout)))
+        return Cout
+
+    def op_weight_grad(self, A, dZ):
+        t = self._torch
+        M, K = A.shape
+        N = dZ.shape[1]
+        dW = t.empty((K, N), dtype=t.float32, device=A.device)
+        prec = LP_BF16 if A.dtype == t.bfloat16 else LP_FP32
+        self._ck(self.lib.lp_op_weight_grad(self.h, C.c_int32(prec), C.c_int64(M), C.c_int32(N), C.c_int32(K), _ptr(A), _ptr(dZ), _ptr(dW)))
+        return dW

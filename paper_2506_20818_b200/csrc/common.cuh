@@ -1,0 +1,63 @@
+// Shared declarations of the link-prediction step library (device helpers, error macros).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "../../include/lp.h"
+
+typedef __nv_bfloat16 bf16;
+
+#define LP_DEVINL __device__ __forceinline__
+
+static inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// ---------------------------------------------------------------------------------------------
+// element conversion helpers: activations are stored as float (FP32 path) or bf16 (BF16 path),
+// all arithmetic is done in float.
+// ---------------------------------------------------------------------------------------------
+template <typename T> struct Vec16;  // 16-byte vector of T
+template <> struct Vec16<float> {
+    static constexpr int N = 4;
+    float4 v;
+    LP_DEVINL void load(const float *p) { v = __ldg(reinterpret_cast<const float4 *>(p)); }
+    LP_DEVINL void store(float *p) const { *reinterpret_cast<float4 *>(p) = v; }
+    LP_DEVINL void to_float(float *f) const { f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w; }
+    LP_DEVINL void from_float(const float *f) { v = make_float4(f[0], f[1], f[2], f[3]); }
+};
+template <> struct Vec16<bf16> {
+    static constexpr int N = 8;
+    uint4 v;
+    LP_DEVINL void load(const bf16 *p) { v = __ldg(reinterpret_cast<const uint4 *>(p)); }
+    LP_DEVINL void store(bf16 *p) const { *reinterpret_cast<uint4 *>(p) = v; }
+    LP_DEVINL void to_float(float *f) const {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {  // bf16 -> float is a 16-bit shift
+            f[2 * i] = __uint_as_float(w[i] << 16);
+            f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
+    LP_DEVINL void from_float(const float *f) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+            w[i] = *reinterpret_cast<uint32_t *>(&h);
+        }
+        v = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+template <typename T> LP_DEVINL float to_f(T x);
+template <> LP_DEVINL float to_f<float>(float x) { return x; }
+template <> LP_DEVINL float to_f<bf16>(bf16 x) { return __bfloat162float(x); }
+template <typename T> LP_DEVINL T from_f(float x);
+template <> LP_DEVINL float from_f<float>(float x) { return x; }
+template <> LP_DEVINL bf16 from_f<bf16>(float x) { return __float2bfloat16_rn(x); }

@@ -1,0 +1,219 @@
+// Edge predictor (Eq. 2, dot product), mean binary cross-entropy over N = |P| + |N| edges
+// (Algorithm 1) and the per-edge score gradients; plus the batch-edge incidence lists that let
+// the gradient with respect to H^(K) be gathered row by row (no float atomics).
+#pragma once
+#include "common.cuh"
+#include "scan_sort.cuh"
+
+constexpr int EDGE_THREADS = 256;
+
+// Node ids arrive from the caller in device memory; every consumer clamps them into [0, n_ids) so
+// that a bad id can never cause an out-of-range access (check_ids_kernel reports it instead).
+LP_DEVINL int clamp_id(int v, int n_ids) { return min(max(v, 0), n_ids - 1); }
+
+__global__ void check_ids_kernel(const int *__restrict__ ids, int64_t m, int n_ids, int *__restrict__ err)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < m && (ids[i] < 0 || ids[i] >= n_ids)) atomicOr(err, 1);
+}
+
+LP_DEVINL float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// ell(s, y) = max(s, 0) - s*y + log(1 + exp(-|s|));   d ell / d s = sigmoid(s) - y
+LP_DEVINL void bce_logits(float s, float y, float &ell, float &dls)
+{
+    const float e = expf(-fabsf(s));
+    ell = fmaxf(s, 0.f) - s * y + log1pf(e);
+    const float sig = (s >= 0.f) ? 1.f / (1.f + e) : e / (1.f + e);
+    dls = sig - y;
+}
+
+// One warp per positive j: loads h_u once, then h_v and the k negative destinations (per-source
+// negatives share the source row).  Writes g for the positive and its negatives (already divided
+// by N), the raw scores if asked, and one loss partial per block.
+//   idmap : optional global id -> row of H (sampled models: position inside the seed frontier)
+template <typename T, int NV>
+__global__ void __launch_bounds__(EDGE_THREADS)
+edge_score_bce_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const int *__restrict__ idmap, const int *__restrict__ pos_src,
+                      const int *__restrict__ pos_dst, int64_t B, const int *__restrict__ neg_src, const int *__restrict__ neg_dst, int k,
+                      float inv_N, float *__restrict__ g_pos, float *__restrict__ g_neg, float *__restrict__ s_pos, float *__restrict__ s_neg,
+                      float *__restrict__ loss_partials)
+{
+    constexpr int VN = Vec16<T>::N;
+    __shared__ float s_loss[EDGE_THREADS / 32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t j = (int64_t)blockIdx.x * (EDGE_THREADS / 32) + warp;
+    const int nchunks = D / VN;
+    float loss = 0.f;
+    if (j < B) {
+        int u = clamp_id(pos_src[j], n_ids), v = clamp_id(pos_dst[j], n_ids);
+        if (idmap) { u = idmap[u]; v = idmap[v]; }
+        float hu[NV][VN];
+        float dot = 0.f;
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const int ch = lane + i * 32;
+            if (ch < nchunks) {
+                Vec16<T> a, b;
+                a.load(H + (size_t)u * ldh + ch * VN);
+                b.load(H + (size_t)v * ldh + ch * VN);
+                float fb[VN];
+                a.to_float(hu[i]);
+                b.to_float(fb);
+#pragma unroll
+                for (int t = 0; t < VN; ++t) dot = fmaf(hu[i][t], fb[t], dot);
+            }
+        }
+        dot = warp_sum(dot);
+        float ell, dls;
+        bce_logits(dot, 1.f, ell, dls);
+        loss += ell;
+        if (lane == 0) {
+            g_pos[j] = dls * inv_N;
+            if (s_pos) s_pos[j] = dot;
+        }
+        for (int kk = 0; kk < k; ++kk) {
+            const int64_t t = j * k + kk;
+            int vn = clamp_id(neg_dst[t], n_ids);
+            if (idmap) vn = idmap[vn];
+            const bool own_src = neg_src != nullptr;
+            int un = u;
+            if (own_src) { un = clamp_id(neg_src[t], n_ids); if (idmap) un = idmap[un]; }
+            float d2 = 0.f;
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const int ch = lane + i * 32;
+                if (ch < nchunks) {
+                    Vec16<T> b;
+                    b.load(H + (size_t)vn * ldh + ch * VN);
+                    float fb[VN];
+                    b.to_float(fb);
+                    if (own_src && un != u) {
+                        Vec16<T> a;
+                        a.load(H + (size_t)un * ldh + ch * VN);
+                        float fa[VN];
+                        a.to_float(fa);
+#pragma unroll
+                        for (int q = 0; q < VN; ++q) d2 = fmaf(fa[q], fb[q], d2);
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < VN; ++q) d2 = fmaf(hu[i][q], fb[q], d2);
+                    }
+                }
+            }
+            d2 = warp_sum(d2);
+            bce_logits(d2, 0.f, ell, dls);
+            loss += ell;
+            if (lane == 0) {
+                g_neg[t] = dls * inv_N;
+                if (s_neg) s_neg[t] = d2;
+            }
+        }
+    }
+    if (lane == 0) s_loss[warp] = loss;
+    __syncthreads();
+    if (threadIdx.x == 0 && loss_partials) {
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < EDGE_THREADS / 32; ++w) s += s_loss[w];
+        loss_partials[blockIdx.x] = s;
+    }
+}
+
+// loss = inv_N * sum of partials, added in index order by one block
+__global__ void loss_reduce_kernel(const float *__restrict__ partials, int64_t m, float inv_N, float *__restrict__ loss)
+{
+    __shared__ float sh[256];
+    float s = 0.f;
+    const int64_t per = (m + 255) / 256;
+    const int64_t b = per * threadIdx.x, e = min(m, b + per);
+    for (int64_t i = b; i < e; ++i) s += partials[i];
+    sh[threadIdx.x] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.f;
+        for (int i = 0; i < 256; ++i) t += sh[i];
+        *loss = t * inv_N;
+    }
+}
+
+// plain scores for lp_score: one warp per edge
+template <typename T, int NV>
+__global__ void __launch_bounds__(EDGE_THREADS)
+edge_score_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const int *__restrict__ idmap, const int *__restrict__ src,
+                  const int *__restrict__ dst, int64_t E, float *__restrict__ scores)
+{
+    constexpr int VN = Vec16<T>::N;
+    const int lane = threadIdx.x & 31;
+    const int64_t e = (int64_t)blockIdx.x * (EDGE_THREADS / 32) + (threadIdx.x >> 5);
+    if (e >= E) return;
+    int u = clamp_id(src[e], n_ids), v = clamp_id(dst[e], n_ids);
+    if (idmap) { u = idmap[u]; v = idmap[v]; }
+    const int nchunks = D / VN;
+    float dot = 0.f;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+        const int ch = lane + i * 32;
+        if (ch < nchunks) {
+            Vec16<T> a, b;
+            a.load(H + (size_t)u * ldh + ch * VN);
+            b.load(H + (size_t)v * ldh + ch * VN);
+            float fa[VN], fb[VN];
+            a.to_float(fa);
+            b.to_float(fb);
+#pragma unroll
+            for (int t = 0; t < VN; ++t) dot = fmaf(fa[t], fb[t], dot);
+        }
+    }
+    dot = warp_sum(dot);
+    if (lane == 0) scores[e] = dot;
+}
+
+// Incidence keys of the scored edges.  Edge slots: positives 0..B-1, negatives B..B+B*k-1.
+// Slot e contributes (node = src_e, other = dst_e) at 2e and (node = dst_e, other = src_e) at 2e+1.
+__global__ void incidence_keys_kernel(int n_ids, const int *__restrict__ idmap, const int *__restrict__ pos_src, const int *__restrict__ pos_dst, int64_t B,
+                                      const int *__restrict__ neg_src, const int *__restrict__ neg_dst, int k, uint32_t *__restrict__ keys,
+                                      uint32_t *__restrict__ vals, int *__restrict__ other, int *__restrict__ counts)
+{
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t E = B * (1 + k);
+    if (e >= E) return;
+    int s, d;
+    if (e < B) {
+        s = pos_src[e];
+        d = pos_dst[e];
+    } else {
+        const int64_t t = e - B;
+        s = neg_src ? neg_src[t] : pos_src[t / k];
+        d = neg_dst[t];
+    }
+    s = clamp_id(s, n_ids);
+    d = clamp_id(d, n_ids);
+    if (idmap) { s = idmap[s]; d = idmap[d]; }
+    keys[2 * e] = (uint32_t)s;
+    keys[2 * e + 1] = (uint32_t)d;
+    vals[2 * e] = (uint32_t)(2 * e);
+    vals[2 * e + 1] = (uint32_t)(2 * e + 1);
+    other[2 * e] = d;
+    other[2 * e + 1] = s;
+    atomicAdd(&counts[s], 1);
+    atomicAdd(&counts[d], 1);
+}
+
+// after the stable sort by node: column (= the other endpoint) and coefficient (= g of the edge)
+__global__ void incidence_fill_kernel(const uint32_t *__restrict__ sorted_slots, int64_t m, const int *__restrict__ other, int64_t B,
+                                      const float *__restrict__ g_pos, const float *__restrict__ g_neg, int *__restrict__ inc_col,
+                                      float *__restrict__ inc_val)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= m) return;
+    const uint32_t slot = sorted_slots[t];
+    const int64_t e = slot >> 1;
+    inc_col[t] = other[slot];
+    inc_val[t] = e < B ? g_pos[e] : g_neg[e - B];
+}

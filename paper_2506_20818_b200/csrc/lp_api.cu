@@ -1,0 +1,1227 @@
+// C ABI of the link-prediction training step: context, validation, workspace and the
+// orchestration of the kernels.  See include/lp.h for the contract of every entry point.
+#include <algorithm>
+#include <cmath>
+#include <new>
+
+#include "common.cuh"
+#include "scan_sort.cuh"
+#include "spmm.cuh"
+#include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
+#include "sampler.cuh"
+#include "edge.cuh"
+#include "optim.cuh"
+
+// ----------------------------------------------------------------------------------------------
+// context
+// ----------------------------------------------------------------------------------------------
+struct HopBlock {  // sampled block of hop h (destinations F_{h-1}, sources F_h)
+    int cap_dst = 0, cap_src = 0;
+    int64_t cap_entries = 0;
+    int n_dst = 0, n_src = 0;  // host mirrors of the last step
+    int64_t entries = 0;
+    int *frontier = nullptr;      // F_h, global ids ascending            [cap_src]
+    int *n_front_dev = nullptr;   // |F_h| on the device
+    int *posmap = nullptr;        // global id -> position in F_h          [n]
+    int *blk_ptr = nullptr;       // offsets per destination               [cap_dst + 1]
+    int *blk_col_global = nullptr, *blk_col_local = nullptr, *blk_row = nullptr;  // [cap_entries]
+    float *inv_deg = nullptr;     // 1 / sampled degree per destination     [cap_dst]
+    int *colptr = nullptr, *rowidx = nullptr, *perm = nullptr;  // transposed block
+    float *valT = nullptr;
+    int *self_idx = nullptr, *inv_self = nullptr;
+};
+
+struct LayerBuf {  // device buffers of one encoder layer (element type fixed by the precision)
+    void *A = nullptr;     // GEMM operand: SAGE [rows, 2 Fi] = [H | mean]; GCN [rows, Fi] = aggregate
+    void *Hin = nullptr;   // input embeddings H^(k) when they are not the left half of A
+    void *Hout = nullptr;  // sampled models: output rows of this layer [rows_dst, Fo]
+    int64_t off_w = 0, off_b = 0;  // offsets in the flat parameter vector
+    int Fi = 0, Fo = 0, Kin = 0;
+};
+
+struct lp_ctx {
+    int device = 0;
+    Exec ex;
+    std::string err;
+    std::vector<void *> graph_allocs, model_allocs;
+    int64_t graph_bytes = 0, model_bytes = 0;
+
+    // graph
+    bool loaded = false;
+    int n = 0, f = 0;
+    int64_t nnz = 0;
+    int *rowptr = nullptr, *col = nullptr;
+    float *w = nullptr;
+    int *colptr = nullptr, *rowidx = nullptr, *perm = nullptr;
+    float *gcn_val = nullptr, *gcn_valT = nullptr, *gcn_self = nullptr;
+    float *inv_deg = nullptr, *meanT_val = nullptr;
+    float *X32 = nullptr;
+    bf16 *X16 = nullptr;
+    int *cand = nullptr;
+    int64_t n_cand = 0;
+    unsigned long long *exhausted_dev = nullptr;
+    int *err_flag = nullptr;
+
+    // model
+    bool model_set = false, sampled = false;
+    lp_model_desc desc{};
+    int64_t n_params = 0, max_batch = 0;
+    int max_k = 0, K = 0;
+    LayerBuf layer[LP_MAX_LAYERS];
+    void *HK = nullptr;                 // H^(K) [rows_out, D]
+    void *dHK = nullptr;                // dL/dH^(K) [rows_out, D]
+    void *dZ[2] = {nullptr, nullptr};   // gradient ping-pong [max_rows, max_width]
+    void *dA = nullptr;                 // [max_rows, max Kin]
+    float *partials = nullptr;          // split-K / column-sum partials
+    int64_t partials_floats = 0;
+    float *g_pos = nullptr, *g_neg = nullptr, *loss_partials = nullptr;
+    uint32_t *inc_keys = nullptr, *inc_slots = nullptr;
+    int *inc_other = nullptr, *inc_ptr = nullptr, *inc_col = nullptr;
+    float *inc_val = nullptr;
+    SortScratch sort;                   // sized for the largest per-step sort
+    TransposeScratch tsp;
+    int *scan_tmp = nullptr;
+    int64_t sort_cap = 0;
+    HopBlock hop[LP_MAX_LAYERS + 1];    // hop[0] holds only the seed frontier F_0
+    unsigned char *mark = nullptr;
+    int *flags = nullptr;
+    int *seed_ids = nullptr;            // pos_src | pos_dst | neg_dst (| neg_src) of the batch
+    int *host_counts = nullptr;         // pinned
+    int *d_neg_tmp = nullptr, *d_pos_tmp = nullptr;  // staging of lp_train_step_host
+    float *d_loss_tmp = nullptr, *d_grads_tmp = nullptr;
+    int rows_out = 0;                   // rows of H^(K) in the last forward
+    bool have_forward = false, have_grad = false;
+    int64_t last_exhausted = 0;
+    TcState tc;                         // tensor-core GEMM state (descriptor encoder, device error word)
+};
+
+static std::string g_create_error;
+
+static lp_status fail(lp_ctx *c, lp_status st, const std::string &msg)
+{
+    if (c) c->err = msg; else g_create_error = msg;
+    return st;
+}
+
+#define CK(call)                                                                                         \
+    do {                                                                                                 \
+        cudaError_t e_ = (call);                                                                         \
+        if (e_ != cudaSuccess)                                                                           \
+            return fail(ctx, e_ == cudaErrorMemoryAllocation ? LP_ENOMEM : LP_ECUDA,                     \
+                        std::string(#call) + ": " + cudaGetErrorString(e_));                             \
+    } while (0)
+
+#define CK_LAUNCH()                                                                                      \
+    do {                                                                                                 \
+        cudaError_t e_ = cudaGetLastError();                                                             \
+        if (e_ != cudaSuccess) return fail(ctx, LP_ECUDA, std::string("kernel launch: ") + cudaGetErrorString(e_)); \
+    } while (0)
+
+template <typename P> static cudaError_t dev_alloc(lp_ctx *c, std::vector<void *> &list, int64_t &bytes_acc, P **out, int64_t count)
+{
+    size_t bytes = sizeof(P) * (size_t)std::max<int64_t>(count, 1);
+    bytes = (bytes + 255) & ~(size_t)255;
+    void *p = nullptr;
+    cudaError_t e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) { *out = nullptr; return e; }
+    list.push_back(p);
+    bytes_acc += (int64_t)bytes;
+    *out = (P *)p;
+    return cudaSuccess;
+}
+#define GALLOC(ptr, count) CK(dev_alloc(ctx, ctx->graph_allocs, ctx->graph_bytes, &(ptr), (count)))
+#define MALLOC(ptr, count) CK(dev_alloc(ctx, ctx->model_allocs, ctx->model_bytes, &(ptr), (count)))
+
+static void free_list(std::vector<void *> &l)
+{
+    for (void *p : l) cudaFree(p);
+    l.clear();
+}
+
+static inline unsigned nblk(int64_t n, int t = 256) { return (unsigned)std::max<int64_t>(1, ceil_div64(n, t)); }
+
+// ----------------------------------------------------------------------------------------------
+// load-time kernels
+// ----------------------------------------------------------------------------------------------
+__global__ void validate_csr_kernel(const int64_t *__restrict__ rowptr64, int n, int64_t nnz, const int *__restrict__ col, int *__restrict__ rowptr32,
+                                    int *__restrict__ err)
+{
+    const int v = blockIdx.x * blockDim.x + threadIdx.x;
+    if (v > n) return;
+    const int64_t a = rowptr64[v];
+    if (v == 0 && a != 0) atomicOr(err, 1);
+    if (v == n) {
+        if (a != nnz) atomicOr(err, 2);
+        rowptr32[v] = (int)min(max(a, (int64_t)0), nnz);
+        return;
+    }
+    const int64_t b = rowptr64[v + 1];
+    if (a < 0 || b < a || b > nnz) { atomicOr(err, 4); rowptr32[v] = (int)min(max(a, (int64_t)0), nnz); return; }
+    rowptr32[v] = (int)a;
+    int prev = -1;
+    for (int64_t e = a; e < b; ++e) {
+        const int c = col[e];
+        if (c < 0 || c >= n) { atomicOr(err, 8); break; }
+        if (c <= prev) { atomicOr(err, 16); break; }
+        prev = c;
+    }
+}
+
+__global__ void degree_kernel(const int *__restrict__ rowptr, const float *__restrict__ w, int n, float *__restrict__ dtilde, float *__restrict__ gcn_self,
+                              float *__restrict__ inv_deg)
+{
+    const int v = blockIdx.x * blockDim.x + threadIdx.x;
+    if (v >= n) return;
+    const int a = rowptr[v], b = rowptr[v + 1];
+    float d = 1.f;  // self-loop of weight 1
+    if (w) { for (int e = a; e < b; ++e) d += w[e]; } else { d += (float)(b - a); }
+    dtilde[v] = d;
+    gcn_self[v] = 1.f / d;
+    inv_deg[v] = b > a ? 1.f / (float)(b - a) : 0.f;
+}
+
+// GCN coefficient of entry e in row v, column u: w_vu / sqrt(d~_v d~_u)
+__global__ void gcn_val_kernel(const int *__restrict__ rows, const int *__restrict__ col, const float *__restrict__ w, const float *__restrict__ dtilde,
+                               int64_t nnz, float *__restrict__ val)
+{
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= nnz) return;
+    val[e] = (w ? w[e] : 1.f) / sqrtf(dtilde[rows[e]] * dtilde[col[e]]);
+}
+
+__global__ void widen_i32_kernel(const int *__restrict__ src, int64_t m, int64_t *__restrict__ dst)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < m) dst[i] = src[i];
+}
+
+// ----------------------------------------------------------------------------------------------
+// life cycle
+// ----------------------------------------------------------------------------------------------
+extern "C" const char *lp_last_error(const lp_ctx *ctx) { return ctx ? ctx->err.c_str() : g_create_error.c_str(); }
+
+extern "C" lp_status lp_create(lp_ctx **out, int32_t device, void *cuda_stream)
+{
+    lp_ctx *ctx = nullptr;
+    if (!out) return fail(nullptr, LP_EINVAL, "lp_create: out is NULL");
+    *out = nullptr;
+    int count = 0;
+    cudaError_t e = cudaGetDeviceCount(&count);
+    if (e != cudaSuccess || count <= 0) return fail(nullptr, LP_ECUDA, std::string("lp_create: no CUDA device: ") + cudaGetErrorString(e));
+    if (device < 0 || device >= count) return fail(nullptr, LP_EINVAL, "lp_create: device index out of range");
+    e = cudaSetDevice(device);
+    if (e != cudaSuccess) return fail(nullptr, LP_ECUDA, std::string("cudaSetDevice: ") + cudaGetErrorString(e));
+    cudaDeviceProp prop;
+    cudaGetDeviceProperties(&prop, device);
+    if (prop.major != 10) return fail(nullptr, LP_EUNSUPPORTED, "lp_create: this library is built for sm_100a (B200) only");
+    ctx = new (std::nothrow) lp_ctx();
+    if (!ctx) return fail(nullptr, LP_ENOMEM, "lp_create: host allocation failed");
+    ctx->device = device;
+    ctx->ex.st = (cudaStream_t)cuda_stream;
+    if (cudaMalloc((void **)&ctx->err_flag, 256) != cudaSuccess || cudaMalloc((void **)&ctx->exhausted_dev, 256) != cudaSuccess ||
+        cudaMallocHost((void **)&ctx->host_counts, 64 * sizeof(int)) != cudaSuccess) {
+        delete ctx;
+        return fail(nullptr, LP_ENOMEM, "lp_create: allocation failed");
+    }
+    cudaMemset(ctx->err_flag, 0, 256);
+    cudaMemset(ctx->exhausted_dev, 0, 256);
+    std::string tc_err;
+    if (!tc_init(ctx->tc, tc_err)) {
+        cudaFree(ctx->err_flag); cudaFree(ctx->exhausted_dev); cudaFreeHost(ctx->host_counts);
+        delete ctx;
+        return fail(nullptr, LP_ECUDA, "lp_create: " + tc_err);
+    }
+    *out = ctx;
+    return LP_OK;
+}
+
+extern "C" void lp_destroy(lp_ctx *ctx)
+{
+    if (!ctx) return;
+    cudaSetDevice(ctx->device);
+    cudaStreamSynchronize(ctx->ex.st);
+    free_list(ctx->model_allocs);
+    free_list(ctx->graph_allocs);
+    tc_destroy(ctx->tc);
+    cudaFree(ctx->err_flag);
+    cudaFree(ctx->exhausted_dev);
+    cudaFreeHost(ctx->host_counts);
+    delete ctx;
+}
+
+static void drop_model(lp_ctx *ctx)
+{
+    free_list(ctx->model_allocs);
+    ctx->model_bytes = 0;
+    ctx->model_set = false;
+    ctx->have_forward = ctx->have_grad = false;
+    for (auto &l : ctx->layer) l = LayerBuf();
+    for (auto &h : ctx->hop) h = HopBlock();
+}
+
+// ----------------------------------------------------------------------------------------------
+// graph
+// ----------------------------------------------------------------------------------------------
+extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const int64_t *rowptr, const int32_t *col, const float *w,
+                                   const float *X, int32_t f, int32_t ptrs_on_device)
+{
+    if (!ctx) return LP_EINVAL;
+    if (n <= 0 || n >= (int64_t)1 << 31) return fail(ctx, LP_EINVAL, "lp_load_graph: n must be in [1, 2^31)");
+    if (nnz < 0 || nnz >= (int64_t)1 << 31) return fail(ctx, LP_EINVAL, "lp_load_graph: nnz must be in [0, 2^31)");
+    if (!rowptr || (!col && nnz > 0) || !X) return fail(ctx, LP_EINVAL, "lp_load_graph: null array");
+    if (f <= 0 || f % 8 != 0 || f > 512) return fail(ctx, LP_EINVAL, "lp_load_graph: feature width must be a multiple of 8 in [8, 512]");
+    CK(cudaSetDevice(ctx->device));
+    CK(cudaStreamSynchronize(ctx->ex.st));
+    drop_model(ctx);
+    free_list(ctx->graph_allocs);
+    ctx->graph_bytes = 0;
+    ctx->loaded = false;
+    ctx->cand = nullptr;
+    ctx->n_cand = 0;
+    cudaStream_t st = ctx->ex.st;
+    const cudaMemcpyKind kind = ptrs_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+
+    int64_t *rowptr64 = nullptr;
+    std::vector<void *> tmp;
+    int64_t tmp_bytes = 0;
+#define TALLOC(ptr, count) do { cudaError_t e__ = dev_alloc(ctx, tmp, tmp_bytes, &(ptr), (count)); if (e__ != cudaSuccess) { free_list(tmp); CK(e__); } } while (0)
+    TALLOC(rowptr64, n + 1);
+    GALLOC(ctx->rowptr, n + 1);
+    GALLOC(ctx->col, nnz);
+    GALLOC(ctx->X32, n * (int64_t)f);
+    GALLOC(ctx->X16, n * (int64_t)f);
+    if (w) GALLOC(ctx->w, nnz); else ctx->w = nullptr;
+    cudaError_t e = cudaMemcpyAsync(rowptr64, rowptr, sizeof(int64_t) * (size_t)(n + 1), kind, st);
+    if (e == cudaSuccess && nnz > 0) e = cudaMemcpyAsync(ctx->col, col, sizeof(int) * (size_t)nnz, kind, st);
+    if (e == cudaSuccess && w && nnz > 0) e = cudaMemcpyAsync(ctx->w, w, sizeof(float) * (size_t)nnz, kind, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->X32, X, sizeof(float) * (size_t)n * f, kind, st);
+    if (e != cudaSuccess) { free_list(tmp); CK(e); }
+
+    cudaMemsetAsync(ctx->err_flag, 0, sizeof(int), st);
+    validate_csr_kernel<<<nblk(n + 1), 256, 0, st>>>(rowptr64, (int)n, nnz, ctx->col, ctx->rowptr, ctx->err_flag);
+    int flag = 0;
+    e = cudaMemcpyAsync(&flag, ctx->err_flag, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) { free_list(tmp); CK(e); }
+    if (flag) {
+        free_list(tmp);
+        free_list(ctx->graph_allocs);
+        char buf[160];
+        snprintf(buf, sizeof buf, "lp_load_graph: malformed CSR (flags %d: 1/2 rowptr ends, 4 rowptr order, 8 column range, 16 columns not strictly ascending)", flag);
+        return fail(ctx, LP_EINVAL, buf);
+    }
+    ctx->n = (int)n;
+    ctx->nnz = nnz;
+    ctx->f = f;
+
+    // transposed structure
+    GALLOC(ctx->colptr, n + 1);
+    GALLOC(ctx->rowidx, nnz);
+    GALLOC(ctx->perm, nnz);
+    TransposeScratch ts;
+    TALLOC(ts.keys, nnz);
+    TALLOC(ts.vals, nnz);
+    TALLOC(ts.rows, nnz);
+    TALLOC(ts.sort.keys_alt, nnz);
+    TALLOC(ts.sort.vals_alt, nnz);
+    TALLOC(ts.sort.hist, SortScratch::hist_ints(nnz));
+    TALLOC(ts.sort.scan_tmp, SortScratch::scan_ints(nnz));
+    TALLOC(ts.scan_tmp, ceil_div64(n + 1, SCAN_TILE) + 1);
+    transpose_csr(ctx->ex, ctx->rowptr, (int)n, (int)n, ctx->col, nnz, ctx->colptr, ctx->rowidx, ctx->perm, ts);
+
+    // normalisations
+    float *dtilde = nullptr;
+    TALLOC(dtilde, n);
+    GALLOC(ctx->gcn_self, n);
+    GALLOC(ctx->inv_deg, n);
+    GALLOC(ctx->gcn_val, nnz);
+    GALLOC(ctx->gcn_valT, nnz);
+    GALLOC(ctx->meanT_val, nnz);
+    degree_kernel<<<nblk(n), 256, 0, st>>>(ctx->rowptr, ctx->w, (int)n, dtilde, ctx->gcn_self, ctx->inv_deg);
+    if (nnz > 0) {
+        gcn_val_kernel<<<nblk(nnz), 256, 0, st>>>(ts.rows, ctx->col, ctx->w, dtilde, nnz, ctx->gcn_val);
+        gather_f32_kernel<<<nblk(nnz), 256, 0, st>>>(ctx->gcn_val, ctx->perm, nnz, ctx->gcn_valT);
+        gather_f32_kernel<<<nblk(nnz), 256, 0, st>>>(ctx->inv_deg, ctx->rowidx, nnz, ctx->meanT_val);
+    }
+    convert_kernel<float, bf16><<<nblk(n * (int64_t)f), 256, 0, st>>>(ctx->X32, ctx->X16, n * (int64_t)f);
+    ctx->ex.launches += 6;
+    e = cudaStreamSynchronize(st);
+    free_list(tmp);
+#undef TALLOC
+    CK(e);
+    CK_LAUNCH();
+    ctx->loaded = true;
+    return LP_OK;
+}
+
+extern "C" lp_status lp_get_structure(lp_ctx *ctx, int64_t *colptr, int32_t *rowidx, int64_t *perm)
+{
+    if (!ctx) return LP_EINVAL;
+    if (!ctx->loaded) return fail(ctx, LP_ESTATE, "lp_get_structure: no graph loaded");
+    CK(cudaSetDevice(ctx->device));
+    cudaStream_t st = ctx->ex.st;
+    if (colptr) widen_i32_kernel<<<nblk(ctx->n + 1), 256, 0, st>>>(ctx->colptr, ctx->n + 1, colptr);
+    if (rowidx && ctx->nnz > 0) CK(cudaMemcpyAsync(rowidx, ctx->rowidx, sizeof(int) * (size_t)ctx->nnz, cudaMemcpyDeviceToDevice, st));
+    if (perm && ctx->nnz > 0) widen_i32_kernel<<<nblk(ctx->nnz), 256, 0, st>>>(ctx->perm, ctx->nnz, perm);
+    CK_LAUNCH();
+    return LP_OK;
+}
+
+extern "C" lp_status lp_set_candidates(lp_ctx *ctx, const int32_t *cand, int64_t n_cand)
+{
+    if (!ctx) return LP_EINVAL;
+    if (!ctx->loaded) return fail(ctx, LP_ESTATE, "lp_set_candidates: no graph loaded");
+    CK(cudaSetDevice(ctx->device));
+    if (!cand || n_cand <= 0) { ctx->cand = nullptr; ctx->n_cand = 0; return LP_OK; }
+    if (n_cand >= (int64_t)1 << 31) return fail(ctx, LP_EINVAL, "lp_set_candidates: too many candidates");
+    GALLOC(ctx->cand, n_cand);  // lives with the graph
+    CK(cudaMemcpyAsync(ctx->cand, cand, sizeof(int) * (size_t)n_cand, cudaMemcpyDeviceToDevice, ctx->ex.st));
+    check_ids_kernel<<<nblk(n_cand), 256, 0, ctx->ex.st>>>(ctx->cand, n_cand, ctx->n, ctx->err_flag);
+    int bad = 0;
+    CK(cudaMemcpyAsync(&bad, ctx->err_flag, sizeof bad, cudaMemcpyDeviceToHost, ctx->ex.st));
+    CK(cudaStreamSynchronize(ctx->ex.st));
+    if (bad) {
+        cudaMemsetAsync(ctx->err_flag, 0, sizeof(int), ctx->ex.st);
+        ctx->cand = nullptr;
+        return fail(ctx, LP_EINVAL, "lp_set_candidates: candidate id outside [0, n)");
+    }
+    ctx->n_cand = n_cand;
+    return LP_OK;
+}
+
+// ----------------------------------------------------------------------------------------------
+// model
+// ----------------------------------------------------------------------------------------------
+extern "C" lp_status lp_param_count(const lp_ctx *ctx, int64_t *n_params)
+{
+    if (!ctx || !n_params) return LP_EINVAL;
+    if (!ctx->model_set) return fail(const_cast<lp_ctx *>(ctx), LP_ESTATE, "lp_param_count: no model set");
+    *n_params = ctx->n_params;
+    return LP_OK;
+}
+
+extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t max_batch, int32_t max_k)
+{
+    if (!ctx || !d) return LP_EINVAL;
+    if (!ctx->loaded) return fail(ctx, LP_ESTATE, "lp_set_model: load a graph first");
+    if (d->arch != LP_GCN && d->arch != LP_SAGE_MEAN) return fail(ctx, LP_EINVAL, "lp_set_model: unknown architecture");
+    if (d->prec != LP_FP32 && d->prec != LP_BF16) return fail(ctx, LP_EINVAL, "lp_set_model: unknown precision");
+    if (d->n_layers < 1 || d->n_layers > LP_MAX_LAYERS) return fail(ctx, LP_EINVAL, "lp_set_model: n_layers out of range");
+    if (d->dims[0] != ctx->f) return fail(ctx, LP_EINVAL, "lp_set_model: dims[0] differs from the feature width of the graph");
+    const int align = d->prec == LP_BF16 ? 64 : 8;
+    for (int k = 0; k <= d->n_layers; ++k)
+        if (d->dims[k] <= 0 || d->dims[k] % align != 0 || d->dims[k] > 512)
+            return fail(ctx, LP_EINVAL, "lp_set_model: widths must be multiples of 8 (FP32) or 64 (BF16), at most 512");
+    bool sampled = false;
+    for (int h = 0; h < d->n_layers; ++h) {
+        if (d->fanout[h] < 0 || d->fanout[h] > MAX_FANOUT) return fail(ctx, LP_EINVAL, "lp_set_model: fanout must be in [0, 32]");
+        sampled |= d->fanout[h] > 0;
+    }
+    if (sampled) {
+        for (int h = 0; h < d->n_layers; ++h)
+            if (d->fanout[h] == 0) return fail(ctx, LP_EINVAL, "lp_set_model: fanouts must be all zero or all positive");
+        if (d->arch != LP_SAGE_MEAN) return fail(ctx, LP_EUNSUPPORTED, "lp_set_model: neighbour sampling is implemented for SAGE-mean only");
+    }
+    if (max_batch <= 0 || max_k < 0 || max_k > 255) return fail(ctx, LP_EINVAL, "lp_set_model: max_batch must be positive, max_k in [0, 255]");
+    if (d->reject_edges && (d->max_attempts < 1 || d->max_attempts > 255)) return fail(ctx, LP_EINVAL, "lp_set_model: max_attempts must be in [1, 255]");
+    if (max_batch * (int64_t)(1 + max_k) * 2 >= (int64_t)1 << 31) return fail(ctx, LP_EINVAL, "lp_set_model: batch too large");
+    CK(cudaSetDevice(ctx->device));
+    CK(cudaStreamSynchronize(ctx->ex.st));
+    drop_model(ctx);
+    ctx->desc = *d;
+    ctx->K = d->n_layers;
+    ctx->sampled = sampled;
+    ctx->max_batch = max_batch;
+    ctx->max_k = max_k;
+    const int K = ctx->K;
+    const size_t es = d->prec == LP_BF16 ? 2 : 4;
+    const bool sage = d->arch == LP_SAGE_MEAN;
+    const int64_t n = ctx->n;
+    const int64_t E = max_batch * (1 + (int64_t)max_k);
+
+    int64_t off = 0;
+    for (int k = 0; k < K; ++k) {
+        LayerBuf &L = ctx->layer[k];
+        L.Fi = d->dims[k];
+        L.Fo = d->dims[k + 1];
+        L.Kin = sage ? 2 * L.Fi : L.Fi;
+        L.off_w = off;
+        off += (int64_t)L.Kin * L.Fo;
+        L.off_b = off;
+        off += L.Fo;
+    }
+    ctx->n_params = off;
+
+    // row capacities per hop (frontier sizes are bounded by n and by the fan-out product)
+    int64_t cap_rows[LP_MAX_LAYERS + 1];
+    if (sampled) {
+        cap_rows[0] = std::min<int64_t>(n, max_batch * (2 + 2 * (int64_t)max_k));
+        for (int h = 1; h <= K; ++h) cap_rows[h] = std::min<int64_t>(n, cap_rows[h - 1] * (1 + (int64_t)d->fanout[h - 1]));
+    } else {
+        for (int h = 0; h <= K; ++h) cap_rows[h] = n;
+    }
+    int64_t max_rows = 0;
+    for (int h = 0; h <= K; ++h) max_rows = std::max(max_rows, cap_rows[h]);
+    int maxF = 0, maxKin = 0;
+    for (int k = 0; k < K; ++k) { maxF = std::max(maxF, std::max(ctx->layer[k].Fi, ctx->layer[k].Fo)); maxKin = std::max(maxKin, ctx->layer[k].Kin); }
+
+    char *p = nullptr;
+    for (int k = 0; k < K; ++k) {
+        LayerBuf &L = ctx->layer[k];
+        // rows of layer k: destinations of hop K-k  (F_{K-k-1}); full graph: n
+        const int64_t rows = sampled ? cap_rows[K - k - 1] : n;
+        MALLOC(p, rows * L.Kin * (int64_t)es);
+        L.A = p;
+        if (!sage) {
+            if (k == 0) {
+                L.Hin = d->prec == LP_BF16 ? (void *)ctx->X16 : (void *)ctx->X32;
+            } else {
+                MALLOC(p, n * L.Fi * (int64_t)es);
+                L.Hin = p;
+            }
+        }
+        if (sampled && k < K - 1) {
+            MALLOC(p, rows * L.Fo * (int64_t)es);
+            L.Hout = p;
+        }
+    }
+    {
+        const int64_t rows = sampled ? cap_rows[0] : n;
+        MALLOC(p, rows * d->dims[K] * (int64_t)es);
+        ctx->HK = p;
+        MALLOC(p, rows * d->dims[K] * (int64_t)es);
+        ctx->dHK = p;
+    }
+    if (sage && !sampled) {  // the left half of the first operand is X itself, written once
+        LayerBuf &L = ctx->layer[0];
+        if (d->prec == LP_BF16)
+            copy_rows_kernel<bf16, bf16><<<nblk(n * L.Fi), 256, 0, ctx->ex.st>>>(ctx->X16, L.Fi, (bf16 *)L.A, L.Kin, n, L.Fi);
+        else
+            copy_rows_kernel<float, float><<<nblk(n * L.Fi), 256, 0, ctx->ex.st>>>(ctx->X32, L.Fi, (float *)L.A, L.Kin, n, L.Fi);
+        ctx->ex.launches += 1;
+    }
+    for (int i = 0; i < 2; ++i) { MALLOC(p, max_rows * maxF * (int64_t)es); ctx->dZ[i] = p; }
+    MALLOC(p, max_rows * maxKin * (int64_t)es);
+    ctx->dA = p;
+    ctx->partials_floats = std::max<int64_t>((int64_t)weight_grad_splits(max_rows) * maxKin * maxF, (int64_t)colsum_splits(max_rows) * maxF);
+    ctx->partials_floats = std::max<int64_t>(ctx->partials_floats, tc_weight_grad_partials(max_rows, maxKin, maxF));
+    MALLOC(ctx->partials, ctx->partials_floats);
+
+    // scoring and incidence
+    MALLOC(ctx->g_pos, max_batch);
+    MALLOC(ctx->g_neg, max_batch * std::max<int64_t>(max_k, 1));
+    MALLOC(ctx->loss_partials, ceil_div64(max_batch, EDGE_THREADS / 32) + 1);
+    MALLOC(ctx->inc_keys, 2 * E);
+    MALLOC(ctx->inc_slots, 2 * E);
+    MALLOC(ctx->inc_other, 2 * E);
+    MALLOC(ctx->inc_col, 2 * E);
+    MALLOC(ctx->inc_val, 2 * E);
+    MALLOC(ctx->inc_ptr, cap_rows[0] + 1);
+    MALLOC(ctx->d_pos_tmp, 2 * max_batch);
+    MALLOC(ctx->d_neg_tmp, max_batch * std::max<int64_t>(max_k, 1));
+    MALLOC(ctx->d_loss_tmp, 64);
+    MALLOC(ctx->d_grads_tmp, ctx->n_params);
+
+    // per-step sort capacity: incidence lists and (sampled) block transposes
+    int64_t sort_cap = 2 * E;
+    if (sampled) {
+        for (int h = 1; h <= K; ++h) {
+            HopBlock &hb = ctx->hop[h];
+            hb.cap_dst = (int)cap_rows[h - 1];
+            hb.cap_src = (int)cap_rows[h];
+            hb.cap_entries = (int64_t)hb.cap_dst * d->fanout[h - 1];
+            if (hb.cap_entries >= (int64_t)1 << 31) return fail(ctx, LP_EINVAL, "lp_set_model: sampled block too large");
+            if (h < K) sort_cap = std::max(sort_cap, hb.cap_entries);
+        }
+        ctx->hop[0].cap_src = (int)cap_rows[0];
+        for (int h = 0; h <= K; ++h) {
+            HopBlock &hb = ctx->hop[h];
+            MALLOC(hb.n_front_dev, 64);
+            if (h < K) {  // the outermost frontier is never materialised: layer 1 reads X by global id
+                MALLOC(hb.frontier, hb.cap_src);
+                MALLOC(hb.posmap, n);
+            }
+            if (h >= 1) {
+                MALLOC(hb.blk_ptr, (int64_t)hb.cap_dst + 1);
+                MALLOC(hb.blk_col_global, hb.cap_entries);
+                MALLOC(hb.blk_row, hb.cap_entries);
+                MALLOC(hb.inv_deg, hb.cap_dst);
+                if (h < K) {
+                    MALLOC(hb.blk_col_local, hb.cap_entries);
+                    MALLOC(hb.colptr, (int64_t)hb.cap_src + 1);
+                    MALLOC(hb.rowidx, hb.cap_entries);
+                    MALLOC(hb.perm, hb.cap_entries);
+                    MALLOC(hb.valT, hb.cap_entries);
+                    MALLOC(hb.self_idx, hb.cap_dst);
+                    MALLOC(hb.inv_self, hb.cap_src);
+                }
+            }
+        }
+        MALLOC(ctx->mark, n);
+        MALLOC(ctx->flags, n);
+        MALLOC(ctx->seed_ids, max_batch * (2 + 2 * (int64_t)max_k));
+    }
+    ctx->sort_cap = sort_cap;
+    MALLOC(ctx->sort.keys_alt, sort_cap);
+    MALLOC(ctx->sort.vals_alt, sort_cap);
+    MALLOC(ctx->sort.hist, SortScratch::hist_ints(sort_cap));
+    MALLOC(ctx->sort.scan_tmp, SortScratch::scan_ints(sort_cap));
+    MALLOC(ctx->tsp.keys, sort_cap);
+    MALLOC(ctx->tsp.vals, sort_cap);
+    MALLOC(ctx->tsp.rows, sort_cap);
+    ctx->tsp.sort = ctx->sort;
+    MALLOC(ctx->scan_tmp, ceil_div64(n + 1, SCAN_TILE) + 2);
+    ctx->tsp.scan_tmp = ctx->scan_tmp;
+    CK(cudaStreamSynchronize(ctx->ex.st));
+    CK_LAUNCH();
+    ctx->model_set = true;
+    return LP_OK;
+}
+
+// ----------------------------------------------------------------------------------------------
+// negatives
+// ----------------------------------------------------------------------------------------------
+extern "C" lp_status lp_sample_negatives(lp_ctx *ctx, uint64_t seed, uint64_t step, int32_t k, int32_t mode, const int32_t *pos_src,
+                                         int64_t B, int64_t edge_index_base, int32_t *neg_src, int32_t *neg_dst)
+{
+    if (!ctx) return LP_EINVAL;
+    if (!ctx->loaded) return fail(ctx, LP_ESTATE, "lp_sample_negatives: no graph loaded");
+    if (k < 0 || k > 255 || B < 0 || edge_index_base < 0) return fail(ctx, LP_EINVAL, "lp_sample_negatives: k in [0, 255], B >= 0, base >= 0");
+    if (mode != LP_NEG_PER_SOURCE && mode != LP_NEG_GLOBAL_PAIR) return fail(ctx, LP_EINVAL, "lp_sample_negatives: unknown mode");
+    if (B * (int64_t)k == 0) return LP_OK;
+    if (!neg_dst) return fail(ctx, LP_EINVAL, "lp_sample_negatives: neg_dst is NULL");
+    if (mode == LP_NEG_PER_SOURCE && !pos_src) return fail(ctx, LP_EINVAL, "lp_sample_negatives: pos_src is NULL");
+    if (mode == LP_NEG_GLOBAL_PAIR && !neg_src) return fail(ctx, LP_EINVAL, "lp_sample_negatives: global-pair mode needs neg_src");
+    CK(cudaSetDevice(ctx->device));
+    const int reject = ctx->model_set ? ctx->desc.reject_edges : 1;
+    const int attempts = (ctx->model_set && ctx->desc.reject_edges) ? ctx->desc.max_attempts : (reject ? 8 : 1);
+    const uint32_t space = (uint32_t)(ctx->cand ? ctx->n_cand : ctx->n);
+    cudaMemsetAsync(ctx->exhausted_dev, 0, sizeof(unsigned long long), ctx->ex.st);
+    sample_negatives_kernel<<<nblk(B * k), 256, 0, ctx->ex.st>>>(ctx->n, ctx->rowptr, ctx->col, ctx->cand, space,
+                                                                make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)), (uint32_t)step, k, mode, reject,
+                                                                attempts, pos_src, B, edge_index_base, neg_src, neg_dst, ctx->exhausted_dev);
+    ctx->ex.launches += 1;
+    CK_LAUNCH();
+    return LP_OK;
+}
+
+// ----------------------------------------------------------------------------------------------
+// the step
+// ----------------------------------------------------------------------------------------------
+template <typename T> static T *tptr(void *p) { return (T *)p; }
+
+// dense transform of one layer: Out = act(A W + b)
+template <typename T>
+static lp_status layer_linear(lp_ctx *ctx, int64_t rows, const LayerBuf &L, const float *params, T *out, int ldo, bool relu)
+{
+    if (rows <= 0) return LP_OK;
+    if (sizeof(T) == 2 && tc_linear_supported(L.Kin, L.Fo)) {
+        std::string err;
+        if (!tc_linear(ctx->tc, ctx->ex, rows, L.Fo, L.Kin, (const bf16 *)L.A, L.Kin, params + L.off_w, /*w_is_kn=*/true, params + L.off_b, relu,
+                       (bf16 *)out, ldo, err))
+            return fail(ctx, LP_ECUDA, "tensor-core GEMM: " + err);
+        return LP_OK;
+    }
+    gemm_simt<T, float, T, false, true>(ctx->ex, rows, L.Fo, L.Kin, (const T *)L.A, L.Kin, params + L.off_w, L.Fo, out, ldo, params + L.off_b, relu ? 1 : 0);
+    return LP_OK;
+}
+
+// dA[rows, Kin] = dZ[rows, Fo] * W^T
+template <typename T>
+static lp_status layer_input_grad(lp_ctx *ctx, int64_t rows, const LayerBuf &L, const float *params, const T *dZ, T *dA)
+{
+    if (rows <= 0) return LP_OK;
+    if (sizeof(T) == 2 && tc_linear_supported(L.Fo, L.Kin)) {
+        std::string err;
+        if (!tc_linear(ctx->tc, ctx->ex, rows, L.Kin, L.Fo, (const bf16 *)dZ, L.Fo, params + L.off_w, /*w_is_kn=*/false, nullptr, false, (bf16 *)dA, L.Kin,
+                       err))
+            return fail(ctx, LP_ECUDA, "tensor-core GEMM: " + err);
+        return LP_OK;
+    }
+    gemm_simt<T, float, T, false, false>(ctx->ex, rows, L.Kin, L.Fo, dZ, L.Fo, params + L.off_w, L.Fo, dA, L.Kin, nullptr, 0);
+    return LP_OK;
+}
+
+template <typename T>
+static lp_status layer_weight_grad(lp_ctx *ctx, int64_t rows, const LayerBuf &L, const T *dZ, float *grads, int accumulate)
+{
+    if (rows <= 0) {
+        if (!accumulate) cudaMemsetAsync(grads + L.off_w, 0, sizeof(float) * ((size_t)L.Kin * L.Fo + L.Fo), ctx->ex.st);
+        return LP_OK;
+    }
+    if (sizeof(T) == 2 && tc_weight_grad_supported(L.Kin, L.Fo)) {
+        std::string err;
+        if (!tc_weight_grad(ctx->tc, ctx->ex, rows, L.Kin, L.Fo, (const bf16 *)L.A, L.Kin, (const bf16 *)dZ, L.Fo, grads + L.off_w, accumulate, ctx->partials, err))
+            return fail(ctx, LP_ECUDA, "tensor-core GEMM: " + err);
+    } else {
+        weight_grad_simt<T>(ctx->ex, rows, L.Kin, L.Fo, (const T *)L.A, L.Kin, dZ, L.Fo, grads + L.off_w, accumulate, ctx->partials);
+    }
+    colsum<T>(ctx->ex, dZ, rows, L.Fo, L.Fo, grads + L.off_b, accumulate, ctx->partials);
+    return LP_OK;
+}
+
+static lp_status sync_counts(lp_ctx *ctx, const int *dev_a, const int *dev_b, int *out_a, int *out_b)
+{
+    CK(cudaMemcpyAsync(ctx->host_counts, dev_a, sizeof(int), cudaMemcpyDeviceToHost, ctx->ex.st));
+    if (dev_b) CK(cudaMemcpyAsync(ctx->host_counts + 1, dev_b, sizeof(int), cudaMemcpyDeviceToHost, ctx->ex.st));
+    CK(cudaStreamSynchronize(ctx->ex.st));
+    *out_a = ctx->host_counts[0];
+    if (dev_b) *out_b = ctx->host_counts[1];
+    return LP_OK;
+}
+
+// Sampled computational graph of the batch: F_0 = unique(seeds); hop h samples fanout[h-1]
+// in-neighbours of every node of F_{h-1}; F_h = unique(F_{h-1} u sampled).
+static lp_status build_blocks(lp_ctx *ctx, const int *pos_src, const int *pos_dst, int64_t B, const int *neg_src, const int *neg_dst, int k,
+                              uint64_t seed, uint64_t step)
+{
+    cudaStream_t st = ctx->ex.st;
+    const int n = ctx->n, K = ctx->K;
+    const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
+    CK(cudaMemsetAsync(ctx->mark, 0, (size_t)n, st));
+    mark_ids_kernel<<<nblk(B), 256, 0, st>>>(pos_src, B, n, ctx->mark);
+    mark_ids_kernel<<<nblk(B), 256, 0, st>>>(pos_dst, B, n, ctx->mark);
+    if (k > 0) mark_ids_kernel<<<nblk(B * k), 256, 0, st>>>(neg_dst, B * k, n, ctx->mark);
+    if (k > 0 && neg_src) mark_ids_kernel<<<nblk(B * k), 256, 0, st>>>(neg_src, B * k, n, ctx->mark);
+    ctx->ex.launches += 4;
+    for (int h = 0; h <= K; ++h) {
+        HopBlock &hb = ctx->hop[h];
+        if (h >= 1) {
+            HopBlock &prev = ctx->hop[h - 1];
+            hb.n_dst = prev.n_src;
+            // sample: counts -> offsets -> columns (also marks the sampled ids; F_{h-1} is still marked)
+            nbr_count_kernel<<<nblk(hb.n_dst + 1), 256, 0, st>>>(ctx->rowptr, prev.frontier, prev.n_front_dev, ctx->desc.fanout[h - 1], hb.blk_ptr, hb.n_dst);
+            exclusive_scan_i32(ctx->ex, hb.blk_ptr, hb.n_dst, hb.blk_ptr, hb.blk_ptr + hb.n_dst, ctx->scan_tmp);
+            nbr_sample_kernel<<<nblk(hb.n_dst), 256, 0, st>>>(ctx->rowptr, ctx->col, prev.frontier, prev.n_front_dev, ctx->desc.fanout[h - 1], key,
+                                                              (uint32_t)step, (uint32_t)h, hb.blk_ptr, hb.blk_col_global, hb.blk_row, ctx->mark);
+            inv_degree_kernel<<<nblk(hb.n_dst), 256, 0, st>>>(hb.blk_ptr, hb.n_dst, nullptr, hb.inv_deg);
+            ctx->ex.launches += 3;
+            if (h == K) {  // outermost hop: only the entry count is needed
+                int entries = 0, dummy = 0;
+                lp_status s = sync_counts(ctx, hb.blk_ptr + hb.n_dst, nullptr, &entries, &dummy);
+                if (s != LP_OK) return s;
+                hb.entries = entries;
+                hb.n_src = n;
+                break;
+            }
+        }
+        // frontier F_h from the marks
+        mark_to_int_kernel<<<nblk(n), 256, 0, st>>>(ctx->mark, n, ctx->flags);
+        exclusive_scan_i32(ctx->ex, ctx->flags, n, hb.posmap, hb.n_front_dev, ctx->scan_tmp);
+        compact_frontier_kernel<<<nblk(n), 256, 0, st>>>(ctx->mark, hb.posmap, n, hb.frontier);
+        ctx->ex.launches += 2;
+        int nf = 0, entries = 0;
+        lp_status s = sync_counts(ctx, hb.n_front_dev, h >= 1 ? hb.blk_ptr + hb.n_dst : nullptr, &nf, &entries);
+        if (s != LP_OK) return s;
+        hb.n_src = nf;
+        if (h >= 1) {
+            hb.entries = entries;
+            // local ids, self positions, transposed block
+            fill_i32_kernel<<<nblk(hb.n_src), 256, 0, st>>>(hb.inv_self, hb.n_src, -1);
+            self_index_kernel<<<nblk(hb.n_dst), 256, 0, st>>>(ctx->hop[h - 1].frontier, ctx->hop[h - 1].n_front_dev, hb.posmap, hb.self_idx, hb.inv_self);
+            ctx->ex.launches += 2;
+            if (hb.entries > 0) {
+                relabel_kernel<<<nblk(hb.entries), 256, 0, st>>>(hb.blk_col_global, hb.blk_ptr + hb.n_dst, hb.entries, hb.posmap, hb.blk_col_local);
+                ctx->ex.launches += 1;
+            }
+            transpose_csr(ctx->ex, hb.blk_ptr, hb.n_dst, hb.n_src, hb.blk_col_local, hb.entries, hb.colptr, hb.rowidx, hb.perm, ctx->tsp);
+            if (hb.entries > 0) {
+                gather_f32_kernel<<<nblk(hb.entries), 256, 0, st>>>(hb.inv_deg, hb.rowidx, hb.entries, hb.valT);
+                ctx->ex.launches += 1;
+            }
+        }
+    }
+    CK_LAUNCH();
+    return LP_OK;
+}
+
+template <typename T> static lp_status forward_impl(lp_ctx *ctx, const float *params)
+{
+    const int K = ctx->K;
+    const bool sage = ctx->desc.arch == LP_SAGE_MEAN;
+    const int n = ctx->n;
+    const T *Xt = sizeof(T) == 2 ? (const T *)ctx->X16 : (const T *)ctx->X32;
+    for (int k = 0; k < K; ++k) {
+        LayerBuf &L = ctx->layer[k];
+        SpmmArgs<T> a;
+        int64_t rows;
+        T *out;
+        int ldo;
+        if (!ctx->sampled) {
+            rows = n;
+            a.n_rows = n;
+            a.rowptr = ctx->rowptr;
+            a.col = ctx->col;
+            a.F = L.Fi;
+            if (sage) {
+                a.X = tptr<T>(L.A);
+                a.ldx = L.Kin;
+                a.Y = tptr<T>(L.A) + L.Fi;
+                a.ldy = L.Kin;
+                a.row_scale = ctx->inv_deg;
+            } else {
+                a.X = tptr<T>(L.Hin);
+                a.ldx = L.Fi;
+                a.Y = tptr<T>(L.A);
+                a.ldy = L.Fi;
+                a.val = ctx->gcn_val;
+                a.init = a.X;
+                a.ldinit = L.Fi;
+                a.init_coef = ctx->gcn_self;
+            }
+            if (k == K - 1) { out = tptr<T>(ctx->HK); ldo = L.Fo; }
+            else if (sage) { out = tptr<T>(ctx->layer[k + 1].A); ldo = ctx->layer[k + 1].Kin; }
+            else { out = tptr<T>(ctx->layer[k + 1].Hin); ldo = L.Fo; }
+        } else {
+            HopBlock &hb = ctx->hop[K - k];
+            rows = hb.n_dst;
+            a.n_rows = hb.n_dst;
+            a.rowptr = hb.blk_ptr;
+            a.F = L.Fi;
+            a.row_scale = hb.inv_deg;
+            a.Y = tptr<T>(L.A) + L.Fi;
+            a.ldy = L.Kin;
+            a.self_out = tptr<T>(L.A);
+            a.ldself = L.Kin;
+            if (k == 0) {  // innermost layer reads the feature matrix by global id
+                a.X = Xt;
+                a.ldx = L.Fi;
+                a.col = hb.blk_col_global;
+                a.self_idx = ctx->hop[K - 1].frontier;
+            } else {
+                a.X = tptr<T>(ctx->layer[k - 1].Hout);
+                a.ldx = L.Fi;
+                a.col = hb.blk_col_local;
+                a.self_idx = hb.self_idx;
+            }
+            if (k == K - 1) { out = tptr<T>(ctx->HK); ldo = L.Fo; } else { out = tptr<T>(L.Hout); ldo = L.Fo; }
+        }
+        if (rows > 0 && !spmm_launch<T>(ctx->ex, a)) return fail(ctx, LP_EUNSUPPORTED, "aggregation width not supported");
+        lp_status s = layer_linear<T>(ctx, rows, L, params, out, ldo, k < K - 1);
+        if (s != LP_OK) return s;
+    }
+    ctx->rows_out = ctx->sampled ? ctx->hop[0].n_src : n;
+    ctx->have_forward = true;
+    CK_LAUNCH();
+    return LP_OK;
+}
+
+template <typename T>
+static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src, const int *pos_dst, int64_t B, const int *neg_src, const int *neg_dst,
+                            int k, uint64_t seed, uint64_t step, float *loss, float *grads, int accumulate)
+{
+    cudaStream_t st = ctx->ex.st;
+    const int K = ctx->K;
+    const bool sage = ctx->desc.arch == LP_SAGE_MEAN;
+    const int D = ctx->desc.dims[K];
+    // bad ids are clamped by every consumer and reported through the context's error word
+    check_ids_kernel<<<nblk(B), 256, 0, st>>>(pos_src, B, ctx->n, ctx->err_flag);
+    check_ids_kernel<<<nblk(B), 256, 0, st>>>(pos_dst, B, ctx->n, ctx->err_flag);
+    if (k > 0) check_ids_kernel<<<nblk(B * k), 256, 0, st>>>(neg_dst, B * k, ctx->n, ctx->err_flag);
+    if (k > 0 && neg_src) check_ids_kernel<<<nblk(B * k), 256, 0, st>>>(neg_src, B * k, ctx->n, ctx->err_flag);
+    ctx->ex.launches += 2 + (k > 0) + (k > 0 && neg_src);
+    if (ctx->sampled) {
+        lp_status s = build_blocks(ctx, pos_src, pos_dst, B, neg_src, neg_dst, k, seed, step);
+        if (s != LP_OK) return s;
+    }
+    lp_status s = forward_impl<T>(ctx, params);
+    if (s != LP_OK) return s;
+    const int rows_out = ctx->rows_out;
+    const int *idmap = ctx->sampled ? ctx->hop[0].posmap : nullptr;
+    const int64_t E = B * (1 + (int64_t)k);
+    const float inv_N = 1.f / (float)E;
+    T *HK = tptr<T>(ctx->HK);
+
+    // scores, loss, per-edge gradients
+    const unsigned eblocks = nblk(B, EDGE_THREADS / 32);
+    constexpr int VN = Vec16<T>::N;
+    const int chunks = D / VN;
+    if (chunks <= 32) edge_score_bce_kernel<T, 1><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials);
+    else if (chunks <= 64) edge_score_bce_kernel<T, 2><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials);
+    else edge_score_bce_kernel<T, 4><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials);
+    loss_reduce_kernel<<<1, 256, 0, st>>>(ctx->loss_partials, eblocks, inv_N, loss);
+
+    // incidence lists of the scored edges, grouped by node (stable sort => fixed summation order)
+    CK(cudaMemsetAsync(ctx->inc_ptr, 0, sizeof(int) * ((size_t)rows_out + 1), st));
+    incidence_keys_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->inc_keys, ctx->inc_slots, ctx->inc_other, ctx->inc_ptr);
+    exclusive_scan_i32(ctx->ex, ctx->inc_ptr, rows_out, ctx->inc_ptr, ctx->inc_ptr + rows_out, ctx->scan_tmp);
+    radix_sort_pairs(ctx->ex, ctx->inc_keys, ctx->inc_slots, 2 * E, bits_for(rows_out), ctx->sort);
+    incidence_fill_kernel<<<nblk(2 * E), 256, 0, st>>>(ctx->inc_slots, 2 * E, ctx->inc_other, B, ctx->g_pos, ctx->g_neg, ctx->inc_col, ctx->inc_val);
+    ctx->ex.launches += 4;
+
+    // dL/dH^(K)[v] = sum over incident scored edges of g_e * h_other
+    T *dZ = tptr<T>(ctx->dHK);
+    int cur = 1;
+    {
+        SpmmArgs<T> a;
+        a.n_rows = rows_out;
+        a.rowptr = ctx->inc_ptr;
+        a.col = ctx->inc_col;
+        a.val = ctx->inc_val;
+        a.X = HK;
+        a.ldx = D;
+        a.F = D;
+        a.Y = dZ;
+        a.ldy = D;
+        if (rows_out > 0 && !spmm_launch<T>(ctx->ex, a)) return fail(ctx, LP_EUNSUPPORTED, "embedding width not supported");
+    }
+    ctx->have_grad = true;
+
+    // backward through the layers
+    for (int l = K - 1; l >= 0; --l) {
+        LayerBuf &L = ctx->layer[l];
+        const int64_t rows = ctx->sampled ? ctx->hop[K - l].n_dst : ctx->n;
+        s = layer_weight_grad<T>(ctx, rows, L, dZ, grads, accumulate);
+        if (s != LP_OK) return s;
+        if (l == 0) break;
+        T *dA = tptr<T>(ctx->dA);
+        s = layer_input_grad<T>(ctx, rows, L, params, dZ, dA);
+        if (s != LP_OK) return s;
+        T *dZn = tptr<T>(ctx->dZ[cur ^ 1]);
+        SpmmArgs<T> a;
+        a.F = L.Fi;
+        a.Y = dZn;
+        a.ldy = L.Fi;
+        if (!ctx->sampled) {
+            a.n_rows = ctx->n;
+            a.rowptr = ctx->colptr;
+            a.col = ctx->rowidx;
+            if (sage) {
+                a.val = ctx->meanT_val;
+                a.X = dA + L.Fi;
+                a.ldx = L.Kin;
+                a.init = dA;
+                a.ldinit = L.Kin;
+                a.relu_ref = tptr<T>(L.A);  // left half = H^(l)
+                a.ldref = L.Kin;
+            } else {
+                a.val = ctx->gcn_valT;
+                a.X = dA;
+                a.ldx = L.Fi;
+                a.init = dA;
+                a.ldinit = L.Fi;
+                a.init_coef = ctx->gcn_self;
+                a.relu_ref = tptr<T>(L.Hin);
+                a.ldref = L.Fi;
+            }
+        } else {
+            HopBlock &hb = ctx->hop[K - l];
+            a.n_rows = hb.n_src;
+            a.rowptr = hb.colptr;
+            a.col = hb.rowidx;
+            a.val = hb.valT;
+            a.X = dA + L.Fi;
+            a.ldx = L.Kin;
+            a.init = dA;
+            a.ldinit = L.Kin;
+            a.init_idx = hb.inv_self;
+            a.relu_ref = tptr<T>(ctx->layer[l - 1].Hout);
+            a.ldref = L.Fi;
+        }
+        if (a.n_rows > 0 && !spmm_launch<T>(ctx->ex, a)) return fail(ctx, LP_EUNSUPPORTED, "aggregation width not supported");
+        dZ = dZn;
+        cur ^= 1;
+    }
+    CK_LAUNCH();
+    return LP_OK;
+}
+
+static lp_status check_step_args(lp_ctx *ctx, const char *who, const void *params, const void *a, const void *b, int64_t B, const void *neg_dst, int k)
+{
+    if (!ctx->model_set) return fail(ctx, LP_ESTATE, std::string(who) + ": set a model first");
+    if (!params) return fail(ctx, LP_EINVAL, std::string(who) + ": params is NULL");
+    if (B <= 0 || B > ctx->max_batch) return fail(ctx, LP_EINVAL, std::string(who) + ": B must be in [1, max_batch]");
+    if (k < 0 || k > ctx->max_k) return fail(ctx, LP_EINVAL, std::string(who) + ": k must be in [0, max_k]");
+    if (!a || !b) return fail(ctx, LP_EINVAL, std::string(who) + ": edge arrays are NULL");
+    if (k > 0 && !neg_dst) return fail(ctx, LP_EINVAL, std::string(who) + ": neg_dst is NULL");
+    return LP_OK;
+}
+
+extern "C" lp_status lp_train_step(lp_ctx *ctx, const float *params, const int32_t *pos_src, const int32_t *pos_dst, int64_t B,
+                                   const int32_t *neg_src, const int32_t *neg_dst, int32_t k, uint64_t seed, uint64_t step, float *loss,
+                                   float *grads, int32_t accumulate)
+{
+    if (!ctx) return LP_EINVAL;
+    lp_status s = check_step_args(ctx, "lp_train_step", params, pos_src, pos_dst, B, neg_dst, k);
+    if (s != LP_OK) return s;
+    if (!loss || !grads) return fail(ctx, LP_EINVAL, "lp_train_step: loss or grads is NULL");
+    CK(cudaSetDevice(ctx->device));
+    if (ctx->desc.prec == LP_BF16) s = train_impl<bf16>(ctx, params, pos_src, pos_dst, B, neg_src, neg_dst, k, seed, step, loss, grads, accumulate);
+    else s = train_impl<float>(ctx, params, pos_src, pos_dst, B, neg_src, neg_dst, k, seed, step, loss, grads, accumulate);
+    if (s != LP_OK) return s;
+    return tc_check(ctx->tc, ctx->ex, false, ctx->err);
+}
+
+extern "C" lp_status lp_adam_step(lp_ctx *ctx, float *params, float *adam_m, float *adam_v, const float *grads, float grad_scale, float lr,
+                                  float beta1, float beta2, float eps, int64_t t)
+{
+    if (!ctx) return LP_EINVAL;
+    if (!ctx->model_set) return fail(ctx, LP_ESTATE, "lp_adam_step: set a model first");
+    if (!params || !grads) return fail(ctx, LP_EINVAL, "lp_adam_step: params or grads is NULL");
+    if ((adam_m == nullptr) != (adam_v == nullptr)) return fail(ctx, LP_EINVAL, "lp_adam_step: pass both moment arrays or neither");
+    if (adam_m && t < 1) return fail(ctx, LP_EINVAL, "lp_adam_step: t counts from 1");
+    CK(cudaSetDevice(ctx->device));
+    const int64_t np = ctx->n_params;
+    if (adam_m) {
+        const double c1 = 1.0 - std::pow((double)beta1, (double)t), c2 = 1.0 - std::pow((double)beta2, (double)t);
+        adam_kernel<<<nblk(np), 256, 0, ctx->ex.st>>>(params, adam_m, adam_v, grads, np, grad_scale, lr, beta1, beta2, eps, (float)(1.0 / c1), (float)(1.0 / c2));
+    } else {
+        sgd_kernel<<<nblk(np), 256, 0, ctx->ex.st>>>(params, grads, np, grad_scale, lr);
+    }
+    ctx->ex.launches += 1;
+    CK_LAUNCH();
+    return LP_OK;
+}
+
+extern "C" lp_status lp_train_step_host(lp_ctx *ctx, float *params, const int32_t *pos_src_host, const int32_t *pos_dst_host, int64_t B, int32_t k,
+                                        uint64_t seed, uint64_t step, int64_t edge_index_base, float *adam_m, float *adam_v, int64_t adam_t,
+                                        float *loss_host, float *grads_host)
+{
+    if (!ctx) return LP_EINVAL;
+    lp_status s = check_step_args(ctx, "lp_train_step_host", params, pos_src_host, pos_dst_host, B, (const void *)1, k);
+    if (s != LP_OK) return s;
+    if (!loss_host) return fail(ctx, LP_EINVAL, "lp_train_step_host: loss_host is NULL");
+    CK(cudaSetDevice(ctx->device));
+    cudaStream_t st = ctx->ex.st;
+    int *ps = ctx->d_pos_tmp, *pd = ctx->d_pos_tmp + ctx->max_batch;
+    CK(cudaMemcpyAsync(ps, pos_src_host, sizeof(int) * (size_t)B, cudaMemcpyHostToDevice, st));
+    CK(cudaMemcpyAsync(pd, pos_dst_host, sizeof(int) * (size_t)B, cudaMemcpyHostToDevice, st));
+    if (k > 0) {
+        s = lp_sample_negatives(ctx, seed, step, k, LP_NEG_PER_SOURCE, ps, B, edge_index_base, nullptr, ctx->d_neg_tmp);
+        if (s != LP_OK) return s;
+    }
+    s = lp_train_step(ctx, params, ps, pd, B, nullptr, ctx->d_neg_tmp, k, seed, step, ctx->d_loss_tmp, ctx->d_grads_tmp, 0);
+    if (s != LP_OK) return s;
+    if (adam_m || adam_v) {
+        s = lp_adam_step(ctx, params, adam_m, adam_v, ctx->d_grads_tmp, 1.f, 1e-3f, 0.9f, 0.999f, 1e-8f, adam_t);
+        if (s != LP_OK) return s;
+    }
+    CK(cudaMemcpyAsync(loss_host, ctx->d_loss_tmp, sizeof(float), cudaMemcpyDeviceToHost, st));
+    if (grads_host) CK(cudaMemcpyAsync(grads_host, ctx->d_grads_tmp, sizeof(float) * (size_t)ctx->n_params, cudaMemcpyDeviceToHost, st));
+    int bad = 0;
+    CK(cudaMemcpyAsync(&bad, ctx->err_flag, sizeof bad, cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    if (bad) {
+        cudaMemsetAsync(ctx->err_flag, 0, sizeof(int), st);
+        return fail(ctx, LP_EINVAL, "lp_train_step_host: a node id is outside [0, n)");
+    }
+    return tc_check(ctx->tc, ctx->ex, true, ctx->err);
+}
+
+template <typename T>
+static lp_status score_impl(lp_ctx *ctx, const float *params, const int *src, const int *dst, int64_t E, uint64_t seed, uint64_t step, float *scores)
+{
+    if (ctx->sampled) {
+        lp_status s = build_blocks(ctx, src, dst, E, nullptr, nullptr, 0, seed, step);
+        if (s != LP_OK) return s;
+    }
+    lp_status s = forward_impl<T>(ctx, params);
+    if (s != LP_OK) return s;
+    const int D = ctx->desc.dims[ctx->K];
+    const int *idmap = ctx->sampled ? ctx->hop[0].posmap : nullptr;
+    constexpr int VN = Vec16<T>::N;
+    const int chunks = D / VN;
+    const unsigned blocks = nblk(E, EDGE_THREADS / 32);
+    if (chunks <= 32) edge_score_kernel<T, 1><<<blocks, EDGE_THREADS, 0, ctx->ex.st>>>(tptr<T>(ctx->HK), D, D, ctx->n, idmap, src, dst, E, scores);
+    else if (chunks <= 64) edge_score_kernel<T, 2><<<blocks, EDGE_THREADS, 0, ctx->ex.st>>>(tptr<T>(ctx->HK), D, D, ctx->n, idmap, src, dst, E, scores);
+    else edge_score_kernel<T, 4><<<blocks, EDGE_THREADS, 0, ctx->ex.st>>>(tptr<T>(ctx->HK), D, D, ctx->n, idmap, src, dst, E, scores);
+    ctx->ex.launches += 1;
+    CK_LAUNCH();
+    return LP_OK;
+}
+
+extern "C" lp_status lp_score(lp_ctx *ctx, const float *params, const int32_t *src, const int32_t *dst, int64_t E, uint64_t seed, uint64_t step,
+                              float *scores)
+{
+    if (!ctx) return LP_EINVAL;
+    if (!ctx->model_set) return fail(ctx, LP_ESTATE, "lp_score: set a model first");
+    if (!params || !src || !dst || !scores) return fail(ctx, LP_EINVAL, "lp_score: null array");
+    if (E <= 0) return fail(ctx, LP_EINVAL, "lp_score: E must be positive");
+    if (ctx->sampled && E > ctx->max_batch) return fail(ctx, LP_EINVAL, "lp_score: sampled models score at most max_batch pairs per call");
+    CK(cudaSetDevice(ctx->device));
+    lp_status s = ctx->desc.prec == LP_BF16 ? score_impl<bf16>(ctx, params, src, dst, E, seed, step, scores)
+                                            : score_impl<float>(ctx, params, src, dst, E, seed, step, scores);
+    if (s != LP_OK) return s;
+    return tc_check(ctx->tc, ctx->ex, false, ctx->err);
+}
+
+// ----------------------------------------------------------------------------------------------
+// inspection
+// ----------------------------------------------------------------------------------------------
+template <typename T> static void to_f32(lp_ctx *ctx, const T *src, int64_t lds, float *dst, int64_t rows, int F)
+{
+    if (rows <= 0) return;
+    copy_rows_kernel<T, float><<<nblk(rows * F), 256, 0, ctx->ex.st>>>(src, lds, dst, F, rows, F);
+    ctx->ex.launches += 1;
+}
+
+extern "C" lp_status lp_get_embeddings(lp_ctx *ctx, int32_t layer, float *out)
+{
+    if (!ctx || !out) return LP_EINVAL;
+    if (!ctx->model_set || !ctx->have_forward) return fail(ctx, LP_ESTATE, "lp_get_embeddings: run a forward pass first");
+    const int K = ctx->K;
+    if (layer < 1 || layer > K) return fail(ctx, LP_EINVAL, "lp_get_embeddings: layer must be in [1, K]");
+    CK(cudaSetDevice(ctx->device));
+    const bool b16 = ctx->desc.prec == LP_BF16;
+    const int F = ctx->desc.dims[layer];
+    const void *src;
+    int64_t ld, rows;
+    if (layer == K) { src = ctx->HK; ld = F; rows = ctx->rows_out; }
+    else if (ctx->sampled) { src = ctx->layer[layer - 1].Hout; ld = F; rows = ctx->hop[K - layer + 1].n_dst; }
+    else if (ctx->desc.arch == LP_SAGE_MEAN) { src = ctx->layer[layer].A; ld = ctx->layer[layer].Kin; rows = ctx->n; }
+    else { src = ctx->layer[layer].Hin; ld = F; rows = ctx->n; }
+    if (b16) to_f32<bf16>(ctx, (const bf16 *)src, ld, out, rows, F); else to_f32<float>(ctx, (const float *)src, ld, out, rows, F);
+    CK_LAUNCH();
+    return LP_OK;
+}
+
+extern "C" lp_status lp_get_output_gradient(lp_ctx *ctx, float *out)
+{
+    if (!ctx || !out) return LP_EINVAL;
+    if (!ctx->model_set || !ctx->have_grad) return fail(ctx, LP_ESTATE, "lp_get_output_gradient: run lp_train_step first");
+    CK(cudaSetDevice(ctx->device));
+    const int D = ctx->desc.dims[ctx->K];
+    if (ctx->desc.prec == LP_BF16) to_f32<bf16>(ctx, (const bf16 *)ctx->dHK, D, out, ctx->rows_out, D);
+    else to_f32<float>(ctx, (const float *)ctx->dHK, D, out, ctx->rows_out, D);
+    CK_LAUNCH();
+    return LP_OK;
+}
+
+extern "C" lp_status lp_get_block(lp_ctx *ctx, int32_t hop, int32_t *frontier, int64_t *blk_ptr, int32_t *blk_col)
+{
+    if (!ctx) return LP_EINVAL;
+    if (!ctx->model_set || !ctx->sampled || !ctx->have_forward) return fail(ctx, LP_ESTATE, "lp_get_block: no sampled step has run");
+    if (hop < 0 || hop > ctx->K) return fail(ctx, LP_EINVAL, "lp_get_block: hop out of range");
+    CK(cudaSetDevice(ctx->device));
+    HopBlock &hb = ctx->hop[hop];
+    cudaStream_t st = ctx->ex.st;
+    if (frontier) {
+        if (hop == ctx->K) return fail(ctx, LP_EUNSUPPORTED, "lp_get_block: the outermost frontier is not materialised (use the block columns)");
+        if (hb.n_src > 0) CK(cudaMemcpyAsync(frontier, hb.frontier, sizeof(int) * (size_t)hb.n_src, cudaMemcpyDeviceToDevice, st));
+    }
+    if (hop >= 1) {
+        if (blk_ptr) widen_i32_kernel<<<nblk(hb.n_dst + 1), 256, 0, st>>>(hb.blk_ptr, hb.n_dst + 1, blk_ptr);
+        if (blk_col && hb.entries > 0) CK(cudaMemcpyAsync(blk_col, hb.blk_col_global, sizeof(int) * (size_t)hb.entries, cudaMemcpyDeviceToDevice, st));
+    }
+    CK_LAUNCH();
+    return LP_OK;
+}
+
+extern "C" lp_status lp_get_stats(lp_ctx *ctx, lp_stats *out)
+{
+    if (!ctx || !out) return LP_EINVAL;
+    CK(cudaSetDevice(ctx->device));
+    memset(out, 0, sizeof *out);
+    unsigned long long ex = 0;
+    int bad = 0;
+    CK(cudaMemcpyAsync(&ex, ctx->exhausted_dev, sizeof ex, cudaMemcpyDeviceToHost, ctx->ex.st));
+    CK(cudaMemcpyAsync(&bad, ctx->err_flag, sizeof bad, cudaMemcpyDeviceToHost, ctx->ex.st));
+    CK(cudaStreamSynchronize(ctx->ex.st));
+    if (bad) {
+        cudaMemsetAsync(ctx->err_flag, 0, sizeof(int), ctx->ex.st);
+        return fail(ctx, LP_EINVAL, "a node id outside [0, n) was passed to an earlier call (it was clamped; results of that call are invalid)");
+    }
+    out->negatives_exhausted = (int64_t)ex;
+    if (ctx->model_set && ctx->sampled) {
+        for (int h = 0; h <= ctx->K; ++h) out->block_nodes[h] = ctx->hop[h].n_src;
+        for (int h = 1; h <= ctx->K; ++h) out->block_edges[h - 1] = ctx->hop[h].entries;
+    }
+    out->workspace_bytes = ctx->graph_bytes + ctx->model_bytes;
+    out->kernel_launches = ctx->ex.launches;
+    return LP_OK;
+}
+
+// ----------------------------------------------------------------------------------------------
+// single operators
+// ----------------------------------------------------------------------------------------------
+template <typename T> static lp_status op_aggregate_impl(lp_ctx *ctx, int arch, int transpose, const T *H, int F, T *M)
+{
+    SpmmArgs<T> a;
+    a.n_rows = ctx->n;
+    a.X = H;
+    a.ldx = F;
+    a.F = F;
+    a.Y = M;
+    a.ldy = F;
+    if (!transpose) {
+        a.rowptr = ctx->rowptr;
+        a.col = ctx->col;
+        if (arch == LP_GCN) { a.val = ctx->gcn_val; a.init = H; a.ldinit = F; a.init_coef = ctx->gcn_self; }
+        else a.row_scale = ctx->inv_deg;
+    } else {
+        a.rowptr = ctx->colptr;
+        a.col = ctx->rowidx;
+        if (arch == LP_GCN) { a.val = ctx->gcn_valT; a.init = H; a.ldinit = F; a.init_coef = ctx->gcn_self; }
+        else a.val = ctx->meanT_val;
+    }
+    if (!spmm_launch<T>(ctx->ex, a)) return fail(ctx, LP_EINVAL, "lp_op_aggregate: F must be a multiple of 8, at most 512");
+    CK_LAUNCH();
+    return LP_OK;
+}
+
+extern "C" lp_status lp_op_aggregate(lp_ctx *ctx, int32_t arch, int32_t transpose, int32_t is_bf16, const void *H, int32_t F, void *M)
+{
+    if (!ctx) return LP_EINVAL;
+    if (!ctx->loaded) return fail(ctx, LP_ESTATE, "lp_op_aggregate: no graph loaded");
+    if (!H || !M || H == M) return fail(ctx, LP_EINVAL, "lp_op_aggregate: H and M must be distinct non-null arrays");
+    if (arch != LP_GCN && arch != LP_SAGE_MEAN) return fail(ctx, LP_EINVAL, "lp_op_aggregate: unknown architecture");
+    if (F <= 0 || F % 8 != 0 || F > 512) return fail(ctx, LP_EINVAL, "lp_op_aggregate: F must be a multiple of 8, at most 512");
+    CK(cudaSetDevice(ctx->device));
+    return is_bf16 ? op_aggregate_impl<bf16>(ctx, arch, transpose, (const bf16 *)H, F, (bf16 *)M)
+                   : op_aggregate_impl<float>(ctx, arch, transpose, (const float *)H, F, (float *)M);
+}
+
+extern "C" lp_status lp_op_linear(lp_ctx *ctx, int32_t prec, int64_t M, int32_t N, int32_t K, const void *A, const void *B, int32_t trans_b,
+                                  const float *bias, int32_t relu, void *C)
+{
+    if (!ctx) return LP_EINVAL;
+    if (!A || !B || !C || M <= 0 || N <= 0 || K <= 0) return fail(ctx, LP_EINVAL, "lp_op_linear: bad argument");
+    CK(cudaSetDevice(ctx->device));
+    if (prec == LP_FP32) {
+        if (trans_b) gemm_simt<float, float, float, false, false>(ctx->ex, M, N, K, (const float *)A, K, (const float *)B, K, (float *)C, N, bias, relu);
+        else gemm_simt<float, float, float, false, true>(ctx->ex, M, N, K, (const float *)A, K, (const float *)B, N, (float *)C, N, bias, relu);
+    } else if (prec == LP_BF16) {
+        if (tc_linear_supported(K, N)) {
+            std::string err;
+            if (!tc_linear_bf16_b(ctx->tc, ctx->ex, M, N, K, (const bf16 *)A, K, (const bf16 *)B, trans_b != 0, bias, relu != 0, (bf16 *)C, N, err))
+                return fail(ctx, LP_ECUDA, "lp_op_linear: " + err);
+        } else if (trans_b) {
+            gemm_simt<bf16, bf16, bf16, false, false>(ctx->ex, M, N, K, (const bf16 *)A, K, (const bf16 *)B, K, (bf16 *)C, N, bias, relu);
+        } else {
+            gemm_simt<bf16, bf16, bf16, false, true>(ctx->ex, M, N, K, (const bf16 *)A, K, (const bf16 *)B, N, (bf16 *)C, N, bias, relu);
+        }
+    } else {
+        return fail(ctx, LP_EINVAL, "lp_op_linear: unknown precision");
+    }
+    CK_LAUNCH();
+    return tc_check(ctx->tc, ctx->ex, false, ctx->err);
+}
+
+extern "C" lp_status lp_op_weight_grad(lp_ctx *ctx, int32_t prec, int64_t M, int32_t N, int32_t K, const void *A, const void *dZ, float *dW)
+{
+    if (!ctx) return LP_EINVAL;
+    if (!A || !dZ || !dW || M <= 0 || N <= 0 || K <= 0) return fail(ctx, LP_EINVAL, "lp_op_weight_grad: bad argument");
+    CK(cudaSetDevice(ctx->device));
+    float *partials = nullptr;
+    const int64_t need = std::max<int64_t>((int64_t)weight_grad_splits(M) * K * N, tc_weight_grad_partials(M, K, N));
+    CK(cudaMalloc((void **)&partials, sizeof(float) * (size_t)need));
+    lp_status rc = LP_OK;
+    if (prec == LP_FP32) {
+        weight_grad_simt<float>(ctx->ex, M, K, N, (const float *)A, K, (const float *)dZ, N, dW, 0, partials);
+    } else if (prec == LP_BF16) {
+        std::string err;
+        if (tc_weight_grad_supported(K, N)) {
+            if (!tc_weight_grad(ctx->tc, ctx->ex, M, K, N, (const bf16 *)A, K, (const bf16 *)dZ, N, dW, 0, partials, err)) rc = fail(ctx, LP_ECUDA, "lp_op_weight_grad: " + err);
+        } else {
+            weight_grad_simt<bf16>(ctx->ex, M, K, N, (const bf16 *)A, K, (const bf16 *)dZ, N, dW, 0, partials);
+        }
+    } else {
+        rc = fail(ctx, LP_EINVAL, "lp_op_weight_grad: unknown precision");
+    }
+    cudaStreamSynchronize(ctx->ex.st);
+    cudaFree(partials);
+    if (rc != LP_OK) return rc;
+    CK_LAUNCH();
+    return tc_check(ctx->tc, ctx->ex, false, ctx->err);
+}

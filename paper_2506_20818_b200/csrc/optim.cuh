@@ -1,0 +1,54 @@
+// Weight update (Algorithm 1: average the workers' gradients, then update; Section IV: Adam with
+// learning rate 1e-3) and small element-wise helpers.
+#pragma once
+#include "common.cuh"
+#include "scan_sort.cuh"
+
+// g = scale * grad;  m = b1 m + (1-b1) g;  v = b2 v + (1-b2) g^2;
+// p -= lr * (m / c1) / (sqrt(v / c2) + eps),  c1 = 1 - b1^t, c2 = 1 - b2^t (computed on the host in double)
+__global__ void adam_kernel(float *__restrict__ p, float *__restrict__ m, float *__restrict__ v, const float *__restrict__ grad, int64_t n,
+                            float scale, float lr, float b1, float b2, float eps, float inv_c1, float inv_c2)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const float g = scale * grad[i];
+    const float mi = b1 * m[i] + (1.f - b1) * g;
+    const float vi = b2 * v[i] + (1.f - b2) * g * g;
+    m[i] = mi;
+    v[i] = vi;
+    p[i] -= lr * (mi * inv_c1) / (sqrtf(vi * inv_c2) + eps);
+}
+
+__global__ void sgd_kernel(float *__restrict__ p, const float *__restrict__ grad, int64_t n, float scale, float lr)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) p[i] -= lr * scale * grad[i];
+}
+
+template <typename TS, typename TD> __global__ void convert_kernel(const TS *__restrict__ src, TD *__restrict__ dst, int64_t n)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) dst[i] = from_f<TD>(to_f<TS>(src[i]));
+}
+
+// dst[r, 0:F] (leading dimension ldd) = src[r, 0:F] (leading dimension lds), with conversion
+template <typename TS, typename TD>
+__global__ void copy_rows_kernel(const TS *__restrict__ src, int64_t lds, TD *__restrict__ dst, int64_t ldd, int64_t rows, int F)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= rows * F) return;
+    const int64_t r = i / F;
+    const int c = (int)(i - r * F);
+    dst[r * ldd + c] = from_f<TD>(to_f<TS>(src[r * lds + c]));
+}
+
+// W[K, N] row-major float -> Wt[N, K] row-major bf16 (K contiguous) and, optionally, W as bf16
+__global__ void weights_to_bf16_kernel(const float *__restrict__ W, int K, int N, bf16 *__restrict__ Wt, bf16 *__restrict__ Wc)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= K * N) return;
+    const int k = i / N, n = i - k * N;
+    const bf16 x = __float2bfloat16_rn(W[i]);
+    if (Wt) Wt[(size_t)n * K + k] = x;
+    if (Wc) Wc[i] = x;
+}
