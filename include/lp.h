@@ -176,9 +176,11 @@ lp_status lp_train_step_host(lp_ctx *ctx, float *params, const int32_t *pos_src_
  * m = b1 m + (1-b1) g;  v = b2 v + (1-b2) g^2;
  * params -= lr * (m / (1 - b1^t)) / (sqrt(v / (1 - b2^t)) + eps).   t counts from 1.
  * With adam_m == NULL the plain rule W <- W - lr * g of Algorithm 1 is applied.
- * All arrays are device float32 [n_params].  Does not synchronise. */
-lp_status lp_adam_step(lp_ctx *ctx, float *params, float *adam_m, float *adam_v, const float *grads, float grad_scale,
-                       float lr, float beta1, float beta2, float eps, int64_t t);
+ * All arrays are device float32 [n_params].  The scalar hyper-parameters are doubles so that
+ * 1 - beta and the bias corrections are formed exactly on the host before being rounded to
+ * float32 for the kernel.  Does not synchronise. */
+lp_status lp_adam_step(lp_ctx *ctx, float *params, float *adam_m, float *adam_v, const float *grads, double grad_scale,
+                       double lr, double beta1, double beta2, double eps, int64_t t);
 
 /* ---- inference, Eq. 2 ------------------------------------------------------------------- */
 
@@ -207,7 +209,8 @@ lp_status lp_get_output_gradient(lp_ctx *ctx, float *out);
 lp_status lp_get_block(lp_ctx *ctx, int32_t hop, int32_t *frontier, int64_t *blk_ptr, int32_t *blk_col);
 
 /* Counters.  Synchronises the stream.  Returns LP_EINVAL (once) when an earlier step was
- * given a node id outside [0, n). */
+ * given a node id outside [0, n), and LP_ETIMEOUT (once) when a bounded wait inside a
+ * tensor-core kernel of an earlier call expired. */
 lp_status lp_get_stats(lp_ctx *ctx, lp_stats *out);
 
 /* ---- single operators (used by the parity tests and the roofline benchmark) -------------- */

@@ -56,13 +56,20 @@ def _layer_graphs(g, n_layers: int, blocks):
     return out
 
 
-def forward(g, X: np.ndarray, params: np.ndarray, arch: str, dims: Sequence[int], blocks=None):
+def forward(g, X: np.ndarray, params: np.ndarray, arch: str, dims: Sequence[int], blocks=None, relu_ties=None,
+            tie_tol: float = 0.0):
     """K-layer encoder (Eq. 1).  Layer k: A = AGG(H^(k-1)) [gcn] or [H^(k-1) | mean] [sage];
-    Z = A W + b; H^(k) = ReLU(Z) for k < K and Z for k = K.  Returns the per-layer cache."""
+    Z = A W + b; H^(k) = ReLU(Z) for k < K and Z for k = K.  Returns the per-layer cache.
+
+    ReLU turns a floating-point value into a yes/no decision (is the unit active?).  When a
+    pre-activation is zero up to rounding, FP64 and the FP32 arithmetic under test may decide
+    differently although both are right.  relu_ties[k] (bool [n, F_{k+1}], the decisions of the
+    implementation under test) is adopted ONLY where |Z| <= tie_tol * max|Z|; everywhere else the
+    oracle decides by itself.  cache["ties"] counts the adopted decisions that differ."""
     K = len(dims) - 1
     P = split_params(arch, dims, np.asarray(params, dtype=np.float64))
     H = np.asarray(X, dtype=np.float64)
-    cache = {"H": [H], "M": [], "Z": [], "graphs": _layer_graphs(g, K, blocks)}
+    cache = {"H": [H], "M": [], "Z": [], "active": [], "ties": 0, "graphs": _layer_graphs(g, K, blocks)}
     mode = "gcn" if arch == "gcn" else "mean"
     for k in range(K):
         rp, cc, w, act = cache["graphs"][k]
@@ -71,7 +78,16 @@ def forward(g, X: np.ndarray, params: np.ndarray, arch: str, dims: Sequence[int]
             Z = M @ P[k]["W"] + P[k]["b"]
         else:
             Z = H @ P[k]["W_self"] + M @ P[k]["W_neigh"] + P[k]["b"]
-        Hn = np.maximum(Z, 0.0) if k < K - 1 else Z
+        if k < K - 1:
+            active = Z > 0.0
+            if relu_ties is not None and relu_ties[k] is not None and tie_tol > 0.0:
+                near = np.abs(Z) <= tie_tol * np.abs(Z).max()
+                cache["ties"] += int((near & (active != relu_ties[k])).sum())
+                active = np.where(near, relu_ties[k], active)
+            cache["active"].append(active)
+            Hn = np.where(active, Z, 0.0)
+        else:
+            Hn = Z
         if act is not None:  # rows outside the frontier are not part of the computational graph
             keep = np.zeros(g.n, dtype=bool)
             keep[act] = True
@@ -92,13 +108,13 @@ def bce_with_logits(s: np.ndarray, y: np.ndarray):
     return ell, sig - y
 
 
-def train_step(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst, blocks=None):
+def train_step(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst, blocks=None, relu_ties=None, tie_tol=0.0):
     """One training step of Algorithm 1 for one worker: scores of Eq. 2 (dot product) for
     positives (label 1) and negatives (label 0), loss L = (1/N) sum ell with N = |P| + |N|,
     and the gradient with respect to every parameter in the flat layout."""
     K = len(dims) - 1
     P = split_params(arch, dims, np.asarray(params, dtype=np.float64))
-    cache = forward(g, X, params, arch, dims, blocks)
+    cache = forward(g, X, params, arch, dims, blocks, relu_ties, tie_tol)
     HK = cache["H"][K]
     src = np.concatenate([pos_src, neg_src]).astype(np.int32)
     dst = np.concatenate([pos_dst, neg_dst]).astype(np.int32)
@@ -116,7 +132,7 @@ def train_step(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst, blo
     mode = "gcn" if arch == "gcn" else "mean"
     for k in range(K - 1, -1, -1):
         rp, cc, w, act = cache["graphs"][k]
-        dZ = dH if k == K - 1 else dH * (cache["Z"][k] > 0.0)
+        dZ = dH if k == K - 1 else dH * cache["active"][k]
         if act is not None:
             keep = np.zeros(g.n, dtype=bool)
             keep[act] = True

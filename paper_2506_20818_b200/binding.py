@@ -184,8 +184,8 @@ class Context:
 
     def adam_step(self, params, m, v, grads, t: int, grad_scale: float = 1.0, lr: float = 1e-3, beta1: float = 0.9, beta2: float = 0.999,
                   eps: float = 1e-8):
-        self._ck(self.lib.lp_adam_step(self.h, _ptr(params), _ptr(m), _ptr(v), _ptr(grads), C.c_float(grad_scale), C.c_float(lr),
-                                       C.c_float(beta1), C.c_float(beta2), C.c_float(eps), C.c_int64(t)))
+        self._ck(self.lib.lp_adam_step(self.h, _ptr(params), _ptr(m), _ptr(v), _ptr(grads), C.c_double(grad_scale), C.c_double(lr),
+                                       C.c_double(beta1), C.c_double(beta2), C.c_double(eps), C.c_int64(t)))
 
     def score(self, params, src, dst, seed: int = 0, step: int = 0):
         t = self._torch

@@ -128,17 +128,17 @@ edge_score_bce_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const 
 // loss = inv_N * sum of partials, added in index order by one block
 __global__ void loss_reduce_kernel(const float *__restrict__ partials, int64_t m, float inv_N, float *__restrict__ loss)
 {
-    __shared__ float sh[256];
-    float s = 0.f;
+    __shared__ double sh[256];  // the block partials are added in double: tens of thousands of nearly equal terms
+    double s = 0.0;
     const int64_t per = (m + 255) / 256;
     const int64_t b = per * threadIdx.x, e = min(m, b + per);
-    for (int64_t i = b; i < e; ++i) s += partials[i];
+    for (int64_t i = b; i < e; ++i) s += (double)partials[i];
     sh[threadIdx.x] = s;
     __syncthreads();
     if (threadIdx.x == 0) {
-        float t = 0.f;
+        double t = 0.0;
         for (int i = 0; i < 256; ++i) t += sh[i];
-        *loss = t * inv_N;
+        *loss = (float)(t * (double)inv_N);
     }
 }
 

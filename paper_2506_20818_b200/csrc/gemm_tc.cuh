@@ -1,18 +1,507 @@
-// Tensor-core (tcgen05) dense transforms of the BF16 path -- placeholder interface: until the
-// tcgen05 kernels land every shape reports "not supported" and the callers use the SIMT kernels.
+// Dense transforms of the BF16 path on the 5th-generation tensor cores (tcgen05, sm_100a).
+//
+//   tc_gemm_kmajor_kernel : C[M, N] = act(A[M, K] * Bt[N, K]^T + bias)       (forward, input gradient)
+//   tc_gemm_mnmajor_kernel: P[z][Kin, N] = A[rows_z, Kin]^T * dZ[rows_z, N]   (weight gradient, split over rows)
+//
+// Both kernels: one CTA owns a 128-row accumulator tile in tensor memory (128 lanes x BN FP32
+// columns); operand tiles are brought in by TMA (cp.async.bulk.tensor, 128-byte swizzle, no
+// multicast) into a ring of shared-memory stages guarded by full/empty mbarriers; one elected
+// thread issues tcgen05.mma (kind::f16, BF16 x BF16 -> FP32) and releases stages with
+// tcgen05.commit; all four warps drain the accumulator with tcgen05.ld and apply the epilogue.
+// Every mbarrier wait is bounded: on expiry the kernel records an error word, frees its tensor
+// memory and returns, and the host reports LP_ETIMEOUT.
 #pragma once
+#include <cuda.h>
+
 #include "common.cuh"
 #include "scan_sort.cuh"
+#include "gemm_simt.cuh"
+#include "optim.cuh"
+
+typedef CUresult (*lp_encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                       const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                       CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 struct TcState {
-    int *err_word = nullptr;
+    lp_encode_tiled_fn encode = nullptr;
+    int *err_word = nullptr;  // device: 0 = fine, else code of the wait that expired
+    bf16 *wbuf = nullptr;     // device scratch: BF16 copy of one layer's weights
+    int *host_err = nullptr;  // pinned
 };
-static bool tc_init(TcState &, std::string &) { return true; }
-static void tc_destroy(TcState &) {}
-static lp_status tc_check(TcState &, Exec &, bool, std::string &) { return LP_OK; }
-static bool tc_linear_supported(int, int) { return false; }
-static bool tc_weight_grad_supported(int, int) { return false; }
-static int64_t tc_weight_grad_partials(int64_t, int, int) { return 0; }
-static bool tc_linear(TcState &, Exec &, int64_t, int, int, const bf16 *, int, const float *, bool, const float *, bool, bf16 *, int, std::string &e) { e = "not built"; return false; }
-static bool tc_linear_bf16_b(TcState &, Exec &, int64_t, int, int, const bf16 *, int, const bf16 *, bool, const float *, bool, bf16 *, int, std::string &e) { e = "not built"; return false; }
-static bool tc_weight_grad(TcState &, Exec &, int64_t, int, int, const bf16 *, int, const bf16 *, int, float *, int, float *, std::string &e) { e = "not built"; return false; }
+
+constexpr int TC_BM = 128;          // accumulator rows (UMMA M)
+constexpr int TC_BK = 64;           // K elements per stage: 64 bf16 = one 128-byte swizzle row
+constexpr int TC_UMMA_K = 16;       // K per tcgen05.mma for 16-bit operands
+constexpr int TC_THREADS = 128;
+constexpr int TC_WBUF_ELEMS = 512 * 512;
+constexpr unsigned long long TC_WAIT_LIMIT_NS = 2000000000ull;  // every mbarrier wait gives up after two seconds
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+LP_DEVINL uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+LP_DEVINL void mbar_init(uint32_t bar, uint32_t count) { asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory"); }
+LP_DEVINL void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+LP_DEVINL bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+LP_DEVINL unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// bounded wait: false when the time limit was reached
+LP_DEVINL bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (global_timer_ns() - t0 > TC_WAIT_LIMIT_NS) return false;
+    }
+}
+LP_DEVINL void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+LP_DEVINL void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+LP_DEVINL void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst), "l"(map),
+                 "r"(bar), "r"(x), "r"(y)
+                 : "memory");
+}
+LP_DEVINL void tma_prefetch_desc(const CUtensorMap *map) { asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory"); }
+
+LP_DEVINL void tmem_alloc(uint32_t smem_dst, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+LP_DEVINL void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+LP_DEVINL void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+LP_DEVINL void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+LP_DEVINL void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+LP_DEVINL void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 lanes x 32 consecutive FP32 columns: thread t of the warp receives lane (32 * (warp % 4) + t)
+LP_DEVINL void tmem_ld_32x32(uint32_t taddr, float *v)
+{
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]),
+          "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
+          "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]),
+          "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor (tcgen05): start address, leading / stride byte offsets in
+// 16-byte units, descriptor version 1, 128-byte swizzle.
+LP_DEVINL uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;  // descriptor version
+    d |= (uint64_t)2 << 61;  // SWIZZLE_128B
+    return d;
+}
+
+// Instruction descriptor, kind::f16: D = FP32, A = B = BF16, M = 128, N = n; *_mn = operand stored MN-major
+static __host__ __device__ inline uint32_t make_idesc_bf16(int n, bool a_mn, bool b_mn)
+{
+    uint32_t d = 0;
+    d |= 1u << 4;                      // accumulator format F32
+    d |= 1u << 7;                      // A format BF16
+    d |= 1u << 10;                     // B format BF16
+    d |= (a_mn ? 1u : 0u) << 15;
+    d |= (b_mn ? 1u : 0u) << 16;
+    d |= (uint32_t)(n >> 3) << 17;
+    d |= (uint32_t)(TC_BM >> 4) << 24;
+    return d;
+}
+
+// ---------------------------------------------------------------------------------------------
+// kernel 1: K-major operands.  A tile = 128 rows x 64 K (16 KiB), B tile = BN rows x 64 K.
+// ---------------------------------------------------------------------------------------------
+struct TcGemmParams {
+    int64_t M;
+    int N, K;
+    int BN;             // accumulator columns of this launch (N tile), multiple of 16, <= 256
+    int stages;
+    const float *bias;  // [N] or null
+    int relu;
+    bf16 *C;            // output (BF16) when out_f32 == null
+    int64_t ldc;
+    float *out_f32;     // FP32 partial output [gridDim.z][M_tiles * 128, N] (weight gradient)
+    int64_t rows;       // weight gradient: reduction length; rows_per_split rows per blockIdx.z
+    int64_t rows_per_split;
+    int *err;
+};
+
+template <bool MN_MAJOR>
+__global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                                                             const TcGemmParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[8], bar_empty[8], bar_acc;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);  // swizzle atoms need 1024-byte alignment
+    const int BN = p.BN;
+    const uint32_t a_bytes = TC_BM * TC_BK * 2;  // 16384
+    const uint32_t b_bytes = (uint32_t)BN * TC_BK * 2;
+    const uint32_t stage_bytes = a_bytes + b_bytes;
+    const int S = p.stages;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < BN) tmem_cols <<= 1;
+
+    // reduction range of this CTA
+    int64_t k_begin = 0, k_end = p.K;
+    if (MN_MAJOR) {
+        k_begin = (int64_t)blockIdx.z * p.rows_per_split;
+        k_end = min(p.rows, k_begin + p.rows_per_split);
+    }
+    const int num_kb = (int)((k_end - k_begin + TC_BK - 1) / TC_BK);
+    const int m0 = blockIdx.x * TC_BM;
+    const int n0 = blockIdx.y * BN;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_empty[s]), 1);
+        }
+        mbar_init(smem_u32(&bar_acc), 1);
+        abort_s = 0;
+        fence_barrier_init();
+        fence_async_proxy();
+        tma_prefetch_desc(&mapA);
+        tma_prefetch_desc(&mapB);
+    }
+    if (warp == 0) {
+        __syncwarp();
+        tmem_alloc(smem_u32(&tmem_base_s), tmem_cols);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_d = tmem_base_s;
+
+    if (num_kb > 0) {
+        if (warp == 0 && lane == 0) {
+            // ---- producer: TMA loads into the stage ring
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % S;
+                if (kb >= S && !mbar_wait(smem_u32(&bar_empty[s]), ((kb / S) & 1) ^ 1)) {
+                    atomicExch(p.err, 1);
+                    abort_s = 1;
+                    break;
+                }
+                const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes), sb = sa + a_bytes;
+                const uint32_t bar = smem_u32(&bar_full[s]);
+                mbar_expect_tx(bar, stage_bytes);
+                const int kk = (int)(k_begin + (int64_t)kb * TC_BK);
+                if (!MN_MAJOR) {
+                    tma_load_2d(sa, &mapA, bar, kk, m0);  // box {64 K, 128 rows}
+                    tma_load_2d(sb, &mapB, bar, kk, n0);  // box {64 K, BN rows}
+                } else {
+                    // boxes {64 columns, 64 reduction rows}: 2 for A (128 features), BN / 64 for B
+                    for (int c = 0; c < TC_BM / 64; ++c) tma_load_2d(sa + c * 8192, &mapA, bar, m0 + c * 64, kk);
+                    for (int c = 0; c < BN / 64; ++c) tma_load_2d(sb + c * 8192, &mapB, bar, n0 + c * 64, kk);
+                }
+            }
+        } else if (warp == 1 && lane == 0) {
+            // ---- MMA issuer
+            const uint32_t idesc = make_idesc_bf16(BN, MN_MAJOR, MN_MAJOR);
+            bool ok = true;
+            for (int kb = 0; kb < num_kb && ok; ++kb) {
+                const int s = kb % S;
+                if (!mbar_wait(smem_u32(&bar_full[s]), (kb / S) & 1)) {
+                    atomicExch(p.err, 2);
+                    abort_s = 1;
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes), sb = sa + a_bytes;
+#pragma unroll
+                for (int k = 0; k < TC_BK / TC_UMMA_K; ++k) {
+                    uint64_t da, db;
+                    if (!MN_MAJOR) {
+                        // K-major, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart;
+                        // a K step of 16 elements moves the start by 32 bytes inside the swizzle row
+                        da = make_smem_desc(sa + k * 32, 16, 1024);
+                        db = make_smem_desc(sb + k * 32, 16, 1024);
+                    } else {
+                        // MN-major, 128-byte swizzle: 64 MN elements per 128-byte row, 8 K rows per 1024-byte
+                        // atom (stride), next 64 MN elements 8192 bytes further (leading); 16 K = 2 atoms
+                        da = make_smem_desc(sa + k * 2048, 8192, 1024);
+                        db = make_smem_desc(sb + k * 2048, 8192, 1024);
+                    }
+                    umma_bf16(tmem_d, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+                }
+                umma_commit(smem_u32(&bar_empty[s]));  // frees the stage when these MMAs have read it
+            }
+            if (ok) umma_commit(smem_u32(&bar_acc));   // accumulator complete
+        }
+        __syncwarp();
+
+        // ---- epilogue: all four warps
+        bool ready = mbar_wait(smem_u32(&bar_acc), 0);
+        if (!ready && lane == 0) atomicExch(p.err, 3);
+        ready = ready && (*(volatile int *)&abort_s == 0);
+        ready = __all_sync(0xffffffffu, ready);
+        tc_fence_after();
+        if (ready) {
+            const int row_in_tile = warp * 32 + lane;
+            const int64_t row = (int64_t)m0 + row_in_tile;
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                float v[32];
+                tmem_ld_32x32(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+                if (p.out_f32) {
+                    // FP32 partial tile of the weight gradient: [split][row][N]
+                    float *dst = p.out_f32 + ((int64_t)blockIdx.z * p.M + row) * p.N + n0 + c0;
+                    if (row < p.M) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4 *>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                    }
+                } else if (row < p.M) {
+                    if (p.bias) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] += __ldg(p.bias + n0 + c0 + i);
+                    }
+                    if (p.relu) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = fmaxf(v[i], 0.f);
+                    }
+                    bf16 *dst = p.C + row * p.ldc + n0 + c0;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        Vec16<bf16> o;
+                        o.from_float(v + i);
+                        o.store(dst + i);
+                    }
+                }
+            }
+        }
+    } else if (p.out_f32) {
+        // empty reduction range: the partial tile is zero
+        const int64_t row = (int64_t)m0 + threadIdx.x;
+        if (row < p.M)
+            for (int c = 0; c < BN; ++c) p.out_f32[((int64_t)blockIdx.z * p.M + row) * p.N + n0 + c] = 0.f;
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        tmem_dealloc(tmem_d, tmem_cols);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+static bool tc_init(TcState &tc, std::string &err)
+{
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+        err = "cuTensorMapEncodeTiled is not available from the driver";
+        return false;
+    }
+    tc.encode = (lp_encode_tiled_fn)fn;
+    if (cudaMalloc((void **)&tc.err_word, 256) != cudaSuccess || cudaMalloc((void **)&tc.wbuf, sizeof(bf16) * TC_WBUF_ELEMS) != cudaSuccess ||
+        cudaMallocHost((void **)&tc.host_err, sizeof(int)) != cudaSuccess) {
+        err = "allocation of the tensor-core GEMM state failed";
+        return false;
+    }
+    cudaMemset(tc.err_word, 0, 256);
+    if (cudaFuncSetAttribute(tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) {
+        err = "cannot raise the dynamic shared memory limit of the tensor-core GEMM";
+        return false;
+    }
+    return true;
+}
+
+static void tc_destroy(TcState &tc)
+{
+    cudaFree(tc.err_word);
+    cudaFree(tc.wbuf);
+    cudaFreeHost(tc.host_err);
+    tc = TcState();
+}
+
+// Reads the device error word.  `synced` = the stream has already been synchronised by the caller;
+// otherwise the word is only inspected when the caller asks for a synchronising check.
+static lp_status tc_check(TcState &tc, Exec &ex, bool synced, std::string &err)
+{
+    if (!synced) return LP_OK;
+    if (cudaMemcpyAsync(tc.host_err, tc.err_word, sizeof(int), cudaMemcpyDeviceToHost, ex.st) != cudaSuccess) return LP_OK;
+    cudaStreamSynchronize(ex.st);
+    if (*tc.host_err != 0) {
+        char buf[128];
+        snprintf(buf, sizeof buf, "tensor-core GEMM: bounded wait %d expired (1 = stage free, 2 = operands, 3 = accumulator)", *tc.host_err);
+        err = buf;
+        cudaMemsetAsync(tc.err_word, 0, sizeof(int), ex.st);
+        return LP_ETIMEOUT;
+    }
+    return LP_OK;
+}
+
+// 2-D BF16 tensor map over a row-major matrix [rows, cols] with leading dimension ld (elements);
+// box = {box_cols (inner, 128 bytes), box_rows}, 128-byte swizzle, zero fill outside.
+static bool tc_make_map(const TcState &tc, CUtensorMap *map, const bf16 *base, int64_t rows, int64_t cols, int64_t ld, int box_cols, int box_rows,
+                        std::string &err)
+{
+    if (((uintptr_t)base & 15) != 0 || (ld * 2) % 16 != 0) { err = "operand is not 16-byte aligned"; return false; }
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = tc.encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void *)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled failed"; return false; }
+    return true;
+}
+
+static int tc_pick_bn(int N) { return N <= 256 ? N : 256; }
+static bool tc_linear_supported(int K, int N) { return K >= 64 && K % 64 == 0 && N >= 64 && N % 64 == 0 && N <= 512 && (N <= 256 || N % 256 == 0) && (int64_t)K * N <= TC_WBUF_ELEMS; }
+static bool tc_weight_grad_supported(int Kin, int N) { return Kin >= 128 && Kin % 128 == 0 && N >= 64 && N % 64 == 0 && N <= 512 && (N <= 256 || N % 256 == 0); }
+
+static int tc_stages(int BN, int num_kb)
+{
+    // two CTAs per SM when the stage ring allows it (smem per CTA <= ~110 KiB)
+    const int stage = TC_BM * TC_BK * 2 + BN * TC_BK * 2;
+    int s = (108 * 1024) / stage;
+    s = std::max(2, std::min(s, 8));
+    return std::max(1, std::min(s, std::max(num_kb, 1)));
+}
+
+// C[M, N] (BF16, leading dimension ldc) = act(A[M, K] * Bt[N, K]^T + bias); Bt is BF16, K contiguous.
+static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const bf16 *A, int64_t lda, const bf16 *Bt, const float *bias, bool relu,
+                           bf16 *C, int64_t ldc, std::string &err)
+{
+    const int BN = tc_pick_bn(N);
+    CUtensorMap mapA, mapB;
+    if (!tc_make_map(tc, &mapA, A, M, K, lda, TC_BK, TC_BM, err)) return false;
+    if (!tc_make_map(tc, &mapB, Bt, N, K, K, TC_BK, BN, err)) return false;
+    TcGemmParams p{};
+    p.M = M; p.N = N; p.K = K; p.BN = BN;
+    p.stages = tc_stages(BN, K / TC_BK);
+    p.bias = bias; p.relu = relu ? 1 : 0; p.C = C; p.ldc = ldc; p.out_f32 = nullptr; p.rows = 0; p.rows_per_split = 0; p.err = tc.err_word;
+    const size_t smem = (size_t)p.stages * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024;
+    dim3 grid((unsigned)ceil_div64(M, TC_BM), (unsigned)(N / BN), 1);
+    tc_gemm_kernel<false><<<grid, TC_THREADS, smem, ex.st>>>(mapA, mapB, p);
+    ex.launches += 1;
+    return true;
+}
+
+// Layer transform with FP32 weights: converts the layer's weights to BF16 (transposing when they
+// are stored [K, N]) into the scratch buffer, then runs the K-major GEMM.
+//   w_is_kn = true : W is [K, N] row-major and the product is A * W        (forward)
+//   w_is_kn = false: W is [N, K] row-major and the product is A * W^T      (input gradient)
+static bool tc_linear(TcState &tc, Exec &ex, int64_t M, int N, int K, const bf16 *A, int lda, const float *W, bool w_is_kn, const float *bias,
+                      bool relu, bf16 *C, int ldc, std::string &err)
+{
+    const int total = K * N;
+    if (w_is_kn) weights_to_bf16_kernel<<<(total + 255) / 256, 256, 0, ex.st>>>(W, K, N, tc.wbuf, nullptr);
+    else convert_kernel<float, bf16><<<(total + 255) / 256, 256, 0, ex.st>>>(W, tc.wbuf, total);
+    ex.launches += 1;
+    return tc_gemm_kmajor(tc, ex, M, N, K, A, lda, tc.wbuf, bias, relu, C, ldc, err);
+}
+
+// the same with a BF16 B operand given as [K, N] (b_is_nk = false) or [N, K] (b_is_nk = true)
+__global__ void transpose_bf16_kernel(const bf16 *__restrict__ B, int K, int N, bf16 *__restrict__ Bt)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= K * N) return;
+    const int k = i / N, n = i - k * N;
+    Bt[(size_t)n * K + k] = B[i];
+}
+
+static bool tc_linear_bf16_b(TcState &tc, Exec &ex, int64_t M, int N, int K, const bf16 *A, int lda, const bf16 *B, bool b_is_nk, const float *bias,
+                             bool relu, bf16 *C, int ldc, std::string &err)
+{
+    const bf16 *Bt = B;
+    if (!b_is_nk) {
+        transpose_bf16_kernel<<<(K * N + 255) / 256, 256, 0, ex.st>>>(B, K, N, tc.wbuf);
+        ex.launches += 1;
+        Bt = tc.wbuf;
+    }
+    return tc_gemm_kmajor(tc, ex, M, N, K, A, lda, Bt, bias, relu, C, ldc, err);
+}
+
+// weight gradient: dW[Kin, N] (+)= A[rows, Kin]^T dZ[rows, N]; partial tiles per row split, then a
+// fixed-order reduction
+static int tc_weight_grad_splits(int64_t rows, int Kin, int N)
+{
+    const int tiles = (Kin / TC_BM) * (N / tc_pick_bn(N));
+    int splits = std::max(1, (2 * 148) / std::max(tiles, 1));
+    const int64_t max_by_rows = std::max<int64_t>(1, ceil_div64(rows, 4 * TC_BK));
+    return (int)std::min<int64_t>(splits, max_by_rows);
+}
+static int64_t tc_weight_grad_partials(int64_t rows, int Kin, int N)
+{
+    if (!tc_weight_grad_supported(Kin, N)) return 0;
+    return (int64_t)tc_weight_grad_splits(rows, Kin, N) * Kin * N;
+}
+
+static bool tc_weight_grad(TcState &tc, Exec &ex, int64_t rows, int Kin, int N, const bf16 *A, int lda, const bf16 *dZ, int ldz, float *dW, int accumulate,
+                           float *partials, std::string &err)
+{
+    const int BN = tc_pick_bn(N);
+    const int splits = tc_weight_grad_splits(rows, Kin, N);
+    CUtensorMap mapA, mapB;
+    if (!tc_make_map(tc, &mapA, A, rows, Kin, lda, 64, TC_BK, err)) return false;
+    if (!tc_make_map(tc, &mapB, dZ, rows, N, ldz, 64, TC_BK, err)) return false;
+    TcGemmParams p{};
+    p.M = Kin; p.N = N; p.K = 0; p.BN = BN;
+    p.rows = rows;
+    p.rows_per_split = ceil_div64(ceil_div64(rows, splits), TC_BK) * TC_BK;
+    p.stages = tc_stages(BN, (int)(p.rows_per_split / TC_BK));
+    p.bias = nullptr; p.relu = 0; p.C = nullptr; p.ldc = 0; p.out_f32 = partials; p.err = tc.err_word;
+    const size_t smem = (size_t)p.stages * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024;
+    dim3 grid((unsigned)(Kin / TC_BM), (unsigned)(N / BN), (unsigned)splits);
+    tc_gemm_kernel<true><<<grid, TC_THREADS, smem, ex.st>>>(mapA, mapB, p);
+    const int64_t count = (int64_t)Kin * N;
+    reduce_partials_kernel<<<(unsigned)ceil_div64(count, 256), 256, 0, ex.st>>>(partials, count, splits, dW, accumulate);
+    ex.launches += 2;
+    return true;
+}

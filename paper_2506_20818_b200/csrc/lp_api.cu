@@ -953,8 +953,8 @@ extern "C" lp_status lp_train_step(lp_ctx *ctx, const float *params, const int32
     return tc_check(ctx->tc, ctx->ex, false, ctx->err);
 }
 
-extern "C" lp_status lp_adam_step(lp_ctx *ctx, float *params, float *adam_m, float *adam_v, const float *grads, float grad_scale, float lr,
-                                  float beta1, float beta2, float eps, int64_t t)
+extern "C" lp_status lp_adam_step(lp_ctx *ctx, float *params, float *adam_m, float *adam_v, const float *grads, double grad_scale, double lr,
+                                  double beta1, double beta2, double eps, int64_t t)
 {
     if (!ctx) return LP_EINVAL;
     if (!ctx->model_set) return fail(ctx, LP_ESTATE, "lp_adam_step: set a model first");
@@ -964,10 +964,11 @@ extern "C" lp_status lp_adam_step(lp_ctx *ctx, float *params, float *adam_m, flo
     CK(cudaSetDevice(ctx->device));
     const int64_t np = ctx->n_params;
     if (adam_m) {
-        const double c1 = 1.0 - std::pow((double)beta1, (double)t), c2 = 1.0 - std::pow((double)beta2, (double)t);
-        adam_kernel<<<nblk(np), 256, 0, ctx->ex.st>>>(params, adam_m, adam_v, grads, np, grad_scale, lr, beta1, beta2, eps, (float)(1.0 / c1), (float)(1.0 / c2));
+        const double c1 = 1.0 - std::pow(beta1, (double)t), c2 = 1.0 - std::pow(beta2, (double)t);
+        adam_kernel<<<nblk(np), 256, 0, ctx->ex.st>>>(params, adam_m, adam_v, grads, np, (float)grad_scale, (float)lr, (float)beta1, (float)(1.0 - beta1),
+                                                      (float)beta2, (float)(1.0 - beta2), (float)eps, (float)(1.0 / c1), (float)(1.0 / c2));
     } else {
-        sgd_kernel<<<nblk(np), 256, 0, ctx->ex.st>>>(params, grads, np, grad_scale, lr);
+        sgd_kernel<<<nblk(np), 256, 0, ctx->ex.st>>>(params, grads, np, (float)grad_scale, (float)lr);
     }
     ctx->ex.launches += 1;
     CK_LAUNCH();
@@ -994,7 +995,7 @@ extern "C" lp_status lp_train_step_host(lp_ctx *ctx, float *params, const int32_
     s = lp_train_step(ctx, params, ps, pd, B, nullptr, ctx->d_neg_tmp, k, seed, step, ctx->d_loss_tmp, ctx->d_grads_tmp, 0);
     if (s != LP_OK) return s;
     if (adam_m || adam_v) {
-        s = lp_adam_step(ctx, params, adam_m, adam_v, ctx->d_grads_tmp, 1.f, 1e-3f, 0.9f, 0.999f, 1e-8f, adam_t);
+        s = lp_adam_step(ctx, params, adam_m, adam_v, ctx->d_grads_tmp, 1.0, 1e-3, 0.9, 0.999, 1e-8, adam_t);
         if (s != LP_OK) return s;
     }
     CK(cudaMemcpyAsync(loss_host, ctx->d_loss_tmp, sizeof(float), cudaMemcpyDeviceToHost, st));
@@ -1129,7 +1130,7 @@ extern "C" lp_status lp_get_stats(lp_ctx *ctx, lp_stats *out)
     }
     out->workspace_bytes = ctx->graph_bytes + ctx->model_bytes;
     out->kernel_launches = ctx->ex.launches;
-    return LP_OK;
+    return tc_check(ctx->tc, ctx->ex, true, ctx->err);
 }
 
 // ----------------------------------------------------------------------------------------------
@@ -1195,7 +1196,12 @@ extern "C" lp_status lp_op_linear(lp_ctx *ctx, int32_t prec, int64_t M, int32_t 
         return fail(ctx, LP_EINVAL, "lp_op_linear: unknown precision");
     }
     CK_LAUNCH();
-    return tc_check(ctx->tc, ctx->ex, false, ctx->err);
+    {
+        lp_status ts = tc_check(ctx->tc, ctx->ex, true, ctx->err);
+        if (ts != LP_OK) return ts;
+    }
+    CK(cudaStreamSynchronize(ctx->ex.st));
+    return LP_OK;
 }
 
 extern "C" lp_status lp_op_weight_grad(lp_ctx *ctx, int32_t prec, int64_t M, int32_t N, int32_t K, const void *A, const void *dZ, float *dW)
@@ -1223,5 +1229,5 @@ extern "C" lp_status lp_op_weight_grad(lp_ctx *ctx, int32_t prec, int64_t M, int
     cudaFree(partials);
     if (rc != LP_OK) return rc;
     CK_LAUNCH();
-    return tc_check(ctx->tc, ctx->ex, false, ctx->err);
+    return tc_check(ctx->tc, ctx->ex, true, ctx->err);
 }
