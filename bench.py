@@ -1,0 +1,362 @@
+#!/usr/bin/env python
+"""Benchmark of the link-prediction training step.
+
+One "step" = everything a worker does for one batch in Algorithm 1: draw the negatives, run the
+encoder forward, score positives and negatives, take the loss, back-propagate, update the weights
+with Adam.  The metric is training edges per second (positives + negatives) over the whole job.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line (see the design doc for the meaning of every key).
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+WORKLOAD = "c2_chunglu_sage2"
+METRIC = "training edges/sec (pos+neg) per step"
+UNIT = "edges/s"
+K_NEG = 1
+SEED = 1234
+
+# DRAM traffic of the dominant kernel (aggregation, F = 256 BF16 on the benchmark graph) from one ncu
+# capture, bytes per launch, valid only for the kernel source it was taken with.
+NCU_TRAFFIC = {"spmm_sha1": None, "bytes_per_launch": None}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), float(d.get("bf16_tflops_sustained", d.get("bf16_tflops", 0))), "measured"
+    return 6650.0, 1400.0, "fallback"
+
+
+def spmm_source_hash():
+    h = hashlib.sha1()
+    with open(os.path.join(ROOT, "paper_2506_20818_b200", "csrc", "spmm.cuh"), "rb") as f:
+        h.update(f.read())
+    return h.hexdigest()
+
+
+class ClockSampler:
+    """nvidia-smi sampling of SM clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.device_index = device_index
+        self.proc = None
+        self.path = f"/tmp/lp_bench_clocks_{os.getpid()}.csv"
+
+    def start(self):
+        try:
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                                          "-i", str(self.device_index)], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, smax, reasons, power = [], [], set(), []
+        for line in open(self.path):
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                smax.append(float(parts[2]))
+                power.append(float(parts[3]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.remove(self.path)
+        except OSError:
+            pass
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = [c for c, p in zip(sm, power) if p >= 0.5 * max(power)] or sm
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(smax), "reasons": sorted(reasons), "samples": len(sm),
+                "power_w_max": max(power)}
+
+
+def cpu_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def run_oracle_steps(g, X, params, dims, pos, B, steps, warmup):
+    """Times the CPU oracle, as it stands, on full steps of the benchmark workload."""
+    import oracle
+    times = []
+    p = params.astype(np.float64)
+    m = np.zeros_like(p)
+    v = np.zeros_like(p)
+    nb = max(1, len(pos[0]) // B)
+    for i in range(warmup + steps):
+        lo = (i % nb) * B
+        u, w = pos[0][lo:lo + B], pos[1][lo:lo + B]
+        t0 = time.perf_counter()
+        ns, nd, _ = oracle.sample_negatives(g.n, g.rowptr, g.col, u, SEED, i, K_NEG, edge_index_base=lo)
+        out = oracle.train_step(g, X, p, "sage", dims, u, w, ns, nd)
+        p, m, v = oracle.adam_step(p, m, v, out["grads"], i + 1)
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            times.append(dt)
+    return times
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--scale", type=float, default=1.0, help="shrink the workload (for quick checks and ncu captures)")
+    ap.add_argument("--batch", type=int, default=65536)
+    ap.add_argument("--cpu-baseline-steps", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--breakdown", action="store_true", help="print a per-category time breakdown to stderr")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    import workloads as wl
+
+    if args.impl == "reference":
+        # the CPU oracle, as it stands, on the host cores: rank 0 alone
+        if rank != 0:
+            return 0
+        g, X, params, pos, cfg = wl.make_config(WORKLOAD, scale=args.scale)
+        B = min(args.batch, len(pos[0]))
+        steps = max(1, min(args.steps, 4))
+        warm = min(args.warmup, 1)
+        times = run_oracle_steps(g, X, params, cfg["dims"], pos, B, steps, warm)
+        t = sum(times)
+        val = steps * B * (1 + K_NEG) / t
+        line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps, "warmup": warm,
+                "ms_per_step": 1e3 * t / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                "data": "synthetic", "config": {"workload": WORKLOAD, "nodes": g.n, "entries": g.nnz, "batch_pos": B, "neg_per_pos": K_NEG,
+                                                "scale": args.scale},
+                "cpu_baseline": {"value": val, "unit": UNIT, "cores": cpu_cores(), "kind": "oracle",
+                                 "sample": f"{steps} full steps of the workload (requested {args.steps}, bounded to keep the run to minutes)"},
+                "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(line))
+        return 0
+
+    import torch
+    import paper_2506_20818_b200 as pkg
+    from paper_2506_20818_b200 import build as lpbuild
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fall-back exists)")
+    if rank == 0:
+        lpbuild.build()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+        dist.barrier()
+    dev = f"cuda:{local_rank}"
+    torch.cuda.set_device(local_rank)
+
+    g, X, params, pos, cfg = wl.make_config(WORKLOAD, scale=args.scale)
+    dims = cfg["dims"]
+    B = min(args.batch, len(pos[0]))
+    nb = max(1, len(pos[0]) // B)
+
+    stream = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(stream):
+        ctx = pkg.Context(local_rank, stream=stream)
+        ctx.load_graph(g.n, g.rowptr, g.col, g.w, X)
+        ctx.set_model("sage", dims, prec="bf16", max_batch=B, max_k=K_NEG)
+        pu = torch.from_numpy(pos[0]).to(dev)
+        pv = torch.from_numpy(pos[1]).to(dev)
+        p = torch.from_numpy(params).to(dev)
+        m = torch.zeros_like(p)
+        v = torch.zeros_like(p)
+        grads = torch.zeros_like(p)
+        loss = torch.zeros(1, device=dev)
+        neg = torch.empty(B * K_NEG, dtype=torch.int32, device=dev)
+    lib = ctx.lib
+    import ctypes as C
+
+    def one_step(i, t_adam):
+        # data-parallel over batches: rank r takes batches r, r + world, ...
+        b = (i * world + rank) % nb
+        lo = b * B
+        su, sv = pu[lo:lo + B], pv[lo:lo + B]
+        ctx._ck(lib.lp_sample_negatives(ctx.h, C.c_uint64(SEED), C.c_uint64(i), C.c_int32(K_NEG), C.c_int32(0), C.c_void_p(su.data_ptr()),
+                                        C.c_int64(B), C.c_int64(lo), None, C.c_void_p(neg.data_ptr())))
+        ctx.train_step(p, su, sv, None, neg, K_NEG, loss, grads, seed=SEED, step=i)
+        if world > 1:
+            with torch.cuda.stream(stream):
+                dist.all_reduce(grads)  # gradient synchronisation of Algorithm 1 (sum; 1/p folded into the update)
+        ctx.adam_step(p, m, v, grads, t_adam, grad_scale=1.0 / world)
+
+    # ---- warm-up
+    with torch.cuda.stream(stream):
+        for i in range(args.warmup):
+            one_step(i, i + 1)
+    stream.synchronize()
+
+    # ---- timed region: K steps, events on the launching stream, aggregation launches timed inside
+    launches0 = ctx.stats().kernel_launches
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.2)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ctx.profile_begin(["agg_fwd", "agg_bwd"])
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for i in range(args.steps):
+            one_step(args.warmup + i, args.warmup + i + 1)
+        e1.record(stream)
+    stream.synchronize()
+    prof = ctx.profile_end()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    elapsed_ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    launches = ctx.stats().kernel_launches - launches0
+    loss_value = float(loss.item())
+    if world > 1:
+        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    edges_per_step = B * (1 + K_NEG) * world
+    value = args.steps * edges_per_step / (elapsed_ms * 1e-3)
+
+    # ---- roofline of the dominant kernel (aggregation launches timed inside the region above)
+    hbm_peak, bf16_peak, peak_kind = measured_peaks()
+    agg_ms = prof["agg_fwd"]["ms"] + prof["agg_bwd"]["ms"]
+    agg_bytes = prof["agg_fwd"]["bytes"] + prof["agg_bwd"]["bytes"]
+    agg_spans = prof["agg_fwd"]["spans"] + prof["agg_bwd"]["spans"]
+    achieved = agg_bytes / (agg_ms * 1e-3) / 1e9 if agg_ms > 0 else None
+    traffic = NCU_TRAFFIC["bytes_per_launch"] if NCU_TRAFFIC["spmm_sha1"] == spmm_source_hash() and args.scale == 1.0 else None
+    roofline = {"bound": "hbm", "kernel": "spmm_csr_kernel (aggregation forward + adjoint)", "achieved": achieved, "peak": hbm_peak,
+                "unit": "GB/s", "frac": (achieved / hbm_peak) if achieved else None, "peak_source": f"of {peak_kind}",
+                "frac_of_nominal_8000": (achieved / 8000.0) if achieved else None, "traffic": traffic,
+                "launches_timed": agg_spans, "avg_launch_us": 1e3 * agg_ms / max(agg_spans, 1),
+                "bytes_per_launch": agg_bytes / max(agg_spans, 1), "share_of_step": agg_ms / elapsed_ms,
+                "note": "algorithmic bytes, gather convention (each stored entry reads one source row); activations of this workload "
+                        "partly fit the 126 MB L2, so the figure can exceed DRAM bandwidth"}
+
+    # ---- optional breakdown of a few more steps, outside the timed region
+    breakdown = None
+    if args.breakdown or rank == 0:
+        ctx.profile_begin()
+        nbk = min(50, args.steps)
+        with torch.cuda.stream(stream):
+            for i in range(nbk):
+                one_step(args.warmup + args.steps + i, args.warmup + args.steps + i + 1)
+        bp = ctx.profile_end()
+        breakdown = {k: {"us_per_step": 1e3 * d["ms"] / nbk, "GBps": (d["bytes"] / (d["ms"] * 1e-3) / 1e9) if d["ms"] > 0 else None,
+                         "TFLOPs": (d["flops"] / (d["ms"] * 1e-3) / 1e12) if d["ms"] > 0 else None} for k, d in bp.items() if d["spans"]}
+        if args.breakdown and rank == 0:
+            print(json.dumps({"breakdown_per_step": breakdown}, indent=1), file=sys.stderr)
+
+    # ---- end to end through the host-buffer entry point: H2D of the batch, step, update, D2H of the loss
+    e2e = None
+    if not args.no_e2e:
+        hu = torch.from_numpy(pos[0]).pin_memory()
+        hv = torch.from_numpy(pos[1]).pin_memory()
+        loss_h = torch.zeros(1).pin_memory()
+        n_e2e = max(3, min(args.steps, 200))
+        t_base = args.warmup + args.steps + 100
+
+        def host_step(i):
+            b = (i * world + rank) % nb
+            lo = b * B
+            ctx.train_step_host(p, hu[lo:lo + B], hv[lo:lo + B], K_NEG, seed=SEED, step=i, edge_index_base=lo, adam_m=m, adam_v=v,
+                                adam_t=i + 1, loss_host=loss_h)
+
+        for i in range(3):
+            host_step(t_base + i)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        for i in range(n_e2e):
+            host_step(t_base + 3 + i)
+        f1.record(stream)
+        stream.synchronize()
+        e2e_ms = max(f0.elapsed_time(f1), 1e3 * (time.perf_counter() - t0))
+        if world > 1:
+            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        e2e = {"value": n_e2e * edges_per_step / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 2 * B * 4, "d2h_bytes_per_step": 4,
+               "steps": n_e2e, "note": "lp_train_step_host: pinned host batch -> device, negatives, step, Adam, loss -> host; "
+                                       "single-GPU update (no gradient all-reduce inside this entry point)"}
+
+    # ---- CPU baseline: the oracle on the host cores, rank 0 at N = 1 only
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        try:
+            times = run_oracle_steps(g, X, params, dims, pos, B, args.cpu_baseline_steps, 0)
+            cpu = {"value": len(times) * B * (1 + K_NEG) / sum(times), "unit": UNIT, "cores": cpu_cores(), "kind": "oracle",
+                   "sample": f"{len(times)} full steps of the same workload (full-graph encoder, {B} positives + {B * K_NEG} negatives each)",
+                   "s_per_step": sum(times) / len(times)}
+        except Exception as ex:  # the baseline must never take the GPU result down with it
+            cpu = {"value": None, "unit": UNIT, "cores": cpu_cores(), "kind": "oracle", "sample": f"failed: {ex}"}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+                "data": "synthetic",
+                "config": {"workload": WORKLOAD, "graph": "Chung-Lu power law, exponent 2.1, mean degree 20", "nodes": g.n, "entries": g.nnz,
+                           "model": "2-layer GraphSAGE-mean 128-256-256, dot-product predictor", "batch_pos": B, "neg_per_pos": K_NEG,
+                           "scale": args.scale, "parallelism": f"dp{world}" if world > 1 else "single GPU",
+                           "l2": "no flush: the step streams ~1 GB of activations per pass, several times the 126 MB L2"},
+                "clocks": clocks, "gpu_launches": int(launches), "loss_last": loss_value, "roofline": roofline, "cpu_baseline": cpu,
+                "e2e": e2e, "breakdown_us_per_step": breakdown}
+        print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -213,6 +213,40 @@ lp_status lp_get_block(lp_ctx *ctx, int32_t hop, int32_t *frontier, int64_t *blk
  * tensor-core kernel of an earlier call expired. */
 lp_status lp_get_stats(lp_ctx *ctx, lp_stats *out);
 
+/* ---- per-kernel timing (roofline measurement) ------------------------------------------------ */
+
+/* Kernel categories of the step. */
+enum {
+    LP_PROF_AGG_FWD = 0,   /* neighbour aggregation, forward (Eq. 1 AGG)                    */
+    LP_PROF_AGG_BWD = 1,   /* its adjoint over the transposed structure                     */
+    LP_PROF_GEMM_FWD = 2,  /* dense transform Z = A W + b (Eq. 1 UPDATE)                    */
+    LP_PROF_GEMM_DGRAD = 3,/* dA = dZ W^T                                                   */
+    LP_PROF_GEMM_WGRAD = 4,/* dW = A^T dZ and db                                            */
+    LP_PROF_SCORE = 5,     /* edge scores, loss, per-edge gradients (Eq. 2, Algorithm 1)    */
+    LP_PROF_INCIDENCE = 6, /* grouping the scored edges by node (integer sort)              */
+    LP_PROF_SCATTER = 7,   /* dL/dH^(K) gathered per node                                   */
+    LP_PROF_NEGATIVES = 8, /* negative sampling                                             */
+    LP_PROF_BLOCKS = 9,    /* neighbour sampling and block construction                     */
+    LP_PROF_ADAM = 10,     /* optimiser                                                     */
+    LP_PROF_CATEGORIES = 11
+};
+
+typedef struct {
+    double ms[LP_PROF_CATEGORIES];      /* device time between CUDA events on the context's stream      */
+    double bytes[LP_PROF_CATEGORIES];   /* algorithmic bytes of the timed launches (gather convention:  */
+                                        /* every stored entry reads its source row once, nothing cached) */
+    double flops[LP_PROF_CATEGORIES];   /* algorithmic floating-point operations                        */
+    int64_t spans[LP_PROF_CATEGORIES];  /* number of timed spans                                        */
+} lp_profile;
+
+/* Start timing the categories selected by `category_mask` (bit c = category c) with CUDA events
+ * recorded on the context's stream around the corresponding launches of every later call.
+ * A mask of 0 switches timing off.  Event records cost about a microsecond each. */
+lp_status lp_profile_begin(lp_ctx *ctx, uint32_t category_mask);
+
+/* Stop timing, synchronise the stream and return the sums per category since lp_profile_begin. */
+lp_status lp_profile_end(lp_ctx *ctx, lp_profile *out);
+
 /* ---- single operators (used by the parity tests and the roofline benchmark) -------------- */
 
 /* AGG of Eq. 1 on the loaded graph, float32 in / float32 out (bf16 = 0) or BF16 in / BF16 out

@@ -64,8 +64,9 @@ def forward(g, X: np.ndarray, params: np.ndarray, arch: str, dims: Sequence[int]
     ReLU turns a floating-point value into a yes/no decision (is the unit active?).  When a
     pre-activation is zero up to rounding, FP64 and the FP32 arithmetic under test may decide
     differently although both are right.  relu_ties[k] (bool [n, F_{k+1}], the decisions of the
-    implementation under test) is adopted ONLY where |Z| <= tie_tol * max|Z|; everywhere else the
-    oracle decides by itself.  cache["ties"] counts the adopted decisions that differ."""
+    implementation under test) is adopted ONLY where |Z| <= tie_tol * rms(Z), with tie_tol the
+    floating-point tolerance of the comparison; everywhere else the oracle decides by itself.
+    cache["ties"] counts the adopted decisions that differ from the oracle's own."""
     K = len(dims) - 1
     P = split_params(arch, dims, np.asarray(params, dtype=np.float64))
     H = np.asarray(X, dtype=np.float64)
@@ -81,7 +82,8 @@ def forward(g, X: np.ndarray, params: np.ndarray, arch: str, dims: Sequence[int]
         if k < K - 1:
             active = Z > 0.0
             if relu_ties is not None and relu_ties[k] is not None and tie_tol > 0.0:
-                near = np.abs(Z) <= tie_tol * np.abs(Z).max()
+                rows = Z if act is None else Z[act]
+                near = np.abs(Z) <= tie_tol * np.sqrt(np.mean(rows * rows))
                 cache["ties"] += int((near & (active != relu_ties[k])).sum())
                 active = np.where(near, relu_ties[k], active)
             cache["active"].append(active)

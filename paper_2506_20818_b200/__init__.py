@@ -6,6 +6,7 @@ from .binding import (  # noqa: F401
     Stats,
     load_library,
     EXPORTS,
+    PROF_CATEGORIES,
     LP_GCN,
     LP_SAGE_MEAN,
     LP_FP32,

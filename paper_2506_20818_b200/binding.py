@@ -26,8 +26,11 @@ EXPORTS = [
     "lp_create", "lp_destroy", "lp_last_error", "lp_load_graph", "lp_get_structure", "lp_set_model",
     "lp_param_count", "lp_set_candidates", "lp_sample_negatives", "lp_train_step", "lp_train_step_host",
     "lp_adam_step", "lp_score", "lp_get_embeddings", "lp_get_output_gradient", "lp_get_block",
-    "lp_get_stats", "lp_op_aggregate", "lp_op_linear", "lp_op_weight_grad",
+    "lp_get_stats", "lp_op_aggregate", "lp_op_linear", "lp_op_weight_grad", "lp_profile_begin", "lp_profile_end",
 ]
+
+PROF_CATEGORIES = ["agg_fwd", "agg_bwd", "gemm_fwd", "gemm_dgrad", "gemm_wgrad", "score", "incidence", "scatter",
+                   "negatives", "blocks", "adam"]
 
 
 class LpError(RuntimeError):
@@ -46,6 +49,10 @@ class Stats(C.Structure):
     _fields_ = [("negatives_exhausted", C.c_int64), ("block_nodes", C.c_int64 * (LP_MAX_LAYERS + 1)),
                 ("block_edges", C.c_int64 * LP_MAX_LAYERS), ("workspace_bytes", C.c_int64),
                 ("kernel_launches", C.c_int64)]
+
+
+class Profile(C.Structure):
+    _fields_ = [("ms", C.c_double * 11), ("bytes", C.c_double * 11), ("flops", C.c_double * 11), ("spans", C.c_int64 * 11)]
 
 
 _lib = None
@@ -230,6 +237,19 @@ class Context:
         if col is not None:
             col = col[: int(s.block_edges[hop - 1])]
         return frontier, ptr, col
+
+    # ---- per-kernel timing
+    def profile_begin(self, categories=None):
+        mask = 0
+        for c in (categories if categories is not None else PROF_CATEGORIES):
+            mask |= 1 << PROF_CATEGORIES.index(c)
+        self._ck(self.lib.lp_profile_begin(self.h, C.c_uint32(mask)))
+
+    def profile_end(self):
+        p = Profile()
+        self._ck(self.lib.lp_profile_end(self.h, C.byref(p)))
+        return {name: {"ms": p.ms[i], "bytes": p.bytes[i], "flops": p.flops[i], "spans": int(p.spans[i])}
+                for i, name in enumerate(PROF_CATEGORIES)}
 
     # ---- single operators
     def op_aggregate(self, arch: str, H, transpose: bool = False):

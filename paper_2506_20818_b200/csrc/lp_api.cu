@@ -141,6 +141,21 @@ static void free_list(std::vector<void *> &l)
 
 static inline unsigned nblk(int64_t n, int t = 256) { return (unsigned)std::max<int64_t>(1, ceil_div64(n, t)); }
 
+// Algorithmic bytes of one aggregation launch, gather convention: every stored entry reads one
+// source row of F elements plus its column index (and coefficient), nothing is assumed cached;
+// plus row offsets, the output rows and the optional per-row operands.
+template <typename T> static double spmm_bytes(const SpmmArgs<T> &a, int64_t nnz)
+{
+    const double s = sizeof(T), rows = a.n_rows, F = a.F;
+    double b = (double)nnz * (F * s + 4.0 + (a.val ? 4.0 : 0.0)) + (rows + 1.0) * 4.0 + rows * F * s;
+    if (a.init) b += rows * F * s;
+    if (a.relu_ref) b += rows * F * s;
+    if (a.self_out) b += 2.0 * rows * F * s;
+    if (a.row_scale) b += rows * 4.0;
+    return b;
+}
+static double gemm_bytes(double M, double N, double K, double s_in, double s_out) { return M * K * s_in + K * N * s_in + M * N * s_out; }
+
 // ----------------------------------------------------------------------------------------------
 // load-time kernels
 // ----------------------------------------------------------------------------------------------
@@ -244,6 +259,7 @@ extern "C" void lp_destroy(lp_ctx *ctx)
     free_list(ctx->model_allocs);
     free_list(ctx->graph_allocs);
     tc_destroy(ctx->tc);
+    for (cudaEvent_t e : ctx->ex.prof.pool) cudaEventDestroy(e);
     cudaFree(ctx->err_flag);
     cudaFree(ctx->exhausted_dev);
     cudaFreeHost(ctx->host_counts);
@@ -597,6 +613,7 @@ extern "C" lp_status lp_sample_negatives(lp_ctx *ctx, uint64_t seed, uint64_t st
     const int reject = ctx->model_set ? ctx->desc.reject_edges : 1;
     const int attempts = (ctx->model_set && ctx->desc.reject_edges) ? ctx->desc.max_attempts : (reject ? 8 : 1);
     const uint32_t space = (uint32_t)(ctx->cand ? ctx->n_cand : ctx->n);
+    ProfScope prof(ctx->ex, LP_PROF_NEGATIVES, (double)B * k * 8.0);
     cudaMemsetAsync(ctx->exhausted_dev, 0, sizeof(unsigned long long), ctx->ex.st);
     sample_negatives_kernel<<<nblk(B * k), 256, 0, ctx->ex.st>>>(ctx->n, ctx->rowptr, ctx->col, ctx->cand, space,
                                                                 make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)), (uint32_t)step, k, mode, reject,
@@ -616,6 +633,7 @@ template <typename T>
 static lp_status layer_linear(lp_ctx *ctx, int64_t rows, const LayerBuf &L, const float *params, T *out, int ldo, bool relu)
 {
     if (rows <= 0) return LP_OK;
+    ProfScope prof(ctx->ex, LP_PROF_GEMM_FWD, gemm_bytes((double)rows, L.Fo, L.Kin, sizeof(T), sizeof(T)), 2.0 * rows * L.Fo * L.Kin);
     if (sizeof(T) == 2 && tc_linear_supported(L.Kin, L.Fo)) {
         std::string err;
         if (!tc_linear(ctx->tc, ctx->ex, rows, L.Fo, L.Kin, (const bf16 *)L.A, L.Kin, params + L.off_w, /*w_is_kn=*/true, params + L.off_b, relu,
@@ -632,6 +650,7 @@ template <typename T>
 static lp_status layer_input_grad(lp_ctx *ctx, int64_t rows, const LayerBuf &L, const float *params, const T *dZ, T *dA)
 {
     if (rows <= 0) return LP_OK;
+    ProfScope prof(ctx->ex, LP_PROF_GEMM_DGRAD, gemm_bytes((double)rows, L.Kin, L.Fo, sizeof(T), sizeof(T)), 2.0 * rows * L.Fo * L.Kin);
     if (sizeof(T) == 2 && tc_linear_supported(L.Fo, L.Kin)) {
         std::string err;
         if (!tc_linear(ctx->tc, ctx->ex, rows, L.Kin, L.Fo, (const bf16 *)dZ, L.Fo, params + L.off_w, /*w_is_kn=*/false, nullptr, false, (bf16 *)dA, L.Kin,
@@ -650,6 +669,7 @@ static lp_status layer_weight_grad(lp_ctx *ctx, int64_t rows, const LayerBuf &L,
         if (!accumulate) cudaMemsetAsync(grads + L.off_w, 0, sizeof(float) * ((size_t)L.Kin * L.Fo + L.Fo), ctx->ex.st);
         return LP_OK;
     }
+    ProfScope prof(ctx->ex, LP_PROF_GEMM_WGRAD, (double)rows * (L.Kin + 2.0 * L.Fo) * sizeof(T) + 4.0 * (L.Kin + 1.0) * L.Fo, 2.0 * rows * L.Fo * (L.Kin + 1.0));
     if (sizeof(T) == 2 && tc_weight_grad_supported(L.Kin, L.Fo)) {
         std::string err;
         if (!tc_weight_grad(ctx->tc, ctx->ex, rows, L.Kin, L.Fo, (const bf16 *)L.A, L.Kin, (const bf16 *)dZ, L.Fo, grads + L.off_w, accumulate, ctx->partials, err))
@@ -679,6 +699,7 @@ static lp_status build_blocks(lp_ctx *ctx, const int *pos_src, const int *pos_ds
     cudaStream_t st = ctx->ex.st;
     const int n = ctx->n, K = ctx->K;
     const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
+    ProfScope prof(ctx->ex, LP_PROF_BLOCKS);
     CK(cudaMemsetAsync(ctx->mark, 0, (size_t)n, st));
     mark_ids_kernel<<<nblk(B), 256, 0, st>>>(pos_src, B, n, ctx->mark);
     mark_ids_kernel<<<nblk(B), 256, 0, st>>>(pos_dst, B, n, ctx->mark);
@@ -797,7 +818,10 @@ template <typename T> static lp_status forward_impl(lp_ctx *ctx, const float *pa
             }
             if (k == K - 1) { out = tptr<T>(ctx->HK); ldo = L.Fo; } else { out = tptr<T>(L.Hout); ldo = L.Fo; }
         }
-        if (rows > 0 && !spmm_launch<T>(ctx->ex, a)) return fail(ctx, LP_EUNSUPPORTED, "aggregation width not supported");
+        {
+            ProfScope prof(ctx->ex, LP_PROF_AGG_FWD, spmm_bytes(a, ctx->sampled ? ctx->hop[K - k].entries : ctx->nnz), 2.0 * (ctx->sampled ? ctx->hop[K - k].entries : ctx->nnz) * L.Fi);
+            if (rows > 0 && !spmm_launch<T>(ctx->ex, a)) return fail(ctx, LP_EUNSUPPORTED, "aggregation width not supported");
+        }
         lp_status s = layer_linear<T>(ctx, rows, L, params, out, ldo, k < K - 1);
         if (s != LP_OK) return s;
     }
@@ -834,6 +858,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     T *HK = tptr<T>(ctx->HK);
 
     // scores, loss, per-edge gradients
+    ProfScope *pscore = new ProfScope(ctx->ex, LP_PROF_SCORE, (double)B * (2.0 + k) * D * sizeof(T) + (double)E * 12.0, 2.0 * E * D);
     const unsigned eblocks = nblk(B, EDGE_THREADS / 32);
     constexpr int VN = Vec16<T>::N;
     const int chunks = D / VN;
@@ -841,14 +866,18 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     else if (chunks <= 64) edge_score_bce_kernel<T, 2><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials);
     else edge_score_bce_kernel<T, 4><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials);
     loss_reduce_kernel<<<1, 256, 0, st>>>(ctx->loss_partials, eblocks, inv_N, loss);
+    delete pscore;
+    ctx->ex.launches += 2;
 
     // incidence lists of the scored edges, grouped by node (stable sort => fixed summation order)
+    ProfScope *pinc = new ProfScope(ctx->ex, LP_PROF_INCIDENCE, (double)E * 2.0 * 40.0);
     CK(cudaMemsetAsync(ctx->inc_ptr, 0, sizeof(int) * ((size_t)rows_out + 1), st));
     incidence_keys_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->inc_keys, ctx->inc_slots, ctx->inc_other, ctx->inc_ptr);
     exclusive_scan_i32(ctx->ex, ctx->inc_ptr, rows_out, ctx->inc_ptr, ctx->inc_ptr + rows_out, ctx->scan_tmp);
     radix_sort_pairs(ctx->ex, ctx->inc_keys, ctx->inc_slots, 2 * E, bits_for(rows_out), ctx->sort);
     incidence_fill_kernel<<<nblk(2 * E), 256, 0, st>>>(ctx->inc_slots, 2 * E, ctx->inc_other, B, ctx->g_pos, ctx->g_neg, ctx->inc_col, ctx->inc_val);
-    ctx->ex.launches += 4;
+    ctx->ex.launches += 2;
+    delete pinc;
 
     // dL/dH^(K)[v] = sum over incident scored edges of g_e * h_other
     T *dZ = tptr<T>(ctx->dHK);
@@ -864,6 +893,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         a.F = D;
         a.Y = dZ;
         a.ldy = D;
+        ProfScope prof(ctx->ex, LP_PROF_SCATTER, spmm_bytes(a, 2 * E), 4.0 * E * D);
         if (rows_out > 0 && !spmm_launch<T>(ctx->ex, a)) return fail(ctx, LP_EUNSUPPORTED, "embedding width not supported");
     }
     ctx->have_grad = true;
@@ -919,7 +949,11 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
             a.relu_ref = tptr<T>(ctx->layer[l - 1].Hout);
             a.ldref = L.Fi;
         }
-        if (a.n_rows > 0 && !spmm_launch<T>(ctx->ex, a)) return fail(ctx, LP_EUNSUPPORTED, "aggregation width not supported");
+        {
+            const int64_t nnz_l = ctx->sampled ? ctx->hop[K - l].entries : ctx->nnz;
+            ProfScope prof(ctx->ex, LP_PROF_AGG_BWD, spmm_bytes(a, nnz_l), 2.0 * nnz_l * L.Fi);
+            if (a.n_rows > 0 && !spmm_launch<T>(ctx->ex, a)) return fail(ctx, LP_EUNSUPPORTED, "aggregation width not supported");
+        }
         dZ = dZn;
         cur ^= 1;
     }
@@ -963,6 +997,7 @@ extern "C" lp_status lp_adam_step(lp_ctx *ctx, float *params, float *adam_m, flo
     if (adam_m && t < 1) return fail(ctx, LP_EINVAL, "lp_adam_step: t counts from 1");
     CK(cudaSetDevice(ctx->device));
     const int64_t np = ctx->n_params;
+    ProfScope prof(ctx->ex, LP_PROF_ADAM, (double)np * (adam_m ? 28.0 : 12.0));
     if (adam_m) {
         const double c1 = 1.0 - std::pow(beta1, (double)t), c2 = 1.0 - std::pow(beta2, (double)t);
         adam_kernel<<<nblk(np), 256, 0, ctx->ex.st>>>(params, adam_m, adam_v, grads, np, (float)grad_scale, (float)lr, (float)beta1, (float)(1.0 - beta1),
@@ -1133,6 +1168,37 @@ extern "C" lp_status lp_get_stats(lp_ctx *ctx, lp_stats *out)
     return tc_check(ctx->tc, ctx->ex, true, ctx->err);
 }
 
+extern "C" lp_status lp_profile_begin(lp_ctx *ctx, uint32_t category_mask)
+{
+    if (!ctx) return LP_EINVAL;
+    CK(cudaSetDevice(ctx->device));
+    CK(cudaStreamSynchronize(ctx->ex.st));
+    ctx->ex.prof.spans.clear();
+    ctx->ex.prof.used = 0;
+    ctx->ex.prof.mask = category_mask & ((1u << LP_PROF_CATEGORIES) - 1u);
+    return LP_OK;
+}
+
+extern "C" lp_status lp_profile_end(lp_ctx *ctx, lp_profile *out)
+{
+    if (!ctx || !out) return LP_EINVAL;
+    CK(cudaSetDevice(ctx->device));
+    ctx->ex.prof.mask = 0;
+    CK(cudaStreamSynchronize(ctx->ex.st));
+    memset(out, 0, sizeof *out);
+    for (const Profiler::Span &s : ctx->ex.prof.spans) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, s.a, s.b) != cudaSuccess) continue;
+        out->ms[s.cat] += ms;
+        out->bytes[s.cat] += s.bytes;
+        out->flops[s.cat] += s.flops;
+        out->spans[s.cat] += 1;
+    }
+    ctx->ex.prof.spans.clear();
+    ctx->ex.prof.used = 0;
+    return LP_OK;
+}
+
 // ----------------------------------------------------------------------------------------------
 // single operators
 // ----------------------------------------------------------------------------------------------
@@ -1156,6 +1222,7 @@ template <typename T> static lp_status op_aggregate_impl(lp_ctx *ctx, int arch, 
         if (arch == LP_GCN) { a.val = ctx->gcn_valT; a.init = H; a.ldinit = F; a.init_coef = ctx->gcn_self; }
         else a.val = ctx->meanT_val;
     }
+    ProfScope prof(ctx->ex, transpose ? LP_PROF_AGG_BWD : LP_PROF_AGG_FWD, spmm_bytes(a, ctx->nnz), 2.0 * ctx->nnz * F);
     if (!spmm_launch<T>(ctx->ex, a)) return fail(ctx, LP_EINVAL, "lp_op_aggregate: F must be a multiple of 8, at most 512");
     CK_LAUNCH();
     return LP_OK;

@@ -4,9 +4,48 @@
 #pragma once
 #include "common.cuh"
 
+// Optional per-category timing with CUDA events on the launching stream (lp_profile_begin/_end).
+struct Profiler {
+    uint32_t mask = 0;  // categories being timed; 0 = off
+    struct Span { int cat; cudaEvent_t a, b; double bytes, flops; };
+    std::vector<Span> spans;
+    std::vector<cudaEvent_t> pool;
+    size_t used = 0;
+    cudaEvent_t get()
+    {
+        if (used == pool.size()) {
+            cudaEvent_t e = nullptr;
+            cudaEventCreate(&e);
+            pool.push_back(e);
+        }
+        return pool[used++];
+    }
+};
+
 struct Exec {
     cudaStream_t st = nullptr;
     int64_t launches = 0;
+    Profiler prof;
+};
+
+// Times everything enqueued on the stream between construction and destruction when the category
+// is selected; `bytes` / `flops` are the algorithmic figures of the enclosed launches.
+struct ProfScope {
+    Exec &ex;
+    int idx = -1;
+    ProfScope(Exec &e, int cat, double bytes = 0.0, double flops = 0.0) : ex(e)
+    {
+        if (ex.prof.mask & (1u << cat)) {
+            Profiler::Span s{cat, ex.prof.get(), ex.prof.get(), bytes, flops};
+            cudaEventRecord(s.a, ex.st);
+            idx = (int)ex.prof.spans.size();
+            ex.prof.spans.push_back(s);
+        }
+    }
+    ~ProfScope()
+    {
+        if (idx >= 0) cudaEventRecord(ex.prof.spans[idx].b, ex.st);
+    }
 };
 
 // ------------------------------------------------------------------------------------------

@@ -440,3 +440,21 @@ def test_sampled_step_backward_finite_differences():
         pm[i] -= 1e-6
         fd[i] = (bf_loss(pp) - bf_loss(pm)) / 2e-6
     assert rel_l2(out["grads"], fd) < 1e-7
+
+
+def test_relu_tie_window_only_touches_near_zero_units():
+    g = wl.erdos_renyi(60, 200, seed=3)
+    dims = [6, 8, 4]
+    X = wl.node_features(g.n, 6, 0)
+    p = wl.glorot_params("gcn", dims, 1, 0.2)
+    base = oracle.forward(g, X, p, "gcn", dims)
+    Z = base["Z"][0]
+    flipped = ~(Z > 0)  # decisions that are all wrong
+    out = oracle.forward(g, X, p, "gcn", dims, relu_ties=[flipped], tie_tol=1e-3)
+    rms = np.sqrt(np.mean(Z * Z))
+    near = np.abs(Z) <= 1e-3 * rms
+    assert out["ties"] == int(near.sum())
+    assert np.array_equal(out["active"][0][~near], (Z > 0)[~near])  # untouched outside the window
+    assert np.array_equal(out["active"][0][near], flipped[near])
+    # window of zero width: nothing adopted
+    assert oracle.forward(g, X, p, "gcn", dims, relu_ties=[flipped], tie_tol=0.0)["ties"] == 0
