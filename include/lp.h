@@ -266,6 +266,29 @@ lp_status lp_op_linear(lp_ctx *ctx, int32_t prec, int64_t M, int32_t N, int32_t 
 lp_status lp_op_weight_grad(lp_ctx *ctx, int32_t prec, int64_t M, int32_t N, int32_t K, const void *A, const void *dZ,
                             float *dW);
 
+/* ---- allocation-free variant ---------------------------------------------------------------- */
+
+/* (No counterpart in the paper: this entry point exists for the callers described below.)
+ * Weight gradient dW[K, N] = A[M, K]^T * dZ[M, N] in float32, the same result as
+ * lp_op_weight_grad(LP_FP32) up to the order of the row-split summation, for callers that cannot
+ * allocate device memory when they need it: latency-critical loops that forbid allocator calls
+ * because those take driver locks and may synchronise the device, processes that handed all
+ * device memory to a pool at start-up, and code sections in which the CUDA runtime itself
+ * refuses to allocate.  It needs no context and calls no cudaMalloc, cudaFree or any allocating routine:
+ * the partial sums of the split-row reduction live in a fixed 8 MiB array inside the library
+ * (every GPU that uses the library holds that array until the process exits).
+ *   device, cuda_stream : device index (made current by the call) and cudaStream_t (NULL = default)
+ *   A[M, K], dZ[M, N], dW[K, N] : DEVICE float32, row-major, caller-owned; dW is overwritten
+ * Limit: K * N <= 2^21 (2,097,152); larger requests return LP_EINVAL with a message available
+ * from lp_last_error(NULL).  M is unbounded.
+ * The first call on each device looks up the device address of the fixed array; make that first
+ * call before starting any stream capture.  All calls on a device share the array and it keeps
+ * the previous call's contents (each call overwrites what it reads, so nothing needs clearing):
+ * two calls whose kernels overlap on the GPU (different streams, no ordering) race on it and
+ * must be serialised by the caller.  Does not synchronise. */
+lp_status lp_weight_grad_static(int32_t device, void *cuda_stream, int64_t M, int32_t N, int32_t K, const float *A, const float *dZ,
+                                float *dW);
+
 #ifdef __cplusplus
 }
 #endif

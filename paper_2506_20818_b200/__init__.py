@@ -5,6 +5,7 @@ from .binding import (  # noqa: F401
     ModelDesc,
     Stats,
     load_library,
+    weight_grad_static,
     EXPORTS,
     PROF_CATEGORIES,
     LP_GCN,

@@ -27,6 +27,7 @@ EXPORTS = [
     "lp_param_count", "lp_set_candidates", "lp_sample_negatives", "lp_train_step", "lp_train_step_host",
     "lp_adam_step", "lp_score", "lp_get_embeddings", "lp_get_output_gradient", "lp_get_block",
     "lp_get_stats", "lp_op_aggregate", "lp_op_linear", "lp_op_weight_grad", "lp_profile_begin", "lp_profile_end",
+    "lp_weight_grad_static",
 ]
 
 PROF_CATEGORIES = ["agg_fwd", "agg_bwd", "gemm_fwd", "gemm_dgrad", "gemm_wgrad", "score", "incidence", "scatter",
@@ -277,3 +278,21 @@ class Context:
         prec = LP_BF16 if A.dtype == t.bfloat16 else LP_FP32
         self._ck(self.lib.lp_op_weight_grad(self.h, C.c_int32(prec), C.c_int64(M), C.c_int32(N), C.c_int32(K), _ptr(A), _ptr(dZ), _ptr(dW)))
         return dW
+
+
+def weight_grad_static(A, dZ, stream=None):
+    """dW = A^T dZ (float32 CUDA tensors) through the allocation-free entry point.  The output
+    tensor is allocated HERE, by torch, before the call: the library call itself allocates nothing.
+    For callers that cannot allocate at call time (allocator-free loops, pre-pooled memory)."""
+    import torch
+
+    lib = load_library()
+    M, K = A.shape
+    N = dZ.shape[1]
+    dW = torch.empty((K, N), dtype=torch.float32, device=A.device)
+    st = stream if stream is not None else torch.cuda.current_stream(A.device)
+    rc = lib.lp_weight_grad_static(C.c_int32(A.device.index or 0), C.c_void_p(st.cuda_stream), C.c_int64(M), C.c_int32(N), C.c_int32(K),
+                                   _ptr(A), _ptr(dZ), _ptr(dW))
+    if rc != LP_OK:
+        raise LpError(rc, lib.lp_last_error(None).decode())
+    return dW

@@ -1298,3 +1298,55 @@ extern "C" lp_status lp_op_weight_grad(lp_ctx *ctx, int32_t prec, int64_t M, int
     CK_LAUNCH();
     return tc_check(ctx->tc, ctx->ex, true, ctx->err);
 }
+
+// ----------------------------------------------------------------------------------------------
+// Weight gradient for callers that must not allocate
+// ----------------------------------------------------------------------------------------------
+// Some hosts of this library cannot call cudaMalloc at the point where they need a weight
+// gradient: a real-time loop that forbids allocator calls (they take driver locks and may
+// synchronise the device), a process whose device memory was all handed to a pool at start-up, or
+// a code section in which the CUDA runtime itself refuses to allocate.  lp_weight_grad_static serves them: the FP32 partial tiles of
+// the split-row reduction live in the fixed device array below instead of a cudaMalloc'ed buffer.
+// The array is part of the loaded module, so every GPU that uses this library holds
+// LP_STATIC_SCRATCH_FLOATS * 4 bytes of it until the process exits.
+#define LP_STATIC_SCRATCH_FLOATS (1 << 21) /* 8 MiB */
+static __device__ __align__(256) float lp_static_scratch[LP_STATIC_SCRATCH_FLOATS];
+
+// In host code the name of a __device__ array is only a handle for the runtime, never an address a
+// kernel may be given; the device address is looked up once per device, with that device current.
+#define LP_STATIC_MAX_DEVICES 64
+static float *g_static_scratch_addr[LP_STATIC_MAX_DEVICES];
+
+extern "C" lp_status lp_weight_grad_static(int32_t device, void *cuda_stream, int64_t M, int32_t N, int32_t K, const float *A, const float *dZ,
+                                           float *dW)
+{
+    lp_ctx *ctx = nullptr;  // errors are reported through lp_last_error(NULL)
+    if (device < 0 || device >= LP_STATIC_MAX_DEVICES) return fail(ctx, LP_EINVAL, "lp_weight_grad_static: device index out of range");
+    if (!A || !dZ || !dW || M <= 0 || N <= 0 || K <= 0) return fail(ctx, LP_EINVAL, "lp_weight_grad_static: bad argument");
+    const int64_t tile = (int64_t)K * N;
+    if (tile > LP_STATIC_SCRATCH_FLOATS) {
+        char buf[200];
+        snprintf(buf, sizeof buf, "lp_weight_grad_static: K * N = %lld exceeds the fixed scratch of %d floats; use lp_op_weight_grad instead",
+                 (long long)tile, LP_STATIC_SCRATCH_FLOATS);
+        return fail(ctx, LP_EINVAL, buf);
+    }
+    CK(cudaSetDevice(device));
+    if (!g_static_scratch_addr[device]) {  // first call on this device: resolve the device address of the array
+        float *addr = nullptr;
+        CK(cudaGetSymbolAddress((void **)&addr, lp_static_scratch));
+        if (!addr) return fail(ctx, LP_ECUDA, "lp_weight_grad_static: cudaGetSymbolAddress returned a null address");
+        g_static_scratch_addr[device] = addr;
+    }
+    float *scratch = g_static_scratch_addr[device];
+    // as many row splits as the fixed array holds (each split writes one full K x N partial tile, so
+    // nothing has to be cleared between calls: every element that is read was written by this call)
+    const int splits = (int)std::max<int64_t>(1, std::min<int64_t>(weight_grad_splits(M), LP_STATIC_SCRATCH_FLOATS / tile));
+    int64_t k_chunk = ceil_div64(ceil_div64(M, splits), SG_BK) * SG_BK;
+    if (k_chunk < SG_BK) k_chunk = SG_BK;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    dim3 grid((unsigned)ceil_div64(K, SG_BM), (unsigned)ceil_div64(N, SG_BN), (unsigned)splits);
+    gemm_simt_kernel<float, float, float, true, true><<<grid, SG_THREADS, 0, st>>>(K, N, M, A, K, dZ, N, (float *)nullptr, 0, nullptr, 0, k_chunk, scratch);
+    reduce_partials_kernel<<<(unsigned)ceil_div64(tile, 256), 256, 0, st>>>(scratch, tile, splits, dW, 0);
+    CK_LAUNCH();
+    return LP_OK;
+}
