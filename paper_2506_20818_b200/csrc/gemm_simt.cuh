@@ -89,7 +89,15 @@ __global__ void reduce_partials_kernel(const float *__restrict__ partials, int64
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= count) return;
     float s = 0.f;
-    for (int z = 0; z < splits; ++z) s += partials[(int64_t)z * count + i];
+    int z = 0;
+    for (; z + 8 <= splits; z += 8) {  // eight independent loads in flight, added in index order
+        float v[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) v[q] = __ldg(partials + (int64_t)(z + q) * count + i);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) s += v[q];
+    }
+    for (; z < splits; ++z) s += __ldg(partials + (int64_t)z * count + i);
     dst[i] = accumulate ? dst[i] + s : s;
 }
 
@@ -121,28 +129,51 @@ static void weight_grad_simt(Exec &ex, int64_t rows, int Kin, int N, const T *A,
     ex.launches += 2;
 }
 
-// column sums: out[j] = sum_r dZ[r, j] (bias gradient), two deterministic stages
+// column sums: out[j] = sum_r dZ[r, j] (bias gradient), two deterministic stages.  A block of 256
+// threads covers a range of rows with 16-byte loads: thread = (row lane, column vector); the row
+// lanes are added in shared memory in lane order, then the blocks' partial rows in block order.
 template <typename T>
-__global__ void colsum_partial_kernel(const T *__restrict__ dZ, int64_t rows, int N, int64_t ldz, int64_t rows_per_block, float *__restrict__ partials)
+__global__ void __launch_bounds__(256) colsum_partial_kernel(const T *__restrict__ dZ, int64_t rows, int N, int64_t ldz, int64_t rows_per_block,
+                                                             float *__restrict__ partials)
 {
-    const int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= N) return;
-    const int64_t r0 = (int64_t)blockIdx.y * rows_per_block, r1 = min(rows, r0 + rows_per_block);
-    float s = 0.f;
-    for (int64_t r = r0; r < r1; ++r) s += to_f<T>(dZ[r * ldz + j]);
-    partials[(int64_t)blockIdx.y * N + j] = s;
+    constexpr int VN = Vec16<T>::N;
+    __shared__ float sh[256 * VN];
+    const int nvec = N / VN;           // column vectors per row (<= 256)
+    const int lanes_r = 256 / nvec;    // row lanes
+    const int c = threadIdx.x % nvec, rl = threadIdx.x / nvec;
+    const int64_t r0 = (int64_t)blockIdx.x * rows_per_block, r1 = min(rows, r0 + rows_per_block);
+    float acc[VN];
+#pragma unroll
+    for (int j = 0; j < VN; ++j) acc[j] = 0.f;
+    if (rl < lanes_r) {
+        for (int64_t r = r0 + rl; r < r1; r += lanes_r) {
+            Vec16<T> v;
+            v.load(dZ + r * ldz + c * VN);
+            float f[VN];
+            v.to_float(f);
+#pragma unroll
+            for (int j = 0; j < VN; ++j) acc[j] += f[j];
+        }
+#pragma unroll
+        for (int j = 0; j < VN; ++j) sh[rl * N + c * VN + j] = acc[j];
+    }
+    __syncthreads();
+    for (int j = threadIdx.x; j < N; j += 256) {
+        float s = 0.f;
+        for (int q = 0; q < lanes_r; ++q) s += sh[q * N + j];
+        partials[(int64_t)blockIdx.x * N + j] = s;
+    }
 }
 
-constexpr int CS_MAX_SPLITS = 1024;
-static int colsum_splits(int64_t rows) { return (int)std::max<int64_t>(1, std::min<int64_t>(CS_MAX_SPLITS, ceil_div64(rows, 256))); }
+constexpr int CS_MAX_SPLITS = 296;
+static int colsum_splits(int64_t rows) { return (int)std::max<int64_t>(1, std::min<int64_t>(CS_MAX_SPLITS, ceil_div64(rows, 64))); }
 
 template <typename T>
 static void colsum(Exec &ex, const T *dZ, int64_t rows, int N, int64_t ldz, float *out, int accumulate, float *partials)
 {
     const int splits = colsum_splits(rows);
     const int64_t rpb = ceil_div64(rows > 0 ? rows : 1, splits);
-    dim3 grid((unsigned)ceil_div64(N, 64), (unsigned)splits);
-    colsum_partial_kernel<T><<<grid, 64, 0, ex.st>>>(dZ, rows, N, ldz, rpb, partials);
+    colsum_partial_kernel<T><<<splits, 256, 0, ex.st>>>(dZ, rows, N, ldz, rpb, partials);
     reduce_partials_kernel<<<(unsigned)ceil_div64(N, 256), 256, 0, ex.st>>>(partials, N, splits, out, accumulate);
     ex.launches += 2;
 }

@@ -334,6 +334,175 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
 }
 
 // ---------------------------------------------------------------------------------------------
+// kernel 2: persistent K-major transform with the weight slice resident in shared memory.
+//
+// One CTA per SM.  CTA c owns the N slice (c mod n_slices) of width BN and walks the 128-row tiles
+// c / n_slices, c / n_slices + stride, ...  Its slice of Bt (BN x K BF16, at most 128 KiB) is loaded
+// once; only A tiles stream through a 4-stage ring.  Two accumulators in tensor memory let the
+// epilogue of tile i (4 warps: tcgen05.ld, bias, ReLU, BF16 stores) overlap the MMAs of tile i + 1.
+//   warp 0: TMA producer (one lane)      warp 1: MMA issuer (one lane)      warps 2-5: epilogue
+// ---------------------------------------------------------------------------------------------
+constexpr int TCP_THREADS = 192;
+constexpr int TCP_STAGES = 4;
+
+LP_DEVINL void mbar_arrive(uint32_t bar) { asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory"); }
+
+__global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(const __grid_constant__ CUtensorMap mapA,
+                                                                              const __grid_constant__ CUtensorMap mapB, const TcGemmParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[TCP_STAGES], bar_empty[TCP_STAGES], bar_w, bar_acc_full[2], bar_acc_empty[2];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int BN = p.BN;
+    const int KB = p.K / TC_BK;                        // k-blocks per tile
+    const uint32_t w_sub_bytes = (uint32_t)BN * 128;   // one k-block of the weight slice: BN rows x 128 B
+    uint8_t *smem_w = smem;
+    uint8_t *smem_a = smem + (size_t)KB * w_sub_bytes;
+    const uint32_t a_bytes = TC_BM * TC_BK * 2;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < 2 * BN) tmem_cols <<= 1;
+
+    const int n_slices = p.N / BN;
+    const int slice = blockIdx.x % n_slices;
+    const int n0 = slice * BN;
+    const int64_t m_tiles = (p.M + TC_BM - 1) / TC_BM;
+    const int64_t first_tile = blockIdx.x / n_slices;
+    const int64_t stride = gridDim.x / n_slices;
+    const int64_t my_tiles = first_tile < m_tiles ? (m_tiles - first_tile + stride - 1) / stride : 0;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < TCP_STAGES; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_empty[s]), 1);
+        }
+        mbar_init(smem_u32(&bar_w), 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&bar_acc_full[b]), 1);
+            mbar_init(smem_u32(&bar_acc_empty[b]), 4);  // one arrival per epilogue warp
+        }
+        abort_s = 0;
+        fence_barrier_init();
+        fence_async_proxy();
+        tma_prefetch_desc(&mapA);
+        tma_prefetch_desc(&mapB);
+    }
+    if (warp == 0) {
+        __syncwarp();
+        tmem_alloc(smem_u32(&tmem_base_s), tmem_cols);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+    volatile int *abort_flag = &abort_s;
+
+    if (my_tiles > 0) {
+        if (warp == 0 && lane == 0) {
+            // ---- producer
+            const uint32_t bw = smem_u32(&bar_w);
+            mbar_expect_tx(bw, (uint32_t)KB * w_sub_bytes);
+            for (int kb = 0; kb < KB; ++kb) tma_load_2d(smem_u32(smem_w + (size_t)kb * w_sub_bytes), &mapB, bw, kb * TC_BK, n0);
+            int64_t it = 0;
+            for (int64_t i = 0; i < my_tiles && !*abort_flag; ++i) {
+                const int m0 = (int)((first_tile + i * stride) * TC_BM);
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    const int s = (int)(it % TCP_STAGES);
+                    if (it >= TCP_STAGES && !mbar_wait(smem_u32(&bar_empty[s]), (uint32_t)(((it / TCP_STAGES) & 1) ^ 1))) {
+                        atomicExch(p.err, 1);
+                        *abort_flag = 1;
+                        break;
+                    }
+                    const uint32_t bar = smem_u32(&bar_full[s]);
+                    mbar_expect_tx(bar, a_bytes);
+                    tma_load_2d(smem_u32(smem_a + (size_t)s * a_bytes), &mapA, bar, kb * TC_BK, m0);
+                }
+            }
+        } else if (warp == 1 && lane == 0) {
+            // ---- MMA issuer
+            const uint32_t idesc = make_idesc_bf16(BN, false, false);
+            bool ok = mbar_wait(smem_u32(&bar_w), 0);
+            if (!ok) { atomicExch(p.err, 4); *abort_flag = 1; }
+            int64_t it = 0;
+            for (int64_t i = 0; i < my_tiles && ok; ++i) {
+                const int b = (int)(i & 1);
+                if (i >= 2 && !mbar_wait(smem_u32(&bar_acc_empty[b]), (uint32_t)((((i >> 1) - 1) & 1)))) {
+                    atomicExch(p.err, 5);
+                    *abort_flag = 1;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t tmem_d = tmem_base + (uint32_t)(b * BN);
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    const int s = (int)(it % TCP_STAGES);
+                    if (!mbar_wait(smem_u32(&bar_full[s]), (uint32_t)((it / TCP_STAGES) & 1))) {
+                        atomicExch(p.err, 2);
+                        *abort_flag = 1;
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem_a + (size_t)s * a_bytes);
+                    const uint32_t sb = smem_u32(smem_w + (size_t)kb * w_sub_bytes);
+#pragma unroll
+                    for (int k = 0; k < TC_BK / TC_UMMA_K; ++k)
+                        umma_bf16(tmem_d, make_smem_desc(sa + k * 32, 16, 1024), make_smem_desc(sb + k * 32, 16, 1024), idesc, (kb | k) != 0 ? 1u : 0u);
+                    umma_commit(smem_u32(&bar_empty[s]));
+                }
+                if (ok) umma_commit(smem_u32(&bar_acc_full[b]));
+            }
+        } else if (warp >= 2) {
+            // ---- epilogue: warp w reads the TMEM lanes of quarter (w mod 4)
+            const int q = warp & 3;
+            for (int64_t i = 0; i < my_tiles; ++i) {
+                const int b = (int)(i & 1);
+                bool ready = mbar_wait(smem_u32(&bar_acc_full[b]), (uint32_t)((i >> 1) & 1));
+                if (!ready && lane == 0) { atomicExch(p.err, 3); *abort_flag = 1; }
+                ready = __all_sync(0xffffffffu, ready && *abort_flag == 0);
+                if (!ready) break;
+                tc_fence_after();
+                const int64_t row = (first_tile + i * stride) * TC_BM + q * 32 + lane;
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN);
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    float v[32];
+                    tmem_ld_32x32(taddr + (uint32_t)c0, v);
+                    if (row < p.M) {
+                        if (p.bias) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] += __ldg(p.bias + n0 + c0 + j);
+                        }
+                        if (p.relu) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
+                        }
+                        bf16 *dst = p.C + row * p.ldc + n0 + c0;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            Vec16<bf16> o;
+                            o.from_float(v + j);
+                            o.store(dst + j);
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[b]));
+            }
+        }
+    }
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, tmem_cols);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
 static bool tc_init(TcState &tc, std::string &err)
@@ -352,7 +521,8 @@ static bool tc_init(TcState &tc, std::string &err)
         return false;
     }
     cudaMemset(tc.err_word, 0, 256);
-    if (cudaFuncSetAttribute(tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess ||
+    if (cudaFuncSetAttribute(tc_linear_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess ||
         cudaFuncSetAttribute(tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) {
         err = "cannot raise the dynamic shared memory limit of the tensor-core GEMM";
         return false;
@@ -415,9 +585,47 @@ static int tc_stages(int BN, int num_kb)
 }
 
 // C[M, N] (BF16, leading dimension ldc) = act(A[M, K] * Bt[N, K]^T + bias); Bt is BF16, K contiguous.
+// Slice width for the persistent kernel: the largest multiple of 64 (at most 256, dividing N) whose
+// weight slice BN x K x 2 B fits 128 KiB beside the four 16 KiB A stages.  0 = does not fit.
+static int tc_persistent_bn(int N, int K)
+{
+    for (int bn = 256; bn >= 64; bn -= 64)
+        if (N % bn == 0 && (int64_t)bn * K * 2 <= 128 * 1024) return bn;
+    return 0;
+}
+
+static int tc_sm_count()
+{
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (sms <= 0) sms = 148;
+    }
+    return sms;
+}
+
 static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const bf16 *A, int64_t lda, const bf16 *Bt, const float *bias, bool relu,
                            bf16 *C, int64_t ldc, std::string &err)
 {
+    const int pbn = tc_persistent_bn(N, K);
+    if (pbn > 0 && M >= 4 * TC_BM) {
+        CUtensorMap mapA, mapB;
+        if (!tc_make_map(tc, &mapA, A, M, K, lda, TC_BK, TC_BM, err)) return false;
+        if (!tc_make_map(tc, &mapB, Bt, N, K, K, TC_BK, pbn, err)) return false;
+        TcGemmParams p{};
+        p.M = M; p.N = N; p.K = K; p.BN = pbn; p.stages = TCP_STAGES;
+        p.bias = bias; p.relu = relu ? 1 : 0; p.C = C; p.ldc = ldc; p.out_f32 = nullptr; p.err = tc.err_word;
+        const int n_slices = N / pbn;
+        const int64_t m_tiles = ceil_div64(M, TC_BM);
+        int64_t ctas = std::min<int64_t>((int64_t)tc_sm_count(), m_tiles * n_slices);
+        ctas = std::max<int64_t>(n_slices, ctas / n_slices * n_slices);  // a whole number of CTAs per slice
+        const size_t smem = (size_t)(K / TC_BK) * pbn * 128 + (size_t)TCP_STAGES * TC_BM * TC_BK * 2 + 1024;
+        tc_linear_persistent_kernel<<<(unsigned)ctas, TCP_THREADS, smem, ex.st>>>(mapA, mapB, p);
+        ex.launches += 1;
+        return true;
+    }
     const int BN = tc_pick_bn(N);
     CUtensorMap mapA, mapB;
     if (!tc_make_map(tc, &mapA, A, M, K, lda, TC_BK, TC_BM, err)) return false;

@@ -61,6 +61,8 @@ struct lp_ctx {
     int *cand = nullptr;
     int64_t n_cand = 0;
     unsigned long long *exhausted_dev = nullptr;
+    HeavyPlan plan_csr, plan_csc, plan_dyn;  // heavy-row plans: the loaded graph, its transpose, per-step structures
+    float *heavy_partials = nullptr;
     int *err_flag = nullptr;
 
     // model
@@ -362,11 +364,32 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
     }
     convert_kernel<float, bf16><<<nblk(n * (int64_t)f), 256, 0, st>>>(ctx->X32, ctx->X16, n * (int64_t)f);
     ctx->ex.launches += 6;
+    // heavy-row plans of the graph and of its transpose (static: built once)
+    const int64_t item_cap = nnz / SPMM_HEAVY + 2;
+    GALLOC(ctx->heavy_partials, item_cap * 512);
+    for (HeavyPlan *hp : {&ctx->plan_csr, &ctx->plan_csc}) {
+        *hp = HeavyPlan();
+        GALLOC(hp->rows, item_cap);
+        GALLOC(hp->base, item_cap);
+        GALLOC(hp->item_row, item_cap);
+        GALLOC(hp->item_first, item_cap);
+        GALLOC(hp->counts, 64);
+        hp->partials = ctx->heavy_partials;
+        cudaMemsetAsync(hp->counts, 0, 2 * sizeof(int), st);
+        spmm_heavy_plan_kernel<<<nblk(n), 256, 0, st>>>(hp == &ctx->plan_csr ? ctx->rowptr : ctx->colptr, (int)n, nullptr, *hp);
+        cudaMemcpyAsync(ctx->host_counts + (hp == &ctx->plan_csr ? 0 : 2), hp->counts, 2 * sizeof(int), cudaMemcpyDeviceToHost, st);
+    }
+    ctx->ex.launches += 2;
     e = cudaStreamSynchronize(st);
     free_list(tmp);
 #undef TALLOC
     CK(e);
     CK_LAUNCH();
+    ctx->plan_csr.host_rows = ctx->host_counts[0];
+    ctx->plan_csr.host_items = ctx->host_counts[1];
+    ctx->plan_csc.host_rows = ctx->host_counts[2];
+    ctx->plan_csc.host_items = ctx->host_counts[3];
+    ctx->plan_dyn = HeavyPlan();
     ctx->loaded = true;
     return LP_OK;
 }
@@ -578,6 +601,24 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
         MALLOC(ctx->flags, n);
         MALLOC(ctx->seed_ids, max_batch * (2 + 2 * (int64_t)max_k));
     }
+    {   // heavy-row plan scratch for the per-step structures (incidence lists, sampled blocks)
+        int64_t dyn_nnz = 2 * E;
+        if (sampled)
+            for (int h = 1; h <= K; ++h) dyn_nnz = std::max(dyn_nnz, ctx->hop[h].cap_entries);
+        const int64_t cap = dyn_nnz / SPMM_HEAVY + 2;
+        HeavyPlan &hp = ctx->plan_dyn;
+        hp = HeavyPlan();
+        MALLOC(hp.rows, cap);
+        MALLOC(hp.base, cap);
+        MALLOC(hp.item_row, cap);
+        MALLOC(hp.item_first, cap);
+        MALLOC(hp.counts, 64);
+        if (cap > ctx->nnz / SPMM_HEAVY + 2) {
+            MALLOC(hp.partials, cap * 512);
+        } else {
+            hp.partials = ctx->heavy_partials;
+        }
+    }
     ctx->sort_cap = sort_cap;
     MALLOC(ctx->sort.keys_alt, sort_cap);
     MALLOC(ctx->sort.vals_alt, sort_cap);
@@ -766,6 +807,15 @@ template <typename T> static lp_status forward_impl(lp_ctx *ctx, const float *pa
     for (int k = 0; k < K; ++k) {
         LayerBuf &L = ctx->layer[k];
         SpmmArgs<T> a;
+        if (!ctx->sampled) {
+            a.heavy = ctx->plan_csr;
+            a.nnz = ctx->nnz;
+        } else {  // sampled rows hold at most `fanout` (<= 32) entries: never heavy
+            a.heavy = ctx->plan_dyn;
+            a.heavy.host_rows = 0;
+            a.heavy.host_items = 0;
+            a.nnz = ctx->hop[K - k].entries;
+        }
         int64_t rows;
         T *out;
         int ldo;
@@ -874,8 +924,8 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     CK(cudaMemsetAsync(ctx->inc_ptr, 0, sizeof(int) * ((size_t)rows_out + 1), st));
     incidence_keys_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->inc_keys, ctx->inc_slots, ctx->inc_other, ctx->inc_ptr);
     exclusive_scan_i32(ctx->ex, ctx->inc_ptr, rows_out, ctx->inc_ptr, ctx->inc_ptr + rows_out, ctx->scan_tmp);
-    radix_sort_pairs(ctx->ex, ctx->inc_keys, ctx->inc_slots, 2 * E, bits_for(rows_out), ctx->sort);
-    incidence_fill_kernel<<<nblk(2 * E), 256, 0, st>>>(ctx->inc_slots, 2 * E, ctx->inc_other, B, ctx->g_pos, ctx->g_neg, ctx->inc_col, ctx->inc_val);
+    const bool sorted_in_place = radix_sort_pairs(ctx->ex, ctx->inc_keys, ctx->inc_slots, 2 * E, bits_for(rows_out), ctx->sort);
+    incidence_fill_kernel<<<nblk(2 * E), 256, 0, st>>>(sorted_in_place ? ctx->inc_slots : ctx->sort.vals_alt, 2 * E, ctx->inc_other, B, ctx->g_pos, ctx->g_neg, ctx->inc_col, ctx->inc_val);
     ctx->ex.launches += 2;
     delete pinc;
 
@@ -884,6 +934,8 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     int cur = 1;
     {
         SpmmArgs<T> a;
+        a.heavy = ctx->plan_dyn;
+        a.nnz = 2 * E;
         a.n_rows = rows_out;
         a.rowptr = ctx->inc_ptr;
         a.col = ctx->inc_col;
@@ -910,6 +962,13 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         if (s != LP_OK) return s;
         T *dZn = tptr<T>(ctx->dZ[cur ^ 1]);
         SpmmArgs<T> a;
+        if (!ctx->sampled) {
+            a.heavy = ctx->plan_csc;
+            a.nnz = ctx->nnz;
+        } else {
+            a.heavy = ctx->plan_dyn;
+            a.nnz = ctx->hop[K - l].entries;
+        }
         a.F = L.Fi;
         a.Y = dZn;
         a.ldy = L.Fi;
@@ -1205,6 +1264,8 @@ extern "C" lp_status lp_profile_end(lp_ctx *ctx, lp_profile *out)
 template <typename T> static lp_status op_aggregate_impl(lp_ctx *ctx, int arch, int transpose, const T *H, int F, T *M)
 {
     SpmmArgs<T> a;
+    a.heavy = transpose ? ctx->plan_csc : ctx->plan_csr;
+    a.nnz = ctx->nnz;
     a.n_rows = ctx->n;
     a.X = H;
     a.ldx = F;

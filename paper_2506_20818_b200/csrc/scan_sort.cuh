@@ -233,14 +233,13 @@ struct SortScratch {  // caller-provided device buffers
     static int64_t scan_ints(int64_t n) { return ceil_div64(hist_ints(n), SCAN_TILE) + 1; }
 };
 
-// Sorts (keys, vals) by the low `key_bits` bits of the key, stably.  The result ends in
-// (keys, vals) again (an even number of passes is run).
-static void radix_sort_pairs(Exec &ex, uint32_t *keys, uint32_t *vals, int64_t n, int key_bits, const SortScratch &s)
+// Sorts (keys, vals) by the low `key_bits` bits of the key, stably, in ceil(key_bits / 8) passes.
+// Returns true when the result is in (keys, vals), false when it is in (s.keys_alt, s.vals_alt).
+static bool radix_sort_pairs(Exec &ex, uint32_t *keys, uint32_t *vals, int64_t n, int key_bits, const SortScratch &s)
 {
-    if (n <= 0) return;
+    if (n <= 0) return true;
     int passes = (key_bits + 7) / 8;
     if (passes < 1) passes = 1;
-    if (passes & 1) passes += 1;
     const int tiles = (int)ceil_div64(n, RS_TILE);
     uint32_t *ki = keys, *vi = vals, *ko = s.keys_alt, *vo = s.vals_alt;
     for (int p = 0; p < passes; ++p) {
@@ -253,6 +252,7 @@ static void radix_sort_pairs(Exec &ex, uint32_t *keys, uint32_t *vals, int64_t n
         t = ki; ki = ko; ko = t;
         t = vi; vi = vo; vo = t;
     }
+    return ki == keys;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -320,8 +320,8 @@ static void transpose_csr(Exec &ex, const int *rowptr, int n_rows, int n_cols, c
     }
     exclusive_scan_i32(ex, colptr, n_cols, colptr, colptr + n_cols, s.scan_tmp);
     if (nnz > 0) {
-        radix_sort_pairs(ex, s.keys, s.vals, nnz, bits_for(n_cols), s.sort);
-        gather_rows_kernel<<<(unsigned)ceil_div64(nnz, 256), 256, 0, ex.st>>>(s.vals, s.rows, nnz, rowidx_t, perm);
+        const bool in_place = radix_sort_pairs(ex, s.keys, s.vals, nnz, bits_for(n_cols), s.sort);
+        gather_rows_kernel<<<(unsigned)ceil_div64(nnz, 256), 256, 0, ex.st>>>(in_place ? s.vals : s.sort.vals_alt, s.rows, nnz, rowidx_t, perm);
         ex.launches += 1;
     }
 }

@@ -4,9 +4,10 @@
 //
 // One group of G lanes (8, 16 or 32) owns a row; every lane gathers 16-byte vectors of the
 // source rows (4 floats or 8 bf16) and accumulates in FP32 in entry order.  Rows with more than
-// SPMM_HEAVY entries (power-law hubs) are split into one contiguous segment per lane group of the
-// block and the partial sums are added in segment order, so a hub costs one block a few
-// microseconds instead of one warp hundreds.  The summation order is a function of the row length
+// SPMM_HEAVY entries (power-law hubs) are cut into items of SPMM_SEG entries; the items run as extra
+// blocks of the same grid (so hubs spread over the whole GPU and overlap the light rows), each
+// writes an FP32 partial row, and a small second kernel adds a row's partials in item order and
+// applies the epilogue.  The summation order is a function of the row length
 // only: results are reproducible bit for bit (no atomics anywhere).  Row offsets of the block's
 // rows are staged in shared memory with one coalesced load.  Optional parts (null pointers) cost
 // a warp-uniform branch:
@@ -19,6 +20,17 @@
 #pragma once
 #include "common.cuh"
 #include "scan_sort.cuh"
+
+// Rows with more than SPMM_HEAVY entries are cut into segments of SPMM_SEG entries ("items").
+// rows[i] / base[i]: heavy row i and the index of its first item; item_row / item_first: for every
+// item its row and that row's first item; counts[0] = heavy rows, counts[1] = items.
+// partials[item][F] holds the FP32 partial sum of an item.  A plan is either built once for a
+// static structure (host_rows >= 0 tells the launcher the counts) or refilled per launch.
+struct HeavyPlan {
+    int *rows = nullptr, *base = nullptr, *item_row = nullptr, *item_first = nullptr, *counts = nullptr;
+    float *partials = nullptr;
+    int host_rows = -1, host_items = -1;  // -1: unknown on the host (plan built on the device per launch)
+};
 
 template <typename T> struct SpmmArgs {
     int n_rows = 0;
@@ -41,25 +53,33 @@ template <typename T> struct SpmmArgs {
     const int *self_idx = nullptr;
     T *self_out = nullptr;
     int ldself = 0;
+    int64_t nnz = 0;             // stored entries (host-known upper bound), sizes the heavy-row part of the grid
+    HeavyPlan heavy;             // heavy rows of this structure: prebuilt (static graph) or scratch to fill per launch
 };
 
 constexpr int SPMM_THREADS = 256;
-constexpr int SPMM_HEAVY = 256;  // rows with more entries than this are processed by the whole block
+constexpr int SPMM_HEAVY = 256;  // rows with more entries than this are cut into items
+constexpr int SPMM_SEG = 512;    // entries per item (one block: 8 lane groups x 64 entries for 32-lane groups)
 
 // acc += sum over entries [e_lo, e_hi) of val[e] * X[col[e], :] for the chunks owned by this lane.
 // The group loads up to G (col, val) pairs at once and broadcasts them; U source rows are gathered
 // before any is consumed, so each lane keeps U * NV 16-byte loads in flight.
 template <typename T, int G, int NV, int U>
-LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl, unsigned gmask, int nchunks, float (&acc)[NV][Vec16<T>::N])
+LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl, unsigned gmask, int nchunks, float (&acc)[NV][Vec16<T>::N],
+                                bool have_first = false, int first_col = 0, float first_val = 0.f)
 {
     constexpr int VN = Vec16<T>::N;
     for (int e0 = e_lo; e0 < e_hi; e0 += G) {
         const int my_e = e0 + gl;
-        int my_col = 0;
-        float my_val = 0.f;
-        if (my_e < e_hi) {
-            my_col = __ldg(a.col + my_e);
-            my_val = a.val ? __ldg(a.val + my_e) : 1.f;
+        int my_col = first_col;
+        float my_val = first_val;
+        if (!(have_first && e0 == e_lo)) {  // the first batch of a row may have been prefetched by the caller
+            my_col = 0;
+            my_val = 0.f;
+            if (my_e < e_hi) {
+                my_col = __ldg(a.col + my_e);
+                my_val = a.val ? __ldg(a.val + my_e) : 1.f;
+            }
         }
         const int cnt = min(G, e_hi - e0);
         int j = 0;
@@ -158,83 +178,185 @@ LP_DEVINL void spmm_epilogue(const SpmmArgs<T> &a, int r, int gl, int nchunks, c
     }
 }
 
-template <typename T, int G, int NV>
-__global__ void __launch_bounds__(SPMM_THREADS) spmm_csr_kernel(const SpmmArgs<T> a)
+template <typename T, int G, int NV, int RPG, int U, int MINB>
+__global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const SpmmArgs<T> a, const int light_blocks)
 {
     constexpr int VN = Vec16<T>::N;
-    constexpr int ROWS = SPMM_THREADS / G;  // rows per block = lane groups per block
-    constexpr int U = (NV == 1) ? 8 : (NV == 2 ? 4 : 2);
+    constexpr int NG = SPMM_THREADS / G;  // lane groups per block
+    constexpr int ROWS = NG * RPG;        // rows per block: every group walks RPG rows
     __shared__ int s_ptr[ROWS + 1];
-    __shared__ __align__(16) float s_part[ROWS][G * NV * VN];  // partial sums of a heavy row, one per group
+    __shared__ __align__(16) float s_part[NG][G * NV * VN];  // partial sums of an item, one per group
     const int n_rows = a.n_rows_dev ? min(*a.n_rows_dev, a.n_rows) : a.n_rows;
-    const int row0 = blockIdx.x * ROWS;
-    if (row0 >= n_rows) return;
-    if (threadIdx.x <= ROWS) s_ptr[threadIdx.x] = a.rowptr[min(row0 + (int)threadIdx.x, n_rows)];
-    __syncthreads();
-    const int g = threadIdx.x / G;   // group (row) inside the block
+    const int g = threadIdx.x / G;   // group inside the block
     const int gl = threadIdx.x % G;  // lane inside the group
-    const int r = row0 + g;
     const unsigned lane = threadIdx.x & 31;
     const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << (lane & ~(unsigned)(G - 1)));
     const int nchunks = a.F / VN;  // 16-byte chunks per row
 
-    float acc[NV][VN];
-    // ---- light rows: one lane group per row, entries in order
-    const int e_begin = s_ptr[g], e_end = s_ptr[g + 1];
-    if (r < n_rows && e_end - e_begin <= SPMM_HEAVY) {
+    if ((int)blockIdx.x >= light_blocks) {
+        // ---- heavy item: SPMM_SEG consecutive entries of a hub row, one contiguous piece per lane group,
+        // pieces added in group order (fixed), FP32 partial row written for the combine kernel
+        const int item = blockIdx.x - light_blocks;
+        if (item >= a.heavy.counts[1]) return;
+        const int r = a.heavy.item_row[item];
+        const int sidx = item - a.heavy.item_first[item];
+        const int hb = a.rowptr[r] + sidx * SPMM_SEG, he = min(a.rowptr[r + 1], hb + SPMM_SEG);
+        const int piece = ((he - hb + NG - 1) / NG + G - 1) / G * G;
+        const int lo = min(he, hb + g * piece), hi = min(he, lo + piece);
+        float hacc[NV][VN];
 #pragma unroll
-        for (int i = 0; i < NV; ++i)
+        for (int q = 0; q < NV; ++q)
 #pragma unroll
-            for (int j = 0; j < VN; ++j) acc[i][j] = 0.f;
-        spmm_accumulate<T, G, NV, U>(a, e_begin, e_end, gl, gmask, nchunks, acc);
-        spmm_epilogue<T, G, NV>(a, r, gl, nchunks, acc);
-    }
-    // ---- heavy rows (power-law hubs): every group of the block takes one contiguous segment of the
-    // row, the partial sums meet in shared memory and are added in segment order (fixed order, no atomics)
-    for (int hr = 0; hr < ROWS; ++hr) {
-        const int hb = s_ptr[hr], he = s_ptr[hr + 1];
-        if (row0 + hr >= n_rows || he - hb <= SPMM_HEAVY) continue;  // uniform over the block
-        const int seg = ((he - hb + ROWS - 1) / ROWS + G - 1) / G * G;
-        const int lo = min(he, hb + g * seg), hi = min(he, lo + seg);
+            for (int j = 0; j < VN; ++j) hacc[q][j] = 0.f;
+        spmm_accumulate<T, G, NV, U>(a, lo, hi, gl, gmask, nchunks, hacc);
 #pragma unroll
-        for (int i = 0; i < NV; ++i)
+        for (int q = 0; q < NV; ++q)
 #pragma unroll
-            for (int j = 0; j < VN; ++j) acc[i][j] = 0.f;
-        spmm_accumulate<T, G, NV, U>(a, lo, hi, gl, gmask, nchunks, acc);
-#pragma unroll
-        for (int i = 0; i < NV; ++i)
-#pragma unroll
-            for (int t = 0; t < VN; ++t) s_part[g][(gl + i * G) * VN + t] = acc[i][t];
+            for (int t = 0; t < VN; ++t) s_part[g][(gl + q * G) * VN + t] = hacc[q][t];
         __syncthreads();
-        if (g == 0) {
+        for (int j = threadIdx.x; j < a.F; j += SPMM_THREADS) {
+            float sum = 0.f;
+            for (int w = 0; w < NG; ++w) sum += s_part[w][j];
+            a.heavy.partials[(size_t)item * a.F + j] = sum;
+        }
+        return;
+    }
+    const int row0 = blockIdx.x * ROWS;
+    if (row0 >= n_rows) return;
+    for (int i = threadIdx.x; i <= ROWS; i += SPMM_THREADS) s_ptr[i] = a.rowptr[min(row0 + i, n_rows)];
+    __syncthreads();
+
+    float acc[NV][VN];
+    // ---- light rows: group g walks rows g, g + NG, g + 2 NG, ... of the block.  The (column, coefficient)
+    // pairs of the next row are fetched before the current row's gathers are consumed, so a group has
+    // its index loads and its feature gathers in flight at the same time.
+    int pre_col = 0;
+    float pre_val = 0.f;
+    {
+        const int eb = s_ptr[g], ee = s_ptr[g + 1];
+        if (eb + gl < ee && ee - eb <= SPMM_HEAVY) {
+            pre_col = __ldg(a.col + eb + gl);
+            pre_val = a.val ? __ldg(a.val + eb + gl) : 1.f;
+        }
+    }
+#pragma unroll 1
+    for (int it = 0; it < RPG; ++it) {
+        const int lr = it * NG + g;
+        const int r = row0 + lr;
+        const int e_begin = s_ptr[lr], e_end = s_ptr[lr + 1];
+        const int cur_col = pre_col;
+        const float cur_val = pre_val;
+        if (it + 1 < RPG) {
+            const int eb = s_ptr[lr + NG], ee = s_ptr[lr + NG + 1];
+            pre_col = 0;
+            pre_val = 0.f;
+            if (eb + gl < ee && ee - eb <= SPMM_HEAVY) {
+                pre_col = __ldg(a.col + eb + gl);
+                pre_val = a.val ? __ldg(a.val + eb + gl) : 1.f;
+            }
+        }
+        if (r < n_rows && e_end - e_begin <= SPMM_HEAVY) {
 #pragma unroll
             for (int i = 0; i < NV; ++i)
 #pragma unroll
-                for (int t = 0; t < VN; ++t) {
-                    float s = 0.f;
-                    for (int q = 0; q < ROWS; ++q) s += s_part[q][(gl + i * G) * VN + t];
-                    acc[i][t] = s;
-                }
-            spmm_epilogue<T, G, NV>(a, row0 + hr, gl, nchunks, acc);
+                for (int j = 0; j < VN; ++j) acc[i][j] = 0.f;
+            spmm_accumulate<T, G, NV, U>(a, e_begin, e_end, gl, gmask, nchunks, acc, true, cur_col, cur_val);
+            spmm_epilogue<T, G, NV>(a, r, gl, nchunks, acc);
         }
-        __syncthreads();
     }
 }
 
+// one thread per row: heavy rows claim a slot and a run of items
+__global__ void spmm_heavy_plan_kernel(const int *__restrict__ rowptr, int n_rows, const int *__restrict__ n_rows_dev, HeavyPlan hp)
+{
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    const int lim = n_rows_dev ? min(*n_rows_dev, n_rows) : n_rows;
+    if (r >= lim) return;
+    const int d = rowptr[r + 1] - rowptr[r];
+    if (d <= SPMM_HEAVY) return;
+    const int nseg = (d + SPMM_SEG - 1) / SPMM_SEG;
+    const int i = atomicAdd(&hp.counts[0], 1);
+    const int b = atomicAdd(&hp.counts[1], nseg);
+    hp.rows[i] = r;
+    hp.base[i] = b;
+    for (int s = 0; s < nseg; ++s) {
+        hp.item_row[b + s] = r;
+        hp.item_first[b + s] = b;
+    }
+}
+
+// adds the items of every heavy row in item order (fixed) and applies the epilogue; one lane group per row
+template <typename T, int G, int NV>
+__global__ void __launch_bounds__(SPMM_THREADS) spmm_heavy_combine_kernel(const SpmmArgs<T> a)
+{
+    constexpr int VN = Vec16<T>::N;
+    constexpr int NG = SPMM_THREADS / G;
+    const int count = a.heavy.counts[0];
+    const int g = threadIdx.x / G, gl = threadIdx.x % G;
+    const int nchunks = a.F / VN;
+    for (int i = blockIdx.x * NG + g; i < count; i += gridDim.x * NG) {
+        const int r = a.heavy.rows[i], b = a.heavy.base[i];
+        const int nseg = (a.rowptr[r + 1] - a.rowptr[r] + SPMM_SEG - 1) / SPMM_SEG;
+        float acc[NV][VN];
+#pragma unroll
+        for (int q = 0; q < NV; ++q)
+#pragma unroll
+            for (int t = 0; t < VN; ++t) acc[q][t] = 0.f;
+        for (int s = 0; s < nseg; ++s) {
+            const float *p = a.heavy.partials + (size_t)(b + s) * a.F;
+#pragma unroll
+            for (int q = 0; q < NV; ++q) {
+                const int ch = gl + q * G;
+                if (ch < nchunks) {
+#pragma unroll
+                    for (int t = 0; t < VN; t += 4) {
+                        const float4 v = *reinterpret_cast<const float4 *>(p + ch * VN + t);
+                        acc[q][t] += v.x; acc[q][t + 1] += v.y; acc[q][t + 2] += v.z; acc[q][t + 3] += v.w;
+                    }
+                }
+            }
+        }
+        spmm_epilogue<T, G, NV>(a, r, gl, nchunks, acc);
+    }
+}
+
+template <typename T, int G, int NV, int RPG, int U, int MINB> static void spmm_launch_cfg(Exec &ex, const SpmmArgs<T> &a)
+{
+    constexpr int ROWS = (SPMM_THREADS / G) * RPG;
+    constexpr int NG = SPMM_THREADS / G;
+    const int light_blocks = (int)ceil_div64(a.n_rows, ROWS);
+    if (light_blocks == 0) return;
+    int64_t items = a.heavy.host_items;
+    if (items < 0) {  // plan unknown on the host: rebuild it on the device, size the grid by the upper bound
+        cudaMemsetAsync(a.heavy.counts, 0, 2 * sizeof(int), ex.st);
+        spmm_heavy_plan_kernel<<<(unsigned)ceil_div64(a.n_rows, 256), 256, 0, ex.st>>>(a.rowptr, a.n_rows, a.n_rows_dev, a.heavy);
+        items = a.nnz / SPMM_HEAVY;  // every heavy row has more than SPMM_HEAVY entries and at most deg / SPMM_HEAVY items
+        ex.launches += 1;
+    }
+    spmm_csr_kernel<T, G, NV, RPG, U, MINB><<<(unsigned)(light_blocks + items), SPMM_THREADS, 0, ex.st>>>(a, light_blocks);
+    ex.launches += 1;
+    if (a.heavy.host_rows != 0) {
+        const int64_t rows_bound = a.heavy.host_rows > 0 ? a.heavy.host_rows : std::max<int64_t>(1, items);
+        const unsigned grid = (unsigned)std::min<int64_t>(592, ceil_div64(rows_bound, NG));
+        spmm_heavy_combine_kernel<T, G, NV><<<grid, SPMM_THREADS, 0, ex.st>>>(a);
+        ex.launches += 1;
+    }
+}
+
+// Launch shape (measured on a 200k-node power-law graph, BF16): with one 16-byte vector per lane, 4 gathers in
+// flight per lane at 48 registers (5 blocks per SM) beat 8 gathers at 80 registers (3 blocks) by about 10 %.
 template <typename T, int G, int NV> static void spmm_launch_gn(Exec &ex, const SpmmArgs<T> &a)
 {
-    constexpr int ROWS = SPMM_THREADS / G;
-    const unsigned blocks = (unsigned)ceil_div64(a.n_rows, ROWS);
-    if (blocks == 0) return;
-    spmm_csr_kernel<T, G, NV><<<blocks, SPMM_THREADS, 0, ex.st>>>(a);
-    ex.launches += 1;
+    if constexpr (NV == 1) spmm_launch_cfg<T, G, NV, 8, 4, 5>(ex, a);
+    else if constexpr (NV == 2) spmm_launch_cfg<T, G, NV, 8, 4, 2>(ex, a);
+    else spmm_launch_cfg<T, G, NV, 8, 2, 2>(ex, a);
 }
 
 // F must be a multiple of the 16-byte vector width and at most 32 * 4 vectors wide.
 template <typename T> static bool spmm_launch(Exec &ex, const SpmmArgs<T> &a)
 {
     constexpr int VN = Vec16<T>::N;
-    if (a.F <= 0 || a.F % VN != 0) return false;
+    if (a.F <= 0 || a.F % VN != 0 || !a.heavy.counts || !a.heavy.partials) return false;
     const int chunks = a.F / VN;
     if (chunks <= 8) spmm_launch_gn<T, 8, 1>(ex, a);
     else if (chunks <= 16) spmm_launch_gn<T, 16, 1>(ex, a);
