@@ -365,7 +365,8 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
     convert_kernel<float, bf16><<<nblk(n * (int64_t)f), 256, 0, st>>>(ctx->X32, ctx->X16, n * (int64_t)f);
     ctx->ex.launches += 6;
     // heavy-row plans of the graph and of its transpose (static: built once)
-    const int64_t item_cap = nnz / SPMM_HEAVY + 2;
+    const int64_t item_cap = nnz / SPMM_HEAVY_MIN + 2;
+    const int static_threshold = 128;  // measured best on a 200k-node power-law graph (64: 282 us, 128: 249 us, 256: 241 us at F=256; 176 / 163 / 193 us at F=128)
     GALLOC(ctx->heavy_partials, item_cap * 512);
     for (HeavyPlan *hp : {&ctx->plan_csr, &ctx->plan_csc}) {
         *hp = HeavyPlan();
@@ -375,6 +376,7 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
         GALLOC(hp->item_first, item_cap);
         GALLOC(hp->counts, 64);
         hp->partials = ctx->heavy_partials;
+        hp->threshold = static_threshold;
         cudaMemsetAsync(hp->counts, 0, 2 * sizeof(int), st);
         spmm_heavy_plan_kernel<<<nblk(n), 256, 0, st>>>(hp == &ctx->plan_csr ? ctx->rowptr : ctx->colptr, (int)n, nullptr, *hp);
         cudaMemcpyAsync(ctx->host_counts + (hp == &ctx->plan_csr ? 0 : 2), hp->counts, 2 * sizeof(int), cudaMemcpyDeviceToHost, st);
@@ -605,7 +607,7 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
         int64_t dyn_nnz = 2 * E;
         if (sampled)
             for (int h = 1; h <= K; ++h) dyn_nnz = std::max(dyn_nnz, ctx->hop[h].cap_entries);
-        const int64_t cap = dyn_nnz / SPMM_HEAVY + 2;
+        const int64_t cap = dyn_nnz / SPMM_HEAVY_MIN + 2;
         HeavyPlan &hp = ctx->plan_dyn;
         hp = HeavyPlan();
         MALLOC(hp.rows, cap);
@@ -613,7 +615,7 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
         MALLOC(hp.item_row, cap);
         MALLOC(hp.item_first, cap);
         MALLOC(hp.counts, 64);
-        if (cap > ctx->nnz / SPMM_HEAVY + 2) {
+        if (cap > ctx->nnz / SPMM_HEAVY_MIN + 2) {
             MALLOC(hp.partials, cap * 512);
         } else {
             hp.partials = ctx->heavy_partials;

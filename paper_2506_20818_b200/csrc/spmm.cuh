@@ -4,7 +4,7 @@
 //
 // One group of G lanes (8, 16 or 32) owns a row; every lane gathers 16-byte vectors of the
 // source rows (4 floats or 8 bf16) and accumulates in FP32 in entry order.  Rows with more than
-// SPMM_HEAVY entries (power-law hubs) are cut into items of SPMM_SEG entries; the items run as extra
+// a per-structure threshold of entries (power-law hubs) are cut into items of SPMM_SEG entries; the items run as extra
 // blocks of the same grid (so hubs spread over the whole GPU and overlap the light rows), each
 // writes an FP32 partial row, and a small second kernel adds a row's partials in item order and
 // applies the epilogue.  The summation order is a function of the row length
@@ -21,7 +21,7 @@
 #include "common.cuh"
 #include "scan_sort.cuh"
 
-// Rows with more than SPMM_HEAVY entries are cut into segments of SPMM_SEG entries ("items").
+// Rows with more than `threshold` entries are cut into segments of SPMM_SEG entries ("items").
 // rows[i] / base[i]: heavy row i and the index of its first item; item_row / item_first: for every
 // item its row and that row's first item; counts[0] = heavy rows, counts[1] = items.
 // partials[item][F] holds the FP32 partial sum of an item.  A plan is either built once for a
@@ -30,6 +30,7 @@ struct HeavyPlan {
     int *rows = nullptr, *base = nullptr, *item_row = nullptr, *item_first = nullptr, *counts = nullptr;
     float *partials = nullptr;
     int host_rows = -1, host_items = -1;  // -1: unknown on the host (plan built on the device per launch)
+    int threshold = 64;                   // rows with more entries than this are heavy (>= SPMM_HEAVY_MIN)
 };
 
 template <typename T> struct SpmmArgs {
@@ -58,7 +59,10 @@ template <typename T> struct SpmmArgs {
 };
 
 constexpr int SPMM_THREADS = 256;
-constexpr int SPMM_HEAVY = 256;  // rows with more entries than this are cut into items
+constexpr int SPMM_HEAVY_MIN = 64;  // smallest heavy-row threshold a plan may use (bounds the item count by nnz / 64).
+                                    // A lane group keeps only a few gathers in flight, so a long row handled by one
+                                    // group is a long dependent chain: long rows are cut into items instead.
+constexpr int SPMM_ITEM_BLOCKS = 1184;  // blocks that walk the item list (grid-stride)
 constexpr int SPMM_SEG = 512;    // entries per item (one block: 8 lane groups x 64 entries for 32-lane groups)
 
 // acc += sum over entries [e_lo, e_hi) of val[e] * X[col[e], :] for the chunks owned by this lane.
@@ -196,8 +200,8 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
     if ((int)blockIdx.x >= light_blocks) {
         // ---- heavy item: SPMM_SEG consecutive entries of a hub row, one contiguous piece per lane group,
         // pieces added in group order (fixed), FP32 partial row written for the combine kernel
-        const int item = blockIdx.x - light_blocks;
-        if (item >= a.heavy.counts[1]) return;
+        const int n_items = a.heavy.counts[1];
+        for (int item = blockIdx.x - light_blocks; item < n_items; item += gridDim.x - light_blocks) {
         const int r = a.heavy.item_row[item];
         const int sidx = item - a.heavy.item_first[item];
         const int hb = a.rowptr[r] + sidx * SPMM_SEG, he = min(a.rowptr[r + 1], hb + SPMM_SEG);
@@ -219,6 +223,8 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
             for (int w = 0; w < NG; ++w) sum += s_part[w][j];
             a.heavy.partials[(size_t)item * a.F + j] = sum;
         }
+        __syncthreads();
+        }
         return;
     }
     const int row0 = blockIdx.x * ROWS;
@@ -234,7 +240,7 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
     float pre_val = 0.f;
     {
         const int eb = s_ptr[g], ee = s_ptr[g + 1];
-        if (eb + gl < ee && ee - eb <= SPMM_HEAVY) {
+        if (eb + gl < ee && ee - eb <= a.heavy.threshold) {
             pre_col = __ldg(a.col + eb + gl);
             pre_val = a.val ? __ldg(a.val + eb + gl) : 1.f;
         }
@@ -250,12 +256,12 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
             const int eb = s_ptr[lr + NG], ee = s_ptr[lr + NG + 1];
             pre_col = 0;
             pre_val = 0.f;
-            if (eb + gl < ee && ee - eb <= SPMM_HEAVY) {
+            if (eb + gl < ee && ee - eb <= a.heavy.threshold) {
                 pre_col = __ldg(a.col + eb + gl);
                 pre_val = a.val ? __ldg(a.val + eb + gl) : 1.f;
             }
         }
-        if (r < n_rows && e_end - e_begin <= SPMM_HEAVY) {
+        if (r < n_rows && e_end - e_begin <= a.heavy.threshold) {
 #pragma unroll
             for (int i = 0; i < NV; ++i)
 #pragma unroll
@@ -273,7 +279,7 @@ __global__ void spmm_heavy_plan_kernel(const int *__restrict__ rowptr, int n_row
     const int lim = n_rows_dev ? min(*n_rows_dev, n_rows) : n_rows;
     if (r >= lim) return;
     const int d = rowptr[r + 1] - rowptr[r];
-    if (d <= SPMM_HEAVY) return;
+    if (d <= hp.threshold) return;
     const int nseg = (d + SPMM_SEG - 1) / SPMM_SEG;
     const int i = atomicAdd(&hp.counts[0], 1);
     const int b = atomicAdd(&hp.counts[1], nseg);
@@ -330,10 +336,11 @@ template <typename T, int G, int NV, int RPG, int U, int MINB> static void spmm_
     if (items < 0) {  // plan unknown on the host: rebuild it on the device, size the grid by the upper bound
         cudaMemsetAsync(a.heavy.counts, 0, 2 * sizeof(int), ex.st);
         spmm_heavy_plan_kernel<<<(unsigned)ceil_div64(a.n_rows, 256), 256, 0, ex.st>>>(a.rowptr, a.n_rows, a.n_rows_dev, a.heavy);
-        items = a.nnz / SPMM_HEAVY;  // every heavy row has more than SPMM_HEAVY entries and at most deg / SPMM_HEAVY items
+        items = a.nnz / SPMM_HEAVY_MIN;  // a heavy row has more than SPMM_HEAVY_MIN entries and at most deg / SPMM_HEAVY_MIN items
         ex.launches += 1;
     }
-    spmm_csr_kernel<T, G, NV, RPG, U, MINB><<<(unsigned)(light_blocks + items), SPMM_THREADS, 0, ex.st>>>(a, light_blocks);
+    const int item_blocks = (int)std::min<int64_t>(items, SPMM_ITEM_BLOCKS);
+    spmm_csr_kernel<T, G, NV, RPG, U, MINB><<<(unsigned)(light_blocks + item_blocks), SPMM_THREADS, 0, ex.st>>>(a, light_blocks);
     ex.launches += 1;
     if (a.heavy.host_rows != 0) {
         const int64_t rows_bound = a.heavy.host_rows > 0 ? a.heavy.host_rows : std::max<int64_t>(1, items);
