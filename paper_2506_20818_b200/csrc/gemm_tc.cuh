@@ -339,17 +339,32 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
 // One CTA per SM.  CTA c owns the N slice (c mod n_slices) of width BN and walks the 128-row tiles
 // c / n_slices, c / n_slices + stride, ...  Its slice of Bt (BN x K BF16, at most 128 KiB) is loaded
 // once; only A tiles stream through a 4-stage ring.  Two accumulators in tensor memory let the
-// epilogue of tile i (4 warps: tcgen05.ld, bias, ReLU, BF16 stores) overlap the MMAs of tile i + 1.
+// epilogue of tile i overlap the MMAs of tile i + 1.  The epilogue (4 warps: tcgen05.ld, bias, ReLU,
+// BF16) writes 128-column halves of the tile into a swizzled shared-memory staging area that one
+// thread hands to TMA stores (full 128-byte rows instead of 16-byte pieces of 32 different rows per
+// store instruction; rows beyond M are clipped by the tensor map).
 //   warp 0: TMA producer (one lane)      warp 1: MMA issuer (one lane)      warps 2-5: epilogue
 // ---------------------------------------------------------------------------------------------
 constexpr int TCP_THREADS = 192;
 constexpr int TCP_STAGES = 4;
+constexpr int TCP_STAGE_OUT_BYTES = 2 * 16384;  // output staging: two boxes of 128 rows x 64 BF16 columns
+
+LP_DEVINL void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+}
+LP_DEVINL void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+LP_DEVINL void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+LP_DEVINL void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+LP_DEVINL void epilogue_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }  // the four epilogue warps only
 
 LP_DEVINL void mbar_arrive(uint32_t bar) { asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory"); }
 
 __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(const __grid_constant__ CUtensorMap mapA,
-                                                                              const __grid_constant__ CUtensorMap mapB, const TcGemmParams p)
+                                                                              const __grid_constant__ CUtensorMap mapB,
+                                                                              const __grid_constant__ CUtensorMap mapC, const TcGemmParams p)
 {
+    __shared__ float s_bias[256];
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[TCP_STAGES], bar_empty[TCP_STAGES], bar_w, bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_base_s;
@@ -363,6 +378,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
     uint8_t *smem_w = smem;
     uint8_t *smem_a = smem + (size_t)KB * w_sub_bytes;
     const uint32_t a_bytes = TC_BM * TC_BK * 2;
+    uint8_t *smem_out = smem_a + (size_t)TCP_STAGES * a_bytes;
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < 2 * BN) tmem_cols <<= 1;
 
@@ -389,11 +405,13 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
         fence_async_proxy();
         tma_prefetch_desc(&mapA);
         tma_prefetch_desc(&mapB);
+        tma_prefetch_desc(&mapC);
     }
     if (warp == 0) {
         __syncwarp();
         tmem_alloc(smem_u32(&tmem_base_s), tmem_cols);
     }
+    for (int j = threadIdx.x; j < BN; j += TCP_THREADS) s_bias[j] = p.bias ? p.bias[n0 + j] : 0.f;
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -461,30 +479,45 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
                 const int b = (int)(i & 1);
                 bool ready = mbar_wait(smem_u32(&bar_acc_full[b]), (uint32_t)((i >> 1) & 1));
                 if (!ready && lane == 0) { atomicExch(p.err, 3); *abort_flag = 1; }
-                ready = __all_sync(0xffffffffu, ready && *abort_flag == 0);
-                if (!ready) break;
+                if (!__all_sync(0xffffffffu, ready) && lane == 0) *abort_flag = 1;
+                epilogue_barrier();             // the four warps take the same decision: all continue or all leave
+                if (*abort_flag != 0) break;
                 tc_fence_after();
-                const int64_t row = (first_tile + i * stride) * TC_BM + q * 32 + lane;
+                const int m0 = (int)((first_tile + i * stride) * TC_BM);
+                const int row_t = q * 32 + lane;  // row inside the tile
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN);
-                for (int c0 = 0; c0 < BN; c0 += 32) {
-                    float v[32];
-                    tmem_ld_32x32(taddr + (uint32_t)c0, v);
-                    if (row < p.M) {
-                        if (p.bias) {
+                const bool store_thread = (warp == 2 && lane == 0);
+                for (int half = 0; half < BN; half += 128) {
+                    const int nbox = min(2, (BN - half) / 64);
+                    if (store_thread) tma_store_wait_read();  // the previous stores have read the staging area
+                    epilogue_barrier();
+                    for (int c0 = half; c0 < half + nbox * 64; c0 += 32) {
+                        float v[32];
+                        tmem_ld_32x32(taddr + (uint32_t)c0, v);
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) v[j] += __ldg(p.bias + n0 + c0 + j);
+                        for (int j = 0; j < 32; j += 4) {
+                            const float4 bb = *reinterpret_cast<const float4 *>(&s_bias[c0 + j]);
+                            v[j] += bb.x; v[j + 1] += bb.y; v[j + 2] += bb.z; v[j + 3] += bb.w;
                         }
                         if (p.relu) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
                         }
-                        bf16 *dst = p.C + row * p.ldc + n0 + c0;
+                        // 128-byte swizzle of the staging box: 16-byte chunk index XOR (row mod 8)
+                        uint8_t *box = smem_out + (size_t)((c0 - half) / 64) * 16384 + (size_t)row_t * 128;
+                        const int chunk0 = (c0 & 63) >> 3;
 #pragma unroll
-                        for (int j = 0; j < 32; j += 8) {
+                        for (int j = 0; j < 4; ++j) {
                             Vec16<bf16> o;
-                            o.from_float(v + j);
-                            o.store(dst + j);
+                            o.from_float(v + 8 * j);
+                            *reinterpret_cast<uint4 *>(box + (((chunk0 + j) ^ (row_t & 7)) << 4)) = o.v;
                         }
+                    }
+                    fence_async_proxy();  // generic-proxy writes -> visible to the TMA engine
+                    epilogue_barrier();
+                    if (store_thread) {
+                        for (int bx = 0; bx < nbox; ++bx) tma_store_2d(&mapC, smem_u32(smem_out + (size_t)bx * 16384), n0 + half + bx * 64, m0);
+                        tma_store_commit();
                     }
                 }
                 tc_fence_before();
@@ -493,6 +526,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
             }
         }
     }
+    if (warp == 2 && lane == 0) tma_store_wait_all();  // output tiles are in global memory before the CTA leaves
     __syncwarp();
     tc_fence_before();
     __syncthreads();
@@ -521,7 +555,7 @@ static bool tc_init(TcState &tc, std::string &err)
         return false;
     }
     cudaMemset(tc.err_word, 0, 256);
-    if (cudaFuncSetAttribute(tc_linear_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess ||
+    if (cudaFuncSetAttribute(tc_linear_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024 + 512) != cudaSuccess ||
         cudaFuncSetAttribute(tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess ||
         cudaFuncSetAttribute(tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) {
         err = "cannot raise the dynamic shared memory limit of the tensor-core GEMM";
@@ -586,7 +620,7 @@ static int tc_stages(int BN, int num_kb)
 
 // C[M, N] (BF16, leading dimension ldc) = act(A[M, K] * Bt[N, K]^T + bias); Bt is BF16, K contiguous.
 // Slice width for the persistent kernel: the largest multiple of 64 (at most 256, dividing N) whose
-// weight slice BN x K x 2 B fits 128 KiB beside the four 16 KiB A stages.  0 = does not fit.
+// weight slice BN x K x 2 B fits 128 KiB beside the four 16 KiB A stages and the 32 KiB output staging.  0 = does not fit.
 static int tc_persistent_bn(int N, int K)
 {
     for (int bn = 256; bn >= 64; bn -= 64)
@@ -614,6 +648,8 @@ static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const
         CUtensorMap mapA, mapB;
         if (!tc_make_map(tc, &mapA, A, M, K, lda, TC_BK, TC_BM, err)) return false;
         if (!tc_make_map(tc, &mapB, Bt, N, K, K, TC_BK, pbn, err)) return false;
+        CUtensorMap mapC;
+        if (!tc_make_map(tc, &mapC, C, M, N, ldc, 64, TC_BM, err)) return false;
         TcGemmParams p{};
         p.M = M; p.N = N; p.K = K; p.BN = pbn; p.stages = TCP_STAGES;
         p.bias = bias; p.relu = relu ? 1 : 0; p.C = C; p.ldc = ldc; p.out_f32 = nullptr; p.err = tc.err_word;
@@ -621,8 +657,8 @@ static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const
         const int64_t m_tiles = ceil_div64(M, TC_BM);
         int64_t ctas = std::min<int64_t>((int64_t)tc_sm_count(), m_tiles * n_slices);
         ctas = std::max<int64_t>(n_slices, ctas / n_slices * n_slices);  // a whole number of CTAs per slice
-        const size_t smem = (size_t)(K / TC_BK) * pbn * 128 + (size_t)TCP_STAGES * TC_BM * TC_BK * 2 + 1024;
-        tc_linear_persistent_kernel<<<(unsigned)ctas, TCP_THREADS, smem, ex.st>>>(mapA, mapB, p);
+        const size_t smem = (size_t)(K / TC_BK) * pbn * 128 + (size_t)TCP_STAGES * TC_BM * TC_BK * 2 + TCP_STAGE_OUT_BYTES + 1024;
+        tc_linear_persistent_kernel<<<(unsigned)ctas, TCP_THREADS, smem, ex.st>>>(mapA, mapB, mapC, p);
         ex.launches += 1;
         return true;
     }
