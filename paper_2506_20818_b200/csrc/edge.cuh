@@ -53,6 +53,19 @@ edge_score_bce_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const 
     if (j < B) {
         int u = clamp_id(pos_src[j], n_ids), v = clamp_id(pos_dst[j], n_ids);
         if (idmap) { u = idmap[u]; v = idmap[v]; }
+        // the first negative row is requested together with h_u and h_v, and each further negative row while
+        // the previous one is reduced: one memory round trip per edge instead of two dependent ones
+        Vec16<T> nxt[NV];
+        int vn_nxt = 0;
+        if (k > 0) {
+            vn_nxt = clamp_id(neg_dst[j * k], n_ids);
+            if (idmap) vn_nxt = idmap[vn_nxt];
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const int ch = lane + i * 32;
+                if (ch < nchunks) nxt[i].load(H + (size_t)vn_nxt * ldh + ch * VN);
+            }
+        }
         float hu[NV][VN];
         float dot = 0.f;
 #pragma unroll
@@ -79,8 +92,18 @@ edge_score_bce_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const 
         }
         for (int kk = 0; kk < k; ++kk) {
             const int64_t t = j * k + kk;
-            int vn = clamp_id(neg_dst[t], n_ids);
-            if (idmap) vn = idmap[vn];
+            Vec16<T> cur[NV];
+#pragma unroll
+            for (int i = 0; i < NV; ++i) cur[i] = nxt[i];
+            if (kk + 1 < k) {
+                vn_nxt = clamp_id(neg_dst[t + 1], n_ids);
+                if (idmap) vn_nxt = idmap[vn_nxt];
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    const int ch = lane + i * 32;
+                    if (ch < nchunks) nxt[i].load(H + (size_t)vn_nxt * ldh + ch * VN);
+                }
+            }
             const bool own_src = neg_src != nullptr;
             int un = u;
             if (own_src) { un = clamp_id(neg_src[t], n_ids); if (idmap) un = idmap[un]; }
@@ -89,10 +112,8 @@ edge_score_bce_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const 
             for (int i = 0; i < NV; ++i) {
                 const int ch = lane + i * 32;
                 if (ch < nchunks) {
-                    Vec16<T> b;
-                    b.load(H + (size_t)vn * ldh + ch * VN);
                     float fb[VN];
-                    b.to_float(fb);
+                    cur[i].to_float(fb);
                     if (own_src && un != u) {
                         Vec16<T> a;
                         a.load(H + (size_t)un * ldh + ch * VN);

@@ -146,7 +146,20 @@ __global__ void __launch_bounds__(256) colsum_partial_kernel(const T *__restrict
 #pragma unroll
     for (int j = 0; j < VN; ++j) acc[j] = 0.f;
     if (rl < lanes_r) {
-        for (int64_t r = r0 + rl; r < r1; r += lanes_r) {
+        int64_t r = r0 + rl;
+        for (; r + 3 * (int64_t)lanes_r < r1; r += 4 * (int64_t)lanes_r) {  // four loads in flight, added in row order
+            Vec16<T> v[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) v[q].load(dZ + (r + q * (int64_t)lanes_r) * ldz + c * VN);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                float f[VN];
+                v[q].to_float(f);
+#pragma unroll
+                for (int j = 0; j < VN; ++j) acc[j] += f[j];
+            }
+        }
+        for (; r < r1; r += lanes_r) {
             Vec16<T> v;
             v.load(dZ + r * ldz + c * VN);
             float f[VN];
