@@ -108,6 +108,25 @@ lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const int64_t *rowp
  * entry that transposed entry t came from).  Any of the three may be NULL. */
 lp_status lp_get_structure(lp_ctx *ctx, int64_t *colptr, int32_t *rowidx, int64_t *perm);
 
+/* ---- graph sparsification, Algorithm 1 (sparsification block), Theorems 1 and 2 -------- */
+
+/* Sparsify the loaded graph (which must be symmetric: every stored entry has its mirror) by the
+ * degree-based approximation of effective resistance: L = floor(alpha * |E|) draws with
+ * replacement (|E| = nnz / 2 undirected edges), edge {u, v} drawn with probability
+ * p = (1/d_u + 1/d_v) / n' (n' = number of non-isolated nodes), each draw adding 1 / (L p) to the
+ * weight of its edge; edges never drawn are removed, all nodes are kept.  Draw l picks
+ * u = nz[floor(x0 n' / 2^32)] among the non-isolated nodes (ascending) and then the neighbour at
+ * position floor(x1 d_u / 2^32) of u's row, with (x0, x1) = words 0 and 1 of
+ * philox(counter = (lo32(l), hi32(l), 0, 4), key = (lo32(seed), hi32(seed))).
+ * The result stays inside the context until the next lp_sparsify / lp_load_graph; *nnz_out receives
+ * its number of stored entries (both orientations).  Synchronises.
+ * LP_EINVAL when alpha is not in (0, 1e6] or the graph is not symmetric. */
+lp_status lp_sparsify(lp_ctx *ctx, double alpha, uint64_t seed, int64_t *nnz_out);
+
+/* Copy the last sparsified graph out (DEVICE arrays): rowptr[n+1] int64, col[nnz_out] int32
+ * ascending inside a row, w[nnz_out] float32 accumulated weights.  Any pointer may be NULL. */
+lp_status lp_get_sparsified(lp_ctx *ctx, int64_t *rowptr, int32_t *col, float *w);
+
 /* ---- model -------------------------------------------------------------------------- */
 
 /* Fix the encoder (Eq. 1) and allocate the activation workspace.  `max_batch` bounds the

@@ -27,7 +27,7 @@ EXPORTS = [
     "lp_param_count", "lp_set_candidates", "lp_sample_negatives", "lp_train_step", "lp_train_step_host",
     "lp_adam_step", "lp_score", "lp_get_embeddings", "lp_get_output_gradient", "lp_get_block",
     "lp_get_stats", "lp_op_aggregate", "lp_op_linear", "lp_op_weight_grad", "lp_profile_begin", "lp_profile_end",
-    "lp_weight_grad_static",
+    "lp_weight_grad_static", "lp_sparsify", "lp_get_sparsified",
 ]
 
 PROF_CATEGORIES = ["agg_fwd", "agg_bwd", "gemm_fwd", "gemm_dgrad", "gemm_wgrad", "score", "incidence", "scatter",
@@ -140,6 +140,19 @@ class Context:
         perm = t.empty(max(self.nnz, 1), dtype=t.int64, device=dev)
         self._ck(self.lib.lp_get_structure(self.h, _ptr(colptr), _ptr(rowidx), _ptr(perm)))
         return colptr, rowidx[: self.nnz], perm[: self.nnz]
+
+    def sparsify(self, alpha: float, seed: int):
+        """Algorithm 1's sparsification of the loaded (symmetric) graph: (rowptr int64, col int32, w float32) on the device."""
+        t = self._torch
+        dev = f"cuda:{self.device}"
+        nnz = C.c_int64()
+        self._ck(self.lib.lp_sparsify(self.h, C.c_double(alpha), C.c_uint64(seed), C.byref(nnz)))
+        k = int(nnz.value)
+        rowptr = t.empty(self.n + 1, dtype=t.int64, device=dev)
+        col = t.empty(max(k, 1), dtype=t.int32, device=dev)
+        w = t.empty(max(k, 1), dtype=t.float32, device=dev)
+        self._ck(self.lib.lp_get_sparsified(self.h, _ptr(rowptr), _ptr(col), _ptr(w)))
+        return rowptr, col[:k], w[:k]
 
     # ---- model
     def set_model(self, arch: str, dims: Sequence[int], prec: str = "fp32", fanout: Optional[Sequence[int]] = None,

@@ -12,6 +12,7 @@
 #include "sampler.cuh"
 #include "edge.cuh"
 #include "optim.cuh"
+#include "sparsify.cuh"
 
 // ----------------------------------------------------------------------------------------------
 // context
@@ -44,8 +45,12 @@ struct lp_ctx {
     int device = 0;
     Exec ex;
     std::string err;
-    std::vector<void *> graph_allocs, model_allocs;
-    int64_t graph_bytes = 0, model_bytes = 0;
+    std::vector<void *> graph_allocs, model_allocs, sparse_allocs;
+    int64_t graph_bytes = 0, model_bytes = 0, sparse_bytes = 0;
+    int64_t *sp_ptr = nullptr;  // last sparsified graph
+    int *sp_col = nullptr;
+    float *sp_w = nullptr;
+    int64_t sp_nnz = -1;
 
     // graph
     bool loaded = false;
@@ -259,6 +264,7 @@ extern "C" void lp_destroy(lp_ctx *ctx)
     cudaSetDevice(ctx->device);
     cudaStreamSynchronize(ctx->ex.st);
     free_list(ctx->model_allocs);
+    free_list(ctx->sparse_allocs);
     free_list(ctx->graph_allocs);
     tc_destroy(ctx->tc);
     for (cudaEvent_t e : ctx->ex.prof.pool) cudaEventDestroy(e);
@@ -292,6 +298,8 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
     CK(cudaSetDevice(ctx->device));
     CK(cudaStreamSynchronize(ctx->ex.st));
     drop_model(ctx);
+    free_list(ctx->sparse_allocs);
+    ctx->sp_nnz = -1;
     free_list(ctx->graph_allocs);
     ctx->graph_bytes = 0;
     ctx->loaded = false;
@@ -428,6 +436,81 @@ extern "C" lp_status lp_set_candidates(lp_ctx *ctx, const int32_t *cand, int64_t
         return fail(ctx, LP_EINVAL, "lp_set_candidates: candidate id outside [0, n)");
     }
     ctx->n_cand = n_cand;
+    return LP_OK;
+}
+
+// ----------------------------------------------------------------------------------------------
+// sparsification
+// ----------------------------------------------------------------------------------------------
+static lp_status sync_counts(lp_ctx *ctx, const int *dev_a, const int *dev_b, int *out_a, int *out_b);
+
+#define SALLOC(ptr, count) CK(dev_alloc(ctx, ctx->sparse_allocs, ctx->sparse_bytes, &(ptr), (count)))
+
+extern "C" lp_status lp_sparsify(lp_ctx *ctx, double alpha, uint64_t seed, int64_t *nnz_out)
+{
+    if (!ctx || !nnz_out) return LP_EINVAL;
+    if (!ctx->loaded) return fail(ctx, LP_ESTATE, "lp_sparsify: no graph loaded");
+    if (!(alpha > 0.0) || alpha > 1e6) return fail(ctx, LP_EINVAL, "lp_sparsify: alpha must be in (0, 1e6]");
+    CK(cudaSetDevice(ctx->device));
+    cudaStream_t st = ctx->ex.st;
+    CK(cudaStreamSynchronize(st));
+    free_list(ctx->sparse_allocs);
+    ctx->sparse_bytes = 0;
+    ctx->sp_nnz = -1;
+    const int n = ctx->n;
+    const int64_t nnz = ctx->nnz;
+    const int64_t L = (int64_t)std::floor(alpha * (double)(nnz / 2));
+    int *flags = nullptr, *pos = nullptr, *nz = nullptr, *hits = nullptr, *scan_tmp = nullptr;
+    const int64_t m = std::max<int64_t>(n, nnz) + 2;
+    SALLOC(flags, m);
+    SALLOC(pos, m);
+    SALLOC(nz, n + 1);
+    SALLOC(hits, nnz + 1);
+    SALLOC(scan_tmp, ceil_div64(m, SCAN_TILE) + 2);
+    SALLOC(ctx->sp_ptr, n + 1);
+    // non-isolated nodes, ascending
+    sp_nonisolated_kernel<<<nblk(n), 256, 0, st>>>(ctx->rowptr, n, flags);
+    exclusive_scan_i32(ctx->ex, flags, n, pos, pos + n, scan_tmp);
+    sp_compact_kernel<<<nblk(n), 256, 0, st>>>(ctx->rowptr, pos, n, nz);
+    int n_nz = 0, dummy = 0;
+    lp_status s = sync_counts(ctx, pos + n, nullptr, &n_nz, &dummy);
+    if (s != LP_OK) return s;
+    CK(cudaMemsetAsync(hits, 0, sizeof(int) * (size_t)(nnz + 1), st));
+    CK(cudaMemsetAsync(ctx->err_flag, 0, sizeof(int), st));
+    if (L > 0 && n_nz > 0)
+        sp_draw_kernel<<<nblk(L), 256, 0, st>>>(ctx->rowptr, ctx->col, nz, (uint32_t)n_nz, make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)), L, hits,
+                                                ctx->err_flag);
+    // kept entries -> positions; pos has nnz + 1 slots so that pos[rowptr[n]] is the total
+    sp_keep_flags_kernel<<<nblk(nnz + 1), 256, 0, st>>>(hits, nnz + 1, flags);
+    exclusive_scan_i32(ctx->ex, flags, nnz + 1, pos, nullptr, scan_tmp);
+    int kept = 0, bad = 0;
+    s = sync_counts(ctx, pos + nnz, ctx->err_flag, &kept, &bad);
+    if (s != LP_OK) return s;
+    if (bad) {
+        cudaMemsetAsync(ctx->err_flag, 0, sizeof(int), st);
+        return fail(ctx, LP_EINVAL, "lp_sparsify: the loaded graph is not symmetric (a drawn entry has no mirror)");
+    }
+    SALLOC(ctx->sp_col, kept);
+    SALLOC(ctx->sp_w, kept);
+    sp_emit_kernel<<<nblk(n + 1), 256, 0, st>>>(ctx->rowptr, ctx->col, hits, pos, n, (double)n_nz, (double)std::max<int64_t>(L, 1), ctx->sp_ptr, ctx->sp_col,
+                                                ctx->sp_w);
+    ctx->ex.launches += 5;
+    CK(cudaStreamSynchronize(st));
+    CK_LAUNCH();
+    ctx->sp_nnz = kept;
+    *nnz_out = kept;
+    return LP_OK;
+}
+
+extern "C" lp_status lp_get_sparsified(lp_ctx *ctx, int64_t *rowptr, int32_t *col, float *w)
+{
+    if (!ctx) return LP_EINVAL;
+    if (ctx->sp_nnz < 0) return fail(ctx, LP_ESTATE, "lp_get_sparsified: call lp_sparsify first");
+    CK(cudaSetDevice(ctx->device));
+    cudaStream_t st = ctx->ex.st;
+    if (rowptr) CK(cudaMemcpyAsync(rowptr, ctx->sp_ptr, sizeof(int64_t) * ((size_t)ctx->n + 1), cudaMemcpyDeviceToDevice, st));
+    if (col && ctx->sp_nnz > 0) CK(cudaMemcpyAsync(col, ctx->sp_col, sizeof(int) * (size_t)ctx->sp_nnz, cudaMemcpyDeviceToDevice, st));
+    if (w && ctx->sp_nnz > 0) CK(cudaMemcpyAsync(w, ctx->sp_w, sizeof(float) * (size_t)ctx->sp_nnz, cudaMemcpyDeviceToDevice, st));
     return LP_OK;
 }
 

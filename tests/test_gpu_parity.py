@@ -521,3 +521,33 @@ def test_host_buffer_step_matches_device_step(pkg):
     ctx.adam_step(p2, m2, v2, grads, 1)
     assert torch.equal(p, p2)
     ctx.close()
+
+
+# ------------------------------------------------------------------------------------------ sparsifier (Algorithm 1)
+@pytest.mark.parametrize("alpha", [0.05, 0.2, 1.5])
+def test_sparsifier_matches_oracle(pkg, alpha):
+    g = wl.chung_lu(30000, 16.0, 2.1, seed=8)
+    assert (np.diff(g.rowptr) == 0).any()  # isolated nodes are skipped by the node draw
+    ctx = make_ctx(pkg, g, wl.node_features(g.n, 8, 0))
+    seed = (3 << 40) + 17
+    rp, col, w = ctx.sparsify(alpha, seed)
+    torch.cuda.synchronize()
+    orp, ocol, ow = oracle.sparsified_graph(g.n, g.rowptr, g.col, alpha, seed)
+    assert np.array_equal(rp.cpu().numpy(), orp) and np.array_equal(col.cpu().numpy(), ocol)  # structure bit-exact
+    assert np.max(np.abs(w.cpu().numpy() - ow) / ow) < 1e-6
+    # the sparsified graph can be loaded and trained on (it is symmetric with ascending columns)
+    ctx2 = pkg.Context(0)
+    ctx2.load_graph(g.n, rp.cpu().numpy(), col.cpu().numpy(), w.cpu().numpy(), wl.node_features(g.n, 8, 0))
+    ctx2.close()
+    ctx.close()
+
+
+def test_sparsifier_rejects_directed_graph(pkg):
+    g = wl.citation_directed(2000, 20000, 2.2, seed=1)
+    ctx = make_ctx(pkg, g, wl.node_features(g.n, 8, 0))
+    with pytest.raises(pkg.LpError) as ei:
+        ctx.sparsify(0.5, 1)
+    assert ei.value.status == -1
+    with pytest.raises(pkg.LpError):
+        ctx.sparsify(0.0, 1)
+    ctx.close()
