@@ -179,6 +179,7 @@ def main():
     import torch
     import paper_2506_20818_b200 as pkg
     from paper_2506_20818_b200 import build as lpbuild
+    from paper_2506_20818_b200.dp import batch_for, sync_gradients
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (no CPU fall-back exists)")
@@ -216,16 +217,15 @@ def main():
 
     def one_step(i, t_adam):
         # data-parallel over batches: rank r takes batches r, r + world, ...
-        b = (i * world + rank) % nb
+        b = batch_for(i, rank, world, nb)
         lo = b * B
         su, sv = pu[lo:lo + B], pv[lo:lo + B]
         ctx._ck(lib.lp_sample_negatives(ctx.h, C.c_uint64(SEED), C.c_uint64(i), C.c_int32(K_NEG), C.c_int32(0), C.c_void_p(su.data_ptr()),
                                         C.c_int64(B), C.c_int64(lo), None, C.c_void_p(neg.data_ptr())))
         ctx.train_step(p, su, sv, None, neg, K_NEG, loss, grads, seed=SEED, step=i)
-        if world > 1:
-            with torch.cuda.stream(stream):
-                dist.all_reduce(grads)  # gradient synchronisation of Algorithm 1 (sum; 1/p folded into the update)
-        ctx.adam_step(p, m, v, grads, t_adam, grad_scale=1.0 / world)
+        with torch.cuda.stream(stream):
+            scale = sync_gradients(grads, world, dist)  # gradient synchronisation of Algorithm 1 (sum; 1/p folded into the update)
+        ctx.adam_step(p, m, v, grads, t_adam, grad_scale=scale)
 
     # ---- warm-up
     with torch.cuda.stream(stream):
@@ -304,7 +304,7 @@ def main():
         t_base = args.warmup + args.steps + 100
 
         def host_step(i):
-            b = (i * world + rank) % nb
+            b = batch_for(i, rank, world, nb)
             lo = b * B
             ctx.train_step_host(p, hu[lo:lo + B], hv[lo:lo + B], K_NEG, seed=SEED, step=i, edge_index_base=lo, adam_m=m, adam_v=v,
                                 adam_t=i + 1, loss_host=loss_h)
