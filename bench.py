@@ -32,9 +32,11 @@ UNIT = "edges/s"
 K_NEG = 1
 SEED = 1234
 
-# DRAM traffic of the dominant kernel (aggregation, F = 256 BF16 on the benchmark graph) from one ncu
-# capture, bytes per launch, valid only for the kernel source it was taken with.
-NCU_TRAFFIC = {"spmm_sha1": None, "bytes_per_launch": None}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the aggregation launches of one step on the
+# benchmark workload, from one ncu capture (profiles/spmm_csr_bf16_config2.md): layer-1 forward 134.7 MB,
+# layer-2 forward 433.4 MB, adjoint 733.7 MB -> mean per timed launch.  Valid only for the kernel source it
+# was taken with (sha1 of csrc/spmm.cuh); reported as null otherwise.
+NCU_TRAFFIC = {"spmm_sha1": "d7a11d4a7910cc49bfe26c8fcf5c5d400edfec16", "bytes_per_launch": (134.7e6 + 433.4e6 + 733.7e6) / 3.0}
 
 
 def measured_peaks():
