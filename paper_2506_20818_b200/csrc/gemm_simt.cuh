@@ -147,12 +147,12 @@ __global__ void __launch_bounds__(256) colsum_partial_kernel(const T *__restrict
     for (int j = 0; j < VN; ++j) acc[j] = 0.f;
     if (rl < lanes_r) {
         int64_t r = r0 + rl;
-        for (; r + 3 * (int64_t)lanes_r < r1; r += 4 * (int64_t)lanes_r) {  // four loads in flight, added in row order
-            Vec16<T> v[4];
+        for (; r + 7 * (int64_t)lanes_r < r1; r += 8 * (int64_t)lanes_r) {  // eight loads in flight, added in row order
+            Vec16<T> v[8];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) v[q].load(dZ + (r + q * (int64_t)lanes_r) * ldz + c * VN);
+            for (int q = 0; q < 8; ++q) v[q].load(dZ + (r + q * (int64_t)lanes_r) * ldz + c * VN);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
+            for (int q = 0; q < 8; ++q) {
                 float f[VN];
                 v[q].to_float(f);
 #pragma unroll
@@ -178,7 +178,30 @@ __global__ void __launch_bounds__(256) colsum_partial_kernel(const T *__restrict
     }
 }
 
-constexpr int CS_MAX_SPLITS = 296;
+// dst[j] = (accumulate ? dst[j] : 0) + sum_z partials[z][j] for a SHORT vector (count <= a few hundred) and many
+// splits: 32 columns per block, eight groups each add a contiguous range of splits in order, then the
+// eight group sums are added in group order (a fixed tree, so the result is reproducible).
+__global__ void __launch_bounds__(256) reduce_partials_short_kernel(const float *__restrict__ partials, int count, int splits, float *__restrict__ dst,
+                                                                    int accumulate)
+{
+    __shared__ float sh[8][32];
+    const int c = blockIdx.x * 32 + (threadIdx.x & 31), g = threadIdx.x >> 5;
+    const int per = (splits + 7) / 8;
+    const int z0 = g * per, z1 = min(splits, z0 + per);
+    float s = 0.f;
+    if (c < count)
+        for (int z = z0; z < z1; ++z) s += __ldg(partials + (int64_t)z * count + c);
+    sh[g][threadIdx.x & 31] = s;
+    __syncthreads();
+    if (g == 0 && c < count) {
+        float t = 0.f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) t += sh[q][threadIdx.x];
+        dst[c] = accumulate ? dst[c] + t : t;
+    }
+}
+
+constexpr int CS_MAX_SPLITS = 592;
 static int colsum_splits(int64_t rows) { return (int)std::max<int64_t>(1, std::min<int64_t>(CS_MAX_SPLITS, ceil_div64(rows, 64))); }
 
 template <typename T>
@@ -187,6 +210,6 @@ static void colsum(Exec &ex, const T *dZ, int64_t rows, int N, int64_t ldz, floa
     const int splits = colsum_splits(rows);
     const int64_t rpb = ceil_div64(rows > 0 ? rows : 1, splits);
     colsum_partial_kernel<T><<<splits, 256, 0, ex.st>>>(dZ, rows, N, ldz, rpb, partials);
-    reduce_partials_kernel<<<(unsigned)ceil_div64(N, 256), 256, 0, ex.st>>>(partials, N, splits, out, accumulate);
+    reduce_partials_short_kernel<<<(unsigned)ceil_div64(N, 32), 256, 0, ex.st>>>(partials, N, splits, out, accumulate);
     ex.launches += 2;
 }
