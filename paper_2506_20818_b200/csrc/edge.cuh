@@ -195,16 +195,14 @@ edge_score_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const int 
     if (lane == 0) scores[e] = dot;
 }
 
-// Incidence keys of the scored edges.  Edge slots: positives 0..B-1, negatives B..B+B*k-1.
-// Slot e contributes (node = src_e, other = dst_e) at 2e and (node = dst_e, other = src_e) at 2e+1.
-__global__ void incidence_keys_kernel(int n_ids, const int *__restrict__ idmap, const int *__restrict__ pos_src, const int *__restrict__ pos_dst, int64_t B,
-                                      const int *__restrict__ neg_src, const int *__restrict__ neg_dst, int k, uint32_t *__restrict__ keys,
-                                      uint32_t *__restrict__ vals, int *__restrict__ other, int *__restrict__ counts)
+// Incidence lists of the scored edges, grouped by node: dL/dH^(K)[v] = sum over incident edges of g_e * h_other.
+// Edge slots: positives 0..B-1, negatives B..B+B*k-1; slot e contributes (node src_e, other dst_e) and
+// (node dst_e, other src_e).  Counts and slot claims use integer atomics, so the ORDER of a node's entries
+// is not reproducible; the gather that consumes the lists therefore sums exactly (64-bit fixed point),
+// which makes its result independent of that order and reproducible bit for bit.
+LP_DEVINL void incidence_endpoints(int n_ids, const int *idmap, const int *pos_src, const int *pos_dst, int64_t B, const int *neg_src,
+                                   const int *neg_dst, int k, int64_t e, int &s, int &d)
 {
-    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int64_t E = B * (1 + k);
-    if (e >= E) return;
-    int s, d;
     if (e < B) {
         s = pos_src[e];
         d = pos_dst[e];
@@ -216,25 +214,34 @@ __global__ void incidence_keys_kernel(int n_ids, const int *__restrict__ idmap, 
     s = clamp_id(s, n_ids);
     d = clamp_id(d, n_ids);
     if (idmap) { s = idmap[s]; d = idmap[d]; }
-    keys[2 * e] = (uint32_t)s;
-    keys[2 * e + 1] = (uint32_t)d;
-    vals[2 * e] = (uint32_t)(2 * e);
-    vals[2 * e + 1] = (uint32_t)(2 * e + 1);
-    other[2 * e] = d;
-    other[2 * e + 1] = s;
+}
+
+__global__ void incidence_count_kernel(int n_ids, const int *__restrict__ idmap, const int *__restrict__ pos_src, const int *__restrict__ pos_dst,
+                                       int64_t B, const int *__restrict__ neg_src, const int *__restrict__ neg_dst, int k, int *__restrict__ counts)
+{
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= B * (1 + k)) return;
+    int s, d;
+    incidence_endpoints(n_ids, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, e, s, d);
     atomicAdd(&counts[s], 1);
     atomicAdd(&counts[d], 1);
 }
 
-// after the stable sort by node: column (= the other endpoint) and coefficient (= g of the edge)
-__global__ void incidence_fill_kernel(const uint32_t *__restrict__ sorted_slots, int64_t m, const int *__restrict__ other, int64_t B,
-                                      const float *__restrict__ g_pos, const float *__restrict__ g_neg, int *__restrict__ inc_col,
-                                      float *__restrict__ inc_val)
+// cursor[v] starts at the offset of node v's list and is advanced by every claim
+__global__ void incidence_fill_kernel(int n_ids, const int *__restrict__ idmap, const int *__restrict__ pos_src, const int *__restrict__ pos_dst,
+                                      int64_t B, const int *__restrict__ neg_src, const int *__restrict__ neg_dst, int k,
+                                      const float *__restrict__ g_pos, const float *__restrict__ g_neg, int *__restrict__ cursor,
+                                      int *__restrict__ inc_col, float *__restrict__ inc_val)
 {
-    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= m) return;
-    const uint32_t slot = sorted_slots[t];
-    const int64_t e = slot >> 1;
-    inc_col[t] = other[slot];
-    inc_val[t] = e < B ? g_pos[e] : g_neg[e - B];
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= B * (1 + k)) return;
+    int s, d;
+    incidence_endpoints(n_ids, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, e, s, d);
+    const float g = e < B ? g_pos[e] : g_neg[e - B];
+    const int ps = atomicAdd(&cursor[s], 1);
+    inc_col[ps] = d;
+    inc_val[ps] = g;
+    const int pd = atomicAdd(&cursor[d], 1);
+    inc_col[pd] = s;
+    inc_val[pd] = g;
 }

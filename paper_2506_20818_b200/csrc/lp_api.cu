@@ -83,8 +83,8 @@ struct lp_ctx {
     float *partials = nullptr;          // split-K / column-sum partials
     int64_t partials_floats = 0;
     float *g_pos = nullptr, *g_neg = nullptr, *loss_partials = nullptr;
-    uint32_t *inc_keys = nullptr, *inc_slots = nullptr;
-    int *inc_other = nullptr, *inc_ptr = nullptr, *inc_col = nullptr;
+    int *inc_cursor = nullptr, *inc_ptr = nullptr, *inc_col = nullptr;
+    float *inc_partials = nullptr;      // 64-bit item partials of the exact gather over the incidence lists
     float *inc_val = nullptr;
     SortScratch sort;                   // sized for the largest per-step sort
     TransposeScratch tsp;
@@ -636,9 +636,8 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
     MALLOC(ctx->g_pos, max_batch);
     MALLOC(ctx->g_neg, max_batch * std::max<int64_t>(max_k, 1));
     MALLOC(ctx->loss_partials, ceil_div64(max_batch, EDGE_THREADS / 32) + 1);
-    MALLOC(ctx->inc_keys, 2 * E);
-    MALLOC(ctx->inc_slots, 2 * E);
-    MALLOC(ctx->inc_other, 2 * E);
+    MALLOC(ctx->inc_cursor, cap_rows[0] + 1);
+    MALLOC(ctx->inc_partials, (2 * E / SPMM_HEAVY_MIN + 2) * 2 * (int64_t)d->dims[K]);
     MALLOC(ctx->inc_col, 2 * E);
     MALLOC(ctx->inc_val, 2 * E);
     MALLOC(ctx->inc_ptr, cap_rows[0] + 1);
@@ -1004,13 +1003,14 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     delete pscore;
     ctx->ex.launches += 2;
 
-    // incidence lists of the scored edges, grouped by node (stable sort => fixed summation order)
-    ProfScope *pinc = new ProfScope(ctx->ex, LP_PROF_INCIDENCE, (double)E * 2.0 * 40.0);
+    // incidence lists of the scored edges, grouped by node (slots claimed with integer atomics)
+    ProfScope *pinc = new ProfScope(ctx->ex, LP_PROF_INCIDENCE, (double)E * 2.0 * 24.0);
     CK(cudaMemsetAsync(ctx->inc_ptr, 0, sizeof(int) * ((size_t)rows_out + 1), st));
-    incidence_keys_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->inc_keys, ctx->inc_slots, ctx->inc_other, ctx->inc_ptr);
+    incidence_count_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->inc_ptr);
     exclusive_scan_i32(ctx->ex, ctx->inc_ptr, rows_out, ctx->inc_ptr, ctx->inc_ptr + rows_out, ctx->scan_tmp);
-    const bool sorted_in_place = radix_sort_pairs(ctx->ex, ctx->inc_keys, ctx->inc_slots, 2 * E, bits_for(rows_out), ctx->sort);
-    incidence_fill_kernel<<<nblk(2 * E), 256, 0, st>>>(sorted_in_place ? ctx->inc_slots : ctx->sort.vals_alt, 2 * E, ctx->inc_other, B, ctx->g_pos, ctx->g_neg, ctx->inc_col, ctx->inc_val);
+    CK(cudaMemcpyAsync(ctx->inc_cursor, ctx->inc_ptr, sizeof(int) * (size_t)rows_out, cudaMemcpyDeviceToDevice, st));
+    incidence_fill_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->g_pos, ctx->g_neg, ctx->inc_cursor, ctx->inc_col,
+                                                   ctx->inc_val);
     ctx->ex.launches += 2;
     delete pinc;
 
@@ -1020,6 +1020,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     {
         SpmmArgs<T> a;
         a.heavy = ctx->plan_dyn;
+        a.heavy.partials = ctx->inc_partials;
         a.nnz = 2 * E;
         a.n_rows = rows_out;
         a.rowptr = ctx->inc_ptr;
@@ -1031,7 +1032,8 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         a.Y = dZ;
         a.ldy = D;
         ProfScope prof(ctx->ex, LP_PROF_SCATTER, spmm_bytes(a, 2 * E), 4.0 * E * D);
-        if (rows_out > 0 && !spmm_launch<T>(ctx->ex, a)) return fail(ctx, LP_EUNSUPPORTED, "embedding width not supported");
+        // the order of a node's entries is not reproducible, so the sum is taken exactly (64-bit fixed point)
+        if (rows_out > 0 && !spmm_launch<T, long long>(ctx->ex, a)) return fail(ctx, LP_EUNSUPPORTED, "embedding width not supported");
     }
     ctx->have_grad = true;
 

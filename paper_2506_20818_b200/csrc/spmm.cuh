@@ -59,6 +59,19 @@ template <typename T> struct SpmmArgs {
 };
 
 constexpr int SPMM_THREADS = 256;
+
+// Accumulator of one output element.  float: FMA in entry order (the result depends on the order of a
+// row's entries, which is fixed for every structure built by a stable sort).  long long: each product
+// is rounded once to a multiple of 2^-40 and added as an integer -- exact and therefore independent of
+// the order of the entries; used for lists whose entry order is not reproducible (slots claimed with
+// integer atomics), so that their sums still are, bit for bit.
+constexpr float SPMM_EXACT_SCALE = 1099511627776.f;  // 2^40: products up to 2^23 in magnitude, resolution 9.1e-13
+template <typename ACC> LP_DEVINL void acc_add(ACC &a, float w, float f);
+template <> LP_DEVINL void acc_add<float>(float &a, float w, float f) { a = fmaf(w, f, a); }
+template <> LP_DEVINL void acc_add<long long>(long long &a, float w, float f) { a += __float2ll_rn(w * f * SPMM_EXACT_SCALE); }
+template <typename ACC> LP_DEVINL float acc_value(ACC a);
+template <> LP_DEVINL float acc_value<float>(float a) { return a; }
+template <> LP_DEVINL float acc_value<long long>(long long a) { return (float)((double)a * (1.0 / 1099511627776.0)); }
 constexpr int SPMM_HEAVY_MIN = 64;  // smallest heavy-row threshold a plan may use (bounds the item count by nnz / 64).
                                     // A lane group keeps only a few gathers in flight, so a long row handled by one
                                     // group is a long dependent chain: long rows are cut into items instead.
@@ -68,8 +81,8 @@ constexpr int SPMM_SEG = 512;    // entries per item (one block: 8 lane groups x
 // acc += sum over entries [e_lo, e_hi) of val[e] * X[col[e], :] for the chunks owned by this lane.
 // The group loads up to G (col, val) pairs at once and broadcasts them; U source rows are gathered
 // before any is consumed, so each lane keeps U * NV 16-byte loads in flight.
-template <typename T, int G, int NV, int U>
-LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl, unsigned gmask, int nchunks, float (&acc)[NV][Vec16<T>::N],
+template <typename T, int G, int NV, int U, typename ACC>
+LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl, unsigned gmask, int nchunks, ACC (&acc)[NV][Vec16<T>::N],
                                 bool have_first = false, int first_col = 0, float first_val = 0.f)
 {
     constexpr int VN = Vec16<T>::N;
@@ -112,7 +125,7 @@ LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl,
                         float f[VN];
                         v[q][i].to_float(f);
 #pragma unroll
-                        for (int t = 0; t < VN; ++t) acc[i][t] = fmaf(w[q], f[t], acc[i][t]);
+                        for (int t = 0; t < VN; ++t) acc_add<ACC>(acc[i][t], w[q], f[t]);
                     }
                 }
         }
@@ -128,7 +141,7 @@ LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl,
                     float f[VN];
                     v.to_float(f);
 #pragma unroll
-                    for (int t = 0; t < VN; ++t) acc[i][t] = fmaf(w, f[t], acc[i][t]);
+                    for (int t = 0; t < VN; ++t) acc_add<ACC>(acc[i][t], w, f[t]);
                 }
             }
         }
@@ -136,8 +149,8 @@ LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl,
 }
 
 // scale, extra term, ReLU mask, store, optional copy of the self row
-template <typename T, int G, int NV>
-LP_DEVINL void spmm_epilogue(const SpmmArgs<T> &a, int r, int gl, int nchunks, const float (&acc)[NV][Vec16<T>::N])
+template <typename T, int G, int NV, typename ACC>
+LP_DEVINL void spmm_epilogue(const SpmmArgs<T> &a, int r, int gl, int nchunks, const ACC (&acc)[NV][Vec16<T>::N])
 {
     constexpr int VN = Vec16<T>::N;
     const float scale = a.row_scale ? __ldg(a.row_scale + r) : 1.f;
@@ -154,7 +167,7 @@ LP_DEVINL void spmm_epilogue(const SpmmArgs<T> &a, int r, int gl, int nchunks, c
         if (ch >= nchunks) continue;
         float o[VN];
 #pragma unroll
-        for (int t = 0; t < VN; ++t) o[t] = acc[i][t] * scale;
+        for (int t = 0; t < VN; ++t) o[t] = acc_value<ACC>(acc[i][t]) * scale;
         if (irow >= 0) {
             Vec16<T> v;
             v.load(a.init + (size_t)irow * a.ldinit + ch * VN);
@@ -182,14 +195,14 @@ LP_DEVINL void spmm_epilogue(const SpmmArgs<T> &a, int r, int gl, int nchunks, c
     }
 }
 
-template <typename T, int G, int NV, int RPG, int U, int MINB>
+template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC>
 __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const SpmmArgs<T> a, const int light_blocks)
 {
     constexpr int VN = Vec16<T>::N;
     constexpr int NG = SPMM_THREADS / G;  // lane groups per block
     constexpr int ROWS = NG * RPG;        // rows per block: every group walks RPG rows
     __shared__ int s_ptr[ROWS + 1];
-    __shared__ __align__(16) float s_part[NG][G * NV * VN];  // partial sums of an item, one per group
+    __shared__ __align__(16) ACC s_part[NG][G * NV * VN];  // partial sums of an item, one per group
     const int n_rows = a.n_rows_dev ? min(*a.n_rows_dev, a.n_rows) : a.n_rows;
     const int g = threadIdx.x / G;   // group inside the block
     const int gl = threadIdx.x % G;  // lane inside the group
@@ -207,21 +220,21 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
         const int hb = a.rowptr[r] + sidx * SPMM_SEG, he = min(a.rowptr[r + 1], hb + SPMM_SEG);
         const int piece = ((he - hb + NG - 1) / NG + G - 1) / G * G;
         const int lo = min(he, hb + g * piece), hi = min(he, lo + piece);
-        float hacc[NV][VN];
+        ACC hacc[NV][VN];
 #pragma unroll
         for (int q = 0; q < NV; ++q)
 #pragma unroll
-            for (int j = 0; j < VN; ++j) hacc[q][j] = 0.f;
-        spmm_accumulate<T, G, NV, U>(a, lo, hi, gl, gmask, nchunks, hacc);
+            for (int j = 0; j < VN; ++j) hacc[q][j] = ACC(0);
+        spmm_accumulate<T, G, NV, U, ACC>(a, lo, hi, gl, gmask, nchunks, hacc);
 #pragma unroll
         for (int q = 0; q < NV; ++q)
 #pragma unroll
             for (int t = 0; t < VN; ++t) s_part[g][(gl + q * G) * VN + t] = hacc[q][t];
         __syncthreads();
         for (int j = threadIdx.x; j < a.F; j += SPMM_THREADS) {
-            float sum = 0.f;
+            ACC sum = ACC(0);
             for (int w = 0; w < NG; ++w) sum += s_part[w][j];
-            a.heavy.partials[(size_t)item * a.F + j] = sum;
+            reinterpret_cast<ACC *>(a.heavy.partials)[(size_t)item * a.F + j] = sum;
         }
         __syncthreads();
         }
@@ -232,7 +245,7 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
     for (int i = threadIdx.x; i <= ROWS; i += SPMM_THREADS) s_ptr[i] = a.rowptr[min(row0 + i, n_rows)];
     __syncthreads();
 
-    float acc[NV][VN];
+    ACC acc[NV][VN];
     // ---- light rows: group g walks rows g, g + NG, g + 2 NG, ... of the block.  The (column, coefficient)
     // pairs of the next row are fetched before the current row's gathers are consumed, so a group has
     // its index loads and its feature gathers in flight at the same time.
@@ -265,9 +278,9 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
 #pragma unroll
             for (int i = 0; i < NV; ++i)
 #pragma unroll
-                for (int j = 0; j < VN; ++j) acc[i][j] = 0.f;
-            spmm_accumulate<T, G, NV, U>(a, e_begin, e_end, gl, gmask, nchunks, acc, true, cur_col, cur_val);
-            spmm_epilogue<T, G, NV>(a, r, gl, nchunks, acc);
+                for (int j = 0; j < VN; ++j) acc[i][j] = ACC(0);
+            spmm_accumulate<T, G, NV, U, ACC>(a, e_begin, e_end, gl, gmask, nchunks, acc, true, cur_col, cur_val);
+            spmm_epilogue<T, G, NV, ACC>(a, r, gl, nchunks, acc);
         }
     }
 }
@@ -292,7 +305,7 @@ __global__ void spmm_heavy_plan_kernel(const int *__restrict__ rowptr, int n_row
 }
 
 // adds the items of every heavy row in item order (fixed) and applies the epilogue; one lane group per row
-template <typename T, int G, int NV>
+template <typename T, int G, int NV, typename ACC>
 __global__ void __launch_bounds__(SPMM_THREADS) spmm_heavy_combine_kernel(const SpmmArgs<T> a)
 {
     constexpr int VN = Vec16<T>::N;
@@ -303,30 +316,27 @@ __global__ void __launch_bounds__(SPMM_THREADS) spmm_heavy_combine_kernel(const 
     for (int i = blockIdx.x * NG + g; i < count; i += gridDim.x * NG) {
         const int r = a.heavy.rows[i], b = a.heavy.base[i];
         const int nseg = (a.rowptr[r + 1] - a.rowptr[r] + SPMM_SEG - 1) / SPMM_SEG;
-        float acc[NV][VN];
+        ACC acc[NV][VN];
 #pragma unroll
         for (int q = 0; q < NV; ++q)
 #pragma unroll
-            for (int t = 0; t < VN; ++t) acc[q][t] = 0.f;
+            for (int t = 0; t < VN; ++t) acc[q][t] = ACC(0);
         for (int s = 0; s < nseg; ++s) {
-            const float *p = a.heavy.partials + (size_t)(b + s) * a.F;
+            const ACC *p = reinterpret_cast<const ACC *>(a.heavy.partials) + (size_t)(b + s) * a.F;
 #pragma unroll
             for (int q = 0; q < NV; ++q) {
                 const int ch = gl + q * G;
                 if (ch < nchunks) {
 #pragma unroll
-                    for (int t = 0; t < VN; t += 4) {
-                        const float4 v = *reinterpret_cast<const float4 *>(p + ch * VN + t);
-                        acc[q][t] += v.x; acc[q][t + 1] += v.y; acc[q][t + 2] += v.z; acc[q][t + 3] += v.w;
-                    }
+                    for (int t = 0; t < VN; ++t) acc[q][t] += p[ch * VN + t];
                 }
             }
         }
-        spmm_epilogue<T, G, NV>(a, r, gl, nchunks, acc);
+        spmm_epilogue<T, G, NV, ACC>(a, r, gl, nchunks, acc);
     }
 }
 
-template <typename T, int G, int NV, int RPG, int U, int MINB> static void spmm_launch_cfg(Exec &ex, const SpmmArgs<T> &a)
+template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC> static void spmm_launch_cfg(Exec &ex, const SpmmArgs<T> &a)
 {
     constexpr int ROWS = (SPMM_THREADS / G) * RPG;
     constexpr int NG = SPMM_THREADS / G;
@@ -340,36 +350,42 @@ template <typename T, int G, int NV, int RPG, int U, int MINB> static void spmm_
         ex.launches += 1;
     }
     const int item_blocks = (int)std::min<int64_t>(items, SPMM_ITEM_BLOCKS);
-    spmm_csr_kernel<T, G, NV, RPG, U, MINB><<<(unsigned)(light_blocks + item_blocks), SPMM_THREADS, 0, ex.st>>>(a, light_blocks);
+    spmm_csr_kernel<T, G, NV, RPG, U, MINB, ACC><<<(unsigned)(light_blocks + item_blocks), SPMM_THREADS, 0, ex.st>>>(a, light_blocks);
     ex.launches += 1;
     if (a.heavy.host_rows != 0) {
         const int64_t rows_bound = a.heavy.host_rows > 0 ? a.heavy.host_rows : std::max<int64_t>(1, items);
         const unsigned grid = (unsigned)std::min<int64_t>(592, ceil_div64(rows_bound, NG));
-        spmm_heavy_combine_kernel<T, G, NV><<<grid, SPMM_THREADS, 0, ex.st>>>(a);
+        spmm_heavy_combine_kernel<T, G, NV, ACC><<<grid, SPMM_THREADS, 0, ex.st>>>(a);
         ex.launches += 1;
     }
 }
 
 // Launch shape (measured on a 200k-node power-law graph, BF16): with one 16-byte vector per lane, 4 gathers in
 // flight per lane at 48 registers (5 blocks per SM) beat 8 gathers at 80 registers (3 blocks) by about 10 %.
-template <typename T, int G, int NV> static void spmm_launch_gn(Exec &ex, const SpmmArgs<T> &a)
+template <typename T, int G, int NV, typename ACC> static void spmm_launch_gn(Exec &ex, const SpmmArgs<T> &a)
 {
-    if constexpr (NV == 1) spmm_launch_cfg<T, G, NV, 8, 4, 5>(ex, a);
-    else if constexpr (NV == 2) spmm_launch_cfg<T, G, NV, 8, 4, 2>(ex, a);
-    else spmm_launch_cfg<T, G, NV, 8, 2, 2>(ex, a);
+    constexpr bool EXACT = sizeof(ACC) == 8;  // 64-bit accumulators need twice the registers
+    if constexpr (NV == 1) spmm_launch_cfg<T, G, NV, 8, 4, EXACT ? 3 : 5, ACC>(ex, a);
+    else if constexpr (NV == 2) spmm_launch_cfg<T, G, NV, 8, EXACT ? 2 : 4, 2, ACC>(ex, a);
+    else spmm_launch_cfg<T, G, NV, 8, 2, EXACT ? 1 : 2, ACC>(ex, a);
 }
 
-// F must be a multiple of the 16-byte vector width and at most 32 * 4 vectors wide.
-template <typename T> static bool spmm_launch(Exec &ex, const SpmmArgs<T> &a)
+// F must be a multiple of the 16-byte vector width and at most 32 * 4 vectors wide.  ACC = float sums a
+// row's entries in their stored order; ACC = long long sums exactly (order-free), for lists whose entry
+// order is not reproducible.  The item partials then hold 8 bytes per element.
+template <typename T, typename ACC = float> static bool spmm_launch(Exec &ex, const SpmmArgs<T> &a)
 {
     constexpr int VN = Vec16<T>::N;
     if (a.F <= 0 || a.F % VN != 0 || !a.heavy.counts || !a.heavy.partials) return false;
     const int chunks = a.F / VN;
-    if (chunks <= 8) spmm_launch_gn<T, 8, 1>(ex, a);
-    else if (chunks <= 16) spmm_launch_gn<T, 16, 1>(ex, a);
-    else if (chunks <= 32) spmm_launch_gn<T, 32, 1>(ex, a);
-    else if (chunks <= 64) spmm_launch_gn<T, 32, 2>(ex, a);
-    else if (chunks <= 128) spmm_launch_gn<T, 32, 4>(ex, a);
-    else return false;
+    if (chunks <= 8) spmm_launch_gn<T, 8, 1, ACC>(ex, a);
+    else if (chunks <= 16) spmm_launch_gn<T, 16, 1, ACC>(ex, a);
+    else if (chunks <= 32) spmm_launch_gn<T, 32, 1, ACC>(ex, a);
+    else if (chunks <= 64) spmm_launch_gn<T, 32, 2, ACC>(ex, a);
+    else if (chunks <= 128) {
+        // 64-bit partials of 1024 BF16 columns would not fit the static shared memory; widths stop at 512 anyway
+        if constexpr (sizeof(ACC) == 8 && sizeof(T) == 2) return false;
+        else spmm_launch_gn<T, 32, 4, ACC>(ex, a);
+    } else return false;
     return true;
 }
