@@ -551,3 +551,28 @@ def test_sparsifier_rejects_directed_graph(pkg):
     with pytest.raises(pkg.LpError):
         ctx.sparsify(0.0, 1)
     ctx.close()
+
+
+def test_step_on_a_caller_stream_matches_default_stream(pkg):
+    g, X, params, pos, cfg = wl.make_config("c2_chunglu_sage2", scale=0.02)
+    dims = cfg["dims"]
+    u, v = pos[0][:3000].copy(), pos[1][:3000].copy()
+    results = []
+    for stream in (None, torch.cuda.Stream(device=DEV)):
+        ctx = pkg.Context(0, stream=stream)
+        cm = torch.cuda.stream(stream) if stream is not None else torch.cuda.stream(torch.cuda.current_stream())
+        with cm:
+            ctx.load_graph(g.n, g.rowptr, g.col, g.w, X)
+            ctx.set_model("sage", dims, prec="bf16", max_batch=len(u), max_k=1)
+            du, dv, p = t32(u), t32(v), t32(params)
+            _, nd = ctx.sample_negatives(3, 1, 1, du)
+            loss = torch.zeros(1, device=DEV)
+            grads = torch.zeros(ctx.n_params, device=DEV)
+            if stream is not None:
+                stream.wait_stream(torch.cuda.default_stream())
+            ctx.train_step(p, du, dv, None, nd, 1, loss, grads)
+            (stream or torch.cuda.current_stream()).synchronize()
+        results.append((loss.clone(), grads.clone(), nd.clone()))
+        ctx.close()
+    assert torch.equal(results[0][2], results[1][2])
+    assert torch.equal(results[0][0], results[1][0]) and torch.equal(results[0][1], results[1][1])
