@@ -148,6 +148,7 @@ def main():
     ap.add_argument("--cpu-baseline-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--cache-input-agg", action="store_true", help="reuse the weight-independent first-layer aggregation across steps (not the default, not the headline)")
     ap.add_argument("--breakdown", action="store_true", help="print a per-category time breakdown to stderr")
     args = ap.parse_args()
 
@@ -205,7 +206,7 @@ def main():
     with torch.cuda.stream(stream):
         ctx = pkg.Context(local_rank, stream=stream)
         ctx.load_graph(g.n, g.rowptr, g.col, g.w, X)
-        ctx.set_model("sage", dims, prec="bf16", max_batch=B, max_k=K_NEG)
+        ctx.set_model("sage", dims, prec="bf16", max_batch=B, max_k=K_NEG, cache_input_aggregation=args.cache_input_agg)
         pu = torch.from_numpy(pos[0]).to(dev)
         pv = torch.from_numpy(pos[1]).to(dev)
         p = torch.from_numpy(params).to(dev)
@@ -349,7 +350,7 @@ def main():
                 "data": "synthetic",
                 "config": {"workload": WORKLOAD, "graph": "Chung-Lu power law, exponent 2.1, mean degree 20", "nodes": g.n, "entries": g.nnz,
                            "model": "2-layer GraphSAGE-mean 128-256-256, dot-product predictor", "batch_pos": B, "neg_per_pos": K_NEG,
-                           "scale": args.scale, "parallelism": f"dp{world}" if world > 1 else "single GPU",
+                           "scale": args.scale, "cache_input_aggregation": bool(args.cache_input_agg), "parallelism": f"dp{world}" if world > 1 else "single GPU",
                            "l2": "no flush: the step streams ~1 GB of activations per pass, several times the 126 MB L2"},
                 "clocks": clocks, "gpu_launches": int(launches), "loss_last": loss_value, "roofline": roofline, "cpu_baseline": cpu,
                 "e2e": e2e, "breakdown_us_per_step": breakdown}

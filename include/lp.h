@@ -64,6 +64,9 @@ typedef struct {
     int32_t fanout[LP_MAX_LAYERS];
     int32_t reject_edges;            /* negatives: redraw self pairs and true edges */
     int32_t max_attempts;            /* draws per negative when reject_edges (1..255) */
+    int32_t cache_input_aggregation; /* full-graph models only: AGG(X) of the first layer does not depend on the
+                                        weights, so compute it in the first step and reuse it afterwards (off = 0:
+                                        every step recomputes it) */
 } lp_model_desc;
 
 typedef struct {

@@ -43,7 +43,7 @@ class LpError(RuntimeError):
 class ModelDesc(C.Structure):
     _fields_ = [("arch", C.c_int32), ("n_layers", C.c_int32), ("dims", C.c_int32 * (LP_MAX_LAYERS + 1)),
                 ("prec", C.c_int32), ("fanout", C.c_int32 * LP_MAX_LAYERS), ("reject_edges", C.c_int32),
-                ("max_attempts", C.c_int32)]
+                ("max_attempts", C.c_int32), ("cache_input_aggregation", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -156,7 +156,8 @@ class Context:
 
     # ---- model
     def set_model(self, arch: str, dims: Sequence[int], prec: str = "fp32", fanout: Optional[Sequence[int]] = None,
-                  reject_edges: bool = True, max_attempts: int = 8, max_batch: int = 65536, max_k: int = 1):
+                  reject_edges: bool = True, max_attempts: int = 8, max_batch: int = 65536, max_k: int = 1,
+                  cache_input_aggregation: bool = False):
         d = ModelDesc()
         d.arch = LP_GCN if arch == "gcn" else LP_SAGE_MEAN
         d.n_layers = len(dims) - 1
@@ -167,6 +168,7 @@ class Context:
             d.fanout[i] = int(v)
         d.reject_edges = int(bool(reject_edges))
         d.max_attempts = int(max_attempts)
+        d.cache_input_aggregation = int(bool(cache_input_aggregation))
         self._ck(self.lib.lp_set_model(self.h, C.byref(d), C.c_int64(max_batch), C.c_int32(max_k)))
         np_ = C.c_int64()
         self._ck(self.lib.lp_param_count(self.h, C.byref(np_)))

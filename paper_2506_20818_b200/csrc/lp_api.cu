@@ -99,6 +99,7 @@ struct lp_ctx {
     float *d_loss_tmp = nullptr, *d_grads_tmp = nullptr;
     int rows_out = 0;                   // rows of H^(K) in the last forward
     bool have_forward = false, have_grad = false;
+    bool input_agg_valid = false;       // cached AGG(X) of layer 1 is present (cache_input_aggregation)
     int64_t last_exhausted = 0;
     TcState tc;                         // tensor-core GEMM state (descriptor encoder, device error word)
 };
@@ -280,6 +281,7 @@ static void drop_model(lp_ctx *ctx)
     ctx->model_bytes = 0;
     ctx->model_set = false;
     ctx->have_forward = ctx->have_grad = false;
+    ctx->input_agg_valid = false;
     for (auto &l : ctx->layer) l = LayerBuf();
     for (auto &h : ctx->hop) h = HopBlock();
 }
@@ -546,6 +548,7 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
         for (int h = 0; h < d->n_layers; ++h)
             if (d->fanout[h] == 0) return fail(ctx, LP_EINVAL, "lp_set_model: fanouts must be all zero or all positive");
         if (d->arch != LP_SAGE_MEAN) return fail(ctx, LP_EUNSUPPORTED, "lp_set_model: neighbour sampling is implemented for SAGE-mean only");
+        if (d->cache_input_aggregation) return fail(ctx, LP_EINVAL, "lp_set_model: cache_input_aggregation needs a full-graph model (sampled neighbourhoods change every step)");
     }
     if (max_batch <= 0 || max_k < 0 || max_k > 255) return fail(ctx, LP_EINVAL, "lp_set_model: max_batch must be positive, max_k in [0, 255]");
     if (d->reject_edges && (d->max_attempts < 1 || d->max_attempts > 255)) return fail(ctx, LP_EINVAL, "lp_set_model: max_attempts must be in [1, 255]");
@@ -952,9 +955,11 @@ template <typename T> static lp_status forward_impl(lp_ctx *ctx, const float *pa
             }
             if (k == K - 1) { out = tptr<T>(ctx->HK); ldo = L.Fo; } else { out = tptr<T>(L.Hout); ldo = L.Fo; }
         }
-        {
+        const bool cached = (k == 0 && !ctx->sampled && ctx->desc.cache_input_aggregation && ctx->input_agg_valid);
+        if (!cached) {
             ProfScope prof(ctx->ex, LP_PROF_AGG_FWD, spmm_bytes(a, ctx->sampled ? ctx->hop[K - k].entries : ctx->nnz), 2.0 * (ctx->sampled ? ctx->hop[K - k].entries : ctx->nnz) * L.Fi);
             if (rows > 0 && !spmm_launch<T>(ctx->ex, a)) return fail(ctx, LP_EUNSUPPORTED, "aggregation width not supported");
+            if (k == 0 && !ctx->sampled) ctx->input_agg_valid = true;  // AGG(X) stays in layer 1's operand buffer
         }
         lp_status s = layer_linear<T>(ctx, rows, L, params, out, ldo, k < K - 1);
         if (s != LP_OK) return s;

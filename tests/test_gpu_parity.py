@@ -576,3 +576,30 @@ def test_step_on_a_caller_stream_matches_default_stream(pkg):
         ctx.close()
     assert torch.equal(results[0][2], results[1][2])
     assert torch.equal(results[0][0], results[1][0]) and torch.equal(results[0][1], results[1][1])
+
+
+@pytest.mark.parametrize("arch", ["gcn", "sage"])
+def test_cached_input_aggregation_gives_identical_steps(pkg, arch):
+    g, X, params, pos, cfg = wl.make_config("c3_coauthor_gcn3", scale=0.02)
+    dims = [128, 64, 64]
+    params = wl.glorot_params(arch, dims, 1, 0.05)
+    u, v = pos[0][:2000].copy(), pos[1][:2000].copy()
+    out = []
+    for cache in (False, True):
+        ctx = make_ctx(pkg, g, X)
+        ctx.set_model(arch, dims, prec="bf16", max_batch=len(u), max_k=1, cache_input_aggregation=cache)
+        du, dv, p = t32(u), t32(v), t32(params)
+        m, vv = torch.zeros_like(p), torch.zeros_like(p)
+        loss, grads = torch.zeros(1, device=DEV), torch.zeros(ctx.n_params, device=DEV)
+        for step in range(3):  # the weights change between steps; the cached aggregate must not
+            _, nd = ctx.sample_negatives(9, step, 1, du)
+            ctx.train_step(p, du, dv, None, nd, 1, loss, grads)
+            ctx.adam_step(p, m, vv, grads, step + 1)
+        torch.cuda.synchronize()
+        out.append((loss.clone(), grads.clone(), p.clone()))
+        ctx.close()
+    assert all(torch.equal(a, b) for a, b in zip(out[0], out[1]))
+    ctx = make_ctx(pkg, wl.citation_directed(500, 4000, 2.2, seed=1), wl.node_features(500, 64, 0))
+    with pytest.raises(pkg.LpError):
+        ctx.set_model("sage", [64, 64], fanout=[3], max_batch=8, cache_input_aggregation=True)
+    ctx.close()
