@@ -81,7 +81,7 @@ constexpr int SPMM_SEG = 512;    // entries per item (one block: 8 lane groups x
 // acc += sum over entries [e_lo, e_hi) of val[e] * X[col[e], :] for the chunks owned by this lane.
 // The group loads up to G (col, val) pairs at once and broadcasts them; U source rows are gathered
 // before any is consumed, so each lane keeps U * NV 16-byte loads in flight.
-template <typename T, int G, int NV, int U, typename ACC>
+template <typename T, int G, int NV, int U, typename ACC, bool HAS_VAL>
 LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl, unsigned gmask, int nchunks, ACC (&acc)[NV][Vec16<T>::N],
                                 bool have_first = false, int first_col = 0, float first_val = 0.f)
 {
@@ -95,7 +95,7 @@ LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl,
             my_val = 0.f;
             if (my_e < e_hi) {
                 my_col = __ldg(a.col + my_e);
-                my_val = a.val ? __ldg(a.val + my_e) : 1.f;
+                if (HAS_VAL) my_val = __ldg(a.val + my_e);
             }
         }
         const int cnt = min(G, e_hi - e0);
@@ -107,7 +107,7 @@ LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl,
 #pragma unroll
             for (int q = 0; q < U; ++q) {
                 c[q] = __shfl_sync(gmask, my_col, j + q, G);
-                w[q] = __shfl_sync(gmask, my_val, j + q, G);
+                w[q] = HAS_VAL ? __shfl_sync(gmask, my_val, j + q, G) : 1.f;
             }
 #pragma unroll
             for (int q = 0; q < U; ++q)
@@ -131,7 +131,7 @@ LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl,
         }
         for (; j < cnt; ++j) {
             const int c = __shfl_sync(gmask, my_col, j, G);
-            const float w = __shfl_sync(gmask, my_val, j, G);
+            const float w = HAS_VAL ? __shfl_sync(gmask, my_val, j, G) : 1.f;
 #pragma unroll
             for (int i = 0; i < NV; ++i) {
                 const int ch = gl + i * G;
@@ -195,7 +195,7 @@ LP_DEVINL void spmm_epilogue(const SpmmArgs<T> &a, int r, int gl, int nchunks, c
     }
 }
 
-template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC>
+template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC, bool HAS_VAL>
 __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const SpmmArgs<T> a, const int light_blocks)
 {
     constexpr int VN = Vec16<T>::N;
@@ -225,7 +225,7 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
         for (int q = 0; q < NV; ++q)
 #pragma unroll
             for (int j = 0; j < VN; ++j) hacc[q][j] = ACC(0);
-        spmm_accumulate<T, G, NV, U, ACC>(a, lo, hi, gl, gmask, nchunks, hacc);
+        spmm_accumulate<T, G, NV, U, ACC, HAS_VAL>(a, lo, hi, gl, gmask, nchunks, hacc);
 #pragma unroll
         for (int q = 0; q < NV; ++q)
 #pragma unroll
@@ -255,7 +255,7 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
         const int eb = s_ptr[g], ee = s_ptr[g + 1];
         if (eb + gl < ee && ee - eb <= a.heavy.threshold) {
             pre_col = __ldg(a.col + eb + gl);
-            pre_val = a.val ? __ldg(a.val + eb + gl) : 1.f;
+            pre_val = HAS_VAL ? __ldg(a.val + eb + gl) : 1.f;
         }
     }
 #pragma unroll 1
@@ -271,7 +271,7 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
             pre_val = 0.f;
             if (eb + gl < ee && ee - eb <= a.heavy.threshold) {
                 pre_col = __ldg(a.col + eb + gl);
-                pre_val = a.val ? __ldg(a.val + eb + gl) : 1.f;
+                pre_val = HAS_VAL ? __ldg(a.val + eb + gl) : 1.f;
             }
         }
         if (r < n_rows && e_end - e_begin <= a.heavy.threshold) {
@@ -279,7 +279,7 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
             for (int i = 0; i < NV; ++i)
 #pragma unroll
                 for (int j = 0; j < VN; ++j) acc[i][j] = ACC(0);
-            spmm_accumulate<T, G, NV, U, ACC>(a, e_begin, e_end, gl, gmask, nchunks, acc, true, cur_col, cur_val);
+            spmm_accumulate<T, G, NV, U, ACC, HAS_VAL>(a, e_begin, e_end, gl, gmask, nchunks, acc, true, cur_col, cur_val);
             spmm_epilogue<T, G, NV, ACC>(a, r, gl, nchunks, acc);
         }
     }
@@ -350,7 +350,8 @@ template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC> sta
         ex.launches += 1;
     }
     const int item_blocks = (int)std::min<int64_t>(items, SPMM_ITEM_BLOCKS);
-    spmm_csr_kernel<T, G, NV, RPG, U, MINB, ACC><<<(unsigned)(light_blocks + item_blocks), SPMM_THREADS, 0, ex.st>>>(a, light_blocks);
+    if (a.val) spmm_csr_kernel<T, G, NV, RPG, U, MINB, ACC, true><<<(unsigned)(light_blocks + item_blocks), SPMM_THREADS, 0, ex.st>>>(a, light_blocks);
+    else spmm_csr_kernel<T, G, NV, RPG, U, MINB, ACC, false><<<(unsigned)(light_blocks + item_blocks), SPMM_THREADS, 0, ex.st>>>(a, light_blocks);
     ex.launches += 1;
     if (a.heavy.host_rows != 0) {
         const int64_t rows_bound = a.heavy.host_rows > 0 ? a.heavy.host_rows : std::max<int64_t>(1, items);
