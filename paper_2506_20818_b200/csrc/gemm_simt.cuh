@@ -14,7 +14,8 @@ constexpr int SG_BM = 64, SG_BN = 64, SG_BK = 16, SG_THREADS = 256;
 template <typename TA, typename TB, typename TC, bool A_MCONTIG, bool B_NCONTIG>
 __global__ void __launch_bounds__(SG_THREADS)
 gemm_simt_kernel(int64_t M, int N, int64_t K, const TA *__restrict__ A, int64_t lda, const TB *__restrict__ B, int64_t ldb,
-                 TC *__restrict__ C, int64_t ldc, const float *__restrict__ bias, int relu, int64_t k_chunk, float *__restrict__ partials)
+                 TC *__restrict__ C, int64_t ldc, const float *__restrict__ bias, int relu, int64_t k_chunk, float *__restrict__ partials,
+                 const float *__restrict__ row_scale = nullptr, int scale_col0 = 0)
 {
     __shared__ __align__(16) float As[SG_BK][SG_BM + 4];
     __shared__ __align__(16) float Bs[SG_BK][SG_BN + 4];
@@ -77,6 +78,7 @@ gemm_simt_kernel(int64_t M, int N, int64_t K, const TA *__restrict__ A, int64_t 
             } else {
                 float v = acc[i][j] + (bias ? bias[n] : 0.f);
                 if (relu) v = fmaxf(v, 0.f);
+                if (row_scale && n >= scale_col0) v *= row_scale[m];  // per-row factor on the trailing columns
                 C[m * ldc + n] = from_f<TC>(v);
             }
         }
@@ -103,11 +105,11 @@ __global__ void reduce_partials_kernel(const float *__restrict__ partials, int64
 
 template <typename TA, typename TB, typename TC, bool A_MCONTIG, bool B_NCONTIG>
 static void gemm_simt(Exec &ex, int64_t M, int N, int64_t K, const TA *A, int64_t lda, const TB *B, int64_t ldb, TC *C, int64_t ldc,
-                      const float *bias, int relu)
+                      const float *bias, int relu, const float *row_scale = nullptr, int scale_col0 = 0)
 {
     if (M <= 0 || N <= 0) return;
     dim3 grid((unsigned)ceil_div64(M, SG_BM), (unsigned)ceil_div64(N, SG_BN), 1);
-    gemm_simt_kernel<TA, TB, TC, A_MCONTIG, B_NCONTIG><<<grid, SG_THREADS, 0, ex.st>>>(M, N, K, A, lda, B, ldb, C, ldc, bias, relu, K > 0 ? K : 1, nullptr);
+    gemm_simt_kernel<TA, TB, TC, A_MCONTIG, B_NCONTIG><<<grid, SG_THREADS, 0, ex.st>>>(M, N, K, A, lda, B, ldb, C, ldc, bias, relu, K > 0 ? K : 1, nullptr, row_scale, scale_col0);
     ex.launches += 1;
 }
 

@@ -164,6 +164,8 @@ struct TcGemmParams {
     int stages;
     const float *bias;  // [N] or null
     int relu;
+    const float *row_scale;  // [M] or null: columns >= scale_col0 of row m are multiplied by row_scale[m]
+    int scale_col0;          // (the 1 / |N(v)| of the mean adjoint, folded into the input-gradient transform)
     bf16 *C;            // output (BF16) when out_f32 == null
     int64_t ldc;
     float *out_f32;     // FP32 partial output [gridDim.z][M_tiles * 128, N] (weight gradient)
@@ -308,6 +310,11 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
                     if (p.relu) {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) v[i] = fmaxf(v[i], 0.f);
+                    }
+                    if (p.row_scale && n0 + c0 >= p.scale_col0) {
+                        const float rs = __ldg(p.row_scale + row);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] *= rs;
                     }
                     bf16 *dst = p.C + row * p.ldc + n0 + c0;
 #pragma unroll
@@ -487,6 +494,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
                 const int row_t = q * 32 + lane;  // row inside the tile
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN);
                 const bool store_thread = (warp == 2 && lane == 0);
+                const float rs = (p.row_scale && (int64_t)m0 + row_t < p.M) ? __ldg(p.row_scale + m0 + row_t) : 1.f;
                 for (int half = 0; half < BN; half += 128) {
                     const int nbox = min(2, (BN - half) / 64);
                     if (store_thread) tma_store_wait_read();  // the previous stores have read the staging area
@@ -502,6 +510,10 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
                         if (p.relu) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
+                        }
+                        if (p.row_scale && n0 + c0 >= p.scale_col0) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] *= rs;
                         }
                         // 128-byte swizzle of the staging box: 16-byte chunk index XOR (row mod 8)
                         uint8_t *box = smem_out + (size_t)((c0 - half) / 64) * 16384 + (size_t)row_t * 128;
@@ -641,7 +653,7 @@ static int tc_sm_count()
 }
 
 static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const bf16 *A, int64_t lda, const bf16 *Bt, const float *bias, bool relu,
-                           bf16 *C, int64_t ldc, std::string &err)
+                           bf16 *C, int64_t ldc, std::string &err, const float *row_scale = nullptr, int scale_col0 = 0)
 {
     const int pbn = tc_persistent_bn(N, K);
     if (pbn > 0 && M >= 4 * TC_BM) {
@@ -653,6 +665,7 @@ static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const
         TcGemmParams p{};
         p.M = M; p.N = N; p.K = K; p.BN = pbn; p.stages = TCP_STAGES;
         p.bias = bias; p.relu = relu ? 1 : 0; p.C = C; p.ldc = ldc; p.out_f32 = nullptr; p.err = tc.err_word;
+        p.row_scale = row_scale; p.scale_col0 = scale_col0;
         const int n_slices = N / pbn;
         const int64_t m_tiles = ceil_div64(M, TC_BM);
         int64_t ctas = std::min<int64_t>((int64_t)tc_sm_count(), m_tiles * n_slices);
@@ -670,6 +683,7 @@ static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const
     p.M = M; p.N = N; p.K = K; p.BN = BN;
     p.stages = tc_stages(BN, K / TC_BK);
     p.bias = bias; p.relu = relu ? 1 : 0; p.C = C; p.ldc = ldc; p.out_f32 = nullptr; p.rows = 0; p.rows_per_split = 0; p.err = tc.err_word;
+    p.row_scale = row_scale; p.scale_col0 = scale_col0;
     const size_t smem = (size_t)p.stages * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024;
     dim3 grid((unsigned)ceil_div64(M, TC_BM), (unsigned)(N / BN), 1);
     tc_gemm_kernel<false><<<grid, TC_THREADS, smem, ex.st>>>(mapA, mapB, p);
@@ -682,13 +696,13 @@ static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const
 //   w_is_kn = true : W is [K, N] row-major and the product is A * W        (forward)
 //   w_is_kn = false: W is [N, K] row-major and the product is A * W^T      (input gradient)
 static bool tc_linear(TcState &tc, Exec &ex, int64_t M, int N, int K, const bf16 *A, int lda, const float *W, bool w_is_kn, const float *bias,
-                      bool relu, bf16 *C, int ldc, std::string &err)
+                      bool relu, bf16 *C, int ldc, std::string &err, const float *row_scale = nullptr, int scale_col0 = 0)
 {
     const int total = K * N;
     if (w_is_kn) weights_to_bf16_kernel<<<(total + 255) / 256, 256, 0, ex.st>>>(W, K, N, tc.wbuf, nullptr);
     else convert_kernel<float, bf16><<<(total + 255) / 256, 256, 0, ex.st>>>(W, tc.wbuf, total);
     ex.launches += 1;
-    return tc_gemm_kmajor(tc, ex, M, N, K, A, lda, tc.wbuf, bias, relu, C, ldc, err);
+    return tc_gemm_kmajor(tc, ex, M, N, K, A, lda, tc.wbuf, bias, relu, C, ldc, err, row_scale, scale_col0);
 }
 
 // the same with a BF16 B operand given as [K, N] (b_is_nk = false) or [N, K] (b_is_nk = true)

@@ -29,7 +29,6 @@ struct HopBlock {  // sampled block of hop h (destinations F_{h-1}, sources F_h)
     int *blk_col_global = nullptr, *blk_col_local = nullptr, *blk_row = nullptr;  // [cap_entries]
     float *inv_deg = nullptr;     // 1 / sampled degree per destination     [cap_dst]
     int *colptr = nullptr, *rowidx = nullptr, *perm = nullptr;  // transposed block
-    float *valT = nullptr;
     int *self_idx = nullptr, *inv_self = nullptr;
 };
 
@@ -678,7 +677,6 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
                     MALLOC(hb.colptr, (int64_t)hb.cap_src + 1);
                     MALLOC(hb.rowidx, hb.cap_entries);
                     MALLOC(hb.perm, hb.cap_entries);
-                    MALLOC(hb.valT, hb.cap_entries);
                     MALLOC(hb.self_idx, hb.cap_dst);
                     MALLOC(hb.inv_self, hb.cap_src);
                 }
@@ -774,19 +772,23 @@ static lp_status layer_linear(lp_ctx *ctx, int64_t rows, const LayerBuf &L, cons
 }
 
 // dA[rows, Kin] = dZ[rows, Fo] * W^T
+// dA[rows, Kin] = dZ[rows, Fo] * W^T.  For SAGE-mean the right half of dA (the gradient of the mean) is
+// multiplied by row_scale = 1 / |N(v)| on the way out, so the adjoint aggregation needs no per-entry
+// coefficient: dH[u] = sum over v with u in N(v) of dA_mean[v] / |N(v)|.
 template <typename T>
-static lp_status layer_input_grad(lp_ctx *ctx, int64_t rows, const LayerBuf &L, const float *params, const T *dZ, T *dA)
+static lp_status layer_input_grad(lp_ctx *ctx, int64_t rows, const LayerBuf &L, const float *params, const T *dZ, T *dA, const float *row_scale,
+                                  int scale_col0)
 {
     if (rows <= 0) return LP_OK;
     ProfScope prof(ctx->ex, LP_PROF_GEMM_DGRAD, gemm_bytes((double)rows, L.Kin, L.Fo, sizeof(T), sizeof(T)), 2.0 * rows * L.Fo * L.Kin);
     if (sizeof(T) == 2 && tc_linear_supported(L.Fo, L.Kin)) {
         std::string err;
         if (!tc_linear(ctx->tc, ctx->ex, rows, L.Kin, L.Fo, (const bf16 *)dZ, L.Fo, params + L.off_w, /*w_is_kn=*/false, nullptr, false, (bf16 *)dA, L.Kin,
-                       err))
+                       err, row_scale, scale_col0))
             return fail(ctx, LP_ECUDA, "tensor-core GEMM: " + err);
         return LP_OK;
     }
-    gemm_simt<T, float, T, false, false>(ctx->ex, rows, L.Kin, L.Fo, dZ, L.Fo, params + L.off_w, L.Fo, dA, L.Kin, nullptr, 0);
+    gemm_simt<T, float, T, false, false>(ctx->ex, rows, L.Kin, L.Fo, dZ, L.Fo, params + L.off_w, L.Fo, dA, L.Kin, nullptr, 0, row_scale, scale_col0);
     return LP_OK;
 }
 
@@ -875,10 +877,6 @@ static lp_status build_blocks(lp_ctx *ctx, const int *pos_src, const int *pos_ds
                 ctx->ex.launches += 1;
             }
             transpose_csr(ctx->ex, hb.blk_ptr, hb.n_dst, hb.n_src, hb.blk_col_local, hb.entries, hb.colptr, hb.rowidx, hb.perm, ctx->tsp);
-            if (hb.entries > 0) {
-                gather_f32_kernel<<<nblk(hb.entries), 256, 0, st>>>(hb.inv_deg, hb.rowidx, hb.entries, hb.valT);
-                ctx->ex.launches += 1;
-            }
         }
     }
     CK_LAUNCH();
@@ -1050,7 +1048,8 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         if (s != LP_OK) return s;
         if (l == 0) break;
         T *dA = tptr<T>(ctx->dA);
-        s = layer_input_grad<T>(ctx, rows, L, params, dZ, dA);
+        const float *mean_scale = sage ? (ctx->sampled ? ctx->hop[K - l].inv_deg : ctx->inv_deg) : nullptr;
+        s = layer_input_grad<T>(ctx, rows, L, params, dZ, dA, mean_scale, L.Fi);
         if (s != LP_OK) return s;
         T *dZn = tptr<T>(ctx->dZ[cur ^ 1]);
         SpmmArgs<T> a;
@@ -1069,7 +1068,6 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
             a.rowptr = ctx->colptr;
             a.col = ctx->rowidx;
             if (sage) {
-                a.val = ctx->meanT_val;
                 a.X = dA + L.Fi;
                 a.ldx = L.Kin;
                 a.init = dA;
@@ -1091,7 +1089,6 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
             a.n_rows = hb.n_src;
             a.rowptr = hb.colptr;
             a.col = hb.rowidx;
-            a.val = hb.valT;
             a.X = dA + L.Fi;
             a.ldx = L.Kin;
             a.init = dA;
