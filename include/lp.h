@@ -130,6 +130,33 @@ lp_status lp_sparsify(lp_ctx *ctx, double alpha, uint64_t seed, int64_t *nnz_out
  * ascending inside a row, w[nnz_out] float32 accumulated weights.  Any pointer may be NULL. */
 lp_status lp_get_sparsified(lp_ctx *ctx, int64_t *rowptr, int32_t *col, float *w);
 
+/* ---- worker view, Section III (data sharing for negative sampling) ----------------------- */
+
+typedef struct {
+    int64_t own_entries;     /* stored entries of the worker's own rows                                   */
+    int64_t foreign_entries; /* stored entries of the other partitions' rows: the graph data shared with   */
+    int64_t foreign_rows;    /*   this worker, and the number of foreign rows that carry any               */
+    int64_t own_nodes;       /* |V^i|                                                                      */
+} lp_view_stats;
+
+/* Build the graph that worker `worker` trains on from the loaded (global) graph and a node -> partition
+ * assignment part[n] (DEVICE int32):
+ *   rows of the worker's own nodes: their list in the loaded graph -- every neighbour when
+ *     keep_cross_edges != 0 (the full-neighbour partitions of the method), else only neighbours in the
+ *     same partition (node-induced subgraph);
+ *   rows of other partitions' nodes, foreign_mode 0: empty (no data sharing, local negatives only);
+ *     1: their lists in the last lp_sparsify result (the method: sparsified subgraphs shared for global
+ *     negatives); 2: their full lists (complete data sharing).
+ * The four variants compared in the paper's ablation are (keep_cross, foreign_mode) = (1, 1), (1, 2),
+ * (1, 0) and (0, 0).  The result stays in the context; *nnz_out receives its entry count and *stats (may be
+ * NULL) the sizes from which the shared graph data volume follows.  Synchronises.
+ * LP_ESTATE when foreign_mode is 1 and lp_sparsify has not been called. */
+lp_status lp_worker_view(lp_ctx *ctx, const int32_t *part, int32_t worker, int32_t keep_cross_edges, int32_t foreign_mode, int64_t *nnz_out,
+                         lp_view_stats *stats);
+
+/* Copy the last worker view out (DEVICE arrays): rowptr[n+1] int64, col[nnz_out] int32 ascending per row. */
+lp_status lp_get_worker_view(lp_ctx *ctx, int64_t *rowptr, int32_t *col);
+
 /* ---- model -------------------------------------------------------------------------- */
 
 /* Fix the encoder (Eq. 1) and allocate the activation workspace.  `max_batch` bounds the

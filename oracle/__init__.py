@@ -23,6 +23,7 @@ from .sparse import (  # noqa: F401
     build_blocks,
     sparsify,
     sparsified_graph,
+    worker_view,
 )
 from .model import (  # noqa: F401
     split_params,

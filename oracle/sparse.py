@@ -168,3 +168,38 @@ def sparsified_graph(n: int, rowptr, col, alpha: float, seed: int):
     new_ptr = np.zeros(n + 1, dtype=np.int64)
     np.cumsum(counts, out=new_ptr[1:])
     return new_ptr, _i32(col)[keep].copy(), wsum[keep].astype(np.float32)
+
+
+def worker_view(n: int, rowptr, col, part, worker: int, keep_cross_edges: bool = True, foreign_mode: int = 1, sparsified=None):
+    """Graph that one worker trains on (Section III; Algorithm 1's use of G^i and the shared sparsified
+    subgraphs): own rows (part[v] == worker) keep every neighbour (full-neighbour partition) or only
+    neighbours of the same partition (node-induced subgraph); foreign rows are empty (foreign_mode 0), taken
+    from the sparsified graph `sparsified = (rowptr, col)` (1) or kept in full (2).
+    Returns (rowptr int64, col int32, stats)."""
+    rowptr, col = _i64(rowptr), _i32(col)
+    part = np.asarray(part)
+    rows = np.repeat(np.arange(n, dtype=np.int64), np.diff(rowptr))
+    own_row = part[rows] == worker
+    keep = own_row if keep_cross_edges else (own_row & (part[col] == worker))
+    out_rows, out_cols = [rows[keep]], [col[keep].astype(np.int64)]
+    own_entries = int(keep.sum())
+    foreign_entries = 0
+    foreign_rows = 0
+    if foreign_mode == 1:
+        sp_ptr, sp_col = _i64(sparsified[0]), _i32(sparsified[1])
+        srows = np.repeat(np.arange(n, dtype=np.int64), np.diff(sp_ptr))
+        f = part[srows] != worker
+        out_rows.append(srows[f]); out_cols.append(sp_col[f].astype(np.int64))
+        foreign_entries = int(f.sum()); foreign_rows = int(np.unique(srows[f]).shape[0])
+    elif foreign_mode == 2:
+        f = ~own_row
+        out_rows.append(rows[f]); out_cols.append(col[f].astype(np.int64))
+        foreign_entries = int(f.sum()); foreign_rows = int(np.unique(rows[f]).shape[0])
+    r = np.concatenate(out_rows); c = np.concatenate(out_cols)
+    order = np.lexsort((c, r))
+    r, c = r[order], c[order]
+    ptr = np.zeros(n + 1, dtype=np.int64)
+    np.cumsum(np.bincount(r, minlength=n), out=ptr[1:])
+    stats = {"own_entries": own_entries, "foreign_entries": foreign_entries, "foreign_rows": foreign_rows,
+             "own_nodes": int((part == worker).sum())}
+    return ptr, c.astype(np.int32), stats

@@ -28,6 +28,7 @@ EXPORTS = [
     "lp_adam_step", "lp_score", "lp_get_embeddings", "lp_get_output_gradient", "lp_get_block",
     "lp_get_stats", "lp_op_aggregate", "lp_op_linear", "lp_op_weight_grad", "lp_profile_begin", "lp_profile_end",
     "lp_weight_grad_static", "lp_sparsify", "lp_get_sparsified",
+    "lp_worker_view", "lp_get_worker_view",
 ]
 
 PROF_CATEGORIES = ["agg_fwd", "agg_bwd", "gemm_fwd", "gemm_dgrad", "gemm_wgrad", "score", "incidence", "scatter",
@@ -50,6 +51,10 @@ class Stats(C.Structure):
     _fields_ = [("negatives_exhausted", C.c_int64), ("block_nodes", C.c_int64 * (LP_MAX_LAYERS + 1)),
                 ("block_edges", C.c_int64 * LP_MAX_LAYERS), ("workspace_bytes", C.c_int64),
                 ("kernel_launches", C.c_int64)]
+
+
+class ViewStats(C.Structure):
+    _fields_ = [("own_entries", C.c_int64), ("foreign_entries", C.c_int64), ("foreign_rows", C.c_int64), ("own_nodes", C.c_int64)]
 
 
 class Profile(C.Structure):
@@ -153,6 +158,21 @@ class Context:
         w = t.empty(max(k, 1), dtype=t.float32, device=dev)
         self._ck(self.lib.lp_get_sparsified(self.h, _ptr(rowptr), _ptr(col), _ptr(w)))
         return rowptr, col[:k], w[:k]
+
+    def worker_view(self, part, worker: int, keep_cross_edges: bool = True, foreign_mode: int = 1):
+        """Graph that `worker` trains on (Section III): (rowptr int64, col int32, stats dict) on the device.
+        foreign_mode 0 = no sharing, 1 = sparsified rows of the last sparsify(), 2 = full rows."""
+        t = self._torch
+        dev = f"cuda:{self.device}"
+        nnz, st = C.c_int64(), ViewStats()
+        self._ck(self.lib.lp_worker_view(self.h, _ptr(part), C.c_int32(worker), C.c_int32(int(keep_cross_edges)), C.c_int32(foreign_mode),
+                                         C.byref(nnz), C.byref(st)))
+        k = int(nnz.value)
+        rowptr = t.empty(self.n + 1, dtype=t.int64, device=dev)
+        col = t.empty(max(k, 1), dtype=t.int32, device=dev)
+        self._ck(self.lib.lp_get_worker_view(self.h, _ptr(rowptr), _ptr(col)))
+        return rowptr, col[:k], {"own_entries": st.own_entries, "foreign_entries": st.foreign_entries,
+                                 "foreign_rows": st.foreign_rows, "own_nodes": st.own_nodes}
 
     # ---- model
     def set_model(self, arch: str, dims: Sequence[int], prec: str = "fp32", fanout: Optional[Sequence[int]] = None,

@@ -13,6 +13,7 @@
 #include "edge.cuh"
 #include "optim.cuh"
 #include "sparsify.cuh"
+#include "view.cuh"
 
 // ----------------------------------------------------------------------------------------------
 // context
@@ -50,6 +51,9 @@ struct lp_ctx {
     int *sp_col = nullptr;
     float *sp_w = nullptr;
     int64_t sp_nnz = -1;
+    std::vector<void *> view_allocs;
+    int64_t view_bytes = 0, view_nnz = -1;
+    int *view_ptr = nullptr, *view_col = nullptr;  // last worker view
 
     // graph
     bool loaded = false;
@@ -265,6 +269,7 @@ extern "C" void lp_destroy(lp_ctx *ctx)
     cudaStreamSynchronize(ctx->ex.st);
     free_list(ctx->model_allocs);
     free_list(ctx->sparse_allocs);
+    free_list(ctx->view_allocs);
     free_list(ctx->graph_allocs);
     tc_destroy(ctx->tc);
     for (cudaEvent_t e : ctx->ex.prof.pool) cudaEventDestroy(e);
@@ -301,6 +306,8 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
     drop_model(ctx);
     free_list(ctx->sparse_allocs);
     ctx->sp_nnz = -1;
+    free_list(ctx->view_allocs);
+    ctx->view_nnz = -1;
     free_list(ctx->graph_allocs);
     ctx->graph_bytes = 0;
     ctx->loaded = false;
@@ -512,6 +519,68 @@ extern "C" lp_status lp_get_sparsified(lp_ctx *ctx, int64_t *rowptr, int32_t *co
     if (rowptr) CK(cudaMemcpyAsync(rowptr, ctx->sp_ptr, sizeof(int64_t) * ((size_t)ctx->n + 1), cudaMemcpyDeviceToDevice, st));
     if (col && ctx->sp_nnz > 0) CK(cudaMemcpyAsync(col, ctx->sp_col, sizeof(int) * (size_t)ctx->sp_nnz, cudaMemcpyDeviceToDevice, st));
     if (w && ctx->sp_nnz > 0) CK(cudaMemcpyAsync(w, ctx->sp_w, sizeof(float) * (size_t)ctx->sp_nnz, cudaMemcpyDeviceToDevice, st));
+    return LP_OK;
+}
+
+// ----------------------------------------------------------------------------------------------
+// worker view
+// ----------------------------------------------------------------------------------------------
+#define VALLOC(ptr, count) CK(dev_alloc(ctx, ctx->view_allocs, ctx->view_bytes, &(ptr), (count)))
+
+extern "C" lp_status lp_worker_view(lp_ctx *ctx, const int32_t *part, int32_t worker, int32_t keep_cross_edges, int32_t foreign_mode,
+                                    int64_t *nnz_out, lp_view_stats *stats)
+{
+    if (!ctx || !nnz_out) return LP_EINVAL;
+    if (!ctx->loaded) return fail(ctx, LP_ESTATE, "lp_worker_view: no graph loaded");
+    if (!part) return fail(ctx, LP_EINVAL, "lp_worker_view: part is NULL");
+    if (foreign_mode < 0 || foreign_mode > 2) return fail(ctx, LP_EINVAL, "lp_worker_view: foreign_mode must be 0, 1 or 2");
+    if (foreign_mode == VIEW_FOREIGN_SPARSIFIED && ctx->sp_nnz < 0) return fail(ctx, LP_ESTATE, "lp_worker_view: call lp_sparsify first");
+    CK(cudaSetDevice(ctx->device));
+    cudaStream_t st = ctx->ex.st;
+    CK(cudaStreamSynchronize(st));
+    free_list(ctx->view_allocs);
+    ctx->view_bytes = 0;
+    ctx->view_nnz = -1;
+    const int n = ctx->n;
+    int *scan_tmp = nullptr;
+    unsigned long long *dstats = nullptr;
+    VALLOC(ctx->view_ptr, n + 1);
+    VALLOC(scan_tmp, ceil_div64(n + 1, SCAN_TILE) + 2);
+    VALLOC(dstats, 8);
+    CK(cudaMemsetAsync(dstats, 0, 8 * sizeof(unsigned long long), st));
+    view_count_kernel<<<nblk(n), 256, 0, st>>>(n, ctx->rowptr, ctx->col, part, worker, keep_cross_edges, foreign_mode, ctx->sp_ptr, ctx->view_ptr, dstats);
+    exclusive_scan_i32(ctx->ex, ctx->view_ptr, n, ctx->view_ptr, ctx->view_ptr + n, scan_tmp);
+    unsigned long long hs[4] = {0, 0, 0, 0};
+    CK(cudaMemcpyAsync(hs, dstats, sizeof hs, cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    const unsigned long long total = hs[0] + hs[1];
+    if (total >= (1ull << 31)) return fail(ctx, LP_EINVAL, "lp_worker_view: the view has 2^31 entries or more");
+    VALLOC(ctx->view_col, (int64_t)total);
+    view_fill_kernel<<<nblk(n), 256, 0, st>>>(n, ctx->rowptr, ctx->col, part, worker, keep_cross_edges, foreign_mode, ctx->sp_ptr, ctx->sp_col,
+                                              ctx->view_ptr, ctx->view_col);
+    ctx->ex.launches += 2;
+    CK(cudaStreamSynchronize(st));
+    CK_LAUNCH();
+    ctx->view_nnz = (int64_t)total;
+    *nnz_out = (int64_t)total;
+    if (stats) {
+        stats->own_entries = (int64_t)hs[0];
+        stats->foreign_entries = (int64_t)hs[1];
+        stats->foreign_rows = (int64_t)hs[2];
+        stats->own_nodes = (int64_t)hs[3];
+    }
+    return LP_OK;
+}
+
+extern "C" lp_status lp_get_worker_view(lp_ctx *ctx, int64_t *rowptr, int32_t *col)
+{
+    if (!ctx) return LP_EINVAL;
+    if (ctx->view_nnz < 0) return fail(ctx, LP_ESTATE, "lp_get_worker_view: call lp_worker_view first");
+    CK(cudaSetDevice(ctx->device));
+    cudaStream_t st = ctx->ex.st;
+    if (rowptr) widen_i32_kernel<<<nblk(ctx->n + 1), 256, 0, st>>>(ctx->view_ptr, ctx->n + 1, rowptr);
+    if (col && ctx->view_nnz > 0) CK(cudaMemcpyAsync(col, ctx->view_col, sizeof(int) * (size_t)ctx->view_nnz, cudaMemcpyDeviceToDevice, st));
+    CK_LAUNCH();
     return LP_OK;
 }
 

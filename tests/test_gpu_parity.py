@@ -603,3 +603,26 @@ def test_cached_input_aggregation_gives_identical_steps(pkg, arch):
     with pytest.raises(pkg.LpError):
         ctx.set_model("sage", [64, 64], fanout=[3], max_batch=8, cache_input_aggregation=True)
     ctx.close()
+
+
+# ------------------------------------------------------------------------------------------ worker views (Section III)
+def test_worker_views_match_oracle(pkg):
+    g = wl.chung_lu(20000, 14.0, 2.1, seed=6)
+    part = wl.random_partition(g.n, 4, seed=3)
+    ctx = make_ctx(pkg, g, wl.node_features(g.n, 8, 0))
+    dpart = t32(part)
+    with pytest.raises(pkg.LpError) as ei:
+        ctx.worker_view(dpart, 0, True, 1)  # sparsified rows requested before lp_sparsify
+    assert ei.value.status == -2
+    srp, scol, _ = ctx.sparsify(0.2, 9)
+    sp = (srp.cpu().numpy(), scol.cpu().numpy())
+    for worker in (0, 3):
+        for keep_cross, mode in ((True, 1), (True, 2), (True, 0), (False, 0)):  # SpLPG, SpLPG+, SpLPG-, SpLPG--
+            rp, col, st = ctx.worker_view(dpart, worker, keep_cross, mode)
+            orp, ocol, ost = oracle.worker_view(g.n, g.rowptr, g.col, part, worker, keep_cross, mode, sparsified=sp)
+            assert np.array_equal(rp.cpu().numpy(), orp) and np.array_equal(col.cpu().numpy(), ocol) and st == ost
+    # the sparsified sharing moves far fewer foreign entries than complete sharing (the method's point)
+    _, _, s1 = ctx.worker_view(dpart, 0, True, 1)
+    _, _, s2 = ctx.worker_view(dpart, 0, True, 2)
+    assert s1["foreign_entries"] < 0.45 * s2["foreign_entries"]
+    ctx.close()

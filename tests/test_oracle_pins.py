@@ -458,3 +458,28 @@ def test_relu_tie_window_only_touches_near_zero_units():
     assert np.array_equal(out["active"][0][near], flipped[near])
     # window of zero width: nothing adopted
     assert oracle.forward(g, X, p, "gcn", dims, relu_ties=[flipped], tie_tol=0.0)["ties"] == 0
+
+
+def test_worker_view_bruteforce():
+    g = wl.chung_lu(300, 8.0, 2.1, seed=4)
+    part = wl.random_partition(g.n, 3, seed=1)
+    sp = oracle.sparsified_graph(g.n, g.rowptr, g.col, 0.3, seed=2)
+    for keep_cross in (True, False):
+        for mode in (0, 1, 2):
+            ptr, col, st = oracle.worker_view(g.n, g.rowptr, g.col, part, 1, keep_cross, mode, sparsified=sp[:2])
+            own = foreign = frows = 0
+            for v in range(g.n):  # row by row, straight from the definition
+                if part[v] == 1:
+                    exp = [u for u in g.col[g.rowptr[v]:g.rowptr[v + 1]] if keep_cross or part[u] == 1]
+                    own += len(exp)
+                elif mode == 1:
+                    exp = list(sp[1][sp[0][v]:sp[0][v + 1]])
+                elif mode == 2:
+                    exp = list(g.col[g.rowptr[v]:g.rowptr[v + 1]])
+                else:
+                    exp = []
+                if part[v] != 1:
+                    foreign += len(exp)
+                    frows += 1 if exp else 0
+                assert col[ptr[v]:ptr[v + 1]].tolist() == exp
+            assert st == {"own_entries": own, "foreign_entries": foreign, "foreign_rows": frows, "own_nodes": int((part == 1).sum())}
