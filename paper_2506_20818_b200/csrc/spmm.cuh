@@ -69,6 +69,26 @@ constexpr float SPMM_EXACT_SCALE = 1099511627776.f;  // 2^40: products up to 2^2
 template <typename ACC> LP_DEVINL void acc_add(ACC &a, float w, float f);
 template <> LP_DEVINL void acc_add<float>(float &a, float w, float f) { a = fmaf(w, f, a); }
 template <> LP_DEVINL void acc_add<long long>(long long &a, float w, float f) { a += __float2ll_rn(w * f * SPMM_EXACT_SCALE); }
+// acc[0..VN) += w * v for one 16-byte vector.  Unit coefficients on BF16 data into FP32 accumulators use the
+// mixed-precision add of sm_100 (add.rn.f32.bf16: the BF16 operand is widened exactly, one rounding, the
+// same result as convert-then-add) and so skip the eight conversion instructions per vector.
+template <typename T, typename ACC, bool HAS_VAL> LP_DEVINL void acc_add_vec(ACC *acc, float w, const Vec16<T> &v)
+{
+    constexpr int VN = Vec16<T>::N;
+    float f[VN];
+    v.to_float(f);
+#pragma unroll
+    for (int t = 0; t < VN; ++t) acc_add<ACC>(acc[t], w, f[t]);
+}
+template <> LP_DEVINL void acc_add_vec<bf16, float, false>(float *acc, float, const Vec16<bf16> &v)
+{
+    const uint32_t x[4] = {v.v.x, v.v.y, v.v.z, v.v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tadd.rn.f32.bf16 %0, lo, %0;\n\tadd.rn.f32.bf16 %1, hi, %1;\n\t}"
+            : "+f"(acc[2 * i]), "+f"(acc[2 * i + 1])
+            : "r"(x[i]));
+}
 template <typename ACC> LP_DEVINL float acc_value(ACC a);
 template <> LP_DEVINL float acc_value<float>(float a) { return a; }
 template <> LP_DEVINL float acc_value<long long>(long long a) { return (float)((double)a * (1.0 / 1099511627776.0)); }
@@ -121,12 +141,7 @@ LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl,
 #pragma unroll
                 for (int i = 0; i < NV; ++i) {
                     const int ch = gl + i * G;
-                    if (ch < nchunks) {
-                        float f[VN];
-                        v[q][i].to_float(f);
-#pragma unroll
-                        for (int t = 0; t < VN; ++t) acc_add<ACC>(acc[i][t], w[q], f[t]);
-                    }
+                    if (ch < nchunks) acc_add_vec<T, ACC, HAS_VAL>(acc[i], w[q], v[q][i]);
                 }
         }
         for (; j < cnt; ++j) {
@@ -138,10 +153,7 @@ LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl,
                 if (ch < nchunks) {
                     Vec16<T> v;
                     v.load(a.X + (size_t)c * a.ldx + ch * VN);
-                    float f[VN];
-                    v.to_float(f);
-#pragma unroll
-                    for (int t = 0; t < VN; ++t) acc_add<ACC>(acc[i][t], w, f[t]);
+                    acc_add_vec<T, ACC, HAS_VAL>(acc[i], w, v);
                 }
             }
         }
