@@ -114,7 +114,8 @@ static void gemm_simt(Exec &ex, int64_t M, int N, int64_t K, const TA *A, int64_
 }
 
 constexpr int WG_MAX_SPLITS = 256;
-static int weight_grad_splits(int64_t rows) { return (int)std::max<int64_t>(1, std::min<int64_t>(WG_MAX_SPLITS, ceil_div64(rows, 1024))); }
+// one split per 256 rows (small graphs still fill the GPU), at most WG_MAX_SPLITS
+static int weight_grad_splits(int64_t rows) { return (int)std::max<int64_t>(1, std::min<int64_t>(WG_MAX_SPLITS, ceil_div64(rows, 256))); }
 
 // dW[Kin, N] = A[rows, Kin]^T * dZ[rows, N]; `partials` needs weight_grad_splits(rows) * Kin * N floats.
 template <typename T>

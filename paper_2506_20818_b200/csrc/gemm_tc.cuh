@@ -108,7 +108,23 @@ LP_DEVINL void umma_commit(uint32_t bar)
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// 32 lanes x 32 consecutive FP32 columns: thread t of the warp receives lane (32 * (warp % 4) + t)
+// 32 lanes x 32 consecutive FP32 columns: thread t of the warp receives lane (32 * (warp % 4) + t).
+// tmem_ld_32x32_issue starts the load, tmem_ld_wait makes every issued load's registers valid.
+LP_DEVINL void tmem_ld_32x32_issue(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]),
+          "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
+          "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]),
+          "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+LP_DEVINL void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 LP_DEVINL void tmem_ld_32x32(uint32_t taddr, float *v)
 {
     uint32_t r[32];
@@ -350,10 +366,13 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
 // BF16) writes 128-column halves of the tile into a swizzled shared-memory staging area that one
 // thread hands to TMA stores (full 128-byte rows instead of 16-byte pieces of 32 different rows per
 // store instruction; rows beyond M are clipped by the tensor map).
-//   warp 0: TMA producer (one lane)      warp 1: MMA issuer (one lane)      warps 2-5: epilogue
+//   warp 0: TMA producer (one lane)      warp 1: MMA issuer (one lane)      warps 2-9: epilogue
+// (two warps per tensor-memory lane quarter, one per 64-column box of the 128-column round; each issues
+// both of its 32-column loads before waiting)
 // ---------------------------------------------------------------------------------------------
-constexpr int TCP_THREADS = 192;
-constexpr int TCP_STAGES = 4;
+constexpr int TCP_THREADS = 320;       // warp 0 producer, warp 1 MMA issuer, warps 2-9 epilogue
+constexpr int TCP_EPI_THREADS = 256;
+constexpr int TCP_MAX_STAGES = 8;  // A-tile ring: as many 16 KiB stages as fit beside the weight slice (4..8)
 constexpr int TCP_STAGE_OUT_BYTES = 2 * 16384;  // output staging: two boxes of 128 rows x 64 BF16 columns
 
 LP_DEVINL void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y)
@@ -363,7 +382,7 @@ LP_DEVINL void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y)
 LP_DEVINL void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 LP_DEVINL void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 LP_DEVINL void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-LP_DEVINL void epilogue_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }  // the four epilogue warps only
+LP_DEVINL void epilogue_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }  // the eight epilogue warps only
 
 LP_DEVINL void mbar_arrive(uint32_t bar) { asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory"); }
 
@@ -373,7 +392,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
 {
     __shared__ float s_bias[256];
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_full[TCP_STAGES], bar_empty[TCP_STAGES], bar_w, bar_acc_full[2], bar_acc_empty[2];
+    __shared__ __align__(8) uint64_t bar_full[TCP_MAX_STAGES], bar_empty[TCP_MAX_STAGES], bar_w, bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
 
@@ -385,7 +404,8 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
     uint8_t *smem_w = smem;
     uint8_t *smem_a = smem + (size_t)KB * w_sub_bytes;
     const uint32_t a_bytes = TC_BM * TC_BK * 2;
-    uint8_t *smem_out = smem_a + (size_t)TCP_STAGES * a_bytes;
+    const int S = p.stages;
+    uint8_t *smem_out = smem_a + (size_t)S * a_bytes;
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < 2 * BN) tmem_cols <<= 1;
 
@@ -398,14 +418,14 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
     const int64_t my_tiles = first_tile < m_tiles ? (m_tiles - first_tile + stride - 1) / stride : 0;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < TCP_STAGES; ++s) {
+        for (int s = 0; s < S; ++s) {
             mbar_init(smem_u32(&bar_full[s]), 1);
             mbar_init(smem_u32(&bar_empty[s]), 1);
         }
         mbar_init(smem_u32(&bar_w), 1);
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&bar_acc_full[b]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[b]), 4);  // one arrival per epilogue warp
+            mbar_init(smem_u32(&bar_acc_empty[b]), 8);  // one arrival per epilogue warp
         }
         abort_s = 0;
         fence_barrier_init();
@@ -435,8 +455,8 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
             for (int64_t i = 0; i < my_tiles && !*abort_flag; ++i) {
                 const int m0 = (int)((first_tile + i * stride) * TC_BM);
                 for (int kb = 0; kb < KB; ++kb, ++it) {
-                    const int s = (int)(it % TCP_STAGES);
-                    if (it >= TCP_STAGES && !mbar_wait(smem_u32(&bar_empty[s]), (uint32_t)(((it / TCP_STAGES) & 1) ^ 1))) {
+                    const int s = (int)(it % S);
+                    if (it >= S && !mbar_wait(smem_u32(&bar_empty[s]), (uint32_t)(((it / S) & 1) ^ 1))) {
                         atomicExch(p.err, 1);
                         *abort_flag = 1;
                         break;
@@ -462,8 +482,8 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + (uint32_t)(b * BN);
                 for (int kb = 0; kb < KB; ++kb, ++it) {
-                    const int s = (int)(it % TCP_STAGES);
-                    if (!mbar_wait(smem_u32(&bar_full[s]), (uint32_t)((it / TCP_STAGES) & 1))) {
+                    const int s = (int)(it % S);
+                    if (!mbar_wait(smem_u32(&bar_full[s]), (uint32_t)((it / S) & 1))) {
                         atomicExch(p.err, 2);
                         *abort_flag = 1;
                         ok = false;
@@ -480,14 +500,16 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
                 if (ok) umma_commit(smem_u32(&bar_acc_full[b]));
             }
         } else if (warp >= 2) {
-            // ---- epilogue: warp w reads the TMEM lanes of quarter (w mod 4)
+            // ---- epilogue: warp w reads the TMEM lanes of quarter (w mod 4); warps 2-5 take the first 64-column
+            // box of every 128-column round, warps 6-9 the second
             const int q = warp & 3;
+            const int my_box = (warp - 2) >> 2;
             for (int64_t i = 0; i < my_tiles; ++i) {
                 const int b = (int)(i & 1);
                 bool ready = mbar_wait(smem_u32(&bar_acc_full[b]), (uint32_t)((i >> 1) & 1));
                 if (!ready && lane == 0) { atomicExch(p.err, 3); *abort_flag = 1; }
                 if (!__all_sync(0xffffffffu, ready) && lane == 0) *abort_flag = 1;
-                epilogue_barrier();             // the four warps take the same decision: all continue or all leave
+                epilogue_barrier();             // the eight warps take the same decision: all continue or all leave
                 if (*abort_flag != 0) break;
                 tc_fence_after();
                 const int m0 = (int)((first_tile + i * stride) * TC_BM);
@@ -499,30 +521,41 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
                     const int nbox = min(2, (BN - half) / 64);
                     if (store_thread) tma_store_wait_read();  // the previous stores have read the staging area
                     epilogue_barrier();
-                    for (int c0 = half; c0 < half + nbox * 64; c0 += 32) {
-                        float v[32];
-                        tmem_ld_32x32(taddr + (uint32_t)c0, v);
+                    if (my_box < nbox) {
+                        const int cb = half + my_box * 64;
+                        uint32_t r[2][32];
+                        tmem_ld_32x32_issue(taddr + (uint32_t)cb, r[0]);
+                        tmem_ld_32x32_issue(taddr + (uint32_t)(cb + 32), r[1]);
+                        tmem_ld_wait();
+                        uint8_t *box = smem_out + (size_t)my_box * 16384 + (size_t)row_t * 128;
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            const float4 bb = *reinterpret_cast<const float4 *>(&s_bias[c0 + j]);
-                            v[j] += bb.x; v[j + 1] += bb.y; v[j + 2] += bb.z; v[j + 3] += bb.w;
-                        }
-                        if (p.relu) {
+                        for (int h2 = 0; h2 < 2; ++h2) {
+                            const int c0 = cb + 32 * h2;
+                            float v[32];
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
-                        }
-                        if (p.row_scale && n0 + c0 >= p.scale_col0) {
+                            for (int j = 0; j < 32; j += 4) {
+                                const float4 bb = *reinterpret_cast<const float4 *>(&s_bias[c0 + j]);
+                                v[j] = __uint_as_float(r[h2][j]) + bb.x;
+                                v[j + 1] = __uint_as_float(r[h2][j + 1]) + bb.y;
+                                v[j + 2] = __uint_as_float(r[h2][j + 2]) + bb.z;
+                                v[j + 3] = __uint_as_float(r[h2][j + 3]) + bb.w;
+                            }
+                            if (p.relu) {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) v[j] *= rs;
-                        }
-                        // 128-byte swizzle of the staging box: 16-byte chunk index XOR (row mod 8)
-                        uint8_t *box = smem_out + (size_t)((c0 - half) / 64) * 16384 + (size_t)row_t * 128;
-                        const int chunk0 = (c0 & 63) >> 3;
+                                for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
+                            }
+                            if (p.row_scale && n0 + c0 >= p.scale_col0) {
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            Vec16<bf16> o;
-                            o.from_float(v + 8 * j);
-                            *reinterpret_cast<uint4 *>(box + (((chunk0 + j) ^ (row_t & 7)) << 4)) = o.v;
+                                for (int j = 0; j < 32; ++j) v[j] *= rs;
+                            }
+                            // 128-byte swizzle of the staging box: 16-byte chunk index XOR (row mod 8)
+                            const int chunk0 = 4 * h2;
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                Vec16<bf16> o;
+                                o.from_float(v + 8 * j);
+                                *reinterpret_cast<uint4 *>(box + (((chunk0 + j) ^ (row_t & 7)) << 4)) = o.v;
+                            }
                         }
                     }
                     fence_async_proxy();  // generic-proxy writes -> visible to the TMA engine
@@ -663,14 +696,17 @@ static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const
         CUtensorMap mapC;
         if (!tc_make_map(tc, &mapC, C, M, N, ldc, 64, TC_BM, err)) return false;
         TcGemmParams p{};
-        p.M = M; p.N = N; p.K = K; p.BN = pbn; p.stages = TCP_STAGES;
+        const int64_t smem_cap = 225 * 1024 + 512 - 1024;
+        const int64_t w_bytes = (int64_t)(K / TC_BK) * pbn * 128;
+        p.M = M; p.N = N; p.K = K; p.BN = pbn;
+        p.stages = (int)std::max<int64_t>(4, std::min<int64_t>(TCP_MAX_STAGES, (smem_cap - w_bytes - TCP_STAGE_OUT_BYTES) / (TC_BM * TC_BK * 2)));
         p.bias = bias; p.relu = relu ? 1 : 0; p.C = C; p.ldc = ldc; p.out_f32 = nullptr; p.err = tc.err_word;
         p.row_scale = row_scale; p.scale_col0 = scale_col0;
         const int n_slices = N / pbn;
         const int64_t m_tiles = ceil_div64(M, TC_BM);
         int64_t ctas = std::min<int64_t>((int64_t)tc_sm_count(), m_tiles * n_slices);
         ctas = std::max<int64_t>(n_slices, ctas / n_slices * n_slices);  // a whole number of CTAs per slice
-        const size_t smem = (size_t)(K / TC_BK) * pbn * 128 + (size_t)TCP_STAGES * TC_BM * TC_BK * 2 + TCP_STAGE_OUT_BYTES + 1024;
+        const size_t smem = (size_t)w_bytes + (size_t)p.stages * TC_BM * TC_BK * 2 + TCP_STAGE_OUT_BYTES + 1024;
         tc_linear_persistent_kernel<<<(unsigned)ctas, TCP_THREADS, smem, ex.st>>>(mapA, mapB, mapC, p);
         ex.launches += 1;
         return true;
