@@ -33,4 +33,7 @@ from .model import (  # noqa: F401
     score,
     adam_step,
     average_gradients,
+    hits_at_k,
+    encoder_param_count,
+    split_predictor,
 )

@@ -32,6 +32,65 @@ def split_params(arch: str, dims: Sequence[int], params: np.ndarray):
     return out
 
 
+def encoder_param_count(arch: str, dims: Sequence[int]) -> int:
+    return sum((2 if arch == "sage" else 1) * dims[k] * dims[k + 1] + dims[k + 1] for k in range(len(dims) - 1))
+
+
+def split_predictor(D: int, Hp: int, tail: np.ndarray):
+    """Views into the predictor part of the flat parameter vector: W0[D,Hp], b0[Hp], W1[Hp,Hp], b1[Hp], w2[Hp], b2[1]."""
+    o = 0
+    out = {}
+    for name, shape in (("W0", (D, Hp)), ("b0", (Hp,)), ("W1", (Hp, Hp)), ("b1", (Hp,)), ("w2", (Hp,)), ("b2", (1,))):
+        size = int(np.prod(shape))
+        out[name] = tail[o:o + size].reshape(shape)
+        o += size
+    assert o == tail.shape[0], "predictor parameters have the wrong length"
+    return out
+
+
+def mlp_predictor_forward(HK, src, dst, pred, ties=None, tie_tol=0.0):
+    """EdgePredictor of Eq. 2 as the 3-layer MLP of the paper's experiments (Section IV) on the Hadamard
+    product of the two embeddings: z0 = h_u * h_v; p1 = ReLU(z0 W0 + b0); p2 = ReLU(p1 W1 + b1);
+    s = p2 . w2 + b2.  ties = (active1, active2) decisions of the implementation under test, adopted only
+    inside the tie window (see forward())."""
+    def relu_decisions(a, given):
+        active = a > 0.0
+        flipped = 0
+        if given is not None and tie_tol > 0.0:
+            near = np.abs(a) <= tie_tol * np.sqrt(np.mean(a * a))
+            flipped = int((near & (active != given)).sum())
+            active = np.where(near, given, active)
+        return active, flipped
+
+    z0 = HK[src] * HK[dst]
+    a1 = z0 @ pred["W0"] + pred["b0"]
+    active1, t1 = relu_decisions(a1, None if ties is None else ties[0])
+    p1 = np.where(active1, a1, 0.0)
+    a2 = p1 @ pred["W1"] + pred["b1"]
+    active2, t2 = relu_decisions(a2, None if ties is None else ties[1])
+    p2 = np.where(active2, a2, 0.0)
+    s = p2 @ pred["w2"] + pred["b2"][0]
+    return s, {"z0": z0, "p1": p1, "p2": p2, "active1": active1, "active2": active2, "ties": t1 + t2}
+
+
+def mlp_predictor_backward(HK, src, dst, pred, cache, gs):
+    """Chain rule through the MLP predictor: returns (gradient dict, dL/dH^(K))."""
+    G = {}
+    G["w2"] = cache["p2"].T @ gs
+    G["b2"] = np.array([gs.sum()])
+    dp2 = np.outer(gs, pred["w2"]) * cache["active2"]
+    G["W1"] = cache["p1"].T @ dp2
+    G["b1"] = dp2.sum(axis=0)
+    dp1 = (dp2 @ pred["W1"].T) * cache["active1"]
+    G["W0"] = cache["z0"].T @ dp1
+    G["b0"] = dp1.sum(axis=0)
+    dz0 = dp1 @ pred["W0"].T
+    dH = np.zeros_like(HK)
+    np.add.at(dH, src, dz0 * HK[dst])
+    np.add.at(dH, dst, dz0 * HK[src])
+    return G, dH
+
+
 def _block_as_global_csr(n: int, frontier: np.ndarray, ptr: np.ndarray, cols: np.ndarray):
     counts = np.zeros(n, dtype=np.int64)
     counts[frontier] = np.diff(ptr)
@@ -110,27 +169,43 @@ def bce_with_logits(s: np.ndarray, y: np.ndarray):
     return ell, sig - y
 
 
-def train_step(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst, blocks=None, relu_ties=None, tie_tol=0.0):
+def train_step(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst, blocks=None, relu_ties=None, tie_tol=0.0,
+               pred_hidden: int = 0, pred_ties=None):
     """One training step of Algorithm 1 for one worker: scores of Eq. 2 (dot product) for
     positives (label 1) and negatives (label 0), loss L = (1/N) sum ell with N = |P| + |N|,
     and the gradient with respect to every parameter in the flat layout."""
     K = len(dims) - 1
-    P = split_params(arch, dims, np.asarray(params, dtype=np.float64))
-    cache = forward(g, X, params, arch, dims, blocks, relu_ties, tie_tol)
+    params = np.asarray(params, dtype=np.float64)
+    n_enc = encoder_param_count(arch, dims)
+    enc_params = params[:n_enc]
+    P = split_params(arch, dims, enc_params)
+    cache = forward(g, X, enc_params, arch, dims, blocks, relu_ties, tie_tol)
     HK = cache["H"][K]
     src = np.concatenate([pos_src, neg_src]).astype(np.int32)
     dst = np.concatenate([pos_dst, neg_dst]).astype(np.int32)
     y = np.concatenate([np.ones(len(pos_src)), np.zeros(len(neg_src))])
-    s = np.einsum("ij,ij->i", HK[src], HK[dst])
+    pred = pcache = None
+    if pred_hidden > 0:
+        pred = split_predictor(dims[K], pred_hidden, params[n_enc:])
+        s, pcache = mlp_predictor_forward(HK, src, dst, pred, pred_ties, tie_tol)
+    else:
+        s = np.einsum("ij,ij->i", HK[src], HK[dst])
     ell, dls = bce_with_logits(s, y)
     N = s.shape[0]
     loss = ell.sum() / N
     gs = dls / N
-    dH = sparse.edge_grad(HK, src, dst, gs)
+    grads_full = np.zeros(params.shape[0], dtype=np.float64)
+    if pred_hidden > 0:
+        PG, dH = mlp_predictor_backward(HK, src, dst, pred, pcache, gs)
+        GP = split_predictor(dims[K], pred_hidden, grads_full[n_enc:])
+        for name in GP:
+            GP[name][...] = PG[name]
+    else:
+        dH = sparse.edge_grad(HK, src, dst, gs)
     dHK = dH
 
-    grads = np.zeros(params.shape[0], dtype=np.float64)
-    G = split_params(arch, dims, grads)
+    grads = grads_full
+    G = split_params(arch, dims, grads[:n_enc])
     mode = "gcn" if arch == "gcn" else "mean"
     for k in range(K - 1, -1, -1):
         rp, cc, w, act = cache["graphs"][k]
@@ -151,7 +226,7 @@ def train_step(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst, blo
             if k > 0:
                 dH = dZ @ P[k]["W_self"].T + sparse.aggregate_backward(mode, g.n, rp, cc, None, dZ @ P[k]["W_neigh"].T)
     return {"loss": loss, "grads": grads, "scores": s, "g": gs, "dHK": dHK,
-            "cache": cache, "src": src, "dst": dst}
+            "cache": cache, "src": src, "dst": dst, "pred_cache": pcache}
 
 
 def input_gradient(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst):
@@ -178,10 +253,26 @@ def input_gradient(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst)
     return dH
 
 
-def score(g, X, params, arch, dims, src, dst, blocks=None) -> np.ndarray:
-    """Edge scores s_(u,v) = <h_u^(K), h_v^(K)> (Eq. 2, dot-product predictor)."""
-    HK = forward(g, X, params, arch, dims, blocks)["H"][len(dims) - 1]
+def score(g, X, params, arch, dims, src, dst, blocks=None, pred_hidden: int = 0) -> np.ndarray:
+    """Edge scores of Eq. 2: <h_u^(K), h_v^(K)> (dot product) or the MLP predictor's output."""
+    params = np.asarray(params, dtype=np.float64)
+    n_enc = encoder_param_count(arch, dims)
+    HK = forward(g, X, params[:n_enc], arch, dims, blocks)["H"][len(dims) - 1]
+    if pred_hidden > 0:
+        pred = split_predictor(dims[-1], pred_hidden, params[n_enc:])
+        return mlp_predictor_forward(HK, np.asarray(src), np.asarray(dst), pred)[0]
     return np.einsum("ij,ij->i", HK[np.asarray(src)], HK[np.asarray(dst)])
+
+
+def hits_at_k(pos_scores, neg_scores, k: int) -> float:
+    """Hits@K (Section IV's accuracy metric): the fraction of positive scores that are strictly greater
+    than the K-th largest negative score (1.0 when there are fewer than K negatives)."""
+    pos = np.asarray(pos_scores, dtype=np.float64)
+    neg = np.asarray(neg_scores, dtype=np.float64)
+    if neg.shape[0] < k:
+        return 1.0
+    kth = np.sort(neg)[-k]
+    return float((pos > kth).mean())
 
 
 def average_gradients(grads_per_worker: List[np.ndarray]) -> np.ndarray:

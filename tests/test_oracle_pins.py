@@ -483,3 +483,62 @@ def test_worker_view_bruteforce():
                     frows += 1 if exp else 0
                 assert col[ptr[v]:ptr[v + 1]].tolist() == exp
             assert st == {"own_entries": own, "foreign_entries": foreign, "foreign_rows": frows, "own_nodes": int((part == 1).sum())}
+
+
+# ------------------------------------------------------------------ MLP edge predictor, Hits@K
+def _dense_mlp_loss(g, X, p, arch, dims, Hp, src, dst, y):
+    """Loss with the 3-layer MLP predictor written independently of the oracle (dense operators)."""
+    n_enc = wl.model_dims_param_count(arch, dims)
+    H, _ = dense_forward(g, X, p[:n_enc], arch, dims)
+    t, D = p[n_enc:], dims[-1]
+    o = 0
+    W0 = t[o:o + D * Hp].reshape(D, Hp); o += D * Hp
+    b0 = t[o:o + Hp]; o += Hp
+    W1 = t[o:o + Hp * Hp].reshape(Hp, Hp); o += Hp * Hp
+    b1 = t[o:o + Hp]; o += Hp
+    w2 = t[o:o + Hp]; o += Hp
+    b2 = t[o]
+    z = H[src] * H[dst]
+    s = np.maximum(np.maximum(z @ W0 + b0, 0) @ W1 + b1, 0) @ w2 + b2
+    return float(np.mean(y * np.logaddexp(0.0, -s) + (1 - y) * np.logaddexp(0.0, s))), s
+
+
+@pytest.mark.parametrize("arch", ["gcn", "sage"])
+def test_mlp_predictor_forward_and_finite_differences(arch):
+    g = wl.erdos_renyi(26, 70, seed=4)
+    dims, Hp = [3, 4, 3], 5
+    X = wl.node_features(g.n, 3, 2)
+    p = wl.glorot_params(arch, dims, 5, bias_scale=0.3, pred_hidden=Hp).astype(np.float64)
+    assert p.shape[0] == wl.model_dims_param_count(arch, dims, Hp)
+    rng = np.random.default_rng(1)
+    src = rng.integers(0, g.n, 30).astype(np.int32)
+    dst = rng.integers(0, g.n, 30).astype(np.int32)
+    dst[:2] = src[:2]
+    nsrc, ndst = src[:15], rng.integers(0, g.n, 15).astype(np.int32)
+    s_all, d_all = np.concatenate([src, nsrc]), np.concatenate([dst, ndst])
+    y = np.concatenate([np.ones(30), np.zeros(15)])
+    out = oracle.train_step(g, X, p, arch, dims, src, dst, nsrc, ndst, pred_hidden=Hp)
+    ref_loss, ref_s = _dense_mlp_loss(g, X, p, arch, dims, Hp, s_all, d_all, y)
+    assert abs(out["loss"] - ref_loss) < 1e-13 and np.allclose(out["scores"], ref_s, atol=1e-13)
+    assert np.allclose(oracle.score(g, X, p, arch, dims, s_all, d_all, pred_hidden=Hp), ref_s, atol=1e-13)
+    fd = np.zeros_like(p)
+    for i in range(p.shape[0]):
+        pp, pm = p.copy(), p.copy()
+        pp[i] += 1e-6
+        pm[i] -= 1e-6
+        fd[i] = (_dense_mlp_loss(g, X, pp, arch, dims, Hp, s_all, d_all, y)[0] - _dense_mlp_loss(g, X, pm, arch, dims, Hp, s_all, d_all, y)[0]) / 2e-6
+    assert rel_l2(out["grads"], fd) < 1e-7 and np.max(np.abs(out["grads"] - fd)) < 1e-8
+    n_enc = wl.model_dims_param_count(arch, dims)
+    assert np.linalg.norm(out["grads"][n_enc:]) > 0 and np.linalg.norm(out["grads"][:n_enc]) > 0
+
+
+def test_hits_at_k_definition():
+    rng = np.random.default_rng(0)
+    pos, neg = rng.standard_normal(200), rng.standard_normal(1000)
+    for k in (1, 10, 100, 1000):
+        brute = np.mean([(neg >= p_).sum() < k for p_ in pos])  # fewer than k negatives score at least as high
+        assert abs(oracle.hits_at_k(pos, neg, k) - brute) < 1e-15
+    assert oracle.hits_at_k(pos, neg, 1001) == 1.0                 # fewer negatives than K
+    assert oracle.hits_at_k(np.array([5.0, 6.0]), np.array([1.0, 2.0, 3.0]), 1) == 1.0
+    assert oracle.hits_at_k(np.array([2.5, 0.0]), np.array([1.0, 2.0, 3.0]), 2) == 0.5
+    assert oracle.hits_at_k(np.array([2.0]), np.array([1.0, 2.0, 3.0]), 2) == 0.0  # ties do not count as hits

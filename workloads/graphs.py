@@ -172,18 +172,23 @@ def node_features(n: int, f: int, seed: int) -> np.ndarray:
     return rng.standard_normal((n, f), dtype=np.float32)
 
 
-def model_dims_param_count(arch: str, dims) -> int:
+def model_dims_param_count(arch: str, dims, pred_hidden: int = 0) -> int:
     """Flat parameter layout: per layer W_self? / W then bias.
     gcn : W[in,out] row-major, b[out]
-    sage: W_self[in,out], W_neigh[in,out] (both row-major), b[out]"""
+    sage: W_self[in,out], W_neigh[in,out] (both row-major), b[out]
+    With an MLP edge predictor (pred_hidden > 0) three more layers follow the encoder:
+    W0[D, Hp], b0[Hp], W1[Hp, Hp], b1[Hp], w2[Hp], b2[1]  (D = dims[-1], Hp = pred_hidden)."""
     total = 0
     for k in range(len(dims) - 1):
         fi, fo = dims[k], dims[k + 1]
         total += (2 if arch == "sage" else 1) * fi * fo + fo
+    if pred_hidden > 0:
+        D, Hp = dims[-1], pred_hidden
+        total += D * Hp + Hp + Hp * Hp + Hp + Hp + 1
     return total
 
 
-def glorot_params(arch: str, dims, seed: int, bias_scale: float = 0.0) -> np.ndarray:
+def glorot_params(arch: str, dims, seed: int, bias_scale: float = 0.0, pred_hidden: int = 0) -> np.ndarray:
     """Glorot-uniform weights in the flat layout; biases zero unless bias_scale > 0
     (non-zero biases make parity tests sensitive to the bias path)."""
     rng = np.random.Generator(np.random.PCG64(seed + 104729))
@@ -194,6 +199,11 @@ def glorot_params(arch: str, dims, seed: int, bias_scale: float = 0.0) -> np.nda
         for _ in range(2 if arch == "sage" else 1):
             parts.append(rng.uniform(-lim, lim, size=fi * fo).astype(np.float32))
         parts.append((bias_scale * rng.standard_normal(fo)).astype(np.float32))
+    if pred_hidden > 0:
+        for fi, fo in ((dims[-1], pred_hidden), (pred_hidden, pred_hidden), (pred_hidden, 1)):
+            lim = np.sqrt(6.0 / (fi + fo))
+            parts.append(rng.uniform(-lim, lim, size=fi * fo).astype(np.float32))
+            parts.append((bias_scale * rng.standard_normal(fo)).astype(np.float32))
     return np.concatenate(parts)
 
 
