@@ -149,6 +149,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cache-input-agg", action="store_true", help="reuse the weight-independent first-layer aggregation across steps (not the default, not the headline)")
+    ap.add_argument("--predictor", default="dot", choices=["dot", "mlp"], help="mlp: the 3-layer MLP predictor of width 256 instead of the dot product (not the headline)")
     ap.add_argument("--breakdown", action="store_true", help="print a per-category time breakdown to stderr")
     args = ap.parse_args()
 
@@ -202,11 +203,16 @@ def main():
     B = min(args.batch, len(pos[0]))
     nb = max(1, len(pos[0]) // B)
 
+    pred_hidden = 256 if args.predictor == "mlp" else 0
+    if pred_hidden:
+        params = wl.glorot_params("sage", dims, SEED, pred_hidden=pred_hidden)
+        args.no_cpu_baseline = True  # the baseline leg times the headline (dot-product) workload only
+
     stream = torch.cuda.Stream(device=dev)
     with torch.cuda.stream(stream):
         ctx = pkg.Context(local_rank, stream=stream)
         ctx.load_graph(g.n, g.rowptr, g.col, g.w, X)
-        ctx.set_model("sage", dims, prec="bf16", max_batch=B, max_k=K_NEG, cache_input_aggregation=args.cache_input_agg)
+        ctx.set_model("sage", dims, prec="bf16", max_batch=B, max_k=K_NEG, cache_input_aggregation=args.cache_input_agg, pred_hidden=pred_hidden)
         pu = torch.from_numpy(pos[0]).to(dev)
         pv = torch.from_numpy(pos[1]).to(dev)
         p = torch.from_numpy(params).to(dev)
@@ -349,7 +355,7 @@ def main():
                 "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
                 "data": "synthetic",
                 "config": {"workload": WORKLOAD, "graph": "Chung-Lu power law, exponent 2.1, mean degree 20", "nodes": g.n, "entries": g.nnz,
-                           "model": "2-layer GraphSAGE-mean 128-256-256, dot-product predictor", "batch_pos": B, "neg_per_pos": K_NEG,
+                           "model": "2-layer GraphSAGE-mean 128-256-256, " + ("3-layer MLP predictor (256)" if pred_hidden else "dot-product predictor"), "batch_pos": B, "neg_per_pos": K_NEG,
                            "scale": args.scale, "cache_input_aggregation": bool(args.cache_input_agg), "parallelism": f"dp{world}" if world > 1 else "single GPU",
                            "l2": "no flush: the step streams ~1 GB of activations per pass, several times the 126 MB L2"},
                 "clocks": clocks, "gpu_launches": int(launches), "loss_last": loss_value, "roofline": roofline, "cpu_baseline": cpu,

@@ -48,6 +48,11 @@ typedef enum {
 typedef enum { LP_GCN = 0, LP_SAGE_MEAN = 1 } lp_arch;
 typedef enum { LP_FP32 = 0, LP_BF16 = 1 } lp_prec;
 typedef enum { LP_NEG_PER_SOURCE = 0, LP_NEG_GLOBAL_PAIR = 1 } lp_neg_mode;
+/* Edge predictor of Eq. 2: the dot product <h_u, h_v>, or the 3-layer MLP of the paper's experiments
+ * (Section IV) on the element-wise product: z0 = h_u * h_v; p1 = ReLU(z0 W0 + b0); p2 = ReLU(p1 W1 + b1);
+ * s = p2 . w2 + b2.  Its parameters follow the encoder's in the flat vector:
+ * W0[D, Hp] row-major, b0[Hp], W1[Hp, Hp], b1[Hp], w2[Hp], b2[1]  (D = dims[K]). */
+typedef enum { LP_PRED_DOT = 0, LP_PRED_MLP = 1 } lp_predictor;
 
 #define LP_MAX_LAYERS 4
 
@@ -67,6 +72,8 @@ typedef struct {
     int32_t cache_input_aggregation; /* full-graph models only: AGG(X) of the first layer does not depend on the
                                         weights, so compute it in the first step and reuse it afterwards (off = 0:
                                         every step recomputes it) */
+    int32_t predictor;               /* lp_predictor: edge predictor of Eq. 2 */
+    int32_t pred_hidden;             /* LP_PRED_MLP: hidden width Hp (multiple of 8, or of 64 in BF16; <= 512) */
 } lp_model_desc;
 
 typedef struct {
@@ -239,12 +246,22 @@ lp_status lp_adam_step(lp_ctx *ctx, float *params, float *adam_m, float *adam_v,
 lp_status lp_score(lp_ctx *ctx, const float *params, const int32_t *src, const int32_t *dst, int64_t E,
                    uint64_t seed, uint64_t step, float *scores);
 
+/* Hits@K (the accuracy metric of Section IV): the fraction of the n_pos positive scores that are
+ * strictly greater than the K-th largest of the n_neg negative scores (1 when n_neg < K).  Scores are
+ * DEVICE float32 arrays (as written by lp_score); *hits is a HOST double.  Allocates temporary device
+ * memory and synchronises. */
+lp_status lp_hits_at_k(lp_ctx *ctx, const float *pos_scores, int64_t n_pos, const float *neg_scores, int64_t n_neg, int64_t K, double *hits);
+
 /* ---- inspection (parity checks) ---------------------------------------------------------- */
 
 /* Embeddings H^(layer) of the last forward pass as float32, layer in 1..K.  For full-graph
  * models `out` is [n, dims[layer]].  For sampled models `out` is [|F_{K-layer}|, dims[layer]],
  * row i belonging to node frontier[i] of that frontier (see lp_get_block).  Device output. */
 lp_status lp_get_embeddings(lp_ctx *ctx, int32_t layer, float *out);
+
+/* Hidden activations of the MLP predictor in the last lp_train_step or lp_score: layer 1 (p1) or 2 (p2)
+ * as float32 [E, pred_hidden], one row per scored edge (positives, then negatives).  Device output. */
+lp_status lp_get_predictor_activations(lp_ctx *ctx, int32_t layer, int64_t E, float *out);
 
 /* Gradient of the loss with respect to H^(K) from the last lp_train_step, float32, same row
  * indexing as lp_get_embeddings(K).  Device output. */

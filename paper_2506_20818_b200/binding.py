@@ -28,7 +28,7 @@ EXPORTS = [
     "lp_adam_step", "lp_score", "lp_get_embeddings", "lp_get_output_gradient", "lp_get_block",
     "lp_get_stats", "lp_op_aggregate", "lp_op_linear", "lp_op_weight_grad", "lp_profile_begin", "lp_profile_end",
     "lp_weight_grad_static", "lp_sparsify", "lp_get_sparsified",
-    "lp_worker_view", "lp_get_worker_view",
+    "lp_worker_view", "lp_get_worker_view", "lp_hits_at_k", "lp_get_predictor_activations",
 ]
 
 PROF_CATEGORIES = ["agg_fwd", "agg_bwd", "gemm_fwd", "gemm_dgrad", "gemm_wgrad", "score", "incidence", "scatter",
@@ -44,7 +44,8 @@ class LpError(RuntimeError):
 class ModelDesc(C.Structure):
     _fields_ = [("arch", C.c_int32), ("n_layers", C.c_int32), ("dims", C.c_int32 * (LP_MAX_LAYERS + 1)),
                 ("prec", C.c_int32), ("fanout", C.c_int32 * LP_MAX_LAYERS), ("reject_edges", C.c_int32),
-                ("max_attempts", C.c_int32), ("cache_input_aggregation", C.c_int32)]
+                ("max_attempts", C.c_int32), ("cache_input_aggregation", C.c_int32), ("predictor", C.c_int32),
+                ("pred_hidden", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -177,7 +178,8 @@ class Context:
     # ---- model
     def set_model(self, arch: str, dims: Sequence[int], prec: str = "fp32", fanout: Optional[Sequence[int]] = None,
                   reject_edges: bool = True, max_attempts: int = 8, max_batch: int = 65536, max_k: int = 1,
-                  cache_input_aggregation: bool = False):
+                  cache_input_aggregation: bool = False, pred_hidden: int = 0):
+        """pred_hidden = 0: dot-product predictor; > 0: 3-layer MLP predictor with that hidden width."""
         d = ModelDesc()
         d.arch = LP_GCN if arch == "gcn" else LP_SAGE_MEAN
         d.n_layers = len(dims) - 1
@@ -189,6 +191,8 @@ class Context:
         d.reject_edges = int(bool(reject_edges))
         d.max_attempts = int(max_attempts)
         d.cache_input_aggregation = int(bool(cache_input_aggregation))
+        d.predictor = 1 if pred_hidden > 0 else 0
+        d.pred_hidden = int(pred_hidden)
         self._ck(self.lib.lp_set_model(self.h, C.byref(d), C.c_int64(max_batch), C.c_int32(max_k)))
         np_ = C.c_int64()
         self._ck(self.lib.lp_param_count(self.h, C.byref(np_)))
@@ -237,6 +241,13 @@ class Context:
                                    _ptr(out)))
         return out
 
+    def hits_at_k(self, pos_scores, neg_scores, k: int) -> float:
+        """Hits@K of device score vectors (float32)."""
+        out = C.c_double()
+        self._ck(self.lib.lp_hits_at_k(self.h, _ptr(pos_scores), C.c_int64(pos_scores.numel()), _ptr(neg_scores), C.c_int64(neg_scores.numel()),
+                                       C.c_int64(k), C.byref(out)))
+        return float(out.value)
+
     # ---- inspection
     def stats(self) -> Stats:
         s = Stats()
@@ -248,6 +259,12 @@ class Context:
         rows = self.n if rows is None else rows
         out = t.empty((rows, self.dims[layer]), dtype=t.float32, device=f"cuda:{self.device}")
         self._ck(self.lib.lp_get_embeddings(self.h, C.c_int32(layer), _ptr(out)))
+        return out
+
+    def predictor_activations(self, layer: int, E: int):
+        t = self._torch
+        out = t.empty((E, int(self.desc.pred_hidden)), dtype=t.float32, device=f"cuda:{self.device}")
+        self._ck(self.lib.lp_get_predictor_activations(self.h, C.c_int32(layer), C.c_int64(E), _ptr(out)))
         return out
 
     def output_gradient(self, rows: Optional[int] = None):

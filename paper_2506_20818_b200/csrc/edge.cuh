@@ -231,17 +231,17 @@ __global__ void incidence_count_kernel(int n_ids, const int *__restrict__ idmap,
 __global__ void incidence_fill_kernel(int n_ids, const int *__restrict__ idmap, const int *__restrict__ pos_src, const int *__restrict__ pos_dst,
                                       int64_t B, const int *__restrict__ neg_src, const int *__restrict__ neg_dst, int k,
                                       const float *__restrict__ g_pos, const float *__restrict__ g_neg, int *__restrict__ cursor,
-                                      int *__restrict__ inc_col, float *__restrict__ inc_val)
+                                      int *__restrict__ inc_col, float *__restrict__ inc_val, int *__restrict__ inc_edge)
 {
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= B * (1 + k)) return;
     int s, d;
     incidence_endpoints(n_ids, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, e, s, d);
-    const float g = e < B ? g_pos[e] : g_neg[e - B];
+    const float g = g_pos ? (e < B ? g_pos[e] : g_neg[e - B]) : 0.f;
     const int ps = atomicAdd(&cursor[s], 1);
     inc_col[ps] = d;
-    inc_val[ps] = g;
     const int pd = atomicAdd(&cursor[d], 1);
     inc_col[pd] = s;
-    inc_val[pd] = g;
+    if (inc_val) { inc_val[ps] = g; inc_val[pd] = g; }
+    if (inc_edge) { inc_edge[ps] = (int)e; inc_edge[pd] = (int)e; }  // MLP predictor: the entry's edge (row of dL/dz0)
 }

@@ -14,6 +14,7 @@
 #include "optim.cuh"
 #include "sparsify.cuh"
 #include "view.cuh"
+#include "predictor.cuh"
 
 // ----------------------------------------------------------------------------------------------
 // context
@@ -86,6 +87,15 @@ struct lp_ctx {
     float *partials = nullptr;          // split-K / column-sum partials
     int64_t partials_floats = 0;
     float *g_pos = nullptr, *g_neg = nullptr, *loss_partials = nullptr;
+    // MLP edge predictor
+    bool mlp = false;
+    int Hp = 0;
+    int64_t n_enc_params = 0;           // parameters of the encoder; the predictor's follow
+    int64_t off_w2 = 0, off_b2 = 0;
+    LayerBuf pred[2];                   // the two wide predictor layers (A = Z0, then P1)
+    void *P2 = nullptr, *dPa = nullptr, *dPb = nullptr, *dZ0 = nullptr;
+    float *pred_scores = nullptr;       // [E]
+    int *inc_edge = nullptr;            // edge of every incidence entry (row of dL/dz0)
     int *inc_cursor = nullptr, *inc_ptr = nullptr, *inc_col = nullptr;
     float *inc_partials = nullptr;      // 64-bit item partials of the exact gather over the incidence lists
     float *inc_val = nullptr;
@@ -618,6 +628,9 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
         if (d->arch != LP_SAGE_MEAN) return fail(ctx, LP_EUNSUPPORTED, "lp_set_model: neighbour sampling is implemented for SAGE-mean only");
         if (d->cache_input_aggregation) return fail(ctx, LP_EINVAL, "lp_set_model: cache_input_aggregation needs a full-graph model (sampled neighbourhoods change every step)");
     }
+    if (d->predictor != LP_PRED_DOT && d->predictor != LP_PRED_MLP) return fail(ctx, LP_EINVAL, "lp_set_model: unknown predictor");
+    if (d->predictor == LP_PRED_MLP && (d->pred_hidden <= 0 || d->pred_hidden % align != 0 || d->pred_hidden > 512))
+        return fail(ctx, LP_EINVAL, "lp_set_model: pred_hidden must be a multiple of 8 (FP32) or 64 (BF16), at most 512");
     if (max_batch <= 0 || max_k < 0 || max_k > 255) return fail(ctx, LP_EINVAL, "lp_set_model: max_batch must be positive, max_k in [0, 255]");
     if (d->reject_edges && (d->max_attempts < 1 || d->max_attempts > 255)) return fail(ctx, LP_EINVAL, "lp_set_model: max_attempts must be in [1, 255]");
     if (max_batch * (int64_t)(1 + max_k) * 2 >= (int64_t)1 << 31) return fail(ctx, LP_EINVAL, "lp_set_model: batch too large");
@@ -645,6 +658,18 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
         off += (int64_t)L.Kin * L.Fo;
         L.off_b = off;
         off += L.Fo;
+    }
+    ctx->n_enc_params = off;
+    ctx->mlp = d->predictor == LP_PRED_MLP;
+    ctx->Hp = ctx->mlp ? d->pred_hidden : 0;
+    if (ctx->mlp) {
+        const int Dk = d->dims[K], Hp = ctx->Hp;
+        LayerBuf &P0 = ctx->pred[0], &P1 = ctx->pred[1];
+        P0 = LayerBuf(); P1 = LayerBuf();
+        P0.Fi = P0.Kin = Dk; P0.Fo = Hp; P0.off_w = off; off += (int64_t)Dk * Hp; P0.off_b = off; off += Hp;
+        P1.Fi = P1.Kin = Hp; P1.Fo = Hp; P1.off_w = off; off += (int64_t)Hp * Hp; P1.off_b = off; off += Hp;
+        ctx->off_w2 = off; off += Hp;
+        ctx->off_b2 = off; off += 1;
     }
     ctx->n_params = off;
 
@@ -699,14 +724,31 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
     for (int i = 0; i < 2; ++i) { MALLOC(p, max_rows * maxF * (int64_t)es); ctx->dZ[i] = p; }
     MALLOC(p, max_rows * maxKin * (int64_t)es);
     ctx->dA = p;
-    ctx->partials_floats = std::max<int64_t>((int64_t)weight_grad_splits(max_rows) * maxKin * maxF, (int64_t)colsum_splits(max_rows) * maxF);
-    ctx->partials_floats = std::max<int64_t>(ctx->partials_floats, tc_weight_grad_partials(max_rows, maxKin, maxF));
+    int64_t part_rows = max_rows;
+    if (ctx->mlp) {  // the predictor's layers run over the scored edges
+        part_rows = std::max<int64_t>(part_rows, E);
+        maxKin = std::max(maxKin, std::max(d->dims[K], ctx->Hp));
+        maxF = std::max(maxF, std::max(d->dims[K], ctx->Hp));
+    }
+    ctx->partials_floats = std::max<int64_t>((int64_t)weight_grad_splits(part_rows) * maxKin * maxF, (int64_t)colsum_splits(part_rows) * (maxF + 1));
+    ctx->partials_floats = std::max<int64_t>(ctx->partials_floats, tc_weight_grad_partials(part_rows, maxKin, maxF));
     MALLOC(ctx->partials, ctx->partials_floats);
 
     // scoring and incidence
-    MALLOC(ctx->g_pos, max_batch);
+    MALLOC(ctx->g_pos, ctx->mlp ? E : max_batch);  // MLP predictor: one array for positives then negatives
     MALLOC(ctx->g_neg, max_batch * std::max<int64_t>(max_k, 1));
-    MALLOC(ctx->loss_partials, ceil_div64(max_batch, EDGE_THREADS / 32) + 1);
+    MALLOC(ctx->loss_partials, std::max<int64_t>(ceil_div64(max_batch, EDGE_THREADS / 32), ceil_div64(E, 256)) + 1);
+    if (ctx->mlp) {
+        const int Dk = d->dims[K], Hp = ctx->Hp;
+        MALLOC(p, E * Dk * (int64_t)es); ctx->pred[0].A = p;
+        MALLOC(p, E * Hp * (int64_t)es); ctx->pred[1].A = p;
+        MALLOC(p, E * Hp * (int64_t)es); ctx->P2 = p;
+        MALLOC(p, E * Hp * (int64_t)es); ctx->dPa = p;
+        MALLOC(p, E * Hp * (int64_t)es); ctx->dPb = p;
+        MALLOC(p, E * Dk * (int64_t)es); ctx->dZ0 = p;
+        MALLOC(ctx->pred_scores, E);
+        MALLOC(ctx->inc_edge, 2 * E);
+    }
     MALLOC(ctx->inc_cursor, cap_rows[0] + 1);
     MALLOC(ctx->inc_partials, (2 * E / SPMM_HEAVY_MIN + 2) * 2 * (int64_t)d->dims[K]);
     MALLOC(ctx->inc_col, 2 * E);
@@ -1037,6 +1079,61 @@ template <typename T> static lp_status forward_impl(lp_ctx *ctx, const float *pa
     return LP_OK;
 }
 
+// ---- MLP edge predictor ----------------------------------------------------------------------
+// scores of the E = B (1 + k) edges (positives, then negatives) into ctx->pred_scores; keeps z0, p1, p2
+template <typename T>
+static lp_status predictor_forward(lp_ctx *ctx, const float *params, const int *idmap, const int *pos_src, const int *pos_dst, int64_t B,
+                                   const int *neg_src, const int *neg_dst, int k)
+{
+    cudaStream_t st = ctx->ex.st;
+    const int D = ctx->desc.dims[ctx->K], Hp = ctx->Hp;
+    const int64_t E = B * (1 + (int64_t)k);
+    constexpr int VN = Vec16<T>::N;
+    const int chunks = D / VN;
+    const unsigned blocks = nblk(E, EDGE_THREADS / 32);
+    T *Z0 = tptr<T>(ctx->pred[0].A), *P1 = tptr<T>(ctx->pred[1].A), *P2 = tptr<T>(ctx->P2), *HK = tptr<T>(ctx->HK);
+    if (chunks <= 32) edge_hadamard_kernel<T, 1><<<blocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, Z0);
+    else if (chunks <= 64) edge_hadamard_kernel<T, 2><<<blocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, Z0);
+    else edge_hadamard_kernel<T, 4><<<blocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, Z0);
+    ctx->ex.launches += 1;
+    lp_status s = layer_linear<T>(ctx, E, ctx->pred[0], params, P1, Hp, true);
+    if (s != LP_OK) return s;
+    s = layer_linear<T>(ctx, E, ctx->pred[1], params, P2, Hp, true);
+    if (s != LP_OK) return s;
+    edge_gemv_kernel<T><<<blocks, EDGE_THREADS, 0, st>>>(P2, Hp, E, params + ctx->off_w2, params + ctx->off_b2, ctx->pred_scores);
+    ctx->ex.launches += 1;
+    CK_LAUNCH();
+    return LP_OK;
+}
+
+// gradients of the predictor's parameters and dL/dz0 (ctx->dZ0) from the per-edge score gradients g
+template <typename T>
+static lp_status predictor_backward(lp_ctx *ctx, const float *params, int64_t E, const float *g, float *grads, int accumulate)
+{
+    cudaStream_t st = ctx->ex.st;
+    const int Hp = ctx->Hp;
+    T *P1 = tptr<T>(ctx->pred[1].A), *P2 = tptr<T>(ctx->P2), *dPa = tptr<T>(ctx->dPa), *dPb = tptr<T>(ctx->dPb), *dZ0 = tptr<T>(ctx->dZ0);
+    // last layer: dw2 = P2^T g, db2 = sum g (two fixed-order stages)
+    const int splits = colsum_splits(E);
+    const int64_t rpb = ceil_div64(E, splits);
+    pred_last_layer_grad_kernel<T><<<splits, 256, 0, st>>>(P2, Hp, E, g, rpb, ctx->partials);
+    reduce_partials_short_kernel<<<nblk(Hp + 1, 32), 256, 0, st>>>(ctx->partials, Hp + 1, splits, grads + ctx->off_w2, accumulate);
+    pred_out_grad_kernel<T><<<nblk(E * Hp), 256, 0, st>>>(P2, Hp, E, g, params + ctx->off_w2, dPa);
+    ctx->ex.launches += 3;
+    lp_status s = layer_weight_grad<T>(ctx, E, ctx->pred[1], dPa, grads, accumulate);
+    if (s != LP_OK) return s;
+    s = layer_input_grad<T>(ctx, E, ctx->pred[1], params, dPa, dPb, nullptr, 0);
+    if (s != LP_OK) return s;
+    relu_mask_kernel<T><<<nblk(E * Hp), 256, 0, st>>>(dPb, P1, E * Hp);
+    ctx->ex.launches += 1;
+    s = layer_weight_grad<T>(ctx, E, ctx->pred[0], dPb, grads, accumulate);
+    if (s != LP_OK) return s;
+    s = layer_input_grad<T>(ctx, E, ctx->pred[0], params, dPb, dZ0, nullptr, 0);
+    if (s != LP_OK) return s;
+    CK_LAUNCH();
+    return LP_OK;
+}
+
 template <typename T>
 static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src, const int *pos_dst, int64_t B, const int *neg_src, const int *neg_dst,
                             int k, uint64_t seed, uint64_t step, float *loss, float *grads, int accumulate)
@@ -1068,10 +1165,22 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     const unsigned eblocks = nblk(B, EDGE_THREADS / 32);
     constexpr int VN = Vec16<T>::N;
     const int chunks = D / VN;
-    if (chunks <= 32) edge_score_bce_kernel<T, 1><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials);
-    else if (chunks <= 64) edge_score_bce_kernel<T, 2><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials);
-    else edge_score_bce_kernel<T, 4><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials);
-    loss_reduce_kernel<<<1, 256, 0, st>>>(ctx->loss_partials, eblocks, inv_N, loss);
+    const float *g_pos = ctx->g_pos, *g_neg = ctx->g_neg;
+    if (ctx->mlp) {
+        s = predictor_forward<T>(ctx, params, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k);
+        if (s != LP_OK) { delete pscore; return s; }
+        const unsigned lblocks = nblk(E, 256);
+        bce_from_scores_kernel<<<lblocks, 256, 0, st>>>(ctx->pred_scores, E, B, inv_N, ctx->g_pos, ctx->loss_partials);
+        loss_reduce_kernel<<<1, 256, 0, st>>>(ctx->loss_partials, lblocks, inv_N, loss);
+        g_neg = ctx->g_pos + B;  // one array: positives, then negatives
+        s = predictor_backward<T>(ctx, params, E, ctx->g_pos, grads, accumulate);
+        if (s != LP_OK) { delete pscore; return s; }
+    } else {
+        if (chunks <= 32) edge_score_bce_kernel<T, 1><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials);
+        else if (chunks <= 64) edge_score_bce_kernel<T, 2><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials);
+        else edge_score_bce_kernel<T, 4><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials);
+        loss_reduce_kernel<<<1, 256, 0, st>>>(ctx->loss_partials, eblocks, inv_N, loss);
+    }
     delete pscore;
     ctx->ex.launches += 2;
 
@@ -1081,8 +1190,8 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     incidence_count_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->inc_ptr);
     exclusive_scan_i32(ctx->ex, ctx->inc_ptr, rows_out, ctx->inc_ptr, ctx->inc_ptr + rows_out, ctx->scan_tmp);
     CK(cudaMemcpyAsync(ctx->inc_cursor, ctx->inc_ptr, sizeof(int) * (size_t)rows_out, cudaMemcpyDeviceToDevice, st));
-    incidence_fill_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->g_pos, ctx->g_neg, ctx->inc_cursor, ctx->inc_col,
-                                                   ctx->inc_val);
+    incidence_fill_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, g_pos, g_neg, ctx->inc_cursor, ctx->inc_col,
+                                                   ctx->mlp ? nullptr : ctx->inc_val, ctx->mlp ? ctx->inc_edge : nullptr);
     ctx->ex.launches += 2;
     delete pinc;
 
@@ -1097,12 +1206,18 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         a.n_rows = rows_out;
         a.rowptr = ctx->inc_ptr;
         a.col = ctx->inc_col;
-        a.val = ctx->inc_val;
         a.X = HK;
         a.ldx = D;
         a.F = D;
         a.Y = dZ;
         a.ldy = D;
+        if (ctx->mlp) {  // dL/dh_node = sum over incident edges of dL/dz0[edge] * h_other
+            a.X2 = tptr<T>(ctx->dZ0);
+            a.ldx2 = D;
+            a.col2 = ctx->inc_edge;
+        } else {         // dot product: g_e * h_other
+            a.val = ctx->inc_val;
+        }
         ProfScope prof(ctx->ex, LP_PROF_SCATTER, spmm_bytes(a, 2 * E), 4.0 * E * D);
         // the order of a node's entries is not reproducible, so the sum is taken exactly (64-bit fixed point)
         if (rows_out > 0 && !spmm_launch<T, long long>(ctx->ex, a)) return fail(ctx, LP_EUNSUPPORTED, "embedding width not supported");
@@ -1275,6 +1390,16 @@ static lp_status score_impl(lp_ctx *ctx, const float *params, const int *src, co
     const int *idmap = ctx->sampled ? ctx->hop[0].posmap : nullptr;
     constexpr int VN = Vec16<T>::N;
     const int chunks = D / VN;
+    if (ctx->mlp) {  // in pieces of at most the predictor's buffer size
+        const int64_t cap = ctx->max_batch * (1 + (int64_t)ctx->max_k);
+        for (int64_t off = 0; off < E; off += cap) {
+            const int64_t m = std::min<int64_t>(cap, E - off);
+            s = predictor_forward<T>(ctx, params, idmap, src + off, dst + off, m, nullptr, nullptr, 0);
+            if (s != LP_OK) return s;
+            CK(cudaMemcpyAsync(scores + off, ctx->pred_scores, sizeof(float) * (size_t)m, cudaMemcpyDeviceToDevice, ctx->ex.st));
+        }
+        return LP_OK;
+    }
     const unsigned blocks = nblk(E, EDGE_THREADS / 32);
     if (chunks <= 32) edge_score_kernel<T, 1><<<blocks, EDGE_THREADS, 0, ctx->ex.st>>>(tptr<T>(ctx->HK), D, D, ctx->n, idmap, src, dst, E, scores);
     else if (chunks <= 64) edge_score_kernel<T, 2><<<blocks, EDGE_THREADS, 0, ctx->ex.st>>>(tptr<T>(ctx->HK), D, D, ctx->n, idmap, src, dst, E, scores);
@@ -1297,6 +1422,42 @@ extern "C" lp_status lp_score(lp_ctx *ctx, const float *params, const int32_t *s
                                             : score_impl<float>(ctx, params, src, dst, E, seed, step, scores);
     if (s != LP_OK) return s;
     return tc_check(ctx->tc, ctx->ex, false, ctx->err);
+}
+
+extern "C" lp_status lp_hits_at_k(lp_ctx *ctx, const float *pos_scores, int64_t n_pos, const float *neg_scores, int64_t n_neg, int64_t K, double *hits)
+{
+    if (!ctx || !hits) return LP_EINVAL;
+    if (!pos_scores || n_pos <= 0 || (n_neg > 0 && !neg_scores) || n_neg < 0 || K <= 0 || n_neg >= ((int64_t)1 << 31))
+        return fail(ctx, LP_EINVAL, "lp_hits_at_k: bad argument");
+    if (n_neg < K) { *hits = 1.0; return LP_OK; }
+    CK(cudaSetDevice(ctx->device));
+    cudaStream_t st = ctx->ex.st;
+    std::vector<void *> tmp;
+    int64_t tmp_bytes = 0;
+    uint32_t *keys = nullptr, *vals = nullptr;
+    unsigned long long *count = nullptr;
+    SortScratch sc;
+    cudaError_t e = dev_alloc(ctx, tmp, tmp_bytes, &keys, n_neg);
+    if (e == cudaSuccess) e = dev_alloc(ctx, tmp, tmp_bytes, &vals, n_neg);
+    if (e == cudaSuccess) e = dev_alloc(ctx, tmp, tmp_bytes, &sc.keys_alt, n_neg);
+    if (e == cudaSuccess) e = dev_alloc(ctx, tmp, tmp_bytes, &sc.vals_alt, n_neg);
+    if (e == cudaSuccess) e = dev_alloc(ctx, tmp, tmp_bytes, &sc.hist, SortScratch::hist_ints(n_neg));
+    if (e == cudaSuccess) e = dev_alloc(ctx, tmp, tmp_bytes, &sc.scan_tmp, SortScratch::scan_ints(n_neg));
+    if (e == cudaSuccess) e = dev_alloc(ctx, tmp, tmp_bytes, &count, 8);
+    if (e != cudaSuccess) { free_list(tmp); CK(e); }
+    float_keys_kernel<<<nblk(n_neg), 256, 0, st>>>(neg_scores, n_neg, keys, vals);
+    const bool in_place = radix_sort_pairs(ctx->ex, keys, vals, n_neg, 32, sc);  // ascending
+    cudaMemsetAsync(count, 0, sizeof(unsigned long long), st);
+    count_above_kernel<<<nblk(n_pos), 256, 0, st>>>(pos_scores, n_pos, in_place ? keys : sc.keys_alt, n_neg - K, count);
+    ctx->ex.launches += 2;
+    unsigned long long h = 0;
+    e = cudaMemcpyAsync(&h, count, sizeof h, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    free_list(tmp);
+    CK(e);
+    CK_LAUNCH();
+    *hits = (double)h / (double)n_pos;
+    return LP_OK;
 }
 
 // ----------------------------------------------------------------------------------------------
@@ -1325,6 +1486,19 @@ extern "C" lp_status lp_get_embeddings(lp_ctx *ctx, int32_t layer, float *out)
     else if (ctx->desc.arch == LP_SAGE_MEAN) { src = ctx->layer[layer].A; ld = ctx->layer[layer].Kin; rows = ctx->n; }
     else { src = ctx->layer[layer].Hin; ld = F; rows = ctx->n; }
     if (b16) to_f32<bf16>(ctx, (const bf16 *)src, ld, out, rows, F); else to_f32<float>(ctx, (const float *)src, ld, out, rows, F);
+    CK_LAUNCH();
+    return LP_OK;
+}
+
+extern "C" lp_status lp_get_predictor_activations(lp_ctx *ctx, int32_t layer, int64_t E, float *out)
+{
+    if (!ctx || !out) return LP_EINVAL;
+    if (!ctx->model_set || !ctx->mlp || !ctx->have_forward) return fail(ctx, LP_ESTATE, "lp_get_predictor_activations: no MLP predictor pass has run");
+    if (layer < 1 || layer > 2 || E <= 0 || E > ctx->max_batch * (1 + (int64_t)ctx->max_k)) return fail(ctx, LP_EINVAL, "lp_get_predictor_activations: bad layer or E");
+    CK(cudaSetDevice(ctx->device));
+    const void *src = layer == 1 ? ctx->pred[1].A : ctx->P2;
+    if (ctx->desc.prec == LP_BF16) to_f32<bf16>(ctx, (const bf16 *)src, ctx->Hp, out, E, ctx->Hp);
+    else to_f32<float>(ctx, (const float *)src, ctx->Hp, out, E, ctx->Hp);
     CK_LAUNCH();
     return LP_OK;
 }

@@ -42,6 +42,9 @@ template <typename T> struct SpmmArgs {
     const float *row_scale = nullptr;
     const T *X = nullptr;
     int ldx = 0;
+    const T *X2 = nullptr;       // optional second operand: entry e contributes X[col[e], :] * X2[col2[e], :] (element-wise)
+    int ldx2 = 0;
+    const int *col2 = nullptr;
     int F = 0;
     T *Y = nullptr;
     int ldy = 0;
@@ -101,7 +104,7 @@ constexpr int SPMM_SEG = 512;    // entries per item (one block: 8 lane groups x
 // acc += sum over entries [e_lo, e_hi) of val[e] * X[col[e], :] for the chunks owned by this lane.
 // The group loads up to G (col, val) pairs at once and broadcasts them; U source rows are gathered
 // before any is consumed, so each lane keeps U * NV 16-byte loads in flight.
-template <typename T, int G, int NV, int U, typename ACC, bool HAS_VAL>
+template <typename T, int G, int NV, int U, typename ACC, bool HAS_VAL, bool HAS_X2 = false>
 LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl, unsigned gmask, int nchunks, ACC (&acc)[NV][Vec16<T>::N],
                                 bool have_first = false, int first_col = 0, float first_val = 0.f)
 {
@@ -118,6 +121,8 @@ LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl,
                 if (HAS_VAL) my_val = __ldg(a.val + my_e);
             }
         }
+        int my_col2 = 0;
+        if (HAS_X2 && my_e < e_hi) my_col2 = __ldg(a.col2 + my_e);
         const int cnt = min(G, e_hi - e0);
         int j = 0;
         for (; j + U <= cnt; j += U) {
@@ -136,24 +141,55 @@ LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl,
                     const int ch = gl + i * G;
                     if (ch < nchunks) v[q][i].load(a.X + (size_t)c[q] * a.ldx + ch * VN);
                 }
+            if (HAS_X2) {
 #pragma unroll
-            for (int q = 0; q < U; ++q)
+                for (int q = 0; q < U; ++q) {
+                    const int c2 = __shfl_sync(gmask, my_col2, j + q, G);
 #pragma unroll
-                for (int i = 0; i < NV; ++i) {
-                    const int ch = gl + i * G;
-                    if (ch < nchunks) acc_add_vec<T, ACC, HAS_VAL>(acc[i], w[q], v[q][i]);
+                    for (int i = 0; i < NV; ++i) {
+                        const int ch = gl + i * G;
+                        if (ch < nchunks) {
+                            Vec16<T> v2;
+                            v2.load(a.X2 + (size_t)c2 * a.ldx2 + ch * VN);
+                            float f[VN], f2[VN];
+                            v[q][i].to_float(f);
+                            v2.to_float(f2);
+#pragma unroll
+                            for (int t = 0; t < VN; ++t) acc_add<ACC>(acc[i][t], w[q], f[t] * f2[t]);
+                        }
+                    }
                 }
+            } else {
+#pragma unroll
+                for (int q = 0; q < U; ++q)
+#pragma unroll
+                    for (int i = 0; i < NV; ++i) {
+                        const int ch = gl + i * G;
+                        if (ch < nchunks) acc_add_vec<T, ACC, HAS_VAL>(acc[i], w[q], v[q][i]);
+                    }
+            }
         }
         for (; j < cnt; ++j) {
             const int c = __shfl_sync(gmask, my_col, j, G);
             const float w = HAS_VAL ? __shfl_sync(gmask, my_val, j, G) : 1.f;
+            const int c2 = HAS_X2 ? __shfl_sync(gmask, my_col2, j, G) : 0;
 #pragma unroll
             for (int i = 0; i < NV; ++i) {
                 const int ch = gl + i * G;
                 if (ch < nchunks) {
                     Vec16<T> v;
                     v.load(a.X + (size_t)c * a.ldx + ch * VN);
-                    acc_add_vec<T, ACC, HAS_VAL>(acc[i], w, v);
+                    if (HAS_X2) {
+                        Vec16<T> v2;
+                        v2.load(a.X2 + (size_t)c2 * a.ldx2 + ch * VN);
+                        float f[VN], f2[VN];
+                        v.to_float(f);
+                        v2.to_float(f2);
+#pragma unroll
+                        for (int t = 0; t < VN; ++t) acc_add<ACC>(acc[i][t], w, f[t] * f2[t]);
+                    } else {
+                        acc_add_vec<T, ACC, HAS_VAL>(acc[i], w, v);
+                    }
                 }
             }
         }
@@ -207,7 +243,7 @@ LP_DEVINL void spmm_epilogue(const SpmmArgs<T> &a, int r, int gl, int nchunks, c
     }
 }
 
-template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC, bool HAS_VAL>
+template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC, bool HAS_VAL, bool HAS_X2>
 __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const SpmmArgs<T> a, const int light_blocks)
 {
     constexpr int VN = Vec16<T>::N;
@@ -237,7 +273,7 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
         for (int q = 0; q < NV; ++q)
 #pragma unroll
             for (int j = 0; j < VN; ++j) hacc[q][j] = ACC(0);
-        spmm_accumulate<T, G, NV, U, ACC, HAS_VAL>(a, lo, hi, gl, gmask, nchunks, hacc);
+        spmm_accumulate<T, G, NV, U, ACC, HAS_VAL, HAS_X2>(a, lo, hi, gl, gmask, nchunks, hacc);
 #pragma unroll
         for (int q = 0; q < NV; ++q)
 #pragma unroll
@@ -291,7 +327,7 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
             for (int i = 0; i < NV; ++i)
 #pragma unroll
                 for (int j = 0; j < VN; ++j) acc[i][j] = ACC(0);
-            spmm_accumulate<T, G, NV, U, ACC, HAS_VAL>(a, e_begin, e_end, gl, gmask, nchunks, acc, true, cur_col, cur_val);
+            spmm_accumulate<T, G, NV, U, ACC, HAS_VAL, HAS_X2>(a, e_begin, e_end, gl, gmask, nchunks, acc, !HAS_X2, cur_col, cur_val);
             spmm_epilogue<T, G, NV, ACC>(a, r, gl, nchunks, acc);
         }
     }
@@ -362,8 +398,18 @@ template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC> sta
         ex.launches += 1;
     }
     const int item_blocks = (int)std::min<int64_t>(items, SPMM_ITEM_BLOCKS);
-    if (a.val) spmm_csr_kernel<T, G, NV, RPG, U, MINB, ACC, true><<<(unsigned)(light_blocks + item_blocks), SPMM_THREADS, 0, ex.st>>>(a, light_blocks);
-    else spmm_csr_kernel<T, G, NV, RPG, U, MINB, ACC, false><<<(unsigned)(light_blocks + item_blocks), SPMM_THREADS, 0, ex.st>>>(a, light_blocks);
+    const unsigned grid = (unsigned)(light_blocks + item_blocks);
+    bool launched = false;
+    if constexpr (sizeof(ACC) == 8) {  // the two-operand form exists for the exact accumulator only
+        if (a.X2) {
+            spmm_csr_kernel<T, G, NV, RPG, U, MINB, ACC, false, true><<<grid, SPMM_THREADS, 0, ex.st>>>(a, light_blocks);
+            launched = true;
+        }
+    }
+    if (!launched) {
+        if (a.val) spmm_csr_kernel<T, G, NV, RPG, U, MINB, ACC, true, false><<<grid, SPMM_THREADS, 0, ex.st>>>(a, light_blocks);
+        else spmm_csr_kernel<T, G, NV, RPG, U, MINB, ACC, false, false><<<grid, SPMM_THREADS, 0, ex.st>>>(a, light_blocks);
+    }
     ex.launches += 1;
     if (a.heavy.host_rows != 0) {
         const int64_t rows_bound = a.heavy.host_rows > 0 ? a.heavy.host_rows : std::max<int64_t>(1, items);
@@ -390,6 +436,7 @@ template <typename T, typename ACC = float> static bool spmm_launch(Exec &ex, co
 {
     constexpr int VN = Vec16<T>::N;
     if (a.F <= 0 || a.F % VN != 0 || !a.heavy.counts || !a.heavy.partials) return false;
+    if (a.X2 && (sizeof(ACC) != 8 || a.val || !a.col2)) return false;
     const int chunks = a.F / VN;
     if (chunks <= 8) spmm_launch_gn<T, 8, 1, ACC>(ex, a);
     else if (chunks <= 16) spmm_launch_gn<T, 16, 1, ACC>(ex, a);

@@ -36,8 +36,8 @@ def test_binding_covers_header():
 
 def test_struct_layouts_match_header():
     import paper_2506_20818_b200 as pkg
-    # lp_model_desc: 2 + 5 + 1 + 4 + 3 int32; lp_stats: 1 + 5 + 4 + 2 int64
-    assert ctypes.sizeof(pkg.ModelDesc) == 4 * 15
+    # lp_model_desc: 2 + 5 + 1 + 4 + 5 int32; lp_stats: 1 + 5 + 4 + 2 int64
+    assert ctypes.sizeof(pkg.ModelDesc) == 4 * 17
     assert ctypes.sizeof(pkg.Stats) == 8 * 12
 
 

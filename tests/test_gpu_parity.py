@@ -626,3 +626,75 @@ def test_worker_views_match_oracle(pkg):
     _, _, s2 = ctx.worker_view(dpart, 0, True, 2)
     assert s1["foreign_entries"] < 0.45 * s2["foreign_entries"]
     ctx.close()
+
+
+# ------------------------------------------------------------------------------------------ MLP edge predictor, Hits@K
+@pytest.mark.parametrize("arch,prec,fanout", [("sage", "fp32", None), ("gcn", "fp32", None), ("sage", "bf16", None), ("sage", "fp32", [4, 3])])
+def test_mlp_predictor_step(pkg, arch, prec, fanout):
+    if fanout:
+        g = wl.citation_directed(5000, 60000, 2.2, seed=5)
+        rows = np.repeat(np.arange(g.n, dtype=np.int32), np.diff(g.rowptr))
+        sel = np.random.default_rng(3).choice(g.nnz, 900, replace=False)
+        u, v = g.col[sel].copy(), rows[sel].copy()
+    else:
+        g = wl.chung_lu(6000, 14.0, 2.1, seed=5)
+        pu, pv = wl.undirected_edge_list(g)
+        sel = np.random.default_rng(3).choice(len(pu), 2500, replace=False)
+        u, v = pu[sel].copy(), pv[sel].copy()
+    dims, Hp, k = [64, 128, 64], 128, 2
+    X = wl.node_features(g.n, 64, 1)
+    params = wl.glorot_params(arch, dims, 2, bias_scale=0.05, pred_hidden=Hp)
+    ctx = make_ctx(pkg, g, X)
+    assert ctx.set_model(arch, dims, prec=prec, fanout=fanout, max_batch=len(u), max_k=k, pred_hidden=Hp) == len(params)
+    du, dv, p = t32(u), t32(v), t32(params)
+    seed, step = 21, 4
+    _, nd = ctx.sample_negatives(seed, step, k, du)
+    loss, grads = torch.zeros(1, device=DEV), torch.full((len(params),), 3.0, device=DEV)
+    ctx.train_step(p, du, dv, None, nd, k, loss, grads, seed=seed, step=step)
+    torch.cuda.synchronize()
+    ons, ond, _ = oracle.sample_negatives(g.n, g.rowptr, g.col, u, seed, step, k)
+    assert np.array_equal(nd.cpu().numpy(), ond)
+    blocks = oracle.build_blocks(g.n, g.rowptr, g.col, np.concatenate([u, v, ond]), fanout, seed, step) if fanout else None
+    rows0 = blocks[0][0] if fanout else np.arange(g.n)
+    ties = None
+    if not fanout:
+        ties = [ctx.embeddings(1).cpu().numpy() > 0]
+    E = len(u) * (1 + k)
+    pred_ties = [ctx.predictor_activations(1, E).cpu().numpy() > 0, ctx.predictor_activations(2, E).cpu().numpy() > 0]
+    ref = oracle.train_step(g, X, params, arch, dims, u, v, ons, ond, blocks=blocks, relu_ties=ties, tie_tol=TOL[prec], pred_hidden=Hp,
+                            pred_ties=pred_ties)
+    assert ref["pred_cache"]["ties"] <= (8 if prec == "fp32" else 0.01 * 2 * E * Hp)
+    n_enc = oracle.encoder_param_count(arch, dims)
+    gg = grads.cpu().numpy()
+    err = {"loss": abs(loss.item() - ref["loss"]) / abs(ref["loss"]),
+           "HK": rel_l2(ctx.embeddings(2, rows=len(rows0)).cpu().numpy(), ref["cache"]["H"][2][rows0]),
+           "dHK": rel_l2(ctx.output_gradient(rows=len(rows0)).cpu().numpy(), ref["dHK"][rows0]),
+           "enc_grads": rel_l2(gg[:n_enc], ref["grads"][:n_enc]),
+           "pred_grads": rel_l2(gg[n_enc:], ref["grads"][n_enc:])}
+    D = dims[-1]
+    o = n_enc
+    for name, size in (("W0", D * Hp), ("b0", Hp), ("W1", Hp * Hp), ("b1", Hp), ("w2", Hp), ("b2", 1)):
+        err["d" + name] = rel_l2(gg[o:o + size], ref["grads"][o:o + size])
+        o += size
+    tol = TOL[prec]
+    bad = {kk: e for kk, e in err.items() if not e < tol}
+    assert not bad, f"outside {tol}: {bad} (all {err})"
+    # scores through lp_score agree with the oracle's predictor
+    s_gpu = ctx.score(p, du, dv, seed=seed, step=step).cpu().numpy()
+    s_ref = oracle.score(g, X, params, arch, dims, u, v, blocks=oracle.build_blocks(g.n, g.rowptr, g.col, np.concatenate([u, v]), fanout, seed, step) if fanout else None, pred_hidden=Hp)
+    assert rel_l2(s_gpu, s_ref) < (2e-2 if prec == "bf16" else 1e-5)
+    ctx.close()
+
+
+def test_hits_at_k(pkg):
+    g = wl.erdos_renyi(50, 100, seed=0)
+    ctx = make_ctx(pkg, g, wl.node_features(g.n, 8, 0))
+    rng = np.random.default_rng(0)
+    pos = rng.standard_normal(5000).astype(np.float32)
+    neg = np.concatenate([rng.standard_normal(300000), [0.0, -0.0, 1.5, 1.5]]).astype(np.float32)
+    for k in (1, 100, 5000, len(neg)):
+        assert ctx.hits_at_k(t32(pos), t32(neg), k) == oracle.hits_at_k(pos, neg, k)
+    assert ctx.hits_at_k(t32(pos), t32(neg[:50]), 100) == 1.0
+    small_pos, small_neg = np.array([2.0, 0.0, -0.0], dtype=np.float32), np.array([1.0, 2.0, 3.0, 0.0], dtype=np.float32)
+    assert ctx.hits_at_k(t32(small_pos), t32(small_neg), 3) == oracle.hits_at_k(small_pos, small_neg, 3)
+    ctx.close()
