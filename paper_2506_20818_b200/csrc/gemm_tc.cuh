@@ -42,6 +42,7 @@ constexpr unsigned long long TC_WAIT_LIMIT_NS = 2000000000ull;  // every mbarrie
 LP_DEVINL uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 LP_DEVINL void mbar_init(uint32_t bar, uint32_t count) { asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory"); }
+LP_DEVINL void mbar_arrive(uint32_t bar) { asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory"); }
 LP_DEVINL void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -184,7 +185,9 @@ struct TcGemmParams {
     int scale_col0;          // (the 1 / |N(v)| of the mean adjoint, folded into the input-gradient transform)
     bf16 *C;            // output (BF16) when out_f32 == null
     int64_t ldc;
-    float *out_f32;     // FP32 partial output [gridDim.z][M_tiles * 128, N] (weight gradient)
+    float *out_f32;     // FP32 partial output [gridDim.z][M + colsum, N] (weight gradient)
+    int colsum;         // weight gradient only: 1 = row M of every partial tile receives the column sums of the B operand
+                        // over the split's rows (the bias gradient), taken from the staged tiles by the otherwise idle warps
     int64_t rows;       // weight gradient: reduction length; rows_per_split rows per blockIdx.z
     int64_t rows_per_split;
     int *err;
@@ -218,11 +221,14 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
     const int num_kb = (int)((k_end - k_begin + TC_BK - 1) / TC_BK);
     const int m0 = blockIdx.x * TC_BM;
     const int n0 = blockIdx.y * BN;
+    // the CTAs of the first M tile also sum the columns of their B tiles (warps 2 and 3)
+    const bool do_colsum = MN_MAJOR && p.colsum != 0 && blockIdx.x == 0;
+    const int64_t part_rows = p.M + (MN_MAJOR && p.colsum != 0 ? 1 : 0);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(smem_u32(&bar_full[s]), 1);
-            mbar_init(smem_u32(&bar_empty[s]), 1);
+            mbar_init(smem_u32(&bar_empty[s]), do_colsum ? 3 : 1);  // the MMA commit, plus one lane of each summing warp
         }
         mbar_init(smem_u32(&bar_acc), 1);
         abort_s = 0;
@@ -296,6 +302,41 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
                 umma_commit(smem_u32(&bar_empty[s]));  // frees the stage when these MMAs have read it
             }
             if (ok) umma_commit(smem_u32(&bar_acc));   // accumulator complete
+        } else if (do_colsum && warp >= 2) {
+            // ---- column sums of the B tiles (bias gradient): thread t owns columns 4t .. 4t+3 of the N tile.
+            // A staged B tile is BN / 64 boxes of 64 reduction rows x 128 bytes; the 16-byte piece c of row k
+            // sits at piece c ^ (k & 7) (128-byte swizzle).  Rows are added in order, so the sum is reproducible.
+            const int t = threadIdx.x - 64;
+            const int c4 = t * 4;
+            const bool active = c4 < BN;
+            const uint32_t box_off = (uint32_t)(c4 >> 6) * 8192u;
+            const uint32_t piece = (uint32_t)((c4 & 63) >> 3), within = (uint32_t)(c4 & 7) * 2u;
+            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+            bool ok = true;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % S;
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_full[s]), (kb / S) & 1));
+                if (!ok) {
+                    if (lane == 0) atomicExch(p.err, 4);
+                    abort_s = 1;
+                    break;
+                }
+                if (active) {
+                    const uint8_t *sb = smem + (size_t)s * stage_bytes + a_bytes + box_off;
+#pragma unroll 8
+                    for (int k = 0; k < TC_BK; ++k) {
+                        const uint2 v = *reinterpret_cast<const uint2 *>(sb + k * 128 + (((piece ^ (uint32_t)(k & 7)) << 4) | within));
+                        s0 += __uint_as_float(v.x << 16);
+                        s1 += __uint_as_float(v.x & 0xffff0000u);
+                        s2 += __uint_as_float(v.y << 16);
+                        s3 += __uint_as_float(v.y & 0xffff0000u);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bar_empty[s]));  // this warp has read the stage
+            }
+            if (ok && active)
+                *reinterpret_cast<float4 *>(p.out_f32 + ((int64_t)blockIdx.z * part_rows + p.M) * p.N + n0 + c4) = make_float4(s0, s1, s2, s3);
         }
         __syncwarp();
 
@@ -313,7 +354,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
                 tmem_ld_32x32(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
                 if (p.out_f32) {
                     // FP32 partial tile of the weight gradient: [split][row][N]
-                    float *dst = p.out_f32 + ((int64_t)blockIdx.z * p.M + row) * p.N + n0 + c0;
+                    float *dst = p.out_f32 + ((int64_t)blockIdx.z * part_rows + row) * p.N + n0 + c0;
                     if (row < p.M) {
 #pragma unroll
                         for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4 *>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
@@ -346,7 +387,9 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
         // empty reduction range: the partial tile is zero
         const int64_t row = (int64_t)m0 + threadIdx.x;
         if (row < p.M)
-            for (int c = 0; c < BN; ++c) p.out_f32[((int64_t)blockIdx.z * p.M + row) * p.N + n0 + c] = 0.f;
+            for (int c = 0; c < BN; ++c) p.out_f32[((int64_t)blockIdx.z * part_rows + row) * p.N + n0 + c] = 0.f;
+        if (do_colsum)
+            for (int c = threadIdx.x; c < BN; c += TC_THREADS) p.out_f32[((int64_t)blockIdx.z * part_rows + p.M) * p.N + n0 + c] = 0.f;
     }
     tc_fence_before();
     __syncthreads();
@@ -384,7 +427,6 @@ LP_DEVINL void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.re
 LP_DEVINL void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 LP_DEVINL void epilogue_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }  // the eight epilogue warps only
 
-LP_DEVINL void mbar_arrive(uint32_t bar) { asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory"); }
 
 __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(const __grid_constant__ CUtensorMap mapA,
                                                                               const __grid_constant__ CUtensorMap mapB,
@@ -626,7 +668,7 @@ static lp_status tc_check(TcState &tc, Exec &ex, bool synced, std::string &err)
     cudaStreamSynchronize(ex.st);
     if (*tc.host_err != 0) {
         char buf[128];
-        snprintf(buf, sizeof buf, "tensor-core GEMM: bounded wait %d expired (1 = stage free, 2 = operands, 3 = accumulator)", *tc.host_err);
+        snprintf(buf, sizeof buf, "tensor-core GEMM: bounded wait %d expired (1 = stage free, 2 = operands, 3 = accumulator, 4 = operands for the column sums)", *tc.host_err);
         err = buf;
         cudaMemsetAsync(tc.err_word, 0, sizeof(int), ex.st);
         return LP_ETIMEOUT;
@@ -762,6 +804,36 @@ static bool tc_linear_bf16_b(TcState &tc, Exec &ex, int64_t M, int N, int K, con
     return tc_gemm_kmajor(tc, ex, M, N, K, A, lda, Bt, bias, relu, C, ldc, err);
 }
 
+// dst[i] = (accumulate ? dst[i] : 0) + sum_z partials[z][i]: a block covers 64 consecutive elements, its four
+// thread rows each add a quarter of the splits in index order, and the quarters are added in order
+__global__ void __launch_bounds__(256) reduce_partials_wide_kernel(const float *__restrict__ partials, int64_t count, int splits, float *__restrict__ dst,
+                                                                   int accumulate)
+{
+    __shared__ float part[4][64];
+    const int e = threadIdx.x & 63, q = threadIdx.x >> 6;
+    const int64_t i = (int64_t)blockIdx.x * 64 + e;
+    const int per = (splits + 3) / 4;
+    const int z0 = q * per, z1 = min(splits, z0 + per);
+    float s = 0.f;
+    if (i < count) {
+        int z = z0;
+        for (; z + 8 <= z1; z += 8) {
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = __ldg(partials + (int64_t)(z + u) * count + i);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) s += v[u];
+        }
+        for (; z < z1; ++z) s += __ldg(partials + (int64_t)z * count + i);
+    }
+    part[q][e] = s;
+    __syncthreads();
+    if (q == 0 && i < count) {
+        const float r = ((part[0][e] + part[1][e]) + part[2][e]) + part[3][e];
+        dst[i] = accumulate ? dst[i] + r : r;
+    }
+}
+
 // weight gradient: dW[Kin, N] (+)= A[rows, Kin]^T dZ[rows, N]; partial tiles per row split, then a
 // fixed-order reduction
 static int tc_weight_grad_splits(int64_t rows, int Kin, int N)
@@ -774,11 +846,13 @@ static int tc_weight_grad_splits(int64_t rows, int Kin, int N)
 static int64_t tc_weight_grad_partials(int64_t rows, int Kin, int N)
 {
     if (!tc_weight_grad_supported(Kin, N)) return 0;
-    return (int64_t)tc_weight_grad_splits(rows, Kin, N) * Kin * N;
+    return (int64_t)tc_weight_grad_splits(rows, Kin, N) * (Kin + 1) * N;
 }
 
+// With fuse_bias the N floats that follow dW receive the column sums of dZ (the bias gradient): the
+// partial tiles get one more row, filled by the first M tile's CTAs, and one reduction serves both.
 static bool tc_weight_grad(TcState &tc, Exec &ex, int64_t rows, int Kin, int N, const bf16 *A, int lda, const bf16 *dZ, int ldz, float *dW, int accumulate,
-                           float *partials, std::string &err)
+                           float *partials, std::string &err, bool fuse_bias = false)
 {
     const int BN = tc_pick_bn(N);
     const int splits = tc_weight_grad_splits(rows, Kin, N);
@@ -791,11 +865,12 @@ static bool tc_weight_grad(TcState &tc, Exec &ex, int64_t rows, int Kin, int N, 
     p.rows_per_split = ceil_div64(ceil_div64(rows, splits), TC_BK) * TC_BK;
     p.stages = tc_stages(BN, (int)(p.rows_per_split / TC_BK));
     p.bias = nullptr; p.relu = 0; p.C = nullptr; p.ldc = 0; p.out_f32 = partials; p.err = tc.err_word;
+    p.colsum = fuse_bias ? 1 : 0;
     const size_t smem = (size_t)p.stages * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024;
     dim3 grid((unsigned)(Kin / TC_BM), (unsigned)(N / BN), (unsigned)splits);
     tc_gemm_kernel<true><<<grid, TC_THREADS, smem, ex.st>>>(mapA, mapB, p);
-    const int64_t count = (int64_t)Kin * N;
-    reduce_partials_kernel<<<(unsigned)ceil_div64(count, 256), 256, 0, ex.st>>>(partials, count, splits, dW, accumulate);
+    const int64_t count = (int64_t)(Kin + (fuse_bias ? 1 : 0)) * N;
+    reduce_partials_wide_kernel<<<(unsigned)ceil_div64(count, 64), 256, 0, ex.st>>>(partials, count, splits, dW, accumulate);
     ex.launches += 2;
     return true;
 }

@@ -913,8 +913,12 @@ static lp_status layer_weight_grad(lp_ctx *ctx, int64_t rows, const LayerBuf &L,
     ProfScope prof(ctx->ex, LP_PROF_GEMM_WGRAD, (double)rows * (L.Kin + 2.0 * L.Fo) * sizeof(T) + 4.0 * (L.Kin + 1.0) * L.Fo, 2.0 * rows * L.Fo * (L.Kin + 1.0));
     if (sizeof(T) == 2 && tc_weight_grad_supported(L.Kin, L.Fo)) {
         std::string err;
-        if (!tc_weight_grad(ctx->tc, ctx->ex, rows, L.Kin, L.Fo, (const bf16 *)L.A, L.Kin, (const bf16 *)dZ, L.Fo, grads + L.off_w, accumulate, ctx->partials, err))
+        // the bias gradient follows the weights in the flat vector: one launch pair produces both
+        const bool fuse_bias = L.off_b == L.off_w + (int64_t)L.Kin * L.Fo;
+        if (!tc_weight_grad(ctx->tc, ctx->ex, rows, L.Kin, L.Fo, (const bf16 *)L.A, L.Kin, (const bf16 *)dZ, L.Fo, grads + L.off_w, accumulate, ctx->partials, err,
+                            fuse_bias))
             return fail(ctx, LP_ECUDA, "tensor-core GEMM: " + err);
+        if (fuse_bias) return LP_OK;
     } else {
         weight_grad_simt<T>(ctx->ex, rows, L.Kin, L.Fo, (const T *)L.A, L.Kin, dZ, L.Fo, grads + L.off_w, accumulate, ctx->partials);
     }
