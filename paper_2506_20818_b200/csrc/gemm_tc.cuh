@@ -33,6 +33,7 @@ constexpr int TC_BM = 128;          // accumulator rows (UMMA M)
 constexpr int TC_BK = 64;           // K elements per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int TC_UMMA_K = 16;       // K per tcgen05.mma for 16-bit operands
 constexpr int TC_THREADS = 128;
+constexpr int TC_COLSUM_BOXES = 4;  // 64-column boxes of the B tile one CTA may have to add up (BN <= 256)
 constexpr int TC_WBUF_ELEMS = 512 * 512;
 constexpr unsigned long long TC_WAIT_LIMIT_NS = 2000000000ull;  // every mbarrier wait gives up after two seconds
 
@@ -43,6 +44,7 @@ LP_DEVINL uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_
 
 LP_DEVINL void mbar_init(uint32_t bar, uint32_t count) { asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory"); }
 LP_DEVINL void mbar_arrive(uint32_t bar) { asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory"); }
+LP_DEVINL void named_barrier_sync(int id, int threads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory"); }
 LP_DEVINL void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -200,7 +202,8 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[8], bar_empty[8], bar_acc;
     __shared__ uint32_t tmem_base_s;
-    __shared__ int abort_s;
+    __shared__ int abort_s, colsum_fail_s;
+    __shared__ float colsum_s[8][64];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);  // swizzle atoms need 1024-byte alignment
@@ -221,8 +224,9 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
     const int num_kb = (int)((k_end - k_begin + TC_BK - 1) / TC_BK);
     const int m0 = blockIdx.x * TC_BM;
     const int n0 = blockIdx.y * BN;
-    // the CTAs of the first M tile also sum the columns of their B tiles (warps 2 and 3)
-    const bool do_colsum = MN_MAJOR && p.colsum != 0 && blockIdx.x == 0;
+    // bias gradient: the 64-column boxes of the B tile are dealt out over the M tiles of the split; warps 2 and 3 add them up
+    const int n_boxes = BN / 64;
+    const bool do_colsum = MN_MAJOR && p.colsum != 0 && (int)blockIdx.x < n_boxes;
     const int64_t part_rows = p.M + (MN_MAJOR && p.colsum != 0 ? 1 : 0);
 
     if (threadIdx.x == 0) {
@@ -232,6 +236,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
         }
         mbar_init(smem_u32(&bar_acc), 1);
         abort_s = 0;
+        colsum_fail_s = 0;
         fence_barrier_init();
         fence_async_proxy();
         tma_prefetch_desc(&mapA);
@@ -303,15 +308,18 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
             }
             if (ok) umma_commit(smem_u32(&bar_acc));   // accumulator complete
         } else if (do_colsum && warp >= 2) {
-            // ---- column sums of the B tiles (bias gradient): thread t owns columns 4t .. 4t+3 of the N tile.
-            // A staged B tile is BN / 64 boxes of 64 reduction rows x 128 bytes; the 16-byte piece c of row k
-            // sits at piece c ^ (k & 7) (128-byte swizzle).  Rows are added in order, so the sum is reproducible.
+            // ---- column sums of the B tiles (bias gradient).  A staged B tile is BN / 64 boxes of 64 reduction
+            // rows x 128 bytes (64 columns); the 16-byte piece c of row k sits at piece c ^ (k & 7) (128-byte
+            // swizzle).  The boxes are dealt out over the CTAs of the split (box b to M tile b mod gridDim.x).
+            // Thread t = (rq, c8) adds rows 8 rq .. 8 rq + 7 of every stage for the eight columns of piece c8;
+            // the eight row groups are added in order at the end, so the sum is reproducible.
             const int t = threadIdx.x - 64;
-            const int c4 = t * 4;
-            const bool active = c4 < BN;
-            const uint32_t box_off = (uint32_t)(c4 >> 6) * 8192u;
-            const uint32_t piece = (uint32_t)((c4 & 63) >> 3), within = (uint32_t)(c4 & 7) * 2u;
-            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+            const int c8 = t & 7, rq = t >> 3;
+            float acc[TC_COLSUM_BOXES][8];
+#pragma unroll
+            for (int j = 0; j < TC_COLSUM_BOXES; ++j)
+#pragma unroll
+                for (int q = 0; q < 8; ++q) acc[j][q] = 0.f;
             bool ok = true;
             for (int kb = 0; kb < num_kb; ++kb) {
                 const int s = kb % S;
@@ -321,22 +329,46 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
                     abort_s = 1;
                     break;
                 }
-                if (active) {
-                    const uint8_t *sb = smem + (size_t)s * stage_bytes + a_bytes + box_off;
-#pragma unroll 8
-                    for (int k = 0; k < TC_BK; ++k) {
-                        const uint2 v = *reinterpret_cast<const uint2 *>(sb + k * 128 + (((piece ^ (uint32_t)(k & 7)) << 4) | within));
-                        s0 += __uint_as_float(v.x << 16);
-                        s1 += __uint_as_float(v.x & 0xffff0000u);
-                        s2 += __uint_as_float(v.y << 16);
-                        s3 += __uint_as_float(v.y & 0xffff0000u);
+                const uint8_t *sb = smem + (size_t)s * stage_bytes + a_bytes + (size_t)rq * 1024;
+#pragma unroll
+                for (int j = 0; j < TC_COLSUM_BOXES; ++j) {
+                    const int b = (int)blockIdx.x + j * (int)gridDim.x;
+                    if (b < n_boxes) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const uint4 v = *reinterpret_cast<const uint4 *>(sb + (size_t)b * 8192 + i * 128 + ((c8 ^ i) << 4));
+                            acc[j][0] += __uint_as_float(v.x << 16);
+                            acc[j][1] += __uint_as_float(v.x & 0xffff0000u);
+                            acc[j][2] += __uint_as_float(v.y << 16);
+                            acc[j][3] += __uint_as_float(v.y & 0xffff0000u);
+                            acc[j][4] += __uint_as_float(v.z << 16);
+                            acc[j][5] += __uint_as_float(v.z & 0xffff0000u);
+                            acc[j][6] += __uint_as_float(v.w << 16);
+                            acc[j][7] += __uint_as_float(v.w & 0xffff0000u);
+                        }
                     }
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bar_empty[s]));  // this warp has read the stage
             }
-            if (ok && active)
-                *reinterpret_cast<float4 *>(p.out_f32 + ((int64_t)blockIdx.z * part_rows + p.M) * p.N + n0 + c4) = make_float4(s0, s1, s2, s3);
+            // both warps take the same path here: `ok` is decided per warp, so exchange it through shared memory
+            if (!ok) colsum_fail_s = 1;
+            named_barrier_sync(1, 64);
+            ok = colsum_fail_s == 0;
+#pragma unroll
+            for (int j = 0; j < TC_COLSUM_BOXES; ++j) {
+                const int b = (int)blockIdx.x + j * (int)gridDim.x;
+                if (b < n_boxes) {  // uniform over the 64 threads
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) colsum_s[rq][c8 * 8 + q] = acc[j][q];
+                    named_barrier_sync(1, 64);
+                    float r = 0.f;
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) r += colsum_s[g][t];
+                    if (ok) p.out_f32[((int64_t)blockIdx.z * part_rows + p.M) * p.N + n0 + b * 64 + t] = r;
+                    named_barrier_sync(1, 64);
+                }
+            }
         }
         __syncwarp();
 
@@ -388,7 +420,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
         const int64_t row = (int64_t)m0 + threadIdx.x;
         if (row < p.M)
             for (int c = 0; c < BN; ++c) p.out_f32[((int64_t)blockIdx.z * part_rows + row) * p.N + n0 + c] = 0.f;
-        if (do_colsum)
+        if (MN_MAJOR && p.colsum != 0 && blockIdx.x == 0)
             for (int c = threadIdx.x; c < BN; c += TC_THREADS) p.out_f32[((int64_t)blockIdx.z * part_rows + p.M) * p.N + n0 + c] = 0.f;
     }
     tc_fence_before();
@@ -804,36 +836,6 @@ static bool tc_linear_bf16_b(TcState &tc, Exec &ex, int64_t M, int N, int K, con
     return tc_gemm_kmajor(tc, ex, M, N, K, A, lda, Bt, bias, relu, C, ldc, err);
 }
 
-// dst[i] = (accumulate ? dst[i] : 0) + sum_z partials[z][i]: a block covers 64 consecutive elements, its four
-// thread rows each add a quarter of the splits in index order, and the quarters are added in order
-__global__ void __launch_bounds__(256) reduce_partials_wide_kernel(const float *__restrict__ partials, int64_t count, int splits, float *__restrict__ dst,
-                                                                   int accumulate)
-{
-    __shared__ float part[4][64];
-    const int e = threadIdx.x & 63, q = threadIdx.x >> 6;
-    const int64_t i = (int64_t)blockIdx.x * 64 + e;
-    const int per = (splits + 3) / 4;
-    const int z0 = q * per, z1 = min(splits, z0 + per);
-    float s = 0.f;
-    if (i < count) {
-        int z = z0;
-        for (; z + 8 <= z1; z += 8) {
-            float v[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) v[u] = __ldg(partials + (int64_t)(z + u) * count + i);
-#pragma unroll
-            for (int u = 0; u < 8; ++u) s += v[u];
-        }
-        for (; z < z1; ++z) s += __ldg(partials + (int64_t)z * count + i);
-    }
-    part[q][e] = s;
-    __syncthreads();
-    if (q == 0 && i < count) {
-        const float r = ((part[0][e] + part[1][e]) + part[2][e]) + part[3][e];
-        dst[i] = accumulate ? dst[i] + r : r;
-    }
-}
-
 // weight gradient: dW[Kin, N] (+)= A[rows, Kin]^T dZ[rows, N]; partial tiles per row split, then a
 // fixed-order reduction
 static int tc_weight_grad_splits(int64_t rows, int Kin, int N)
@@ -870,7 +872,7 @@ static bool tc_weight_grad(TcState &tc, Exec &ex, int64_t rows, int Kin, int N, 
     dim3 grid((unsigned)(Kin / TC_BM), (unsigned)(N / BN), (unsigned)splits);
     tc_gemm_kernel<true><<<grid, TC_THREADS, smem, ex.st>>>(mapA, mapB, p);
     const int64_t count = (int64_t)(Kin + (fuse_bias ? 1 : 0)) * N;
-    reduce_partials_wide_kernel<<<(unsigned)ceil_div64(count, 64), 256, 0, ex.st>>>(partials, count, splits, dW, accumulate);
+    reduce_partials_kernel<<<(unsigned)ceil_div64(count, 256), 256, 0, ex.st>>>(partials, count, splits, dW, accumulate);
     ex.launches += 2;
     return true;
 }
