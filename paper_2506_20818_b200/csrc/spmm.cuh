@@ -83,6 +83,21 @@ template <typename T, typename ACC, bool HAS_VAL> LP_DEVINL void acc_add_vec(ACC
 #pragma unroll
     for (int t = 0; t < VN; ++t) acc_add<ACC>(acc[t], w, f[t]);
 }
+// exact accumulator: the power-of-two scale is folded into the coefficient once per vector (exact), leaving one
+// multiplication, one conversion and one 64-bit addition per element
+template <typename T, bool HAS_VAL> LP_DEVINL void acc_add_vec_exact(long long *acc, float w, const Vec16<T> &v)
+{
+    constexpr int VN = Vec16<T>::N;
+    float f[VN];
+    v.to_float(f);
+    const float ws = w * SPMM_EXACT_SCALE;
+#pragma unroll
+    for (int t = 0; t < VN; ++t) acc[t] += __float2ll_rn(ws * f[t]);
+}
+template <> LP_DEVINL void acc_add_vec<bf16, long long, true>(long long *acc, float w, const Vec16<bf16> &v) { acc_add_vec_exact<bf16, true>(acc, w, v); }
+template <> LP_DEVINL void acc_add_vec<bf16, long long, false>(long long *acc, float w, const Vec16<bf16> &v) { acc_add_vec_exact<bf16, false>(acc, w, v); }
+template <> LP_DEVINL void acc_add_vec<float, long long, true>(long long *acc, float w, const Vec16<float> &v) { acc_add_vec_exact<float, true>(acc, w, v); }
+template <> LP_DEVINL void acc_add_vec<float, long long, false>(long long *acc, float w, const Vec16<float> &v) { acc_add_vec_exact<float, false>(acc, w, v); }
 template <> LP_DEVINL void acc_add_vec<bf16, float, false>(float *acc, float, const Vec16<bf16> &v)
 {
     const uint32_t x[4] = {v.v.x, v.v.y, v.v.z, v.v.w};
@@ -94,7 +109,8 @@ template <> LP_DEVINL void acc_add_vec<bf16, float, false>(float *acc, float, co
 }
 template <typename ACC> LP_DEVINL float acc_value(ACC a);
 template <> LP_DEVINL float acc_value<float>(float a) { return a; }
-template <> LP_DEVINL float acc_value<long long>(long long a) { return (float)((double)a * (1.0 / 1099511627776.0)); }
+// one rounding (64-bit integer to FP32, to nearest); the power-of-two scale is exact
+template <> LP_DEVINL float acc_value<long long>(long long a) { return __ll2float_rn(a) * (1.f / SPMM_EXACT_SCALE); }
 constexpr int SPMM_HEAVY_MIN = 64;  // smallest heavy-row threshold a plan may use (bounds the item count by nnz / 64).
                                     // A lane group keeps only a few gathers in flight, so a long row handled by one
                                     // group is a long dependent chain: long rows are cut into items instead.
@@ -322,7 +338,19 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
                 pre_val = HAS_VAL ? __ldg(a.val + eb + gl) : 1.f;
             }
         }
-        if (r < n_rows && e_end - e_begin <= a.heavy.threshold) {
+        if (r < n_rows && e_end == e_begin && !a.init && !a.self_out) {
+            // empty row without an extra term: the output row is zero
+            Vec16<T> z;
+            float zf[VN];
+#pragma unroll
+            for (int j = 0; j < VN; ++j) zf[j] = 0.f;
+            z.from_float(zf);
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const int ch = gl + i * G;
+                if (ch < nchunks) z.store(a.Y + (size_t)r * a.ldy + ch * VN);
+            }
+        } else if (r < n_rows && e_end - e_begin <= a.heavy.threshold) {
 #pragma unroll
             for (int i = 0; i < NV; ++i)
 #pragma unroll
