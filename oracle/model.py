@@ -99,19 +99,41 @@ def _block_as_global_csr(n: int, frontier: np.ndarray, ptr: np.ndarray, cols: np
     return rowptr, cols
 
 
-def _layer_graphs(g, n_layers: int, blocks):
-    """Per layer l = 1..K: (rowptr, col, w, active_rows or None).
+def _sampled_gcn_weights(g, frontier: np.ndarray, ptr: np.ndarray, cols: np.ndarray) -> np.ndarray:
+    """Per-entry weights of a sampled block for the GCN aggregation: the weight the entry has in
+    the loaded graph, times |N(v)| / |S(v)| for its destination v -- every neighbour is drawn
+    with probability |S(v)| / |N(v)|, so the sampled sum estimates the full neighbour sum
+    without bias.  The normalisation 1 / sqrt(d~_v d~_u) keeps the degrees of the full graph."""
+    w = np.zeros(cols.shape[0], dtype=np.float64)
+    for i, v in enumerate(frontier):
+        lo, hi = int(ptr[i]), int(ptr[i + 1])
+        if hi == lo:
+            continue
+        r0, r1 = int(g.rowptr[v]), int(g.rowptr[v + 1])
+        pos = r0 + np.searchsorted(g.col[r0:r1], cols[lo:hi])
+        assert np.array_equal(g.col[pos], cols[lo:hi])
+        full = np.ones(hi - lo) if g.w is None else g.w[pos].astype(np.float64)
+        w[lo:hi] = full * ((r1 - r0) / (hi - lo))
+    return w.astype(np.float32)  # the aggregation routine takes float32 weights; the ratio of two small integers times a
+    #                              float32 weight is rounded once here
+
+
+def _layer_graphs(g, n_layers: int, blocks, arch: str = "sage"):
+    """Per layer l = 1..K: (rowptr, col, w, active_rows or None, dtilde or None).
     Full-graph training uses the loaded graph at every layer.  With a sampled computational
-    graph, layer l works on hop h = K - l + 1: rows F_{h-1} aggregate their sampled neighbours."""
+    graph, layer l works on hop h = K - l + 1: rows F_{h-1} aggregate their sampled neighbours
+    (mean over the sample; GCN: rescaled sample with the full graph's degrees, self term exact)."""
     if blocks is None:
-        return [(g.rowptr, g.col, g.w, None)] * n_layers
+        return [(g.rowptr, g.col, g.w, None, None)] * n_layers
     frontiers, blks = blocks
+    dt = sparse.gcn_degree(g.n, g.rowptr, g.w) if arch == "gcn" else None
     out = []
     for l in range(1, n_layers + 1):
         h = n_layers - l + 1
         ptr, cols = blks[h - 1]
         rp, cc = _block_as_global_csr(g.n, frontiers[h - 1], ptr, cols)
-        out.append((rp, cc, None, frontiers[h - 1]))
+        w = _sampled_gcn_weights(g, frontiers[h - 1], ptr, cols) if arch == "gcn" else None
+        out.append((rp, cc, w, frontiers[h - 1], dt))
     return out
 
 
@@ -129,11 +151,11 @@ def forward(g, X: np.ndarray, params: np.ndarray, arch: str, dims: Sequence[int]
     K = len(dims) - 1
     P = split_params(arch, dims, np.asarray(params, dtype=np.float64))
     H = np.asarray(X, dtype=np.float64)
-    cache = {"H": [H], "M": [], "Z": [], "active": [], "ties": 0, "graphs": _layer_graphs(g, K, blocks)}
+    cache = {"H": [H], "M": [], "Z": [], "active": [], "ties": 0, "graphs": _layer_graphs(g, K, blocks, arch)}
     mode = "gcn" if arch == "gcn" else "mean"
     for k in range(K):
-        rp, cc, w, act = cache["graphs"][k]
-        M = sparse.aggregate(mode, g.n, rp, cc, w if arch == "gcn" else None, H)
+        rp, cc, w, act, dt = cache["graphs"][k]
+        M = sparse.aggregate(mode, g.n, rp, cc, w if arch == "gcn" else None, H, dt)
         if arch == "gcn":
             Z = M @ P[k]["W"] + P[k]["b"]
         else:
@@ -208,7 +230,7 @@ def train_step(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst, blo
     G = split_params(arch, dims, grads[:n_enc])
     mode = "gcn" if arch == "gcn" else "mean"
     for k in range(K - 1, -1, -1):
-        rp, cc, w, act = cache["graphs"][k]
+        rp, cc, w, act, dt = cache["graphs"][k]
         dZ = dH if k == K - 1 else dH * cache["active"][k]
         if act is not None:
             keep = np.zeros(g.n, dtype=bool)
@@ -219,7 +241,7 @@ def train_step(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst, blo
         if arch == "gcn":
             G[k]["W"][:] = M.T @ dZ
             dM = dZ @ P[k]["W"].T
-            dH = sparse.aggregate_backward(mode, g.n, rp, cc, w, dM) if k > 0 else None
+            dH = sparse.aggregate_backward(mode, g.n, rp, cc, w, dM, dt) if k > 0 else None
         else:
             G[k]["W_self"][:] = Hprev.T @ dZ
             G[k]["W_neigh"][:] = M.T @ dZ

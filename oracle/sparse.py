@@ -64,26 +64,32 @@ def gcn_degree(n: int, rowptr, w) -> np.ndarray:
 _MODE = {"gcn": 0, "mean": 1, "sage": 1}
 
 
-def aggregate(mode: str, n: int, rowptr, col, w, H: np.ndarray) -> np.ndarray:
-    """AGG of Eq. 1 over every row: 'gcn' (renormalised adjacency) or 'mean'."""
+def aggregate(mode: str, n: int, rowptr, col, w, H: np.ndarray, dtilde=None) -> np.ndarray:
+    """AGG of Eq. 1 over every row: 'gcn' (renormalised adjacency) or 'mean'.
+    dtilde: the GCN degrees to normalise with; by default those of the structure given
+    (a sampled block passes the degrees of the full graph)."""
     rowptr, col = _i64(rowptr), _i32(col)
     w = None if w is None else np.ascontiguousarray(w, dtype=np.float32)
     H = np.ascontiguousarray(H, dtype=np.float64)
     F = H.shape[1]
-    dt = gcn_degree(n, rowptr, w) if _MODE[mode] == 0 else None
+    dt = None
+    if _MODE[mode] == 0:
+        dt = gcn_degree(n, rowptr, w) if dtilde is None else np.ascontiguousarray(dtilde, dtype=np.float64)
     M = np.zeros((n, F), dtype=np.float64)
     lib().orc_aggregate(C.c_int(_MODE[mode]), C.c_int64(n), _p(rowptr, C.c_int64), _p(col, C.c_int32),
                         _p(w, C.c_float), _p(dt, C.c_double), _p(H, C.c_double), C.c_int64(F), _p(M, C.c_double))
     return M
 
 
-def aggregate_backward(mode: str, n: int, rowptr, col, w, dM: np.ndarray) -> np.ndarray:
+def aggregate_backward(mode: str, n: int, rowptr, col, w, dM: np.ndarray, dtilde=None) -> np.ndarray:
     """Gradient of AGG with respect to its input embeddings (scatter form)."""
     rowptr, col = _i64(rowptr), _i32(col)
     w = None if w is None else np.ascontiguousarray(w, dtype=np.float32)
     dM = np.ascontiguousarray(dM, dtype=np.float64)
     F = dM.shape[1]
-    dt = gcn_degree(n, rowptr, w) if _MODE[mode] == 0 else None
+    dt = None
+    if _MODE[mode] == 0:
+        dt = gcn_degree(n, rowptr, w) if dtilde is None else np.ascontiguousarray(dtilde, dtype=np.float64)
     dH = np.zeros((n, F), dtype=np.float64)
     lib().orc_aggregate_backward(C.c_int(_MODE[mode]), C.c_int64(n), _p(rowptr, C.c_int64), _p(col, C.c_int32),
                                  _p(w, C.c_float), _p(dt, C.c_double), _p(dM, C.c_double), C.c_int64(F),

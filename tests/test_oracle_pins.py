@@ -442,6 +442,106 @@ def test_sampled_step_backward_finite_differences():
     assert rel_l2(out["grads"], fd) < 1e-7
 
 
+def _dense_sampled_gcn_operator(g, frontier, ptr, cols):
+    """Dense operator of one sampled GCN hop, written from the definition: self term 1 / d~_v, sampled entries
+    w_vu / sqrt(d~_v d~_u) * |N(v)| / |S(v)|, degrees of the full graph."""
+    A = dense_adjacency(g)
+    dt = 1.0 + A.sum(axis=1)
+    S = np.zeros((g.n, g.n))
+    for i, v in enumerate(frontier):
+        nb = cols[ptr[i]:ptr[i + 1]]
+        deg = int(g.rowptr[v + 1] - g.rowptr[v])
+        S[v, v] += 1.0 / dt[v]
+        for u in nb:
+            S[v, u] += A[v, u] / math.sqrt(dt[v] * dt[u]) * deg / len(nb)
+    return S
+
+
+def test_sampled_gcn_with_full_fanout_equals_full_graph_training():
+    # a fan-out at least as large as every degree samples every neighbour: the sampled step must then give
+    # the loss and the parameter gradients of full-graph training (pinned elsewhere against dense operators)
+    g = wl.coauthor_weighted(70, 260, seed=4)
+    fan = int(np.diff(g.rowptr).max())
+    dims = [4, 5, 3]
+    X = wl.node_features(g.n, 4, 0).astype(np.float64)
+    p = wl.glorot_params("gcn", dims, 3, 0.2).astype(np.float64)
+    src = np.array([1, 5, 9, 30], dtype=np.int32)
+    dst = np.array([2, 7, 9, 41], dtype=np.int32)
+    nsrc, ndst = src.copy(), np.array([50, 3, 22, 8], dtype=np.int32)
+    blocks = oracle.build_blocks(g.n, g.rowptr, g.col, np.concatenate([src, dst, ndst]), [fan, fan], seed=1, step=0)
+    a = oracle.train_step(g, X, p, "gcn", dims, src, dst, nsrc, ndst, blocks=blocks)
+    b = oracle.train_step(g, X, p, "gcn", dims, src, dst, nsrc, ndst)
+    assert abs(a["loss"] - b["loss"]) < 1e-12
+    assert rel_l2(a["grads"], b["grads"]) < 1e-6  # float32 rounding of the per-entry ratio-times-weight only
+
+
+def test_sampled_gcn_forward_bruteforce_and_unbiased():
+    g = wl.coauthor_weighted(90, 700, seed=8)
+    assert g.w is not None and np.diff(g.rowptr).max() > 6
+    dims = [4, 5, 3]
+    X = wl.node_features(g.n, 4, 0).astype(np.float64)
+    p = wl.glorot_params("gcn", dims, 2, 0.2).astype(np.float64)
+    P = oracle.split_params("gcn", dims, p)
+    seeds = np.array([3, 17, 40, 77], dtype=np.int32)
+    fr, blks = oracle.build_blocks(g.n, g.rowptr, g.col, seeds, [3, 2], seed=5, step=0)
+    HK = oracle.forward(g, X, p, "gcn", dims, blocks=(fr, blks))["H"][2]
+    H = X
+    for l in (1, 2):
+        h = 2 - l + 1
+        S = _dense_sampled_gcn_operator(g, fr[h - 1], *blks[h - 1])
+        Z = (S @ H) @ P[l - 1]["W"] + P[l - 1]["b"]
+        Hn = np.maximum(Z, 0) if l < 2 else Z
+        keep = np.zeros(g.n, dtype=bool)
+        keep[fr[h - 1]] = True
+        H = np.where(keep[:, None], Hn, 0.0)
+    assert rel_l2(HK, H) < 1e-6
+    # the sampled operator averages to the full one over many independent samples
+    v = int(np.argmax(np.diff(g.rowptr)))
+    full = dense_gcn_operator(g)[v]
+    acc = np.zeros(g.n)
+    T = 3000
+    for step in range(T):
+        fr1, blk1 = oracle.build_blocks(g.n, g.rowptr, g.col, np.array([v], dtype=np.int32), [3], seed=9, step=step)
+        acc += _dense_sampled_gcn_operator(g, fr1[0], *blk1[0])[v]
+    nz = full > 0
+    assert np.abs(acc[nz] / T - full[nz]).max() < 0.12 * full[nz].max()
+    assert np.abs(acc[~nz]).max() == 0.0
+
+
+def test_sampled_gcn_step_backward_finite_differences():
+    g = wl.coauthor_weighted(60, 300, seed=6)
+    dims = [3, 4, 3]
+    X = wl.node_features(g.n, 3, 0).astype(np.float64)
+    p = wl.glorot_params("gcn", dims, 2, 0.2).astype(np.float64)
+    src = np.array([1, 5, 9, 30], dtype=np.int32)
+    dst = np.array([2, 7, 9, 41], dtype=np.int32)
+    nsrc, ndst = src.copy(), np.array([50, 3, 22, 8], dtype=np.int32)
+    fr, blks = oracle.build_blocks(g.n, g.rowptr, g.col, np.concatenate([src, dst, ndst]), [3, 2], seed=1, step=7)
+    out = oracle.train_step(g, X, p, "gcn", dims, src, dst, nsrc, ndst, blocks=(fr, blks))
+    ops = [_dense_sampled_gcn_operator(g, fr[2 - l], *blks[2 - l]) for l in (1, 2)]
+    s_all, d_all = np.concatenate([src, nsrc]), np.concatenate([dst, ndst])
+    y = np.concatenate([np.ones(4), np.zeros(4)])
+
+    def bf_loss(pp):
+        P = oracle.split_params("gcn", dims, pp)
+        H1 = np.maximum((ops[0] @ X) @ P[0]["W"] + P[0]["b"], 0)
+        keep = np.zeros(g.n, dtype=bool)
+        keep[fr[1]] = True
+        H1 = np.where(keep[:, None], H1, 0.0)
+        H2 = (ops[1] @ H1) @ P[1]["W"] + P[1]["b"]
+        s = (H2[s_all] * H2[d_all]).sum(axis=1)
+        return float(np.mean(y * np.logaddexp(0, -s) + (1 - y) * np.logaddexp(0, s)))
+
+    assert abs(bf_loss(p) - out["loss"]) < 1e-7
+    fd = np.zeros_like(p)
+    for i in range(p.shape[0]):
+        pp, pm = p.copy(), p.copy()
+        pp[i] += 1e-6
+        pm[i] -= 1e-6
+        fd[i] = (bf_loss(pp) - bf_loss(pm)) / 2e-6
+    assert rel_l2(out["grads"], fd) < 1e-5
+
+
 def test_relu_tie_window_only_touches_near_zero_units():
     g = wl.erdos_renyi(60, 200, seed=3)
     dims = [6, 8, 4]
