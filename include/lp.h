@@ -60,7 +60,9 @@ typedef enum { LP_PRED_DOT = 0, LP_PRED_MLP = 1 } lp_predictor;
  * fanouts).  dims = {input, hidden.., output}; every width must be a multiple of 8 (FP32)
  * or of 64 (BF16 tensor-core path).  fanout[h] is the number of in-neighbours sampled at hop
  * h+1 (hop 1 feeds the LAST layer); all zeros = full-graph training (every node aggregates
- * its full neighbour list).  Sampling is supported for LP_SAGE_MEAN only. */
+ * its full neighbour list).  Over a sample S(v) of N(v), LP_SAGE_MEAN takes the mean of the sample;
+ * LP_GCN keeps the coefficients and degrees of the loaded graph, multiplies the sampled entries of v
+ * by |N(v)| / |S(v)| (an unbiased estimate of the full sum) and keeps the self term exact. */
 typedef struct {
     int32_t arch;                    /* lp_arch */
     int32_t n_layers;                /* K, 1..LP_MAX_LAYERS */

@@ -165,6 +165,10 @@ def forward(g, X: np.ndarray, params: np.ndarray, arch: str, dims: Sequence[int]
             if relu_ties is not None and relu_ties[k] is not None and tie_tol > 0.0:
                 rows = Z if act is None else Z[act]
                 near = np.abs(Z) <= tie_tol * np.sqrt(np.mean(rows * rows))
+                if act is not None:  # rows outside the frontier are not computed at all: nothing to adopt there
+                    in_frontier = np.zeros(g.n, dtype=bool)
+                    in_frontier[act] = True
+                    near &= in_frontier[:, None]
                 cache["ties"] += int((near & (active != relu_ties[k])).sum())
                 active = np.where(near, relu_ties[k], active)
             cache["active"].append(active)

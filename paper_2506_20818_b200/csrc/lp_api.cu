@@ -32,6 +32,10 @@ struct HopBlock {  // sampled block of hop h (destinations F_{h-1}, sources F_h)
     float *inv_deg = nullptr;     // 1 / sampled degree per destination     [cap_dst]
     int *colptr = nullptr, *rowidx = nullptr, *perm = nullptr;  // transposed block
     int *self_idx = nullptr, *inv_self = nullptr;
+    // GCN only: CSR position of every sampled entry, its rescaled coefficient (block order and transposed
+    // order) and the self coefficients 1 / d~ of the destination and of the source rows
+    int *blk_eid = nullptr;
+    float *blk_val = nullptr, *blk_valT = nullptr, *self_coef_dst = nullptr, *self_coef_src = nullptr;
 };
 
 struct LayerBuf {  // device buffers of one encoder layer (element type fixed by the precision)
@@ -625,7 +629,6 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
     if (sampled) {
         for (int h = 0; h < d->n_layers; ++h)
             if (d->fanout[h] == 0) return fail(ctx, LP_EINVAL, "lp_set_model: fanouts must be all zero or all positive");
-        if (d->arch != LP_SAGE_MEAN) return fail(ctx, LP_EUNSUPPORTED, "lp_set_model: neighbour sampling is implemented for SAGE-mean only");
         if (d->cache_input_aggregation) return fail(ctx, LP_EINVAL, "lp_set_model: cache_input_aggregation needs a full-graph model (sampled neighbourhoods change every step)");
     }
     if (d->predictor != LP_PRED_DOT && d->predictor != LP_PRED_MLP) return fail(ctx, LP_EINVAL, "lp_set_model: unknown predictor");
@@ -693,7 +696,7 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
         const int64_t rows = sampled ? cap_rows[K - k - 1] : n;
         MALLOC(p, rows * L.Kin * (int64_t)es);
         L.A = p;
-        if (!sage) {
+        if (!sage && !sampled) {
             if (k == 0) {
                 L.Hin = d->prec == LP_BF16 ? (void *)ctx->X16 : (void *)ctx->X32;
             } else {
@@ -783,6 +786,15 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
                 MALLOC(hb.blk_col_global, hb.cap_entries);
                 MALLOC(hb.blk_row, hb.cap_entries);
                 MALLOC(hb.inv_deg, hb.cap_dst);
+                if (!sage) {
+                    MALLOC(hb.blk_eid, hb.cap_entries);
+                    MALLOC(hb.blk_val, hb.cap_entries);
+                    MALLOC(hb.self_coef_dst, hb.cap_dst);
+                    if (h < K) {
+                        MALLOC(hb.blk_valT, hb.cap_entries);
+                        MALLOC(hb.self_coef_src, hb.cap_src);
+                    }
+                }
                 if (h < K) {
                     MALLOC(hb.blk_col_local, hb.cap_entries);
                     MALLOC(hb.colptr, (int64_t)hb.cap_src + 1);
@@ -936,6 +948,17 @@ static lp_status sync_counts(lp_ctx *ctx, const int *dev_a, const int *dev_b, in
     return LP_OK;
 }
 
+// GCN coefficients of a sampled block (entries and destination self terms); hb.entries and hb.n_dst are known
+static void gcn_block_coefficients(lp_ctx *ctx, HopBlock &hb, HopBlock &prev)
+{
+    cudaStream_t st = ctx->ex.st;
+    if (hb.entries > 0)
+        gcn_block_coef_kernel<<<nblk(hb.entries), 256, 0, st>>>(ctx->rowptr, prev.frontier, hb.blk_ptr, hb.blk_row, hb.blk_eid, hb.blk_ptr + hb.n_dst,
+                                                                ctx->gcn_val, hb.blk_val);
+    if (hb.n_dst > 0) gather_by_id_kernel<<<nblk(hb.n_dst), 256, 0, st>>>(ctx->gcn_self, prev.frontier, prev.n_front_dev, hb.cap_dst, hb.self_coef_dst);
+    ctx->ex.launches += 2;
+}
+
 // Sampled computational graph of the batch: F_0 = unique(seeds); hop h samples fanout[h-1]
 // in-neighbours of every node of F_{h-1}; F_h = unique(F_{h-1} u sampled).
 static lp_status build_blocks(lp_ctx *ctx, const int *pos_src, const int *pos_dst, int64_t B, const int *neg_src, const int *neg_dst, int k,
@@ -944,6 +967,7 @@ static lp_status build_blocks(lp_ctx *ctx, const int *pos_src, const int *pos_ds
     cudaStream_t st = ctx->ex.st;
     const int n = ctx->n, K = ctx->K;
     const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
+    const bool gcn = ctx->desc.arch == LP_GCN;
     ProfScope prof(ctx->ex, LP_PROF_BLOCKS);
     CK(cudaMemsetAsync(ctx->mark, 0, (size_t)n, st));
     mark_ids_kernel<<<nblk(B), 256, 0, st>>>(pos_src, B, n, ctx->mark);
@@ -960,7 +984,7 @@ static lp_status build_blocks(lp_ctx *ctx, const int *pos_src, const int *pos_ds
             nbr_count_kernel<<<nblk(hb.n_dst + 1), 256, 0, st>>>(ctx->rowptr, prev.frontier, prev.n_front_dev, ctx->desc.fanout[h - 1], hb.blk_ptr, hb.n_dst);
             exclusive_scan_i32(ctx->ex, hb.blk_ptr, hb.n_dst, hb.blk_ptr, hb.blk_ptr + hb.n_dst, ctx->scan_tmp);
             nbr_sample_kernel<<<nblk(hb.n_dst), 256, 0, st>>>(ctx->rowptr, ctx->col, prev.frontier, prev.n_front_dev, ctx->desc.fanout[h - 1], key,
-                                                              (uint32_t)step, (uint32_t)h, hb.blk_ptr, hb.blk_col_global, hb.blk_row, ctx->mark);
+                                                              (uint32_t)step, (uint32_t)h, hb.blk_ptr, hb.blk_col_global, hb.blk_row, ctx->mark, hb.blk_eid);
             inv_degree_kernel<<<nblk(hb.n_dst), 256, 0, st>>>(hb.blk_ptr, hb.n_dst, nullptr, hb.inv_deg);
             ctx->ex.launches += 3;
             if (h == K) {  // outermost hop: only the entry count is needed
@@ -969,6 +993,7 @@ static lp_status build_blocks(lp_ctx *ctx, const int *pos_src, const int *pos_ds
                 if (s != LP_OK) return s;
                 hb.entries = entries;
                 hb.n_src = n;
+                if (gcn) gcn_block_coefficients(ctx, hb, prev);
                 break;
             }
         }
@@ -992,6 +1017,12 @@ static lp_status build_blocks(lp_ctx *ctx, const int *pos_src, const int *pos_ds
                 ctx->ex.launches += 1;
             }
             transpose_csr(ctx->ex, hb.blk_ptr, hb.n_dst, hb.n_src, hb.blk_col_local, hb.entries, hb.colptr, hb.rowidx, hb.perm, ctx->tsp);
+            if (gcn) {
+                gcn_block_coefficients(ctx, hb, ctx->hop[h - 1]);
+                if (hb.entries > 0) gather_f32_kernel<<<nblk(hb.entries), 256, 0, st>>>(hb.blk_val, hb.perm, hb.entries, hb.blk_valT);
+                gather_by_id_kernel<<<nblk(hb.n_src), 256, 0, st>>>(ctx->gcn_self, hb.frontier, hb.n_front_dev, hb.cap_src, hb.self_coef_src);
+                ctx->ex.launches += 2;
+            }
         }
     }
     CK_LAUNCH();
@@ -1050,21 +1081,32 @@ template <typename T> static lp_status forward_impl(lp_ctx *ctx, const float *pa
             a.n_rows = hb.n_dst;
             a.rowptr = hb.blk_ptr;
             a.F = L.Fi;
-            a.row_scale = hb.inv_deg;
-            a.Y = tptr<T>(L.A) + L.Fi;
-            a.ldy = L.Kin;
-            a.self_out = tptr<T>(L.A);
-            a.ldself = L.Kin;
+            a.ldx = L.Fi;
+            const int *self_rows;
             if (k == 0) {  // innermost layer reads the feature matrix by global id
                 a.X = Xt;
-                a.ldx = L.Fi;
                 a.col = hb.blk_col_global;
-                a.self_idx = ctx->hop[K - 1].frontier;
+                self_rows = ctx->hop[K - 1].frontier;
             } else {
                 a.X = tptr<T>(ctx->layer[k - 1].Hout);
-                a.ldx = L.Fi;
                 a.col = hb.blk_col_local;
-                a.self_idx = hb.self_idx;
+                self_rows = hb.self_idx;
+            }
+            if (sage) {  // [h_v | mean over the sample]
+                a.row_scale = hb.inv_deg;
+                a.Y = tptr<T>(L.A) + L.Fi;
+                a.ldy = L.Kin;
+                a.self_out = tptr<T>(L.A);
+                a.ldself = L.Kin;
+                a.self_idx = self_rows;
+            } else {     // h_v / d~_v + rescaled sample with the graph's coefficients
+                a.val = hb.blk_val;
+                a.Y = tptr<T>(L.A);
+                a.ldy = L.Fi;
+                a.init = a.X;
+                a.ldinit = L.Fi;
+                a.init_idx = self_rows;
+                a.init_coef = hb.self_coef_dst;
             }
             if (k == K - 1) { out = tptr<T>(ctx->HK); ldo = L.Fo; } else { out = tptr<T>(L.Hout); ldo = L.Fo; }
         }
@@ -1277,11 +1319,18 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
             a.n_rows = hb.n_src;
             a.rowptr = hb.colptr;
             a.col = hb.rowidx;
-            a.X = dA + L.Fi;
-            a.ldx = L.Kin;
             a.init = dA;
             a.ldinit = L.Kin;
             a.init_idx = hb.inv_self;
+            if (sage) {
+                a.X = dA + L.Fi;
+                a.ldx = L.Kin;
+            } else {
+                a.val = hb.blk_valT;
+                a.X = dA;
+                a.ldx = L.Fi;
+                a.init_coef = hb.self_coef_src;
+            }
             a.relu_ref = tptr<T>(ctx->layer[l - 1].Hout);
             a.ldref = L.Fi;
         }

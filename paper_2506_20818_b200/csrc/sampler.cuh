@@ -89,7 +89,7 @@ __global__ void nbr_count_kernel(const int *__restrict__ rowptr, const int *__re
 __global__ void nbr_sample_kernel(const int *__restrict__ rowptr, const int *__restrict__ col, const int *__restrict__ frontier,
                                   const int *__restrict__ n_front_dev, int fanout, uint2 key, uint32_t step_lo, uint32_t hop,
                                   const int *__restrict__ blk_ptr, int *__restrict__ blk_col_global, int *__restrict__ blk_row,
-                                  unsigned char *__restrict__ mark)
+                                  unsigned char *__restrict__ mark, int *__restrict__ blk_eid = nullptr)
 {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= *n_front_dev) return;
@@ -101,6 +101,7 @@ __global__ void nbr_sample_kernel(const int *__restrict__ rowptr, const int *__r
             const int u = col[r0 + e];
             blk_col_global[out + e] = u;
             blk_row[out + e] = i;
+            if (blk_eid) blk_eid[out + e] = r0 + e;  // position of the sampled entry in the graph's CSR
             mark[u] = 1;
         }
         return;
@@ -124,8 +125,32 @@ __global__ void nbr_sample_kernel(const int *__restrict__ rowptr, const int *__r
         const int u = col[r0 + pos[q]];
         blk_col_global[out + q] = u;
         blk_row[out + q] = i;
+        if (blk_eid) blk_eid[out + q] = r0 + pos[q];
         mark[u] = 1;
     }
+}
+
+// GCN over a sampled block: entry e of destination i = frontier position of v keeps the graph's coefficient
+// w_vu / sqrt(d~_v d~_u), rescaled by |N(v)| / |S(v)| (every neighbour is kept with probability |S(v)| / |N(v)|, so the
+// sampled sum estimates the full one without bias); the self coefficient 1 / d~_v is exact.
+__global__ void gcn_block_coef_kernel(const int *__restrict__ rowptr, const int *__restrict__ frontier, const int *__restrict__ blk_ptr,
+                                      const int *__restrict__ blk_row, const int *__restrict__ blk_eid, const int *__restrict__ n_entries_dev,
+                                      const float *__restrict__ gcn_val, float *__restrict__ blk_val)
+{
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= *n_entries_dev) return;
+    const int i = blk_row[e];
+    const int v = frontier[i];
+    const float ratio = (float)(rowptr[v + 1] - rowptr[v]) / (float)(blk_ptr[i + 1] - blk_ptr[i]);
+    blk_val[e] = gcn_val[blk_eid[e]] * ratio;
+}
+
+// out[i] = table[ids[i]] for i < *count
+__global__ void gather_by_id_kernel(const float *__restrict__ table, const int *__restrict__ ids, const int *__restrict__ count_dev, int cap,
+                                    float *__restrict__ out)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < min(*count_dev, cap)) out[i] = table[ids[i]];
 }
 
 __global__ void mark_ids_kernel(const int *__restrict__ ids, int64_t m, int n, unsigned char *__restrict__ mark)

@@ -81,9 +81,10 @@ def test_bad_graphs_are_rejected(pkg):
     ctx.load_graph(g.n, g.rowptr, g.col, None, wl.node_features(g.n, 8, 0))
     with pytest.raises(pkg.LpError):
         ctx.set_model("gcn", [16, 8], max_batch=4)  # dims[0] != f
-    with pytest.raises(pkg.LpError) as ei:
-        ctx.set_model("gcn", [8, 8], fanout=[3], max_batch=4)  # sampling is SAGE only
-    assert ei.value.status == -5
+    with pytest.raises(pkg.LpError):
+        ctx.set_model("gcn", [8, 8, 8], fanout=[3, 0], max_batch=4)  # fanouts must be all zero or all positive
+    with pytest.raises(pkg.LpError):
+        ctx.set_model("sage", [8, 8], fanout=[33], max_batch=4)  # above the largest supported fan-out
     ctx.close()
 
 
@@ -337,6 +338,49 @@ def test_sampled_two_layer_and_one_layer(pkg):
         params = wl.glorot_params("sage", dims, 2, 0.05)
         err, _, _ = run_step(pkg, g, X, params, "sage", dims, "fp32", pos, fanout=fan, k=2)
         assert_within(err, TOL["fp32"])
+
+
+@pytest.mark.parametrize("prec", ["fp32", "bf16"])
+def test_sampled_gcn_minibatch(pkg, prec):
+    # mini-batch training of the weighted 3-layer GCN configuration with the fan-outs 25 / 10 / 5 of Section IV
+    g, X, params, pos, cfg = wl.make_config("c3_coauthor_gcn3", scale=0.04)
+    sel = np.random.default_rng(3).choice(len(pos[0]), 256, replace=False)
+    err, _, _ = run_step(pkg, g, X, params, "gcn", cfg["dims"], prec, (pos[0][sel], pos[1][sel]), fanout=[25, 10, 5], step=2)
+    assert_within(err, TOL[prec])
+
+
+@pytest.mark.parametrize("prec", ["fp32", "bf16"])
+def test_sampled_sage_minibatch_fanout_25_10(pkg, prec):
+    g, X, params, pos, cfg = wl.make_config("c2_chunglu_sage2", scale=0.05)
+    sel = np.random.default_rng(4).choice(len(pos[0]), 1024, replace=False)
+    err, _, _ = run_step(pkg, g, X, params, "sage", cfg["dims"], prec, (pos[0][sel], pos[1][sel]), fanout=[25, 10], step=1)
+    assert_within(err, TOL[prec])
+
+
+def test_sampled_gcn_full_fanout_matches_full_graph_step(pkg):
+    # every degree below the fan-out: the sampled GCN step is the full-graph step on the seeds' neighbourhood
+    g = wl.erdos_renyi(400, 1200, seed=5)
+    assert np.diff(g.rowptr).max() <= 32
+    dims = [16, 24, 8]
+    X = wl.node_features(g.n, 16, 1)
+    params = wl.glorot_params("gcn", dims, 2, 0.05)
+    u, v = wl.undirected_edge_list(g)
+    pos = (u[:64].astype(np.int32), v[:64].astype(np.int32))
+    ctx = pkg.Context(0)
+    ctx.load_graph(g.n, g.rowptr, g.col, g.w, X)
+    out = {}
+    for name, fan in (("full", None), ("sampled", [32, 32])):
+        ctx.set_model("gcn", dims, prec="fp32", fanout=fan, max_batch=64, max_k=1)
+        du, dv = t32(pos[0]), t32(pos[1])
+        _, nd = ctx.sample_negatives(3, 0, 1, du)
+        p = t32(params)
+        grads = torch.zeros_like(p)
+        loss = torch.zeros(1, device="cuda:0")
+        ctx.train_step(p, du, dv, None, nd, 1, loss, grads, seed=3, step=0)
+        out[name] = (loss.item(), grads.cpu().numpy())
+    ctx.close()
+    assert abs(out["full"][0] - out["sampled"][0]) <= 1e-6 * abs(out["full"][0])
+    assert rel_l2(out["sampled"][1], out["full"][1]) < 1e-5
 
 
 def test_step_edge_cases(pkg):
