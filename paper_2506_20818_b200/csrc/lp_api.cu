@@ -983,7 +983,7 @@ static lp_status build_blocks(lp_ctx *ctx, const int *pos_src, const int *pos_ds
             // sample: counts -> offsets -> columns (also marks the sampled ids; F_{h-1} is still marked)
             nbr_count_kernel<<<nblk(hb.n_dst + 1), 256, 0, st>>>(ctx->rowptr, prev.frontier, prev.n_front_dev, ctx->desc.fanout[h - 1], hb.blk_ptr, hb.n_dst);
             exclusive_scan_i32(ctx->ex, hb.blk_ptr, hb.n_dst, hb.blk_ptr, hb.blk_ptr + hb.n_dst, ctx->scan_tmp);
-            nbr_sample_kernel<<<nblk(hb.n_dst), 256, 0, st>>>(ctx->rowptr, ctx->col, prev.frontier, prev.n_front_dev, ctx->desc.fanout[h - 1], key,
+            nbr_sample_kernel<<<nblk((int64_t)hb.n_dst * 32), 256, 0, st>>>(ctx->rowptr, ctx->col, prev.frontier, prev.n_front_dev, ctx->desc.fanout[h - 1], key,
                                                               (uint32_t)step, (uint32_t)h, hb.blk_ptr, hb.blk_col_global, hb.blk_row, ctx->mark, hb.blk_eid);
             inv_degree_kernel<<<nblk(hb.n_dst), 256, 0, st>>>(hb.blk_ptr, hb.n_dst, nullptr, hb.inv_deg);
             ctx->ex.launches += 3;
