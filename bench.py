@@ -281,9 +281,19 @@ def main():
     agg_spans = prof["agg_fwd"]["spans"] + prof["agg_bwd"]["spans"]
     achieved = agg_bytes / (agg_ms * 1e-3) / 1e9 if agg_ms > 0 else None
     traffic = NCU_TRAFFIC["bytes_per_launch"] if NCU_TRAFFIC["spmm_sha1"] == spmm_source_hash() and args.scale == 1.0 else None
+    # compulsory bytes of the same launches: every source row read once instead of once per stored entry
+    # (three aggregation launches per step: widths dims[0], dims[1], dims[1]; BF16)
+    widths = [dims[0]] + [dims[k] for k in range(1, len(dims) - 1) for _ in (0, 1)]
+    gather_minus_min = sum((g.nnz - g.n) * f * 2 for f in widths) / max(len(widths), 1)
+    avg_launch_s = 1e-3 * agg_ms / max(agg_spans, 1)
+    min_bytes = agg_bytes / max(agg_spans, 1) - gather_minus_min
     roofline = {"bound": "hbm", "kernel": "spmm_csr_kernel (aggregation forward + adjoint)", "achieved": achieved, "peak": hbm_peak,
                 "unit": "GB/s", "frac": (achieved / hbm_peak) if achieved else None, "peak_source": f"of {peak_kind}",
                 "frac_of_nominal_8000": (achieved / 8000.0) if achieved else None, "traffic": traffic,
+                "dram_frac": (traffic / avg_launch_s / 1e9 / hbm_peak) if traffic and avg_launch_s > 0 else None,
+                "min_bytes_per_launch": min_bytes,
+                "t_bound_over_t": (min_bytes / (hbm_peak * 1e9) / avg_launch_s) if avg_launch_s > 0 else None,
+                "source_rows_fit_l2": bool(g.n * max(widths) * 2 <= 126e6),
                 "launches_timed": agg_spans, "avg_launch_us": 1e3 * agg_ms / max(agg_spans, 1),
                 "bytes_per_launch": agg_bytes / max(agg_spans, 1), "share_of_step": agg_ms / elapsed_ms,
                 "note": "algorithmic bytes, gather convention (each stored entry reads one source row); activations of this workload "

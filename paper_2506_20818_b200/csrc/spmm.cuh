@@ -234,7 +234,7 @@ LP_DEVINL void spmm_epilogue(const SpmmArgs<T> &a, int r, int gl, int nchunks, c
         for (int t = 0; t < VN; ++t) o[t] = acc_value<ACC>(acc[i][t]) * scale;
         if (irow >= 0) {
             Vec16<T> v;
-            v.load(a.init + (size_t)irow * a.ldinit + ch * VN);
+            v.load_once(a.init + (size_t)irow * a.ldinit + ch * VN);
             float f[VN];
             v.to_float(f);
 #pragma unroll
@@ -242,7 +242,7 @@ LP_DEVINL void spmm_epilogue(const SpmmArgs<T> &a, int r, int gl, int nchunks, c
         }
         if (a.relu_ref) {
             Vec16<T> v;
-            v.load(a.relu_ref + (size_t)r * a.ldref + ch * VN);
+            v.load_once(a.relu_ref + (size_t)r * a.ldref + ch * VN);
             float f[VN];
             v.to_float(f);
 #pragma unroll
@@ -250,7 +250,7 @@ LP_DEVINL void spmm_epilogue(const SpmmArgs<T> &a, int r, int gl, int nchunks, c
         }
         Vec16<T> out;
         out.from_float(o);
-        out.store(a.Y + (size_t)r * a.ldy + ch * VN);
+        out.store_once(a.Y + (size_t)r * a.ldy + ch * VN);
         if (srow >= 0) {
             Vec16<T> v;
             v.load(a.X + (size_t)srow * a.ldx + ch * VN);
