@@ -983,8 +983,19 @@ static lp_status build_blocks(lp_ctx *ctx, const int *pos_src, const int *pos_ds
             // sample: counts -> offsets -> columns (also marks the sampled ids; F_{h-1} is still marked)
             nbr_count_kernel<<<nblk(hb.n_dst + 1), 256, 0, st>>>(ctx->rowptr, prev.frontier, prev.n_front_dev, ctx->desc.fanout[h - 1], hb.blk_ptr, hb.n_dst);
             exclusive_scan_i32(ctx->ex, hb.blk_ptr, hb.n_dst, hb.blk_ptr, hb.blk_ptr + hb.n_dst, ctx->scan_tmp);
-            nbr_sample_kernel<<<nblk((int64_t)hb.n_dst * 32), 256, 0, st>>>(ctx->rowptr, ctx->col, prev.frontier, prev.n_front_dev, ctx->desc.fanout[h - 1], key,
-                                                              (uint32_t)step, (uint32_t)h, hb.blk_ptr, hb.blk_col_global, hb.blk_row, ctx->mark, hb.blk_eid);
+            {
+                const int fo = ctx->desc.fanout[h - 1];
+                const uint32_t st32 = (uint32_t)step, h32 = (uint32_t)h;
+                if (fo <= 8)
+                    nbr_sample_kernel<8><<<nblk((int64_t)hb.n_dst * 8), 256, 0, st>>>(ctx->rowptr, ctx->col, prev.frontier, prev.n_front_dev, fo, key, st32, h32,
+                                                                                      hb.blk_ptr, hb.blk_col_global, hb.blk_row, ctx->mark, hb.blk_eid);
+                else if (fo <= 16)
+                    nbr_sample_kernel<16><<<nblk((int64_t)hb.n_dst * 16), 256, 0, st>>>(ctx->rowptr, ctx->col, prev.frontier, prev.n_front_dev, fo, key, st32, h32,
+                                                                                        hb.blk_ptr, hb.blk_col_global, hb.blk_row, ctx->mark, hb.blk_eid);
+                else
+                    nbr_sample_kernel<32><<<nblk((int64_t)hb.n_dst * 32), 256, 0, st>>>(ctx->rowptr, ctx->col, prev.frontier, prev.n_front_dev, fo, key, st32, h32,
+                                                                                        hb.blk_ptr, hb.blk_col_global, hb.blk_row, ctx->mark, hb.blk_eid);
+            }
             inv_degree_kernel<<<nblk(hb.n_dst), 256, 0, st>>>(hb.blk_ptr, hb.n_dst, nullptr, hb.inv_deg);
             ctx->ex.launches += 3;
             if (h == K) {  // outermost hop: only the entry count is needed
@@ -1016,7 +1027,7 @@ static lp_status build_blocks(lp_ctx *ctx, const int *pos_src, const int *pos_ds
                 relabel_kernel<<<nblk(hb.entries), 256, 0, st>>>(hb.blk_col_global, hb.blk_ptr + hb.n_dst, hb.entries, hb.posmap, hb.blk_col_local);
                 ctx->ex.launches += 1;
             }
-            transpose_csr(ctx->ex, hb.blk_ptr, hb.n_dst, hb.n_src, hb.blk_col_local, hb.entries, hb.colptr, hb.rowidx, hb.perm, ctx->tsp);
+            transpose_csr(ctx->ex, hb.blk_ptr, hb.n_dst, hb.n_src, hb.blk_col_local, hb.entries, hb.colptr, hb.rowidx, hb.perm, ctx->tsp, hb.blk_row);
             if (gcn) {
                 gcn_block_coefficients(ctx, hb, ctx->hop[h - 1]);
                 if (hb.entries > 0) gather_f32_kernel<<<nblk(hb.entries), 256, 0, st>>>(hb.blk_val, hb.perm, hb.entries, hb.blk_valT);

@@ -86,23 +86,27 @@ __global__ void nbr_count_kernel(const int *__restrict__ rowptr, const int *__re
 
 // Floyd's subset algorithm: for q = 0..fanout-1, j = d - fanout + q, t uniform in [0, j];
 // take t unless already taken, else j.  Positions are emitted in ascending order.
-// One warp per frontier row: lane q evaluates draw q (the draws are independent counter-based
-// numbers), the "already taken" decisions are resolved in order with one ballot per draw, and
-// every lane finds the rank of its position among the (distinct) positions of the row.
+// One group of G lanes (8, 16 or 32, at least the fan-out) per frontier row: lane q evaluates draw q (the
+// draws are independent counter-based numbers), the "already taken" decisions are resolved in order
+// with one ballot per draw, and every lane finds the rank of its position among the (distinct)
+// positions of the row.
+template <int G>
 __global__ void nbr_sample_kernel(const int *__restrict__ rowptr, const int *__restrict__ col, const int *__restrict__ frontier,
                                   const int *__restrict__ n_front_dev, int fanout, uint2 key, uint32_t step_lo, uint32_t hop,
                                   const int *__restrict__ blk_ptr, int *__restrict__ blk_col_global, int *__restrict__ blk_row,
-                                  unsigned char *__restrict__ mark, int *__restrict__ blk_eid = nullptr)
+                                  unsigned char *__restrict__ mark, int *__restrict__ blk_eid)
 {
-    const int lane = threadIdx.x & 31;
-    const int64_t i64 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (i64 >= *n_front_dev) return;  // uniform over the warp
+    const unsigned lane = threadIdx.x & 31;
+    const int gl = threadIdx.x % G;  // lane inside the group
+    const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << (lane & ~(unsigned)(G - 1)));
+    const int64_t i64 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
+    if (i64 >= *n_front_dev) return;  // uniform over the group
     const int i = (int)i64;
     const int v = frontier[i];
     const int r0 = rowptr[v], d = rowptr[v + 1] - r0;
     const int out = blk_ptr[i];
     if (d <= fanout) {
-        for (int e = lane; e < d; e += 32) {
+        for (int e = gl; e < d; e += G) {
             const int u = col[r0 + e];
             blk_col_global[out + e] = u;
             blk_row[out + e] = i;
@@ -111,21 +115,21 @@ __global__ void nbr_sample_kernel(const int *__restrict__ rowptr, const int *__r
         }
         return;
     }
-    const int j = d - fanout + lane;
+    const int j = d - fanout + gl;
     int t = 0;
-    if (lane < fanout) {
-        const uint32_t x = philox4x32_10(make_uint4((uint32_t)v, (uint32_t)lane, step_lo, DRAW_NEIGHBOR | (hop << 8)), key).x;
+    if (gl < fanout) {
+        const uint32_t x = philox4x32_10(make_uint4((uint32_t)v, (uint32_t)gl, step_lo, DRAW_NEIGHBOR | (hop << 8)), key).x;
         t = (int)__umulhi(x, (uint32_t)(j + 1));
     }
     int mypos = -1;
     for (int q = 0; q < fanout; ++q) {
-        const int tq = __shfl_sync(0xffffffffu, t, q);
-        const unsigned taken = __ballot_sync(0xffffffffu, lane < q && mypos == tq);
-        if (lane == q) mypos = taken ? j : tq;
+        const int tq = __shfl_sync(gmask, t, q, G);
+        const unsigned taken = __ballot_sync(gmask, gl < q && mypos == tq);
+        if (gl == q) mypos = taken ? j : tq;
     }
     int rank = 0;
-    for (int z = 0; z < fanout; ++z) rank += __shfl_sync(0xffffffffu, mypos, z) < mypos ? 1 : 0;
-    if (lane < fanout) {
+    for (int z = 0; z < fanout; ++z) rank += __shfl_sync(gmask, mypos, z, G) < mypos ? 1 : 0;
+    if (gl < fanout) {
         const int u = col[r0 + mypos];
         blk_col_global[out + rank] = u;
         blk_row[out + rank] = i;

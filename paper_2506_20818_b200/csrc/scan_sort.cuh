@@ -275,6 +275,18 @@ __global__ void expand_entries_kernel(const int *__restrict__ rowptr, int n_rows
     rows[e] = lo;
 }
 
+// the same when the row of every entry is already known: keys, values and the per-column counts in one pass
+__global__ void expand_known_rows_kernel(const int *__restrict__ col, int64_t nnz, uint32_t *__restrict__ keys, uint32_t *__restrict__ vals,
+                                         int *__restrict__ counts)
+{
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= nnz) return;
+    const int c = col[e];
+    keys[e] = (uint32_t)c;
+    vals[e] = (uint32_t)e;
+    atomicAdd(&counts[c], 1);
+}
+
 __global__ void count_keys_kernel(const int *__restrict__ ids, int64_t m, int *__restrict__ counts)
 {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -309,19 +321,24 @@ struct TransposeScratch {
 // rowidx_t[nnz] (row of each transposed entry, ascending inside a transposed row because the
 // sort is stable and entries are visited in row order) and perm[nnz] (original entry index).
 static void transpose_csr(Exec &ex, const int *rowptr, int n_rows, int n_cols, const int *col, int64_t nnz, int *colptr,
-                          int *rowidx_t, int *perm, const TransposeScratch &s)
+                          int *rowidx_t, int *perm, const TransposeScratch &s, const int *rows_known = nullptr)
 {
     cudaMemsetAsync(colptr, 0, sizeof(int) * ((size_t)n_cols + 1), ex.st);
     if (nnz > 0) {
         const unsigned blocks = (unsigned)ceil_div64(nnz, 256);
-        expand_entries_kernel<<<blocks, 256, 0, ex.st>>>(rowptr, n_rows, col, nnz, s.keys, s.vals, s.rows);
-        count_keys_kernel<<<blocks, 256, 0, ex.st>>>(col, nnz, colptr);
-        ex.launches += 2;
+        if (rows_known) {  // the caller has the row of every entry (sampled blocks record it)
+            expand_known_rows_kernel<<<blocks, 256, 0, ex.st>>>(col, nnz, s.keys, s.vals, colptr);
+            ex.launches += 1;
+        } else {
+            expand_entries_kernel<<<blocks, 256, 0, ex.st>>>(rowptr, n_rows, col, nnz, s.keys, s.vals, s.rows);
+            count_keys_kernel<<<blocks, 256, 0, ex.st>>>(col, nnz, colptr);
+            ex.launches += 2;
+        }
     }
     exclusive_scan_i32(ex, colptr, n_cols, colptr, colptr + n_cols, s.scan_tmp);
     if (nnz > 0) {
         const bool in_place = radix_sort_pairs(ex, s.keys, s.vals, nnz, bits_for(n_cols), s.sort);
-        gather_rows_kernel<<<(unsigned)ceil_div64(nnz, 256), 256, 0, ex.st>>>(in_place ? s.vals : s.sort.vals_alt, s.rows, nnz, rowidx_t, perm);
+        gather_rows_kernel<<<(unsigned)ceil_div64(nnz, 256), 256, 0, ex.st>>>(in_place ? s.vals : s.sort.vals_alt, rows_known ? rows_known : s.rows, nnz, rowidx_t, perm);
         ex.launches += 1;
     }
 }
