@@ -33,10 +33,10 @@ K_NEG = 1
 SEED = 1234
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the aggregation launches of one step on the
-# benchmark workload, from one ncu capture (profiles/spmm_csr_bf16_config2.md): layer-1 forward 134.7 MB,
-# layer-2 forward 433.4 MB, adjoint 733.7 MB -> mean per timed launch.  Valid only for the kernel source it
-# was taken with (sha1 of csrc/spmm.cuh); reported as null otherwise.
-NCU_TRAFFIC = {"spmm_sha1": "d7a11d4a7910cc49bfe26c8fcf5c5d400edfec16", "bytes_per_launch": (134.7e6 + 433.4e6 + 733.7e6) / 3.0}
+# benchmark workload, from one ncu capture (profiles/spmm_csr_bf16_config2.md): layer-1 forward 119.8 MB,
+# layer-2 forward 398.1 MB, adjoint 604.5 MB -> mean per timed launch.  Valid only for the kernel source it
+# was taken with (sha1 of csrc/spmm.cuh + csrc/common.cuh); reported as null otherwise.
+NCU_TRAFFIC = {"spmm_sha1": "95e2e8530e91f695a44d7f992304bcf0fa5d5523", "bytes_per_launch": (119.8e6 + 398.1e6 + 604.5e6) / 3.0}
 
 
 def measured_peaks():
@@ -50,8 +50,9 @@ def measured_peaks():
 
 def spmm_source_hash():
     h = hashlib.sha1()
-    with open(os.path.join(ROOT, "paper_2506_20818_b200", "csrc", "spmm.cuh"), "rb") as f:
-        h.update(f.read())
+    for name in ("spmm.cuh", "common.cuh"):  # the kernel and the vector load / store forms it uses
+        with open(os.path.join(ROOT, "paper_2506_20818_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
     return h.hexdigest()
 
 
