@@ -17,6 +17,17 @@ __global__ void check_ids_kernel(const int *__restrict__ ids, int64_t m, int n_i
     if (i < m && (ids[i] < 0 || ids[i] >= n_ids)) atomicOr(err, 1);
 }
 
+// the same for the up to four id arrays of a step in one launch (null arrays are skipped)
+__global__ void check_step_ids_kernel(const int *__restrict__ a, int64_t na, const int *__restrict__ b, int64_t nb, const int *__restrict__ c, int64_t nc,
+                                      const int *__restrict__ d, int64_t nd, int n_ids, int *__restrict__ err)
+{
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int *p = a;
+    if (i >= na) { i -= na; p = b; if (i >= nb) { i -= nb; p = c; if (i >= nc) { i -= nc; p = d; if (i >= nd) return; } } }
+    const int v = p[i];
+    if (v < 0 || v >= n_ids) atomicOr(err, 1);
+}
+
 LP_DEVINL float warp_sum(float v)
 {
 #pragma unroll
@@ -42,7 +53,7 @@ __global__ void __launch_bounds__(EDGE_THREADS)
 edge_score_bce_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const int *__restrict__ idmap, const int *__restrict__ pos_src,
                       const int *__restrict__ pos_dst, int64_t B, const int *__restrict__ neg_src, const int *__restrict__ neg_dst, int k,
                       float inv_N, float *__restrict__ g_pos, float *__restrict__ g_neg, float *__restrict__ s_pos, float *__restrict__ s_neg,
-                      float *__restrict__ loss_partials)
+                      float *__restrict__ loss_partials, int *__restrict__ inc_counts = nullptr)
 {
     constexpr int VN = Vec16<T>::N;
     __shared__ float s_loss[EDGE_THREADS / 32];
@@ -89,12 +100,17 @@ edge_score_bce_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const 
         if (lane == 0) {
             g_pos[j] = dls * inv_N;
             if (s_pos) s_pos[j] = dot;
+            if (inc_counts) {  // lengths of the per-node incidence lists, counted while the endpoints are at hand
+                atomicAdd(&inc_counts[u], 1);
+                atomicAdd(&inc_counts[v], 1);
+            }
         }
         for (int kk = 0; kk < k; ++kk) {
             const int64_t t = j * k + kk;
             Vec16<T> cur[NV];
 #pragma unroll
             for (int i = 0; i < NV; ++i) cur[i] = nxt[i];
+            const int vn_cur = vn_nxt;
             if (kk + 1 < k) {
                 vn_nxt = clamp_id(neg_dst[t + 1], n_ids);
                 if (idmap) vn_nxt = idmap[vn_nxt];
@@ -133,6 +149,10 @@ edge_score_bce_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const 
             if (lane == 0) {
                 g_neg[t] = dls * inv_N;
                 if (s_neg) s_neg[t] = d2;
+                if (inc_counts) {
+                    atomicAdd(&inc_counts[un], 1);
+                    atomicAdd(&inc_counts[vn_cur], 1);
+                }
             }
         }
     }
@@ -146,21 +166,20 @@ edge_score_bce_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const 
     }
 }
 
-// loss = inv_N * sum of partials, added in index order by one block
-__global__ void loss_reduce_kernel(const float *__restrict__ partials, int64_t m, float inv_N, float *__restrict__ loss)
+// loss = inv_N * sum of partials: one block of 1024 threads, thread t adds partials t, t + 1024, ... in double
+// (tens of thousands of nearly equal terms), then a fixed binary tree over the threads
+__global__ void __launch_bounds__(1024) loss_reduce_kernel(const float *__restrict__ partials, int64_t m, float inv_N, float *__restrict__ loss)
 {
-    __shared__ double sh[256];  // the block partials are added in double: tens of thousands of nearly equal terms
+    __shared__ double sh[1024];
     double s = 0.0;
-    const int64_t per = (m + 255) / 256;
-    const int64_t b = per * threadIdx.x, e = min(m, b + per);
-    for (int64_t i = b; i < e; ++i) s += (double)partials[i];
+    for (int64_t i = threadIdx.x; i < m; i += 1024) s += (double)partials[i];
     sh[threadIdx.x] = s;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        double t = 0.0;
-        for (int i = 0; i < 256; ++i) t += sh[i];
-        *loss = (float)(t * (double)inv_N);
+    for (int w = 512; w > 0; w >>= 1) {
+        if ((int)threadIdx.x < w) sh[threadIdx.x] += sh[threadIdx.x + w];
+        __syncthreads();
     }
+    if (threadIdx.x == 0) *loss = (float)(sh[0] * (double)inv_N);
 }
 
 // plain scores for lp_score: one warp per edge

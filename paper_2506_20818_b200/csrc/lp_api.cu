@@ -1200,11 +1200,11 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     const bool sage = ctx->desc.arch == LP_SAGE_MEAN;
     const int D = ctx->desc.dims[K];
     // bad ids are clamped by every consumer and reported through the context's error word
-    check_ids_kernel<<<nblk(B), 256, 0, st>>>(pos_src, B, ctx->n, ctx->err_flag);
-    check_ids_kernel<<<nblk(B), 256, 0, st>>>(pos_dst, B, ctx->n, ctx->err_flag);
-    if (k > 0) check_ids_kernel<<<nblk(B * k), 256, 0, st>>>(neg_dst, B * k, ctx->n, ctx->err_flag);
-    if (k > 0 && neg_src) check_ids_kernel<<<nblk(B * k), 256, 0, st>>>(neg_src, B * k, ctx->n, ctx->err_flag);
-    ctx->ex.launches += 2 + (k > 0) + (k > 0 && neg_src);
+    {
+        const int64_t nk = k > 0 ? B * k : 0;
+        check_step_ids_kernel<<<nblk(2 * B + 2 * nk), 256, 0, st>>>(pos_src, B, pos_dst, B, neg_dst, nk, neg_src, (k > 0 && neg_src) ? nk : 0, ctx->n, ctx->err_flag);
+        ctx->ex.launches += 1;
+    }
     if (ctx->sampled) {
         lp_status s = build_blocks(ctx, pos_src, pos_dst, B, neg_src, neg_dst, k, seed, step);
         if (s != LP_OK) return s;
@@ -1223,28 +1223,29 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     constexpr int VN = Vec16<T>::N;
     const int chunks = D / VN;
     const float *g_pos = ctx->g_pos, *g_neg = ctx->g_neg;
+    // the dot-product scoring kernel also counts the incidence-list lengths (into the zeroed offsets array)
+    CK(cudaMemsetAsync(ctx->inc_ptr, 0, sizeof(int) * ((size_t)rows_out + 1), st));
     if (ctx->mlp) {
         s = predictor_forward<T>(ctx, params, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k);
         if (s != LP_OK) { delete pscore; return s; }
         const unsigned lblocks = nblk(E, 256);
         bce_from_scores_kernel<<<lblocks, 256, 0, st>>>(ctx->pred_scores, E, B, inv_N, ctx->g_pos, ctx->loss_partials);
-        loss_reduce_kernel<<<1, 256, 0, st>>>(ctx->loss_partials, lblocks, inv_N, loss);
+        loss_reduce_kernel<<<1, 1024, 0, st>>>(ctx->loss_partials, lblocks, inv_N, loss);
         g_neg = ctx->g_pos + B;  // one array: positives, then negatives
         s = predictor_backward<T>(ctx, params, E, ctx->g_pos, grads, accumulate);
         if (s != LP_OK) { delete pscore; return s; }
     } else {
-        if (chunks <= 32) edge_score_bce_kernel<T, 1><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials);
-        else if (chunks <= 64) edge_score_bce_kernel<T, 2><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials);
-        else edge_score_bce_kernel<T, 4><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials);
-        loss_reduce_kernel<<<1, 256, 0, st>>>(ctx->loss_partials, eblocks, inv_N, loss);
+        if (chunks <= 32) edge_score_bce_kernel<T, 1><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials, ctx->inc_ptr);
+        else if (chunks <= 64) edge_score_bce_kernel<T, 2><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials, ctx->inc_ptr);
+        else edge_score_bce_kernel<T, 4><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials, ctx->inc_ptr);
+        loss_reduce_kernel<<<1, 1024, 0, st>>>(ctx->loss_partials, eblocks, inv_N, loss);
     }
     delete pscore;
     ctx->ex.launches += 2;
 
     // incidence lists of the scored edges, grouped by node (slots claimed with integer atomics)
     ProfScope *pinc = new ProfScope(ctx->ex, LP_PROF_INCIDENCE, (double)E * 2.0 * 24.0);
-    CK(cudaMemsetAsync(ctx->inc_ptr, 0, sizeof(int) * ((size_t)rows_out + 1), st));
-    incidence_count_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->inc_ptr);
+    if (ctx->mlp) incidence_count_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->inc_ptr);
     exclusive_scan_i32(ctx->ex, ctx->inc_ptr, rows_out, ctx->inc_ptr, ctx->inc_ptr + rows_out, ctx->scan_tmp);
     CK(cudaMemcpyAsync(ctx->inc_cursor, ctx->inc_ptr, sizeof(int) * (size_t)rows_out, cudaMemcpyDeviceToDevice, st));
     incidence_fill_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, g_pos, g_neg, ctx->inc_cursor, ctx->inc_col,
