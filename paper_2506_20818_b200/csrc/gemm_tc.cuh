@@ -458,6 +458,7 @@ LP_DEVINL void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" :
 LP_DEVINL void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 LP_DEVINL void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 LP_DEVINL void epilogue_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }  // the eight epilogue warps only
+LP_DEVINL void group_barrier(int grp) { asm volatile("bar.sync %0, 128;" ::"r"(2 + grp) : "memory"); }  // the four warps of one box group
 
 
 __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(const __grid_constant__ CUtensorMap mapA,
@@ -589,13 +590,15 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
                 const int m0 = (int)((first_tile + i * stride) * TC_BM);
                 const int row_t = q * 32 + lane;  // row inside the tile
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN);
-                const bool store_thread = (warp == 2 && lane == 0);
+                const bool store_thread = (((warp - 2) & 3) == 0 && lane == 0);  // one per box group (warps 2 and 6)
                 const float rs = (p.row_scale && (int64_t)m0 + row_t < p.M) ? __ldg(p.row_scale + m0 + row_t) : 1.f;
                 for (int half = 0; half < BN; half += 128) {
                     const int nbox = min(2, (BN - half) / 64);
-                    if (store_thread) tma_store_wait_read();  // the previous stores have read the staging area
-                    epilogue_barrier();
+                    // the two box groups (four warps, one 64-column staging box each) run independently: a group waits
+                    // only for its own previous store and synchronises only its own 128 threads
                     if (my_box < nbox) {
+                        if (store_thread) tma_store_wait_read();  // this group's previous store has read its staging box
+                        group_barrier(my_box);
                         const int cb = half + my_box * 64;
                         uint32_t r[2][32];
                         tmem_ld_32x32_issue(taddr + (uint32_t)cb, r[0]);
@@ -631,12 +634,12 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
                                 *reinterpret_cast<uint4 *>(box + (((chunk0 + j) ^ (row_t & 7)) << 4)) = o.v;
                             }
                         }
-                    }
-                    fence_async_proxy();  // generic-proxy writes -> visible to the TMA engine
-                    epilogue_barrier();
-                    if (store_thread) {
-                        for (int bx = 0; bx < nbox; ++bx) tma_store_2d(&mapC, smem_u32(smem_out + (size_t)bx * 16384), n0 + half + bx * 64, m0);
-                        tma_store_commit();
+                        fence_async_proxy();  // generic-proxy writes -> visible to the TMA engine
+                        group_barrier(my_box);
+                        if (store_thread) {
+                            tma_store_2d(&mapC, smem_u32(smem_out + (size_t)my_box * 16384), n0 + half + my_box * 64, m0);
+                            tma_store_commit();
+                        }
                     }
                 }
                 tc_fence_before();
@@ -645,7 +648,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
             }
         }
     }
-    if (warp == 2 && lane == 0) tma_store_wait_all();  // output tiles are in global memory before the CTA leaves
+    if ((warp == 2 || warp == 6) && lane == 0) tma_store_wait_all();  // output tiles are in global memory before the CTA leaves
     __syncwarp();
     tc_fence_before();
     __syncthreads();
