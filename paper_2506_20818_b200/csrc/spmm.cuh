@@ -119,7 +119,9 @@ constexpr int SPMM_SEG = 512;    // entries per item (one block: 8 lane groups x
 
 // acc += sum over entries [e_lo, e_hi) of val[e] * X[col[e], :] for the chunks owned by this lane.
 // The group loads up to G (col, val) pairs at once and broadcasts them; U source rows are gathered
-// before any is consumed, so each lane keeps U * NV 16-byte loads in flight.
+// before any is consumed, so each lane keeps U * NV 16-byte loads in flight.  Lanes beyond the row
+// width repeat the last chunk (their sums are never stored), which keeps the gathers free of
+// per-lane predicates.
 template <typename T, int G, int NV, int U, typename ACC, bool HAS_VAL, bool HAS_X2 = false>
 LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl, unsigned gmask, int nchunks, ACC (&acc)[NV][Vec16<T>::N],
                                 bool have_first = false, int first_col = 0, float first_val = 0.f)
@@ -153,10 +155,7 @@ LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl,
 #pragma unroll
             for (int q = 0; q < U; ++q)
 #pragma unroll
-                for (int i = 0; i < NV; ++i) {
-                    const int ch = gl + i * G;
-                    if (ch < nchunks) v[q][i].load(a.X + (size_t)c[q] * a.ldx + ch * VN);
-                }
+                for (int i = 0; i < NV; ++i) v[q][i].load(a.X + (size_t)c[q] * a.ldx + min(gl + i * G, nchunks - 1) * VN);
             if (HAS_X2) {
 #pragma unroll
                 for (int q = 0; q < U; ++q) {
@@ -179,10 +178,7 @@ LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl,
 #pragma unroll
                 for (int q = 0; q < U; ++q)
 #pragma unroll
-                    for (int i = 0; i < NV; ++i) {
-                        const int ch = gl + i * G;
-                        if (ch < nchunks) acc_add_vec<T, ACC, HAS_VAL>(acc[i], w[q], v[q][i]);
-                    }
+                    for (int i = 0; i < NV; ++i) acc_add_vec<T, ACC, HAS_VAL>(acc[i], w[q], v[q][i]);
             }
         }
         for (; j < cnt; ++j) {
@@ -192,9 +188,9 @@ LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl,
 #pragma unroll
             for (int i = 0; i < NV; ++i) {
                 const int ch = gl + i * G;
-                if (ch < nchunks) {
+                if (HAS_X2 ? ch < nchunks : true) {
                     Vec16<T> v;
-                    v.load(a.X + (size_t)c * a.ldx + ch * VN);
+                    v.load(a.X + (size_t)c * a.ldx + min(ch, nchunks - 1) * VN);
                     if (HAS_X2) {
                         Vec16<T> v2;
                         v2.load(a.X2 + (size_t)c2 * a.ldx2 + ch * VN);
