@@ -33,10 +33,10 @@ K_NEG = 1
 SEED = 1234
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the aggregation launches of one step on the
-# benchmark workload, from one ncu capture (profiles/spmm_csr_bf16_config2.md): layer-1 forward 119.8 MB,
-# layer-2 forward 398.1 MB, adjoint 604.5 MB -> mean per timed launch.  Valid only for the kernel source it
+# benchmark workload, from one ncu capture (profiles/spmm_csr_bf16_config2.md): layer-1 forward 121.5 MB,
+# layer-2 forward 397.9 MB, adjoint 608.0 MB -> mean per timed launch.  Valid only for the kernel source it
 # was taken with (sha1 of csrc/spmm.cuh + csrc/common.cuh); reported as null otherwise.
-NCU_TRAFFIC = {"spmm_sha1": "95e2e8530e91f695a44d7f992304bcf0fa5d5523", "bytes_per_launch": (119.8e6 + 398.1e6 + 604.5e6) / 3.0}
+NCU_TRAFFIC = {"spmm_sha1": "db609f90a1a3efc7130110a97cd8e51e06baad64", "bytes_per_launch": (121.5e6 + 397.9e6 + 608.0e6) / 3.0}
 
 
 def measured_peaks():

@@ -1,0 +1,75 @@
+"""Operator-level timing of the library's single-operator entry points on a synthetic graph.
+
+    python -m paper_2506_20818_b200.opbench --op aggregate --nodes 1000000 --mean-degree 16 --width 256
+
+times `lp_op_aggregate` (AGG of Eq. 1 and, with --transpose, its adjoint) with CUDA events and prints one JSON
+line: microseconds per launch, the algorithmic bytes of the launch in the gather convention (every stored entry
+reads one source row; offsets, indices and the output once) and in the compulsory convention (every source row
+once), and both divided by the time.  The graph is the Chung-Lu power-law generator of the benchmark workloads;
+with --nodes 1000000 --mean-degree 16 it is the graph of the partitioned configuration, whose 512 MB BF16 source
+matrix does not fit the L2 cache, so the launch is bound by HBM rather than by L2 gathers.  Used for the ncu
+captures of single kernels (few launches, small process).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import numpy as np
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--op", choices=["aggregate"], default="aggregate")
+    ap.add_argument("--nodes", type=int, default=1_000_000)
+    ap.add_argument("--mean-degree", type=float, default=16.0)
+    ap.add_argument("--exponent", type=float, default=2.1)
+    ap.add_argument("--width", type=int, default=256)
+    ap.add_argument("--arch", choices=["sage", "gcn"], default="sage")
+    ap.add_argument("--transpose", action="store_true")
+    ap.add_argument("--fp32", action="store_true")
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--seed", type=int, default=5)
+    args = ap.parse_args()
+
+    import torch
+    import workloads as wl
+    from . import Context
+
+    g = wl.chung_lu(args.nodes, args.mean_degree, args.exponent, seed=args.seed)
+    ctx = Context(0)
+    ctx.load_graph(g.n, g.rowptr, g.col, g.w, wl.node_features(g.n, 8, args.seed))
+    torch.manual_seed(args.seed)
+    H = torch.randn(g.n, args.width, device="cuda:0")
+    if not args.fp32:
+        H = H.to(torch.bfloat16)
+    es = H.element_size()
+    for _ in range(args.warmup):
+        ctx.op_aggregate(args.arch, H, transpose=args.transpose)
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(args.iters):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        ctx.op_aggregate(args.arch, H, transpose=args.transpose)
+        b.record()
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b) * 1e3)
+    us = float(np.median(times))
+    per_entry = 4 + (4 if (args.arch == "gcn" or args.transpose) else 0)
+    fixed = (g.n + 1) * 4 + g.n * args.width * es + (g.n * 4 if args.arch == "sage" and not args.transpose else 0)
+    if args.arch == "gcn":
+        fixed += g.n * args.width * es + g.n * 4  # self term
+    gather = g.nnz * (args.width * es + per_entry) + fixed
+    compulsory = g.n * args.width * es + g.nnz * per_entry + fixed
+    print(json.dumps({"op": "aggregate", "arch": args.arch, "transpose": args.transpose, "dtype": "fp32" if args.fp32 else "bf16",
+                      "nodes": g.n, "entries": int(g.nnz), "width": args.width, "us_per_launch": round(us, 1),
+                      "gather_bytes": gather, "gather_GBps": round(gather / us / 1e3, 1),
+                      "compulsory_bytes": compulsory, "compulsory_GBps": round(compulsory / us / 1e3, 1),
+                      "source_matrix_MB": round(g.n * args.width * es / 1e6, 1)}))
+    ctx.close()
+
+
+if __name__ == "__main__":
+    main()
