@@ -300,6 +300,33 @@ def main():
                 "note": "algorithmic bytes, gather convention (each stored entry reads one source row); activations of this workload "
                         "partly fit the 126 MB L2, so the figure can exceed DRAM bandwidth"}
 
+    # ---- gather ceiling of the same launches (outside the timed region): the bare gather of the index streams the
+    # three aggregation launches of a step walk (lp_op_gather_ceiling: no rows, arithmetic or epilogue).  With the source
+    # matrix largely L2 resident this, not the HBM copy bandwidth, is the floor of the aggregation kernel.
+    if rank == 0:
+        def probe_us(width, transpose):
+            Hp = torch.randn((g.n, width), device=dev).to(torch.bfloat16)
+            ev = []
+            with torch.cuda.stream(stream):
+                for it in range(8):
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record(stream)
+                    ctx.op_gather_ceiling(Hp, transpose=transpose)
+                    b.record(stream)
+                    ev.append((a, b))
+            stream.synchronize()
+            return 1e3 * statistics.median(a.elapsed_time(b) for a, b in ev[3:])
+
+        # forward launches walk the CSR, the adjoint launch the transposed structure (layer 1 has no adjoint)
+        shapes = [(dims[k], False) for k in range(len(dims) - 1)] + [(dims[k], True) for k in range(1, len(dims) - 1)]
+        if all(f * 2 in (128, 256, 512) for f, _ in shapes):
+            floor_us = sum(probe_us(f, tr) for f, tr in shapes)
+            agg_us_per_step = 1e3 * agg_ms / args.steps
+            roofline["gather_ceiling"] = {"floor_us_per_step": floor_us, "aggregation_us_per_step": agg_us_per_step,
+                                          "frac": floor_us / agg_us_per_step if agg_us_per_step > 0 else None,
+                                          "note": "time of lp_op_gather_ceiling over the same index streams and row widths "
+                                                  "divided by the aggregation time of a step"}
+
     # ---- optional breakdown of a few more steps, outside the timed region
     breakdown = None
     if args.breakdown or rank == 0:

@@ -324,6 +324,15 @@ lp_status lp_profile_end(lp_ctx *ctx, lp_profile *out);
  * H and M are [n, F] row-major device arrays; F a multiple of 8, F <= 512. */
 lp_status lp_op_aggregate(lp_ctx *ctx, int32_t arch, int32_t transpose, int32_t bf16, const void *H, int32_t F, void *M);
 
+/* (No counterpart in the paper: a measurement aid for the roofline of lp_op_aggregate.)
+ * Bare gather over the loaded graph's index stream: the stored entries (column indices of the CSR, or the row
+ * indices of its transpose when transpose = 1) are cut into runs of 64 consecutive entries; for every run the rows
+ * H[index] (row_bytes bytes each, row-major, n rows) are loaded and folded with bitwise XOR, and folds receives
+ * ceil(nnz / 64) rows of row_bytes bytes.  No row structure, arithmetic or epilogue: the time of this call is the
+ * floor for any kernel that gathers these rows in this order, whether they come from L2 or from HBM.
+ *   H, folds : DEVICE, 16-byte aligned, caller-owned; row_bytes in {128, 256, 512}.  Does not synchronise. */
+lp_status lp_op_gather_ceiling(lp_ctx *ctx, int32_t transpose, const void *H, int32_t row_bytes, void *folds);
+
 /* Dense transform C[M, N] = A[M, K] * B + bias, optional ReLU; B is [K, N] row-major
  * (trans_b = 0) or [N, K] row-major (trans_b = 1).  prec LP_FP32: float32 everywhere;
  * LP_BF16: A, B, C are BF16 words, bias float32, FP32 accumulation on the tensor cores. */

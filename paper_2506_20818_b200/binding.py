@@ -26,7 +26,7 @@ EXPORTS = [
     "lp_create", "lp_destroy", "lp_last_error", "lp_load_graph", "lp_get_structure", "lp_set_model",
     "lp_param_count", "lp_set_candidates", "lp_sample_negatives", "lp_train_step", "lp_train_step_host",
     "lp_adam_step", "lp_score", "lp_get_embeddings", "lp_get_output_gradient", "lp_get_block",
-    "lp_get_stats", "lp_op_aggregate", "lp_op_linear", "lp_op_weight_grad", "lp_profile_begin", "lp_profile_end",
+    "lp_get_stats", "lp_op_aggregate", "lp_op_gather_ceiling", "lp_op_linear", "lp_op_weight_grad", "lp_profile_begin", "lp_profile_end",
     "lp_weight_grad_static", "lp_sparsify", "lp_get_sparsified",
     "lp_worker_view", "lp_get_worker_view", "lp_hits_at_k", "lp_get_predictor_activations",
 ]
@@ -311,6 +311,15 @@ class Context:
         self._ck(self.lib.lp_op_aggregate(self.h, C.c_int32(LP_GCN if arch == "gcn" else LP_SAGE_MEAN), C.c_int32(int(transpose)),
                                           C.c_int32(int(H.dtype == t.bfloat16)), _ptr(H), C.c_int32(H.shape[1]), _ptr(M)))
         return M
+
+    def op_gather_ceiling(self, H, transpose: bool = False):
+        """XOR folds of the rows of H named by every run of 64 stored entries (see lp_op_gather_ceiling)."""
+        t = self._torch
+        row_bytes = H.shape[1] * H.element_size()
+        runs = (self.nnz + 63) // 64
+        folds = t.empty((runs, row_bytes // 4), dtype=t.int32, device=H.device)
+        self._ck(self.lib.lp_op_gather_ceiling(self.h, C.c_int32(int(transpose)), _ptr(H), C.c_int32(row_bytes), _ptr(folds)))
+        return folds
 
     def op_linear(self, A, B, bias=None, relu: bool = False, trans_b: bool = False):
         t = self._torch

@@ -15,6 +15,7 @@
 #include "sparsify.cuh"
 #include "view.cuh"
 #include "predictor.cuh"
+#include "probe.cuh"
 
 // ----------------------------------------------------------------------------------------------
 // context
@@ -1696,6 +1697,19 @@ extern "C" lp_status lp_op_aggregate(lp_ctx *ctx, int32_t arch, int32_t transpos
     CK(cudaSetDevice(ctx->device));
     return is_bf16 ? op_aggregate_impl<bf16>(ctx, arch, transpose, (const bf16 *)H, F, (bf16 *)M)
                    : op_aggregate_impl<float>(ctx, arch, transpose, (const float *)H, F, (float *)M);
+}
+
+extern "C" lp_status lp_op_gather_ceiling(lp_ctx *ctx, int32_t transpose, const void *H, int32_t row_bytes, void *folds)
+{
+    if (!ctx) return LP_EINVAL;
+    if (!ctx->loaded) return fail(ctx, LP_ESTATE, "lp_op_gather_ceiling: no graph loaded");
+    if (!H || !folds) return fail(ctx, LP_EINVAL, "lp_op_gather_ceiling: H and folds must be non-null");
+    if (row_bytes != 128 && row_bytes != 256 && row_bytes != 512) return fail(ctx, LP_EINVAL, "lp_op_gather_ceiling: row_bytes must be 128, 256 or 512");
+    if (((uintptr_t)H & 15) != 0 || ((uintptr_t)folds & 15) != 0) return fail(ctx, LP_EINVAL, "lp_op_gather_ceiling: H and folds must be 16-byte aligned");
+    CK(cudaSetDevice(ctx->device));
+    gather_probe_launch(ctx->ex, transpose ? ctx->rowidx : ctx->col, ctx->nnz, H, row_bytes, folds);
+    CK_LAUNCH();
+    return LP_OK;
 }
 
 extern "C" lp_status lp_op_linear(lp_ctx *ctx, int32_t prec, int64_t M, int32_t N, int32_t K, const void *A, const void *B, int32_t trans_b,

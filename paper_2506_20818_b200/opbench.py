@@ -2,7 +2,8 @@
 
     python -m paper_2506_20818_b200.opbench --op aggregate --nodes 1000000 --mean-degree 16 --width 256
 
-times `lp_op_aggregate` (AGG of Eq. 1 and, with --transpose, its adjoint) with CUDA events and prints one JSON
+times `lp_op_aggregate` (AGG of Eq. 1 and, with --transpose, its adjoint; `--op gather-ceiling`: the bare gather of the
+same index stream, `lp_op_gather_ceiling`, the floor of any such kernel) with CUDA events and prints one JSON
 line: microseconds per launch, the algorithmic bytes of the launch in the gather convention (every stored entry
 reads one source row; offsets, indices and the output once) and in the compulsory convention (every source row
 once), and both divided by the time.  The graph is the Chung-Lu power-law generator of the benchmark workloads;
@@ -20,7 +21,7 @@ import numpy as np
 
 def main() -> None:
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", choices=["aggregate"], default="aggregate")
+    ap.add_argument("--op", choices=["aggregate", "gather-ceiling"], default="aggregate")
     ap.add_argument("--nodes", type=int, default=1_000_000)
     ap.add_argument("--mean-degree", type=float, default=16.0)
     ap.add_argument("--exponent", type=float, default=2.1)
@@ -45,18 +46,29 @@ def main() -> None:
     if not args.fp32:
         H = H.to(torch.bfloat16)
     es = H.element_size()
+    if args.op == "gather-ceiling":
+        run = lambda: ctx.op_gather_ceiling(H, transpose=args.transpose)  # noqa: E731
+    else:
+        run = lambda: ctx.op_aggregate(args.arch, H, transpose=args.transpose)  # noqa: E731
     for _ in range(args.warmup):
-        ctx.op_aggregate(args.arch, H, transpose=args.transpose)
+        run()
     torch.cuda.synchronize()
     times = []
     for _ in range(args.iters):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
-        ctx.op_aggregate(args.arch, H, transpose=args.transpose)
+        run()
         b.record()
         torch.cuda.synchronize()
         times.append(a.elapsed_time(b) * 1e3)
     us = float(np.median(times))
+    if args.op == "gather-ceiling":
+        moved = g.nnz * (args.width * es + 4) + ((g.nnz + 63) // 64) * args.width * es
+        print(json.dumps({"op": "gather-ceiling", "transpose": args.transpose, "nodes": g.n, "entries": int(g.nnz), "row_bytes": args.width * es,
+                          "us_per_launch": round(us, 1), "gather_bytes": moved, "gather_GBps": round(moved / us / 1e3, 1),
+                          "source_matrix_MB": round(g.n * args.width * es / 1e6, 1)}))
+        ctx.close()
+        return
     per_entry = 4 + (4 if (args.arch == "gcn" or args.transpose) else 0)
     fixed = (g.n + 1) * 4 + g.n * args.width * es + (g.n * 4 if args.arch == "sage" and not args.transpose else 0)
     if args.arch == "gcn":

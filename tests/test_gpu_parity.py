@@ -119,6 +119,22 @@ def test_aggregate_bf16(pkg, F):
     ctx.close()
 
 
+@pytest.mark.parametrize("words", [32, 64, 128])
+def test_gather_ceiling_folds_are_exact(pkg, words):
+    # the measurement kernel behind the roofline figures does the gathers it claims: XOR folds of runs of 64 entries,
+    # an integer result, checked against numpy on a graph whose entry count leaves a ragged last run
+    g = wl.chung_lu(5000, 12.0, 2.1, seed=9)
+    assert g.nnz % 64 != 0
+    ctx = make_ctx(pkg, g, wl.node_features(g.n, 8, 0))
+    H = np.random.default_rng(2).integers(-2**31, 2**31 - 1, size=(g.n, words), dtype=np.int64).astype(np.int32)
+    _, rowidx, _ = ctx.get_structure()
+    for transpose, idx in ((False, g.col), (True, rowidx.cpu().numpy())):
+        folds = ctx.op_gather_ceiling(t32(H), transpose=transpose).cpu().numpy()
+        ref = np.bitwise_xor.reduceat(H[idx], np.arange(0, g.nnz, 64), axis=0)
+        assert folds.shape == ref.shape and np.array_equal(folds, ref)
+    ctx.close()
+
+
 # ------------------------------------------------------------------------------------------ dense transforms
 @pytest.mark.parametrize("M,K,N", [(1000, 64, 64), (3333, 256, 256), (517, 512, 256), (129, 128, 264), (1, 8, 8)])
 def test_linear_and_weight_grad_fp32(pkg, M, K, N):
