@@ -28,6 +28,7 @@ template <> struct Vec16<float> {
     float4 v;
     LP_DEVINL void load(const float *p) { v = __ldg(reinterpret_cast<const float4 *>(p)); }
     LP_DEVINL void store(float *p) const { *reinterpret_cast<float4 *>(p) = v; }
+    LP_DEVINL void zero() { v = make_float4(0.f, 0.f, 0.f, 0.f); }
     LP_DEVINL void load_once(const float *p) { v = __ldcs(reinterpret_cast<const float4 *>(p)); }
     LP_DEVINL void store_once(float *p) const { __stcs(reinterpret_cast<float4 *>(p), v); }
     LP_DEVINL void to_float(float *f) const { f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w; }
@@ -38,6 +39,7 @@ template <> struct Vec16<bf16> {
     uint4 v;
     LP_DEVINL void load(const bf16 *p) { v = __ldg(reinterpret_cast<const uint4 *>(p)); }
     LP_DEVINL void store(bf16 *p) const { *reinterpret_cast<uint4 *>(p) = v; }
+    LP_DEVINL void zero() { v = make_uint4(0u, 0u, 0u, 0u); }
     // streaming forms for data touched once per launch (evicted first, so gathered rows keep their place in L2)
     LP_DEVINL void load_once(const bf16 *p) { v = __ldcs(reinterpret_cast<const uint4 *>(p)); }
     LP_DEVINL void store_once(bf16 *p) const { __stcs(reinterpret_cast<uint4 *>(p), v); }

@@ -31,6 +31,22 @@ struct HeavyPlan {
     float *partials = nullptr;
     int host_rows = -1, host_items = -1;  // -1: unknown on the host (plan built on the device per launch)
     int threshold = 64;                   // rows with more entries than this are heavy (>= SPMM_HEAVY_MIN)
+    int seg = 512;                        // entries per item (SPMM_SEG; SPMM_PIECE for the padded form's own plan)
+    // Static structures only: every row again in padded form for spmm_padded_kernel.  A row is cut into pieces of at
+    // most SPMM_PIECE entries (one piece unless it is heavy), a piece into groups of four entries (pad index -1, pad
+    // coefficient 0; an empty row keeps one all-pad group so that its output is written).  pcol / pval hold the groups
+    // back to back; grow[g] is -1 inside a piece, the row r >= 0 when group g finishes the only piece of row r, and
+    // -(2 + slot) when it finishes a piece of a heavy row whose FP32 partial sum goes to slot `slot` of `partials`
+    // (p_rows / p_base / p_counts list the heavy rows and their first slots for the combine kernel).  chunk_start
+    // cuts the groups into chunks that begin at piece starts (n_chunks + 1 offsets).
+    const int4 *pcol = nullptr;
+    const float4 *pval = nullptr;
+    const float *pval_src = nullptr;      // the per-entry coefficient array pval was padded from
+    const int *grow = nullptr;
+    const int *chunk_start = nullptr;
+    int n_chunks = 0;
+    int *p_rows = nullptr, *p_base = nullptr, *p_counts = nullptr;
+    int p_host_rows = 0;
 };
 
 template <typename T> struct SpmmArgs {
@@ -116,6 +132,8 @@ constexpr int SPMM_HEAVY_MIN = 64;  // smallest heavy-row threshold a plan may u
                                     // group is a long dependent chain: long rows are cut into items instead.
 constexpr int SPMM_ITEM_BLOCKS = 1184;  // blocks that walk the item list (grid-stride)
 constexpr int SPMM_SEG = 512;    // entries per item (one block: 8 lane groups x 64 entries for 32-lane groups)
+constexpr int SPMM_PIECE = 128;  // entries per piece of the padded form (= the heavy-row threshold of static structures)
+constexpr int SPMM_CHUNK_GROUPS = 16;  // groups of four entries per chunk of the padded form (one lane group walks a chunk)
 
 // acc += sum over entries [e_lo, e_hi) of val[e] * X[col[e], :] for the chunks owned by this lane.
 // The group loads up to G (col, val) pairs at once and broadcasts them; U source rows are gathered
@@ -277,7 +295,7 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
         for (int item = blockIdx.x - light_blocks; item < n_items; item += gridDim.x - light_blocks) {
         const int r = a.heavy.item_row[item];
         const int sidx = item - a.heavy.item_first[item];
-        const int hb = a.rowptr[r] + sidx * SPMM_SEG, he = min(a.rowptr[r + 1], hb + SPMM_SEG);
+        const int hb = a.rowptr[r] + sidx * a.heavy.seg, he = min(a.rowptr[r + 1], hb + a.heavy.seg);
         const int piece = ((he - hb + NG - 1) / NG + G - 1) / G * G;
         const int lo = min(he, hb + g * piece), hi = min(he, lo + piece);
         ACC hacc[NV][VN];
@@ -357,19 +375,177 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Padded flat form for static structures (one 16-byte vector per lane, FP32 sums, source rows G * MULT vectors apart).
+// A lane group streams the groups of one chunk: the four rows a group names are gathered at once and added in entry
+// order; when the group finishes a piece, the epilogue runs (only piece of a row) or the FP32 partial row is written
+// for the combine kernel (piece of a heavy row), and the sums restart from zero.  A row that is one piece is summed
+// in the same order as by the row-per-group kernel and gives the same bits.  Nothing in the inner loop depends on a
+// row's length: no tails, no per-entry end tests, the next group's indices are fetched while this group's rows are
+// in flight, a short row costs one group instead of a round trip of its own, and hub rows are pieces like any other.
+// Only the last group of a piece can hold pads; there the loads are predicated and the pads add zeros.
+// ---------------------------------------------------------------------------------------------
+// PLAIN: the epilogue is the row scale alone (mean aggregation forward); it is written out here so that the loop
+// keeps the register budget of a bare gather.
+LP_DEVINL void prefetch_l1(const void *p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
+
+template <typename T, int G, int MULT, int MINB, bool HAS_VAL, bool PLAIN>
+__global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_padded_kernel(const SpmmArgs<T> a)
+{
+    constexpr int VN = Vec16<T>::N;
+    constexpr int NG = SPMM_THREADS / G;
+    constexpr unsigned PITCH = (unsigned)(G * VN * MULT);  // elements between source rows
+    const int gl = threadIdx.x % G;
+    const int nchunks = a.F / VN;
+    const int c = blockIdx.x * NG + threadIdx.x / G;
+    if (c >= a.heavy.n_chunks) return;
+    const int gs = __ldg(a.heavy.chunk_start + c), ge = __ldg(a.heavy.chunk_start + c + 1);
+    if (gs >= ge) return;
+    const T *xl = a.X + min(gl, nchunks - 1) * VN;  // lanes beyond the row width repeat the last chunk and store nothing
+    float acc[1][VN];
+#pragma unroll
+    for (int t = 0; t < VN; ++t) acc[0][t] = 0.f;
+    int4 cn = __ldg(a.heavy.pcol + gs);
+    float4 wn = HAS_VAL ? __ldg(a.heavy.pval + gs) : make_float4(1.f, 1.f, 1.f, 1.f);
+    int rn = __ldg(a.heavy.grow + gs);
+    for (int grp = gs; grp < ge; ++grp) {
+        const int4 cc = cn;
+        const float4 ww = wn;
+        const int rr = rn;
+        Vec16<T> v0, v1, v2, v3;
+        if (rr == -1) {  // inside a piece: four real entries
+            v0.load(xl + (size_t)(unsigned)cc.x * PITCH);
+            v1.load(xl + (size_t)(unsigned)cc.y * PITCH);
+            v2.load(xl + (size_t)(unsigned)cc.z * PITCH);
+            v3.load(xl + (size_t)(unsigned)cc.w * PITCH);
+        } else {         // last group of a piece: pads (index -1) load nothing and add zeros
+            v0.zero();
+            v1.zero();
+            v2.zero();
+            v3.zero();
+            if (cc.x >= 0) v0.load(xl + (size_t)(unsigned)cc.x * PITCH);
+            if (cc.y >= 0) v1.load(xl + (size_t)(unsigned)cc.y * PITCH);
+            if (cc.z >= 0) v2.load(xl + (size_t)(unsigned)cc.z * PITCH);
+            if (cc.w >= 0) v3.load(xl + (size_t)(unsigned)cc.w * PITCH);
+        }
+        if (grp + 1 < ge) {
+            cn = __ldg(a.heavy.pcol + grp + 1);
+            if (HAS_VAL) wn = __ldg(a.heavy.pval + grp + 1);
+            rn = __ldg(a.heavy.grow + grp + 1);
+        }
+        if constexpr (!PLAIN) {
+            // the row operands of the epilogue (extra term, ReLU reference) are requested when this group finishes a
+            // row, before its gathers are waited for, so that the epilogue finds them in L1
+            if (rr >= 0 && gl < nchunks) {
+                if (a.init) prefetch_l1(a.init + (size_t)rr * a.ldinit + gl * VN);
+                if (a.relu_ref) prefetch_l1(a.relu_ref + (size_t)rr * a.ldref + gl * VN);
+            }
+        }
+        acc_add_vec<T, float, HAS_VAL>(acc[0], ww.x, v0);
+        acc_add_vec<T, float, HAS_VAL>(acc[0], ww.y, v1);
+        acc_add_vec<T, float, HAS_VAL>(acc[0], ww.z, v2);
+        acc_add_vec<T, float, HAS_VAL>(acc[0], ww.w, v3);
+        if (rr != -1) {
+            if (rr >= 0) {
+                if constexpr (PLAIN) {
+                    if (gl < nchunks) {
+                        const float scale = a.row_scale ? __ldg(a.row_scale + rr) : 1.f;
+                        float o[VN];
+#pragma unroll
+                        for (int t = 0; t < VN; ++t) o[t] = acc[0][t] * scale;
+                        Vec16<T> out;
+                        out.from_float(o);
+                        out.store_once(a.Y + (size_t)rr * a.ldy + gl * VN);
+                    }
+                } else {
+                    spmm_epilogue<T, G, 1, float>(a, rr, gl, nchunks, acc);
+                }
+            } else if (gl < nchunks) {
+                float *dst = a.heavy.partials + (size_t)(-rr - 2) * a.F + gl * VN;
+#pragma unroll
+                for (int t = 0; t < VN; t += 4) *reinterpret_cast<float4 *>(dst + t) = make_float4(acc[0][t], acc[0][t + 1], acc[0][t + 2], acc[0][t + 3]);
+            }
+#pragma unroll
+            for (int t = 0; t < VN; ++t) acc[0][t] = 0.f;
+        }
+    }
+}
+
+// groups owned by every row of the padded form
+LP_DEVINL int padded_row_groups(int d, int threshold)
+{
+    if (d <= threshold) return max(1, (d + 3) / 4);
+    const int rem = d % SPMM_PIECE;
+    return (d / SPMM_PIECE) * (SPMM_PIECE / 4) + (rem + 3) / 4;
+}
+__global__ void padded_count_kernel(const int *__restrict__ rowptr, int n, int threshold, int *__restrict__ ngroups)
+{
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= n) return;
+    ngroups[r] = padded_row_groups(rowptr[r + 1] - rowptr[r], threshold);
+}
+// chunk starts contributed by row r: every piece of a heavy row opens a chunk; a light row opens one when it is the
+// first row, follows a heavy row, or when first_group crosses a multiple of SPMM_CHUNK_GROUPS between rows r - 1 and r
+__global__ void padded_chunk_count_kernel(const int *__restrict__ rowptr, const int *__restrict__ first_group, int n, int threshold, int *__restrict__ count)
+{
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= n) return;
+    const int d = rowptr[r + 1] - rowptr[r];
+    if (d > threshold) {
+        count[r] = (d + SPMM_PIECE - 1) / SPMM_PIECE;
+        return;
+    }
+    const bool opens = r == 0 || rowptr[r] - rowptr[r - 1] > threshold || first_group[r] / SPMM_CHUNK_GROUPS != first_group[r - 1] / SPMM_CHUNK_GROUPS;
+    count[r] = opens ? 1 : 0;
+}
+// one thread per row writes the row's groups, their finishing codes and the chunk offsets it contributes
+__global__ void padded_fill_kernel(const int *__restrict__ rowptr, const int *__restrict__ col, const float *__restrict__ val, int n, int threshold,
+                                   const int *__restrict__ first_group, const int *__restrict__ chunk_count, const int *__restrict__ chunk_of,
+                                   const int *__restrict__ row_base, int *__restrict__ chunk_start, int *__restrict__ pcol, float *__restrict__ pval,
+                                   int *__restrict__ grow)
+{
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= n) return;
+    if (r == n - 1) chunk_start[chunk_of[n]] = first_group[n];  // chunk_of[n] = number of chunks, first_group[n] = all groups
+    const int b = rowptr[r], d = rowptr[r + 1] - b;
+    const bool heavy = d > threshold;
+    const int np = heavy ? (d + SPMM_PIECE - 1) / SPMM_PIECE : 1;
+    int g = first_group[r];
+    if (!heavy && chunk_count[r]) chunk_start[chunk_of[r]] = g;
+    for (int s = 0; s < np; ++s) {
+        const int lo = s * SPMM_PIECE;
+        const int len = heavy ? min(SPMM_PIECE, d - lo) : d;
+        const int ng = max(1, (len + 3) / 4);
+        if (heavy) chunk_start[chunk_of[r] + s] = g;
+        for (int i = 0; i < 4 * ng; ++i) {
+            pcol[4 * (size_t)g + i] = i < len ? col[b + lo + i] : -1;
+            if (pval) pval[4 * (size_t)g + i] = i < len ? val[b + lo + i] : 0.f;
+        }
+        for (int j = 0; j < ng; ++j) grow[g + j] = j < ng - 1 ? -1 : (heavy ? -(2 + row_base[r] + s) : r);
+        g += ng;
+    }
+}
+
 // one thread per row: heavy rows claim a slot and a run of items
-__global__ void spmm_heavy_plan_kernel(const int *__restrict__ rowptr, int n_rows, const int *__restrict__ n_rows_dev, HeavyPlan hp)
+// (row_base, optional: first item of every heavy row, -1 for the others)
+__global__ void spmm_heavy_plan_kernel(const int *__restrict__ rowptr, int n_rows, const int *__restrict__ n_rows_dev, HeavyPlan hp,
+                                       int *__restrict__ row_base = nullptr)
 {
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     const int lim = n_rows_dev ? min(*n_rows_dev, n_rows) : n_rows;
     if (r >= lim) return;
     const int d = rowptr[r + 1] - rowptr[r];
-    if (d <= hp.threshold) return;
-    const int nseg = (d + SPMM_SEG - 1) / SPMM_SEG;
+    if (d <= hp.threshold) {
+        if (row_base) row_base[r] = -1;
+        return;
+    }
+    const int nseg = (d + hp.seg - 1) / hp.seg;
     const int i = atomicAdd(&hp.counts[0], 1);
     const int b = atomicAdd(&hp.counts[1], nseg);
     hp.rows[i] = r;
     hp.base[i] = b;
+    if (row_base) row_base[r] = b;
     for (int s = 0; s < nseg; ++s) {
         hp.item_row[b + s] = r;
         hp.item_first[b + s] = b;
@@ -387,13 +563,32 @@ __global__ void __launch_bounds__(SPMM_THREADS) spmm_heavy_combine_kernel(const 
     const int nchunks = a.F / VN;
     for (int i = blockIdx.x * NG + g; i < count; i += gridDim.x * NG) {
         const int r = a.heavy.rows[i], b = a.heavy.base[i];
-        const int nseg = (a.rowptr[r + 1] - a.rowptr[r] + SPMM_SEG - 1) / SPMM_SEG;
+        const int nseg = (a.rowptr[r + 1] - a.rowptr[r] + a.heavy.seg - 1) / a.heavy.seg;
         ACC acc[NV][VN];
 #pragma unroll
         for (int q = 0; q < NV; ++q)
 #pragma unroll
             for (int t = 0; t < VN; ++t) acc[q][t] = ACC(0);
-        for (int s = 0; s < nseg; ++s) {
+        // four partial rows are fetched before any is added (the additions stay in item order)
+        int s = 0;
+        if constexpr (NV == 1) {
+            if (gl < nchunks) {
+                for (; s + 4 <= nseg; s += 4) {
+                    ACC tmp[4][VN];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const ACC *p = reinterpret_cast<const ACC *>(a.heavy.partials) + (size_t)(b + s + u) * a.F + gl * VN;
+#pragma unroll
+                        for (int t = 0; t < VN; ++t) tmp[u][t] = p[t];
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+#pragma unroll
+                        for (int t = 0; t < VN; ++t) acc[0][t] += tmp[u][t];
+                }
+            }
+        }
+        for (; s < nseg; ++s) {
             const ACC *p = reinterpret_cast<const ACC *>(a.heavy.partials) + (size_t)(b + s) * a.F;
 #pragma unroll
             for (int q = 0; q < NV; ++q) {
@@ -414,6 +609,35 @@ template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC> sta
     constexpr int NG = SPMM_THREADS / G;
     const int light_blocks = (int)ceil_div64(a.n_rows, ROWS);
     if (light_blocks == 0) return;
+    // static structure with a padded plan and source rows G or 2 G vectors apart: the padded kernel walks every row
+    if constexpr (NV == 1 && sizeof(ACC) == 4) {
+        const int pitch = a.ldx / Vec16<T>::N;
+        if (a.heavy.pcol != nullptr && a.heavy.n_chunks > 0 && !a.X2 && !a.self_out && !a.n_rows_dev && !a.init_idx && a.ldx % Vec16<T>::N == 0 &&
+            (pitch == G || pitch == 2 * G) && (a.val == nullptr || (a.val == a.heavy.pval_src && a.heavy.pval != nullptr))) {
+            SpmmArgs<T> b = a;
+            b.heavy.rows = a.heavy.p_rows;
+            b.heavy.base = a.heavy.p_base;
+            b.heavy.counts = a.heavy.p_counts;
+            b.heavy.seg = SPMM_PIECE;
+            const unsigned pgrid = (unsigned)ceil_div64(a.heavy.n_chunks, NG);
+            const bool plain = !a.init && !a.relu_ref;
+#define LP_PADDED(MULT_, VAL_) do { \
+                if (plain) spmm_padded_kernel<T, G, MULT_, 6, VAL_, true><<<pgrid, SPMM_THREADS, 0, ex.st>>>(b); \
+                else spmm_padded_kernel<T, G, MULT_, 5, VAL_, false><<<pgrid, SPMM_THREADS, 0, ex.st>>>(b); } while (0)
+            if (pitch == G) {
+                if (a.val) LP_PADDED(1, true); else LP_PADDED(1, false);
+            } else {
+                if (a.val) LP_PADDED(2, true); else LP_PADDED(2, false);
+            }
+#undef LP_PADDED
+            ex.launches += 1;
+            if (a.heavy.p_host_rows > 0) {
+                spmm_heavy_combine_kernel<T, G, NV, ACC><<<(unsigned)std::min<int64_t>(592, ceil_div64(a.heavy.p_host_rows, NG)), SPMM_THREADS, 0, ex.st>>>(b);
+                ex.launches += 1;
+            }
+            return;
+        }
+    }
     int64_t items = a.heavy.host_items;
     if (items < 0) {  // plan unknown on the host: rebuild it on the device, size the grid by the upper bound
         cudaMemsetAsync(a.heavy.counts, 0, 2 * sizeof(int), ex.st);
