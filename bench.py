@@ -33,10 +33,10 @@ K_NEG = 1
 SEED = 1234
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the aggregation launches of one step on the
-# benchmark workload, from one ncu capture (profiles/spmm_csr_bf16_config2.md): layer-1 forward 121.5 MB,
-# layer-2 forward 397.9 MB, adjoint 608.0 MB -> mean per timed launch.  Valid only for the kernel source it
+# benchmark workload, from one ncu capture (profiles/spmm_padded_bf16_config2.md): layer-1 forward 129.9 MB,
+# layer-2 forward 426.4 MB, adjoint 627.4 MB -> mean per timed launch.  Valid only for the kernel source it
 # was taken with (sha1 of csrc/spmm.cuh + csrc/common.cuh); reported as null otherwise.
-NCU_TRAFFIC = {"spmm_sha1": "db609f90a1a3efc7130110a97cd8e51e06baad64", "bytes_per_launch": (121.5e6 + 397.9e6 + 608.0e6) / 3.0}
+NCU_TRAFFIC = {"spmm_sha1": "a536f7e229120cc78ae42345289239879bd08c9f", "bytes_per_launch": (129.9e6 + 426.4e6 + 627.4e6) / 3.0}
 
 
 def measured_peaks():
@@ -288,7 +288,7 @@ def main():
     gather_minus_min = sum((g.nnz - g.n) * f * 2 for f in widths) / max(len(widths), 1)
     avg_launch_s = 1e-3 * agg_ms / max(agg_spans, 1)
     min_bytes = agg_bytes / max(agg_spans, 1) - gather_minus_min
-    roofline = {"bound": "hbm", "kernel": "spmm_csr_kernel (aggregation forward + adjoint)", "achieved": achieved, "peak": hbm_peak,
+    roofline = {"bound": "hbm", "kernel": "spmm_padded_kernel (aggregation forward + adjoint)", "achieved": achieved, "peak": hbm_peak,
                 "unit": "GB/s", "frac": (achieved / hbm_peak) if achieved else None, "peak_source": f"of {peak_kind}",
                 "frac_of_nominal_8000": (achieved / 8000.0) if achieved else None, "traffic": traffic,
                 "dram_frac": (traffic / avg_launch_s / 1e9 / hbm_peak) if traffic and avg_launch_s > 0 else None,

@@ -417,7 +417,7 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
     // padded form of both structures (for spmm_padded_kernel), with the GCN coefficients padded alongside
     static_assert(SPMM_PIECE % 4 == 0, "pieces are whole groups");
     for (HeavyPlan *hp : {&ctx->plan_csr, &ctx->plan_csc}) {
-        if (e != cudaSuccess || n <= 0 || static_threshold != SPMM_PIECE) break;
+        if (e != cudaSuccess || n <= 0) break;
         const bool csr = hp == &ctx->plan_csr;
         const int *sp = csr ? ctx->rowptr : ctx->colptr, *sc = csr ? ctx->col : ctx->rowidx;
         const float *sv = csr ? ctx->gcn_val : ctx->gcn_valT;
@@ -428,7 +428,7 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
         GALLOC(pp.counts, 64);
         TALLOC(pp.item_row, item_cap);
         TALLOC(pp.item_first, item_cap);
-        pp.threshold = static_threshold;
+        pp.threshold = SPMM_PIECE;
         pp.seg = SPMM_PIECE;
         int *row_base = nullptr, *first_group = nullptr, *chunk_count = nullptr, *chunk_of = nullptr;
         TALLOC(row_base, n + 1);
@@ -437,9 +437,9 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
         TALLOC(chunk_of, n + 1);
         cudaMemsetAsync(pp.counts, 0, 2 * sizeof(int), st);
         spmm_heavy_plan_kernel<<<nblk(n), 256, 0, st>>>(sp, (int)n, nullptr, pp, row_base);
-        padded_count_kernel<<<nblk(n), 256, 0, st>>>(sp, (int)n, static_threshold, first_group);
+        padded_count_kernel<<<nblk(n), 256, 0, st>>>(sp, (int)n, SPMM_PIECE, first_group);
         exclusive_scan_i32(ctx->ex, first_group, n, first_group, first_group + n, ts.scan_tmp);
-        padded_chunk_count_kernel<<<nblk(n), 256, 0, st>>>(sp, first_group, (int)n, static_threshold, chunk_count);
+        padded_chunk_count_kernel<<<nblk(n), 256, 0, st>>>(sp, first_group, (int)n, SPMM_PIECE, chunk_count);
         exclusive_scan_i32(ctx->ex, chunk_count, n, chunk_of, chunk_of + n, ts.scan_tmp);
         cudaMemcpyAsync(ctx->host_counts + 8, first_group + n, sizeof(int), cudaMemcpyDeviceToHost, st);
         cudaMemcpyAsync(ctx->host_counts + 9, chunk_of + n, sizeof(int), cudaMemcpyDeviceToHost, st);
@@ -455,7 +455,7 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
         GALLOC(pval, 4 * n_groups + 4);
         GALLOC(grow, n_groups + 1);
         GALLOC(chunk_start, (int64_t)n_chunks + 2);
-        padded_fill_kernel<<<nblk(n), 256, 0, st>>>(sp, sc, sv, (int)n, static_threshold, first_group, chunk_count, chunk_of, row_base, chunk_start, pcol, pval, grow);
+        padded_fill_kernel<<<nblk(n), 256, 0, st>>>(sp, sc, sv, (int)n, SPMM_PIECE, first_group, chunk_count, chunk_of, row_base, chunk_start, pcol, pval, grow);
         ctx->ex.launches += 5;
         e = cudaStreamSynchronize(st);
         if (e != cudaSuccess) break;

@@ -2,7 +2,10 @@
 //
 //   Y[r, :] = mask_r( init_coef[r] * Init[init_idx[r], :]  +  row_scale[r] * sum_e val[e] * X[col[e], :] )
 //
-// One group of G lanes (8, 16 or 32) owns a row; every lane gathers 16-byte vectors of the
+// Two kernels.  spmm_padded_kernel serves the static structures (the loaded graph and its transpose), for which a
+// padded copy of the rows is built once at load: it is described above its definition.  spmm_csr_kernel serves
+// every structure as it is stored (per-step structures, wide rows, exact sums):
+// one group of G lanes (8, 16 or 32) owns a row; every lane gathers 16-byte vectors of the
 // source rows (4 floats or 8 bf16) and accumulates in FP32 in entry order.  Rows with more than
 // a per-structure threshold of entries (power-law hubs) are cut into items of SPMM_SEG entries; the items run as extra
 // blocks of the same grid (so hubs spread over the whole GPU and overlap the light rows), each
@@ -132,7 +135,7 @@ constexpr int SPMM_HEAVY_MIN = 64;  // smallest heavy-row threshold a plan may u
                                     // group is a long dependent chain: long rows are cut into items instead.
 constexpr int SPMM_ITEM_BLOCKS = 1184;  // blocks that walk the item list (grid-stride)
 constexpr int SPMM_SEG = 512;    // entries per item (one block: 8 lane groups x 64 entries for 32-lane groups)
-constexpr int SPMM_PIECE = 128;  // entries per piece of the padded form (= the heavy-row threshold of static structures)
+constexpr int SPMM_PIECE = 128;  // entries per piece of the padded form; rows with more entries are cut and combined (256: slower by 2 %)
 constexpr int SPMM_CHUNK_GROUPS = 16;  // groups of four entries per chunk of the padded form (one lane group walks a chunk)
 
 // acc += sum over entries [e_lo, e_hi) of val[e] * X[col[e], :] for the chunks owned by this lane.
