@@ -417,7 +417,7 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
     // padded form of both structures (for spmm_padded_kernel), with the GCN coefficients padded alongside
     static_assert(SPMM_PIECE % 4 == 0, "pieces are whole groups");
     for (HeavyPlan *hp : {&ctx->plan_csr, &ctx->plan_csc}) {
-        if (e != cudaSuccess || n <= 0) break;
+        if (e != cudaSuccess || n <= 0 || n >= (1 << 27) || item_cap >= (1 << 27)) break;  // row and slot numbers share 27 bits of the finishing codes
         const bool csr = hp == &ctx->plan_csr;
         const int *sp = csr ? ctx->rowptr : ctx->colptr, *sc = csr ? ctx->col : ctx->rowidx;
         const float *sv = csr ? ctx->gcn_val : ctx->gcn_valT;

@@ -36,11 +36,12 @@ struct HeavyPlan {
     int threshold = 64;                   // rows with more entries than this are heavy (>= SPMM_HEAVY_MIN)
     int seg = 512;                        // entries per item (SPMM_SEG; SPMM_PIECE for the padded form's own plan)
     // Static structures only: every row again in padded form for spmm_padded_kernel.  A row is cut into pieces of at
-    // most SPMM_PIECE entries (one piece unless it is heavy), a piece into groups of four entries (pad index -1, pad
-    // coefficient 0; an empty row keeps one all-pad group so that its output is written).  pcol / pval hold the groups
-    // back to back; grow[g] is -1 inside a piece, the row r >= 0 when group g finishes the only piece of row r, and
-    // -(2 + slot) when it finishes a piece of a heavy row whose FP32 partial sum goes to slot `slot` of `partials`
-    // (p_rows / p_base / p_counts list the heavy rows and their first slots for the combine kernel).  chunk_start
+    // most SPMM_PIECE entries (one piece unless it is heavy), a piece into groups of four entries (a pad repeats the
+    // group's first index, or names row 0 in the all-pad group that an empty row keeps so that its output is written;
+    // pad coefficient 0).  pcol / pval hold the groups back to back; grow[g] is -1 inside a piece and
+    // (id << 4 | kind << 3 | cnt) for the group that finishes a piece: cnt = real entries of that group (0..4), kind 0:
+    // the piece is all of row id, kind 1: the piece belongs to a heavy row and its FP32 partial sum goes to slot id of
+    // `partials` (p_rows / p_base / p_counts list the heavy rows and their first slots for the combine kernel).  chunk_start
     // cuts the groups into chunks that begin at piece starts (n_chunks + 1 offsets).
     const int4 *pcol = nullptr;
     const float4 *pval = nullptr;
@@ -387,7 +388,8 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
 // in the same order as by the row-per-group kernel and gives the same bits.  Nothing in the inner loop depends on a
 // row's length: no tails, no per-entry end tests, the next group's indices are fetched while this group's rows are
 // in flight, a short row costs one group instead of a round trip of its own, and hub rows are pieces like any other.
-// Only the last group of a piece can hold pads; there the loads are predicated and the pads add zeros.
+// Only the last group of a piece can hold pads: they repeat an index of the group (a load that hits L1) and are left
+// out of the sum by a count the finishing code carries (unit coefficients) or by their zero coefficient.
 // ---------------------------------------------------------------------------------------------
 // PLAIN: the epilogue is the row scale alone (mean aggregation forward); it is written out here so that the loop
 // keeps the register budget of a bare gather.
@@ -417,55 +419,55 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_padded_kernel(const S
         const float4 ww = wn;
         const int rr = rn;
         Vec16<T> v0, v1, v2, v3;
-        if (rr == -1) {  // inside a piece: four real entries
-            v0.load(xl + (size_t)(unsigned)cc.x * PITCH);
-            v1.load(xl + (size_t)(unsigned)cc.y * PITCH);
-            v2.load(xl + (size_t)(unsigned)cc.z * PITCH);
-            v3.load(xl + (size_t)(unsigned)cc.w * PITCH);
-        } else {         // last group of a piece: pads (index -1) load nothing and add zeros
-            v0.zero();
-            v1.zero();
-            v2.zero();
-            v3.zero();
-            if (cc.x >= 0) v0.load(xl + (size_t)(unsigned)cc.x * PITCH);
-            if (cc.y >= 0) v1.load(xl + (size_t)(unsigned)cc.y * PITCH);
-            if (cc.z >= 0) v2.load(xl + (size_t)(unsigned)cc.z * PITCH);
-            if (cc.w >= 0) v3.load(xl + (size_t)(unsigned)cc.w * PITCH);
-        }
+        v0.load(xl + (size_t)(unsigned)cc.x * PITCH);
+        v1.load(xl + (size_t)(unsigned)cc.y * PITCH);
+        v2.load(xl + (size_t)(unsigned)cc.z * PITCH);
+        v3.load(xl + (size_t)(unsigned)cc.w * PITCH);
         if (grp + 1 < ge) {
             cn = __ldg(a.heavy.pcol + grp + 1);
             if (HAS_VAL) wn = __ldg(a.heavy.pval + grp + 1);
             rn = __ldg(a.heavy.grow + grp + 1);
         }
+        const int id = rr >> 4;  // row or partial slot finished by this group (when rr != -1)
         if constexpr (!PLAIN) {
             // the row operands of the epilogue (extra term, ReLU reference) are requested when this group finishes a
             // row, before its gathers are waited for, so that the epilogue finds them in L1
-            if (rr >= 0 && gl < nchunks) {
-                if (a.init) prefetch_l1(a.init + (size_t)rr * a.ldinit + gl * VN);
-                if (a.relu_ref) prefetch_l1(a.relu_ref + (size_t)rr * a.ldref + gl * VN);
+            if (rr != -1 && (rr & 8) == 0 && gl < nchunks) {
+                if (a.init) prefetch_l1(a.init + (size_t)id * a.ldinit + gl * VN);
+                if (a.relu_ref) prefetch_l1(a.relu_ref + (size_t)id * a.ldref + gl * VN);
             }
         }
-        acc_add_vec<T, float, HAS_VAL>(acc[0], ww.x, v0);
-        acc_add_vec<T, float, HAS_VAL>(acc[0], ww.y, v1);
-        acc_add_vec<T, float, HAS_VAL>(acc[0], ww.z, v2);
-        acc_add_vec<T, float, HAS_VAL>(acc[0], ww.w, v3);
+        if (rr == -1 || (HAS_VAL && (rr & 7) != 0)) {  // inside a piece all four entries are real; with coefficients a pad
+                                                        // repeats a real entry of its group under a zero coefficient
+            acc_add_vec<T, float, HAS_VAL>(acc[0], ww.x, v0);
+            acc_add_vec<T, float, HAS_VAL>(acc[0], ww.y, v1);
+            acc_add_vec<T, float, HAS_VAL>(acc[0], ww.z, v2);
+            acc_add_vec<T, float, HAS_VAL>(acc[0], ww.w, v3);
+        } else if (!HAS_VAL) {  // (with coefficients what is left is the all-pad group of an empty row: nothing to add)
+            const int cnt = rr & 7;
+            if (cnt > 0) acc_add_vec<T, float, HAS_VAL>(acc[0], ww.x, v0);
+            if (cnt > 1) acc_add_vec<T, float, HAS_VAL>(acc[0], ww.y, v1);
+            if (cnt > 2) acc_add_vec<T, float, HAS_VAL>(acc[0], ww.z, v2);
+            if (cnt > 3) acc_add_vec<T, float, HAS_VAL>(acc[0], ww.w, v3);
+        }
         if (rr != -1) {
-            if (rr >= 0) {
+            if ((rr & 8) == 0) {
+                const int row = id;
                 if constexpr (PLAIN) {
                     if (gl < nchunks) {
-                        const float scale = a.row_scale ? __ldg(a.row_scale + rr) : 1.f;
+                        const float scale = a.row_scale ? __ldg(a.row_scale + row) : 1.f;
                         float o[VN];
 #pragma unroll
                         for (int t = 0; t < VN; ++t) o[t] = acc[0][t] * scale;
                         Vec16<T> out;
                         out.from_float(o);
-                        out.store_once(a.Y + (size_t)rr * a.ldy + gl * VN);
+                        out.store_once(a.Y + (size_t)row * a.ldy + gl * VN);
                     }
                 } else {
-                    spmm_epilogue<T, G, 1, float>(a, rr, gl, nchunks, acc);
+                    spmm_epilogue<T, G, 1, float>(a, row, gl, nchunks, acc);
                 }
             } else if (gl < nchunks) {
-                float *dst = a.heavy.partials + (size_t)(-rr - 2) * a.F + gl * VN;
+                float *dst = a.heavy.partials + (size_t)id * a.F + gl * VN;
 #pragma unroll
                 for (int t = 0; t < VN; t += 4) *reinterpret_cast<float4 *>(dst + t) = make_float4(acc[0][t], acc[0][t + 1], acc[0][t + 2], acc[0][t + 3]);
             }
@@ -522,10 +524,13 @@ __global__ void padded_fill_kernel(const int *__restrict__ rowptr, const int *__
         const int ng = max(1, (len + 3) / 4);
         if (heavy) chunk_start[chunk_of[r] + s] = g;
         for (int i = 0; i < 4 * ng; ++i) {
-            pcol[4 * (size_t)g + i] = i < len ? col[b + lo + i] : -1;
+            const int first = (i / 4) * 4;  // a pad repeats the first index of its group (row 0 in an all-pad group)
+            pcol[4 * (size_t)g + i] = i < len ? col[b + lo + i] : (first < len ? col[b + lo + first] : 0);
             if (pval) pval[4 * (size_t)g + i] = i < len ? val[b + lo + i] : 0.f;
         }
-        for (int j = 0; j < ng; ++j) grow[g + j] = j < ng - 1 ? -1 : (heavy ? -(2 + row_base[r] + s) : r);
+        const int cnt = len - 4 * (ng - 1);  // real entries of the last group: 1..4, 0 for an empty row
+        const int code = heavy ? ((row_base[r] + s) << 4 | 8 | cnt) : (r << 4 | cnt);
+        for (int j = 0; j < ng; ++j) grow[g + j] = j < ng - 1 ? -1 : code;
         g += ng;
     }
 }
