@@ -119,6 +119,49 @@ def test_aggregate_bf16(pkg, F):
     ctx.close()
 
 
+@pytest.mark.parametrize("F", [32, 128])
+def test_aggregate_piece_and_group_boundaries(pkg, F):
+    # the static structures are walked in padded form: rows cut into pieces of 128 entries and groups of four.  This
+    # directed graph has a row of every length around those boundaries (0..9, 127..130, 255..258, 511..514, 1000), in
+    # scattered positions with empty rows between them and at both ends; mean and its adjoint against the oracle, FP32
+    # (one piece per row, pieces combined, pads in the last group, the all-pad group of an empty row)
+    lengths = list(range(0, 10)) + [127, 128, 129, 130, 255, 256, 257, 258, 511, 512, 513, 514, 1000]
+    n = 1200
+    rng = np.random.default_rng(F)
+    rows = rng.permutation(np.arange(3, n - 3))[: len(lengths)]
+    dst, src = [], []
+    for r, d in zip(rows, lengths):
+        cand = np.delete(np.arange(n), r)
+        dst.append(np.full(d, r))
+        src.append(rng.choice(cand, size=d, replace=False))
+    g = wl.csr_from_edges(n, np.concatenate(dst), np.concatenate(src))
+    assert np.array_equal(np.sort(np.diff(g.rowptr)[rows]), np.sort(lengths)) and g.rowptr[3] == 0
+    ctx = make_ctx(pkg, g, wl.node_features(n, 8, 0))
+    H = rng.standard_normal((n, F)).astype(np.float32)
+    for transpose in (False, True):
+        out = ctx.op_aggregate("sage", t32(H), transpose=transpose).cpu().numpy()
+        ref = (oracle.aggregate_backward if transpose else oracle.aggregate)("mean", n, g.rowptr, g.col, None, H)
+        assert rel_l2(out, ref) < 1e-6
+        assert np.max(np.abs(out - ref)) < 1e-5 * max(1.0, np.abs(ref).max())
+        if not transpose:
+            assert not out[np.diff(g.rowptr) == 0].any()  # empty rows are written, as zeros
+    Hb = t32(H).to(torch.bfloat16)
+    outb = ctx.op_aggregate("sage", Hb).float().cpu().numpy()
+    refb = oracle.aggregate("mean", n, g.rowptr, g.col, None, Hb.float().cpu().numpy())
+    assert rel_l2(outb, refb) < 4e-3
+    ctx.close()
+    # the same lengths as COLUMNS (the graph with every entry reversed), with per-entry coefficients: the GCN operator and
+    # its adjoint, so that the padded transposed structure meets the boundaries too
+    gt = wl.csr_from_edges(n, np.concatenate(src), np.concatenate(dst))
+    ctx = make_ctx(pkg, gt, wl.node_features(n, 8, 0))
+    for transpose in (False, True):
+        out = ctx.op_aggregate("gcn", t32(H), transpose=transpose).cpu().numpy()
+        ref = (oracle.aggregate_backward if transpose else oracle.aggregate)("gcn", n, gt.rowptr, gt.col, None, H)
+        assert rel_l2(out, ref) < 1e-6
+        assert np.max(np.abs(out - ref)) < 1e-5 * max(1.0, np.abs(ref).max())
+    ctx.close()
+
+
 @pytest.mark.parametrize("words", [32, 64, 128])
 def test_gather_ceiling_folds_are_exact(pkg, words):
     # the measurement kernel behind the roofline figures does the gathers it claims: XOR folds of runs of 64 entries,
