@@ -166,6 +166,86 @@ edge_score_bce_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const 
     }
 }
 
+// The common case (one negative per positive that shares the positive's source, rows of at most 32 vectors): a warp
+// takes two positives and requests their six rows together before it reduces any, which halves the number of
+// dependent memory round trips per scored edge.  Scores, gradients and incidence counts are those of
+// edge_score_bce_kernel bit for bit (same order of multiply-adds and the same reduction tree); a block's loss
+// partial covers 16 positives instead of 8.
+template <typename T>
+__global__ void __launch_bounds__(EDGE_THREADS)
+edge_score_bce_pair_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const int *__restrict__ idmap, const int *__restrict__ pos_src,
+                           const int *__restrict__ pos_dst, int64_t B, const int *__restrict__ neg_dst, float inv_N, float *__restrict__ g_pos,
+                           float *__restrict__ g_neg, float *__restrict__ loss_partials, int *__restrict__ inc_counts)
+{
+    constexpr int VN = Vec16<T>::N;
+    constexpr int P = 2;
+    __shared__ float s_loss[EDGE_THREADS / 32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t j0 = ((int64_t)blockIdx.x * (EDGE_THREADS / 32) + warp) * P;
+    const int nchunks = D / VN;
+    const bool active = lane < nchunks;
+    const int ch = min(lane, nchunks - 1);
+    float loss = 0.f;
+    if (j0 < B) {
+        int u[P], v[P], vn[P];
+        Vec16<T> ru[P], rv[P], rn[P];
+#pragma unroll
+        for (int p = 0; p < P; ++p) {
+            const int64_t j = min(j0 + p, B - 1);  // a missing second positive repeats the first one's loads and writes nothing
+            u[p] = clamp_id(pos_src[j], n_ids);
+            v[p] = clamp_id(pos_dst[j], n_ids);
+            vn[p] = clamp_id(neg_dst[j], n_ids);
+            if (idmap) { u[p] = idmap[u[p]]; v[p] = idmap[v[p]]; vn[p] = idmap[vn[p]]; }
+        }
+#pragma unroll
+        for (int p = 0; p < P; ++p) {
+            ru[p].load(H + (size_t)u[p] * ldh + ch * VN);
+            rv[p].load(H + (size_t)v[p] * ldh + ch * VN);
+            rn[p].load(H + (size_t)vn[p] * ldh + ch * VN);
+        }
+#pragma unroll
+        for (int p = 0; p < P; ++p) {
+            float fu[VN], fv[VN], fn[VN];
+            ru[p].to_float(fu);
+            rv[p].to_float(fv);
+            rn[p].to_float(fn);
+            float dp = 0.f, dn = 0.f;
+            if (active) {
+#pragma unroll
+                for (int t = 0; t < VN; ++t) dp = fmaf(fu[t], fv[t], dp);
+#pragma unroll
+                for (int t = 0; t < VN; ++t) dn = fmaf(fu[t], fn[t], dn);
+            }
+            dp = warp_sum(dp);
+            dn = warp_sum(dn);
+            float ell_p, dls_p, ell_n, dls_n;
+            bce_logits(dp, 1.f, ell_p, dls_p);
+            bce_logits(dn, 0.f, ell_n, dls_n);
+            if (j0 + p < B) {
+                loss += ell_p;
+                loss += ell_n;
+                if (lane == 0) {
+                    g_pos[j0 + p] = dls_p * inv_N;
+                    g_neg[j0 + p] = dls_n * inv_N;
+                    if (inc_counts) {
+                        atomicAdd(&inc_counts[u[p]], 2);  // source of the positive and of its negative
+                        atomicAdd(&inc_counts[v[p]], 1);
+                        atomicAdd(&inc_counts[vn[p]], 1);
+                    }
+                }
+            }
+        }
+    }
+    if (lane == 0) s_loss[warp] = loss;
+    __syncthreads();
+    if (threadIdx.x == 0 && loss_partials) {
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < EDGE_THREADS / 32; ++w) s += s_loss[w];
+        loss_partials[blockIdx.x] = s;
+    }
+}
+
 // loss = inv_N * sum of partials: one block of 1024 threads, thread t adds partials t, t + 1024, ... in double
 // (tens of thousands of nearly equal terms), then a fixed binary tree over the threads
 __global__ void __launch_bounds__(1024) loss_reduce_kernel(const float *__restrict__ partials, int64_t m, float inv_N, float *__restrict__ loss)

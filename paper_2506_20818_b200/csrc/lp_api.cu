@@ -1292,10 +1292,14 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         s = predictor_backward<T>(ctx, params, E, ctx->g_pos, grads, accumulate);
         if (s != LP_OK) { delete pscore; return s; }
     } else {
-        if (chunks <= 32) edge_score_bce_kernel<T, 1><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials, ctx->inc_ptr);
+        unsigned lparts = eblocks;  // loss partials written
+        if (chunks <= 32 && k == 1 && !neg_src) {
+            lparts = nblk(B, 2 * (EDGE_THREADS / 32));
+            edge_score_bce_pair_kernel<T><<<lparts, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_dst, inv_N, ctx->g_pos, ctx->g_neg, ctx->loss_partials, ctx->inc_ptr);
+        } else if (chunks <= 32) edge_score_bce_kernel<T, 1><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials, ctx->inc_ptr);
         else if (chunks <= 64) edge_score_bce_kernel<T, 2><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials, ctx->inc_ptr);
         else edge_score_bce_kernel<T, 4><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials, ctx->inc_ptr);
-        loss_reduce_kernel<<<1, 1024, 0, st>>>(ctx->loss_partials, eblocks, inv_N, loss);
+        loss_reduce_kernel<<<1, 1024, 0, st>>>(ctx->loss_partials, lparts, inv_N, loss);
     }
     delete pscore;
     ctx->ex.launches += 2;
