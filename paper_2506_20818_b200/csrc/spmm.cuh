@@ -391,11 +391,12 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
 // Only the last group of a piece can hold pads: they repeat an index of the group (a load that hits L1) and are left
 // out of the sum by a count the finishing code carries (unit coefficients) or by their zero coefficient.
 // ---------------------------------------------------------------------------------------------
-// PLAIN: the epilogue is the row scale alone (mean aggregation forward); it is written out here so that the loop
-// keeps the register budget of a bare gather.
+// EPI 1: the epilogue is the row scale alone (mean aggregation forward); EPI 2: extra term with unit coefficient and
+// ReLU mask and nothing else (adjoint of the mean aggregation).  Both are written out compactly so that the loop keeps
+// the register budget of a bare gather; EPI 0 is the general epilogue.
 LP_DEVINL void prefetch_l1(const void *p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
 
-template <typename T, int G, int MULT, int MINB, bool HAS_VAL, bool PLAIN>
+template <typename T, int G, int MULT, int MINB, bool HAS_VAL, int EPI>
 __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_padded_kernel(const SpmmArgs<T> a)
 {
     constexpr int VN = Vec16<T>::N;
@@ -429,7 +430,7 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_padded_kernel(const S
             rn = __ldg(a.heavy.grow + grp + 1);
         }
         const int id = rr >> 4;  // row or partial slot finished by this group (when rr != -1)
-        if constexpr (!PLAIN) {
+        if constexpr (EPI != 1) {
             // the row operands of the epilogue (extra term, ReLU reference) are requested when this group finishes a
             // row, before its gathers are waited for, so that the epilogue finds them in L1
             if (rr != -1 && (rr & 8) == 0 && gl < nchunks) {
@@ -453,7 +454,7 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_padded_kernel(const S
         if (rr != -1) {
             if ((rr & 8) == 0) {
                 const int row = id;
-                if constexpr (PLAIN) {
+                if constexpr (EPI == 1) {
                     if (gl < nchunks) {
                         const float scale = a.row_scale ? __ldg(a.row_scale + row) : 1.f;
                         float o[VN];
@@ -461,6 +462,20 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_padded_kernel(const S
                         for (int t = 0; t < VN; ++t) o[t] = acc[0][t] * scale;
                         Vec16<T> out;
                         out.from_float(o);
+                        out.store_once(a.Y + (size_t)row * a.ldy + gl * VN);
+                    }
+                } else if constexpr (EPI == 2) {
+                    if (gl < nchunks) {  // y = relu_ref > 0 ? sum + init : 0 (the general epilogue's arithmetic with scale and coefficient 1)
+                        Vec16<T> vi, vr;
+                        vi.load_once(a.init + (size_t)row * a.ldinit + gl * VN);
+                        vr.load_once(a.relu_ref + (size_t)row * a.ldref + gl * VN);
+                        float fi[VN], fr[VN];
+                        vi.to_float(fi);
+                        vr.to_float(fr);
+#pragma unroll
+                        for (int t = 0; t < VN; ++t) fi[t] = fr[t] > 0.f ? fmaf(1.f, fi[t], acc[0][t] * 1.f) : 0.f;
+                        Vec16<T> out;
+                        out.from_float(fi);
                         out.store_once(a.Y + (size_t)row * a.ldy + gl * VN);
                     }
                 } else {
@@ -629,9 +644,11 @@ template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC> sta
             b.heavy.seg = SPMM_PIECE;
             const unsigned pgrid = (unsigned)ceil_div64(a.heavy.n_chunks, NG);
             const bool plain = !a.init && !a.relu_ref;
+            const bool self_mask = a.init && a.relu_ref && !a.init_coef && !a.row_scale && !a.val;
 #define LP_PADDED(MULT_, VAL_) do { \
-                if (plain) spmm_padded_kernel<T, G, MULT_, 6, VAL_, true><<<pgrid, SPMM_THREADS, 0, ex.st>>>(b); \
-                else spmm_padded_kernel<T, G, MULT_, 5, VAL_, false><<<pgrid, SPMM_THREADS, 0, ex.st>>>(b); } while (0)
+                if (plain) spmm_padded_kernel<T, G, MULT_, 6, VAL_, 1><<<pgrid, SPMM_THREADS, 0, ex.st>>>(b); \
+                else if (self_mask) spmm_padded_kernel<T, G, MULT_, 5, false, 2><<<pgrid, SPMM_THREADS, 0, ex.st>>>(b); \
+                else spmm_padded_kernel<T, G, MULT_, 5, VAL_, 0><<<pgrid, SPMM_THREADS, 0, ex.st>>>(b); } while (0)
             if (pitch == G) {
                 if (a.val) LP_PADDED(1, true); else LP_PADDED(1, false);
             } else {
