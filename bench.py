@@ -33,10 +33,10 @@ K_NEG = 1
 SEED = 1234
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the aggregation launches of one step on the
-# benchmark workload, from one ncu capture (profiles/spmm_padded_bf16_config2.md): layer-1 forward 127.1 MB,
-# layer-2 forward 408.1 MB, adjoint 635.6 MB -> mean per timed launch.  Valid only for the kernel source it
+# benchmark workload, from one ncu capture (profiles/spmm_padded_bf16_config2.md): layer-1 forward 123.7 MB,
+# layer-2 forward 408.8 MB, adjoint 628.4 MB -> mean per timed launch.  Valid only for the kernel source it
 # was taken with (sha1 of csrc/spmm.cuh + csrc/common.cuh); reported as null otherwise.
-NCU_TRAFFIC = {"spmm_sha1": "68d3db2af47b09a6afc33225e1a3242c3d79c894", "bytes_per_launch": (127.1e6 + 408.1e6 + 635.6e6) / 3.0}
+NCU_TRAFFIC = {"spmm_sha1": "897672ea779116af0d86a2a91421625fa1b531bd", "bytes_per_launch": (123.7e6 + 408.8e6 + 628.4e6) / 3.0}
 
 
 def measured_peaks():
