@@ -111,7 +111,10 @@ const char *lp_last_error(const lp_ctx *ctx);
  * The arrays are copied (the caller may free them afterwards).  The call validates the CSR
  * (LP_EINVAL on any violation), builds the transposed structure used by the backward pass
  * (entries of a transposed row ordered by original row), the degree normalisations
- * (GCN: d~_v = 1 + sum_u w_vu; SAGE: 1/|N(v)|) and a BF16 copy of X.  Synchronises. */
+ * (GCN: d~_v = 1 + sum_u w_vu; SAGE: 1/|N(v)|), a BF16 copy of X, and a padded copy of the graph and
+ * of its transpose for the aggregation kernel (rows in groups of four entries: about 8.6 bytes per
+ * stored entry and structure, a little more where rows are short; lp_get_stats reports the total).
+ * Synchronises. */
 lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const int64_t *rowptr, const int32_t *col,
                         const float *w, const float *X, int32_t f, int32_t ptrs_on_device);
 
