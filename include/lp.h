@@ -213,6 +213,10 @@ lp_status lp_sample_negatives(lp_ctx *ctx, uint64_t seed, uint64_t step, int32_t
  *   loss              : device float32 scalar, L = (1/N) sum_e ell(s_e, y_e), N = B(1+k)
  *   grads[n_params]   : device float32, dL/dW; overwritten, or added to when accumulate != 0
  *                       (gradient accumulation over emulated workers)
+ * The gradient with respect to the embeddings is summed per node in 64-bit fixed point (order-free, hence
+ * reproducible bit for bit) at a resolution of 2^-32 relative to |h| / N (2^-(50 - ceil(log2 N)) for N above
+ * 2^18); embeddings must stay below 4096 in magnitude for that sum not to saturate, and a NaN embedding
+ * contributes 0 to it.
  * Node ids are checked on the device: an id outside [0, n) is clamped into range (so no
  * access ever leaves the arrays), the results of that call are then meaningless, and the
  * next synchronising call (lp_get_stats, lp_train_step_host) returns LP_EINVAL once.

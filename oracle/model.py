@@ -48,29 +48,39 @@ def split_predictor(D: int, Hp: int, tail: np.ndarray):
     return out
 
 
-def mlp_predictor_forward(HK, src, dst, pred, ties=None, tie_tol=0.0):
+def mlp_predictor_forward(HK, src, dst, pred, ties=None, rounding=None, var_HK=None, n_sigma: float = 6.0):
     """EdgePredictor of Eq. 2 as the 3-layer MLP of the paper's experiments (Section IV) on the Hadamard
     product of the two embeddings: z0 = h_u * h_v; p1 = ReLU(z0 W0 + b0); p2 = ReLU(p1 W1 + b1);
     s = p2 . w2 + b2.  ties = (active1, active2) decisions of the implementation under test, adopted only
-    inside the tie window (see forward())."""
-    def relu_decisions(a, given):
-        active = a > 0.0
-        flipped = 0
-        if given is not None and tie_tol > 0.0:
-            near = np.abs(a) <= tie_tol * np.sqrt(np.mean(a * a))
-            flipped = int((near & (active != given)).sum())
-            active = np.where(near, given, active)
-        return active, flipped
-
+    inside the rounding window of the pre-activation (see forward()); var_HK is the rounding-error variance
+    of H^(K) that forward() returns under the same rounding model."""
+    r = rounding_model(rounding)
     z0 = HK[src] * HK[dst]
-    a1 = z0 @ pred["W0"] + pred["b0"]
-    active1, t1 = relu_decisions(a1, None if ties is None else ties[0])
-    p1 = np.where(active1, a1, 0.0)
-    a2 = p1 @ pred["W1"] + pred["b1"]
-    active2, t2 = relu_decisions(a2, None if ties is None else ties[1])
-    p2 = np.where(active2, a2, 0.0)
-    s = p2 @ pred["w2"] + pred["b2"][0]
-    return s, {"z0": z0, "p1": p1, "p2": p2, "active1": active1, "active2": active2, "ties": t1 + t2}
+    out = {"z0": z0, "ties": 0, "n_near": 0, "near": [], "own_active": [], "window": [], "Z": []}
+    V = None
+    if r is not None:
+        vk = np.zeros_like(HK) if var_HK is None else var_HK
+        V = HK[dst] ** 2 * vk[src] + HK[src] ** 2 * vk[dst] + (r["u_store"] * z0) ** 2 / 3.0
+    A = z0
+    for li, (Wn, bn) in enumerate((("W0", "b0"), ("W1", "b1"))):
+        a = A @ pred[Wn] + pred[bn]
+        active = a > 0.0
+        given = None if ties is None else ties[li]
+        if r is not None:
+            var = _dense_error_variance([(A, V, pred[Wn])], pred[bn], r)
+            active, near, win, flipped = _relu_decisions(a, var, given, n_sigma)
+            out["ties"] += flipped
+            out["n_near"] += int(near.sum())
+            out["near"].append(near)
+            out["window"].append(win)
+            V = np.where(active, var + (r["u_store"] * a) ** 2 / 3.0, 0.0)
+        out["own_active"].append(a > 0.0)
+        out["Z"].append(a)
+        A = np.where(active, a, 0.0)
+        out["p%d" % (li + 1)] = A
+        out["active%d" % (li + 1)] = active
+    s = out["p2"] @ pred["w2"] + pred["b2"][0]
+    return s, out
 
 
 def mlp_predictor_backward(HK, src, dst, pred, cache, gs):
@@ -137,22 +147,101 @@ def _layer_graphs(g, n_layers: int, blocks, arch: str = "sage"):
     return out
 
 
+# Unit roundoffs of the two arithmetic paths a checked implementation may take (first-order rounding-error
+# model; the unit roundoff of round-to-nearest with p significand bits is 2^-p: 2^-8 for BF16, 2^-24 for FP32):
+#   u_in    rounding of the input features X when they are stored          (BF16 path: X is converted)
+#   u_store rounding of every stored activation (aggregates, embeddings)
+#   u_w     rounding of the weights before the dense transform             (BF16 path: W is converted)
+#   u_acc   one addition of the dense transform's accumulator; the tensor-core accumulator is credited with
+#           two bits less than FP32 because its additions need not round to nearest
+#   u_coef  one FP32 operation on an aggregation coefficient (1/deg, w / sqrt(d~ d~))
+ROUNDING = {
+    "fp32": {"u_in": 0.0, "u_store": 2.0 ** -24, "u_w": 0.0, "u_acc": 2.0 ** -24, "u_coef": 2.0 ** -24},
+    "bf16": {"u_in": 2.0 ** -8, "u_store": 2.0 ** -8, "u_w": 2.0 ** -8, "u_acc": 2.0 ** -22, "u_coef": 2.0 ** -24},
+}
+
+
+def rounding_model(rounding):
+    """None, the name of a path in ROUNDING, or a dict with the same keys."""
+    if rounding is None:
+        return None
+    return ROUNDING[rounding] if isinstance(rounding, str) else rounding
+
+
+def _dense_error_variance(parts, b, r):
+    """Variance of the rounding error of Z = sum_i A_i W_i + b computed in finite precision with ONE accumulator
+    (parts = [(A_i, VA_i, W_i), ...]), to first order, with every rounding taken as an independent error uniform in
+    +-u|x| (variance (u x)^2 / 3):
+      errors already in A (variance VA) and the rounding of W pass through the product;
+      each of the K additions of the accumulator rounds a partial sum that is at most sum_j |A_j W_j| + |b|."""
+    prop, S, K = 0.0, np.abs(b), 0
+    for A, VA, W in parts:
+        prop = prop + (VA + (r["u_w"] ** 2 / 3.0) * A * A) @ (W * W)
+        S = S + np.abs(A) @ np.abs(W)
+        K += A.shape[1]
+    return prop + K * (r["u_acc"] * S) ** 2 / 3.0
+
+
+def _aggregate_error_variance(mode, n, rp, cc, w, dt, H, VH, M, r):
+    """The same for M = AGG(H): the errors of H pass through with the squared coefficients; the coefficients
+    carry three FP32 roundings; the FP32 accumulator rounds deg partial sums bounded by AGG(|H|); the
+    result is rounded once more when it is stored."""
+    deg = np.diff(rp).astype(np.float64)
+    if mode == "gcn":
+        w32 = np.ones(cc.shape[0], dtype=np.float32) if w is None else np.asarray(w, dtype=np.float32)
+        d1 = sparse.gcn_degree(n, rp, w32) if dt is None else np.asarray(dt, dtype=np.float64)
+        prop = sparse.aggregate("gcn", n, rp, cc, (w32.astype(np.float64) ** 2).astype(np.float32), VH, d1 * d1)
+        absum = sparse.aggregate("gcn", n, rp, cc, w32, np.abs(H), d1)
+        terms = deg + 1.0
+    else:
+        prop = sparse.aggregate("mean", n, rp, cc, None, VH) / np.maximum(deg, 1.0)[:, None]
+        absum = sparse.aggregate("mean", n, rp, cc, None, np.abs(H))
+        terms = deg
+    return (prop + (3.0 * r["u_coef"] * absum) ** 2 / 3.0 + terms[:, None] * (2.0 ** -24 * absum) ** 2 / 3.0
+            + (r["u_store"] * M) ** 2 / 3.0)
+
+
+def _relu_decisions(Z, var, given, n_sigma, rows=None):
+    """The oracle's own decisions Z > 0, and the units whose pre-activation lies within n_sigma standard
+    deviations of the modelled rounding error of zero (the window): only there may the decisions `given`
+    by the implementation under test replace the oracle's own.  Returns (active, near, window, adopted
+    decisions that differ)."""
+    own = Z > 0.0
+    win = n_sigma * np.sqrt(var)
+    near = np.abs(Z) <= win
+    if rows is not None:  # rows outside the frontier are not computed at all: nothing to adopt there
+        inside = np.zeros(Z.shape[0], dtype=bool)
+        inside[rows] = True
+        near &= inside[:, None]
+    if given is None:
+        return own, near, win, 0
+    flipped = int((near & (own != given)).sum())
+    return np.where(near, given, own), near, win, flipped
+
+
 def forward(g, X: np.ndarray, params: np.ndarray, arch: str, dims: Sequence[int], blocks=None, relu_ties=None,
-            tie_tol: float = 0.0):
+            rounding=None, n_sigma: float = 6.0, final_variance: bool = False):
     """K-layer encoder (Eq. 1).  Layer k: A = AGG(H^(k-1)) [gcn] or [H^(k-1) | mean] [sage];
     Z = A W + b; H^(k) = ReLU(Z) for k < K and Z for k = K.  Returns the per-layer cache.
 
     ReLU turns a floating-point value into a yes/no decision (is the unit active?).  When a
-    pre-activation is zero up to rounding, FP64 and the FP32 arithmetic under test may decide
-    differently although both are right.  relu_ties[k] (bool [n, F_{k+1}], the decisions of the
-    implementation under test) is adopted ONLY where |Z| <= tie_tol * rms(Z), with tie_tol the
-    floating-point tolerance of the comparison; everywhere else the oracle decides by itself.
-    cache["ties"] counts the adopted decisions that differ from the oracle's own."""
+    pre-activation is zero up to the rounding of the arithmetic under test, that arithmetic and
+    FP64 may decide differently although both are right.  With `rounding` (a key of ROUNDING or a
+    dict of unit roundoffs) the oracle propagates a first-order model of that arithmetic's rounding
+    error through the layers (variances of independent roundings) and marks the units with
+    |Z| <= n_sigma * sigma(Z) -- cache["near"][k], cache["window"][k].  relu_ties[k] (bool [n, F_{k+1}],
+    the decisions of the implementation under test) is adopted ONLY on those units; everywhere else
+    the oracle decides by itself (cache["own_active"][k] holds its own decision on every unit, so a
+    test can demand equality outside the window).  cache["ties"] counts the adopted decisions that
+    differ from the oracle's own, cache["n_near"] the units inside the windows."""
     K = len(dims) - 1
     P = split_params(arch, dims, np.asarray(params, dtype=np.float64))
     H = np.asarray(X, dtype=np.float64)
-    cache = {"H": [H], "M": [], "Z": [], "active": [], "ties": 0, "graphs": _layer_graphs(g, K, blocks, arch)}
+    r = rounding_model(rounding)
+    cache = {"H": [H], "M": [], "Z": [], "active": [], "own_active": [], "near": [], "window": [], "ties": 0, "n_near": 0,
+             "var_HK": None, "graphs": _layer_graphs(g, K, blocks, arch)}
     mode = "gcn" if arch == "gcn" else "mean"
+    VH = (r["u_in"] * H) ** 2 / 3.0 if r is not None else None
     for k in range(K):
         rp, cc, w, act, dt = cache["graphs"][k]
         M = sparse.aggregate(mode, g.n, rp, cc, w if arch == "gcn" else None, H, dt)
@@ -160,21 +249,31 @@ def forward(g, X: np.ndarray, params: np.ndarray, arch: str, dims: Sequence[int]
             Z = M @ P[k]["W"] + P[k]["b"]
         else:
             Z = H @ P[k]["W_self"] + M @ P[k]["W_neigh"] + P[k]["b"]
+        var = None
+        if r is not None and (k < K - 1 or final_variance):
+            VM = _aggregate_error_variance(mode, g.n, rp, cc, w if arch == "gcn" else None, dt, H, VH, M, r)
+            if arch == "gcn":
+                var = _dense_error_variance([(M, VM, P[k]["W"])], P[k]["b"], r)
+            else:
+                var = _dense_error_variance([(H, VH, P[k]["W_self"]), (M, VM, P[k]["W_neigh"])], P[k]["b"], r)
         if k < K - 1:
             active = Z > 0.0
-            if relu_ties is not None and relu_ties[k] is not None and tie_tol > 0.0:
-                rows = Z if act is None else Z[act]
-                near = np.abs(Z) <= tie_tol * np.sqrt(np.mean(rows * rows))
-                if act is not None:  # rows outside the frontier are not computed at all: nothing to adopt there
-                    in_frontier = np.zeros(g.n, dtype=bool)
-                    in_frontier[act] = True
-                    near &= in_frontier[:, None]
-                cache["ties"] += int((near & (active != relu_ties[k])).sum())
-                active = np.where(near, relu_ties[k], active)
+            cache["own_active"].append(active)
+            if r is not None:
+                given = None if relu_ties is None else relu_ties[k]
+                active, near, win, flipped = _relu_decisions(Z, var, given, n_sigma, act)
+                cache["ties"] += flipped
+                cache["n_near"] += int(near.sum())
+                cache["near"].append(near)
+                cache["window"].append(win)
             cache["active"].append(active)
             Hn = np.where(active, Z, 0.0)
+            if r is not None:
+                VH = np.where(active, var + (r["u_store"] * Z) ** 2 / 3.0, 0.0)
         else:
             Hn = Z
+            if var is not None:
+                cache["var_HK"] = var + (r["u_store"] * Z) ** 2 / 3.0
         if act is not None:  # rows outside the frontier are not part of the computational graph
             keep = np.zeros(g.n, dtype=bool)
             keep[act] = True
@@ -195,8 +294,8 @@ def bce_with_logits(s: np.ndarray, y: np.ndarray):
     return ell, sig - y
 
 
-def train_step(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst, blocks=None, relu_ties=None, tie_tol=0.0,
-               pred_hidden: int = 0, pred_ties=None):
+def train_step(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst, blocks=None, relu_ties=None, rounding=None,
+               pred_hidden: int = 0, pred_ties=None, n_sigma: float = 6.0):
     """One training step of Algorithm 1 for one worker: scores of Eq. 2 (dot product) for
     positives (label 1) and negatives (label 0), loss L = (1/N) sum ell with N = |P| + |N|,
     and the gradient with respect to every parameter in the flat layout."""
@@ -205,7 +304,7 @@ def train_step(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst, blo
     n_enc = encoder_param_count(arch, dims)
     enc_params = params[:n_enc]
     P = split_params(arch, dims, enc_params)
-    cache = forward(g, X, enc_params, arch, dims, blocks, relu_ties, tie_tol)
+    cache = forward(g, X, enc_params, arch, dims, blocks, relu_ties, rounding, n_sigma, final_variance=pred_hidden > 0)
     HK = cache["H"][K]
     src = np.concatenate([pos_src, neg_src]).astype(np.int32)
     dst = np.concatenate([pos_dst, neg_dst]).astype(np.int32)
@@ -213,7 +312,7 @@ def train_step(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst, blo
     pred = pcache = None
     if pred_hidden > 0:
         pred = split_predictor(dims[K], pred_hidden, params[n_enc:])
-        s, pcache = mlp_predictor_forward(HK, src, dst, pred, pred_ties, tie_tol)
+        s, pcache = mlp_predictor_forward(HK, src, dst, pred, pred_ties, rounding, cache["var_HK"], n_sigma)
     else:
         s = np.einsum("ij,ij->i", HK[src], HK[dst])
     ell, dls = bce_with_logits(s, y)

@@ -1330,6 +1330,18 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         a.F = D;
         a.Y = dZ;
         a.ldy = D;
+        // Scale of the exact sum.  Every coefficient carries the 1 / N of the mean loss, so the products are of the order
+        // |h| / N: the power-of-two scale is 2^s * 2^ceil(log2 N) with s = min(32, 50 - ceil(log2 N)), which resolves a
+        // product to 2^-s relative to |h| / N whatever the batch size.  The coefficients of one node add up to at most 1
+        // in magnitude (dot product; a small multiple of it behind the MLP), so a node's sum stays below 2^63 as long
+        // as the embeddings stay below 4096 in magnitude.
+        {
+            int lg = 0;
+            while (((int64_t)1 << lg) < E) ++lg;
+            const int sh = std::min(32, 50 - lg) + lg;
+            a.exact_scale = ldexpf(1.f, sh);
+            a.exact_inv = ldexpf(1.f, -sh);
+        }
         if (ctx->mlp) {  // dL/dh_node = sum over incident edges of dL/dz0[edge] * h_other
             a.X2 = tptr<T>(ctx->dZ0);
             a.ldx2 = D;

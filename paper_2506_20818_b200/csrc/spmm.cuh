@@ -78,6 +78,9 @@ template <typename T> struct SpmmArgs {
     T *self_out = nullptr;
     int ldself = 0;
     int64_t nnz = 0;             // stored entries (host-known upper bound), sizes the heavy-row part of the grid
+    // exact (64-bit fixed-point) sums only: every product is multiplied by exact_scale, a power of two chosen by the caller
+    // from the magnitude of the coefficients, before it is rounded to an integer; the sum is multiplied by exact_inv = 1 / exact_scale
+    float exact_scale = 1099511627776.f, exact_inv = 1.f / 1099511627776.f;  // 2^40
     HeavyPlan heavy;             // heavy rows of this structure: prebuilt (static graph) or scratch to fill per launch
 };
 
@@ -85,13 +88,14 @@ constexpr int SPMM_THREADS = 256;
 
 // Accumulator of one output element.  float: FMA in entry order (the result depends on the order of a
 // row's entries, which is fixed for every structure built by a stable sort).  long long: each product
-// is rounded once to a multiple of 2^-40 and added as an integer -- exact and therefore independent of
-// the order of the entries; used for lists whose entry order is not reproducible (slots claimed with
-// integer atomics), so that their sums still are, bit for bit.
-constexpr float SPMM_EXACT_SCALE = 1099511627776.f;  // 2^40: products up to 2^23 in magnitude, resolution 9.1e-13
+// (coefficient already multiplied by the power-of-two scale of SpmmArgs) is rounded once to an integer and
+// added as an integer -- exact and therefore independent of the order of the entries; used for lists whose
+// entry order is not reproducible (slots claimed with integer atomics), so that their sums still are, bit
+// for bit.  With scale 2^s the resolution of a product is 2^-s and the sum of a row must stay below 2^(63-s)
+// in magnitude; NaN counts as 0 and larger values saturate, so the caller picks s from the data's range.
 template <typename ACC> LP_DEVINL void acc_add(ACC &a, float w, float f);
 template <> LP_DEVINL void acc_add<float>(float &a, float w, float f) { a = fmaf(w, f, a); }
-template <> LP_DEVINL void acc_add<long long>(long long &a, float w, float f) { a += __float2ll_rn(w * f * SPMM_EXACT_SCALE); }
+template <> LP_DEVINL void acc_add<long long>(long long &a, float w, float f) { a += __float2ll_rn(w * f); }
 // acc[0..VN) += w * v for one 16-byte vector.  Unit coefficients on BF16 data into FP32 accumulators use the
 // mixed-precision add of sm_100 (add.rn.f32.bf16: the BF16 operand is widened exactly, one rounding, the
 // same result as convert-then-add) and so skip the eight conversion instructions per vector.
@@ -103,21 +107,6 @@ template <typename T, typename ACC, bool HAS_VAL> LP_DEVINL void acc_add_vec(ACC
 #pragma unroll
     for (int t = 0; t < VN; ++t) acc_add<ACC>(acc[t], w, f[t]);
 }
-// exact accumulator: the power-of-two scale is folded into the coefficient once per vector (exact), leaving one
-// multiplication, one conversion and one 64-bit addition per element
-template <typename T, bool HAS_VAL> LP_DEVINL void acc_add_vec_exact(long long *acc, float w, const Vec16<T> &v)
-{
-    constexpr int VN = Vec16<T>::N;
-    float f[VN];
-    v.to_float(f);
-    const float ws = w * SPMM_EXACT_SCALE;
-#pragma unroll
-    for (int t = 0; t < VN; ++t) acc[t] += __float2ll_rn(ws * f[t]);
-}
-template <> LP_DEVINL void acc_add_vec<bf16, long long, true>(long long *acc, float w, const Vec16<bf16> &v) { acc_add_vec_exact<bf16, true>(acc, w, v); }
-template <> LP_DEVINL void acc_add_vec<bf16, long long, false>(long long *acc, float w, const Vec16<bf16> &v) { acc_add_vec_exact<bf16, false>(acc, w, v); }
-template <> LP_DEVINL void acc_add_vec<float, long long, true>(long long *acc, float w, const Vec16<float> &v) { acc_add_vec_exact<float, true>(acc, w, v); }
-template <> LP_DEVINL void acc_add_vec<float, long long, false>(long long *acc, float w, const Vec16<float> &v) { acc_add_vec_exact<float, false>(acc, w, v); }
 template <> LP_DEVINL void acc_add_vec<bf16, float, false>(float *acc, float, const Vec16<bf16> &v)
 {
     const uint32_t x[4] = {v.v.x, v.v.y, v.v.z, v.v.w};
@@ -129,8 +118,8 @@ template <> LP_DEVINL void acc_add_vec<bf16, float, false>(float *acc, float, co
 }
 template <typename ACC> LP_DEVINL float acc_value(ACC a);
 template <> LP_DEVINL float acc_value<float>(float a) { return a; }
-// one rounding (64-bit integer to FP32, to nearest); the power-of-two scale is exact
-template <> LP_DEVINL float acc_value<long long>(long long a) { return __ll2float_rn(a) * (1.f / SPMM_EXACT_SCALE); }
+// one rounding (64-bit integer to FP32, to nearest); the epilogue multiplies by the exact power-of-two 1 / scale
+template <> LP_DEVINL float acc_value<long long>(long long a) { return __ll2float_rn(a); }
 constexpr int SPMM_HEAVY_MIN = 64;  // smallest heavy-row threshold a plan may use (bounds the item count by nnz / 64).
                                     // A lane group keeps only a few gathers in flight, so a long row handled by one
                                     // group is a long dependent chain: long rows are cut into items instead.
@@ -149,6 +138,7 @@ LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl,
                                 bool have_first = false, int first_col = 0, float first_val = 0.f)
 {
     constexpr int VN = Vec16<T>::N;
+    const float wscale = sizeof(ACC) == 8 ? a.exact_scale : 1.f;  // exact sums: the power-of-two scale rides on the coefficient
     for (int e0 = e_lo; e0 < e_hi; e0 += G) {
         const int my_e = e0 + gl;
         int my_col = first_col;
@@ -172,7 +162,7 @@ LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl,
 #pragma unroll
             for (int q = 0; q < U; ++q) {
                 c[q] = __shfl_sync(gmask, my_col, j + q, G);
-                w[q] = HAS_VAL ? __shfl_sync(gmask, my_val, j + q, G) : 1.f;
+                w[q] = (HAS_VAL ? __shfl_sync(gmask, my_val, j + q, G) : 1.f) * wscale;
             }
 #pragma unroll
             for (int q = 0; q < U; ++q)
@@ -205,7 +195,7 @@ LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl,
         }
         for (; j < cnt; ++j) {
             const int c = __shfl_sync(gmask, my_col, j, G);
-            const float w = HAS_VAL ? __shfl_sync(gmask, my_val, j, G) : 1.f;
+            const float w = (HAS_VAL ? __shfl_sync(gmask, my_val, j, G) : 1.f) * wscale;
             const int c2 = HAS_X2 ? __shfl_sync(gmask, my_col2, j, G) : 0;
 #pragma unroll
             for (int i = 0; i < NV; ++i) {
@@ -235,7 +225,7 @@ template <typename T, int G, int NV, typename ACC>
 LP_DEVINL void spmm_epilogue(const SpmmArgs<T> &a, int r, int gl, int nchunks, const ACC (&acc)[NV][Vec16<T>::N])
 {
     constexpr int VN = Vec16<T>::N;
-    const float scale = a.row_scale ? __ldg(a.row_scale + r) : 1.f;
+    const float scale = (a.row_scale ? __ldg(a.row_scale + r) : 1.f) * (sizeof(ACC) == 8 ? a.exact_inv : 1.f);
     int irow = -1;
     float icoef = 0.f;
     if (a.init) {

@@ -62,3 +62,28 @@ def rel_l2(a, b):
     b = np.asarray(b, dtype=np.float64).ravel()
     den = np.linalg.norm(b)
     return float(np.linalg.norm(a - b) / den) if den > 0 else float(np.linalg.norm(a - b))
+
+
+def assert_relu_decisions_agree(cache, gpu_masks, rows_per_layer=None, label=""):
+    """ReLU is the one place where floating point decides a yes/no.  `cache` is the oracle's forward cache computed
+    with a rounding model: outside the rounding window of a pre-activation the decision is unique, so the decisions of
+    the implementation under test (`gpu_masks[k]`, bool [n, F]) must equal the oracle's OWN decisions there, bit for
+    bit; inside the window either decision is valid.  The number of units inside the window is bounded by what a window
+    of that width can hold: a pre-activation with standard deviation s has density at most 0.4 / s at zero, so a unit
+    falls within +-w of zero with probability about 0.8 w / s (twice that, plus 16, is allowed).
+    Returns (units inside the windows, adopted decisions that differ from the oracle's own)."""
+    inside = differ = 0
+    for k, gm in enumerate(gpu_masks):
+        own, near, win, Z = cache["own_active"][k], cache["near"][k], cache["window"][k], cache["Z"][k]
+        if rows_per_layer is not None:
+            r = rows_per_layer[k]
+            gm, own, near, win, Z = gm[r], own[r], near[r], win[r], Z[r]
+        wrong = (gm != own) & ~near
+        assert not wrong.any(), f"{label} layer {k + 1}: {int(wrong.sum())} ReLU decisions differ outside the rounding window"
+        s = np.sqrt(np.mean(Z * Z))
+        capacity = 16 + 2.0 * float(np.minimum(1.0, 0.8 * win / s).sum()) if s > 0 else 16
+        assert near.sum() <= capacity, f"{label} layer {k + 1}: {int(near.sum())} units inside the window, a window of this width holds {capacity:.0f}"
+        inside += int(near.sum())
+        differ += int((near & (gm != own)).sum())
+    print(f"{label} ReLU windows: {inside} units inside, {differ} decisions adopted from the implementation under test")
+    return inside, differ

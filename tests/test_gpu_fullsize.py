@@ -6,7 +6,7 @@ import pytest
 
 import oracle
 import workloads as wl
-from helpers import rel_l2
+from helpers import assert_relu_decisions_agree, rel_l2
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -55,9 +55,8 @@ def test_config2_full_size_step(pkg, config2, prec):
     ons, ond, oex = oracle.sample_negatives(g.n, g.rowptr, g.col, u, seed, step, 1, edge_index_base=lo)
     assert np.array_equal(nd.cpu().numpy(), ond) and ctx.stats().negatives_exhausted == oex
     H1 = ctx.embeddings(1).cpu().numpy()
-    ref = oracle.train_step(g, X, params, "sage", dims, u, v, ons, ond, relu_ties=[H1 > 0], tie_tol=TOL[prec])
-    n_hidden = ref["cache"]["Z"][0].size
-    assert ref["cache"]["ties"] <= (8 if prec == "fp32" else 0.01 * n_hidden)
+    ref = oracle.train_step(g, X, params, "sage", dims, u, v, ons, ond, relu_ties=[H1 > 0], rounding=prec)
+    assert_relu_decisions_agree(ref["cache"], [H1 > 0], None, f"config 2 full size {prec}")
     err = {"loss": abs(loss.item() - ref["loss"]) / abs(ref["loss"]),
            "H1": rel_l2(H1, ref["cache"]["H"][1]),
            "H2": rel_l2(ctx.embeddings(2).cpu().numpy(), ref["cache"]["H"][2]),

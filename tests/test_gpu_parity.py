@@ -8,7 +8,7 @@ import pytest
 
 import oracle
 import workloads as wl
-from helpers import rel_l2
+from helpers import assert_relu_decisions_agree, rel_l2
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -266,8 +266,10 @@ def test_negatives_exhaustion_counter(pkg):
 
 
 # ------------------------------------------------------------------------------------------ full step
-def run_step(pkg, g, X, params, arch, dims, prec, pos, k=1, seed=5, step=0, fanout=None, cand=None, check_layers=True):
-    """One training step both ways; returns a dict of relative errors and the raw results."""
+def run_step(pkg, g, X, params, arch, dims, prec, pos, k=1, seed=5, step=0, fanout=None, cand=None, check_layers=True, adopt=True):
+    """One training step both ways; returns a dict of relative errors and the raw results.
+    adopt = False: the oracle takes every ReLU decision by itself (the caller has made sure that no pre-activation
+    lies inside a rounding window) and the implementation's decisions must equal them everywhere."""
     u, v = pos
     ctx = make_ctx(pkg, g, X)
     ctx.set_model(arch, dims, prec=prec, fanout=fanout, max_batch=len(u), max_k=max(k, 1))
@@ -292,23 +294,27 @@ def run_step(pkg, g, X, params, arch, dims, prec, pos, k=1, seed=5, step=0, fano
     if fanout:
         seeds = np.concatenate([u, v, ond])
         blocks = oracle.build_blocks(g.n, g.rowptr, g.col, seeds, fanout, seed, step)
-    # ReLU decisions on pre-activations that are zero up to the path's rounding are taken from the GPU
-    # (both sides must take a float-decides-an-integer decision in the same precision); the window is
-    # the path's tolerance times the RMS pre-activation, and the number of adopted decisions is bounded.
-    ties = None
+    # ReLU decisions: where a pre-activation is zero up to the rounding of the path (the oracle's window, derived from
+    # the unit roundoffs of the FP32 or BF16 arithmetic) the oracle adopts the GPU's decision; outside the window the GPU's
+    # decisions must equal the oracle's own, bit for bit.
+    ties, rows_per_layer = None, None
     if K > 1:
         ties = []
+        if fanout:
+            rows_per_layer = [blocks[0][K - layer] for layer in range(1, K)]
         for layer in range(1, K):
             if fanout:
                 full = np.zeros((g.n, dims[layer]), dtype=bool)
-                rows_l = oracle.build_blocks(g.n, g.rowptr, g.col, np.concatenate([u, v, ond]), fanout, seed, step)[0][K - layer]
+                rows_l = rows_per_layer[layer - 1]
                 full[rows_l] = ctx.embeddings(layer, rows=len(rows_l)).cpu().numpy() > 0
                 ties.append(full)
             else:
                 ties.append(ctx.embeddings(layer).cpu().numpy() > 0)
-    ref = oracle.train_step(g, X, params, arch, dims, u, v, ons, ond, blocks=blocks, relu_ties=ties, tie_tol=TOL[prec])
-    n_hidden = sum(z.size for z in ref["cache"]["Z"][:-1])
-    assert ref["cache"]["ties"] <= (4 if prec == "fp32" else 0.01 * n_hidden), f"too many ReLU decisions adopted: {ref['cache']['ties']}"
+    ref = oracle.train_step(g, X, params, arch, dims, u, v, ons, ond, blocks=blocks, relu_ties=ties if adopt else None, rounding=prec)
+    if K > 1:
+        inside, _ = assert_relu_decisions_agree(ref["cache"], ties, rows_per_layer, f"{arch}/{prec}")
+        if not adopt:
+            assert inside == 0 and ref["cache"]["ties"] == 0
     err = {"loss": abs(loss.item() - ref["loss"]) / abs(ref["loss"]),
            "grads": rel_l2(grads.cpu().numpy(), ref["grads"])}
     if fanout:
@@ -376,6 +382,27 @@ def test_config3_coauthor_gcn3_weighted(pkg, prec):
     g, X, params, pos, cfg = wl.make_config("c3_coauthor_gcn3", scale=0.04)
     assert g.w is not None and g.w.max() > 1
     err, _, _ = run_step(pkg, g, X, params, "gcn", cfg["dims"], prec, pos)
+    assert_within(err, TOL[prec])
+
+
+@pytest.mark.parametrize("arch,prec", [("gcn", "fp32"), ("gcn", "bf16"), ("sage", "fp32"), ("sage", "bf16")])
+def test_step_parity_without_adopted_relu_decisions(pkg, arch, prec):
+    # A 3-layer step in which the oracle takes EVERY ReLU decision itself.  The biases of the two hidden layers are set to
+    # +-6 standard deviations of the layer's pre-activations (alternating by unit), so that -- as the oracle alone
+    # establishes -- no pre-activation lies inside a rounding window; the GPU's decisions must then equal the oracle's on
+    # every unit, and the gradients are compared without anything taken from the code under test.
+    g = wl.erdos_renyi(3000, 24000, seed=12)
+    dims = [64, 128, 128, 64]
+    X = wl.node_features(g.n, 64, 2)
+    params = wl.glorot_params(arch, dims, 3, 0.0)
+    P = oracle.split_params(arch, dims, params)  # views into params
+    for k in (0, 1):
+        Z = oracle.forward(g, X, params, arch, dims)["Z"][k]
+        P[k]["b"][:] = 6.0 * np.sqrt(np.mean(Z * Z)) * np.where(np.arange(dims[k + 1]) % 2 == 0, 1.0, -1.0)
+    own = oracle.forward(g, X, params, arch, dims, rounding=prec)
+    assert own["n_near"] == 0 and all(0.3 < a.mean() < 0.7 for a in own["own_active"])
+    u, v = wl.undirected_edge_list(g)
+    err, _, _ = run_step(pkg, g, X, params, arch, dims, prec, (u[:6000].copy(), v[:6000].copy()), adopt=False)
     assert_within(err, TOL[prec])
 
 
@@ -764,9 +791,12 @@ def test_mlp_predictor_step(pkg, arch, prec, fanout):
         ties = [ctx.embeddings(1).cpu().numpy() > 0]
     E = len(u) * (1 + k)
     pred_ties = [ctx.predictor_activations(1, E).cpu().numpy() > 0, ctx.predictor_activations(2, E).cpu().numpy() > 0]
-    ref = oracle.train_step(g, X, params, arch, dims, u, v, ons, ond, blocks=blocks, relu_ties=ties, tie_tol=TOL[prec], pred_hidden=Hp,
+    ref = oracle.train_step(g, X, params, arch, dims, u, v, ons, ond, blocks=blocks, relu_ties=ties, rounding=prec, pred_hidden=Hp,
                             pred_ties=pred_ties)
-    assert ref["pred_cache"]["ties"] <= (8 if prec == "fp32" else 0.01 * 2 * E * Hp)
+    # outside the rounding windows the GPU's ReLU decisions equal the oracle's own (encoder and predictor)
+    if ties is not None:
+        assert_relu_decisions_agree(ref["cache"], ties, None, f"{arch}/{prec} encoder")
+    assert_relu_decisions_agree(ref["pred_cache"], pred_ties, None, f"{arch}/{prec} predictor")
     n_enc = oracle.encoder_param_count(arch, dims)
     gg = grads.cpu().numpy()
     err = {"loss": abs(loss.item() - ref["loss"]) / abs(ref["loss"]),
