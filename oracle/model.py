@@ -286,6 +286,15 @@ def forward(g, X: np.ndarray, params: np.ndarray, arch: str, dims: Sequence[int]
     return cache
 
 
+def edge_dot(HK: np.ndarray, src: np.ndarray, dst: np.ndarray, chunk: int = 65536) -> np.ndarray:
+    """s_e = <h_src(e), h_dst(e)> (Eq. 2 with the dot product), one edge at a time; the edges are taken in slices so that
+    the two gathered row blocks stay small whatever the number of scored edges (no sum is split or reordered)."""
+    out = np.empty(src.shape[0], dtype=np.float64)
+    for lo in range(0, src.shape[0], chunk):
+        out[lo:lo + chunk] = np.einsum("ij,ij->i", HK[src[lo:lo + chunk]], HK[dst[lo:lo + chunk]])
+    return out
+
+
 def bce_with_logits(s: np.ndarray, y: np.ndarray):
     """Per-edge binary cross-entropy of label y and probability sigmoid(s), in the
     overflow-free form  max(s,0) - s*y + log(1 + exp(-|s|)), and d/ds = sigmoid(s) - y."""
@@ -314,7 +323,7 @@ def train_step(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst, blo
         pred = split_predictor(dims[K], pred_hidden, params[n_enc:])
         s, pcache = mlp_predictor_forward(HK, src, dst, pred, pred_ties, rounding, cache["var_HK"], n_sigma)
     else:
-        s = np.einsum("ij,ij->i", HK[src], HK[dst])
+        s = edge_dot(HK, src, dst)
     ell, dls = bce_with_logits(s, y)
     N = s.shape[0]
     loss = ell.sum() / N
@@ -364,7 +373,7 @@ def input_gradient(g, X, params, arch, dims, pos_src, pos_dst, neg_src, neg_dst)
     src = np.concatenate([pos_src, neg_src]).astype(np.int32)
     dst = np.concatenate([pos_dst, neg_dst]).astype(np.int32)
     y = np.concatenate([np.ones(len(pos_src)), np.zeros(len(neg_src))])
-    s = np.einsum("ij,ij->i", HK[src], HK[dst])
+    s = edge_dot(HK, src, dst)
     _, dls = bce_with_logits(s, y)
     dH = sparse.edge_grad(HK, src, dst, dls / s.shape[0])
     mode = "gcn" if arch == "gcn" else "mean"
@@ -386,7 +395,7 @@ def score(g, X, params, arch, dims, src, dst, blocks=None, pred_hidden: int = 0)
     if pred_hidden > 0:
         pred = split_predictor(dims[-1], pred_hidden, params[n_enc:])
         return mlp_predictor_forward(HK, np.asarray(src), np.asarray(dst), pred)[0]
-    return np.einsum("ij,ij->i", HK[np.asarray(src)], HK[np.asarray(dst)])
+    return edge_dot(HK, np.asarray(src), np.asarray(dst))
 
 
 def hits_at_k(pos_scores, neg_scores, k: int) -> float:

@@ -28,12 +28,16 @@ class Graph:
         return int(self.col.shape[0])
 
 
-def csr_from_edges(n: int, dst: np.ndarray, src: np.ndarray, w: Optional[np.ndarray] = None) -> Graph:
-    """Build CSR (rows = dst, cols = src) from a list of distinct directed entries."""
+def csr_from_edges(n: int, dst: np.ndarray, src: np.ndarray, w: Optional[np.ndarray] = None, presorted: bool = False) -> Graph:
+    """Build CSR (rows = dst, cols = src) from a list of distinct directed entries
+    (presorted: the list is already ordered by (dst, src), so the sort is skipped)."""
     dst = np.asarray(dst, dtype=np.int64)
     src = np.asarray(src, dtype=np.int64)
-    order = np.lexsort((src, dst))
-    dst, src = dst[order], src[order]
+    if presorted:
+        order = slice(None)
+    else:
+        order = np.lexsort((src, dst))
+        dst, src = dst[order], src[order]
     counts = np.bincount(dst, minlength=n).astype(np.int64)
     rowptr = np.zeros(n + 1, dtype=np.int64)
     np.cumsum(counts, out=rowptr[1:])
@@ -159,8 +163,9 @@ def citation_directed(n: int, m: int, gamma_in: float, seed: int) -> Graph:
     dst = relabel[_draw_weighted(rng, cdf, m)].astype(np.int64)
     src = rng.integers(0, n, size=m).astype(np.int64)
     keep = dst != src
-    key = np.unique(dst[keep] * n + src[keep])
-    g = csr_from_edges(n, key // n, key % n)
+    key = np.sort(dst[keep] * n + src[keep])  # ascending (dst, src); duplicates are neighbours
+    key = key[np.concatenate([[True], key[1:] != key[:-1]])]
+    g = csr_from_edges(n, key // n, key % n, presorted=True)
     g.directed = True
     g.meta = {"family": "citation_directed", "seed": seed, "gamma_in": gamma_in, "entries": g.nnz}
     return g
