@@ -7,7 +7,12 @@ with Adam.  The metric is training edges per second (positives + negatives) over
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-Prints ONE JSON line (see the design doc for the meaning of every key).
+Prints ONE JSON line.  Keys beyond the usual ones:
+  roofline      the aggregation launches of the timed region (the dominant kernel), algorithmic bytes / time
+  hbm_roofline  the same kernel on a graph whose source matrix does not fit the L2 cache (HBM-bound)
+  configs       the other workload configurations at full size (parity-tested elsewhere; timed here)
+  cpu_baseline  the CPU oracle on the host cores, one thread and all cores
+  e2e           the same metric through the host-buffer entry point, copies inside the timed region
 """
 from __future__ import annotations
 
@@ -15,6 +20,7 @@ import argparse
 import hashlib
 import json
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -33,9 +39,8 @@ K_NEG = 1
 SEED = 1234
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the aggregation launches of one step on the
-# benchmark workload, from one ncu capture (profiles/spmm_padded_bf16_config2.md): layer-1 forward 123.7 MB,
-# layer-2 forward 408.8 MB, adjoint 628.4 MB -> mean per timed launch.  Valid only for the kernel source it
-# was taken with (sha1 of csrc/spmm.cuh + csrc/common.cuh); reported as null otherwise.
+# benchmark workload, from one ncu capture of a whole step at full size: mean per timed launch.  Valid only for the
+# kernel source it was taken with (sha1 of csrc/spmm.cuh + csrc/common.cuh); reported as null otherwise.
 NCU_TRAFFIC = {"spmm_sha1": "897672ea779116af0d86a2a91421625fa1b531bd", "bytes_per_launch": (123.7e6 + 408.8e6 + 628.4e6) / 3.0}
 
 
@@ -138,6 +143,214 @@ def run_oracle_steps(g, X, params, dims, pos, B, steps, warmup):
     return times
 
 
+def oracle_baseline(g, X, params, dims, pos, B, steps_all_cores):
+    """The oracle on the host: the requested number of steps with every core the process may use, and one step held to a
+    single thread (numpy's BLAS pool and the C part's OpenMP team both limited to 1)."""
+    out = {"unit": UNIT, "cores": cpu_cores(), "kind": "oracle"}
+    times = run_oracle_steps(g, X, params, dims, pos, B, steps_all_cores, 0)
+    out["value"] = len(times) * B * (1 + K_NEG) / sum(times)
+    out["s_per_step"] = sum(times) / len(times)
+    out["sample"] = (f"{len(times)} full steps of the same workload on all {out['cores']} cores (full-graph encoder, {B} positives + "
+                     f"{B * K_NEG} negatives each); 1 such step on one thread")
+    try:
+        from threadpoolctl import threadpool_limits
+        with threadpool_limits(limits=1):
+            t1 = run_oracle_steps(g, X, params, dims, pos, B, 1, 0)
+        out["single_thread"] = {"value": B * (1 + K_NEG) / t1[0], "unit": UNIT, "cores": 1, "s_per_step": t1[0]}
+    except Exception as ex:  # the single-thread figure is additional: never lose the other one over it
+        out["single_thread"] = {"value": None, "note": f"failed: {ex}"}
+    return out
+
+
+def free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+# ------------------------------------------------------------------------------------------------------------------
+# the other configurations, timed at full size after the headline region (N = 1, rank 0)
+# ------------------------------------------------------------------------------------------------------------------
+def _events(torch):
+    return torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+
+def time_steps(torch, ctx, params, pu, pv, B, k, steps, warmup, seed=SEED):
+    """ms per step of negatives + step + Adam on consecutive batches of B positives (wrapping around)."""
+    dev = pu.device
+    p = params.clone()
+    m, v, grads = torch.zeros_like(p), torch.zeros_like(p), torch.zeros_like(p)
+    loss = torch.zeros(1, device=dev)
+    nb = max(1, pu.numel() // B)
+
+    def one(i):
+        lo = (i % nb) * B
+        su, sv = pu[lo:lo + B], pv[lo:lo + B]
+        _, nd = ctx.sample_negatives(seed, i, k, su, edge_index_base=lo)
+        ctx.train_step(p, su, sv, None, nd, k, loss, grads, seed=seed, step=i)
+        ctx.adam_step(p, m, v, grads, i + 1)
+
+    for i in range(warmup):
+        one(i)
+    torch.cuda.synchronize()
+    a, b = _events(torch)
+    a.record()
+    for i in range(steps):
+        one(warmup + i)
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / steps
+    Bq = min(B, pu.numel())
+    return {"ms_per_step": ms, "edges_per_s": Bq * (1 + k) / (ms * 1e-3), "batch_pos": Bq, "steps": steps, "loss_last": float(loss.item())}
+
+
+def bench_other_configs(torch, pkg, wl, dev):
+    out = {}
+    t_all = time.perf_counter()
+
+    def t(a):
+        return torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+
+    # ---- config 1: tiny graph, 2-layer GCN, FP32, every edge a positive
+    g, X, params, pos, cfg = wl.make_config("c1_tiny_er_gcn2")
+    ctx = pkg.Context(0)
+    ctx.load_graph(g.n, g.rowptr, g.col, g.w, X)
+    ctx.set_model("gcn", cfg["dims"], prec="fp32", max_batch=len(pos[0]), max_k=1)
+    out["c1_tiny_er_gcn2"] = dict(time_steps(torch, ctx, t(params), t(pos[0]), t(pos[1]), len(pos[0]), 1, 100, 5), nodes=g.n, entries=g.nnz, dtype="f32")
+    ctx.close()
+
+    # ---- config 2 variants: every training positive behind one encoder pass; mini-batches over sampled blocks
+    g, X, params, pos, cfg = wl.make_config("c2_chunglu_sage2")
+    ctx = pkg.Context(0)
+    ctx.load_graph(g.n, g.rowptr, g.col, g.w, X)
+    pu, pv, pp = t(pos[0]), t(pos[1]), t(params)
+    ctx.set_model("sage", cfg["dims"], prec="bf16", max_batch=len(pos[0]), max_k=1)
+    out["c2_one_pass_all_positives"] = dict(time_steps(torch, ctx, pp, pu, pv, len(pos[0]), 1, 20, 3), nodes=g.n, entries=g.nnz, dtype="bf16")
+    for B in (256, 10240, 51200):
+        ctx.set_model("sage", cfg["dims"], prec="bf16", fanout=[25, 10], max_batch=B, max_k=1)
+        out[f"c2_minibatch_fanout25_10_B{B}"] = dict(time_steps(torch, ctx, pp, pu, pv, B, 1, 30, 5), dtype="bf16")
+    ctx.close()
+
+    # ---- config 3: weighted 3-layer GCN, full graph (every training edge a positive; B = 65,536) and mini-batches
+    g, X, params, pos, cfg = wl.make_config("c3_coauthor_gcn3")
+    ctx = pkg.Context(0)
+    ctx.load_graph(g.n, g.rowptr, g.col, g.w, X)
+    pu, pv, pp = t(pos[0]), t(pos[1]), t(params)
+    ctx.set_model("gcn", cfg["dims"], prec="bf16", max_batch=len(pos[0]), max_k=1)
+    out["c3_coauthor_gcn3"] = dict(time_steps(torch, ctx, pp, pu, pv, len(pos[0]), 1, 20, 3), nodes=g.n, entries=g.nnz, dtype="bf16")
+    out["c3_coauthor_gcn3_B65536"] = dict(time_steps(torch, ctx, pp, pu, pv, 65536, 1, 30, 3), dtype="bf16")
+    for B in (256, 10240, 51200):
+        ctx.set_model("gcn", cfg["dims"], prec="bf16", fanout=[25, 10, 5], max_batch=B, max_k=1)
+        out[f"c3_minibatch_fanout25_10_5_B{B}"] = dict(time_steps(torch, ctx, pp, pu, pv, B, 1, 30, 5), dtype="bf16")
+    ctx.close()
+
+    # ---- config 4: directed 2.9 M-node graph, 3-layer SAGE-mean over sampled blocks (fan-outs 15/10/5)
+    g, X, params, pos, cfg = wl.make_config("c4_citation_sage3_sampled")
+    ctx = pkg.Context(0)
+    ctx.load_graph(g.n, g.rowptr, g.col, None, X)
+    ctx.set_model("sage", cfg["dims"], prec="bf16", fanout=cfg["fanout"], max_batch=65536, max_k=1)
+    sel = np.random.default_rng(4).permutation(len(pos[0]))[: 16 * 65536]
+    r = time_steps(torch, ctx, t(params), t(pos[0][sel]), t(pos[1][sel]), 65536, 1, 12, 3)
+    st = ctx.stats()
+    out["c4_citation_sage3_sampled"] = dict(r, nodes=g.n, entries=g.nnz, dtype="bf16", frontier_nodes=[int(st.block_nodes[h]) for h in range(3)],
+                                           block_entries=[int(st.block_edges[h]) for h in range(3)])
+    ctx.close()
+    del X
+
+    # ---- config 5: 8 emulated workers in sequence, gradients accumulated, one update; local vs global negatives
+    g, X, params, pos, cfg = wl.make_config("c5_partitioned_sage2")
+    p_workers, B = cfg["partitions"], 65536
+    part = wl.random_partition(g.n, p_workers, seed=5)
+    ctxG = pkg.Context(0)
+    ctxG.load_graph(g.n, g.rowptr, g.col, None, X)
+    a, b = _events(torch)
+    a.record()
+    ctxG.sparsify(cfg["alpha"], 5)
+    b.record()
+    torch.cuda.synchronize()
+    sparsify_ms = a.elapsed_time(b)
+    dpart, X_dev, pp = t(part), t(X), t(params)
+    rows = np.repeat(np.arange(g.n, dtype=np.int64), np.diff(g.rowptr))
+    upper = g.col > rows
+    prow, pcol = part[rows], part[g.col]
+    for negatives in ("local", "global"):
+        acc = torch.zeros_like(pp)
+        scratch = torch.zeros_like(pp)
+        loss = torch.zeros(1, device=dev)
+        total_ms, edges, n_batches, view_entries = 0.0, 0, 0, 0
+        for i in range(p_workers):
+            rp, col, vstats = ctxG.worker_view(dpart, i, keep_cross_edges=False, foreign_mode=0 if negatives == "local" else 1)
+            view_entries += int(col.numel())
+            ctx = pkg.Context(0)
+            ctx.load_graph(g.n, rp, col, None, X_dev, on_device=True)
+            ctx.set_model("sage", cfg["dims"], prec="bf16", max_batch=B, max_k=1)
+            if negatives == "local":
+                ctx.set_candidates(t(np.nonzero(part == i)[0].astype(np.int32)))
+            keep = upper & (prow == i) & (pcol == i)  # the partition's own undirected edges, each once
+            pu, pv = t(rows[keep].astype(np.int32)), t(g.col[keep].astype(np.int32))
+            nbat = (pu.numel() + B - 1) // B
+            _, nd = ctx.sample_negatives(SEED, 10_000 + i, 1, pu[:B])  # warm-up step into a scratch gradient
+            ctx.train_step(pp, pu[:B], pv[:B], None, nd, 1, loss, scratch, seed=SEED, step=0)
+            torch.cuda.synchronize()
+            a, b = _events(torch)
+            a.record()
+            for j in range(nbat):
+                su, sv = pu[j * B:(j + 1) * B], pv[j * B:(j + 1) * B]
+                _, nd = ctx.sample_negatives(SEED, i * 64 + j, 1, su, edge_index_base=j * B)
+                ctx.train_step(pp, su, sv, None, nd, 1, loss, acc, seed=SEED, step=i * 64 + j, accumulate=True)
+            if i == p_workers - 1:  # Algorithm 1: average over the workers, then one update
+                m, v = torch.zeros_like(pp), torch.zeros_like(pp)
+                ctx.adam_step(pp.clone(), m, v, acc, 1, grad_scale=1.0 / p_workers)
+            b.record()
+            torch.cuda.synchronize()
+            total_ms += a.elapsed_time(b)
+            edges += 2 * int(pu.numel())
+            n_batches += nbat
+            ctx.close()
+        out[f"c5_partitioned_sage2_{negatives}_negatives"] = {"ms_per_pass": total_ms, "edges_per_s": edges / (total_ms * 1e-3), "batches": n_batches, "scored_edges": edges,
+                                                             "workers": p_workers, "nodes": g.n, "entries_global": g.nnz, "entries_all_views": view_entries, "dtype": "bf16",
+                                                             "note": "one pass over every partition's own positives in batches of 65,536, gradients accumulated "
+                                                                     "in partition order, one Adam update; graph loading and view building outside the timed spans"}
+    out["c5_sparsify_global_graph_ms"] = sparsify_ms
+    ctxG.close()
+    out["wall_s"] = time.perf_counter() - t_all
+    return out
+
+
+def bench_hbm_roofline(torch, pkg, wl, dev, hbm_peak, peak_kind):
+    """The aggregation kernel where it is bound by HBM: the 1 M-node graph of the partitioned configuration, whose
+    512 MB BF16 source matrix does not fit the 126 MB L2 (mean aggregation, F = 256, forward and adjoint)."""
+    g = wl.chung_lu(1_000_000, 16.0, 2.1, seed=5)
+    ctx = pkg.Context(0)
+    ctx.load_graph(g.n, g.rowptr, g.col, None, wl.node_features(g.n, 8, 5))
+    F, es = 256, 2
+    H = torch.randn(g.n, F, device=dev).to(torch.bfloat16)
+    out = {"graph": "Chung-Lu, 1,000,000 nodes, mean degree 16", "entries": g.nnz, "width": F, "dtype": "bf16", "source_matrix_MB": g.n * F * es / 1e6,
+           "peak": hbm_peak, "peak_source": f"of {peak_kind}", "unit": "GB/s", "bound": "hbm"}
+    for name, transpose in (("forward", False), ("adjoint", True)):
+        for _ in range(3):
+            ctx.op_aggregate("sage", H, transpose=transpose)
+        torch.cuda.synchronize()
+        ev = []
+        for _ in range(20):
+            a, b = _events(torch)
+            a.record()
+            ctx.op_aggregate("sage", H, transpose=transpose)
+            b.record()
+            ev.append((a, b))
+        torch.cuda.synchronize()
+        us = 1e3 * statistics.median(a.elapsed_time(b) for a, b in ev)
+        per_entry = 4 + (4 if transpose else 0)
+        fixed = (g.n + 1) * 4 + g.n * F * es + (0 if transpose else g.n * 4)
+        gather = g.nnz * (F * es + per_entry) + fixed
+        compulsory = g.n * F * es + g.nnz * per_entry + fixed
+        out[name] = {"us_per_launch": us, "launches": 20, "gather_bytes": gather, "compulsory_bytes": compulsory,
+                     "achieved_gather": gather / us / 1e3, "frac_gather": gather / us / 1e3 / hbm_peak,
+                     "achieved_compulsory": compulsory / us / 1e3, "frac_compulsory": compulsory / us / 1e3 / hbm_peak}
+    ctx.close()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -149,10 +362,17 @@ def main():
     ap.add_argument("--cpu-baseline-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the HBM-bound roofline run and the other configurations")
     ap.add_argument("--cache-input-agg", action="store_true", help="reuse the weight-independent first-layer aggregation across steps (not the default, not the headline)")
     ap.add_argument("--predictor", default="dot", choices=["dot", "mlp"], help="mlp: the 3-layer MLP predictor of width 256 instead of the dot product (not the headline)")
     ap.add_argument("--breakdown", action="store_true", help="print a per-category time breakdown to stderr")
     args = ap.parse_args()
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        # started as a plain process: start one rank per GPU of this node and let rank 0 print the line
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1",
+               "--master-port", str(free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+        return subprocess.call(cmd)
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -188,14 +408,15 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (no CPU fall-back exists)")
-    if rank == 0:
-        lpbuild.build()
     dist = None
     if world > 1:
         import torch.distributed as dist
         torch.cuda.set_device(local_rank)
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
-        dist.barrier()
+    if rank == 0:
+        lpbuild.build()
+    if world > 1:
+        dist.barrier()  # no rank loads the library before rank 0 has (re)built it
     dev = f"cuda:{local_rank}"
     torch.cuda.set_device(local_rank)
 
@@ -288,17 +509,21 @@ def main():
     gather_minus_min = sum((g.nnz - g.n) * f * 2 for f in widths) / max(len(widths), 1)
     avg_launch_s = 1e-3 * agg_ms / max(agg_spans, 1)
     min_bytes = agg_bytes / max(agg_spans, 1) - gather_minus_min
-    roofline = {"bound": "hbm", "kernel": "spmm_padded_kernel (aggregation forward + adjoint)", "achieved": achieved, "peak": hbm_peak,
-                "unit": "GB/s", "frac": (achieved / hbm_peak) if achieved else None, "peak_source": f"of {peak_kind}",
+    fits_l2 = bool(g.n * max(widths) * 2 <= 126e6)
+    roofline = {"bound": "l2" if fits_l2 else "hbm",
+                "bound_note": ("the gathered source matrices (51-102 MB) stay in the 126 MB L2, so the launches are bound by L2 gathers, not by HBM: "
+                               "`achieved` (gather convention) may exceed the HBM peak; read dram_frac, t_bound_over_t and gather_ceiling, and "
+                               "hbm_roofline for the same kernel on an input that does not fit L2") if fits_l2 else "source matrix larger than L2",
+                "kernel": "spmm_padded_kernel (aggregation forward + adjoint)", "achieved": achieved, "peak": hbm_peak,
+                "unit": "GB/s", "frac": (achieved / hbm_peak) if achieved else None, "peak_source": f"of {peak_kind} (HBM copy bandwidth)",
                 "frac_of_nominal_8000": (achieved / 8000.0) if achieved else None, "traffic": traffic,
                 "dram_frac": (traffic / avg_launch_s / 1e9 / hbm_peak) if traffic and avg_launch_s > 0 else None,
                 "min_bytes_per_launch": min_bytes,
                 "t_bound_over_t": (min_bytes / (hbm_peak * 1e9) / avg_launch_s) if avg_launch_s > 0 else None,
-                "source_rows_fit_l2": bool(g.n * max(widths) * 2 <= 126e6),
+                "source_rows_fit_l2": fits_l2,
                 "launches_timed": agg_spans, "avg_launch_us": 1e3 * agg_ms / max(agg_spans, 1),
                 "bytes_per_launch": agg_bytes / max(agg_spans, 1), "share_of_step": agg_ms / elapsed_ms,
-                "note": "algorithmic bytes, gather convention (each stored entry reads one source row); activations of this workload "
-                        "partly fit the 126 MB L2, so the figure can exceed DRAM bandwidth"}
+                "note": "algorithmic bytes, gather convention (each stored entry reads one source row, nothing assumed cached)"}
 
     # ---- gather ceiling of the same launches (outside the timed region): the bare gather of the index streams the
     # three aggregation launches of a step walk (lp_op_gather_ceiling: no rows, arithmetic or epilogue).  With the source
@@ -327,7 +552,7 @@ def main():
                                           "note": "time of lp_op_gather_ceiling over the same index streams and row widths "
                                                   "divided by the aggregation time of a step"}
 
-    # ---- optional breakdown of a few more steps, outside the timed region
+    # ---- breakdown of a few more steps, outside the timed region
     breakdown = None
     if args.breakdown or rank == 0:
         ctx.profile_begin()
@@ -337,11 +562,12 @@ def main():
                 one_step(args.warmup + args.steps + i, args.warmup + args.steps + i + 1)
         bp = ctx.profile_end()
         breakdown = {k: {"us_per_step": 1e3 * d["ms"] / nbk, "GBps": (d["bytes"] / (d["ms"] * 1e-3) / 1e9) if d["ms"] > 0 else None,
+                         "frac_of_hbm_peak": (d["bytes"] / (d["ms"] * 1e-3) / 1e9 / hbm_peak) if d["ms"] > 0 else None,
                          "TFLOPs": (d["flops"] / (d["ms"] * 1e-3) / 1e12) if d["ms"] > 0 else None} for k, d in bp.items() if d["spans"]}
         if args.breakdown and rank == 0:
             print(json.dumps({"breakdown_per_step": breakdown}, indent=1), file=sys.stderr)
 
-    # ---- end to end through the host-buffer entry point: H2D of the batch, step, update, D2H of the loss
+    # ---- end to end: pinned host batch -> device, negatives, step, gradient average, update, loss -> host, every step
     e2e = None
     if not args.no_e2e:
         hu = torch.from_numpy(pos[0]).pin_memory()
@@ -349,12 +575,27 @@ def main():
         loss_h = torch.zeros(1).pin_memory()
         n_e2e = max(3, min(args.steps, 200))
         t_base = args.warmup + args.steps + 100
+        du_stage = torch.empty(B, dtype=torch.int32, device=dev)
+        dv_stage = torch.empty(B, dtype=torch.int32, device=dev)
 
         def host_step(i):
             b = batch_for(i, rank, world, nb)
             lo = b * B
-            ctx.train_step_host(p, hu[lo:lo + B], hv[lo:lo + B], K_NEG, seed=SEED, step=i, edge_index_base=lo, adam_m=m, adam_v=v,
-                                adam_t=i + 1, loss_host=loss_h)
+            if world == 1:  # the library's host-buffer entry point does all of it in one call
+                ctx.train_step_host(p, hu[lo:lo + B], hv[lo:lo + B], K_NEG, seed=SEED, step=i, edge_index_base=lo, adam_m=m, adam_v=v,
+                                    adam_t=i + 1, loss_host=loss_h)
+                return
+            # data parallel: the gradient average of Algorithm 1 sits between the step and the update
+            with torch.cuda.stream(stream):
+                du_stage.copy_(hu[lo:lo + B], non_blocking=True)
+                dv_stage.copy_(hv[lo:lo + B], non_blocking=True)
+                ctx._ck(lib.lp_sample_negatives(ctx.h, C.c_uint64(SEED), C.c_uint64(i), C.c_int32(K_NEG), C.c_int32(0), C.c_void_p(du_stage.data_ptr()),
+                                                C.c_int64(B), C.c_int64(lo), None, C.c_void_p(neg.data_ptr())))
+                ctx.train_step(p, du_stage, dv_stage, None, neg, K_NEG, loss, grads, seed=SEED, step=i)
+                scale = sync_gradients(grads, world, dist)
+                ctx.adam_step(p, m, v, grads, i + 1, grad_scale=scale)
+                loss_h.copy_(loss, non_blocking=True)
+            stream.synchronize()
 
         for i in range(3):
             host_step(t_base + i)
@@ -374,17 +615,27 @@ def main():
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             e2e_ms = float(t.item())
         e2e = {"value": n_e2e * edges_per_step / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 2 * B * 4, "d2h_bytes_per_step": 4,
-               "steps": n_e2e, "note": "lp_train_step_host: pinned host batch -> device, negatives, step, Adam, loss -> host; "
-                                       "single-GPU update (no gradient all-reduce inside this entry point)"}
+               "steps": n_e2e, "note": ("lp_train_step_host: pinned host batch -> device, negatives, step, Adam, loss -> host" if world == 1 else
+                                        "per rank: pinned host batch -> device, negatives, step, all-reduce of the gradient, Adam, loss -> host")}
+
+    # ---- the same kernel where HBM binds it, and the other configurations (rank 0, one GPU)
+    hbm_roofline = other = None
+    ctx.close()
+    if rank == 0 and world == 1 and not args.no_extras and args.scale == 1.0:
+        try:
+            hbm_roofline = bench_hbm_roofline(torch, pkg, wl, dev, hbm_peak, peak_kind)
+        except Exception as ex:
+            hbm_roofline = {"failed": str(ex)}
+        try:
+            other = bench_other_configs(torch, pkg, wl, dev)
+        except Exception as ex:
+            other = {"failed": str(ex)}
 
     # ---- CPU baseline: the oracle on the host cores, rank 0 at N = 1 only
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         try:
-            times = run_oracle_steps(g, X, params, dims, pos, B, args.cpu_baseline_steps, 0)
-            cpu = {"value": len(times) * B * (1 + K_NEG) / sum(times), "unit": UNIT, "cores": cpu_cores(), "kind": "oracle",
-                   "sample": f"{len(times)} full steps of the same workload (full-graph encoder, {B} positives + {B * K_NEG} negatives each)",
-                   "s_per_step": sum(times) / len(times)}
+            cpu = oracle_baseline(g, X, params, dims, pos, B, args.cpu_baseline_steps)
         except Exception as ex:  # the baseline must never take the GPU result down with it
             cpu = {"value": None, "unit": UNIT, "cores": cpu_cores(), "kind": "oracle", "sample": f"failed: {ex}"}
 
@@ -396,10 +647,9 @@ def main():
                            "model": "2-layer GraphSAGE-mean 128-256-256, " + ("3-layer MLP predictor (256)" if pred_hidden else "dot-product predictor"), "batch_pos": B, "neg_per_pos": K_NEG,
                            "scale": args.scale, "cache_input_aggregation": bool(args.cache_input_agg), "parallelism": f"dp{world}" if world > 1 else "single GPU",
                            "l2": "no flush: the step streams ~1 GB of activations per pass, several times the 126 MB L2"},
-                "clocks": clocks, "gpu_launches": int(launches), "loss_last": loss_value, "roofline": roofline, "cpu_baseline": cpu,
-                "e2e": e2e, "breakdown_us_per_step": breakdown}
+                "clocks": clocks, "gpu_launches": int(launches), "loss_last": loss_value, "roofline": roofline, "hbm_roofline": hbm_roofline,
+                "cpu_baseline": cpu, "e2e": e2e, "breakdown_us_per_step": breakdown, "configs": other}
         print(json.dumps(line))
-    ctx.close()
     if world > 1:
         dist.destroy_process_group()
     return 0
