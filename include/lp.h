@@ -249,11 +249,20 @@ lp_status lp_adam_step(lp_ctx *ctx, float *params, float *adam_m, float *adam_v,
 
 /* ---- inference, Eq. 2 ------------------------------------------------------------------- */
 
-/* scores[E] = <h_u^(K), h_v^(K)> for the E pairs (src, dst) after a full forward pass with
- * `params` (sampled models draw neighbours with seed/step as in lp_train_step).  Device
- * arrays.  Does not synchronise. */
+/* scores[E] = <h_u^(K), h_v^(K)> (or the MLP predictor's output) for the E pairs (src, dst) under the
+ * weights `params` (sampled models draw neighbours with seed/step as in lp_train_step).  Device
+ * arrays.  Does not synchronise.
+ * Full-graph models keep H^(K) between calls: an evaluation pass that scores validation positives and
+ * negatives in batches (Section IV) runs the encoder once.  The kept embeddings are used when the call
+ * passes the same `params` pointer as the forward pass that produced them (an lp_score or lp_train_step
+ * of this context) and no lp_adam_step / lp_train_step_host of this context has updated weights since.
+ * A caller that changes the weights behind that pointer by other means must call
+ * lp_invalidate_embeddings before scoring. */
 lp_status lp_score(lp_ctx *ctx, const float *params, const int32_t *src, const int32_t *dst, int64_t E,
                    uint64_t seed, uint64_t step, float *scores);
+
+/* Forget the embeddings kept for lp_score (see there).  Never fails on a valid context. */
+lp_status lp_invalidate_embeddings(lp_ctx *ctx);
 
 /* Hits@K (the accuracy metric of Section IV): the fraction of the n_pos positive scores that are
  * strictly greater than the K-th largest of the n_neg negative scores (1 when n_neg < K).  Scores are
@@ -287,6 +296,16 @@ lp_status lp_get_block(lp_ctx *ctx, int32_t hop, int32_t *frontier, int64_t *blk
  * given a node id outside [0, n), and LP_ETIMEOUT (once) when a bounded wait inside a
  * tensor-core kernel of an earlier call expired. */
 lp_status lp_get_stats(lp_ctx *ctx, lp_stats *out);
+
+/* (No counterpart in the paper: failure detection of the library itself.)
+ * Every device-side wait of the tensor-core kernels (on a shared-memory barrier that a bulk copy or a matrix
+ * instruction completes) is bounded: when it has lasted limit_ns the kernel records which wait gave up, releases
+ * its tensor memory and returns; the next synchronising call returns LP_ETIMEOUT once and the context stays
+ * usable.  limit_ns (default 2e9, allowed 1e3 .. 6e10) sets that bound for later launches of this context.
+ * overdeclare_bytes (normally 0; a multiple of 16, at most 65536) is a self-test of that path: the NEXT tensor-core
+ * launch announces that many bytes more than it copies on its first barrier, so every copy lands but the barrier
+ * never completes and the waits run into the limit.  Nothing faults and nothing is left running. */
+lp_status lp_set_wait_limit(lp_ctx *ctx, uint64_t limit_ns, int32_t overdeclare_bytes);
 
 /* ---- per-kernel timing (roofline measurement) ------------------------------------------------ */
 
@@ -364,7 +383,7 @@ lp_status lp_op_weight_grad(lp_ctx *ctx, int32_t prec, int64_t M, int32_t N, int
  *   device, cuda_stream : device index (made current by the call) and cudaStream_t (NULL = default)
  *   A[M, K], dZ[M, N], dW[K, N] : DEVICE float32, row-major, caller-owned; dW is overwritten
  * Limit: K * N <= 2^21 (2,097,152); larger requests return LP_EINVAL with a message available
- * from lp_last_error(NULL).  M is unbounded.
+ * from lp_last_error(NULL) (that message is kept per host thread).  M is unbounded.
  * The first call on each device looks up the device address of the fixed array; make that first
  * call before starting any stream capture.  All calls on a device share the array and it keeps
  * the previous call's contents (each call overwrites what it reads, so nothing needs clearing):

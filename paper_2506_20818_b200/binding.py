@@ -29,6 +29,7 @@ EXPORTS = [
     "lp_get_stats", "lp_op_aggregate", "lp_op_gather_ceiling", "lp_op_linear", "lp_op_weight_grad", "lp_profile_begin", "lp_profile_end",
     "lp_weight_grad_static", "lp_sparsify", "lp_get_sparsified",
     "lp_worker_view", "lp_get_worker_view", "lp_hits_at_k", "lp_get_predictor_activations",
+    "lp_invalidate_embeddings", "lp_set_wait_limit",
 ]
 
 PROF_CATEGORIES = ["agg_fwd", "agg_bwd", "gemm_fwd", "gemm_dgrad", "gemm_wgrad", "score", "incidence", "scatter",
@@ -240,6 +241,15 @@ class Context:
         self._ck(self.lib.lp_score(self.h, _ptr(params), _ptr(src), _ptr(dst), C.c_int64(src.numel()), C.c_uint64(seed), C.c_uint64(step),
                                    _ptr(out)))
         return out
+
+    def invalidate_embeddings(self):
+        """Tell the library that the weights changed outside its own calls (see lp_score)."""
+        self._ck(self.lib.lp_invalidate_embeddings(self.h))
+
+    def set_wait_limit(self, limit_ns: int, overdeclare_bytes: int = 0):
+        """Bound of the device-side waits of the tensor-core kernels; overdeclare_bytes > 0 makes the next such
+        launch run into that bound (self-test of the LP_ETIMEOUT path)."""
+        self._ck(self.lib.lp_set_wait_limit(self.h, C.c_uint64(limit_ns), C.c_int32(overdeclare_bytes)))
 
     def hits_at_k(self, pos_scores, neg_scores, k: int) -> float:
         """Hits@K of device score vectors (float32)."""

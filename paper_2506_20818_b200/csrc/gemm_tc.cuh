@@ -8,8 +8,8 @@
 // multicast) into a ring of shared-memory stages guarded by full/empty mbarriers; one elected
 // thread issues tcgen05.mma (kind::f16, BF16 x BF16 -> FP32) and releases stages with
 // tcgen05.commit; all four warps drain the accumulator with tcgen05.ld and apply the epilogue.
-// Every mbarrier wait is bounded: on expiry the kernel records an error word, frees its tensor
-// memory and returns, and the host reports LP_ETIMEOUT.
+// Every mbarrier wait is bounded (two seconds unless the host sets another limit): on expiry the kernel
+// records an error word, frees its tensor memory and returns, and the host reports LP_ETIMEOUT.
 #pragma once
 #include <cuda.h>
 
@@ -27,6 +27,8 @@ struct TcState {
     int *err_word = nullptr;  // device: 0 = fine, else code of the wait that expired
     bf16 *wbuf = nullptr;     // device scratch: BF16 copy of one layer's weights
     int *host_err = nullptr;  // pinned
+    unsigned long long wait_limit_ns = 2000000000ull;  // every mbarrier wait gives up after this long (default two seconds)
+    int overdeclare_tx = 0;   // diagnostics: the next launch expects this many bytes more than it copies (consumed by that launch)
 };
 
 constexpr int TC_BM = 128;          // accumulator rows (UMMA M)
@@ -35,7 +37,6 @@ constexpr int TC_UMMA_K = 16;       // K per tcgen05.mma for 16-bit operands
 constexpr int TC_THREADS = 128;
 constexpr int TC_COLSUM_BOXES = 4;  // 64-column boxes of the B tile one CTA may have to add up (BN <= 256)
 constexpr int TC_WBUF_ELEMS = 512 * 512;
-constexpr unsigned long long TC_WAIT_LIMIT_NS = 2000000000ull;  // every mbarrier wait gives up after two seconds
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -66,14 +67,14 @@ LP_DEVINL unsigned long long global_timer_ns()
     return t;
 }
 // bounded wait: false when the time limit was reached
-LP_DEVINL bool mbar_wait(uint32_t bar, uint32_t parity)
+LP_DEVINL bool mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
     for (;;) {
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (global_timer_ns() - t0 > TC_WAIT_LIMIT_NS) return false;
+        if (global_timer_ns() - t0 > limit_ns) return false;
     }
 }
 LP_DEVINL void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
@@ -193,6 +194,8 @@ struct TcGemmParams {
     int64_t rows;       // weight gradient: reduction length; rows_per_split rows per blockIdx.z
     int64_t rows_per_split;
     int *err;
+    unsigned long long wait_ns;  // limit of every mbarrier wait
+    int extra_tx;                // diagnostics: bytes added to the first stage's expected transfer so that its wait expires
 };
 
 template <bool MN_MAJOR>
@@ -256,14 +259,14 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
             // ---- producer: TMA loads into the stage ring
             for (int kb = 0; kb < num_kb; ++kb) {
                 const int s = kb % S;
-                if (kb >= S && !mbar_wait(smem_u32(&bar_empty[s]), ((kb / S) & 1) ^ 1)) {
+                if (kb >= S && !mbar_wait(smem_u32(&bar_empty[s]), ((kb / S) & 1) ^ 1, p.wait_ns)) {
                     atomicExch(p.err, 1);
                     abort_s = 1;
                     break;
                 }
                 const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes), sb = sa + a_bytes;
                 const uint32_t bar = smem_u32(&bar_full[s]);
-                mbar_expect_tx(bar, stage_bytes);
+                mbar_expect_tx(bar, stage_bytes + (kb == 0 ? (uint32_t)p.extra_tx : 0u));
                 const int kk = (int)(k_begin + (int64_t)kb * TC_BK);
                 if (!MN_MAJOR) {
                     tma_load_2d(sa, &mapA, bar, kk, m0);  // box {64 K, 128 rows}
@@ -280,7 +283,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
             bool ok = true;
             for (int kb = 0; kb < num_kb && ok; ++kb) {
                 const int s = kb % S;
-                if (!mbar_wait(smem_u32(&bar_full[s]), (kb / S) & 1)) {
+                if (!mbar_wait(smem_u32(&bar_full[s]), (kb / S) & 1, p.wait_ns)) {
                     atomicExch(p.err, 2);
                     abort_s = 1;
                     ok = false;
@@ -323,7 +326,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
             bool ok = true;
             for (int kb = 0; kb < num_kb; ++kb) {
                 const int s = kb % S;
-                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_full[s]), (kb / S) & 1));
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_full[s]), (kb / S) & 1, p.wait_ns));
                 if (!ok) {
                     if (lane == 0) atomicExch(p.err, 4);
                     abort_s = 1;
@@ -373,7 +376,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
         __syncwarp();
 
         // ---- epilogue: all four warps
-        bool ready = mbar_wait(smem_u32(&bar_acc), 0);
+        bool ready = mbar_wait(smem_u32(&bar_acc), 0, p.wait_ns);
         if (!ready && lane == 0) atomicExch(p.err, 3);
         ready = ready && (*(volatile int *)&abort_s == 0);
         ready = __all_sync(0xffffffffu, ready);
@@ -531,25 +534,25 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
                 const int m0 = (int)((first_tile + i * stride) * TC_BM);
                 for (int kb = 0; kb < KB; ++kb, ++it) {
                     const int s = (int)(it % S);
-                    if (it >= S && !mbar_wait(smem_u32(&bar_empty[s]), (uint32_t)(((it / S) & 1) ^ 1))) {
+                    if (it >= S && !mbar_wait(smem_u32(&bar_empty[s]), (uint32_t)(((it / S) & 1) ^ 1), p.wait_ns)) {
                         atomicExch(p.err, 1);
                         *abort_flag = 1;
                         break;
                     }
                     const uint32_t bar = smem_u32(&bar_full[s]);
-                    mbar_expect_tx(bar, a_bytes);
+                    mbar_expect_tx(bar, a_bytes + (it == 0 ? (uint32_t)p.extra_tx : 0u));
                     tma_load_2d(smem_u32(smem_a + (size_t)s * a_bytes), &mapA, bar, kb * TC_BK, m0);
                 }
             }
         } else if (warp == 1 && lane == 0) {
             // ---- MMA issuer
             const uint32_t idesc = make_idesc_bf16(BN, false, false);
-            bool ok = mbar_wait(smem_u32(&bar_w), 0);
+            bool ok = mbar_wait(smem_u32(&bar_w), 0, p.wait_ns);
             if (!ok) { atomicExch(p.err, 4); *abort_flag = 1; }
             int64_t it = 0;
             for (int64_t i = 0; i < my_tiles && ok; ++i) {
                 const int b = (int)(i & 1);
-                if (i >= 2 && !mbar_wait(smem_u32(&bar_acc_empty[b]), (uint32_t)((((i >> 1) - 1) & 1)))) {
+                if (i >= 2 && !mbar_wait(smem_u32(&bar_acc_empty[b]), (uint32_t)((((i >> 1) - 1) & 1)), p.wait_ns)) {
                     atomicExch(p.err, 5);
                     *abort_flag = 1;
                     break;
@@ -558,7 +561,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
                 const uint32_t tmem_d = tmem_base + (uint32_t)(b * BN);
                 for (int kb = 0; kb < KB; ++kb, ++it) {
                     const int s = (int)(it % S);
-                    if (!mbar_wait(smem_u32(&bar_full[s]), (uint32_t)((it / S) & 1))) {
+                    if (!mbar_wait(smem_u32(&bar_full[s]), (uint32_t)((it / S) & 1), p.wait_ns)) {
                         atomicExch(p.err, 2);
                         *abort_flag = 1;
                         ok = false;
@@ -581,7 +584,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
             const int my_box = (warp - 2) >> 2;
             for (int64_t i = 0; i < my_tiles; ++i) {
                 const int b = (int)(i & 1);
-                bool ready = mbar_wait(smem_u32(&bar_acc_full[b]), (uint32_t)((i >> 1) & 1));
+                bool ready = mbar_wait(smem_u32(&bar_acc_full[b]), (uint32_t)((i >> 1) & 1), p.wait_ns);
                 if (!ready && lane == 0) { atomicExch(p.err, 3); *abort_flag = 1; }
                 if (!__all_sync(0xffffffffu, ready) && lane == 0) *abort_flag = 1;
                 epilogue_barrier();             // the eight warps take the same decision: all continue or all leave
@@ -779,6 +782,7 @@ static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const
         p.stages = (int)std::max<int64_t>(4, std::min<int64_t>(TCP_MAX_STAGES, (smem_cap - w_bytes - TCP_STAGE_OUT_BYTES) / (TC_BM * TC_BK * 2)));
         p.bias = bias; p.relu = relu ? 1 : 0; p.C = C; p.ldc = ldc; p.out_f32 = nullptr; p.err = tc.err_word;
         p.row_scale = row_scale; p.scale_col0 = scale_col0;
+        p.wait_ns = tc.wait_limit_ns; p.extra_tx = tc.overdeclare_tx; tc.overdeclare_tx = 0;
         const int n_slices = N / pbn;
         const int64_t m_tiles = ceil_div64(M, TC_BM);
         int64_t ctas = std::min<int64_t>((int64_t)tc_sm_count(), m_tiles * n_slices);
@@ -797,6 +801,7 @@ static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const
     p.stages = tc_stages(BN, K / TC_BK);
     p.bias = bias; p.relu = relu ? 1 : 0; p.C = C; p.ldc = ldc; p.out_f32 = nullptr; p.rows = 0; p.rows_per_split = 0; p.err = tc.err_word;
     p.row_scale = row_scale; p.scale_col0 = scale_col0;
+    p.wait_ns = tc.wait_limit_ns; p.extra_tx = tc.overdeclare_tx; tc.overdeclare_tx = 0;
     const size_t smem = (size_t)p.stages * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024;
     dim3 grid((unsigned)ceil_div64(M, TC_BM), (unsigned)(N / BN), 1);
     tc_gemm_kernel<false><<<grid, TC_THREADS, smem, ex.st>>>(mapA, mapB, p);
@@ -871,6 +876,7 @@ static bool tc_weight_grad(TcState &tc, Exec &ex, int64_t rows, int Kin, int N, 
     p.stages = tc_stages(BN, (int)(p.rows_per_split / TC_BK));
     p.bias = nullptr; p.relu = 0; p.C = nullptr; p.ldc = 0; p.out_f32 = partials; p.err = tc.err_word;
     p.colsum = fuse_bias ? 1 : 0;
+    p.wait_ns = tc.wait_limit_ns; p.extra_tx = tc.overdeclare_tx; tc.overdeclare_tx = 0;
     const size_t smem = (size_t)p.stages * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024;
     dim3 grid((unsigned)(Kin / TC_BM), (unsigned)(N / BN), (unsigned)splits);
     tc_gemm_kernel<true><<<grid, TC_THREADS, smem, ex.st>>>(mapA, mapB, p);

@@ -2,6 +2,7 @@
 // orchestration of the kernels.  See include/lp.h for the contract of every entry point.
 #include <algorithm>
 #include <cmath>
+#include <memory>
 #include <new>
 
 #include "common.cuh"
@@ -72,7 +73,7 @@ struct lp_ctx {
     float *inv_deg = nullptr, *meanT_val = nullptr;
     float *X32 = nullptr;
     bf16 *X16 = nullptr;
-    int *cand = nullptr;
+    int *cand = nullptr;         // candidate set of the negative sampler (own allocation, replaced by every lp_set_candidates)
     int64_t n_cand = 0;
     unsigned long long *exhausted_dev = nullptr;
     HeavyPlan plan_csr, plan_csc, plan_dyn;  // heavy-row plans: the loaded graph, its transpose, per-step structures
@@ -118,11 +119,16 @@ struct lp_ctx {
     int rows_out = 0;                   // rows of H^(K) in the last forward
     bool have_forward = false, have_grad = false;
     bool input_agg_valid = false;       // cached AGG(X) of layer 1 is present (cache_input_aggregation)
+    // H^(K) of the last full-graph forward pass stays valid for lp_score while the same parameter vector is passed and no
+    // call of this library has changed it (param_version counts such calls)
+    bool hk_valid = false;
+    const float *hk_params = nullptr;
+    uint64_t hk_version = 0, param_version = 0;
     int64_t last_exhausted = 0;
     TcState tc;                         // tensor-core GEMM state (descriptor encoder, device error word)
 };
 
-static std::string g_create_error;
+static thread_local std::string g_create_error;  // errors of calls that have no context: one per host thread
 
 static lp_status fail(lp_ctx *c, lp_status st, const std::string &msg)
 {
@@ -164,6 +170,13 @@ static void free_list(std::vector<void *> &l)
     for (void *p : l) cudaFree(p);
     l.clear();
 }
+
+// temporaries of one call: released on every way out of it
+struct TempAllocs {
+    std::vector<void *> list;
+    int64_t bytes = 0;
+    ~TempAllocs() { free_list(list); }
+};
 
 static inline unsigned nblk(int64_t n, int t = 256) { return (unsigned)std::max<int64_t>(1, ceil_div64(n, t)); }
 
@@ -301,6 +314,7 @@ static void drop_model(lp_ctx *ctx)
     ctx->model_set = false;
     ctx->have_forward = ctx->have_grad = false;
     ctx->input_agg_valid = false;
+    ctx->hk_valid = false;
     for (auto &l : ctx->layer) l = LayerBuf();
     for (auto &h : ctx->hop) h = HopBlock();
 }
@@ -332,9 +346,10 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
     const cudaMemcpyKind kind = ptrs_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
 
     int64_t *rowptr64 = nullptr;
-    std::vector<void *> tmp;
-    int64_t tmp_bytes = 0;
-#define TALLOC(ptr, count) do { cudaError_t e__ = dev_alloc(ctx, tmp, tmp_bytes, &(ptr), (count)); if (e__ != cudaSuccess) { free_list(tmp); CK(e__); } } while (0)
+    TempAllocs tmp_guard;
+    std::vector<void *> &tmp = tmp_guard.list;
+    int64_t &tmp_bytes = tmp_guard.bytes;
+#define TALLOC(ptr, count) CK(dev_alloc(ctx, tmp, tmp_bytes, &(ptr), (count)))
     TALLOC(rowptr64, n + 1);
     GALLOC(ctx->rowptr, n + 1);
     GALLOC(ctx->col, nnz);
@@ -345,16 +360,15 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
     if (e == cudaSuccess && nnz > 0) e = cudaMemcpyAsync(ctx->col, col, sizeof(int) * (size_t)nnz, kind, st);
     if (e == cudaSuccess && w && nnz > 0) e = cudaMemcpyAsync(ctx->w, w, sizeof(float) * (size_t)nnz, kind, st);
     if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->X32, X, sizeof(float) * (size_t)n * f, kind, st);
-    if (e != cudaSuccess) { free_list(tmp); CK(e); }
+    CK(e);
 
     cudaMemsetAsync(ctx->err_flag, 0, sizeof(int), st);
     validate_csr_kernel<<<nblk(n + 1), 256, 0, st>>>(rowptr64, (int)n, nnz, ctx->col, ctx->rowptr, ctx->err_flag);
     int flag = 0;
     e = cudaMemcpyAsync(&flag, ctx->err_flag, sizeof(int), cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-    if (e != cudaSuccess) { free_list(tmp); CK(e); }
+    CK(e);
     if (flag) {
-        free_list(tmp);
         free_list(ctx->graph_allocs);
         char buf[160];
         snprintf(buf, sizeof buf, "lp_load_graph: malformed CSR (flags %d: 1/2 rowptr ends, 4 rowptr order, 8 column range, 16 columns not strictly ascending)", flag);
@@ -470,7 +484,6 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
         hp->p_counts = pp.counts;
         hp->p_host_rows = ctx->host_counts[10];
     }
-    free_list(tmp);
 #undef TALLOC
     CK(e);
     CK_LAUNCH();
@@ -501,7 +514,15 @@ extern "C" lp_status lp_set_candidates(lp_ctx *ctx, const int32_t *cand, int64_t
     if (!ctx) return LP_EINVAL;
     if (!ctx->loaded) return fail(ctx, LP_ESTATE, "lp_set_candidates: no graph loaded");
     CK(cudaSetDevice(ctx->device));
-    if (!cand || n_cand <= 0) { ctx->cand = nullptr; ctx->n_cand = 0; return LP_OK; }
+    CK(cudaStreamSynchronize(ctx->ex.st));  // earlier sampling launches may still read the previous set
+    if (ctx->cand) {                        // the previous set is released: repeated calls do not grow the context
+        auto it = std::find(ctx->graph_allocs.begin(), ctx->graph_allocs.end(), (void *)ctx->cand);
+        if (it != ctx->graph_allocs.end()) ctx->graph_allocs.erase(it);
+        cudaFree(ctx->cand);
+        ctx->cand = nullptr;
+        ctx->n_cand = 0;
+    }
+    if (!cand || n_cand <= 0) return LP_OK;
     if (n_cand >= (int64_t)1 << 31) return fail(ctx, LP_EINVAL, "lp_set_candidates: too many candidates");
     GALLOC(ctx->cand, n_cand);  // lives with the graph
     CK(cudaMemcpyAsync(ctx->cand, cand, sizeof(int) * (size_t)n_cand, cudaMemcpyDeviceToDevice, ctx->ex.st));
@@ -511,6 +532,8 @@ extern "C" lp_status lp_set_candidates(lp_ctx *ctx, const int32_t *cand, int64_t
     CK(cudaStreamSynchronize(ctx->ex.st));
     if (bad) {
         cudaMemsetAsync(ctx->err_flag, 0, sizeof(int), ctx->ex.st);
+        ctx->graph_allocs.erase(std::find(ctx->graph_allocs.begin(), ctx->graph_allocs.end(), (void *)ctx->cand));
+        cudaFree(ctx->cand);
         ctx->cand = nullptr;
         return fail(ctx, LP_EINVAL, "lp_set_candidates: candidate id outside [0, n)");
     }
@@ -1189,6 +1212,9 @@ template <typename T> static lp_status forward_impl(lp_ctx *ctx, const float *pa
     }
     ctx->rows_out = ctx->sampled ? ctx->hop[0].n_src : n;
     ctx->have_forward = true;
+    ctx->hk_valid = !ctx->sampled;
+    ctx->hk_params = params;
+    ctx->hk_version = ctx->param_version;
     CK_LAUNCH();
     return LP_OK;
 }
@@ -1275,7 +1301,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     T *HK = tptr<T>(ctx->HK);
 
     // scores, loss, per-edge gradients
-    ProfScope *pscore = new ProfScope(ctx->ex, LP_PROF_SCORE, (double)B * (2.0 + k) * D * sizeof(T) + (double)E * 12.0, 2.0 * E * D);
+    std::unique_ptr<ProfScope> pscore(new ProfScope(ctx->ex, LP_PROF_SCORE, (double)B * (2.0 + k) * D * sizeof(T) + (double)E * 12.0, 2.0 * E * D));
     const unsigned eblocks = nblk(B, EDGE_THREADS / 32);
     constexpr int VN = Vec16<T>::N;
     const int chunks = D / VN;
@@ -1284,13 +1310,13 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     CK(cudaMemsetAsync(ctx->inc_ptr, 0, sizeof(int) * ((size_t)rows_out + 1), st));
     if (ctx->mlp) {
         s = predictor_forward<T>(ctx, params, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k);
-        if (s != LP_OK) { delete pscore; return s; }
+        if (s != LP_OK) return s;
         const unsigned lblocks = nblk(E, 256);
         bce_from_scores_kernel<<<lblocks, 256, 0, st>>>(ctx->pred_scores, E, B, inv_N, ctx->g_pos, ctx->loss_partials);
         loss_reduce_kernel<<<1, 1024, 0, st>>>(ctx->loss_partials, lblocks, inv_N, loss);
         g_neg = ctx->g_pos + B;  // one array: positives, then negatives
         s = predictor_backward<T>(ctx, params, E, ctx->g_pos, grads, accumulate);
-        if (s != LP_OK) { delete pscore; return s; }
+        if (s != LP_OK) return s;
     } else {
         unsigned lparts = eblocks;  // loss partials written
         if (chunks <= 32 && k == 1 && !neg_src) {
@@ -1301,18 +1327,18 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         else edge_score_bce_kernel<T, 4><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials, ctx->inc_ptr);
         loss_reduce_kernel<<<1, 1024, 0, st>>>(ctx->loss_partials, lparts, inv_N, loss);
     }
-    delete pscore;
+    pscore.reset();
     ctx->ex.launches += 2;
 
     // incidence lists of the scored edges, grouped by node (slots claimed with integer atomics)
-    ProfScope *pinc = new ProfScope(ctx->ex, LP_PROF_INCIDENCE, (double)E * 2.0 * 24.0);
+    std::unique_ptr<ProfScope> pinc(new ProfScope(ctx->ex, LP_PROF_INCIDENCE, (double)E * 2.0 * 24.0));
     if (ctx->mlp) incidence_count_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->inc_ptr);
     exclusive_scan_i32(ctx->ex, ctx->inc_ptr, rows_out, ctx->inc_ptr, ctx->inc_ptr + rows_out, ctx->scan_tmp);
     CK(cudaMemcpyAsync(ctx->inc_cursor, ctx->inc_ptr, sizeof(int) * (size_t)rows_out, cudaMemcpyDeviceToDevice, st));
     incidence_fill_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, g_pos, g_neg, ctx->inc_cursor, ctx->inc_col,
                                                    ctx->mlp ? nullptr : ctx->inc_val, ctx->mlp ? ctx->inc_edge : nullptr);
     ctx->ex.launches += 2;
-    delete pinc;
+    pinc.reset();
 
     // dL/dH^(K)[v] = sum over incident scored edges of g_e * h_other
     T *dZ = tptr<T>(ctx->dHK);
@@ -1467,6 +1493,7 @@ extern "C" lp_status lp_adam_step(lp_ctx *ctx, float *params, float *adam_m, flo
     if (adam_m && t < 1) return fail(ctx, LP_EINVAL, "lp_adam_step: t counts from 1");
     CK(cudaSetDevice(ctx->device));
     const int64_t np = ctx->n_params;
+    ctx->param_version += 1;  // embeddings kept for lp_score belong to the old weights
     ProfScope prof(ctx->ex, LP_PROF_ADAM, (double)np * (adam_m ? 28.0 : 12.0));
     if (adam_m) {
         const double c1 = 1.0 - std::pow(beta1, (double)t), c2 = 1.0 - std::pow(beta2, (double)t);
@@ -1522,7 +1549,10 @@ static lp_status score_impl(lp_ctx *ctx, const float *params, const int *src, co
         lp_status s = build_blocks(ctx, src, dst, E, nullptr, nullptr, 0, seed, step);
         if (s != LP_OK) return s;
     }
-    lp_status s = forward_impl<T>(ctx, params);
+    // full-graph models: H^(K) of the last forward pass is reused while the caller passes the same parameter vector and no
+    // call of this library has updated it since
+    lp_status s = LP_OK;
+    if (!(ctx->hk_valid && ctx->hk_params == params && ctx->hk_version == ctx->param_version)) s = forward_impl<T>(ctx, params);
     if (s != LP_OK) return s;
     const int D = ctx->desc.dims[ctx->K];
     const int *idmap = ctx->sampled ? ctx->hop[0].posmap : nullptr;
@@ -1560,6 +1590,24 @@ extern "C" lp_status lp_score(lp_ctx *ctx, const float *params, const int32_t *s
                                             : score_impl<float>(ctx, params, src, dst, E, seed, step, scores);
     if (s != LP_OK) return s;
     return tc_check(ctx->tc, ctx->ex, false, ctx->err);
+}
+
+extern "C" lp_status lp_invalidate_embeddings(lp_ctx *ctx)
+{
+    if (!ctx) return LP_EINVAL;
+    ctx->hk_valid = false;
+    return LP_OK;
+}
+
+extern "C" lp_status lp_set_wait_limit(lp_ctx *ctx, uint64_t limit_ns, int32_t overdeclare_bytes)
+{
+    if (!ctx) return LP_EINVAL;
+    if (limit_ns < 1000 || limit_ns > 60000000000ull) return fail(ctx, LP_EINVAL, "lp_set_wait_limit: limit must be between 1 us and 60 s");
+    if (overdeclare_bytes < 0 || overdeclare_bytes > 65536 || overdeclare_bytes % 16 != 0)
+        return fail(ctx, LP_EINVAL, "lp_set_wait_limit: overdeclare_bytes must be a multiple of 16 in [0, 65536]");
+    ctx->tc.wait_limit_ns = limit_ns;
+    ctx->tc.overdeclare_tx = overdeclare_bytes;
+    return LP_OK;
 }
 
 extern "C" lp_status lp_hits_at_k(lp_ctx *ctx, const float *pos_scores, int64_t n_pos, const float *neg_scores, int64_t n_neg, int64_t K, double *hits)

@@ -567,6 +567,81 @@ def test_score(pkg, arch, prec):
     ctx.close()
 
 
+def test_score_keeps_embeddings_between_calls(pkg):
+    # an evaluation pass scores positives and negatives in batches (Section IV): the encoder runs once, later calls
+    # with the same weights only score; an update of the weights (or an explicit invalidation) runs it again
+    g = wl.chung_lu(5000, 10.0, 2.1, seed=3)
+    dims = [64, 128, 64]
+    X = wl.node_features(g.n, 64, 3)
+    params = wl.glorot_params("sage", dims, 3, 0.05)
+    ctx = make_ctx(pkg, g, X)
+    ctx.set_model("sage", dims, prec="fp32", max_batch=1024)
+    u, v = wl.undirected_edge_list(g)
+    du, dv, p = t32(u), t32(v), t32(params)
+    half = len(u) // 2
+    n0 = ctx.stats().kernel_launches
+    s_a = ctx.score(p, du[:half].contiguous(), dv[:half].contiguous())
+    n1 = ctx.stats().kernel_launches
+    s_b = ctx.score(p, du[half:].contiguous(), dv[half:].contiguous())
+    n2 = ctx.stats().kernel_launches
+    assert n1 - n0 > 3 and n2 - n1 == 1  # encoder + scoring, then scoring alone
+    ref = oracle.score(g, X, params, "sage", dims, u, v)
+    assert rel_l2(torch.cat([s_a, s_b]).cpu().numpy(), ref) < TOL["fp32"]
+    # another parameter vector, an optimiser step, an explicit invalidation: each runs the encoder again
+    p2 = p.clone()
+    ctx.score(p2, du, dv)
+    n3 = ctx.stats().kernel_launches
+    assert n3 - n2 == n1 - n0
+    m, vv, grads = torch.zeros_like(p2), torch.zeros_like(p2), torch.ones_like(p2)
+    ctx.adam_step(p2, m, vv, grads, 1)
+    n4 = ctx.stats().kernel_launches
+    s_new = ctx.score(p2, du, dv)
+    n5 = ctx.stats().kernel_launches
+    assert n5 - n4 == n1 - n0
+    assert rel_l2(s_new.cpu().numpy(), oracle.score(g, X, p2.cpu().numpy(), "sage", dims, u, v)) < TOL["fp32"]
+    p2.mul_(0.5)  # weights changed behind the library's back: the caller says so
+    ctx.invalidate_embeddings()
+    s_half = ctx.score(p2, du, dv)
+    assert ctx.stats().kernel_launches - n5 == n1 - n0
+    assert rel_l2(s_half.cpu().numpy(), oracle.score(g, X, p2.cpu().numpy(), "sage", dims, u, v)) < TOL["fp32"]
+    # a training step leaves the embeddings of its weights behind as well
+    ctx.set_model("sage", dims, prec="fp32", max_batch=len(u), max_k=1)
+    _, nd = ctx.sample_negatives(1, 0, 1, du)
+    loss, grads = torch.zeros(1, device=DEV), torch.zeros(ctx.n_params, device=DEV)
+    ctx.train_step(p, du, dv, None, nd, 1, loss, grads)
+    n6 = ctx.stats().kernel_launches
+    s_c = ctx.score(p, du, dv)
+    assert ctx.stats().kernel_launches - n6 == 1
+    assert rel_l2(s_c.cpu().numpy(), ref) < TOL["fp32"]
+    ctx.close()
+
+
+@pytest.mark.parametrize("M", [100, 4096])
+def test_bounded_wait_expires_cleanly(pkg, M):
+    # failure detection of the tensor-core kernels, exercised without any fault: the next launch is told to expect 16
+    # bytes more than its copies deliver, so every copy lands but the barrier never completes; with the limit at 2 ms
+    # every wait gives up, the kernel frees its tensor memory and returns, the call reports LP_ETIMEOUT once, and the
+    # context (tensor memory included) works as before.  M = 100 takes the one-tile kernel, M = 4096 the persistent one.
+    g = wl.erdos_renyi(50, 100, seed=0)
+    ctx = make_ctx(pkg, g, wl.node_features(g.n, 8, 0))
+    rng = np.random.default_rng(M)
+    A = torch.from_numpy(rng.standard_normal((M, 256)).astype(np.float32)).to(DEV).to(torch.bfloat16)
+    W = torch.from_numpy((rng.standard_normal((256, 128)) / 16).astype(np.float32)).to(DEV).to(torch.bfloat16)
+    ref = A.float().cpu().numpy().astype(np.float64) @ W.float().cpu().numpy().astype(np.float64)
+    assert rel_l2(ctx.op_linear(A, W).float().cpu().numpy(), ref) < 4e-3
+    ctx.set_wait_limit(2_000_000, overdeclare_bytes=16)
+    with pytest.raises(pkg.LpError) as ei:
+        ctx.op_linear(A, W)
+    assert ei.value.status == -6 and "wait" in str(ei.value)
+    ctx.stats()  # reported once
+    for _ in range(3):  # the self-test was consumed by that launch; tensor memory was released (these launches need all of it again)
+        assert rel_l2(ctx.op_linear(A, W).float().cpu().numpy(), ref) < 4e-3
+    ctx.set_wait_limit(2_000_000_000)
+    with pytest.raises(pkg.LpError):
+        ctx.set_wait_limit(10)
+    ctx.close()
+
+
 # ------------------------------------------------------------------------------------------ emulated workers (config 5)
 def test_config5_partitions_local_vs_global(pkg):
     g, X, params, pos, cfg = wl.make_config("c5_partitioned_sage2", scale=0.01)

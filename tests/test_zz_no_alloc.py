@@ -46,10 +46,36 @@ def test_static_weight_grad_matches_ordinary_entry_twice(pkg):
         assert rel_l2(got.cpu().numpy(), want.cpu().numpy()) < 1e-5  # FP32-path tolerance of the parity tests
         exact = A.double().T @ dZ.double()
         assert rel_l2(got.double().cpu().numpy(), exact.cpu().numpy()) < 1e-5
-    # same inputs again: the result is reproducible bit for bit
-    again = pkg.weight_grad_static(A, dZ)
+    # same inputs again: the result is reproducible bit for bit, and the call takes no device memory: the free
+    # memory of the device is the same before and after it (the output tensor is allocated beforehand)
+    import ctypes as C
+    lib = pkg.load_library()
+    again = torch.empty_like(got)
     torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    rc = lib.lp_weight_grad_static(C.c_int32(0), C.c_void_p(torch.cuda.current_stream().cuda_stream), C.c_int64(A.shape[0]), C.c_int32(dZ.shape[1]),
+                                   C.c_int32(A.shape[1]), C.c_void_p(A.data_ptr()), C.c_void_p(dZ.data_ptr()), C.c_void_p(again.data_ptr()))
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert rc == 0 and free_after == free_before
     assert torch.equal(again, got)
+    ctx.close()
+
+
+def test_static_weight_grad_at_the_size_limit(pkg):
+    # K * N = 2^21 exactly: the fixed array holds one partial tile, so the rows are not split at all
+    import workloads as wl
+    g = wl.erdos_renyi(50, 100, seed=0)
+    ctx = pkg.Context(0)
+    ctx.load_graph(g.n, g.rowptr, g.col, None, wl.node_features(g.n, 8, 0))
+    rng = np.random.default_rng(6)
+    A = torch.from_numpy(rng.standard_normal((37, 2048)).astype(np.float32)).to(DEV)
+    dZ = torch.from_numpy(rng.standard_normal((37, 1024)).astype(np.float32)).to(DEV)
+    for _ in range(2):
+        got = pkg.weight_grad_static(A, dZ)
+        torch.cuda.synchronize()
+        assert rel_l2(got.double().cpu().numpy(), (A.double().T @ dZ.double()).cpu().numpy()) < 1e-5
+    assert rel_l2(got.cpu().numpy(), ctx.op_weight_grad(A, dZ).cpu().numpy()) < 1e-5
     ctx.close()
 
 
