@@ -68,3 +68,28 @@ template <> LP_DEVINL float to_f<bf16>(bf16 x) { return __bfloat162float(x); }
 template <typename T> LP_DEVINL T from_f(float x);
 template <> LP_DEVINL float from_f<float>(float x) { return x; }
 template <> LP_DEVINL bf16 from_f<bf16>(float x) { return __float2bfloat16_rn(x); }
+
+// acc += <a, b> over one 16-byte vector, elements in storage order (one FMA each).  BF16 operands go through the
+// mixed-precision FMA of sm_100 (fma.rn.f32.bf16: both factors widened exactly, one rounding), which gives the
+// same bits as convert-then-fmaf without the conversion instructions.
+template <typename T> LP_DEVINL float dot_vec(const Vec16<T> &a, const Vec16<T> &b, float acc)
+{
+    constexpr int VN = Vec16<T>::N;
+    float fa[VN], fb[VN];
+    a.to_float(fa);
+    b.to_float(fb);
+#pragma unroll
+    for (int t = 0; t < VN; ++t) acc = fmaf(fa[t], fb[t], acc);
+    return acc;
+}
+template <> LP_DEVINL float dot_vec<bf16>(const Vec16<bf16> &a, const Vec16<bf16> &b, float acc)
+{
+    const uint32_t x[4] = {a.v.x, a.v.y, a.v.z, a.v.w}, y[4] = {b.v.x, b.v.y, b.v.z, b.v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        asm("{\n\t.reg .b16 alo, ahi, blo, bhi;\n\tmov.b32 {alo, ahi}, %1;\n\tmov.b32 {blo, bhi}, %2;\n\t"
+            "fma.rn.f32.bf16 %0, alo, blo, %0;\n\tfma.rn.f32.bf16 %0, ahi, bhi, %0;\n\t}"
+            : "+f"(acc)
+            : "r"(x[i]), "r"(y[i]));
+    return acc;
+}

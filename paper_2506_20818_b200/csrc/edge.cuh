@@ -205,16 +205,10 @@ edge_score_bce_pair_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, c
         }
 #pragma unroll
         for (int p = 0; p < P; ++p) {
-            float fu[VN], fv[VN], fn[VN];
-            ru[p].to_float(fu);
-            rv[p].to_float(fv);
-            rn[p].to_float(fn);
             float dp = 0.f, dn = 0.f;
             if (active) {
-#pragma unroll
-                for (int t = 0; t < VN; ++t) dp = fmaf(fu[t], fv[t], dp);
-#pragma unroll
-                for (int t = 0; t < VN; ++t) dn = fmaf(fu[t], fn[t], dn);
+                dp = dot_vec<T>(ru[p], rv[p], 0.f);
+                dn = dot_vec<T>(ru[p], rn[p], 0.f);
             }
             dp = warp_sum(dp);
             dn = warp_sum(dn);
@@ -283,11 +277,7 @@ edge_score_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const int 
             Vec16<T> a, b;
             a.load(H + (size_t)u * ldh + ch * VN);
             b.load(H + (size_t)v * ldh + ch * VN);
-            float fa[VN], fb[VN];
-            a.to_float(fa);
-            b.to_float(fb);
-#pragma unroll
-            for (int t = 0; t < VN; ++t) dot = fmaf(fa[t], fb[t], dot);
+            dot = dot_vec<T>(a, b, dot);
         }
     }
     dot = warp_sum(dot);
@@ -326,20 +316,35 @@ __global__ void incidence_count_kernel(int n_ids, const int *__restrict__ idmap,
     atomicAdd(&counts[d], 1);
 }
 
-// cursor[v] starts at the offset of node v's list and is advanced by every claim
+// cursor[v] starts at the offset of node v's list and is advanced by every claim.  The lanes of a warp that claim
+// slots of the same node (batches often hold runs of positives with a common source) make one claim together: the
+// lowest of them adds their number to the cursor and every lane takes its rank inside the claimed run.
+LP_DEVINL int claim_slot(int *cursor, int node, unsigned active, int lane)
+{
+    const unsigned peers = __match_any_sync(active, node);
+    const int leader = __ffs(peers) - 1;
+    int base = 0;
+    if (lane == leader) base = atomicAdd(&cursor[node], __popc(peers));
+    base = __shfl_sync(peers, base, leader);
+    return base + __popc(peers & ((1u << lane) - 1u));
+}
+
 __global__ void incidence_fill_kernel(int n_ids, const int *__restrict__ idmap, const int *__restrict__ pos_src, const int *__restrict__ pos_dst,
                                       int64_t B, const int *__restrict__ neg_src, const int *__restrict__ neg_dst, int k,
                                       const float *__restrict__ g_pos, const float *__restrict__ g_neg, int *__restrict__ cursor,
                                       int *__restrict__ inc_col, float *__restrict__ inc_val, int *__restrict__ inc_edge)
 {
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= B * (1 + k)) return;
+    const bool valid = e < B * (1 + k);
+    const unsigned active = __ballot_sync(0xffffffffu, valid);
+    if (!valid) return;
+    const int lane = threadIdx.x & 31;
     int s, d;
     incidence_endpoints(n_ids, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, e, s, d);
     const float g = g_pos ? (e < B ? g_pos[e] : g_neg[e - B]) : 0.f;
-    const int ps = atomicAdd(&cursor[s], 1);
+    const int ps = claim_slot(cursor, s, active, lane);
     inc_col[ps] = d;
-    const int pd = atomicAdd(&cursor[d], 1);
+    const int pd = claim_slot(cursor, d, active, lane);
     inc_col[pd] = s;
     if (inc_val) { inc_val[ps] = g; inc_val[pd] = g; }
     if (inc_edge) { inc_edge[ps] = (int)e; inc_edge[pd] = (int)e; }  // MLP predictor: the entry's edge (row of dL/dz0)

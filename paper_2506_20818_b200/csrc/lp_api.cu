@@ -108,6 +108,7 @@ struct lp_ctx {
     SortScratch sort;                   // sized for the largest per-step sort
     TransposeScratch tsp;
     int *scan_tmp = nullptr;
+    OnePassScan scan1;                  // single-launch scan of the step's per-node counts
     int64_t sort_cap = 0;
     HopBlock hop[LP_MAX_LAYERS + 1];    // hop[0] holds only the seed frontier F_0
     unsigned char *mark = nullptr;
@@ -315,6 +316,7 @@ static void drop_model(lp_ctx *ctx)
     ctx->have_forward = ctx->have_grad = false;
     ctx->input_agg_valid = false;
     ctx->hk_valid = false;
+    ctx->scan1 = OnePassScan();
     for (auto &l : ctx->layer) l = LayerBuf();
     for (auto &h : ctx->hop) h = HopBlock();
 }
@@ -918,6 +920,12 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
     ctx->tsp.sort = ctx->sort;
     MALLOC(ctx->scan_tmp, ceil_div64(n + 1, SCAN_TILE) + 2);
     ctx->tsp.scan_tmp = ctx->scan_tmp;
+    ctx->scan1 = OnePassScan();
+    ctx->scan1.tiles_cap = ceil_div64(n + 1, SCAN_TILE) + 1;
+    MALLOC(ctx->scan1.status, ctx->scan1.tiles_cap);
+    MALLOC(ctx->scan1.ticket, 64);
+    CK(cudaMemsetAsync(ctx->scan1.status, 0, sizeof(unsigned long long) * (size_t)ctx->scan1.tiles_cap, ctx->ex.st));
+    CK(cudaMemsetAsync(ctx->scan1.ticket, 0, 64 * sizeof(unsigned), ctx->ex.st));
     CK(cudaStreamSynchronize(ctx->ex.st));
     CK_LAUNCH();
     ctx->model_set = true;
@@ -1333,8 +1341,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     // incidence lists of the scored edges, grouped by node (slots claimed with integer atomics)
     std::unique_ptr<ProfScope> pinc(new ProfScope(ctx->ex, LP_PROF_INCIDENCE, (double)E * 2.0 * 24.0));
     if (ctx->mlp) incidence_count_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->inc_ptr);
-    exclusive_scan_i32(ctx->ex, ctx->inc_ptr, rows_out, ctx->inc_ptr, ctx->inc_ptr + rows_out, ctx->scan_tmp);
-    CK(cudaMemcpyAsync(ctx->inc_cursor, ctx->inc_ptr, sizeof(int) * (size_t)rows_out, cudaMemcpyDeviceToDevice, st));
+    exclusive_scan_i32_onepass(ctx->ex, ctx->inc_ptr, rows_out, ctx->inc_ptr, ctx->inc_cursor, ctx->inc_ptr + rows_out, ctx->scan1, ctx->err_flag, ctx->scan_tmp);
     incidence_fill_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, g_pos, g_neg, ctx->inc_cursor, ctx->inc_col,
                                                    ctx->mlp ? nullptr : ctx->inc_val, ctx->mlp ? ctx->inc_edge : nullptr);
     ctx->ex.launches += 2;
@@ -1537,6 +1544,7 @@ extern "C" lp_status lp_train_step_host(lp_ctx *ctx, float *params, const int32_
     CK(cudaStreamSynchronize(st));
     if (bad) {
         cudaMemsetAsync(ctx->err_flag, 0, sizeof(int), st);
+        if (bad & 2) return fail(ctx, LP_ETIMEOUT, "lp_train_step_host: a bounded wait inside the scan of the step expired");
         return fail(ctx, LP_EINVAL, "lp_train_step_host: a node id is outside [0, n)");
     }
     return tc_check(ctx->tc, ctx->ex, true, ctx->err);
@@ -1733,6 +1741,7 @@ extern "C" lp_status lp_get_stats(lp_ctx *ctx, lp_stats *out)
     CK(cudaStreamSynchronize(ctx->ex.st));
     if (bad) {
         cudaMemsetAsync(ctx->err_flag, 0, sizeof(int), ctx->ex.st);
+        if (bad & 2) return fail(ctx, LP_ETIMEOUT, "a bounded wait inside the scan of an earlier step expired (results of that call are invalid)");
         return fail(ctx, LP_EINVAL, "a node id outside [0, n) was passed to an earlier call (it was clamped; results of that call are invalid)");
     }
     out->negatives_exhausted = (int64_t)ex;

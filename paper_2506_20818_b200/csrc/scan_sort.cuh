@@ -162,6 +162,131 @@ static void exclusive_scan_i32(Exec &ex, const int *in, int64_t n, int *out, int
 }
 
 // ------------------------------------------------------------------------------------------
+// The same scan in ONE launch (for the scans inside a training step, where three dependent launches cost more
+// than the work).  Tiles are handed out by a ticket, so a block only ever waits for tiles whose blocks are
+// already running; a tile publishes its own sum at once and its inclusive prefix as soon as the look-back over its
+// predecessors (one warp, 32 predecessors at a time) has found one.  A tile's status word carries the call's epoch,
+// so the array needs no clearing between calls.  Every wait is bounded: on expiry bit 1 of *err is set, the tile
+// carries on with what it has (the result of that call is wrong, the host reports it) and nothing hangs.
+// ------------------------------------------------------------------------------------------
+struct OnePassScan {
+    unsigned long long *status = nullptr;  // one word per tile: epoch << 34 | flag << 32 | value (flag 1 = tile sum, 2 = inclusive prefix)
+    unsigned *ticket = nullptr;            // next tile; the block that takes the last tile puts it back to 0
+    int64_t tiles_cap = 0;
+    unsigned epoch = 0;                    // host side: incremented by every call
+};
+
+LP_DEVINL unsigned long long scan_status_load(const unsigned long long *p)
+{
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+LP_DEVINL void scan_status_store(unsigned long long *p, unsigned long long v)
+{
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+__global__ void __launch_bounds__(SCAN_THREADS) scan_onepass_kernel(const int *__restrict__ in, int64_t n, int *__restrict__ out, int *__restrict__ out_copy,
+                                                                    int *__restrict__ out_total, unsigned long long *__restrict__ status,
+                                                                    unsigned *__restrict__ ticket, unsigned epoch, int *__restrict__ err)
+{
+    __shared__ int sw[8];
+    __shared__ unsigned tile_s;
+    __shared__ int prefix_s;
+    if (threadIdx.x == 0) {
+        tile_s = atomicAdd(ticket, 1u);
+        if (tile_s == gridDim.x - 1) *ticket = 0;  // every tile of this launch has been handed out
+    }
+    __syncthreads();
+    const unsigned tile = tile_s;
+    const int64_t t0 = (int64_t)tile * SCAN_TILE + (int64_t)threadIdx.x * SCAN_ITEMS;
+    int v[SCAN_ITEMS];
+    int acc = 0;
+#pragma unroll
+    for (int i = 0; i < SCAN_ITEMS; ++i) {
+        v[i] = (t0 + i < n) ? in[t0 + i] : 0;
+        acc += v[i];
+    }
+    int tot;
+    int ex = block_exclusive_scan_256(acc, sw, &tot);
+    const unsigned long long tag = (unsigned long long)epoch << 34;
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x;
+        if (lane == 0) scan_status_store(status + tile, tag | ((tile == 0 ? 2ull : 1ull) << 32) | (unsigned)tot);
+        int exclusive = 0;
+        int64_t base = (int64_t)tile - 1;
+        bool done = tile == 0;
+        while (!done) {
+            const int64_t t = base - lane;
+            int flag = 2, val = 0;  // before the first tile: an inclusive prefix of 0
+            if (t >= 0) {
+                unsigned long long w = scan_status_load(status + t);
+                if ((w >> 34) != epoch || ((w >> 32) & 3ull) == 0) {
+                    unsigned long long t_start;
+                    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_start));
+                    for (;;) {
+                        w = scan_status_load(status + t);
+                        if ((w >> 34) == epoch && ((w >> 32) & 3ull) != 0) break;
+                        unsigned long long now;
+                        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now));
+                        if (now - t_start > 2000000000ull) {  // two seconds: give up, report, carry on
+                            atomicOr(err, 2);
+                            w = tag | (2ull << 32);
+                            break;
+                        }
+                    }
+                }
+                flag = (int)((w >> 32) & 3ull);
+                val = (int)(unsigned)(w & 0xffffffffull);
+            }
+            const unsigned has_prefix = __ballot_sync(0xffffffffu, flag == 2);
+            const int upto = has_prefix ? __ffs(has_prefix) - 1 : 31;  // nearest predecessor that knows its inclusive prefix
+            int contrib = lane <= upto ? val : 0;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) contrib += __shfl_xor_sync(0xffffffffu, contrib, o);
+            exclusive += contrib;
+            if (has_prefix) done = true; else base -= 32;
+        }
+        if (lane == 0) {
+            prefix_s = exclusive;
+            if (tile != 0) scan_status_store(status + tile, tag | (2ull << 32) | (unsigned)(exclusive + tot));
+        }
+    }
+    __syncthreads();
+    ex += prefix_s;
+#pragma unroll
+    for (int i = 0; i < SCAN_ITEMS; ++i) {
+        if (t0 + i < n) {
+            out[t0 + i] = ex;
+            if (out_copy) out_copy[t0 + i] = ex;
+        }
+        ex += v[i];
+    }
+    if (out_total && tile == gridDim.x - 1 && threadIdx.x == SCAN_THREADS - 1) *out_total = ex;
+}
+
+// out[i] = sum_{j<i} in[j]; out_copy (optional) receives the same values; *out_total (optional) the sum of all.
+// in == out is allowed.  Falls back to the three-launch scan when the scratch is too small.
+static void exclusive_scan_i32_onepass(Exec &ex, const int *in, int64_t n, int *out, int *out_copy, int *out_total, OnePassScan &sc, int *err, int *tmp)
+{
+    if (n <= 0) {
+        if (out_total) cudaMemsetAsync(out_total, 0, sizeof(int), ex.st);
+        return;
+    }
+    const int64_t tiles = ceil_div64(n, SCAN_TILE);
+    if (!sc.status || tiles > sc.tiles_cap) {
+        exclusive_scan_i32(ex, in, n, out, out_total, tmp);
+        if (out_copy) cudaMemcpyAsync(out_copy, out, sizeof(int) * (size_t)n, cudaMemcpyDeviceToDevice, ex.st);
+        return;
+    }
+    sc.epoch = (sc.epoch + 1u) & 0x3fffffffu;
+    if (sc.epoch == 0) sc.epoch = 1;
+    scan_onepass_kernel<<<(unsigned)tiles, SCAN_THREADS, 0, ex.st>>>(in, n, out, out_copy, out_total, sc.status, sc.ticket, sc.epoch, err);
+    ex.launches += 1;
+}
+
+// ------------------------------------------------------------------------------------------
 // stable LSD radix sort of pairs, 8 bits per pass
 // ------------------------------------------------------------------------------------------
 constexpr int RS_THREADS = 256;
