@@ -662,6 +662,283 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
 }
 
 // ---------------------------------------------------------------------------------------------
+// kernel 3: the persistent transform on PAIRS of SMs (thread-block clusters of two CTAs, tcgen05 cta_group::2).
+//
+// One tcgen05.mma of the pair multiplies a 256-row tile (128 rows in each CTA's shared memory) by a BN-column weight
+// slice of which each CTA holds half (BN / 2 rows of Bt), and leaves 128 rows x BN FP32 columns in each CTA's tensor
+// memory.  Against kernel 2 a CTA keeps only half of the weight slice resident, so a slice up to 256 columns wide fits
+// for K up to 512 and no operand tile is read by more than one SM.  Roles per CTA as in kernel 2 (warp 0 producer,
+// warp 1 MMA issuer, warps 2-9 epilogue); only the issuer of the pair's first CTA (the leader) issues MMAs.
+//   operand stages : each producer copies its own 128-row A tile and announces the bytes on the LEADER's full barrier
+//                    (two arrivals per phase); the leader's commit releases the stage in both CTAs
+//   accumulators   : two per CTA; the leader's commit tells both CTAs' epilogues that one is complete, the eight epilogue
+//                    warps of BOTH CTAs arrive on the leader's barrier when they have drained it
+//   tensor memory  : allocated and freed by warp 0 of both CTAs (cta_group::2), freed after a cluster barrier
+// No bulk copy here is a multicast (every tile is copied by the CTA that consumes it); only the completion signal of the
+// MMAs goes to both CTAs.  All waits are bounded.
+// ---------------------------------------------------------------------------------------------
+LP_DEVINL uint32_t cluster_cta_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+LP_DEVINL uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank)  // shared::cluster address of the same location in CTA `rank` of the cluster
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+LP_DEVINL void cluster_barrier()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+LP_DEVINL void mbar_arrive_remote(uint32_t cluster_addr) { asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory"); }
+LP_DEVINL void mbar_expect_tx_remote(uint32_t cluster_addr, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr), "r"(bytes) : "memory");
+}
+// tile copy into this CTA's shared memory whose completion is counted on a barrier of either CTA of the pair
+LP_DEVINL void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar_cluster_addr, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+                 "l"(map), "r"(bar_cluster_addr), "r"(x), "r"(y)
+                 : "memory");
+}
+LP_DEVINL void tmem_alloc_pair(uint32_t smem_dst, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+LP_DEVINL void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+LP_DEVINL void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// completion of the pair's earlier MMAs arrives on the barrier at this shared-memory offset in BOTH CTAs of the pair
+// (a barrier signal sent to two CTAs; no data is copied)
+LP_DEVINL void umma_commit_pair(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar), "h"((uint16_t)3)
+                 : "memory");
+}
+// instruction descriptor of the pair's MMA: 256 rows (128 per CTA), n columns
+static __host__ __device__ inline uint32_t make_idesc_bf16_pair(int n)
+{
+    uint32_t d = 0;
+    d |= 1u << 4;                      // accumulator format F32
+    d |= 1u << 7;                      // A format BF16
+    d |= 1u << 10;                     // B format BF16
+    d |= (uint32_t)(n >> 3) << 17;
+    d |= (uint32_t)(256 >> 4) << 24;
+    return d;
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TCP_THREADS, 1)
+    tc_linear_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const __grid_constant__ CUtensorMap mapC,
+                          const TcGemmParams p)
+{
+    __shared__ float s_bias[256];
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[TCP_MAX_STAGES], bar_empty[TCP_MAX_STAGES], bar_w, bar_acc_full[2], bar_acc_empty[2];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_cta_rank();   // 0 = leader of the pair
+    const bool leader = rank == 0;
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int BN = p.BN, HB = BN / 2;           // the pair's slice width and this CTA's half of it
+    const int KB = p.K / TC_BK;
+    const uint32_t w_sub_bytes = (uint32_t)HB * 128;  // one k-block of this CTA's half slice: HB rows x 128 B
+    uint8_t *smem_w = smem;
+    uint8_t *smem_a = smem + (size_t)KB * w_sub_bytes;
+    const uint32_t a_bytes = TC_BM * TC_BK * 2;
+    const int S = p.stages;
+    uint8_t *smem_out = smem_a + (size_t)S * a_bytes;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < 2 * BN) tmem_cols <<= 1;
+
+    const int n_slices = p.N / BN;
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    const int slice = pair % n_slices;
+    const int n0 = slice * BN;
+    const int64_t m_tiles = (p.M + 2 * TC_BM - 1) / (2 * TC_BM);  // tiles of 256 rows
+    const int64_t first_tile = pair / n_slices;
+    const int64_t stride = n_pairs / n_slices;
+    const int64_t my_tiles = first_tile < m_tiles ? (m_tiles - first_tile + stride - 1) / stride : 0;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 2);   // one announcement per CTA of the pair (used in the leader only)
+            mbar_init(smem_u32(&bar_empty[s]), 1);
+        }
+        mbar_init(smem_u32(&bar_w), 2);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&bar_acc_full[b]), 1);
+            mbar_init(smem_u32(&bar_acc_empty[b]), 16);  // eight epilogue warps in each CTA (used in the leader only)
+        }
+        abort_s = 0;
+        fence_barrier_init();
+        fence_async_proxy();
+        tma_prefetch_desc(&mapA);
+        tma_prefetch_desc(&mapB);
+        tma_prefetch_desc(&mapC);
+    }
+    if (warp == 0) {
+        __syncwarp();
+        tmem_alloc_pair(smem_u32(&tmem_base_s), tmem_cols);
+    }
+    for (int j = threadIdx.x; j < BN; j += TCP_THREADS) s_bias[j] = p.bias ? p.bias[n0 + j] : 0.f;
+    tc_fence_before();
+    __syncthreads();
+    cluster_barrier();  // both CTAs' barriers are initialised before either announces anything on them
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+    volatile int *abort_flag = &abort_s;
+
+    if (my_tiles > 0) {
+        if (warp == 0 && lane == 0) {
+            // ---- producer: this CTA's half of the weight slice, then its 128 rows of every tile
+            const uint32_t bw = map_to_cta(smem_u32(&bar_w), 0);
+            mbar_expect_tx_remote(bw, (uint32_t)KB * w_sub_bytes);
+            for (int kb = 0; kb < KB; ++kb) tma_load_2d_pair(smem_u32(smem_w + (size_t)kb * w_sub_bytes), &mapB, bw, kb * TC_BK, n0 + (int)rank * HB);
+            int64_t it = 0;
+            for (int64_t i = 0; i < my_tiles && !*abort_flag; ++i) {
+                const int m0 = (int)((first_tile + i * stride) * (2 * TC_BM)) + (int)rank * TC_BM;
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    const int s = (int)(it % S);
+                    if (it >= S && !mbar_wait(smem_u32(&bar_empty[s]), (uint32_t)(((it / S) & 1) ^ 1), p.wait_ns)) {
+                        atomicExch(p.err, 1);
+                        *abort_flag = 1;
+                        break;
+                    }
+                    const uint32_t bar = map_to_cta(smem_u32(&bar_full[s]), 0);
+                    mbar_expect_tx_remote(bar, a_bytes + (it == 0 && leader ? (uint32_t)p.extra_tx : 0u));
+                    tma_load_2d_pair(smem_u32(smem_a + (size_t)s * a_bytes), &mapA, bar, kb * TC_BK, m0);
+                }
+            }
+        } else if (warp == 1 && lane == 0 && leader) {
+            // ---- MMA issuer of the pair
+            const uint32_t idesc = make_idesc_bf16_pair(BN);
+            bool ok = mbar_wait(smem_u32(&bar_w), 0, p.wait_ns);
+            if (!ok) { atomicExch(p.err, 4); *abort_flag = 1; }
+            int64_t it = 0;
+            for (int64_t i = 0; i < my_tiles && ok; ++i) {
+                const int b = (int)(i & 1);
+                if (i >= 2 && !mbar_wait(smem_u32(&bar_acc_empty[b]), (uint32_t)((((i >> 1) - 1) & 1)), p.wait_ns)) {
+                    atomicExch(p.err, 5);
+                    *abort_flag = 1;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t tmem_d = tmem_base + (uint32_t)(b * BN);
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    const int s = (int)(it % S);
+                    if (!mbar_wait(smem_u32(&bar_full[s]), (uint32_t)((it / S) & 1), p.wait_ns)) {
+                        atomicExch(p.err, 2);
+                        *abort_flag = 1;
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem_a + (size_t)s * a_bytes);
+                    const uint32_t sb = smem_u32(smem_w + (size_t)kb * w_sub_bytes);
+#pragma unroll
+                    for (int k = 0; k < TC_BK / TC_UMMA_K; ++k)
+                        umma_bf16_pair(tmem_d, make_smem_desc(sa + k * 32, 16, 1024), make_smem_desc(sb + k * 32, 16, 1024), idesc, (kb | k) != 0 ? 1u : 0u);
+                    umma_commit_pair(smem_u32(&bar_empty[s]));  // the stage is free again in both CTAs
+                }
+                if (ok) umma_commit_pair(smem_u32(&bar_acc_full[b]));  // both CTAs' epilogues may drain their 128 rows
+            }
+        } else if (warp >= 2) {
+            // ---- epilogue (as in kernel 2, on this CTA's 128 rows; the drained accumulator is reported to the leader)
+            const int q = warp & 3;
+            const int my_box = (warp - 2) >> 2;
+            for (int64_t i = 0; i < my_tiles; ++i) {
+                const int b = (int)(i & 1);
+                bool ready = mbar_wait(smem_u32(&bar_acc_full[b]), (uint32_t)((i >> 1) & 1), p.wait_ns);
+                if (!ready && lane == 0) { atomicExch(p.err, 3); *abort_flag = 1; }
+                if (!__all_sync(0xffffffffu, ready) && lane == 0) *abort_flag = 1;
+                epilogue_barrier();
+                if (*abort_flag != 0) break;
+                tc_fence_after();
+                const int m0 = (int)((first_tile + i * stride) * (2 * TC_BM)) + (int)rank * TC_BM;
+                const int row_t = q * 32 + lane;
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN);
+                const bool store_thread = (((warp - 2) & 3) == 0 && lane == 0);
+                const float rs = (p.row_scale && (int64_t)m0 + row_t < p.M) ? __ldg(p.row_scale + m0 + row_t) : 1.f;
+                for (int half = 0; half < BN; half += 128) {
+                    const int nbox = min(2, (BN - half) / 64);
+                    if (my_box < nbox) {
+                        if (store_thread) tma_store_wait_read();
+                        group_barrier(my_box);
+                        const int cb = half + my_box * 64;
+                        uint32_t r[2][32];
+                        tmem_ld_32x32_issue(taddr + (uint32_t)cb, r[0]);
+                        tmem_ld_32x32_issue(taddr + (uint32_t)(cb + 32), r[1]);
+                        tmem_ld_wait();
+                        uint8_t *box = smem_out + (size_t)my_box * 16384 + (size_t)row_t * 128;
+#pragma unroll
+                        for (int h2 = 0; h2 < 2; ++h2) {
+                            const int c0 = cb + 32 * h2;
+                            float v[32];
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) {
+                                const float4 bb = *reinterpret_cast<const float4 *>(&s_bias[c0 + j]);
+                                v[j] = __uint_as_float(r[h2][j]) + bb.x;
+                                v[j + 1] = __uint_as_float(r[h2][j + 1]) + bb.y;
+                                v[j + 2] = __uint_as_float(r[h2][j + 2]) + bb.z;
+                                v[j + 3] = __uint_as_float(r[h2][j + 3]) + bb.w;
+                            }
+                            if (p.relu) {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
+                            }
+                            if (p.row_scale && n0 + c0 >= p.scale_col0) {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) v[j] *= rs;
+                            }
+                            const int chunk0 = 4 * h2;
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                Vec16<bf16> o;
+                                o.from_float(v + 8 * j);
+                                *reinterpret_cast<uint4 *>(box + (((chunk0 + j) ^ (row_t & 7)) << 4)) = o.v;
+                            }
+                        }
+                        fence_async_proxy();
+                        group_barrier(my_box);
+                        if (store_thread) {
+                            tma_store_2d(&mapC, smem_u32(smem_out + (size_t)my_box * 16384), n0 + half + my_box * 64, m0);
+                            tma_store_commit();
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_remote(map_to_cta(smem_u32(&bar_acc_empty[b]), 0));
+            }
+        }
+    }
+    if ((warp == 2 || warp == 6) && lane == 0) tma_store_wait_all();
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    cluster_barrier();  // neither CTA frees tensor memory, or leaves with barriers the other may still signal, before both are done
+    if (warp == 0) {
+        __syncwarp();
+        tmem_dealloc_pair(tmem_base, tmem_cols);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
 static bool tc_init(TcState &tc, std::string &err)
@@ -681,6 +958,7 @@ static bool tc_init(TcState &tc, std::string &err)
     }
     cudaMemset(tc.err_word, 0, 256);
     if (cudaFuncSetAttribute(tc_linear_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024 + 512) != cudaSuccess ||
+        cudaFuncSetAttribute(tc_linear_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024 + 512) != cudaSuccess ||
         cudaFuncSetAttribute(tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess ||
         cudaFuncSetAttribute(tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) {
         err = "cannot raise the dynamic shared memory limit of the tensor-core GEMM";
@@ -753,6 +1031,15 @@ static int tc_persistent_bn(int N, int K)
     return 0;
 }
 
+// Slice width for the pair kernel: the largest multiple of 128 (at most 256, dividing N) whose half slice BN / 2 x K x 2 B
+// fits 128 KiB beside at least two A stages and the output staging.  0 = does not fit.
+static int tc_pair_bn(int N, int K)
+{
+    for (int bn = 256; bn >= 128; bn -= 128)
+        if (N % bn == 0 && (int64_t)(bn / 2) * K * 2 <= 128 * 1024) return bn;
+    return 0;
+}
+
 static int tc_sm_count()
 {
     static int sms = 0;
@@ -768,6 +1055,30 @@ static int tc_sm_count()
 static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const bf16 *A, int64_t lda, const bf16 *Bt, const float *bias, bool relu,
                            bf16 *C, int64_t ldc, std::string &err, const float *row_scale = nullptr, int scale_col0 = 0)
 {
+    // pairs of SMs: a slice of up to 256 columns whose half (per CTA) fits 128 KiB; worth it from a few hundred tiles on
+    const int pair_bn = tc_pair_bn(N, K);
+    if (pair_bn > 0 && M >= 64 * TC_BM && tc_sm_count() >= 4) {
+        CUtensorMap mapA, mapB, mapC;
+        if (!tc_make_map(tc, &mapA, A, M, K, lda, TC_BK, TC_BM, err)) return false;
+        if (!tc_make_map(tc, &mapB, Bt, N, K, K, TC_BK, pair_bn / 2, err)) return false;
+        if (!tc_make_map(tc, &mapC, C, M, N, ldc, 64, TC_BM, err)) return false;
+        TcGemmParams p{};
+        const int64_t smem_cap = 225 * 1024 + 512 - 1024;
+        const int64_t w_bytes = (int64_t)(K / TC_BK) * (pair_bn / 2) * 128;  // this CTA's half of the slice
+        p.M = M; p.N = N; p.K = K; p.BN = pair_bn;
+        p.stages = (int)std::max<int64_t>(2, std::min<int64_t>(TCP_MAX_STAGES, (smem_cap - w_bytes - TCP_STAGE_OUT_BYTES) / (TC_BM * TC_BK * 2)));
+        p.bias = bias; p.relu = relu ? 1 : 0; p.C = C; p.ldc = ldc; p.out_f32 = nullptr; p.err = tc.err_word;
+        p.row_scale = row_scale; p.scale_col0 = scale_col0;
+        p.wait_ns = tc.wait_limit_ns; p.extra_tx = tc.overdeclare_tx; tc.overdeclare_tx = 0;
+        const int n_slices = N / pair_bn;
+        const int64_t m_tiles = ceil_div64(M, 2 * TC_BM);
+        int64_t pairs = std::min<int64_t>((int64_t)tc_sm_count() / 2, m_tiles * n_slices);
+        pairs = std::max<int64_t>(n_slices, pairs / n_slices * n_slices);  // a whole number of pairs per slice
+        const size_t smem = (size_t)w_bytes + (size_t)p.stages * TC_BM * TC_BK * 2 + TCP_STAGE_OUT_BYTES + 1024;
+        tc_linear_pair_kernel<<<(unsigned)(2 * pairs), TCP_THREADS, smem, ex.st>>>(mapA, mapB, mapC, p);
+        ex.launches += 1;
+        return true;
+    }
     const int pbn = tc_persistent_bn(N, K);
     if (pbn > 0 && M >= 4 * TC_BM) {
         CUtensorMap mapA, mapB;

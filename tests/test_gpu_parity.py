@@ -198,7 +198,8 @@ def test_linear_and_weight_grad_fp32(pkg, M, K, N):
     ctx.close()
 
 
-@pytest.mark.parametrize("M,K,N", [(1000, 64, 64), (4099, 256, 256), (70000, 512, 256), (300, 128, 256), (131, 256, 128), (5, 256, 512)])
+@pytest.mark.parametrize("M,K,N", [(1000, 64, 64), (4099, 256, 256), (70000, 512, 256), (300, 128, 256), (131, 256, 128), (5, 256, 512),
+                                   (8192, 256, 256), (20001, 256, 512), (33000, 512, 512), (9000, 128, 128), (50000, 64, 256)])
 def test_linear_and_weight_grad_bf16(pkg, M, K, N):
     g = wl.erdos_renyi(50, 100, seed=0)
     ctx = make_ctx(pkg, g, wl.node_features(g.n, 8, 0))
