@@ -1120,21 +1120,7 @@ static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const
     return true;
 }
 
-// Layer transform with FP32 weights: converts the layer's weights to BF16 (transposing when they
-// are stored [K, N]) into the scratch buffer, then runs the K-major GEMM.
-//   w_is_kn = true : W is [K, N] row-major and the product is A * W        (forward)
-//   w_is_kn = false: W is [N, K] row-major and the product is A * W^T      (input gradient)
-static bool tc_linear(TcState &tc, Exec &ex, int64_t M, int N, int K, const bf16 *A, int lda, const float *W, bool w_is_kn, const float *bias,
-                      bool relu, bf16 *C, int ldc, std::string &err, const float *row_scale = nullptr, int scale_col0 = 0)
-{
-    const int total = K * N;
-    if (w_is_kn) weights_to_bf16_kernel<<<(total + 255) / 256, 256, 0, ex.st>>>(W, K, N, tc.wbuf, nullptr);
-    else convert_kernel<float, bf16><<<(total + 255) / 256, 256, 0, ex.st>>>(W, tc.wbuf, total);
-    ex.launches += 1;
-    return tc_gemm_kmajor(tc, ex, M, N, K, A, lda, tc.wbuf, bias, relu, C, ldc, err, row_scale, scale_col0);
-}
-
-// the same with a BF16 B operand given as [K, N] (b_is_nk = false) or [N, K] (b_is_nk = true)
+// C = act(A B + bias) with a BF16 B operand given as [K, N] (b_is_nk = false: transposed into the scratch first) or [N, K] (b_is_nk = true)
 __global__ void transpose_bf16_kernel(const bf16 *__restrict__ B, int K, int N, bf16 *__restrict__ Bt)
 {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -1160,7 +1146,7 @@ static bool tc_linear_bf16_b(TcState &tc, Exec &ex, int64_t M, int N, int K, con
 static int tc_weight_grad_splits(int64_t rows, int Kin, int N)
 {
     const int tiles = (Kin / TC_BM) * (N / tc_pick_bn(N));
-    int splits = std::max(1, (2 * 148) / std::max(tiles, 1));
+    int splits = std::max(1, (2 * 148) / std::max(tiles, 1));  // two CTAs per SM (measured: one per SM 156 us, two 145 us, three 207 us per step)
     const int64_t max_by_rows = std::max<int64_t>(1, ceil_div64(rows, 4 * TC_BK));
     return (int)std::min<int64_t>(splits, max_by_rows);
 }

@@ -127,6 +127,7 @@ struct lp_ctx {
     uint64_t hk_version = 0, param_version = 0;
     int64_t last_exhausted = 0;
     TcState tc;                         // tensor-core GEMM state (descriptor encoder, device error word)
+    bf16 *w16 = nullptr, *w16t = nullptr;  // BF16 path: the parameter vector of the current call as BF16, as is and with every weight matrix transposed
 };
 
 static thread_local std::string g_create_error;  // errors of calls that have no context: one per host thread
@@ -317,6 +318,7 @@ static void drop_model(lp_ctx *ctx)
     ctx->input_agg_valid = false;
     ctx->hk_valid = false;
     ctx->scan1 = OnePassScan();
+    ctx->w16 = ctx->w16t = nullptr;
     for (auto &l : ctx->layer) l = LayerBuf();
     for (auto &h : ctx->hop) h = HopBlock();
 }
@@ -843,6 +845,10 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
     MALLOC(ctx->d_neg_tmp, max_batch * std::max<int64_t>(max_k, 1));
     MALLOC(ctx->d_loss_tmp, 64);
     MALLOC(ctx->d_grads_tmp, ctx->n_params);
+    if (d->prec == LP_BF16) {
+        MALLOC(ctx->w16, ctx->n_params);
+        MALLOC(ctx->w16t, ctx->n_params);
+    }
 
     // per-step sort capacity: incidence lists and (sampled) block transposes
     int64_t sort_cap = 2 * E;
@@ -965,6 +971,18 @@ extern "C" lp_status lp_sample_negatives(lp_ctx *ctx, uint64_t seed, uint64_t st
 // ----------------------------------------------------------------------------------------------
 template <typename T> static T *tptr(void *p) { return (T *)p; }
 
+// BF16 path: one launch turns the call's parameter vector into the two BF16 copies the transforms read
+static void cache_weights(lp_ctx *ctx, const float *params)
+{
+    if (ctx->desc.prec != LP_BF16 || !ctx->w16) return;
+    WeightBlocks wb{};
+    for (int k = 0; k < ctx->K; ++k) { wb.off[wb.count] = ctx->layer[k].off_w; wb.kin[wb.count] = ctx->layer[k].Kin; wb.fo[wb.count] = ctx->layer[k].Fo; ++wb.count; }
+    if (ctx->mlp)
+        for (int j = 0; j < 2; ++j) { wb.off[wb.count] = ctx->pred[j].off_w; wb.kin[wb.count] = ctx->pred[j].Kin; wb.fo[wb.count] = ctx->pred[j].Fo; ++wb.count; }
+    weights_cache_kernel<<<nblk(ctx->n_params), 256, 0, ctx->ex.st>>>(params, ctx->n_params, wb, ctx->w16, ctx->w16t);
+    ctx->ex.launches += 1;
+}
+
 // dense transform of one layer: Out = act(A W + b)
 template <typename T>
 static lp_status layer_linear(lp_ctx *ctx, int64_t rows, const LayerBuf &L, const float *params, T *out, int ldo, bool relu)
@@ -972,9 +990,8 @@ static lp_status layer_linear(lp_ctx *ctx, int64_t rows, const LayerBuf &L, cons
     if (rows <= 0) return LP_OK;
     ProfScope prof(ctx->ex, LP_PROF_GEMM_FWD, gemm_bytes((double)rows, L.Fo, L.Kin, sizeof(T), sizeof(T)), 2.0 * rows * L.Fo * L.Kin);
     if (sizeof(T) == 2 && tc_linear_supported(L.Kin, L.Fo)) {
-        std::string err;
-        if (!tc_linear(ctx->tc, ctx->ex, rows, L.Fo, L.Kin, (const bf16 *)L.A, L.Kin, params + L.off_w, /*w_is_kn=*/true, params + L.off_b, relu,
-                       (bf16 *)out, ldo, err))
+        std::string err;  // Out = A W: the K-major GEMM reads W^T [Fo, Kin] from the transposed BF16 copy
+        if (!tc_gemm_kmajor(ctx->tc, ctx->ex, rows, L.Fo, L.Kin, (const bf16 *)L.A, L.Kin, ctx->w16t + L.off_w, params + L.off_b, relu, (bf16 *)out, ldo, err))
             return fail(ctx, LP_ECUDA, "tensor-core GEMM: " + err);
         return LP_OK;
     }
@@ -993,9 +1010,9 @@ static lp_status layer_input_grad(lp_ctx *ctx, int64_t rows, const LayerBuf &L, 
     if (rows <= 0) return LP_OK;
     ProfScope prof(ctx->ex, LP_PROF_GEMM_DGRAD, gemm_bytes((double)rows, L.Kin, L.Fo, sizeof(T), sizeof(T)), 2.0 * rows * L.Fo * L.Kin);
     if (sizeof(T) == 2 && tc_linear_supported(L.Fo, L.Kin)) {
-        std::string err;
-        if (!tc_linear(ctx->tc, ctx->ex, rows, L.Kin, L.Fo, (const bf16 *)dZ, L.Fo, params + L.off_w, /*w_is_kn=*/false, nullptr, false, (bf16 *)dA, L.Kin,
-                       err, row_scale, scale_col0))
+        std::string err;  // dA = dZ W^T: W [Kin, Fo] as stored is the [N, K] operand
+        if (!tc_gemm_kmajor(ctx->tc, ctx->ex, rows, L.Kin, L.Fo, (const bf16 *)dZ, L.Fo, ctx->w16 + L.off_w, nullptr, false, (bf16 *)dA, L.Kin, err, row_scale,
+                            scale_col0))
             return fail(ctx, LP_ECUDA, "tensor-core GEMM: " + err);
         return LP_OK;
     }
@@ -1296,6 +1313,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         check_step_ids_kernel<<<nblk(2 * B + 2 * nk), 256, 0, st>>>(pos_src, B, pos_dst, B, neg_dst, nk, neg_src, (k > 0 && neg_src) ? nk : 0, ctx->n, ctx->err_flag);
         ctx->ex.launches += 1;
     }
+    cache_weights(ctx, params);
     if (ctx->sampled) {
         lp_status s = build_blocks(ctx, pos_src, pos_dst, B, neg_src, neg_dst, k, seed, step);
         if (s != LP_OK) return s;
@@ -1560,7 +1578,9 @@ static lp_status score_impl(lp_ctx *ctx, const float *params, const int *src, co
     // full-graph models: H^(K) of the last forward pass is reused while the caller passes the same parameter vector and no
     // call of this library has updated it since
     lp_status s = LP_OK;
-    if (!(ctx->hk_valid && ctx->hk_params == params && ctx->hk_version == ctx->param_version)) s = forward_impl<T>(ctx, params);
+    const bool reuse = ctx->hk_valid && ctx->hk_params == params && ctx->hk_version == ctx->param_version;
+    if (!reuse || ctx->mlp) cache_weights(ctx, params);  // (the MLP predictor's layers need their weights in any case)
+    if (!reuse) s = forward_impl<T>(ctx, params);
     if (s != LP_OK) return s;
     const int D = ctx->desc.dims[ctx->K];
     const int *idmap = ctx->sampled ? ctx->hop[0].posmap : nullptr;

@@ -54,3 +54,31 @@ __global__ void weights_to_bf16_kernel(const float *__restrict__ W, int K, int N
     if (Wt) Wt[(size_t)n * K + k] = x;
     if (Wc) Wc[i] = x;
 }
+
+// BF16 copies of a whole flat parameter vector in one launch: `asis` element for element, and `transposed` with every
+// weight matrix W[Kin, Fo] (row-major, at offset off) stored as its transpose [Fo, Kin] at the same offset (biases are
+// copied in place in both).  The forward transforms read the transposed blocks, the input-gradient transforms the others.
+struct WeightBlocks {
+    int count;
+    long long off[8];
+    int kin[8], fo[8];
+};
+__global__ void weights_cache_kernel(const float *__restrict__ params, long long n, WeightBlocks blocks, bf16 *__restrict__ asis, bf16 *__restrict__ transposed)
+{
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const bf16 x = __float2bfloat16_rn(params[i]);
+    asis[i] = x;
+    long long dst = i;
+#pragma unroll
+    for (int b = 0; b < 8; ++b) {
+        if (b < blocks.count) {
+            const long long r = i - blocks.off[b];
+            if (r >= 0 && r < (long long)blocks.kin[b] * blocks.fo[b]) {
+                const int k = (int)(r / blocks.fo[b]), c = (int)(r - (long long)k * blocks.fo[b]);
+                dst = blocks.off[b] + (long long)c * blocks.kin[b] + k;
+            }
+        }
+    }
+    transposed[dst] = x;
+}
