@@ -255,7 +255,7 @@ def _gpu_view_step(pkg, ctxG, dpart, X_dev, X, g, part, i, sp, negatives, params
     return ctx, loss, grads, (view, cand, pu, pv, nd, seed, step)
 
 
-@pytest.mark.parametrize("scale,p_check", [(1.0, {"local": [0, 4], "global": [5]}), (0.1, {"local": list(range(8)), "global": list(range(8))})])
+@pytest.mark.parametrize("scale,p_check", [(1.0, {"local": [0], "global": [5]}), (0.1, {"local": list(range(8)), "global": list(range(8))})])
 def test_config5_gpu_built_views(pkg, scale, p_check):
     g, X, params, pos, cfg = wl.make_config("c5_partitioned_sage2", scale=scale)
     dims, p, alpha, prec, B = cfg["dims"], cfg["partitions"], cfg["alpha"], "bf16", 65536
@@ -296,3 +296,49 @@ def test_config5_gpu_built_views(pkg, scale, p_check):
             avg = oracle.average_gradients([ora[i] for i in range(p)])
             assert rel_l2(acc.cpu().numpy() / p, avg) < TOL[prec]
     ctxG.close()
+
+
+def test_config5_full_size_local_partitions_as_own_graphs(pkg):
+    # Local negatives never leave the partition, so a worker can hold its induced subgraph as a graph of its own (about
+    # 125,000 of the 1 M nodes, renumbered in ascending id order) -- the form the benchmark times.  Every partition's BF16 step
+    # against the oracle on the same subgraph, and the 8-way accumulated gradient against the oracle's average (Algorithm 1).
+    g, X, params, pos, cfg = wl.make_config("c5_partitioned_sage2")
+    dims, p, prec, B = cfg["dims"], cfg["partitions"], "bf16", 65536
+    part = wl.random_partition(g.n, p, seed=5)
+    rows = np.repeat(np.arange(g.n, dtype=np.int64), np.diff(g.rowptr))
+    prow, pcol, upper = part[rows], part[g.col], g.col > rows
+    acc = torch.zeros(len(params), device=DEV)
+    ora = []
+    for i in range(p):
+        own = np.nonzero(part == i)[0]
+        new_id = np.full(g.n, -1, dtype=np.int64)
+        new_id[own] = np.arange(own.shape[0])
+        inside = (prow == i) & (pcol == i)
+        sub = wl.csr_from_edges(own.shape[0], new_id[rows[inside]], new_id[g.col[inside]])
+        Xs = np.ascontiguousarray(X[own])
+        keep = inside & upper
+        pu, pv = new_id[rows[keep]].astype(np.int32)[:B].copy(), new_id[g.col[keep]].astype(np.int32)[:B].copy()
+        ctx = pkg.Context(0)
+        ctx.load_graph(sub.n, sub.rowptr, sub.col, None, Xs)
+        ctx.set_model("sage", dims, prec=prec, max_batch=len(pu), max_k=1)
+        du, dv = t32(pu), t32(pv)
+        seed, step = 11, i
+        _, nd = ctx.sample_negatives(seed, step, 1, du)
+        loss, grads = torch.zeros(1, device=DEV), torch.zeros(ctx.n_params, device=DEV)
+        ctx.train_step(t32(params), du, dv, None, nd, 1, loss, grads, seed=seed, step=step)
+        ctx.train_step(t32(params), du, dv, None, nd, 1, loss, acc, seed=seed, step=step, accumulate=True)
+        torch.cuda.synchronize()
+        ons, ond, _ = oracle.sample_negatives(sub.n, sub.rowptr, sub.col, pu, seed, step, 1)
+        assert np.array_equal(nd.cpu().numpy(), ond)
+        # the same negatives as a draw among the partition's nodes in the 1 M-node numbering (candidate set = own nodes)
+        if i == 0:
+            view = wl.induced_subgraph(g, part == i)
+            _, gnd, _ = oracle.sample_negatives(g.n, view.rowptr, view.col, own[pu].astype(np.int32), seed, step, 1, cand=own.astype(np.int32))
+            assert np.array_equal(own[ond], gnd)
+        H1 = ctx.embeddings(1).cpu().numpy() > 0
+        ref = oracle.train_step(sub, Xs, params, "sage", dims, pu, pv, ons, ond, relu_ties=[H1], rounding=prec)
+        assert_relu_decisions_agree(ref["cache"], [H1], None, f"config 5 partition {i} as its own graph")
+        check_step(ctx, ref, loss, grads, "sage", dims, TOL[prec], {"dHK": rel_l2(ctx.output_gradient().cpu().numpy(), ref["dHK"])})
+        ora.append(ref["grads"])
+        ctx.close()
+    assert rel_l2(acc.cpu().numpy() / p, oracle.average_gradients(ora)) < TOL[prec]
