@@ -317,6 +317,7 @@ static void drop_model(lp_ctx *ctx)
     ctx->have_forward = ctx->have_grad = false;
     ctx->input_agg_valid = false;
     ctx->hk_valid = false;
+    ctx->ex.scan1 = nullptr;
     ctx->scan1 = OnePassScan();
     ctx->w16 = ctx->w16t = nullptr;
     for (auto &l : ctx->layer) l = LayerBuf();
@@ -927,11 +928,13 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
     MALLOC(ctx->scan_tmp, ceil_div64(n + 1, SCAN_TILE) + 2);
     ctx->tsp.scan_tmp = ctx->scan_tmp;
     ctx->scan1 = OnePassScan();
-    ctx->scan1.tiles_cap = ceil_div64(n + 1, SCAN_TILE) + 1;
+    ctx->scan1.tiles_cap = std::max<int64_t>(ceil_div64(n + 1, SCAN_TILE), ceil_div64(SortScratch::hist_ints(sort_cap), SCAN_TILE)) + 1;
     MALLOC(ctx->scan1.status, ctx->scan1.tiles_cap);
     MALLOC(ctx->scan1.ticket, 64);
     CK(cudaMemsetAsync(ctx->scan1.status, 0, sizeof(unsigned long long) * (size_t)ctx->scan1.tiles_cap, ctx->ex.st));
     CK(cudaMemsetAsync(ctx->scan1.ticket, 0, 64 * sizeof(unsigned), ctx->ex.st));
+    ctx->ex.scan1 = &ctx->scan1;  // from here on every scan of this context takes one launch
+    ctx->ex.scan_err = ctx->err_flag;
     CK(cudaStreamSynchronize(ctx->ex.st));
     CK_LAUNCH();
     ctx->model_set = true;
@@ -1359,7 +1362,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     // incidence lists of the scored edges, grouped by node (slots claimed with integer atomics)
     std::unique_ptr<ProfScope> pinc(new ProfScope(ctx->ex, LP_PROF_INCIDENCE, (double)E * 2.0 * 24.0));
     if (ctx->mlp) incidence_count_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->inc_ptr);
-    exclusive_scan_i32_onepass(ctx->ex, ctx->inc_ptr, rows_out, ctx->inc_ptr, ctx->inc_cursor, ctx->inc_ptr + rows_out, ctx->scan1, ctx->err_flag, ctx->scan_tmp);
+    exclusive_scan_i32_copy(ctx->ex, ctx->inc_ptr, rows_out, ctx->inc_ptr, ctx->inc_cursor, ctx->inc_ptr + rows_out, ctx->scan_tmp);
     incidence_fill_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, g_pos, g_neg, ctx->inc_cursor, ctx->inc_col,
                                                    ctx->mlp ? nullptr : ctx->inc_val, ctx->mlp ? ctx->inc_edge : nullptr);
     ctx->ex.launches += 2;

@@ -22,10 +22,13 @@ struct Profiler {
     }
 };
 
+struct OnePassScan;
 struct Exec {
     cudaStream_t st = nullptr;
     int64_t launches = 0;
     Profiler prof;
+    OnePassScan *scan1 = nullptr;  // scratch of the one-launch scan (null: every scan takes three launches)
+    int *scan_err = nullptr;       // device word that receives bit 1 when a bounded wait of that scan expires
 };
 
 // Times everything enqueued on the stream between construction and destruction when the category
@@ -146,10 +149,14 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_apply_kernel(const int *__r
     if (out_total && blockIdx.x == gridDim.x - 1 && threadIdx.x == SCAN_THREADS - 1) *out_total = ex;
 }
 
+static bool scan_onepass_try(Exec &ex, const int *in, int64_t n, int *out, int *out_copy, int *out_total);
+
 // out[i] = sum_{j<i} in[j] for i in [0, n); if out_total != nullptr it receives the sum of all.
-// `tmp` needs ceil(n / SCAN_TILE) + 1 ints.  in == out is allowed.
+// `tmp` needs ceil(n / SCAN_TILE) + 1 ints.  in == out is allowed.  One launch when the context has the scratch of the
+// one-launch scan and the input fits it, else three.
 static void exclusive_scan_i32(Exec &ex, const int *in, int64_t n, int *out, int *out_total, int *tmp)
 {
+    if (n > 0 && scan_onepass_try(ex, in, n, out, nullptr, out_total)) return;
     if (n <= 0) {
         if (out_total) cudaMemsetAsync(out_total, 0, sizeof(int), ex.st);
         return;
@@ -266,24 +273,28 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_onepass_kernel(const int *_
     if (out_total && tile == gridDim.x - 1 && threadIdx.x == SCAN_THREADS - 1) *out_total = ex;
 }
 
-// out[i] = sum_{j<i} in[j]; out_copy (optional) receives the same values; *out_total (optional) the sum of all.
-// in == out is allowed.  Falls back to the three-launch scan when the scratch is too small.
-static void exclusive_scan_i32_onepass(Exec &ex, const int *in, int64_t n, int *out, int *out_copy, int *out_total, OnePassScan &sc, int *err, int *tmp)
+static bool scan_onepass_try(Exec &ex, const int *in, int64_t n, int *out, int *out_copy, int *out_total)
+{
+    OnePassScan *sc = ex.scan1;
+    const int64_t tiles = ceil_div64(n, SCAN_TILE);
+    if (!sc || !sc->status || tiles > sc->tiles_cap) return false;
+    sc->epoch = (sc->epoch + 1u) & 0x3fffffffu;
+    if (sc->epoch == 0) sc->epoch = 1;
+    scan_onepass_kernel<<<(unsigned)tiles, SCAN_THREADS, 0, ex.st>>>(in, n, out, out_copy, out_total, sc->status, sc->ticket, sc->epoch, ex.scan_err);
+    ex.launches += 1;
+    return true;
+}
+
+// the same scan with a second copy of the result (out_copy), as the incidence lists want it (offsets and cursors)
+static void exclusive_scan_i32_copy(Exec &ex, const int *in, int64_t n, int *out, int *out_copy, int *out_total, int *tmp)
 {
     if (n <= 0) {
         if (out_total) cudaMemsetAsync(out_total, 0, sizeof(int), ex.st);
         return;
     }
-    const int64_t tiles = ceil_div64(n, SCAN_TILE);
-    if (!sc.status || tiles > sc.tiles_cap) {
-        exclusive_scan_i32(ex, in, n, out, out_total, tmp);
-        if (out_copy) cudaMemcpyAsync(out_copy, out, sizeof(int) * (size_t)n, cudaMemcpyDeviceToDevice, ex.st);
-        return;
-    }
-    sc.epoch = (sc.epoch + 1u) & 0x3fffffffu;
-    if (sc.epoch == 0) sc.epoch = 1;
-    scan_onepass_kernel<<<(unsigned)tiles, SCAN_THREADS, 0, ex.st>>>(in, n, out, out_copy, out_total, sc.status, sc.ticket, sc.epoch, err);
-    ex.launches += 1;
+    if (scan_onepass_try(ex, in, n, out, out_copy, out_total)) return;
+    exclusive_scan_i32(ex, in, n, out, out_total, tmp);
+    cudaMemcpyAsync(out_copy, out, sizeof(int) * (size_t)n, cudaMemcpyDeviceToDevice, ex.st);
 }
 
 // ------------------------------------------------------------------------------------------

@@ -154,66 +154,116 @@ LP_DEVINL void spmm_accumulate(const SpmmArgs<T> &a, int e_lo, int e_hi, int gl,
         int my_col2 = 0;
         if (HAS_X2 && my_e < e_hi) my_col2 = __ldg(a.col2 + my_e);
         const int cnt = min(G, e_hi - e0);
-        int j = 0;
-        for (; j + U <= cnt; j += U) {
-            int c[U];
-            float w[U];
-            Vec16<T> v[U][NV];
-#pragma unroll
-            for (int q = 0; q < U; ++q) {
-                c[q] = __shfl_sync(gmask, my_col, j + q, G);
-                w[q] = (HAS_VAL ? __shfl_sync(gmask, my_val, j + q, G) : 1.f) * wscale;
-            }
-#pragma unroll
-            for (int q = 0; q < U; ++q)
-#pragma unroll
-                for (int i = 0; i < NV; ++i) v[q][i].load(a.X + (size_t)c[q] * a.ldx + min(gl + i * G, nchunks - 1) * VN);
-            if (HAS_X2) {
+        if constexpr (sizeof(ACC) == 8) {
+            // exact sums (batch incidence lists): full batches of U, then the rest one by one
+            int j = 0;
+            for (; j + U <= cnt; j += U) {
+                int c[U];
+                float w[U];
+                Vec16<T> v[U][NV];
 #pragma unroll
                 for (int q = 0; q < U; ++q) {
-                    const int c2 = __shfl_sync(gmask, my_col2, j + q, G);
-#pragma unroll
-                    for (int i = 0; i < NV; ++i) {
-                        const int ch = gl + i * G;
-                        if (ch < nchunks) {
-                            Vec16<T> v2;
-                            v2.load(a.X2 + (size_t)c2 * a.ldx2 + ch * VN);
-                            float f[VN], f2[VN];
-                            v[q][i].to_float(f);
-                            v2.to_float(f2);
-#pragma unroll
-                            for (int t = 0; t < VN; ++t) acc_add<ACC>(acc[i][t], w[q], f[t] * f2[t]);
-                        }
-                    }
+                    c[q] = __shfl_sync(gmask, my_col, j + q, G);
+                    w[q] = (HAS_VAL ? __shfl_sync(gmask, my_val, j + q, G) : 1.f) * wscale;
                 }
-            } else {
 #pragma unroll
                 for (int q = 0; q < U; ++q)
 #pragma unroll
-                    for (int i = 0; i < NV; ++i) acc_add_vec<T, ACC, HAS_VAL>(acc[i], w[q], v[q][i]);
-            }
-        }
-        for (; j < cnt; ++j) {
-            const int c = __shfl_sync(gmask, my_col, j, G);
-            const float w = (HAS_VAL ? __shfl_sync(gmask, my_val, j, G) : 1.f) * wscale;
-            const int c2 = HAS_X2 ? __shfl_sync(gmask, my_col2, j, G) : 0;
+                    for (int i = 0; i < NV; ++i) v[q][i].load(a.X + (size_t)c[q] * a.ldx + min(gl + i * G, nchunks - 1) * VN);
+                if (HAS_X2) {
 #pragma unroll
-            for (int i = 0; i < NV; ++i) {
-                const int ch = gl + i * G;
-                if (HAS_X2 ? ch < nchunks : true) {
-                    Vec16<T> v;
-                    v.load(a.X + (size_t)c * a.ldx + min(ch, nchunks - 1) * VN);
-                    if (HAS_X2) {
-                        Vec16<T> v2;
-                        v2.load(a.X2 + (size_t)c2 * a.ldx2 + ch * VN);
-                        float f[VN], f2[VN];
-                        v.to_float(f);
-                        v2.to_float(f2);
+                    for (int q = 0; q < U; ++q) {
+                        const int c2 = __shfl_sync(gmask, my_col2, j + q, G);
 #pragma unroll
-                        for (int t = 0; t < VN; ++t) acc_add<ACC>(acc[i][t], w, f[t] * f2[t]);
-                    } else {
-                        acc_add_vec<T, ACC, HAS_VAL>(acc[i], w, v);
+                        for (int i = 0; i < NV; ++i) {
+                            const int ch = gl + i * G;
+                            if (ch < nchunks) {
+                                Vec16<T> v2;
+                                v2.load(a.X2 + (size_t)c2 * a.ldx2 + ch * VN);
+                                float f[VN], f2[VN];
+                                v[q][i].to_float(f);
+                                v2.to_float(f2);
+#pragma unroll
+                                for (int t = 0; t < VN; ++t) acc_add<ACC>(acc[i][t], w[q], f[t] * f2[t]);
+                            }
+                        }
                     }
+                } else {
+#pragma unroll
+                    for (int q = 0; q < U; ++q)
+#pragma unroll
+                        for (int i = 0; i < NV; ++i) acc_add_vec<T, ACC, HAS_VAL>(acc[i], w[q], v[q][i]);
+                }
+            }
+            for (; j < cnt; ++j) {
+                const int c = __shfl_sync(gmask, my_col, j, G);
+                const float w = (HAS_VAL ? __shfl_sync(gmask, my_val, j, G) : 1.f) * wscale;
+                const int c2 = HAS_X2 ? __shfl_sync(gmask, my_col2, j, G) : 0;
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    const int ch = gl + i * G;
+                    if (HAS_X2 ? ch < nchunks : true) {
+                        Vec16<T> v;
+                        v.load(a.X + (size_t)c * a.ldx + min(ch, nchunks - 1) * VN);
+                        if (HAS_X2) {
+                            Vec16<T> v2;
+                            v2.load(a.X2 + (size_t)c2 * a.ldx2 + ch * VN);
+                            float f[VN], f2[VN];
+                            v.to_float(f);
+                            v2.to_float(f2);
+#pragma unroll
+                            for (int t = 0; t < VN; ++t) acc_add<ACC>(acc[i][t], w, f[t] * f2[t]);
+                        } else {
+                            acc_add_vec<T, ACC, HAS_VAL>(acc[i], w, v);
+                        }
+                    }
+                }
+            }
+        } else {
+            // U source rows are requested together whatever is left of the batch: a short batch (a row of one to three entries,
+            // the tail of a longer one) repeats its last entry in the unused slots -- a load that hits L1 -- and leaves the
+            // repeats out of the sum, so that it costs one memory round trip instead of one per entry
+            for (int j = 0; j < cnt; j += U) {
+                int c[U];
+                float w[U];
+                Vec16<T> v[U][NV];
+#pragma unroll
+                for (int q = 0; q < U; ++q) {
+                    const int src = min(j + q, cnt - 1);
+                    c[q] = __shfl_sync(gmask, my_col, src, G);
+                    w[q] = (HAS_VAL ? __shfl_sync(gmask, my_val, src, G) : 1.f) * wscale;
+                }
+#pragma unroll
+                for (int q = 0; q < U; ++q)
+#pragma unroll
+                    for (int i = 0; i < NV; ++i) v[q][i].load(a.X + (size_t)c[q] * a.ldx + min(gl + i * G, nchunks - 1) * VN);
+                if (HAS_X2) {
+#pragma unroll
+                    for (int q = 0; q < U; ++q) {
+                        const int c2 = __shfl_sync(gmask, my_col2, min(j + q, cnt - 1), G);
+                        if (j + q < cnt) {
+#pragma unroll
+                            for (int i = 0; i < NV; ++i) {
+                                const int ch = gl + i * G;
+                                if (ch < nchunks) {
+                                    Vec16<T> v2;
+                                    v2.load(a.X2 + (size_t)c2 * a.ldx2 + ch * VN);
+                                    float f[VN], f2[VN];
+                                    v[q][i].to_float(f);
+                                    v2.to_float(f2);
+#pragma unroll
+                                    for (int t = 0; t < VN; ++t) acc_add<ACC>(acc[i][t], w[q], f[t] * f2[t]);
+                                }
+                            }
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int q = 0; q < U; ++q)
+                        if (j + q < cnt) {
+#pragma unroll
+                            for (int i = 0; i < NV; ++i) acc_add_vec<T, ACC, HAS_VAL>(acc[i], w[q], v[q][i]);
+                        }
                 }
             }
         }
