@@ -39,9 +39,10 @@ K_NEG = 1
 SEED = 1234
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the aggregation launches of one step on the
-# benchmark workload, from one ncu capture of a whole step at full size: mean per timed launch.  Valid only for the
-# kernel source it was taken with (sha1 of csrc/spmm.cuh + csrc/common.cuh); reported as null otherwise.
-NCU_TRAFFIC = {"spmm_sha1": "897672ea779116af0d86a2a91421625fa1b531bd", "bytes_per_launch": (123.7e6 + 408.8e6 + 628.4e6) / 3.0}
+# benchmark workload, from one ncu capture of a whole step at full size (layer-1 forward 124.8 MB, layer-2 forward
+# 410.0 MB, adjoint 630.0 MB): mean per timed launch.  Valid only for the kernel source it was taken with (sha1 of
+# csrc/spmm.cuh + csrc/common.cuh); reported as null otherwise.
+NCU_TRAFFIC = {"spmm_sha1": "046a4394dabc84ca4e22d7519eb8b1e5991986a4", "bytes_per_launch": (124.8e6 + 410.0e6 + 630.0e6) / 3.0}
 
 
 def measured_peaks():
@@ -341,7 +342,7 @@ def bench_hbm_roofline(torch, pkg, wl, dev, hbm_peak, peak_kind):
     H = torch.randn(g.n, F, device=dev).to(torch.bfloat16)
     out = {"graph": "Chung-Lu, 1,000,000 nodes, mean degree 16", "entries": g.nnz, "width": F, "dtype": "bf16", "source_matrix_MB": g.n * F * es / 1e6,
            "peak": hbm_peak, "peak_source": f"of {peak_kind}", "unit": "GB/s", "bound": "hbm"}
-    for name, transpose in (("forward", False), ("adjoint", True)):
+    for name, transpose in (("forward", False), ("adjoint_with_coefficients", True)):  # the operator-level adjoint carries 1/|N(v)| per entry
         for _ in range(3):
             ctx.op_aggregate("sage", H, transpose=transpose)
         torch.cuda.synchronize()
