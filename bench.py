@@ -42,7 +42,9 @@ SEED = 1234
 # benchmark workload, from one ncu capture of a whole step at full size (layer-1 forward 124.8 MB, layer-2 forward
 # 410.0 MB, adjoint 630.0 MB): mean per timed launch.  Valid only for the kernel source it was taken with (sha1 of
 # csrc/spmm.cuh + csrc/common.cuh); reported as null otherwise.
-NCU_TRAFFIC = {"spmm_sha1": "046a4394dabc84ca4e22d7519eb8b1e5991986a4", "bytes_per_launch": (124.8e6 + 410.0e6 + 630.0e6) / 3.0}
+NCU_TRAFFIC = {"spmm_sha1": "046a4394dabc84ca4e22d7519eb8b1e5991986a4", "bytes_per_launch": (124.8e6 + 410.0e6 + 630.0e6) / 3.0,
+               # the forward mean aggregation (F = 256, BF16) on the 1 M-node graph of the HBM-bound roofline run: 3416.3 MB read + 559.9 MB written
+               "hbm_forward_bytes_per_launch": 3416.3e6 + 559.9e6}
 
 
 def measured_peaks():
@@ -341,7 +343,8 @@ def bench_hbm_roofline(torch, pkg, wl, dev, hbm_peak, peak_kind):
     F, es = 256, 2
     H = torch.randn(g.n, F, device=dev).to(torch.bfloat16)
     out = {"graph": "Chung-Lu, 1,000,000 nodes, mean degree 16", "entries": g.nnz, "width": F, "dtype": "bf16", "source_matrix_MB": g.n * F * es / 1e6,
-           "peak": hbm_peak, "peak_source": f"of {peak_kind}", "unit": "GB/s", "bound": "hbm"}
+           "peak": hbm_peak, "peak_source": f"of {peak_kind}", "unit": "GB/s", "bound": "hbm",
+           "note": "time includes the combine launch of the hub rows; dram_frac = ncu DRAM bytes of the launch / live time / peak"}
     for name, transpose in (("forward", False), ("adjoint_with_coefficients", True)):  # the operator-level adjoint carries 1/|N(v)| per entry
         for _ in range(3):
             ctx.op_aggregate("sage", H, transpose=transpose)
@@ -362,6 +365,11 @@ def bench_hbm_roofline(torch, pkg, wl, dev, hbm_peak, peak_kind):
         out[name] = {"us_per_launch": us, "launches": 20, "gather_bytes": gather, "compulsory_bytes": compulsory,
                      "achieved_gather": gather / us / 1e3, "frac_gather": gather / us / 1e3 / hbm_peak,
                      "achieved_compulsory": compulsory / us / 1e3, "frac_compulsory": compulsory / us / 1e3 / hbm_peak}
+        if not transpose:  # DRAM traffic of this launch from ncu (valid for the kernel source it was captured with)
+            traffic = NCU_TRAFFIC["hbm_forward_bytes_per_launch"] if NCU_TRAFFIC["spmm_sha1"] == spmm_source_hash() else None
+            out[name]["traffic"] = traffic
+            out[name]["dram_achieved"] = traffic / us / 1e3 if traffic else None
+            out[name]["dram_frac"] = traffic / us / 1e3 / hbm_peak if traffic else None
     ctx.close()
     return out
 
