@@ -596,7 +596,7 @@ def main():
         hu = torch.from_numpy(pos[0]).pin_memory()
         hv = torch.from_numpy(pos[1]).pin_memory()
         loss_h = torch.zeros(1).pin_memory()
-        n_e2e = max(3, min(args.steps, 200))
+        n_e2e = max(50, min(args.steps, 200))  # at least 50 steps: the first ones still warm the pinned-copy path up
         t_base = args.warmup + args.steps + 100
         du_stage = torch.empty(B, dtype=torch.int32, device=dev)
         dv_stage = torch.empty(B, dtype=torch.int32, device=dev)

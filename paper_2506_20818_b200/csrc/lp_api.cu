@@ -415,7 +415,7 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
     convert_kernel<float, bf16><<<nblk(n * (int64_t)f), 256, 0, st>>>(ctx->X32, ctx->X16, n * (int64_t)f);
     ctx->ex.launches += 6;
     // heavy-row plans of the graph and of its transpose (static: built once)
-    const int64_t item_cap = nnz / SPMM_HEAVY_MIN + 2;
+    const int64_t item_cap = nnz / 64 + 2;  // static plans cut rows above 128 entries into pieces of 128 or items of 512: at most deg / 64 of them per row
     const int static_threshold = 128;  // measured best on a 200k-node power-law graph (64: 282 us, 128: 249 us, 256: 241 us at F=256; 176 / 163 / 193 us at F=128)
     GALLOC(ctx->heavy_partials, item_cap * 512);
     for (HeavyPlan *hp : {&ctx->plan_csr, &ctx->plan_csc}) {
@@ -910,7 +910,7 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
         MALLOC(hp.item_row, cap);
         MALLOC(hp.item_first, cap);
         MALLOC(hp.counts, 64);
-        if (cap > ctx->nnz / SPMM_HEAVY_MIN + 2) {
+        if (cap > ctx->nnz / 64 + 2) {  // larger than the partial rows allocated with the graph
             MALLOC(hp.partials, cap * 512);
         } else {
             hp.partials = ctx->heavy_partials;
@@ -1375,6 +1375,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         SpmmArgs<T> a;
         a.heavy = ctx->plan_dyn;
         a.heavy.partials = ctx->inc_partials;
+
         a.nnz = 2 * E;
         a.n_rows = rows_out;
         a.rowptr = ctx->inc_ptr;

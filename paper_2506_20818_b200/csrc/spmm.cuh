@@ -33,7 +33,7 @@ struct HeavyPlan {
     int *rows = nullptr, *base = nullptr, *item_row = nullptr, *item_first = nullptr, *counts = nullptr;
     float *partials = nullptr;
     int host_rows = -1, host_items = -1;  // -1: unknown on the host (plan built on the device per launch)
-    int threshold = 64;                   // rows with more entries than this are heavy (>= SPMM_HEAVY_MIN)
+    int threshold = 32;                   // rows with more entries than this are heavy (>= SPMM_HEAVY_MIN)
     int seg = 512;                        // entries per item (SPMM_SEG; SPMM_PIECE for the padded form's own plan)
     // Static structures only: every row again in padded form for spmm_padded_kernel.  A row is cut into pieces of at
     // most SPMM_PIECE entries (one piece unless it is heavy), a piece into groups of four entries (a pad repeats the
@@ -120,7 +120,7 @@ template <typename ACC> LP_DEVINL float acc_value(ACC a);
 template <> LP_DEVINL float acc_value<float>(float a) { return a; }
 // one rounding (64-bit integer to FP32, to nearest); the epilogue multiplies by the exact power-of-two 1 / scale
 template <> LP_DEVINL float acc_value<long long>(long long a) { return __ll2float_rn(a); }
-constexpr int SPMM_HEAVY_MIN = 64;  // smallest heavy-row threshold a plan may use (bounds the item count by nnz / 64).
+constexpr int SPMM_HEAVY_MIN = 32;  // smallest heavy-row threshold a plan may use (bounds the item count by nnz / 32).
                                     // A lane group keeps only a few gathers in flight, so a long row handled by one
                                     // group is a long dependent chain: long rows are cut into items instead.
 constexpr int SPMM_ITEM_BLOCKS = 1184;  // blocks that walk the item list (grid-stride)
@@ -332,15 +332,17 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
     const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << (lane & ~(unsigned)(G - 1)));
     const int nchunks = a.F / VN;  // 16-byte chunks per row
 
-    if ((int)blockIdx.x >= light_blocks) {
+    const int item_blocks = (int)gridDim.x - light_blocks;
+    if ((int)blockIdx.x < item_blocks) {
         // ---- heavy item: SPMM_SEG consecutive entries of a hub row, one contiguous piece per lane group,
-        // pieces added in group order (fixed), FP32 partial row written for the combine kernel
+        // pieces added in group order (fixed), FP32 partial row written for the combine kernel.  The item blocks come
+        // FIRST in the grid: they are the longest chains of dependent gathers, so they start before the light rows
         const int n_items = a.heavy.counts[1];
-        for (int item = blockIdx.x - light_blocks; item < n_items; item += gridDim.x - light_blocks) {
+        for (int item = blockIdx.x; item < n_items; item += item_blocks) {
         const int r = a.heavy.item_row[item];
         const int sidx = item - a.heavy.item_first[item];
         const int hb = a.rowptr[r] + sidx * a.heavy.seg, he = min(a.rowptr[r + 1], hb + a.heavy.seg);
-        const int piece = ((he - hb + NG - 1) / NG + G - 1) / G * G;
+        const int piece = ((he - hb + NG - 1) / NG + U - 1) / U * U;
         const int lo = min(he, hb + g * piece), hi = min(he, lo + piece);
         ACC hacc[NV][VN];
 #pragma unroll
@@ -362,7 +364,7 @@ __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const Spmm
         }
         return;
     }
-    const int row0 = blockIdx.x * ROWS;
+    const int row0 = ((int)blockIdx.x - item_blocks) * ROWS;
     if (row0 >= n_rows) return;
     for (int i = threadIdx.x; i <= ROWS; i += SPMM_THREADS) s_ptr[i] = a.rowptr[min(row0 + i, n_rows)];
     __syncthreads();
