@@ -168,9 +168,10 @@ edge_score_bce_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const 
 
 // The common case (one negative per positive that shares the positive's source, rows of at most 32 vectors): a warp
 // takes two positives and requests their six rows together before it reduces any, which halves the number of
-// dependent memory round trips per scored edge.  Scores, gradients and incidence counts are those of
-// edge_score_bce_kernel bit for bit (same order of multiply-adds and the same reduction tree); a block's loss
-// partial covers 16 positives instead of 8.
+// dependent memory round trips per scored edge.  The four dot products of the warp are reduced together (lane i of
+// every group of four ends up with the sum of value i: 8 shuffles instead of 20) and their losses and gradients are
+// evaluated side by side, one score per lane, instead of one after the other on every lane: the kernel is bound by
+// instruction issue, not by memory.  A block's loss partial covers 16 positives.
 template <typename T>
 __global__ void __launch_bounds__(EDGE_THREADS)
 edge_score_bce_pair_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const int *__restrict__ idmap, const int *__restrict__ pos_src,
@@ -203,32 +204,45 @@ edge_score_bce_pair_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, c
             rv[p].load(H + (size_t)v[p] * ldh + ch * VN);
             rn[p].load(H + (size_t)vn[p] * ldh + ch * VN);
         }
+        // d[2p] = <h_u, h_v> and d[2p + 1] = <h_u, h_v'> of positive p, this lane's 16 bytes of each
+        float d[4];
 #pragma unroll
         for (int p = 0; p < P; ++p) {
-            float dp = 0.f, dn = 0.f;
-            if (active) {
-                dp = dot_vec<T>(ru[p], rv[p], 0.f);
-                dn = dot_vec<T>(ru[p], rn[p], 0.f);
-            }
-            dp = warp_sum(dp);
-            dn = warp_sum(dn);
-            float ell_p, dls_p, ell_n, dls_n;
-            bce_logits(dp, 1.f, ell_p, dls_p);
-            bce_logits(dn, 0.f, ell_n, dls_n);
-            if (j0 + p < B) {
-                loss += ell_p;
-                loss += ell_n;
-                if (lane == 0) {
-                    g_pos[j0 + p] = dls_p * inv_N;
-                    g_neg[j0 + p] = dls_n * inv_N;
-                    if (inc_counts) {
-                        atomicAdd(&inc_counts[u[p]], 2);  // source of the positive and of its negative
-                        atomicAdd(&inc_counts[v[p]], 1);
-                        atomicAdd(&inc_counts[vn[p]], 1);
-                    }
-                }
+            d[2 * p] = active ? dot_vec<T>(ru[p], rv[p], 0.f) : 0.f;
+            d[2 * p + 1] = active ? dot_vec<T>(ru[p], rn[p], 0.f) : 0.f;
+        }
+        // four sums at once: after two exchange steps lane l holds value (l & 3) summed over the lanes l, l ^ 1, l ^ 2, l ^ 3;
+        // three butterfly steps over the lanes with equal (l & 3) finish it
+        {
+            const bool hi1 = (lane & 1) != 0;
+            const float a0 = hi1 ? d[0] : d[1], k0 = hi1 ? d[1] : d[0];
+            const float a1 = hi1 ? d[2] : d[3], k1 = hi1 ? d[3] : d[2];
+            const float e0 = k0 + __shfl_xor_sync(0xffffffffu, a0, 1);  // lanes with bit 0 clear keep values 0 and 2, the others 1 and 3
+            const float e1 = k1 + __shfl_xor_sync(0xffffffffu, a1, 1);
+            const bool hi2 = (lane & 2) != 0;
+            const float give = hi2 ? e0 : e1, keep = hi2 ? e1 : e0;
+            float sum = keep + __shfl_xor_sync(0xffffffffu, give, 2);      // lane l: value (l & 1) + 2 * ((l >> 1) & 1)
+            sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+            sum += __shfl_xor_sync(0xffffffffu, sum, 8);
+            sum += __shfl_xor_sync(0xffffffffu, sum, 16);
+            // lane l < 4 now evaluates score l: positive p = l >> 1, label 1 for even l (the positive), 0 for odd l (its negative)
+            const int p = (lane >> 1) & 1;
+            const bool is_pos = (lane & 1) == 0;
+            float ell, dls;
+            bce_logits(sum, is_pos ? 1.f : 0.f, ell, dls);
+            if (lane < 4 && j0 + p < B) {
+                loss = ell;
+                (is_pos ? g_pos : g_neg)[j0 + p] = dls * inv_N;
             }
         }
+        if (lane < P && j0 + lane < B && inc_counts) {  // lane p counts the endpoints of positive p and of its negative
+            const int up = lane == 0 ? u[0] : u[1], vp = lane == 0 ? v[0] : v[1], np_ = lane == 0 ? vn[0] : vn[1];
+            atomicAdd(&inc_counts[up], 2);  // source of the positive and of its negative
+            atomicAdd(&inc_counts[vp], 1);
+            atomicAdd(&inc_counts[np_], 1);
+        }
+        loss += __shfl_xor_sync(0xffffffffu, loss, 1);  // the warp's four losses (the other lanes hold 0)
+        loss += __shfl_xor_sync(0xffffffffu, loss, 2);
     }
     if (lane == 0) s_loss[warp] = loss;
     __syncthreads();
