@@ -186,6 +186,11 @@ struct TcGemmParams {
     int relu;
     const float *row_scale;  // [M] or null: columns >= scale_col0 of row m are multiplied by row_scale[m]
     int scale_col0;          // (the 1 / |N(v)| of the mean adjoint, folded into the input-gradient transform)
+    // pair kernel only.  Sign bits of the output, one 32-bit word per row and 32 columns, word (c / 32) * M + row, column
+    // c of the 32 at bit (c / 2) + 16 * (c % 2) (the order in which packed BF16 pairs give them up): mask_out receives
+    // "stored BF16 value > 0" (with relu), mask_in zeroes the outputs whose bit is clear (ReLU backward)
+    uint32_t *mask_out;
+    const uint32_t *mask_in;
     bf16 *C;            // output (BF16) when out_f32 == null
     int64_t ldc;
     float *out_f32;     // FP32 partial output [gridDim.z][M + colsum, N] (weight gradient)
@@ -594,7 +599,8 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
                 const int row_t = q * 32 + lane;  // row inside the tile
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN);
                 const bool store_thread = (((warp - 2) & 3) == 0 && lane == 0);  // one per box group (warps 2 and 6)
-                const float rs = (p.row_scale && (int64_t)m0 + row_t < p.M) ? __ldg(p.row_scale + m0 + row_t) : 1.f;
+                const bool row_ok = (int64_t)m0 + row_t < p.M;
+                const float rs = (p.row_scale && row_ok) ? __ldg(p.row_scale + m0 + row_t) : 1.f;
                 for (int half = 0; half < BN; half += 128) {
                     const int nbox = min(2, (BN - half) / 64);
                     // the two box groups (four warps, one 64-column staging box each) run independently: a group waits
@@ -873,7 +879,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TCP_THREADS, 1)
                 const int row_t = q * 32 + lane;
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN);
                 const bool store_thread = (((warp - 2) & 3) == 0 && lane == 0);
-                const float rs = (p.row_scale && (int64_t)m0 + row_t < p.M) ? __ldg(p.row_scale + m0 + row_t) : 1.f;
+                const bool row_ok = (int64_t)m0 + row_t < p.M;
+                const float rs = (p.row_scale && row_ok) ? __ldg(p.row_scale + m0 + row_t) : 1.f;
                 for (int half = 0; half < BN; half += 128) {
                     const int nbox = min(2, (BN - half) / 64);
                     if (my_box < nbox) {
@@ -905,13 +912,31 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TCP_THREADS, 1)
 #pragma unroll
                                 for (int j = 0; j < 32; ++j) v[j] *= rs;
                             }
+                            if (p.mask_in) {
+                                const uint32_t keep = row_ok ? __ldg(p.mask_in + (size_t)((n0 + c0) >> 5) * (size_t)p.M + (size_t)(m0 + row_t)) : 0u;
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) v[j] = ((keep >> ((j >> 1) + 16 * (j & 1))) & 1u) ? v[j] : 0.f;
+                            }
                             const int chunk0 = 4 * h2;
+                            uint32_t positive = 0;
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
                                 Vec16<bf16> o;
                                 o.from_float(v + 8 * j);
                                 *reinterpret_cast<uint4 *>(box + (((chunk0 + j) ^ (row_t & 7)) << 4)) = o.v;
+                                if (p.mask_out) {
+                                    // a stored value is positive exactly when its magnitude bits are not all zero (the ReLU left no
+                                    // negative ones): adding 0x7fff carries into bit 15 of each half of a packed pair
+                                    const uint32_t w4[4] = {o.v.x, o.v.y, o.v.z, o.v.w};
+#pragma unroll
+                                    for (int t = 0; t < 4; ++t) {
+                                        const int k = 4 * j + t;  // packed pair k holds columns 2 k and 2 k + 1 of these 32
+                                        const uint32_t carry = ((w4[t] & 0x7fff7fffu) + 0x7fff7fffu) >> (15 - k);
+                                        positive |= carry & ((1u << k) | (1u << (16 + k)));
+                                    }
+                                }
                             }
+                            if (p.mask_out && row_ok) p.mask_out[(size_t)((n0 + c0) >> 5) * (size_t)p.M + (size_t)(m0 + row_t)] = positive;
                         }
                         fence_async_proxy();
                         group_barrier(my_box);
@@ -1052,12 +1077,20 @@ static int tc_sm_count()
     return sms;
 }
 
+// whether tc_gemm_kmajor runs this shape on pairs of SMs (the only kernel that reads and writes the sign-bit words)
+static bool tc_pair_applies(int64_t M, int N, int K) { return tc_pair_bn(N, K) > 0 && M >= 64 * TC_BM && tc_sm_count() >= 4; }
+
 static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const bf16 *A, int64_t lda, const bf16 *Bt, const float *bias, bool relu,
-                           bf16 *C, int64_t ldc, std::string &err, const float *row_scale = nullptr, int scale_col0 = 0)
+                           bf16 *C, int64_t ldc, std::string &err, const float *row_scale = nullptr, int scale_col0 = 0, uint32_t *mask_out = nullptr,
+                           const uint32_t *mask_in = nullptr)
 {
     // pairs of SMs: a slice of up to 256 columns whose half (per CTA) fits 128 KiB; worth it from a few hundred tiles on
     const int pair_bn = tc_pair_bn(N, K);
-    if (pair_bn > 0 && M >= 64 * TC_BM && tc_sm_count() >= 4) {
+    if ((mask_out || mask_in) && !(tc_pair_applies(M, N, K) && (!mask_out || relu))) {
+        err = "sign-bit words need the pair kernel (and a ReLU when they are written)";
+        return false;
+    }
+    if (tc_pair_applies(M, N, K)) {
         CUtensorMap mapA, mapB, mapC;
         if (!tc_make_map(tc, &mapA, A, M, K, lda, TC_BK, TC_BM, err)) return false;
         if (!tc_make_map(tc, &mapB, Bt, N, K, K, TC_BK, pair_bn / 2, err)) return false;
@@ -1069,6 +1102,7 @@ static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const
         p.stages = (int)std::max<int64_t>(2, std::min<int64_t>(TCP_MAX_STAGES, (smem_cap - w_bytes - TCP_STAGE_OUT_BYTES) / (TC_BM * TC_BK * 2)));
         p.bias = bias; p.relu = relu ? 1 : 0; p.C = C; p.ldc = ldc; p.out_f32 = nullptr; p.err = tc.err_word;
         p.row_scale = row_scale; p.scale_col0 = scale_col0;
+        p.mask_out = mask_out; p.mask_in = mask_in;
         p.wait_ns = tc.wait_limit_ns; p.extra_tx = tc.overdeclare_tx; tc.overdeclare_tx = 0;
         const int n_slices = N / pair_bn;
         const int64_t m_tiles = ceil_div64(M, 2 * TC_BM);

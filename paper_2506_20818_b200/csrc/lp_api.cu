@@ -128,6 +128,15 @@ struct lp_ctx {
     int64_t last_exhausted = 0;
     TcState tc;                         // tensor-core GEMM state (descriptor encoder, device error word)
     bf16 *w16 = nullptr, *w16t = nullptr;  // BF16 path: the parameter vector of the current call as BF16, as is and with every weight matrix transposed
+    bf16 *w16s = nullptr;                  // ... and with the SAGE layers' [W_self ; W_neigh] stored side by side (see weights_cache_kernel)
+    // One-pass SAGE layers l >= 1 on the tensor-core pair kernel take the input gradient as
+    // dH^(l) = relu'(H^(l)) * ([dZ | A^T dZ / deg] [W_self^T ; W_neigh^T]): the adjoint aggregation runs on dZ (no self term, no mask),
+    // the transform reads the two halves side by side and applies the ReLU mask from sign-bit words the forward transform left.
+    bool cat_grad[LP_MAX_LAYERS] = {};
+    uint32_t *relu_bits[LP_MAX_LAYERS] = {};  // [Fi / 32][n] words of layer l's input H^(l)
+    void *dcat[2] = {nullptr, nullptr};       // [n, 2 * max Fo] gradient operands (dZ | adjoint aggregate)
+    const void *out_grad = nullptr;           // where the last step left dL/dH^(K), and its row pitch
+    int out_grad_ld = 0;
 };
 
 static thread_local std::string g_create_error;  // errors of calls that have no context: one per host thread
@@ -319,7 +328,10 @@ static void drop_model(lp_ctx *ctx)
     ctx->hk_valid = false;
     ctx->ex.scan1 = nullptr;
     ctx->scan1 = OnePassScan();
-    ctx->w16 = ctx->w16t = nullptr;
+    ctx->w16 = ctx->w16t = ctx->w16s = nullptr;
+    for (int l = 0; l < LP_MAX_LAYERS; ++l) { ctx->cat_grad[l] = false; ctx->relu_bits[l] = nullptr; }
+    ctx->dcat[0] = ctx->dcat[1] = nullptr;
+    ctx->out_grad = nullptr;
     for (auto &l : ctx->layer) l = LayerBuf();
     for (auto &h : ctx->hop) h = HopBlock();
 }
@@ -481,6 +493,16 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
         hp->pcol = reinterpret_cast<const int4 *>(pcol);
         hp->pval = reinterpret_cast<const float4 *>(pval);
         hp->pval_src = sv;
+        if (!csr) {  // the transposed structure also carries the mean's coefficients 1 / |N(v)| of the entry's source row v
+            float *pval2 = nullptr;
+            GALLOC(pval2, 4 * n_groups + 4);
+            padded_fill_kernel<<<nblk(n), 256, 0, st>>>(sp, sc, ctx->meanT_val, (int)n, SPMM_PIECE, first_group, chunk_count, chunk_of, row_base, chunk_start, pcol, pval2, grow);
+            ctx->ex.launches += 1;
+            e = cudaStreamSynchronize(st);
+            if (e != cudaSuccess) break;
+            hp->pval2 = reinterpret_cast<const float4 *>(pval2);
+            hp->pval2_src = ctx->meanT_val;
+        }
         hp->grow = grow;
         hp->chunk_start = chunk_start;
         hp->n_chunks = n_groups > 0 ? n_chunks : 0;
@@ -849,6 +871,23 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
     if (d->prec == LP_BF16) {
         MALLOC(ctx->w16, ctx->n_params);
         MALLOC(ctx->w16t, ctx->n_params);
+        // layers whose input gradient is taken as aggregate-then-transform (see cat_grad): the widths must suit the pair
+        // kernel in both directions and the padded adjoint, and aggregating dZ (Fo wide) must not cost more than
+        // aggregating the transformed gradient (Fi wide)
+        int max_fo = 0;
+        for (int l = 1; l < K && sage && !sampled; ++l) {
+            const LayerBuf &L = ctx->layer[l], &P = ctx->layer[l - 1];
+            if (L.Fo <= L.Fi && L.Fi % 32 == 0 && ctx->plan_csc.pval2 && tc_linear_supported(2 * L.Fo, L.Fi) && tc_pair_applies(n, L.Fi, 2 * L.Fo) &&
+                tc_linear_supported(P.Kin, P.Fo) && tc_pair_applies(n, P.Fo, P.Kin)) {
+                ctx->cat_grad[l] = true;
+                MALLOC(ctx->relu_bits[l], (int64_t)(L.Fi / 32) * n);
+                max_fo = std::max(max_fo, L.Fo);
+            }
+        }
+        if (max_fo > 0) {
+            MALLOC(ctx->w16s, ctx->n_params);
+            for (int i = 0; i < 2; ++i) { MALLOC(p, n * 2 * (int64_t)max_fo * es); ctx->dcat[i] = p; }
+        }
     }
 
     // per-step sort capacity: incidence lists and (sampled) block transposes
@@ -979,25 +1018,31 @@ static void cache_weights(lp_ctx *ctx, const float *params)
 {
     if (ctx->desc.prec != LP_BF16 || !ctx->w16) return;
     WeightBlocks wb{};
-    for (int k = 0; k < ctx->K; ++k) { wb.off[wb.count] = ctx->layer[k].off_w; wb.kin[wb.count] = ctx->layer[k].Kin; wb.fo[wb.count] = ctx->layer[k].Fo; ++wb.count; }
+    for (int k = 0; k < ctx->K; ++k) {
+        wb.off[wb.count] = ctx->layer[k].off_w; wb.kin[wb.count] = ctx->layer[k].Kin; wb.fo[wb.count] = ctx->layer[k].Fo;
+        wb.split[wb.count] = ctx->cat_grad[k] ? ctx->layer[k].Fi : 0;
+        ++wb.count;
+    }
     if (ctx->mlp)
         for (int j = 0; j < 2; ++j) { wb.off[wb.count] = ctx->pred[j].off_w; wb.kin[wb.count] = ctx->pred[j].Kin; wb.fo[wb.count] = ctx->pred[j].Fo; ++wb.count; }
-    weights_cache_kernel<<<nblk(ctx->n_params), 256, 0, ctx->ex.st>>>(params, ctx->n_params, wb, ctx->w16, ctx->w16t);
+    weights_cache_kernel<<<nblk(ctx->n_params), 256, 0, ctx->ex.st>>>(params, ctx->n_params, wb, ctx->w16, ctx->w16t, ctx->w16s);
     ctx->ex.launches += 1;
 }
 
 // dense transform of one layer: Out = act(A W + b)
 template <typename T>
-static lp_status layer_linear(lp_ctx *ctx, int64_t rows, const LayerBuf &L, const float *params, T *out, int ldo, bool relu)
+static lp_status layer_linear(lp_ctx *ctx, int64_t rows, const LayerBuf &L, const float *params, T *out, int ldo, bool relu, uint32_t *sign_bits = nullptr)
 {
     if (rows <= 0) return LP_OK;
     ProfScope prof(ctx->ex, LP_PROF_GEMM_FWD, gemm_bytes((double)rows, L.Fo, L.Kin, sizeof(T), sizeof(T)), 2.0 * rows * L.Fo * L.Kin);
     if (sizeof(T) == 2 && tc_linear_supported(L.Kin, L.Fo)) {
         std::string err;  // Out = A W: the K-major GEMM reads W^T [Fo, Kin] from the transposed BF16 copy
-        if (!tc_gemm_kmajor(ctx->tc, ctx->ex, rows, L.Fo, L.Kin, (const bf16 *)L.A, L.Kin, ctx->w16t + L.off_w, params + L.off_b, relu, (bf16 *)out, ldo, err))
+        if (!tc_gemm_kmajor(ctx->tc, ctx->ex, rows, L.Fo, L.Kin, (const bf16 *)L.A, L.Kin, ctx->w16t + L.off_w, params + L.off_b, relu, (bf16 *)out, ldo, err, nullptr, 0,
+                            sign_bits))
             return fail(ctx, LP_ECUDA, "tensor-core GEMM: " + err);
         return LP_OK;
     }
+    if (sign_bits) return fail(ctx, LP_ESTATE, "sign-bit words asked of a transform that does not run on the tensor cores");
     gemm_simt<T, float, T, false, true>(ctx->ex, rows, L.Fo, L.Kin, (const T *)L.A, L.Kin, params + L.off_w, L.Fo, out, ldo, params + L.off_b, relu ? 1 : 0);
     return LP_OK;
 }
@@ -1007,24 +1052,24 @@ static lp_status layer_linear(lp_ctx *ctx, int64_t rows, const LayerBuf &L, cons
 // multiplied by row_scale = 1 / |N(v)| on the way out, so the adjoint aggregation needs no per-entry
 // coefficient: dH[u] = sum over v with u in N(v) of dA_mean[v] / |N(v)|.
 template <typename T>
-static lp_status layer_input_grad(lp_ctx *ctx, int64_t rows, const LayerBuf &L, const float *params, const T *dZ, T *dA, const float *row_scale,
+static lp_status layer_input_grad(lp_ctx *ctx, int64_t rows, const LayerBuf &L, const float *params, const T *dZ, int ldz, T *dA, const float *row_scale,
                                   int scale_col0)
 {
     if (rows <= 0) return LP_OK;
     ProfScope prof(ctx->ex, LP_PROF_GEMM_DGRAD, gemm_bytes((double)rows, L.Kin, L.Fo, sizeof(T), sizeof(T)), 2.0 * rows * L.Fo * L.Kin);
     if (sizeof(T) == 2 && tc_linear_supported(L.Fo, L.Kin)) {
         std::string err;  // dA = dZ W^T: W [Kin, Fo] as stored is the [N, K] operand
-        if (!tc_gemm_kmajor(ctx->tc, ctx->ex, rows, L.Kin, L.Fo, (const bf16 *)dZ, L.Fo, ctx->w16 + L.off_w, nullptr, false, (bf16 *)dA, L.Kin, err, row_scale,
+        if (!tc_gemm_kmajor(ctx->tc, ctx->ex, rows, L.Kin, L.Fo, (const bf16 *)dZ, ldz, ctx->w16 + L.off_w, nullptr, false, (bf16 *)dA, L.Kin, err, row_scale,
                             scale_col0))
             return fail(ctx, LP_ECUDA, "tensor-core GEMM: " + err);
         return LP_OK;
     }
-    gemm_simt<T, float, T, false, false>(ctx->ex, rows, L.Kin, L.Fo, dZ, L.Fo, params + L.off_w, L.Fo, dA, L.Kin, nullptr, 0, row_scale, scale_col0);
+    gemm_simt<T, float, T, false, false>(ctx->ex, rows, L.Kin, L.Fo, dZ, ldz, params + L.off_w, L.Fo, dA, L.Kin, nullptr, 0, row_scale, scale_col0);
     return LP_OK;
 }
 
 template <typename T>
-static lp_status layer_weight_grad(lp_ctx *ctx, int64_t rows, const LayerBuf &L, const T *dZ, float *grads, int accumulate)
+static lp_status layer_weight_grad(lp_ctx *ctx, int64_t rows, const LayerBuf &L, const T *dZ, int ldz, float *grads, int accumulate)
 {
     if (rows <= 0) {
         if (!accumulate) cudaMemsetAsync(grads + L.off_w, 0, sizeof(float) * ((size_t)L.Kin * L.Fo + L.Fo), ctx->ex.st);
@@ -1035,14 +1080,14 @@ static lp_status layer_weight_grad(lp_ctx *ctx, int64_t rows, const LayerBuf &L,
         std::string err;
         // the bias gradient follows the weights in the flat vector: one launch pair produces both
         const bool fuse_bias = L.off_b == L.off_w + (int64_t)L.Kin * L.Fo;
-        if (!tc_weight_grad(ctx->tc, ctx->ex, rows, L.Kin, L.Fo, (const bf16 *)L.A, L.Kin, (const bf16 *)dZ, L.Fo, grads + L.off_w, accumulate, ctx->partials, err,
+        if (!tc_weight_grad(ctx->tc, ctx->ex, rows, L.Kin, L.Fo, (const bf16 *)L.A, L.Kin, (const bf16 *)dZ, ldz, grads + L.off_w, accumulate, ctx->partials, err,
                             fuse_bias))
             return fail(ctx, LP_ECUDA, "tensor-core GEMM: " + err);
         if (fuse_bias) return LP_OK;
     } else {
-        weight_grad_simt<T>(ctx->ex, rows, L.Kin, L.Fo, (const T *)L.A, L.Kin, dZ, L.Fo, grads + L.off_w, accumulate, ctx->partials);
+        weight_grad_simt<T>(ctx->ex, rows, L.Kin, L.Fo, (const T *)L.A, L.Kin, dZ, ldz, grads + L.off_w, accumulate, ctx->partials);
     }
-    colsum<T>(ctx->ex, dZ, rows, L.Fo, L.Fo, grads + L.off_b, accumulate, ctx->partials);
+    colsum<T>(ctx->ex, dZ, rows, L.Fo, ldz, grads + L.off_b, accumulate, ctx->partials);
     return LP_OK;
 }
 
@@ -1235,7 +1280,7 @@ template <typename T> static lp_status forward_impl(lp_ctx *ctx, const float *pa
             if (rows > 0 && !spmm_launch<T>(ctx->ex, a)) return fail(ctx, LP_EUNSUPPORTED, "aggregation width not supported");
             if (k == 0 && !ctx->sampled) ctx->input_agg_valid = true;  // AGG(X) stays in layer 1's operand buffer
         }
-        lp_status s = layer_linear<T>(ctx, rows, L, params, out, ldo, k < K - 1);
+        lp_status s = layer_linear<T>(ctx, rows, L, params, out, ldo, k < K - 1, (k < K - 1 && ctx->cat_grad[k + 1]) ? ctx->relu_bits[k + 1] : nullptr);
         if (s != LP_OK) return s;
     }
     ctx->rows_out = ctx->sampled ? ctx->hop[0].n_src : n;
@@ -1288,15 +1333,15 @@ static lp_status predictor_backward(lp_ctx *ctx, const float *params, int64_t E,
     reduce_partials_short_kernel<<<nblk(Hp + 1, 32), 256, 0, st>>>(ctx->partials, Hp + 1, splits, grads + ctx->off_w2, accumulate);
     pred_out_grad_kernel<T><<<nblk(E * Hp), 256, 0, st>>>(P2, Hp, E, g, params + ctx->off_w2, dPa);
     ctx->ex.launches += 3;
-    lp_status s = layer_weight_grad<T>(ctx, E, ctx->pred[1], dPa, grads, accumulate);
+    lp_status s = layer_weight_grad<T>(ctx, E, ctx->pred[1], dPa, ctx->pred[1].Fo, grads, accumulate);
     if (s != LP_OK) return s;
-    s = layer_input_grad<T>(ctx, E, ctx->pred[1], params, dPa, dPb, nullptr, 0);
+    s = layer_input_grad<T>(ctx, E, ctx->pred[1], params, dPa, ctx->pred[1].Fo, dPb, nullptr, 0);
     if (s != LP_OK) return s;
     relu_mask_kernel<T><<<nblk(E * Hp), 256, 0, st>>>(dPb, P1, E * Hp);
     ctx->ex.launches += 1;
-    s = layer_weight_grad<T>(ctx, E, ctx->pred[0], dPb, grads, accumulate);
+    s = layer_weight_grad<T>(ctx, E, ctx->pred[0], dPb, ctx->pred[0].Fo, grads, accumulate);
     if (s != LP_OK) return s;
-    s = layer_input_grad<T>(ctx, E, ctx->pred[0], params, dPb, dZ0, nullptr, 0);
+    s = layer_input_grad<T>(ctx, E, ctx->pred[0], params, dPb, ctx->pred[0].Fo, dZ0, nullptr, 0);
     if (s != LP_OK) return s;
     CK_LAUNCH();
     return LP_OK;
@@ -1369,8 +1414,13 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     pinc.reset();
 
     // dL/dH^(K)[v] = sum over incident scored edges of g_e * h_other
+    // (a layer that aggregates its gradient before the transform keeps dZ as the left half of a [rows, 2 Fo] operand)
+    int cur = 1, cat_cur = 0;
     T *dZ = tptr<T>(ctx->dHK);
-    int cur = 1;
+    int ldz = D;
+    if (K >= 2 && ctx->cat_grad[K - 1]) { dZ = tptr<T>(ctx->dcat[cat_cur]); ldz = 2 * D; }
+    ctx->out_grad = dZ;
+    ctx->out_grad_ld = ldz;
     {
         SpmmArgs<T> a;
         a.heavy = ctx->plan_dyn;
@@ -1384,7 +1434,12 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         a.ldx = D;
         a.F = D;
         a.Y = dZ;
-        a.ldy = D;
+        a.ldy = ldz;
+        if (K >= 2 && ctx->cat_grad[K - 1]) {  // the adjoint of the mean gathers dZ[v] / |N(v)|: written here, beside dZ, so that it needs no coefficients
+            a.Y2 = tptr<T>(ctx->dHK);
+            a.ldy2 = D;
+            a.y2_scale = ctx->inv_deg;
+        }
         // Scale of the exact sum.  Every coefficient carries the 1 / N of the mean loss, so the products are of the order
         // |h| / N: the power-of-two scale is 2^s * 2^ceil(log2 N) with s = min(32, 50 - ceil(log2 N)), which resolves a
         // product to 2^-s relative to |h| / N whatever the batch size.  The coefficients of one node add up to at most 1
@@ -1414,14 +1469,53 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     for (int l = K - 1; l >= 0; --l) {
         LayerBuf &L = ctx->layer[l];
         const int64_t rows = ctx->sampled ? ctx->hop[K - l].n_dst : ctx->n;
-        s = layer_weight_grad<T>(ctx, rows, L, dZ, grads, accumulate);
+        s = layer_weight_grad<T>(ctx, rows, L, dZ, ldz, grads, accumulate);
         if (s != LP_OK) return s;
         if (l == 0) break;
+        // where the gradient of this layer's input goes: the next layer down may want it as the left half of its own operand
+        T *dZn = tptr<T>(ctx->dZ[cur ^ 1]);
+        int ldn = L.Fi;
+        if (l >= 2 && ctx->cat_grad[l - 1]) { dZn = tptr<T>(ctx->dcat[cat_cur ^ 1]); ldn = 2 * L.Fi; }
+        if (ctx->cat_grad[l]) {
+            // dH^(l) = relu'(H^(l)) * ([dZ | A^T (dZ / deg)] [W_self^T ; W_neigh^T]): aggregate first (plain epilogue, no self
+            // term), then one transform over both halves with the ReLU mask taken from the forward transform's sign bits
+            if constexpr (sizeof(T) == 2) {
+                SpmmArgs<T> a;
+                a.heavy = ctx->plan_csc;
+                a.nnz = ctx->nnz;
+                a.n_rows = ctx->n;
+                a.rowptr = ctx->colptr;
+                a.col = ctx->rowidx;
+                a.F = L.Fo;
+                if (l == K - 1) {  // the top layer's dZ / |N(v)| was written beside dZ
+                    a.X = tptr<T>(ctx->dHK);
+                    a.ldx = L.Fo;
+                } else {           // below it the mean's coefficients ride with the entries
+                    a.val = ctx->meanT_val;
+                    a.X = dZ;
+                    a.ldx = ldz;
+                }
+                a.Y = dZ + L.Fo;
+                a.ldy = ldz;
+                {
+                    ProfScope prof(ctx->ex, LP_PROF_AGG_BWD, spmm_bytes(a, ctx->nnz), 2.0 * ctx->nnz * L.Fo);
+                    if (!spmm_launch<T>(ctx->ex, a)) return fail(ctx, LP_EUNSUPPORTED, "aggregation width not supported");
+                }
+                ProfScope prof(ctx->ex, LP_PROF_GEMM_DGRAD, gemm_bytes((double)rows, L.Fi, 2 * L.Fo, sizeof(T), sizeof(T)), 4.0 * rows * L.Fo * L.Fi);
+                std::string err;
+                if (!tc_gemm_kmajor(ctx->tc, ctx->ex, rows, L.Fi, 2 * L.Fo, (const bf16 *)dZ, ldz, ctx->w16s + L.off_w, nullptr, false, (bf16 *)dZn, ldn, err, nullptr, 0,
+                                    nullptr, ctx->relu_bits[l]))
+                    return fail(ctx, LP_ECUDA, "tensor-core GEMM: " + err);
+            }
+            dZ = dZn;
+            ldz = ldn;
+            if (l >= 2 && ctx->cat_grad[l - 1]) cat_cur ^= 1; else cur ^= 1;
+            continue;
+        }
         T *dA = tptr<T>(ctx->dA);
         const float *mean_scale = sage ? (ctx->sampled ? ctx->hop[K - l].inv_deg : ctx->inv_deg) : nullptr;
-        s = layer_input_grad<T>(ctx, rows, L, params, dZ, dA, mean_scale, L.Fi);
+        s = layer_input_grad<T>(ctx, rows, L, params, dZ, ldz, dA, mean_scale, L.Fi);
         if (s != LP_OK) return s;
-        T *dZn = tptr<T>(ctx->dZ[cur ^ 1]);
         SpmmArgs<T> a;
         if (!ctx->sampled) {
             a.heavy = ctx->plan_csc;
@@ -1432,7 +1526,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         }
         a.F = L.Fi;
         a.Y = dZn;
-        a.ldy = L.Fi;
+        a.ldy = ldn;
         if (!ctx->sampled) {
             a.n_rows = ctx->n;
             a.rowptr = ctx->colptr;
@@ -1480,7 +1574,8 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
             if (a.n_rows > 0 && !spmm_launch<T>(ctx->ex, a)) return fail(ctx, LP_EUNSUPPORTED, "aggregation width not supported");
         }
         dZ = dZn;
-        cur ^= 1;
+        ldz = ldn;
+        if (l >= 2 && ctx->cat_grad[l - 1]) cat_cur ^= 1; else cur ^= 1;
     }
     CK_LAUNCH();
     return LP_OK;
@@ -1727,8 +1822,8 @@ extern "C" lp_status lp_get_output_gradient(lp_ctx *ctx, float *out)
     if (!ctx->model_set || !ctx->have_grad) return fail(ctx, LP_ESTATE, "lp_get_output_gradient: run lp_train_step first");
     CK(cudaSetDevice(ctx->device));
     const int D = ctx->desc.dims[ctx->K];
-    if (ctx->desc.prec == LP_BF16) to_f32<bf16>(ctx, (const bf16 *)ctx->dHK, D, out, ctx->rows_out, D);
-    else to_f32<float>(ctx, (const float *)ctx->dHK, D, out, ctx->rows_out, D);
+    if (ctx->desc.prec == LP_BF16) to_f32<bf16>(ctx, (const bf16 *)ctx->out_grad, ctx->out_grad_ld, out, ctx->rows_out, D);
+    else to_f32<float>(ctx, (const float *)ctx->out_grad, ctx->out_grad_ld, out, ctx->rows_out, D);
     CK_LAUNCH();
     return LP_OK;
 }

@@ -58,12 +58,15 @@ __global__ void weights_to_bf16_kernel(const float *__restrict__ W, int K, int N
 // BF16 copies of a whole flat parameter vector in one launch: `asis` element for element, and `transposed` with every
 // weight matrix W[Kin, Fo] (row-major, at offset off) stored as its transpose [Fo, Kin] at the same offset (biases are
 // copied in place in both).  The forward transforms read the transposed blocks, the input-gradient transforms the others.
+// `stacked` (optional): a block with split = Fi > 0 holds W = [W_self ; W_neigh] (2 Fi rows); it is stored as
+// [Fi, 2 Fo] with row n = (W_self[n, :] | W_neigh[n, :]), the [N, K] operand of dH = [dZ | A^T dZ] [W_self^T ; W_neigh^T].
 struct WeightBlocks {
     int count;
     long long off[8];
-    int kin[8], fo[8];
+    int kin[8], fo[8], split[8];
 };
-__global__ void weights_cache_kernel(const float *__restrict__ params, long long n, WeightBlocks blocks, bf16 *__restrict__ asis, bf16 *__restrict__ transposed)
+__global__ void weights_cache_kernel(const float *__restrict__ params, long long n, WeightBlocks blocks, bf16 *__restrict__ asis, bf16 *__restrict__ transposed,
+                                     bf16 *__restrict__ stacked)
 {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
@@ -77,6 +80,10 @@ __global__ void weights_cache_kernel(const float *__restrict__ params, long long
             if (r >= 0 && r < (long long)blocks.kin[b] * blocks.fo[b]) {
                 const int k = (int)(r / blocks.fo[b]), c = (int)(r - (long long)k * blocks.fo[b]);
                 dst = blocks.off[b] + (long long)c * blocks.kin[b] + k;
+                if (stacked && blocks.split[b] > 0) {
+                    const int half = k / blocks.split[b], row = k - half * blocks.split[b];
+                    stacked[blocks.off[b] + (long long)row * (2 * blocks.fo[b]) + half * blocks.fo[b] + c] = x;
+                }
             }
         }
     }

@@ -46,6 +46,8 @@ struct HeavyPlan {
     const int4 *pcol = nullptr;
     const float4 *pval = nullptr;
     const float *pval_src = nullptr;      // the per-entry coefficient array pval was padded from
+    const float4 *pval2 = nullptr;        // a second padded coefficient array of the same structure
+    const float *pval2_src = nullptr;
     const int *grow = nullptr;
     const int *chunk_start = nullptr;
     int n_chunks = 0;
@@ -77,6 +79,9 @@ template <typename T> struct SpmmArgs {
     const int *self_idx = nullptr;
     T *self_out = nullptr;
     int ldself = 0;
+    T *Y2 = nullptr;             // optional second copy of the output, row r multiplied by y2_scale[r] (row-per-group kernel only)
+    int ldy2 = 0;
+    const float *y2_scale = nullptr;
     int64_t nnz = 0;             // stored entries (host-known upper bound), sizes the heavy-row part of the grid
     // exact (64-bit fixed-point) sums only: every product is multiplied by exact_scale, a power of two chosen by the caller
     // from the magnitude of the coefficients, before it is rounded to an integer; the sum is multiplied by exact_inv = 1 / exact_scale
@@ -309,6 +314,13 @@ LP_DEVINL void spmm_epilogue(const SpmmArgs<T> &a, int r, int gl, int nchunks, c
         Vec16<T> out;
         out.from_float(o);
         out.store_once(a.Y + (size_t)r * a.ldy + ch * VN);
+        if (a.Y2) {  // gathered by the next launch: an ordinary store
+            const float s2 = __ldg(a.y2_scale + r);
+#pragma unroll
+            for (int t = 0; t < VN; ++t) o[t] *= s2;
+            out.from_float(o);
+            out.store(a.Y2 + (size_t)r * a.ldy2 + ch * VN);
+        }
         if (srow >= 0) {
             Vec16<T> v;
             v.load(a.X + (size_t)srow * a.ldx + ch * VN);
@@ -677,9 +689,11 @@ template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC> sta
     // static structure with a padded plan and source rows G or 2 G vectors apart: the padded kernel walks every row
     if constexpr (NV == 1 && sizeof(ACC) == 4) {
         const int pitch = a.ldx / Vec16<T>::N;
-        if (a.heavy.pcol != nullptr && a.heavy.n_chunks > 0 && !a.X2 && !a.self_out && !a.n_rows_dev && !a.init_idx && a.ldx % Vec16<T>::N == 0 &&
-            (pitch == G || pitch == 2 * G) && (a.val == nullptr || (a.val == a.heavy.pval_src && a.heavy.pval != nullptr))) {
+        if (a.heavy.pcol != nullptr && a.heavy.n_chunks > 0 && !a.X2 && !a.self_out && !a.Y2 && !a.n_rows_dev && !a.init_idx && a.ldx % Vec16<T>::N == 0 &&
+            (pitch == G || pitch == 2 * G) &&
+            (a.val == nullptr || (a.val == a.heavy.pval_src && a.heavy.pval != nullptr) || (a.val == a.heavy.pval2_src && a.heavy.pval2 != nullptr))) {
             SpmmArgs<T> b = a;
+            if (a.val && a.val != a.heavy.pval_src) b.heavy.pval = a.heavy.pval2;
             b.heavy.rows = a.heavy.p_rows;
             b.heavy.base = a.heavy.p_base;
             b.heavy.counts = a.heavy.p_counts;
@@ -688,7 +702,7 @@ template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC> sta
             const bool plain = !a.init && !a.relu_ref;
             const bool self_mask = a.init && a.relu_ref && !a.init_coef && !a.row_scale && !a.val;
 #define LP_PADDED(MULT_, VAL_) do { \
-                if (plain) spmm_padded_kernel<T, G, MULT_, 6, VAL_, 1><<<pgrid, SPMM_THREADS, 0, ex.st>>>(b); \
+                if (plain) spmm_padded_kernel<T, G, MULT_, VAL_ ? 5 : 6, VAL_, 1><<<pgrid, SPMM_THREADS, 0, ex.st>>>(b); \
                 else if (self_mask) spmm_padded_kernel<T, G, MULT_, 5, false, 2><<<pgrid, SPMM_THREADS, 0, ex.st>>>(b); \
                 else spmm_padded_kernel<T, G, MULT_, 5, VAL_, 0><<<pgrid, SPMM_THREADS, 0, ex.st>>>(b); } while (0)
             if (pitch == G) {

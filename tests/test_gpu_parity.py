@@ -378,6 +378,22 @@ def test_config2_chunglu_sage(pkg, prec):
     assert_within(err, TOL[prec])
 
 
+@pytest.mark.parametrize("dims", [[64, 128, 128, 64], [64, 64, 128, 128]])
+def test_sage3_one_pass_on_the_pair_kernel(pkg, dims):
+    # Three SAGE layers over 9,001 nodes (35 row tiles of 256 and a ragged one) in BF16: every transform runs on pairs of
+    # SMs, and each layer whose output is not wider than its input takes its input gradient as aggregate-then-transform (the
+    # adjoint aggregation of dZ beside dZ, one transform over both halves, the ReLU mask from the forward pass's sign
+    # bits).  First shape: both upper layers, chained through the two operand buffers; second shape: the top layer only (the
+    # middle layer widens 64 -> 128 and keeps transform-then-aggregate), so the two forms of the input gradient follow one another.
+    g = wl.chung_lu(9001, 14.0, 2.1, seed=21)
+    X = wl.node_features(g.n, dims[0], 3)
+    params = wl.glorot_params("sage", dims, 5, 0.05)
+    u, v = wl.undirected_edge_list(g)
+    sel = np.random.default_rng(1).choice(len(u), 5000, replace=False)
+    err, _, _ = run_step(pkg, g, X, params, "sage", dims, "bf16", (u[sel], v[sel]))
+    assert_within(err, TOL["bf16"])
+
+
 @pytest.mark.parametrize("prec", ["fp32", "bf16"])
 def test_config3_coauthor_gcn3_weighted(pkg, prec):
     g, X, params, pos, cfg = wl.make_config("c3_coauthor_gcn3", scale=0.04)
