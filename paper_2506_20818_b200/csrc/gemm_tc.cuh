@@ -191,6 +191,7 @@ struct TcGemmParams {
     // "stored BF16 value > 0" (with relu), mask_in zeroes the outputs whose bit is clear (ReLU backward)
     uint32_t *mask_out;
     const uint32_t *mask_in;
+    int out_sets;            // pair kernel: 1 or 2 pairs of output staging boxes (a box is refilled once the stores before the latest one or three have read theirs)
     bf16 *C;            // output (BF16) when out_f32 == null
     int64_t ldc;
     float *out_f32;     // FP32 partial output [gridDim.z][M + colsum, N] (weight gradient)
@@ -464,6 +465,9 @@ LP_DEVINL void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y)
 }
 LP_DEVINL void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 LP_DEVINL void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+LP_DEVINL void tma_store_wait_read_but_one() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+LP_DEVINL void tma_store_wait_read_but_three() { asm volatile("cp.async.bulk.wait_group.read 3;" ::: "memory"); }
+LP_DEVINL void box_barrier() { asm volatile("bar.sync 2, 256;" ::: "memory"); }  // the eight epilogue warps, around one staging box
 LP_DEVINL void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 LP_DEVINL void epilogue_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }  // the eight epilogue warps only
 LP_DEVINL void group_barrier(int grp) { asm volatile("bar.sync %0, 128;" ::"r"(2 + grp) : "memory"); }  // the four warps of one box group
@@ -866,7 +870,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TCP_THREADS, 1)
         } else if (warp >= 2) {
             // ---- epilogue (as in kernel 2, on this CTA's 128 rows; the drained accumulator is reported to the leader)
             const int q = warp & 3;
-            const int my_box = (warp - 2) >> 2;
+            const int hsel = (warp - 2) >> 2;  // which 32 columns of a 64-column staging box this warp fills
+            const uint32_t n_boxes = 2u * (uint32_t)p.out_sets;  // staging boxes, filled in turn by all eight warps
+            uint32_t n_stores = 0;
             for (int64_t i = 0; i < my_tiles; ++i) {
                 const int b = (int)(i & 1);
                 bool ready = mbar_wait(smem_u32(&bar_acc_full[b]), (uint32_t)((i >> 1) & 1), p.wait_ns);
@@ -878,70 +884,70 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TCP_THREADS, 1)
                 const int m0 = (int)((first_tile + i * stride) * (2 * TC_BM)) + (int)rank * TC_BM;
                 const int row_t = q * 32 + lane;
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN);
-                const bool store_thread = (((warp - 2) & 3) == 0 && lane == 0);
+                const bool store_thread = (warp == 2 && lane == 0);
                 const bool row_ok = (int64_t)m0 + row_t < p.M;
                 const float rs = (p.row_scale && row_ok) ? __ldg(p.row_scale + m0 + row_t) : 1.f;
                 for (int half = 0; half < BN; half += 128) {
-                    const int nbox = min(2, (BN - half) / 64);
-                    if (my_box < nbox) {
-                        if (store_thread) tma_store_wait_read();
-                        group_barrier(my_box);
-                        const int cb = half + my_box * 64;
-                        uint32_t r[2][32];
-                        tmem_ld_32x32_issue(taddr + (uint32_t)cb, r[0]);
-                        tmem_ld_32x32_issue(taddr + (uint32_t)(cb + 32), r[1]);
-                        tmem_ld_wait();
-                        uint8_t *box = smem_out + (size_t)my_box * 16384 + (size_t)row_t * 128;
+                    uint32_t r[2][32];
+                    tmem_ld_32x32_issue(taddr + (uint32_t)(half + 32 * hsel), r[0]);
+                    tmem_ld_32x32_issue(taddr + (uint32_t)(half + 64 + 32 * hsel), r[1]);
+                    tmem_ld_wait();
 #pragma unroll
-                        for (int h2 = 0; h2 < 2; ++h2) {
-                            const int c0 = cb + 32 * h2;
-                            float v[32];
+                    for (int h2 = 0; h2 < 2; ++h2) {
+                        // the box about to be filled has been read by the store that used it last: all but the n_boxes - 1 latest are done
+                        if (store_thread) { if (n_boxes == 4) tma_store_wait_read_but_three(); else tma_store_wait_read_but_one(); }
+                        box_barrier();
+                        const uint32_t box_id = n_stores & (n_boxes - 1u);
+                        ++n_stores;
+                        const int cb = half + 64 * h2;    // first column of the box
+                        const int c0 = cb + 32 * hsel;    // first of this thread's 32 columns
+                        uint8_t *box = smem_out + (size_t)box_id * 16384 + (size_t)row_t * 128;
+                        float v[32];
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4) {
-                                const float4 bb = *reinterpret_cast<const float4 *>(&s_bias[c0 + j]);
-                                v[j] = __uint_as_float(r[h2][j]) + bb.x;
-                                v[j + 1] = __uint_as_float(r[h2][j + 1]) + bb.y;
-                                v[j + 2] = __uint_as_float(r[h2][j + 2]) + bb.z;
-                                v[j + 3] = __uint_as_float(r[h2][j + 3]) + bb.w;
-                            }
-                            if (p.relu) {
+                        for (int j = 0; j < 32; j += 4) {
+                            const float4 bb = *reinterpret_cast<const float4 *>(&s_bias[c0 + j]);
+                            v[j] = __uint_as_float(r[h2][j]) + bb.x;
+                            v[j + 1] = __uint_as_float(r[h2][j + 1]) + bb.y;
+                            v[j + 2] = __uint_as_float(r[h2][j + 2]) + bb.z;
+                            v[j + 3] = __uint_as_float(r[h2][j + 3]) + bb.w;
+                        }
+                        if (p.relu) {
 #pragma unroll
-                                for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
-                            }
-                            if (p.row_scale && n0 + c0 >= p.scale_col0) {
+                            for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
+                        }
+                        if (p.row_scale && n0 + c0 >= p.scale_col0) {
 #pragma unroll
-                                for (int j = 0; j < 32; ++j) v[j] *= rs;
-                            }
-                            if (p.mask_in) {
-                                const uint32_t keep = row_ok ? __ldg(p.mask_in + (size_t)((n0 + c0) >> 5) * (size_t)p.M + (size_t)(m0 + row_t)) : 0u;
+                            for (int j = 0; j < 32; ++j) v[j] *= rs;
+                        }
+                        if (p.mask_in) {
+                            const uint32_t keep = row_ok ? __ldg(p.mask_in + (size_t)((n0 + c0) >> 5) * (size_t)p.M + (size_t)(m0 + row_t)) : 0u;
 #pragma unroll
-                                for (int j = 0; j < 32; ++j) v[j] = ((keep >> ((j >> 1) + 16 * (j & 1))) & 1u) ? v[j] : 0.f;
-                            }
-                            const int chunk0 = 4 * h2;
-                            uint32_t positive = 0;
+                            for (int j = 0; j < 32; ++j) v[j] = ((keep >> ((j >> 1) + 16 * (j & 1))) & 1u) ? v[j] : 0.f;
+                        }
+                        const int chunk0 = 4 * hsel;
+                        uint32_t positive = 0;
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                Vec16<bf16> o;
-                                o.from_float(v + 8 * j);
-                                *reinterpret_cast<uint4 *>(box + (((chunk0 + j) ^ (row_t & 7)) << 4)) = o.v;
-                                if (p.mask_out) {
-                                    // a stored value is positive exactly when its magnitude bits are not all zero (the ReLU left no
-                                    // negative ones): adding 0x7fff carries into bit 15 of each half of a packed pair
-                                    const uint32_t w4[4] = {o.v.x, o.v.y, o.v.z, o.v.w};
+                        for (int j = 0; j < 4; ++j) {
+                            Vec16<bf16> o;
+                            o.from_float(v + 8 * j);
+                            *reinterpret_cast<uint4 *>(box + (((chunk0 + j) ^ (row_t & 7)) << 4)) = o.v;
+                            if (p.mask_out) {
+                                // a stored value is positive exactly when its magnitude bits are not all zero (the ReLU left no
+                                // negative ones): adding 0x7fff carries into bit 15 of each half of a packed pair
+                                const uint32_t w4[4] = {o.v.x, o.v.y, o.v.z, o.v.w};
 #pragma unroll
-                                    for (int t = 0; t < 4; ++t) {
-                                        const int k = 4 * j + t;  // packed pair k holds columns 2 k and 2 k + 1 of these 32
-                                        const uint32_t carry = ((w4[t] & 0x7fff7fffu) + 0x7fff7fffu) >> (15 - k);
-                                        positive |= carry & ((1u << k) | (1u << (16 + k)));
-                                    }
+                                for (int t = 0; t < 4; ++t) {
+                                    const int k = 4 * j + t;  // packed pair k holds columns 2 k and 2 k + 1 of these 32
+                                    const uint32_t carry = ((w4[t] & 0x7fff7fffu) + 0x7fff7fffu) >> (15 - k);
+                                    positive |= carry & ((1u << k) | (1u << (16 + k)));
                                 }
                             }
-                            if (p.mask_out && row_ok) p.mask_out[(size_t)((n0 + c0) >> 5) * (size_t)p.M + (size_t)(m0 + row_t)] = positive;
                         }
+                        if (p.mask_out && row_ok) p.mask_out[(size_t)((n0 + c0) >> 5) * (size_t)p.M + (size_t)(m0 + row_t)] = positive;
                         fence_async_proxy();
-                        group_barrier(my_box);
+                        box_barrier();
                         if (store_thread) {
-                            tma_store_2d(&mapC, smem_u32(smem_out + (size_t)my_box * 16384), n0 + half + my_box * 64, m0);
+                            tma_store_2d(&mapC, smem_u32(smem_out + (size_t)box_id * 16384), n0 + cb, m0);
                             tma_store_commit();
                         }
                     }
@@ -952,7 +958,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TCP_THREADS, 1)
             }
         }
     }
-    if ((warp == 2 || warp == 6) && lane == 0) tma_store_wait_all();
+    if (warp == 2 && lane == 0) tma_store_wait_all();
     __syncwarp();
     tc_fence_before();
     __syncthreads();
@@ -1099,7 +1105,10 @@ static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const
         const int64_t smem_cap = 225 * 1024 + 512 - 1024;
         const int64_t w_bytes = (int64_t)(K / TC_BK) * (pair_bn / 2) * 128;  // this CTA's half of the slice
         p.M = M; p.N = N; p.K = K; p.BN = pair_bn;
-        p.stages = (int)std::max<int64_t>(2, std::min<int64_t>(TCP_MAX_STAGES, (smem_cap - w_bytes - TCP_STAGE_OUT_BYTES) / (TC_BM * TC_BK * 2)));
+        // a second set of output staging boxes where six A stages still fit beside it
+        p.out_sets = (smem_cap - w_bytes - 2 * TCP_STAGE_OUT_BYTES) / (TC_BM * TC_BK * 2) >= 6 ? 2 : 1;
+        const int64_t out_bytes = (int64_t)p.out_sets * TCP_STAGE_OUT_BYTES;
+        p.stages = (int)std::max<int64_t>(2, std::min<int64_t>(TCP_MAX_STAGES, (smem_cap - w_bytes - out_bytes) / (TC_BM * TC_BK * 2)));
         p.bias = bias; p.relu = relu ? 1 : 0; p.C = C; p.ldc = ldc; p.out_f32 = nullptr; p.err = tc.err_word;
         p.row_scale = row_scale; p.scale_col0 = scale_col0;
         p.mask_out = mask_out; p.mask_in = mask_in;
@@ -1108,7 +1117,7 @@ static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const
         const int64_t m_tiles = ceil_div64(M, 2 * TC_BM);
         int64_t pairs = std::min<int64_t>((int64_t)tc_sm_count() / 2, m_tiles * n_slices);
         pairs = std::max<int64_t>(n_slices, pairs / n_slices * n_slices);  // a whole number of pairs per slice
-        const size_t smem = (size_t)w_bytes + (size_t)p.stages * TC_BM * TC_BK * 2 + TCP_STAGE_OUT_BYTES + 1024;
+        const size_t smem = (size_t)w_bytes + (size_t)p.stages * TC_BM * TC_BK * 2 + (size_t)out_bytes + 1024;
         tc_linear_pair_kernel<<<(unsigned)(2 * pairs), TCP_THREADS, smem, ex.st>>>(mapA, mapB, mapC, p);
         ex.launches += 1;
         return true;
