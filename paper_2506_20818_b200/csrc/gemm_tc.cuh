@@ -875,19 +875,31 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TCP_THREADS, 1)
             uint32_t n_stores = 0;
             for (int64_t i = 0; i < my_tiles; ++i) {
                 const int b = (int)(i & 1);
+                const int m0 = (int)((first_tile + i * stride) * (2 * TC_BM)) + (int)rank * TC_BM;
+                const int row_t = q * 32 + lane;
+                const bool row_ok = (int64_t)m0 + row_t < p.M;
+                // per-row operands of the epilogue are requested before the accumulator is waited for
+                const float rs = (p.row_scale && row_ok) ? __ldg(p.row_scale + m0 + row_t) : 1.f;
+                uint32_t keep4[4] = {0u, 0u, 0u, 0u};  // sign-bit words of this thread's (up to) four 32-column chunks of the tile
+                if (p.mask_in && row_ok) {
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const int c = 128 * (t >> 1) + 64 * (t & 1) + 32 * hsel;
+                        if (c < BN) keep4[t] = __ldg(p.mask_in + (size_t)((n0 + c) >> 5) * (size_t)p.M + (size_t)(m0 + row_t));
+                    }
+                }
                 bool ready = mbar_wait(smem_u32(&bar_acc_full[b]), (uint32_t)((i >> 1) & 1), p.wait_ns);
                 if (!ready && lane == 0) { atomicExch(p.err, 3); *abort_flag = 1; }
                 if (!__all_sync(0xffffffffu, ready) && lane == 0) *abort_flag = 1;
                 epilogue_barrier();
                 if (*abort_flag != 0) break;
                 tc_fence_after();
-                const int m0 = (int)((first_tile + i * stride) * (2 * TC_BM)) + (int)rank * TC_BM;
-                const int row_t = q * 32 + lane;
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN);
                 const bool store_thread = (warp == 2 && lane == 0);
-                const bool row_ok = (int64_t)m0 + row_t < p.M;
-                const float rs = (p.row_scale && row_ok) ? __ldg(p.row_scale + m0 + row_t) : 1.f;
-                for (int half = 0; half < BN; half += 128) {
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int half = 128 * hh;
+                    if (half >= BN) break;
                     uint32_t r[2][32];
                     tmem_ld_32x32_issue(taddr + (uint32_t)(half + 32 * hsel), r[0]);
                     tmem_ld_32x32_issue(taddr + (uint32_t)(half + 64 + 32 * hsel), r[1]);
@@ -920,7 +932,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TCP_THREADS, 1)
                             for (int j = 0; j < 32; ++j) v[j] *= rs;
                         }
                         if (p.mask_in) {
-                            const uint32_t keep = row_ok ? __ldg(p.mask_in + (size_t)((n0 + c0) >> 5) * (size_t)p.M + (size_t)(m0 + row_t)) : 0u;
+                            const uint32_t keep = keep4[2 * hh + h2];
 #pragma unroll
                             for (int j = 0; j < 32; ++j) v[j] = ((keep >> ((j >> 1) + 16 * (j & 1))) & 1u) ? v[j] : 0.f;
                         }
