@@ -436,6 +436,7 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
         GALLOC(hp->base, item_cap);
         GALLOC(hp->item_row, item_cap);
         GALLOC(hp->item_first, item_cap);
+        GALLOC(hp->nseg, item_cap);
         GALLOC(hp->counts, 64);
         hp->partials = ctx->heavy_partials;
         hp->threshold = static_threshold;
@@ -456,6 +457,7 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
         HeavyPlan pp;
         GALLOC(pp.rows, item_cap);
         GALLOC(pp.base, item_cap);
+        GALLOC(pp.nseg, item_cap);
         GALLOC(pp.counts, 64);
         TALLOC(pp.item_row, item_cap);
         TALLOC(pp.item_first, item_cap);
@@ -509,6 +511,7 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
         hp->p_rows = pp.rows;
         hp->p_base = pp.base;
         hp->p_counts = pp.counts;
+        hp->p_nseg = pp.nseg;
         hp->p_host_rows = ctx->host_counts[10];
     }
 #undef TALLOC
@@ -948,6 +951,7 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
         MALLOC(hp.base, cap);
         MALLOC(hp.item_row, cap);
         MALLOC(hp.item_first, cap);
+        MALLOC(hp.nseg, cap);
         MALLOC(hp.counts, 64);
         if (cap > ctx->nnz / 64 + 2) {  // larger than the partial rows allocated with the graph
             MALLOC(hp.partials, cap * 512);

@@ -31,6 +31,7 @@
 // static structure (host_rows >= 0 tells the launcher the counts) or refilled per launch.
 struct HeavyPlan {
     int *rows = nullptr, *base = nullptr, *item_row = nullptr, *item_first = nullptr, *counts = nullptr;
+    int *nseg = nullptr;                  // optional: items of heavy row i (saves the combine kernel the row-offset round trip)
     float *partials = nullptr;
     int host_rows = -1, host_items = -1;  // -1: unknown on the host (plan built on the device per launch)
     int threshold = 32;                   // rows with more entries than this are heavy (>= SPMM_HEAVY_MIN)
@@ -51,7 +52,7 @@ struct HeavyPlan {
     const int *grow = nullptr;
     const int *chunk_start = nullptr;
     int n_chunks = 0;
-    int *p_rows = nullptr, *p_base = nullptr, *p_counts = nullptr;
+    int *p_rows = nullptr, *p_base = nullptr, *p_counts = nullptr, *p_nseg = nullptr;
     int p_host_rows = 0;
 };
 
@@ -622,6 +623,7 @@ __global__ void spmm_heavy_plan_kernel(const int *__restrict__ rowptr, int n_row
     const int b = atomicAdd(&hp.counts[1], nseg);
     hp.rows[i] = r;
     hp.base[i] = b;
+    if (hp.nseg) hp.nseg[i] = nseg;
     if (row_base) row_base[r] = b;
     for (int s = 0; s < nseg; ++s) {
         hp.item_row[b + s] = r;
@@ -640,30 +642,34 @@ __global__ void __launch_bounds__(SPMM_THREADS) spmm_heavy_combine_kernel(const 
     const int nchunks = a.F / VN;
     for (int i = blockIdx.x * NG + g; i < count; i += gridDim.x * NG) {
         const int r = a.heavy.rows[i], b = a.heavy.base[i];
-        const int nseg = (a.rowptr[r + 1] - a.rowptr[r] + a.heavy.seg - 1) / a.heavy.seg;
+        const int nseg = a.heavy.nseg ? a.heavy.nseg[i] : (a.rowptr[r + 1] - a.rowptr[r] + a.heavy.seg - 1) / a.heavy.seg;
         ACC acc[NV][VN];
 #pragma unroll
         for (int q = 0; q < NV; ++q)
 #pragma unroll
             for (int t = 0; t < VN; ++t) acc[q][t] = ACC(0);
-        // four partial rows are fetched before any is added (the additions stay in item order)
+        // a batch of partial rows is fetched before any is added (the additions stay in item order); a batch that reaches
+        // past the row's last item fetches nothing there and adds zero, so that a short row is one round trip, not one per item
         int s = 0;
         if constexpr (NV == 1) {
+            constexpr int W = sizeof(ACC) == 4 ? 8 : 4;
             if (gl < nchunks) {
-                for (; s + 4 <= nseg; s += 4) {
-                    ACC tmp[4][VN];
+                for (; s < nseg; s += W) {
+                    ACC tmp[W][VN];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
+                    for (int u = 0; u < W; ++u) {
                         const ACC *p = reinterpret_cast<const ACC *>(a.heavy.partials) + (size_t)(b + s + u) * a.F + gl * VN;
+                        const bool in = s + u < nseg;
 #pragma unroll
-                        for (int t = 0; t < VN; ++t) tmp[u][t] = p[t];
+                        for (int t = 0; t < VN; ++t) tmp[u][t] = in ? p[t] : ACC(0);
                     }
 #pragma unroll
-                    for (int u = 0; u < 4; ++u)
+                    for (int u = 0; u < W; ++u)
 #pragma unroll
                         for (int t = 0; t < VN; ++t) acc[0][t] += tmp[u][t];
                 }
             }
+            s = nseg;
         }
         for (; s < nseg; ++s) {
             const ACC *p = reinterpret_cast<const ACC *>(a.heavy.partials) + (size_t)(b + s) * a.F;
@@ -697,6 +703,7 @@ template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC> sta
             b.heavy.rows = a.heavy.p_rows;
             b.heavy.base = a.heavy.p_base;
             b.heavy.counts = a.heavy.p_counts;
+            b.heavy.nseg = a.heavy.p_nseg;
             b.heavy.seg = SPMM_PIECE;
             const unsigned pgrid = (unsigned)ceil_div64(a.heavy.n_chunks, NG);
             const bool plain = !a.init && !a.relu_ref;
