@@ -341,6 +341,13 @@ lp_status lp_profile_begin(lp_ctx *ctx, uint32_t category_mask);
 /* Stop timing, synchronise the stream and return the sums per category since lp_profile_begin. */
 lp_status lp_profile_end(lp_ctx *ctx, lp_profile *out);
 
+/* Time only the launches of every n-th call of lp_train_step / lp_train_step_host (n >= 1; 1, the default,
+ * times every call).  An event record between two kernels keeps the second from being made resident while
+ * the first still runs, so timed steps run a few percent slower than untimed ones: sampling keeps the timed
+ * launches representative while the whole run stays close to its untimed speed.  The setting lasts until it
+ * is changed.  LP_EINVAL when n is 0. */
+lp_status lp_profile_sample_every(lp_ctx *ctx, uint32_t n);
+
 /* ---- single operators (used by the parity tests and the roofline benchmark) -------------- */
 
 /* AGG of Eq. 1 on the loaded graph, float32 in / float32 out (bf16 = 0) or BF16 in / BF16 out

@@ -26,7 +26,7 @@ EXPORTS = [
     "lp_create", "lp_destroy", "lp_last_error", "lp_load_graph", "lp_get_structure", "lp_set_model",
     "lp_param_count", "lp_set_candidates", "lp_sample_negatives", "lp_train_step", "lp_train_step_host",
     "lp_adam_step", "lp_score", "lp_get_embeddings", "lp_get_output_gradient", "lp_get_block",
-    "lp_get_stats", "lp_op_aggregate", "lp_op_gather_ceiling", "lp_op_linear", "lp_op_weight_grad", "lp_profile_begin", "lp_profile_end",
+    "lp_get_stats", "lp_op_aggregate", "lp_op_gather_ceiling", "lp_op_linear", "lp_op_weight_grad", "lp_profile_begin", "lp_profile_end", "lp_profile_sample_every",
     "lp_weight_grad_static", "lp_sparsify", "lp_get_sparsified",
     "lp_worker_view", "lp_get_worker_view", "lp_hits_at_k", "lp_get_predictor_activations",
     "lp_invalidate_embeddings", "lp_set_wait_limit",
@@ -307,6 +307,9 @@ class Context:
         for c in (categories if categories is not None else PROF_CATEGORIES):
             mask |= 1 << PROF_CATEGORIES.index(c)
         self._ck(self.lib.lp_profile_begin(self.h, C.c_uint32(mask)))
+
+    def profile_sample_every(self, n: int):
+        self._ck(self.lib.lp_profile_sample_every(self.h, C.c_uint32(n)))
 
     def profile_end(self):
         p = Profile()

@@ -21,6 +21,7 @@ __global__ void check_ids_kernel(const int *__restrict__ ids, int64_t m, int n_i
 __global__ void check_step_ids_kernel(const int *__restrict__ a, int64_t na, const int *__restrict__ b, int64_t nb, const int *__restrict__ c, int64_t nc,
                                       const int *__restrict__ d, int64_t nd, int n_ids, int *__restrict__ err)
 {
+    LP_DEP_ENTER();
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int *p = a;
     if (i >= na) { i -= na; p = b; if (i >= nb) { i -= nb; p = c; if (i >= nc) { i -= nc; p = d; if (i >= nd) return; } } }
@@ -55,6 +56,7 @@ edge_score_bce_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const 
                       float inv_N, float *__restrict__ g_pos, float *__restrict__ g_neg, float *__restrict__ s_pos, float *__restrict__ s_neg,
                       float *__restrict__ loss_partials, int *__restrict__ inc_counts = nullptr)
 {
+    LP_DEP_ENTER();
     constexpr int VN = Vec16<T>::N;
     __shared__ float s_loss[EDGE_THREADS / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -178,6 +180,7 @@ edge_score_bce_pair_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, c
                            const int *__restrict__ pos_dst, int64_t B, const int *__restrict__ neg_dst, float inv_N, float *__restrict__ g_pos,
                            float *__restrict__ g_neg, float *__restrict__ loss_partials, int *__restrict__ inc_counts)
 {
+    LP_DEP_ENTER();
     constexpr int VN = Vec16<T>::N;
     constexpr int P = 2;
     __shared__ float s_loss[EDGE_THREADS / 32];
@@ -258,6 +261,7 @@ edge_score_bce_pair_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, c
 // (tens of thousands of nearly equal terms), then a fixed binary tree over the threads
 __global__ void __launch_bounds__(1024) loss_reduce_kernel(const float *__restrict__ partials, int64_t m, float inv_N, float *__restrict__ loss)
 {
+    LP_DEP_ENTER();
     __shared__ double sh[1024];
     double s = 0.0;
     for (int64_t i = threadIdx.x; i < m; i += 1024) s += (double)partials[i];
@@ -348,6 +352,7 @@ __global__ void incidence_fill_kernel(int n_ids, const int *__restrict__ idmap, 
                                       const float *__restrict__ g_pos, const float *__restrict__ g_neg, int *__restrict__ cursor,
                                       int *__restrict__ inc_col, float *__restrict__ inc_val, int *__restrict__ inc_edge)
 {
+    LP_DEP_ENTER();
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const bool valid = e < B * (1 + k);
     const unsigned active = __ballot_sync(0xffffffffu, valid);

@@ -88,6 +88,7 @@ gemm_simt_kernel(int64_t M, int N, int64_t K, const TA *__restrict__ A, int64_t 
 // dst[i] = (accumulate ? dst[i] : 0) + sum_z partials[z][i], z ascending
 __global__ void reduce_partials_kernel(const float *__restrict__ partials, int64_t count, int splits, float *__restrict__ dst, int accumulate)
 {
+    LP_DEP_ENTER();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= count) return;
     float s = 0.f;
@@ -128,7 +129,7 @@ static void weight_grad_simt(Exec &ex, int64_t rows, int Kin, int N, const T *A,
     dim3 grid((unsigned)ceil_div64(Kin, SG_BM), (unsigned)ceil_div64(N, SG_BN), (unsigned)splits);
     gemm_simt_kernel<T, T, float, true, true><<<grid, SG_THREADS, 0, ex.st>>>(Kin, N, rows, A, lda, dZ, ldz, (float *)nullptr, 0, nullptr, 0, k_chunk, partials);
     const int64_t count = (int64_t)Kin * N;
-    reduce_partials_kernel<<<(unsigned)ceil_div64(count, 256), 256, 0, ex.st>>>(partials, count, splits, dW, accumulate);
+    launch_dep(reduce_partials_kernel, dim3((unsigned)ceil_div64(count, 256)), dim3(256), 0, ex.st, partials, count, splits, dW, accumulate);
     ex.launches += 2;
 }
 

@@ -208,6 +208,7 @@ template <bool MN_MAJOR>
 __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                                                              const TcGemmParams p)
 {
+    LP_DEP_ENTER();
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[8], bar_empty[8], bar_acc;
     __shared__ uint32_t tmem_base_s;
@@ -477,6 +478,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 1) tc_linear_persistent_kernel(co
                                                                               const __grid_constant__ CUtensorMap mapB,
                                                                               const __grid_constant__ CUtensorMap mapC, const TcGemmParams p)
 {
+    LP_DEP_ENTER();
     __shared__ float s_bias[256];
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[TCP_MAX_STAGES], bar_empty[TCP_MAX_STAGES], bar_w, bar_acc_full[2], bar_acc_empty[2];
@@ -754,6 +756,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TCP_THREADS, 1)
     tc_linear_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const __grid_constant__ CUtensorMap mapC,
                           const TcGemmParams p)
 {
+    LP_DEP_ENTER();
     __shared__ float s_bias[256];
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[TCP_MAX_STAGES], bar_empty[TCP_MAX_STAGES], bar_w, bar_acc_full[2], bar_acc_empty[2];
@@ -1130,7 +1133,7 @@ static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const
         int64_t pairs = std::min<int64_t>((int64_t)tc_sm_count() / 2, m_tiles * n_slices);
         pairs = std::max<int64_t>(n_slices, pairs / n_slices * n_slices);  // a whole number of pairs per slice
         const size_t smem = (size_t)w_bytes + (size_t)p.stages * TC_BM * TC_BK * 2 + (size_t)out_bytes + 1024;
-        tc_linear_pair_kernel<<<(unsigned)(2 * pairs), TCP_THREADS, smem, ex.st>>>(mapA, mapB, mapC, p);
+        launch_dep(tc_linear_pair_kernel, dim3((unsigned)(2 * pairs)), dim3(TCP_THREADS), smem, ex.st, mapA, mapB, mapC, p);
         ex.launches += 1;
         return true;
     }
@@ -1154,7 +1157,7 @@ static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const
         int64_t ctas = std::min<int64_t>((int64_t)tc_sm_count(), m_tiles * n_slices);
         ctas = std::max<int64_t>(n_slices, ctas / n_slices * n_slices);  // a whole number of CTAs per slice
         const size_t smem = (size_t)w_bytes + (size_t)p.stages * TC_BM * TC_BK * 2 + TCP_STAGE_OUT_BYTES + 1024;
-        tc_linear_persistent_kernel<<<(unsigned)ctas, TCP_THREADS, smem, ex.st>>>(mapA, mapB, mapC, p);
+        launch_dep(tc_linear_persistent_kernel, dim3((unsigned)ctas), dim3(TCP_THREADS), smem, ex.st, mapA, mapB, mapC, p);
         ex.launches += 1;
         return true;
     }
@@ -1170,7 +1173,7 @@ static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const
     p.wait_ns = tc.wait_limit_ns; p.extra_tx = tc.overdeclare_tx; tc.overdeclare_tx = 0;
     const size_t smem = (size_t)p.stages * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024;
     dim3 grid((unsigned)ceil_div64(M, TC_BM), (unsigned)(N / BN), 1);
-    tc_gemm_kernel<false><<<grid, TC_THREADS, smem, ex.st>>>(mapA, mapB, p);
+    launch_dep(tc_gemm_kernel<false>, dim3(grid), dim3(TC_THREADS), smem, ex.st, mapA, mapB, p);
     ex.launches += 1;
     return true;
 }
@@ -1231,9 +1234,9 @@ static bool tc_weight_grad(TcState &tc, Exec &ex, int64_t rows, int Kin, int N, 
     p.wait_ns = tc.wait_limit_ns; p.extra_tx = tc.overdeclare_tx; tc.overdeclare_tx = 0;
     const size_t smem = (size_t)p.stages * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024;
     dim3 grid((unsigned)(Kin / TC_BM), (unsigned)(N / BN), (unsigned)splits);
-    tc_gemm_kernel<true><<<grid, TC_THREADS, smem, ex.st>>>(mapA, mapB, p);
+    launch_dep(tc_gemm_kernel<true>, dim3(grid), dim3(TC_THREADS), smem, ex.st, mapA, mapB, p);
     const int64_t count = (int64_t)(Kin + (fuse_bias ? 1 : 0)) * N;
-    reduce_partials_kernel<<<(unsigned)ceil_div64(count, 256), 256, 0, ex.st>>>(partials, count, splits, dW, accumulate);
+    launch_dep(reduce_partials_kernel, dim3((unsigned)ceil_div64(count, 256)), dim3(256), 0, ex.st, partials, count, splits, dW, accumulate);
     ex.launches += 2;
     return true;
 }

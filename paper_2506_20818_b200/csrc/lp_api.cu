@@ -441,7 +441,7 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
         hp->partials = ctx->heavy_partials;
         hp->threshold = static_threshold;
         cudaMemsetAsync(hp->counts, 0, 2 * sizeof(int), st);
-        spmm_heavy_plan_kernel<<<nblk(n), 256, 0, st>>>(hp == &ctx->plan_csr ? ctx->rowptr : ctx->colptr, (int)n, nullptr, *hp);
+        launch_dep(spmm_heavy_plan_kernel, dim3(nblk(n)), dim3(256), 0, st, hp == &ctx->plan_csr ? ctx->rowptr : ctx->colptr, (int)n, nullptr, *hp, nullptr);
         cudaMemcpyAsync(ctx->host_counts + (hp == &ctx->plan_csr ? 0 : 2), hp->counts, 2 * sizeof(int), cudaMemcpyDeviceToHost, st);
     }
     ctx->ex.launches += 2;
@@ -469,7 +469,7 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
         TALLOC(chunk_count, n + 1);
         TALLOC(chunk_of, n + 1);
         cudaMemsetAsync(pp.counts, 0, 2 * sizeof(int), st);
-        spmm_heavy_plan_kernel<<<nblk(n), 256, 0, st>>>(sp, (int)n, nullptr, pp, row_base);
+        launch_dep(spmm_heavy_plan_kernel, dim3(nblk(n)), dim3(256), 0, st, sp, (int)n, nullptr, pp, row_base);
         padded_count_kernel<<<nblk(n), 256, 0, st>>>(sp, (int)n, SPMM_PIECE, first_group);
         exclusive_scan_i32(ctx->ex, first_group, n, first_group, first_group + n, ts.scan_tmp);
         padded_chunk_count_kernel<<<nblk(n), 256, 0, st>>>(sp, first_group, (int)n, SPMM_PIECE, chunk_count);
@@ -1029,7 +1029,7 @@ static void cache_weights(lp_ctx *ctx, const float *params)
     }
     if (ctx->mlp)
         for (int j = 0; j < 2; ++j) { wb.off[wb.count] = ctx->pred[j].off_w; wb.kin[wb.count] = ctx->pred[j].Kin; wb.fo[wb.count] = ctx->pred[j].Fo; ++wb.count; }
-    weights_cache_kernel<<<nblk(ctx->n_params), 256, 0, ctx->ex.st>>>(params, ctx->n_params, wb, ctx->w16, ctx->w16t, ctx->w16s);
+    launch_dep(weights_cache_kernel, dim3(nblk(ctx->n_params)), dim3(256), 0, ctx->ex.st, params, ctx->n_params, wb, ctx->w16, ctx->w16t, ctx->w16s);
     ctx->ex.launches += 1;
 }
 
@@ -1359,10 +1359,11 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     const int K = ctx->K;
     const bool sage = ctx->desc.arch == LP_SAGE_MEAN;
     const int D = ctx->desc.dims[K];
+    ctx->ex.prof.tick += 1;  // lp_profile_sample_every counts training steps
     // bad ids are clamped by every consumer and reported through the context's error word
     {
         const int64_t nk = k > 0 ? B * k : 0;
-        check_step_ids_kernel<<<nblk(2 * B + 2 * nk), 256, 0, st>>>(pos_src, B, pos_dst, B, neg_dst, nk, neg_src, (k > 0 && neg_src) ? nk : 0, ctx->n, ctx->err_flag);
+        launch_dep(check_step_ids_kernel, dim3(nblk(2 * B + 2 * nk)), dim3(256), 0, st, pos_src, B, pos_dst, B, neg_dst, nk, neg_src, (k > 0 && neg_src) ? nk : 0, ctx->n, ctx->err_flag);
         ctx->ex.launches += 1;
     }
     cache_weights(ctx, params);
@@ -1391,7 +1392,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         if (s != LP_OK) return s;
         const unsigned lblocks = nblk(E, 256);
         bce_from_scores_kernel<<<lblocks, 256, 0, st>>>(ctx->pred_scores, E, B, inv_N, ctx->g_pos, ctx->loss_partials);
-        loss_reduce_kernel<<<1, 1024, 0, st>>>(ctx->loss_partials, lblocks, inv_N, loss);
+        launch_dep(loss_reduce_kernel, dim3(1), dim3(1024), 0, st, ctx->loss_partials, lblocks, inv_N, loss);
         g_neg = ctx->g_pos + B;  // one array: positives, then negatives
         s = predictor_backward<T>(ctx, params, E, ctx->g_pos, grads, accumulate);
         if (s != LP_OK) return s;
@@ -1399,11 +1400,11 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         unsigned lparts = eblocks;  // loss partials written
         if (chunks <= 32 && k == 1 && !neg_src) {
             lparts = nblk(B, 2 * (EDGE_THREADS / 32));
-            edge_score_bce_pair_kernel<T><<<lparts, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_dst, inv_N, ctx->g_pos, ctx->g_neg, ctx->loss_partials, ctx->inc_ptr);
-        } else if (chunks <= 32) edge_score_bce_kernel<T, 1><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials, ctx->inc_ptr);
-        else if (chunks <= 64) edge_score_bce_kernel<T, 2><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials, ctx->inc_ptr);
-        else edge_score_bce_kernel<T, 4><<<eblocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials, ctx->inc_ptr);
-        loss_reduce_kernel<<<1, 1024, 0, st>>>(ctx->loss_partials, lparts, inv_N, loss);
+            launch_dep(edge_score_bce_pair_kernel<T>, dim3(lparts), dim3(EDGE_THREADS), 0, st, HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_dst, inv_N, ctx->g_pos, ctx->g_neg, ctx->loss_partials, ctx->inc_ptr);
+        } else if (chunks <= 32) launch_dep(edge_score_bce_kernel<T, 1>, dim3(eblocks), dim3(EDGE_THREADS), 0, st, HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials, ctx->inc_ptr);
+        else if (chunks <= 64) launch_dep(edge_score_bce_kernel<T, 2>, dim3(eblocks), dim3(EDGE_THREADS), 0, st, HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials, ctx->inc_ptr);
+        else launch_dep(edge_score_bce_kernel<T, 4>, dim3(eblocks), dim3(EDGE_THREADS), 0, st, HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials, ctx->inc_ptr);
+        launch_dep(loss_reduce_kernel, dim3(1), dim3(1024), 0, st, ctx->loss_partials, lparts, inv_N, loss);
     }
     pscore.reset();
     ctx->ex.launches += 2;
@@ -1412,7 +1413,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     std::unique_ptr<ProfScope> pinc(new ProfScope(ctx->ex, LP_PROF_INCIDENCE, (double)E * 2.0 * 24.0));
     if (ctx->mlp) incidence_count_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->inc_ptr);
     exclusive_scan_i32_copy(ctx->ex, ctx->inc_ptr, rows_out, ctx->inc_ptr, ctx->inc_cursor, ctx->inc_ptr + rows_out, ctx->scan_tmp);
-    incidence_fill_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, g_pos, g_neg, ctx->inc_cursor, ctx->inc_col,
+    launch_dep(incidence_fill_kernel, dim3(nblk(E)), dim3(256), 0, st, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, g_pos, g_neg, ctx->inc_cursor, ctx->inc_col,
                                                    ctx->mlp ? nullptr : ctx->inc_val, ctx->mlp ? ctx->inc_edge : nullptr);
     ctx->ex.launches += 2;
     pinc.reset();
@@ -1625,7 +1626,7 @@ extern "C" lp_status lp_adam_step(lp_ctx *ctx, float *params, float *adam_m, flo
     ProfScope prof(ctx->ex, LP_PROF_ADAM, (double)np * (adam_m ? 28.0 : 12.0));
     if (adam_m) {
         const double c1 = 1.0 - std::pow(beta1, (double)t), c2 = 1.0 - std::pow(beta2, (double)t);
-        adam_kernel<<<nblk(np), 256, 0, ctx->ex.st>>>(params, adam_m, adam_v, grads, np, (float)grad_scale, (float)lr, (float)beta1, (float)(1.0 - beta1),
+        launch_dep(adam_kernel, dim3(nblk(np)), dim3(256), 0, ctx->ex.st, params, adam_m, adam_v, grads, np, (float)grad_scale, (float)lr, (float)beta1, (float)(1.0 - beta1),
                                                       (float)beta2, (float)(1.0 - beta2), (float)eps, (float)(1.0 / c1), (float)(1.0 / c2));
     } else {
         sgd_kernel<<<nblk(np), 256, 0, ctx->ex.st>>>(params, grads, np, (float)grad_scale, (float)lr);
@@ -1888,6 +1889,14 @@ extern "C" lp_status lp_profile_begin(lp_ctx *ctx, uint32_t category_mask)
     return LP_OK;
 }
 
+extern "C" lp_status lp_profile_sample_every(lp_ctx *ctx, uint32_t n)
+{
+    if (!ctx) return LP_EINVAL;
+    if (n == 0) return fail(ctx, LP_EINVAL, "lp_profile_sample_every: n must be at least 1");
+    ctx->ex.prof.period = n;
+    return LP_OK;
+}
+
 extern "C" lp_status lp_profile_end(lp_ctx *ctx, lp_profile *out)
 {
     if (!ctx || !out) return LP_EINVAL;
@@ -2070,7 +2079,7 @@ extern "C" lp_status lp_weight_grad_static(int32_t device, void *cuda_stream, in
     cudaStream_t st = (cudaStream_t)cuda_stream;
     dim3 grid((unsigned)ceil_div64(K, SG_BM), (unsigned)ceil_div64(N, SG_BN), (unsigned)splits);
     gemm_simt_kernel<float, float, float, true, true><<<grid, SG_THREADS, 0, st>>>(K, N, M, A, K, dZ, N, (float *)nullptr, 0, nullptr, 0, k_chunk, scratch);
-    reduce_partials_kernel<<<(unsigned)ceil_div64(tile, 256), 256, 0, st>>>(scratch, tile, splits, dW, 0);
+    launch_dep(reduce_partials_kernel, dim3((unsigned)ceil_div64(tile, 256)), dim3(256), 0, st, scratch, tile, splits, dW, 0);
     CK_LAUNCH();
     return LP_OK;
 }

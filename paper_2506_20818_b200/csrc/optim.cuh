@@ -11,6 +11,7 @@ __global__ void adam_kernel(float *__restrict__ p, float *__restrict__ m, float 
                             float scale, float lr, float b1, float one_minus_b1, float b2, float one_minus_b2, float eps, float inv_c1,
                             float inv_c2)
 {
+    LP_DEP_ENTER();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     const float g = scale * grad[i];
@@ -68,6 +69,7 @@ struct WeightBlocks {
 __global__ void weights_cache_kernel(const float *__restrict__ params, long long n, WeightBlocks blocks, bf16 *__restrict__ asis, bf16 *__restrict__ transposed,
                                      bf16 *__restrict__ stacked)
 {
+    LP_DEP_ENTER();
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     const bf16 x = __float2bfloat16_rn(params[i]);

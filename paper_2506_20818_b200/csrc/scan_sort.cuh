@@ -7,6 +7,9 @@
 // Optional per-category timing with CUDA events on the launching stream (lp_profile_begin/_end).
 struct Profiler {
     uint32_t mask = 0;  // categories being timed; 0 = off
+    uint32_t period = 1;  // only every period-th training step is timed
+    uint64_t tick = 0;    // training steps seen
+    bool live(int cat) const { return (mask & (1u << cat)) && (period <= 1 || tick % period == 0); }
     struct Span { int cat; cudaEvent_t a, b; double bytes, flops; };
     std::vector<Span> spans;
     std::vector<cudaEvent_t> pool;
@@ -38,7 +41,7 @@ struct ProfScope {
     int idx = -1;
     ProfScope(Exec &e, int cat, double bytes = 0.0, double flops = 0.0) : ex(e)
     {
-        if (ex.prof.mask & (1u << cat)) {
+        if (ex.prof.live(cat)) {
             Profiler::Span s{cat, ex.prof.get(), ex.prof.get(), bytes, flops};
             cudaEventRecord(s.a, ex.st);
             idx = (int)ex.prof.spans.size();
@@ -198,6 +201,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_onepass_kernel(const int *_
                                                                     int *__restrict__ out_total, unsigned long long *__restrict__ status,
                                                                     unsigned *__restrict__ ticket, unsigned epoch, int *__restrict__ err)
 {
+    LP_DEP_ENTER();
     __shared__ int sw[8];
     __shared__ unsigned tile_s;
     __shared__ int prefix_s;
@@ -280,7 +284,7 @@ static bool scan_onepass_try(Exec &ex, const int *in, int64_t n, int *out, int *
     if (!sc || !sc->status || tiles > sc->tiles_cap) return false;
     sc->epoch = (sc->epoch + 1u) & 0x3fffffffu;
     if (sc->epoch == 0) sc->epoch = 1;
-    scan_onepass_kernel<<<(unsigned)tiles, SCAN_THREADS, 0, ex.st>>>(in, n, out, out_copy, out_total, sc->status, sc->ticket, sc->epoch, ex.scan_err);
+    launch_dep(scan_onepass_kernel, dim3((unsigned)tiles), dim3(SCAN_THREADS), 0, ex.st, in, n, out, out_copy, out_total, sc->status, sc->ticket, sc->epoch, ex.scan_err);
     ex.launches += 1;
     return true;
 }

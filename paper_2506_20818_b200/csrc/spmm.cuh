@@ -333,6 +333,7 @@ LP_DEVINL void spmm_epilogue(const SpmmArgs<T> &a, int r, int gl, int nchunks, c
 template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC, bool HAS_VAL, bool HAS_X2>
 __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_csr_kernel(const SpmmArgs<T> a, const int light_blocks)
 {
+    LP_DEP_ENTER();
     constexpr int VN = Vec16<T>::N;
     constexpr int NG = SPMM_THREADS / G;  // lane groups per block
     constexpr int ROWS = NG * RPG;        // rows per block: every group walks RPG rows
@@ -454,6 +455,7 @@ LP_DEVINL void prefetch_l1(const void *p) { asm volatile("prefetch.global.L1 [%0
 template <typename T, int G, int MULT, int MINB, bool HAS_VAL, int EPI>
 __global__ void __launch_bounds__(SPMM_THREADS, MINB) spmm_padded_kernel(const SpmmArgs<T> a)
 {
+    LP_DEP_ENTER();
     constexpr int VN = Vec16<T>::N;
     constexpr int NG = SPMM_THREADS / G;
     constexpr unsigned PITCH = (unsigned)(G * VN * MULT);  // elements between source rows
@@ -610,6 +612,7 @@ __global__ void padded_fill_kernel(const int *__restrict__ rowptr, const int *__
 __global__ void spmm_heavy_plan_kernel(const int *__restrict__ rowptr, int n_rows, const int *__restrict__ n_rows_dev, HeavyPlan hp,
                                        int *__restrict__ row_base = nullptr)
 {
+    LP_DEP_ENTER();
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     const int lim = n_rows_dev ? min(*n_rows_dev, n_rows) : n_rows;
     if (r >= lim) return;
@@ -635,6 +638,7 @@ __global__ void spmm_heavy_plan_kernel(const int *__restrict__ rowptr, int n_row
 template <typename T, int G, int NV, typename ACC>
 __global__ void __launch_bounds__(SPMM_THREADS) spmm_heavy_combine_kernel(const SpmmArgs<T> a)
 {
+    LP_DEP_ENTER();
     constexpr int VN = Vec16<T>::N;
     constexpr int NG = SPMM_THREADS / G;
     const int count = a.heavy.counts[0];
@@ -709,9 +713,9 @@ template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC> sta
             const bool plain = !a.init && !a.relu_ref;
             const bool self_mask = a.init && a.relu_ref && !a.init_coef && !a.row_scale && !a.val;
 #define LP_PADDED(MULT_, VAL_) do { \
-                if (plain) spmm_padded_kernel<T, G, MULT_, VAL_ ? 5 : 6, VAL_, 1><<<pgrid, SPMM_THREADS, 0, ex.st>>>(b); \
-                else if (self_mask) spmm_padded_kernel<T, G, MULT_, 5, false, 2><<<pgrid, SPMM_THREADS, 0, ex.st>>>(b); \
-                else spmm_padded_kernel<T, G, MULT_, 5, VAL_, 0><<<pgrid, SPMM_THREADS, 0, ex.st>>>(b); } while (0)
+                if (plain) launch_dep(spmm_padded_kernel<T, G, MULT_, VAL_ ? 5 : 6, VAL_, 1>, dim3(pgrid), dim3(SPMM_THREADS), 0, ex.st, b); \
+                else if (self_mask) launch_dep(spmm_padded_kernel<T, G, MULT_, 5, false, 2>, dim3(pgrid), dim3(SPMM_THREADS), 0, ex.st, b); \
+                else launch_dep(spmm_padded_kernel<T, G, MULT_, 5, VAL_, 0>, dim3(pgrid), dim3(SPMM_THREADS), 0, ex.st, b); } while (0)
             if (pitch == G) {
                 if (a.val) LP_PADDED(1, true); else LP_PADDED(1, false);
             } else {
@@ -720,7 +724,7 @@ template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC> sta
 #undef LP_PADDED
             ex.launches += 1;
             if (a.heavy.p_host_rows > 0) {
-                spmm_heavy_combine_kernel<T, G, NV, ACC><<<(unsigned)std::min<int64_t>(592, ceil_div64(a.heavy.p_host_rows, NG)), SPMM_THREADS, 0, ex.st>>>(b);
+                launch_dep(spmm_heavy_combine_kernel<T, G, NV, ACC>, dim3((unsigned)std::min<int64_t>(592, ceil_div64(a.heavy.p_host_rows, NG))), dim3(SPMM_THREADS), 0, ex.st, b);
                 ex.launches += 1;
             }
             return;
@@ -729,7 +733,7 @@ template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC> sta
     int64_t items = a.heavy.host_items;
     if (items < 0) {  // plan unknown on the host: rebuild it on the device, size the grid by the upper bound
         cudaMemsetAsync(a.heavy.counts, 0, 2 * sizeof(int), ex.st);
-        spmm_heavy_plan_kernel<<<(unsigned)ceil_div64(a.n_rows, 256), 256, 0, ex.st>>>(a.rowptr, a.n_rows, a.n_rows_dev, a.heavy);
+        launch_dep(spmm_heavy_plan_kernel, dim3((unsigned)ceil_div64(a.n_rows, 256)), dim3(256), 0, ex.st, a.rowptr, a.n_rows, a.n_rows_dev, a.heavy, nullptr);
         items = a.nnz / SPMM_HEAVY_MIN;  // a heavy row has more than SPMM_HEAVY_MIN entries and at most deg / SPMM_HEAVY_MIN items
         ex.launches += 1;
     }
@@ -738,19 +742,19 @@ template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC> sta
     bool launched = false;
     if constexpr (sizeof(ACC) == 8) {  // the two-operand form exists for the exact accumulator only
         if (a.X2) {
-            spmm_csr_kernel<T, G, NV, RPG, U, MINB, ACC, false, true><<<grid, SPMM_THREADS, 0, ex.st>>>(a, light_blocks);
+            launch_dep(spmm_csr_kernel<T, G, NV, RPG, U, MINB, ACC, false, true>, dim3(grid), dim3(SPMM_THREADS), 0, ex.st, a, light_blocks);
             launched = true;
         }
     }
     if (!launched) {
-        if (a.val) spmm_csr_kernel<T, G, NV, RPG, U, MINB, ACC, true, false><<<grid, SPMM_THREADS, 0, ex.st>>>(a, light_blocks);
-        else spmm_csr_kernel<T, G, NV, RPG, U, MINB, ACC, false, false><<<grid, SPMM_THREADS, 0, ex.st>>>(a, light_blocks);
+        if (a.val) launch_dep(spmm_csr_kernel<T, G, NV, RPG, U, MINB, ACC, true, false>, dim3(grid), dim3(SPMM_THREADS), 0, ex.st, a, light_blocks);
+        else launch_dep(spmm_csr_kernel<T, G, NV, RPG, U, MINB, ACC, false, false>, dim3(grid), dim3(SPMM_THREADS), 0, ex.st, a, light_blocks);
     }
     ex.launches += 1;
     if (a.heavy.host_rows != 0) {
         const int64_t rows_bound = a.heavy.host_rows > 0 ? a.heavy.host_rows : std::max<int64_t>(1, items);
         const unsigned grid = (unsigned)std::min<int64_t>(592, ceil_div64(rows_bound, NG));
-        spmm_heavy_combine_kernel<T, G, NV, ACC><<<grid, SPMM_THREADS, 0, ex.st>>>(a);
+        launch_dep(spmm_heavy_combine_kernel<T, G, NV, ACC>, dim3(grid), dim3(SPMM_THREADS), 0, ex.st, a);
         ex.launches += 1;
     }
 }
