@@ -19,9 +19,11 @@ __global__ void check_ids_kernel(const int *__restrict__ ids, int64_t m, int n_i
 
 // the same for the up to four id arrays of a step in one launch (null arrays are skipped)
 __global__ void check_step_ids_kernel(const int *__restrict__ a, int64_t na, const int *__restrict__ b, int64_t nb, const int *__restrict__ c, int64_t nc,
-                                      const int *__restrict__ d, int64_t nd, int n_ids, int *__restrict__ err)
+                                      const int *__restrict__ d, int64_t nd, int n_ids, int *__restrict__ err, int *__restrict__ zero, int64_t n_zero)
 {
     LP_DEP_ENTER();
+    // first kernel of a step: it also clears the incidence-list counters the scoring kernel adds into
+    for (int64_t z = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; z < n_zero; z += (int64_t)gridDim.x * blockDim.x) zero[z] = 0;
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int *p = a;
     if (i >= na) { i -= na; p = b; if (i >= nb) { i -= nb; p = c; if (i >= nc) { i -= nc; p = d; if (i >= nd) return; } } }
@@ -350,10 +352,11 @@ LP_DEVINL int claim_slot(int *cursor, int node, unsigned active, int lane)
 __global__ void incidence_fill_kernel(int n_ids, const int *__restrict__ idmap, const int *__restrict__ pos_src, const int *__restrict__ pos_dst,
                                       int64_t B, const int *__restrict__ neg_src, const int *__restrict__ neg_dst, int k,
                                       const float *__restrict__ g_pos, const float *__restrict__ g_neg, int *__restrict__ cursor,
-                                      int *__restrict__ inc_col, float *__restrict__ inc_val, int *__restrict__ inc_edge)
+                                      int *__restrict__ inc_col, float *__restrict__ inc_val, int *__restrict__ inc_edge, int *__restrict__ plan_counts)
 {
     LP_DEP_ENTER();
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e == 0 && plan_counts) { plan_counts[0] = 0; plan_counts[1] = 0; }  // the heavy-row plan of these lists is built by the next launch
     const bool valid = e < B * (1 + k);
     const unsigned active = __ballot_sync(0xffffffffu, valid);
     if (!valid) return;

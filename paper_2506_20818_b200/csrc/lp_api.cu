@@ -75,7 +75,8 @@ struct lp_ctx {
     bf16 *X16 = nullptr;
     int *cand = nullptr;         // candidate set of the negative sampler (own allocation, replaced by every lp_set_candidates)
     int64_t n_cand = 0;
-    unsigned long long *exhausted_dev = nullptr;
+    unsigned long long *exhausted_dev = nullptr;  // 16 counters used in turn: a call of the sampler adds into one and clears the next
+    uint64_t neg_calls = 0;
     HeavyPlan plan_csr, plan_csc, plan_dyn;  // heavy-row plans: the loaded graph, its transpose, per-step structures
     float *heavy_partials = nullptr;
     int *err_flag = nullptr;
@@ -87,6 +88,7 @@ struct lp_ctx {
     int max_k = 0, K = 0;
     LayerBuf layer[LP_MAX_LAYERS];
     void *HK = nullptr;                 // H^(K) [rows_out, D]
+    int64_t inc_cap = 0;                // ints in inc_ptr
     void *dHK = nullptr;                // dL/dH^(K) [rows_out, D]
     void *dZ[2] = {nullptr, nullptr};   // gradient ping-pong [max_rows, max_width]
     void *dA = nullptr;                 // [max_rows, max Kin]
@@ -867,6 +869,7 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
     MALLOC(ctx->inc_col, 2 * E);
     MALLOC(ctx->inc_val, 2 * E);
     MALLOC(ctx->inc_ptr, cap_rows[0] + 1);
+    ctx->inc_cap = cap_rows[0] + 1;
     MALLOC(ctx->d_pos_tmp, 2 * max_batch);
     MALLOC(ctx->d_neg_tmp, max_batch * std::max<int64_t>(max_k, 1));
     MALLOC(ctx->d_loss_tmp, 64);
@@ -1003,10 +1006,11 @@ extern "C" lp_status lp_sample_negatives(lp_ctx *ctx, uint64_t seed, uint64_t st
     const int attempts = (ctx->model_set && ctx->desc.reject_edges) ? ctx->desc.max_attempts : (reject ? 8 : 1);
     const uint32_t space = (uint32_t)(ctx->cand ? ctx->n_cand : ctx->n);
     ProfScope prof(ctx->ex, LP_PROF_NEGATIVES, (double)B * k * 8.0);
-    cudaMemsetAsync(ctx->exhausted_dev, 0, sizeof(unsigned long long), ctx->ex.st);
-    sample_negatives_kernel<<<nblk(B * k), 256, 0, ctx->ex.st>>>(ctx->n, ctx->rowptr, ctx->col, ctx->cand, space,
-                                                                make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)), (uint32_t)step, k, mode, reject,
-                                                                attempts, pos_src, B, edge_index_base, neg_src, neg_dst, ctx->exhausted_dev);
+    unsigned long long *counter = ctx->exhausted_dev + ctx->neg_calls % 16, *next = ctx->exhausted_dev + (ctx->neg_calls + 1) % 16;
+    ctx->neg_calls += 1;
+    launch_dep(sample_negatives_kernel, dim3(nblk(B * k)), dim3(256), 0, ctx->ex.st, ctx->n, ctx->rowptr, ctx->col, ctx->cand, space,
+               make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)), (uint32_t)step, k, mode, reject, attempts, pos_src, B, edge_index_base, neg_src, neg_dst,
+               counter, next);
     ctx->ex.launches += 1;
     CK_LAUNCH();
     return LP_OK;
@@ -1363,7 +1367,8 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     // bad ids are clamped by every consumer and reported through the context's error word
     {
         const int64_t nk = k > 0 ? B * k : 0;
-        launch_dep(check_step_ids_kernel, dim3(nblk(2 * B + 2 * nk)), dim3(256), 0, st, pos_src, B, pos_dst, B, neg_dst, nk, neg_src, (k > 0 && neg_src) ? nk : 0, ctx->n, ctx->err_flag);
+        launch_dep(check_step_ids_kernel, dim3(nblk(2 * B + 2 * nk)), dim3(256), 0, st, pos_src, B, pos_dst, B, neg_dst, nk, neg_src, (k > 0 && neg_src) ? nk : 0, ctx->n, ctx->err_flag,
+                   ctx->inc_ptr, ctx->inc_cap);
         ctx->ex.launches += 1;
     }
     cache_weights(ctx, params);
@@ -1386,7 +1391,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     const int chunks = D / VN;
     const float *g_pos = ctx->g_pos, *g_neg = ctx->g_neg;
     // the dot-product scoring kernel also counts the incidence-list lengths (into the zeroed offsets array)
-    CK(cudaMemsetAsync(ctx->inc_ptr, 0, sizeof(int) * ((size_t)rows_out + 1), st));
+    // (the offsets array was cleared by the first kernel of the step)
     if (ctx->mlp) {
         s = predictor_forward<T>(ctx, params, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k);
         if (s != LP_OK) return s;
@@ -1414,7 +1419,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     if (ctx->mlp) incidence_count_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->inc_ptr);
     exclusive_scan_i32_copy(ctx->ex, ctx->inc_ptr, rows_out, ctx->inc_ptr, ctx->inc_cursor, ctx->inc_ptr + rows_out, ctx->scan_tmp);
     launch_dep(incidence_fill_kernel, dim3(nblk(E)), dim3(256), 0, st, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, g_pos, g_neg, ctx->inc_cursor, ctx->inc_col,
-                                                   ctx->mlp ? nullptr : ctx->inc_val, ctx->mlp ? ctx->inc_edge : nullptr);
+               ctx->mlp ? nullptr : ctx->inc_val, ctx->mlp ? ctx->inc_edge : nullptr, ctx->plan_dyn.counts);
     ctx->ex.launches += 2;
     pinc.reset();
 
@@ -1430,6 +1435,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         SpmmArgs<T> a;
         a.heavy = ctx->plan_dyn;
         a.heavy.partials = ctx->inc_partials;
+        a.heavy.counts_zeroed = true;  // by the kernel that filled the lists
 
         a.nnz = 2 * E;
         a.n_rows = rows_out;
@@ -1860,7 +1866,7 @@ extern "C" lp_status lp_get_stats(lp_ctx *ctx, lp_stats *out)
     memset(out, 0, sizeof *out);
     unsigned long long ex = 0;
     int bad = 0;
-    CK(cudaMemcpyAsync(&ex, ctx->exhausted_dev, sizeof ex, cudaMemcpyDeviceToHost, ctx->ex.st));
+    CK(cudaMemcpyAsync(&ex, ctx->exhausted_dev + (ctx->neg_calls + 15) % 16, sizeof ex, cudaMemcpyDeviceToHost, ctx->ex.st));  // the last call's counter
     CK(cudaMemcpyAsync(&bad, ctx->err_flag, sizeof bad, cudaMemcpyDeviceToHost, ctx->ex.st));
     CK(cudaStreamSynchronize(ctx->ex.st));
     if (bad) {

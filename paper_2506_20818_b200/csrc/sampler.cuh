@@ -39,9 +39,12 @@ LP_DEVINL bool csr_has_entry(const int *__restrict__ rowptr, const int *__restri
 __global__ void sample_negatives_kernel(int n, const int *__restrict__ rowptr, const int *__restrict__ col,
                                         const int *__restrict__ cand, uint32_t n_space, uint2 key, uint32_t step_lo, int k, int mode,
                                         int reject, int max_attempts, const int *__restrict__ pos_src, int64_t B, int64_t base,
-                                        int *__restrict__ neg_src, int *__restrict__ neg_dst, unsigned long long *__restrict__ exhausted)
+                                        int *__restrict__ neg_src, int *__restrict__ neg_dst, unsigned long long *__restrict__ exhausted,
+                                        unsigned long long *__restrict__ exhausted_next)
 {
+    LP_DEP_ENTER();
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t == 0) *exhausted_next = 0ull;  // the counter of the next call (the counters are used in turn, so no call needs a memset)
     if (t >= B * k) return;
     const int64_t j = t / k;
     const uint32_t kk = (uint32_t)(t - j * k);

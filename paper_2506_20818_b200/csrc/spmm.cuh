@@ -34,6 +34,7 @@ struct HeavyPlan {
     int *nseg = nullptr;                  // optional: items of heavy row i (saves the combine kernel the row-offset round trip)
     float *partials = nullptr;
     int host_rows = -1, host_items = -1;  // -1: unknown on the host (plan built on the device per launch)
+    bool counts_zeroed = false;           // per-launch plans: the caller's previous kernel has already cleared `counts`
     int threshold = 32;                   // rows with more entries than this are heavy (>= SPMM_HEAVY_MIN)
     int seg = 512;                        // entries per item (SPMM_SEG; SPMM_PIECE for the padded form's own plan)
     // Static structures only: every row again in padded form for spmm_padded_kernel.  A row is cut into pieces of at
@@ -732,7 +733,7 @@ template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC> sta
     }
     int64_t items = a.heavy.host_items;
     if (items < 0) {  // plan unknown on the host: rebuild it on the device, size the grid by the upper bound
-        cudaMemsetAsync(a.heavy.counts, 0, 2 * sizeof(int), ex.st);
+        if (!a.heavy.counts_zeroed) cudaMemsetAsync(a.heavy.counts, 0, 2 * sizeof(int), ex.st);
         launch_dep(spmm_heavy_plan_kernel, dim3((unsigned)ceil_div64(a.n_rows, 256)), dim3(256), 0, ex.st, a.rowptr, a.n_rows, a.n_rows_dev, a.heavy, nullptr);
         items = a.nnz / SPMM_HEAVY_MIN;  // a heavy row has more than SPMM_HEAVY_MIN entries and at most deg / SPMM_HEAVY_MIN items
         ex.launches += 1;
