@@ -13,6 +13,7 @@ LP_DEVINL int clamp_id(int v, int n_ids) { return min(max(v, 0), n_ids - 1); }
 
 __global__ void check_ids_kernel(const int *__restrict__ ids, int64_t m, int n_ids, int *__restrict__ err)
 {
+    LP_DEP_ENTER();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < m && (ids[i] < 0 || ids[i] >= n_ids)) atomicOr(err, 1);
 }
@@ -282,6 +283,7 @@ __global__ void __launch_bounds__(EDGE_THREADS)
 edge_score_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const int *__restrict__ idmap, const int *__restrict__ src,
                   const int *__restrict__ dst, int64_t E, float *__restrict__ scores)
 {
+    LP_DEP_ENTER();
     constexpr int VN = Vec16<T>::N;
     const int lane = threadIdx.x & 31;
     const int64_t e = (int64_t)blockIdx.x * (EDGE_THREADS / 32) + (threadIdx.x >> 5);
@@ -328,6 +330,7 @@ LP_DEVINL void incidence_endpoints(int n_ids, const int *idmap, const int *pos_s
 __global__ void incidence_count_kernel(int n_ids, const int *__restrict__ idmap, const int *__restrict__ pos_src, const int *__restrict__ pos_dst,
                                        int64_t B, const int *__restrict__ neg_src, const int *__restrict__ neg_dst, int k, int *__restrict__ counts)
 {
+    LP_DEP_ENTER();
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= B * (1 + k)) return;
     int s, d;

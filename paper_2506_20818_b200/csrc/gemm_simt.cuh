@@ -17,6 +17,7 @@ gemm_simt_kernel(int64_t M, int N, int64_t K, const TA *__restrict__ A, int64_t 
                  TC *__restrict__ C, int64_t ldc, const float *__restrict__ bias, int relu, int64_t k_chunk, float *__restrict__ partials,
                  const float *__restrict__ row_scale = nullptr, int scale_col0 = 0)
 {
+    LP_DEP_ENTER();
     __shared__ __align__(16) float As[SG_BK][SG_BM + 4];
     __shared__ __align__(16) float Bs[SG_BK][SG_BN + 4];
     const int64_t m0 = (int64_t)blockIdx.x * SG_BM;
@@ -110,7 +111,7 @@ static void gemm_simt(Exec &ex, int64_t M, int N, int64_t K, const TA *A, int64_
 {
     if (M <= 0 || N <= 0) return;
     dim3 grid((unsigned)ceil_div64(M, SG_BM), (unsigned)ceil_div64(N, SG_BN), 1);
-    gemm_simt_kernel<TA, TB, TC, A_MCONTIG, B_NCONTIG><<<grid, SG_THREADS, 0, ex.st>>>(M, N, K, A, lda, B, ldb, C, ldc, bias, relu, K > 0 ? K : 1, nullptr, row_scale, scale_col0);
+    launch_dep(gemm_simt_kernel<TA, TB, TC, A_MCONTIG, B_NCONTIG>, dim3(grid), dim3(SG_THREADS), 0, ex.st, M, N, K, A, lda, B, ldb, C, ldc, bias, relu, K > 0 ? K : 1, nullptr, row_scale, scale_col0);
     ex.launches += 1;
 }
 
@@ -127,7 +128,7 @@ static void weight_grad_simt(Exec &ex, int64_t rows, int Kin, int N, const T *A,
     int64_t k_chunk = ceil_div64(ceil_div64(rows, splits), SG_BK) * SG_BK;
     if (k_chunk < SG_BK) k_chunk = SG_BK;
     dim3 grid((unsigned)ceil_div64(Kin, SG_BM), (unsigned)ceil_div64(N, SG_BN), (unsigned)splits);
-    gemm_simt_kernel<T, T, float, true, true><<<grid, SG_THREADS, 0, ex.st>>>(Kin, N, rows, A, lda, dZ, ldz, (float *)nullptr, 0, nullptr, 0, k_chunk, partials);
+    launch_dep(gemm_simt_kernel<T, T, float, true, true>, dim3(grid), dim3(SG_THREADS), 0, ex.st, Kin, N, rows, A, lda, dZ, ldz, (float *)nullptr, 0, nullptr, 0, k_chunk, partials, nullptr, 0);
     const int64_t count = (int64_t)Kin * N;
     launch_dep(reduce_partials_kernel, dim3((unsigned)ceil_div64(count, 256)), dim3(256), 0, ex.st, partials, count, splits, dW, accumulate);
     ex.launches += 2;
@@ -140,6 +141,7 @@ template <typename T>
 __global__ void __launch_bounds__(256) colsum_partial_kernel(const T *__restrict__ dZ, int64_t rows, int N, int64_t ldz, int64_t rows_per_block,
                                                              float *__restrict__ partials)
 {
+    LP_DEP_ENTER();
     constexpr int VN = Vec16<T>::N;
     __shared__ float sh[256 * VN];
     const int nvec = N / VN;           // column vectors per row (<= 256)
@@ -188,6 +190,7 @@ __global__ void __launch_bounds__(256) colsum_partial_kernel(const T *__restrict
 __global__ void __launch_bounds__(256) reduce_partials_short_kernel(const float *__restrict__ partials, int count, int splits, float *__restrict__ dst,
                                                                     int accumulate)
 {
+    LP_DEP_ENTER();
     __shared__ float sh[8][32];
     const int c = blockIdx.x * 32 + (threadIdx.x & 31), g = threadIdx.x >> 5;
     const int per = (splits + 7) / 8;
@@ -213,7 +216,7 @@ static void colsum(Exec &ex, const T *dZ, int64_t rows, int N, int64_t ldz, floa
 {
     const int splits = colsum_splits(rows);
     const int64_t rpb = ceil_div64(rows > 0 ? rows : 1, splits);
-    colsum_partial_kernel<T><<<splits, 256, 0, ex.st>>>(dZ, rows, N, ldz, rpb, partials);
-    reduce_partials_short_kernel<<<(unsigned)ceil_div64(N, 32), 256, 0, ex.st>>>(partials, N, splits, out, accumulate);
+    launch_dep(colsum_partial_kernel<T>, dim3(splits), dim3(256), 0, ex.st, dZ, rows, N, ldz, rpb, partials);
+    launch_dep(reduce_partials_short_kernel, dim3((unsigned)ceil_div64(N, 32)), dim3(256), 0, ex.st, partials, N, splits, out, accumulate);
     ex.launches += 2;
 }

@@ -1181,6 +1181,7 @@ static bool tc_gemm_kmajor(TcState &tc, Exec &ex, int64_t M, int N, int K, const
 // C = act(A B + bias) with a BF16 B operand given as [K, N] (b_is_nk = false: transposed into the scratch first) or [N, K] (b_is_nk = true)
 __global__ void transpose_bf16_kernel(const bf16 *__restrict__ B, int K, int N, bf16 *__restrict__ Bt)
 {
+    LP_DEP_ENTER();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= K * N) return;
     const int k = i / N, n = i - k * N;
@@ -1192,7 +1193,7 @@ static bool tc_linear_bf16_b(TcState &tc, Exec &ex, int64_t M, int N, int K, con
 {
     const bf16 *Bt = B;
     if (!b_is_nk) {
-        transpose_bf16_kernel<<<(K * N + 255) / 256, 256, 0, ex.st>>>(B, K, N, tc.wbuf);
+        launch_dep(transpose_bf16_kernel, dim3((K * N + 255) / 256), dim3(256), 0, ex.st, B, K, N, tc.wbuf);
         ex.launches += 1;
         Bt = tc.wbuf;
     }

@@ -214,6 +214,7 @@ static double gemm_bytes(double M, double N, double K, double s_in, double s_out
 __global__ void validate_csr_kernel(const int64_t *__restrict__ rowptr64, int n, int64_t nnz, const int *__restrict__ col, int *__restrict__ rowptr32,
                                     int *__restrict__ err)
 {
+    LP_DEP_ENTER();
     const int v = blockIdx.x * blockDim.x + threadIdx.x;
     if (v > n) return;
     const int64_t a = rowptr64[v];
@@ -238,6 +239,7 @@ __global__ void validate_csr_kernel(const int64_t *__restrict__ rowptr64, int n,
 __global__ void degree_kernel(const int *__restrict__ rowptr, const float *__restrict__ w, int n, float *__restrict__ dtilde, float *__restrict__ gcn_self,
                               float *__restrict__ inv_deg)
 {
+    LP_DEP_ENTER();
     const int v = blockIdx.x * blockDim.x + threadIdx.x;
     if (v >= n) return;
     const int a = rowptr[v], b = rowptr[v + 1];
@@ -252,6 +254,7 @@ __global__ void degree_kernel(const int *__restrict__ rowptr, const float *__res
 __global__ void gcn_val_kernel(const int *__restrict__ rows, const int *__restrict__ col, const float *__restrict__ w, const float *__restrict__ dtilde,
                                int64_t nnz, float *__restrict__ val)
 {
+    LP_DEP_ENTER();
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= nnz) return;
     val[e] = (w ? w[e] : 1.f) / sqrtf(dtilde[rows[e]] * dtilde[col[e]]);
@@ -259,6 +262,7 @@ __global__ void gcn_val_kernel(const int *__restrict__ rows, const int *__restri
 
 __global__ void widen_i32_kernel(const int *__restrict__ src, int64_t m, int64_t *__restrict__ dst)
 {
+    LP_DEP_ENTER();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < m) dst[i] = src[i];
 }
@@ -382,7 +386,7 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
     CK(e);
 
     cudaMemsetAsync(ctx->err_flag, 0, sizeof(int), st);
-    validate_csr_kernel<<<nblk(n + 1), 256, 0, st>>>(rowptr64, (int)n, nnz, ctx->col, ctx->rowptr, ctx->err_flag);
+    launch_dep(validate_csr_kernel, dim3(nblk(n + 1)), dim3(256), 0, st, rowptr64, (int)n, nnz, ctx->col, ctx->rowptr, ctx->err_flag);
     int flag = 0;
     e = cudaMemcpyAsync(&flag, ctx->err_flag, sizeof(int), cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
@@ -420,13 +424,13 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
     GALLOC(ctx->gcn_val, nnz);
     GALLOC(ctx->gcn_valT, nnz);
     GALLOC(ctx->meanT_val, nnz);
-    degree_kernel<<<nblk(n), 256, 0, st>>>(ctx->rowptr, ctx->w, (int)n, dtilde, ctx->gcn_self, ctx->inv_deg);
+    launch_dep(degree_kernel, dim3(nblk(n)), dim3(256), 0, st, ctx->rowptr, ctx->w, (int)n, dtilde, ctx->gcn_self, ctx->inv_deg);
     if (nnz > 0) {
-        gcn_val_kernel<<<nblk(nnz), 256, 0, st>>>(ts.rows, ctx->col, ctx->w, dtilde, nnz, ctx->gcn_val);
-        gather_f32_kernel<<<nblk(nnz), 256, 0, st>>>(ctx->gcn_val, ctx->perm, nnz, ctx->gcn_valT);
-        gather_f32_kernel<<<nblk(nnz), 256, 0, st>>>(ctx->inv_deg, ctx->rowidx, nnz, ctx->meanT_val);
+        launch_dep(gcn_val_kernel, dim3(nblk(nnz)), dim3(256), 0, st, ts.rows, ctx->col, ctx->w, dtilde, nnz, ctx->gcn_val);
+        launch_dep(gather_f32_kernel, dim3(nblk(nnz)), dim3(256), 0, st, ctx->gcn_val, ctx->perm, nnz, ctx->gcn_valT);
+        launch_dep(gather_f32_kernel, dim3(nblk(nnz)), dim3(256), 0, st, ctx->inv_deg, ctx->rowidx, nnz, ctx->meanT_val);
     }
-    convert_kernel<float, bf16><<<nblk(n * (int64_t)f), 256, 0, st>>>(ctx->X32, ctx->X16, n * (int64_t)f);
+    launch_dep(convert_kernel<float, bf16>, dim3(nblk(n * (int64_t)f)), dim3(256), 0, st, ctx->X32, ctx->X16, n * (int64_t)f);
     ctx->ex.launches += 6;
     // heavy-row plans of the graph and of its transpose (static: built once)
     const int64_t item_cap = nnz / 64 + 2;  // static plans cut rows above 128 entries into pieces of 128 or items of 512: at most deg / 64 of them per row
@@ -472,9 +476,9 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
         TALLOC(chunk_of, n + 1);
         cudaMemsetAsync(pp.counts, 0, 2 * sizeof(int), st);
         launch_dep(spmm_heavy_plan_kernel, dim3(nblk(n)), dim3(256), 0, st, sp, (int)n, nullptr, pp, row_base);
-        padded_count_kernel<<<nblk(n), 256, 0, st>>>(sp, (int)n, SPMM_PIECE, first_group);
+        launch_dep(padded_count_kernel, dim3(nblk(n)), dim3(256), 0, st, sp, (int)n, SPMM_PIECE, first_group);
         exclusive_scan_i32(ctx->ex, first_group, n, first_group, first_group + n, ts.scan_tmp);
-        padded_chunk_count_kernel<<<nblk(n), 256, 0, st>>>(sp, first_group, (int)n, SPMM_PIECE, chunk_count);
+        launch_dep(padded_chunk_count_kernel, dim3(nblk(n)), dim3(256), 0, st, sp, first_group, (int)n, SPMM_PIECE, chunk_count);
         exclusive_scan_i32(ctx->ex, chunk_count, n, chunk_of, chunk_of + n, ts.scan_tmp);
         cudaMemcpyAsync(ctx->host_counts + 8, first_group + n, sizeof(int), cudaMemcpyDeviceToHost, st);
         cudaMemcpyAsync(ctx->host_counts + 9, chunk_of + n, sizeof(int), cudaMemcpyDeviceToHost, st);
@@ -490,7 +494,7 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
         GALLOC(pval, 4 * n_groups + 4);
         GALLOC(grow, n_groups + 1);
         GALLOC(chunk_start, (int64_t)n_chunks + 2);
-        padded_fill_kernel<<<nblk(n), 256, 0, st>>>(sp, sc, sv, (int)n, SPMM_PIECE, first_group, chunk_count, chunk_of, row_base, chunk_start, pcol, pval, grow);
+        launch_dep(padded_fill_kernel, dim3(nblk(n)), dim3(256), 0, st, sp, sc, sv, (int)n, SPMM_PIECE, first_group, chunk_count, chunk_of, row_base, chunk_start, pcol, pval, grow);
         ctx->ex.launches += 5;
         e = cudaStreamSynchronize(st);
         if (e != cudaSuccess) break;
@@ -500,7 +504,7 @@ extern "C" lp_status lp_load_graph(lp_ctx *ctx, int64_t n, int64_t nnz, const in
         if (!csr) {  // the transposed structure also carries the mean's coefficients 1 / |N(v)| of the entry's source row v
             float *pval2 = nullptr;
             GALLOC(pval2, 4 * n_groups + 4);
-            padded_fill_kernel<<<nblk(n), 256, 0, st>>>(sp, sc, ctx->meanT_val, (int)n, SPMM_PIECE, first_group, chunk_count, chunk_of, row_base, chunk_start, pcol, pval2, grow);
+            launch_dep(padded_fill_kernel, dim3(nblk(n)), dim3(256), 0, st, sp, sc, ctx->meanT_val, (int)n, SPMM_PIECE, first_group, chunk_count, chunk_of, row_base, chunk_start, pcol, pval2, grow);
             ctx->ex.launches += 1;
             e = cudaStreamSynchronize(st);
             if (e != cudaSuccess) break;
@@ -534,9 +538,9 @@ extern "C" lp_status lp_get_structure(lp_ctx *ctx, int64_t *colptr, int32_t *row
     if (!ctx->loaded) return fail(ctx, LP_ESTATE, "lp_get_structure: no graph loaded");
     CK(cudaSetDevice(ctx->device));
     cudaStream_t st = ctx->ex.st;
-    if (colptr) widen_i32_kernel<<<nblk(ctx->n + 1), 256, 0, st>>>(ctx->colptr, ctx->n + 1, colptr);
+    if (colptr) launch_dep(widen_i32_kernel, dim3(nblk(ctx->n + 1)), dim3(256), 0, st, ctx->colptr, ctx->n + 1, colptr);
     if (rowidx && ctx->nnz > 0) CK(cudaMemcpyAsync(rowidx, ctx->rowidx, sizeof(int) * (size_t)ctx->nnz, cudaMemcpyDeviceToDevice, st));
-    if (perm && ctx->nnz > 0) widen_i32_kernel<<<nblk(ctx->nnz), 256, 0, st>>>(ctx->perm, ctx->nnz, perm);
+    if (perm && ctx->nnz > 0) launch_dep(widen_i32_kernel, dim3(nblk(ctx->nnz)), dim3(256), 0, st, ctx->perm, ctx->nnz, perm);
     CK_LAUNCH();
     return LP_OK;
 }
@@ -558,7 +562,7 @@ extern "C" lp_status lp_set_candidates(lp_ctx *ctx, const int32_t *cand, int64_t
     if (n_cand >= (int64_t)1 << 31) return fail(ctx, LP_EINVAL, "lp_set_candidates: too many candidates");
     GALLOC(ctx->cand, n_cand);  // lives with the graph
     CK(cudaMemcpyAsync(ctx->cand, cand, sizeof(int) * (size_t)n_cand, cudaMemcpyDeviceToDevice, ctx->ex.st));
-    check_ids_kernel<<<nblk(n_cand), 256, 0, ctx->ex.st>>>(ctx->cand, n_cand, ctx->n, ctx->err_flag);
+    launch_dep(check_ids_kernel, dim3(nblk(n_cand)), dim3(256), 0, ctx->ex.st, ctx->cand, n_cand, ctx->n, ctx->err_flag);
     int bad = 0;
     CK(cudaMemcpyAsync(&bad, ctx->err_flag, sizeof bad, cudaMemcpyDeviceToHost, ctx->ex.st));
     CK(cudaStreamSynchronize(ctx->ex.st));
@@ -603,19 +607,19 @@ extern "C" lp_status lp_sparsify(lp_ctx *ctx, double alpha, uint64_t seed, int64
     SALLOC(scan_tmp, ceil_div64(m, SCAN_TILE) + 2);
     SALLOC(ctx->sp_ptr, n + 1);
     // non-isolated nodes, ascending
-    sp_nonisolated_kernel<<<nblk(n), 256, 0, st>>>(ctx->rowptr, n, flags);
+    launch_dep(sp_nonisolated_kernel, dim3(nblk(n)), dim3(256), 0, st, ctx->rowptr, n, flags);
     exclusive_scan_i32(ctx->ex, flags, n, pos, pos + n, scan_tmp);
-    sp_compact_kernel<<<nblk(n), 256, 0, st>>>(ctx->rowptr, pos, n, nz);
+    launch_dep(sp_compact_kernel, dim3(nblk(n)), dim3(256), 0, st, ctx->rowptr, pos, n, nz);
     int n_nz = 0, dummy = 0;
     lp_status s = sync_counts(ctx, pos + n, nullptr, &n_nz, &dummy);
     if (s != LP_OK) return s;
     CK(cudaMemsetAsync(hits, 0, sizeof(int) * (size_t)(nnz + 1), st));
     CK(cudaMemsetAsync(ctx->err_flag, 0, sizeof(int), st));
     if (L > 0 && n_nz > 0)
-        sp_draw_kernel<<<nblk(L), 256, 0, st>>>(ctx->rowptr, ctx->col, nz, (uint32_t)n_nz, make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)), L, hits,
+        launch_dep(sp_draw_kernel, dim3(nblk(L)), dim3(256), 0, st, ctx->rowptr, ctx->col, nz, (uint32_t)n_nz, make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)), L, hits,
                                                 ctx->err_flag);
     // kept entries -> positions; pos has nnz + 1 slots so that pos[rowptr[n]] is the total
-    sp_keep_flags_kernel<<<nblk(nnz + 1), 256, 0, st>>>(hits, nnz + 1, flags);
+    launch_dep(sp_keep_flags_kernel, dim3(nblk(nnz + 1)), dim3(256), 0, st, hits, nnz + 1, flags);
     exclusive_scan_i32(ctx->ex, flags, nnz + 1, pos, nullptr, scan_tmp);
     int kept = 0, bad = 0;
     s = sync_counts(ctx, pos + nnz, ctx->err_flag, &kept, &bad);
@@ -626,7 +630,7 @@ extern "C" lp_status lp_sparsify(lp_ctx *ctx, double alpha, uint64_t seed, int64
     }
     SALLOC(ctx->sp_col, kept);
     SALLOC(ctx->sp_w, kept);
-    sp_emit_kernel<<<nblk(n + 1), 256, 0, st>>>(ctx->rowptr, ctx->col, hits, pos, n, (double)n_nz, (double)std::max<int64_t>(L, 1), ctx->sp_ptr, ctx->sp_col,
+    launch_dep(sp_emit_kernel, dim3(nblk(n + 1)), dim3(256), 0, st, ctx->rowptr, ctx->col, hits, pos, n, (double)n_nz, (double)std::max<int64_t>(L, 1), ctx->sp_ptr, ctx->sp_col,
                                                 ctx->sp_w);
     ctx->ex.launches += 5;
     CK(cudaStreamSynchronize(st));
@@ -674,7 +678,7 @@ extern "C" lp_status lp_worker_view(lp_ctx *ctx, const int32_t *part, int32_t wo
     VALLOC(scan_tmp, ceil_div64(n + 1, SCAN_TILE) + 2);
     VALLOC(dstats, 8);
     CK(cudaMemsetAsync(dstats, 0, 8 * sizeof(unsigned long long), st));
-    view_count_kernel<<<nblk(n), 256, 0, st>>>(n, ctx->rowptr, ctx->col, part, worker, keep_cross_edges, foreign_mode, ctx->sp_ptr, ctx->view_ptr, dstats);
+    launch_dep(view_count_kernel, dim3(nblk(n)), dim3(256), 0, st, n, ctx->rowptr, ctx->col, part, worker, keep_cross_edges, foreign_mode, ctx->sp_ptr, ctx->view_ptr, dstats);
     exclusive_scan_i32(ctx->ex, ctx->view_ptr, n, ctx->view_ptr, ctx->view_ptr + n, scan_tmp);
     unsigned long long hs[4] = {0, 0, 0, 0};
     CK(cudaMemcpyAsync(hs, dstats, sizeof hs, cudaMemcpyDeviceToHost, st));
@@ -682,7 +686,7 @@ extern "C" lp_status lp_worker_view(lp_ctx *ctx, const int32_t *part, int32_t wo
     const unsigned long long total = hs[0] + hs[1];
     if (total >= (1ull << 31)) return fail(ctx, LP_EINVAL, "lp_worker_view: the view has 2^31 entries or more");
     VALLOC(ctx->view_col, (int64_t)total);
-    view_fill_kernel<<<nblk(n), 256, 0, st>>>(n, ctx->rowptr, ctx->col, part, worker, keep_cross_edges, foreign_mode, ctx->sp_ptr, ctx->sp_col,
+    launch_dep(view_fill_kernel, dim3(nblk(n)), dim3(256), 0, st, n, ctx->rowptr, ctx->col, part, worker, keep_cross_edges, foreign_mode, ctx->sp_ptr, ctx->sp_col,
                                               ctx->view_ptr, ctx->view_col);
     ctx->ex.launches += 2;
     CK(cudaStreamSynchronize(st));
@@ -704,7 +708,7 @@ extern "C" lp_status lp_get_worker_view(lp_ctx *ctx, int64_t *rowptr, int32_t *c
     if (ctx->view_nnz < 0) return fail(ctx, LP_ESTATE, "lp_get_worker_view: call lp_worker_view first");
     CK(cudaSetDevice(ctx->device));
     cudaStream_t st = ctx->ex.st;
-    if (rowptr) widen_i32_kernel<<<nblk(ctx->n + 1), 256, 0, st>>>(ctx->view_ptr, ctx->n + 1, rowptr);
+    if (rowptr) launch_dep(widen_i32_kernel, dim3(nblk(ctx->n + 1)), dim3(256), 0, st, ctx->view_ptr, ctx->n + 1, rowptr);
     if (col && ctx->view_nnz > 0) CK(cudaMemcpyAsync(col, ctx->view_col, sizeof(int) * (size_t)ctx->view_nnz, cudaMemcpyDeviceToDevice, st));
     CK_LAUNCH();
     return LP_OK;
@@ -831,9 +835,9 @@ extern "C" lp_status lp_set_model(lp_ctx *ctx, const lp_model_desc *d, int64_t m
     if (sage && !sampled) {  // the left half of the first operand is X itself, written once
         LayerBuf &L = ctx->layer[0];
         if (d->prec == LP_BF16)
-            copy_rows_kernel<bf16, bf16><<<nblk(n * L.Fi), 256, 0, ctx->ex.st>>>(ctx->X16, L.Fi, (bf16 *)L.A, L.Kin, n, L.Fi);
+            launch_dep(copy_rows_kernel<bf16, bf16>, dim3(nblk(n * L.Fi)), dim3(256), 0, ctx->ex.st, ctx->X16, L.Fi, (bf16 *)L.A, L.Kin, n, L.Fi);
         else
-            copy_rows_kernel<float, float><<<nblk(n * L.Fi), 256, 0, ctx->ex.st>>>(ctx->X32, L.Fi, (float *)L.A, L.Kin, n, L.Fi);
+            launch_dep(copy_rows_kernel<float, float>, dim3(nblk(n * L.Fi)), dim3(256), 0, ctx->ex.st, ctx->X32, L.Fi, (float *)L.A, L.Kin, n, L.Fi);
         ctx->ex.launches += 1;
     }
     for (int i = 0; i < 2; ++i) { MALLOC(p, max_rows * maxF * (int64_t)es); ctx->dZ[i] = p; }
@@ -1114,9 +1118,9 @@ static void gcn_block_coefficients(lp_ctx *ctx, HopBlock &hb, HopBlock &prev)
 {
     cudaStream_t st = ctx->ex.st;
     if (hb.entries > 0)
-        gcn_block_coef_kernel<<<nblk(hb.entries), 256, 0, st>>>(ctx->rowptr, prev.frontier, hb.blk_ptr, hb.blk_row, hb.blk_eid, hb.blk_ptr + hb.n_dst,
+        launch_dep(gcn_block_coef_kernel, dim3(nblk(hb.entries)), dim3(256), 0, st, ctx->rowptr, prev.frontier, hb.blk_ptr, hb.blk_row, hb.blk_eid, hb.blk_ptr + hb.n_dst,
                                                                 ctx->gcn_val, hb.blk_val);
-    if (hb.n_dst > 0) gather_by_id_kernel<<<nblk(hb.n_dst), 256, 0, st>>>(ctx->gcn_self, prev.frontier, prev.n_front_dev, hb.cap_dst, hb.self_coef_dst);
+    if (hb.n_dst > 0) launch_dep(gather_by_id_kernel, dim3(nblk(hb.n_dst)), dim3(256), 0, st, ctx->gcn_self, prev.frontier, prev.n_front_dev, hb.cap_dst, hb.self_coef_dst);
     ctx->ex.launches += 2;
 }
 
@@ -1131,10 +1135,10 @@ static lp_status build_blocks(lp_ctx *ctx, const int *pos_src, const int *pos_ds
     const bool gcn = ctx->desc.arch == LP_GCN;
     ProfScope prof(ctx->ex, LP_PROF_BLOCKS);
     CK(cudaMemsetAsync(ctx->mark, 0, (size_t)n, st));
-    mark_ids_kernel<<<nblk(B), 256, 0, st>>>(pos_src, B, n, ctx->mark);
-    mark_ids_kernel<<<nblk(B), 256, 0, st>>>(pos_dst, B, n, ctx->mark);
-    if (k > 0) mark_ids_kernel<<<nblk(B * k), 256, 0, st>>>(neg_dst, B * k, n, ctx->mark);
-    if (k > 0 && neg_src) mark_ids_kernel<<<nblk(B * k), 256, 0, st>>>(neg_src, B * k, n, ctx->mark);
+    launch_dep(mark_ids_kernel, dim3(nblk(B)), dim3(256), 0, st, pos_src, B, n, ctx->mark);
+    launch_dep(mark_ids_kernel, dim3(nblk(B)), dim3(256), 0, st, pos_dst, B, n, ctx->mark);
+    if (k > 0) launch_dep(mark_ids_kernel, dim3(nblk(B * k)), dim3(256), 0, st, neg_dst, B * k, n, ctx->mark);
+    if (k > 0 && neg_src) launch_dep(mark_ids_kernel, dim3(nblk(B * k)), dim3(256), 0, st, neg_src, B * k, n, ctx->mark);
     ctx->ex.launches += 4;
     for (int h = 0; h <= K; ++h) {
         HopBlock &hb = ctx->hop[h];
@@ -1142,22 +1146,22 @@ static lp_status build_blocks(lp_ctx *ctx, const int *pos_src, const int *pos_ds
             HopBlock &prev = ctx->hop[h - 1];
             hb.n_dst = prev.n_src;
             // sample: counts -> offsets -> columns (also marks the sampled ids; F_{h-1} is still marked)
-            nbr_count_kernel<<<nblk(hb.n_dst + 1), 256, 0, st>>>(ctx->rowptr, prev.frontier, prev.n_front_dev, ctx->desc.fanout[h - 1], hb.blk_ptr, hb.n_dst);
+            launch_dep(nbr_count_kernel, dim3(nblk(hb.n_dst + 1)), dim3(256), 0, st, ctx->rowptr, prev.frontier, prev.n_front_dev, ctx->desc.fanout[h - 1], hb.blk_ptr, hb.n_dst);
             exclusive_scan_i32(ctx->ex, hb.blk_ptr, hb.n_dst, hb.blk_ptr, hb.blk_ptr + hb.n_dst, ctx->scan_tmp);
             {
                 const int fo = ctx->desc.fanout[h - 1];
                 const uint32_t st32 = (uint32_t)step, h32 = (uint32_t)h;
                 if (fo <= 8)
-                    nbr_sample_kernel<8><<<nblk((int64_t)hb.n_dst * 8), 256, 0, st>>>(ctx->rowptr, ctx->col, prev.frontier, prev.n_front_dev, fo, key, st32, h32,
+                    launch_dep(nbr_sample_kernel<8>, dim3(nblk((int64_t)hb.n_dst * 8)), dim3(256), 0, st, ctx->rowptr, ctx->col, prev.frontier, prev.n_front_dev, fo, key, st32, h32,
                                                                                       hb.blk_ptr, hb.blk_col_global, hb.blk_row, ctx->mark, hb.blk_eid);
                 else if (fo <= 16)
-                    nbr_sample_kernel<16><<<nblk((int64_t)hb.n_dst * 16), 256, 0, st>>>(ctx->rowptr, ctx->col, prev.frontier, prev.n_front_dev, fo, key, st32, h32,
+                    launch_dep(nbr_sample_kernel<16>, dim3(nblk((int64_t)hb.n_dst * 16)), dim3(256), 0, st, ctx->rowptr, ctx->col, prev.frontier, prev.n_front_dev, fo, key, st32, h32,
                                                                                         hb.blk_ptr, hb.blk_col_global, hb.blk_row, ctx->mark, hb.blk_eid);
                 else
-                    nbr_sample_kernel<32><<<nblk((int64_t)hb.n_dst * 32), 256, 0, st>>>(ctx->rowptr, ctx->col, prev.frontier, prev.n_front_dev, fo, key, st32, h32,
+                    launch_dep(nbr_sample_kernel<32>, dim3(nblk((int64_t)hb.n_dst * 32)), dim3(256), 0, st, ctx->rowptr, ctx->col, prev.frontier, prev.n_front_dev, fo, key, st32, h32,
                                                                                         hb.blk_ptr, hb.blk_col_global, hb.blk_row, ctx->mark, hb.blk_eid);
             }
-            inv_degree_kernel<<<nblk(hb.n_dst), 256, 0, st>>>(hb.blk_ptr, hb.n_dst, nullptr, hb.inv_deg);
+            launch_dep(inv_degree_kernel, dim3(nblk(hb.n_dst)), dim3(256), 0, st, hb.blk_ptr, hb.n_dst, nullptr, hb.inv_deg);
             ctx->ex.launches += 3;
             if (h == K) {  // outermost hop: only the entry count is needed
                 int entries = 0, dummy = 0;
@@ -1170,9 +1174,9 @@ static lp_status build_blocks(lp_ctx *ctx, const int *pos_src, const int *pos_ds
             }
         }
         // frontier F_h from the marks
-        mark_to_int_kernel<<<nblk(n), 256, 0, st>>>(ctx->mark, n, ctx->flags);
+        launch_dep(mark_to_int_kernel, dim3(nblk(n)), dim3(256), 0, st, ctx->mark, n, ctx->flags);
         exclusive_scan_i32(ctx->ex, ctx->flags, n, hb.posmap, hb.n_front_dev, ctx->scan_tmp);
-        compact_frontier_kernel<<<nblk(n), 256, 0, st>>>(ctx->mark, hb.posmap, n, hb.frontier);
+        launch_dep(compact_frontier_kernel, dim3(nblk(n)), dim3(256), 0, st, ctx->mark, hb.posmap, n, hb.frontier);
         ctx->ex.launches += 2;
         int nf = 0, entries = 0;
         lp_status s = sync_counts(ctx, hb.n_front_dev, h >= 1 ? hb.blk_ptr + hb.n_dst : nullptr, &nf, &entries);
@@ -1181,18 +1185,18 @@ static lp_status build_blocks(lp_ctx *ctx, const int *pos_src, const int *pos_ds
         if (h >= 1) {
             hb.entries = entries;
             // local ids, self positions, transposed block
-            fill_i32_kernel<<<nblk(hb.n_src), 256, 0, st>>>(hb.inv_self, hb.n_src, -1);
-            self_index_kernel<<<nblk(hb.n_dst), 256, 0, st>>>(ctx->hop[h - 1].frontier, ctx->hop[h - 1].n_front_dev, hb.posmap, hb.self_idx, hb.inv_self);
+            launch_dep(fill_i32_kernel, dim3(nblk(hb.n_src)), dim3(256), 0, st, hb.inv_self, hb.n_src, -1);
+            launch_dep(self_index_kernel, dim3(nblk(hb.n_dst)), dim3(256), 0, st, ctx->hop[h - 1].frontier, ctx->hop[h - 1].n_front_dev, hb.posmap, hb.self_idx, hb.inv_self);
             ctx->ex.launches += 2;
             if (hb.entries > 0) {
-                relabel_kernel<<<nblk(hb.entries), 256, 0, st>>>(hb.blk_col_global, hb.blk_ptr + hb.n_dst, hb.entries, hb.posmap, hb.blk_col_local);
+                launch_dep(relabel_kernel, dim3(nblk(hb.entries)), dim3(256), 0, st, hb.blk_col_global, hb.blk_ptr + hb.n_dst, hb.entries, hb.posmap, hb.blk_col_local);
                 ctx->ex.launches += 1;
             }
             transpose_csr(ctx->ex, hb.blk_ptr, hb.n_dst, hb.n_src, hb.blk_col_local, hb.entries, hb.colptr, hb.rowidx, hb.perm, ctx->tsp, hb.blk_row);
             if (gcn) {
                 gcn_block_coefficients(ctx, hb, ctx->hop[h - 1]);
-                if (hb.entries > 0) gather_f32_kernel<<<nblk(hb.entries), 256, 0, st>>>(hb.blk_val, hb.perm, hb.entries, hb.blk_valT);
-                gather_by_id_kernel<<<nblk(hb.n_src), 256, 0, st>>>(ctx->gcn_self, hb.frontier, hb.n_front_dev, hb.cap_src, hb.self_coef_src);
+                if (hb.entries > 0) launch_dep(gather_f32_kernel, dim3(nblk(hb.entries)), dim3(256), 0, st, hb.blk_val, hb.perm, hb.entries, hb.blk_valT);
+                launch_dep(gather_by_id_kernel, dim3(nblk(hb.n_src)), dim3(256), 0, st, ctx->gcn_self, hb.frontier, hb.n_front_dev, hb.cap_src, hb.self_coef_src);
                 ctx->ex.launches += 2;
             }
         }
@@ -1313,15 +1317,15 @@ static lp_status predictor_forward(lp_ctx *ctx, const float *params, const int *
     const int chunks = D / VN;
     const unsigned blocks = nblk(E, EDGE_THREADS / 32);
     T *Z0 = tptr<T>(ctx->pred[0].A), *P1 = tptr<T>(ctx->pred[1].A), *P2 = tptr<T>(ctx->P2), *HK = tptr<T>(ctx->HK);
-    if (chunks <= 32) edge_hadamard_kernel<T, 1><<<blocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, Z0);
-    else if (chunks <= 64) edge_hadamard_kernel<T, 2><<<blocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, Z0);
-    else edge_hadamard_kernel<T, 4><<<blocks, EDGE_THREADS, 0, st>>>(HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, Z0);
+    if (chunks <= 32) launch_dep(edge_hadamard_kernel<T, 1>, dim3(blocks), dim3(EDGE_THREADS), 0, st, HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, Z0);
+    else if (chunks <= 64) launch_dep(edge_hadamard_kernel<T, 2>, dim3(blocks), dim3(EDGE_THREADS), 0, st, HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, Z0);
+    else launch_dep(edge_hadamard_kernel<T, 4>, dim3(blocks), dim3(EDGE_THREADS), 0, st, HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, Z0);
     ctx->ex.launches += 1;
     lp_status s = layer_linear<T>(ctx, E, ctx->pred[0], params, P1, Hp, true);
     if (s != LP_OK) return s;
     s = layer_linear<T>(ctx, E, ctx->pred[1], params, P2, Hp, true);
     if (s != LP_OK) return s;
-    edge_gemv_kernel<T><<<blocks, EDGE_THREADS, 0, st>>>(P2, Hp, E, params + ctx->off_w2, params + ctx->off_b2, ctx->pred_scores);
+    launch_dep(edge_gemv_kernel<T>, dim3(blocks), dim3(EDGE_THREADS), 0, st, P2, Hp, E, params + ctx->off_w2, params + ctx->off_b2, ctx->pred_scores);
     ctx->ex.launches += 1;
     CK_LAUNCH();
     return LP_OK;
@@ -1337,15 +1341,15 @@ static lp_status predictor_backward(lp_ctx *ctx, const float *params, int64_t E,
     // last layer: dw2 = P2^T g, db2 = sum g (two fixed-order stages)
     const int splits = colsum_splits(E);
     const int64_t rpb = ceil_div64(E, splits);
-    pred_last_layer_grad_kernel<T><<<splits, 256, 0, st>>>(P2, Hp, E, g, rpb, ctx->partials);
-    reduce_partials_short_kernel<<<nblk(Hp + 1, 32), 256, 0, st>>>(ctx->partials, Hp + 1, splits, grads + ctx->off_w2, accumulate);
-    pred_out_grad_kernel<T><<<nblk(E * Hp), 256, 0, st>>>(P2, Hp, E, g, params + ctx->off_w2, dPa);
+    launch_dep(pred_last_layer_grad_kernel<T>, dim3(splits), dim3(256), 0, st, P2, Hp, E, g, rpb, ctx->partials);
+    launch_dep(reduce_partials_short_kernel, dim3(nblk(Hp + 1, 32)), dim3(256), 0, st, ctx->partials, Hp + 1, splits, grads + ctx->off_w2, accumulate);
+    launch_dep(pred_out_grad_kernel<T>, dim3(nblk(E * Hp)), dim3(256), 0, st, P2, Hp, E, g, params + ctx->off_w2, dPa);
     ctx->ex.launches += 3;
     lp_status s = layer_weight_grad<T>(ctx, E, ctx->pred[1], dPa, ctx->pred[1].Fo, grads, accumulate);
     if (s != LP_OK) return s;
     s = layer_input_grad<T>(ctx, E, ctx->pred[1], params, dPa, ctx->pred[1].Fo, dPb, nullptr, 0);
     if (s != LP_OK) return s;
-    relu_mask_kernel<T><<<nblk(E * Hp), 256, 0, st>>>(dPb, P1, E * Hp);
+    launch_dep(relu_mask_kernel<T>, dim3(nblk(E * Hp)), dim3(256), 0, st, dPb, P1, E * Hp);
     ctx->ex.launches += 1;
     s = layer_weight_grad<T>(ctx, E, ctx->pred[0], dPb, ctx->pred[0].Fo, grads, accumulate);
     if (s != LP_OK) return s;
@@ -1396,7 +1400,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         s = predictor_forward<T>(ctx, params, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k);
         if (s != LP_OK) return s;
         const unsigned lblocks = nblk(E, 256);
-        bce_from_scores_kernel<<<lblocks, 256, 0, st>>>(ctx->pred_scores, E, B, inv_N, ctx->g_pos, ctx->loss_partials);
+        launch_dep(bce_from_scores_kernel, dim3(lblocks), dim3(256), 0, st, ctx->pred_scores, E, B, inv_N, ctx->g_pos, ctx->loss_partials);
         launch_dep(loss_reduce_kernel, dim3(1), dim3(1024), 0, st, ctx->loss_partials, lblocks, inv_N, loss);
         g_neg = ctx->g_pos + B;  // one array: positives, then negatives
         s = predictor_backward<T>(ctx, params, E, ctx->g_pos, grads, accumulate);
@@ -1416,7 +1420,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
 
     // incidence lists of the scored edges, grouped by node (slots claimed with integer atomics)
     std::unique_ptr<ProfScope> pinc(new ProfScope(ctx->ex, LP_PROF_INCIDENCE, (double)E * 2.0 * 24.0));
-    if (ctx->mlp) incidence_count_kernel<<<nblk(E), 256, 0, st>>>(ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->inc_ptr);
+    if (ctx->mlp) launch_dep(incidence_count_kernel, dim3(nblk(E)), dim3(256), 0, st, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->inc_ptr);
     exclusive_scan_i32_copy(ctx->ex, ctx->inc_ptr, rows_out, ctx->inc_ptr, ctx->inc_cursor, ctx->inc_ptr + rows_out, ctx->scan_tmp);
     launch_dep(incidence_fill_kernel, dim3(nblk(E)), dim3(256), 0, st, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, g_pos, g_neg, ctx->inc_cursor, ctx->inc_col,
                ctx->mlp ? nullptr : ctx->inc_val, ctx->mlp ? ctx->inc_edge : nullptr, ctx->plan_dyn.counts);
@@ -1635,7 +1639,7 @@ extern "C" lp_status lp_adam_step(lp_ctx *ctx, float *params, float *adam_m, flo
         launch_dep(adam_kernel, dim3(nblk(np)), dim3(256), 0, ctx->ex.st, params, adam_m, adam_v, grads, np, (float)grad_scale, (float)lr, (float)beta1, (float)(1.0 - beta1),
                                                       (float)beta2, (float)(1.0 - beta2), (float)eps, (float)(1.0 / c1), (float)(1.0 / c2));
     } else {
-        sgd_kernel<<<nblk(np), 256, 0, ctx->ex.st>>>(params, grads, np, (float)grad_scale, (float)lr);
+        launch_dep(sgd_kernel, dim3(nblk(np)), dim3(256), 0, ctx->ex.st, params, grads, np, (float)grad_scale, (float)lr);
     }
     ctx->ex.launches += 1;
     CK_LAUNCH();
@@ -1707,9 +1711,9 @@ static lp_status score_impl(lp_ctx *ctx, const float *params, const int *src, co
         return LP_OK;
     }
     const unsigned blocks = nblk(E, EDGE_THREADS / 32);
-    if (chunks <= 32) edge_score_kernel<T, 1><<<blocks, EDGE_THREADS, 0, ctx->ex.st>>>(tptr<T>(ctx->HK), D, D, ctx->n, idmap, src, dst, E, scores);
-    else if (chunks <= 64) edge_score_kernel<T, 2><<<blocks, EDGE_THREADS, 0, ctx->ex.st>>>(tptr<T>(ctx->HK), D, D, ctx->n, idmap, src, dst, E, scores);
-    else edge_score_kernel<T, 4><<<blocks, EDGE_THREADS, 0, ctx->ex.st>>>(tptr<T>(ctx->HK), D, D, ctx->n, idmap, src, dst, E, scores);
+    if (chunks <= 32) launch_dep(edge_score_kernel<T, 1>, dim3(blocks), dim3(EDGE_THREADS), 0, ctx->ex.st, tptr<T>(ctx->HK), D, D, ctx->n, idmap, src, dst, E, scores);
+    else if (chunks <= 64) launch_dep(edge_score_kernel<T, 2>, dim3(blocks), dim3(EDGE_THREADS), 0, ctx->ex.st, tptr<T>(ctx->HK), D, D, ctx->n, idmap, src, dst, E, scores);
+    else launch_dep(edge_score_kernel<T, 4>, dim3(blocks), dim3(EDGE_THREADS), 0, ctx->ex.st, tptr<T>(ctx->HK), D, D, ctx->n, idmap, src, dst, E, scores);
     ctx->ex.launches += 1;
     CK_LAUNCH();
     return LP_OK;
@@ -1769,10 +1773,10 @@ extern "C" lp_status lp_hits_at_k(lp_ctx *ctx, const float *pos_scores, int64_t 
     if (e == cudaSuccess) e = dev_alloc(ctx, tmp, tmp_bytes, &sc.scan_tmp, SortScratch::scan_ints(n_neg));
     if (e == cudaSuccess) e = dev_alloc(ctx, tmp, tmp_bytes, &count, 8);
     if (e != cudaSuccess) { free_list(tmp); CK(e); }
-    float_keys_kernel<<<nblk(n_neg), 256, 0, st>>>(neg_scores, n_neg, keys, vals);
+    launch_dep(float_keys_kernel, dim3(nblk(n_neg)), dim3(256), 0, st, neg_scores, n_neg, keys, vals);
     const bool in_place = radix_sort_pairs(ctx->ex, keys, vals, n_neg, 32, sc);  // ascending
     cudaMemsetAsync(count, 0, sizeof(unsigned long long), st);
-    count_above_kernel<<<nblk(n_pos), 256, 0, st>>>(pos_scores, n_pos, in_place ? keys : sc.keys_alt, n_neg - K, count);
+    launch_dep(count_above_kernel, dim3(nblk(n_pos)), dim3(256), 0, st, pos_scores, n_pos, in_place ? keys : sc.keys_alt, n_neg - K, count);
     ctx->ex.launches += 2;
     unsigned long long h = 0;
     e = cudaMemcpyAsync(&h, count, sizeof h, cudaMemcpyDeviceToHost, st);
@@ -1790,7 +1794,7 @@ extern "C" lp_status lp_hits_at_k(lp_ctx *ctx, const float *pos_scores, int64_t 
 template <typename T> static void to_f32(lp_ctx *ctx, const T *src, int64_t lds, float *dst, int64_t rows, int F)
 {
     if (rows <= 0) return;
-    copy_rows_kernel<T, float><<<nblk(rows * F), 256, 0, ctx->ex.st>>>(src, lds, dst, F, rows, F);
+    launch_dep(copy_rows_kernel<T, float>, dim3(nblk(rows * F)), dim3(256), 0, ctx->ex.st, src, lds, dst, F, rows, F);
     ctx->ex.launches += 1;
 }
 
@@ -1852,7 +1856,7 @@ extern "C" lp_status lp_get_block(lp_ctx *ctx, int32_t hop, int32_t *frontier, i
         if (hb.n_src > 0) CK(cudaMemcpyAsync(frontier, hb.frontier, sizeof(int) * (size_t)hb.n_src, cudaMemcpyDeviceToDevice, st));
     }
     if (hop >= 1) {
-        if (blk_ptr) widen_i32_kernel<<<nblk(hb.n_dst + 1), 256, 0, st>>>(hb.blk_ptr, hb.n_dst + 1, blk_ptr);
+        if (blk_ptr) launch_dep(widen_i32_kernel, dim3(nblk(hb.n_dst + 1)), dim3(256), 0, st, hb.blk_ptr, hb.n_dst + 1, blk_ptr);
         if (blk_col && hb.entries > 0) CK(cudaMemcpyAsync(blk_col, hb.blk_col_global, sizeof(int) * (size_t)hb.entries, cudaMemcpyDeviceToDevice, st));
     }
     CK_LAUNCH();
@@ -2084,7 +2088,7 @@ extern "C" lp_status lp_weight_grad_static(int32_t device, void *cuda_stream, in
     if (k_chunk < SG_BK) k_chunk = SG_BK;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     dim3 grid((unsigned)ceil_div64(K, SG_BM), (unsigned)ceil_div64(N, SG_BN), (unsigned)splits);
-    gemm_simt_kernel<float, float, float, true, true><<<grid, SG_THREADS, 0, st>>>(K, N, M, A, K, dZ, N, (float *)nullptr, 0, nullptr, 0, k_chunk, scratch);
+    launch_dep(gemm_simt_kernel<float, float, float, true, true>, dim3(grid), dim3(SG_THREADS), 0, st, K, N, M, A, K, dZ, N, (float *)nullptr, 0, nullptr, 0, k_chunk, scratch, nullptr, 0);
     launch_dep(reduce_partials_kernel, dim3((unsigned)ceil_div64(tile, 256)), dim3(256), 0, st, scratch, tile, splits, dW, 0);
     CK_LAUNCH();
     return LP_OK;

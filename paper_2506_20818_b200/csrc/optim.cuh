@@ -24,12 +24,14 @@ __global__ void adam_kernel(float *__restrict__ p, float *__restrict__ m, float 
 
 __global__ void sgd_kernel(float *__restrict__ p, const float *__restrict__ grad, int64_t n, float scale, float lr)
 {
+    LP_DEP_ENTER();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) p[i] -= lr * scale * grad[i];
 }
 
 template <typename TS, typename TD> __global__ void convert_kernel(const TS *__restrict__ src, TD *__restrict__ dst, int64_t n)
 {
+    LP_DEP_ENTER();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) dst[i] = from_f<TD>(to_f<TS>(src[i]));
 }
@@ -38,6 +40,7 @@ template <typename TS, typename TD> __global__ void convert_kernel(const TS *__r
 template <typename TS, typename TD>
 __global__ void copy_rows_kernel(const TS *__restrict__ src, int64_t lds, TD *__restrict__ dst, int64_t ldd, int64_t rows, int F)
 {
+    LP_DEP_ENTER();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= rows * F) return;
     const int64_t r = i / F;
@@ -48,6 +51,7 @@ __global__ void copy_rows_kernel(const TS *__restrict__ src, int64_t lds, TD *__
 // W[K, N] row-major float -> Wt[N, K] row-major bf16 (K contiguous) and, optionally, W as bf16
 __global__ void weights_to_bf16_kernel(const float *__restrict__ W, int K, int N, bf16 *__restrict__ Wt, bf16 *__restrict__ Wc)
 {
+    LP_DEP_ENTER();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= K * N) return;
     const int k = i / N, n = i - k * N;

@@ -14,6 +14,7 @@ edge_hadamard_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, const i
                      const int *__restrict__ pos_dst, int64_t B, const int *__restrict__ neg_src, const int *__restrict__ neg_dst, int k,
                      T *__restrict__ Z0)
 {
+    LP_DEP_ENTER();
     constexpr int VN = Vec16<T>::N;
     const int lane = threadIdx.x & 31;
     const int64_t e = (int64_t)blockIdx.x * (EDGE_THREADS / 32) + (threadIdx.x >> 5);
@@ -44,6 +45,7 @@ template <typename T>
 __global__ void __launch_bounds__(EDGE_THREADS)
 edge_gemv_kernel(const T *__restrict__ P, int Hp, int64_t E, const float *__restrict__ w, const float *__restrict__ b, float *__restrict__ s)
 {
+    LP_DEP_ENTER();
     const int lane = threadIdx.x & 31;
     const int64_t e = (int64_t)blockIdx.x * (EDGE_THREADS / 32) + (threadIdx.x >> 5);
     if (e >= E) return;
@@ -57,6 +59,7 @@ edge_gemv_kernel(const T *__restrict__ P, int Hp, int64_t E, const float *__rest
 __global__ void __launch_bounds__(256)
 bce_from_scores_kernel(const float *__restrict__ s, int64_t E, int64_t B, float inv_N, float *__restrict__ g, float *__restrict__ loss_partials)
 {
+    LP_DEP_ENTER();
     __shared__ float sh[8];
     const int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x;
     float ell = 0.f;
@@ -81,6 +84,7 @@ template <typename T>
 __global__ void pred_out_grad_kernel(const T *__restrict__ P2, int Hp, int64_t E, const float *__restrict__ g, const float *__restrict__ w2,
                                      T *__restrict__ dP2)
 {
+    LP_DEP_ENTER();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= E * Hp) return;
     const int64_t e = i / Hp;
@@ -94,6 +98,7 @@ __global__ void __launch_bounds__(256)
 pred_last_layer_grad_kernel(const T *__restrict__ P2, int Hp, int64_t E, const float *__restrict__ g, int64_t rows_per_block,
                             float *__restrict__ partials)
 {
+    LP_DEP_ENTER();
     const int64_t r0 = (int64_t)blockIdx.x * rows_per_block, r1 = min(E, r0 + rows_per_block);
     for (int j = threadIdx.x; j <= Hp; j += 256) {
         float acc = 0.f;
@@ -109,6 +114,7 @@ pred_last_layer_grad_kernel(const T *__restrict__ P2, int Hp, int64_t E, const f
 template <typename T>
 __global__ void relu_mask_kernel(T *__restrict__ x, const T *__restrict__ ref, int64_t count)
 {
+    LP_DEP_ENTER();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < count && !(to_f<T>(ref[i]) > 0.f)) x[i] = from_f<T>(0.f);
 }
@@ -123,6 +129,7 @@ LP_DEVINL uint32_t float_sort_key(float f)
 
 __global__ void float_keys_kernel(const float *__restrict__ x, int64_t n, uint32_t *__restrict__ keys, uint32_t *__restrict__ vals)
 {
+    LP_DEP_ENTER();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) { keys[i] = float_sort_key(x[i]); vals[i] = (uint32_t)i; }
 }
@@ -131,6 +138,7 @@ __global__ void float_keys_kernel(const float *__restrict__ x, int64_t n, uint32
 __global__ void count_above_kernel(const float *__restrict__ pos, int64_t n_pos, const uint32_t *__restrict__ sorted_keys, int64_t thr_index,
                                    unsigned long long *__restrict__ count)
 {
+    LP_DEP_ENTER();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t thr = sorted_keys[thr_index];
     const bool hit = i < n_pos && float_sort_key(pos[i]) > thr;

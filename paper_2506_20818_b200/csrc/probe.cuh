@@ -14,6 +14,7 @@ template <int LANES>
 __global__ void __launch_bounds__(256) gather_probe_kernel(const int *__restrict__ col, int64_t nnz, const uint4 *__restrict__ X, int64_t pitch16,
                                                            uint4 *__restrict__ out)
 {
+    LP_DEP_ENTER();
     const int64_t gid = ((int64_t)blockIdx.x * 256 + threadIdx.x) / LANES;
     const int gl = threadIdx.x % LANES;
     const int64_t e0 = gid * PROBE_RUN;
@@ -45,9 +46,9 @@ static bool gather_probe_launch(Exec &ex, const int *col, int64_t nnz, const voi
     const int lanes = row_bytes / 16;
     const int64_t groups = ceil_div64(nnz, PROBE_RUN);
     const unsigned blocks = (unsigned)ceil_div64(groups * lanes, 256);
-    if (lanes == 32) gather_probe_kernel<32><<<blocks, 256, 0, ex.st>>>(col, nnz, (const uint4 *)X, lanes, (uint4 *)out);
-    else if (lanes == 16) gather_probe_kernel<16><<<blocks, 256, 0, ex.st>>>(col, nnz, (const uint4 *)X, lanes, (uint4 *)out);
-    else if (lanes == 8) gather_probe_kernel<8><<<blocks, 256, 0, ex.st>>>(col, nnz, (const uint4 *)X, lanes, (uint4 *)out);
+    if (lanes == 32) launch_dep(gather_probe_kernel<32>, dim3(blocks), dim3(256), 0, ex.st, col, nnz, (const uint4 *)X, lanes, (uint4 *)out);
+    else if (lanes == 16) launch_dep(gather_probe_kernel<16>, dim3(blocks), dim3(256), 0, ex.st, col, nnz, (const uint4 *)X, lanes, (uint4 *)out);
+    else if (lanes == 8) launch_dep(gather_probe_kernel<8>, dim3(blocks), dim3(256), 0, ex.st, col, nnz, (const uint4 *)X, lanes, (uint4 *)out);
     else return false;
     ex.launches += 1;
     return true;

@@ -79,6 +79,7 @@ constexpr int MAX_FANOUT = 32;
 __global__ void nbr_count_kernel(const int *__restrict__ rowptr, const int *__restrict__ frontier, const int *__restrict__ n_front_dev,
                                  int fanout, int *__restrict__ counts, int max_front)
 {
+    LP_DEP_ENTER();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= max_front) return;
     const int nf = *n_front_dev;
@@ -99,6 +100,7 @@ __global__ void nbr_sample_kernel(const int *__restrict__ rowptr, const int *__r
                                   const int *__restrict__ blk_ptr, int *__restrict__ blk_col_global, int *__restrict__ blk_row,
                                   unsigned char *__restrict__ mark, int *__restrict__ blk_eid)
 {
+    LP_DEP_ENTER();
     const unsigned lane = threadIdx.x & 31;
     const int gl = threadIdx.x % G;  // lane inside the group
     const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << (lane & ~(unsigned)(G - 1)));
@@ -148,6 +150,7 @@ __global__ void gcn_block_coef_kernel(const int *__restrict__ rowptr, const int 
                                       const int *__restrict__ blk_row, const int *__restrict__ blk_eid, const int *__restrict__ n_entries_dev,
                                       const float *__restrict__ gcn_val, float *__restrict__ blk_val)
 {
+    LP_DEP_ENTER();
     const int e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= *n_entries_dev) return;
     const int i = blk_row[e];
@@ -160,18 +163,21 @@ __global__ void gcn_block_coef_kernel(const int *__restrict__ rowptr, const int 
 __global__ void gather_by_id_kernel(const float *__restrict__ table, const int *__restrict__ ids, const int *__restrict__ count_dev, int cap,
                                     float *__restrict__ out)
 {
+    LP_DEP_ENTER();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < min(*count_dev, cap)) out[i] = table[ids[i]];
 }
 
 __global__ void mark_ids_kernel(const int *__restrict__ ids, int64_t m, int n, unsigned char *__restrict__ mark)
 {
+    LP_DEP_ENTER();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < m) mark[min(max(ids[i], 0), n - 1)] = 1;
 }
 
 __global__ void mark_to_int_kernel(const unsigned char *__restrict__ mark, int n, int *__restrict__ flags)
 {
+    LP_DEP_ENTER();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) flags[i] = mark[i] ? 1 : 0;
 }
@@ -179,6 +185,7 @@ __global__ void mark_to_int_kernel(const unsigned char *__restrict__ mark, int n
 // frontier[posmap[v]] = v for marked v (posmap = exclusive scan of the marks): sorted and unique
 __global__ void compact_frontier_kernel(const unsigned char *__restrict__ mark, const int *__restrict__ posmap, int n, int *__restrict__ frontier)
 {
+    LP_DEP_ENTER();
     const int v = blockIdx.x * blockDim.x + threadIdx.x;
     if (v < n && mark[v]) frontier[posmap[v]] = v;
 }
@@ -187,6 +194,7 @@ __global__ void compact_frontier_kernel(const unsigned char *__restrict__ mark, 
 __global__ void relabel_kernel(const int *__restrict__ ids_global, const int *__restrict__ count_dev, int64_t max_count,
                                const int *__restrict__ posmap, int *__restrict__ ids_local)
 {
+    LP_DEP_ENTER();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < max_count && i < (int64_t)*count_dev) ids_local[i] = posmap[ids_global[i]];
 }
@@ -196,6 +204,7 @@ __global__ void relabel_kernel(const int *__restrict__ ids_global, const int *__
 __global__ void self_index_kernel(const int *__restrict__ prev_frontier, const int *__restrict__ n_prev_dev, const int *__restrict__ posmap,
                                   int *__restrict__ self_idx, int *__restrict__ inv_self)
 {
+    LP_DEP_ENTER();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= *n_prev_dev) return;
     const int p = posmap[prev_frontier[i]];
@@ -205,6 +214,7 @@ __global__ void self_index_kernel(const int *__restrict__ prev_frontier, const i
 
 __global__ void fill_i32_kernel(int *__restrict__ p, int64_t m, int v)
 {
+    LP_DEP_ENTER();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < m) p[i] = v;
 }
@@ -212,6 +222,7 @@ __global__ void fill_i32_kernel(int *__restrict__ p, int64_t m, int v)
 // 1 / |sampled neighbours| per destination row, and the same value per transposed entry
 __global__ void inv_degree_kernel(const int *__restrict__ ptr, int n_rows, const int *__restrict__ n_rows_dev, float *__restrict__ inv)
 {
+    LP_DEP_ENTER();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     const int lim = n_rows_dev ? min(*n_rows_dev, n_rows) : n_rows;
     if (i >= lim) return;
@@ -221,6 +232,7 @@ __global__ void inv_degree_kernel(const int *__restrict__ ptr, int n_rows, const
 
 __global__ void gather_f32_kernel(const float *__restrict__ src, const int *__restrict__ idx, int64_t m, float *__restrict__ dst)
 {
+    LP_DEP_ENTER();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < m) dst[i] = src[idx[i]];
 }

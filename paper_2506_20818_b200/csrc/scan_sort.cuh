@@ -86,6 +86,7 @@ LP_DEVINL int block_exclusive_scan_256(int x, int *smem_warp /*>=8 ints*/, int *
 
 __global__ void __launch_bounds__(SCAN_THREADS) scan_tile_sums_kernel(const int *__restrict__ in, int64_t n, int *__restrict__ sums)
 {
+    LP_DEP_ENTER();
     __shared__ int sw[8];
     const int64_t base = (int64_t)blockIdx.x * SCAN_TILE;
     int acc = 0;
@@ -102,6 +103,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_tile_sums_kernel(const int 
 // one block scans `m` values in place (exclusive), writes the grand total to *total if non-null
 __global__ void __launch_bounds__(SCAN_THREADS) scan_single_block_kernel(int *__restrict__ data, int64_t m, int *__restrict__ total)
 {
+    LP_DEP_ENTER();
     __shared__ int sw[8];
     __shared__ int carry_s;
     if (threadIdx.x == 0) carry_s = 0;
@@ -132,6 +134,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_single_block_kernel(int *__
 __global__ void __launch_bounds__(SCAN_THREADS) scan_apply_kernel(const int *__restrict__ in, int64_t n, const int *__restrict__ tile_off,
                                                                   int *__restrict__ out, int *__restrict__ out_total)
 {
+    LP_DEP_ENTER();
     __shared__ int sw[8];
     const int64_t t0 = (int64_t)blockIdx.x * SCAN_TILE + (int64_t)threadIdx.x * SCAN_ITEMS;
     int v[SCAN_ITEMS];
@@ -165,9 +168,9 @@ static void exclusive_scan_i32(Exec &ex, const int *in, int64_t n, int *out, int
         return;
     }
     const int64_t tiles = ceil_div64(n, SCAN_TILE);
-    scan_tile_sums_kernel<<<(unsigned)tiles, SCAN_THREADS, 0, ex.st>>>(in, n, tmp);
-    scan_single_block_kernel<<<1, SCAN_THREADS, 0, ex.st>>>(tmp, tiles, nullptr);
-    scan_apply_kernel<<<(unsigned)tiles, SCAN_THREADS, 0, ex.st>>>(in, n, tmp, out, out_total);
+    launch_dep(scan_tile_sums_kernel, dim3((unsigned)tiles), dim3(SCAN_THREADS), 0, ex.st, in, n, tmp);
+    launch_dep(scan_single_block_kernel, dim3(1), dim3(SCAN_THREADS), 0, ex.st, tmp, tiles, nullptr);
+    launch_dep(scan_apply_kernel, dim3((unsigned)tiles), dim3(SCAN_THREADS), 0, ex.st, in, n, tmp, out, out_total);
     ex.launches += 3;
 }
 
@@ -312,6 +315,7 @@ constexpr int RS_RADIX = 256;
 __global__ void __launch_bounds__(RS_THREADS) rs_hist_kernel(const uint32_t *__restrict__ keys, int64_t n, int shift,
                                                              int *__restrict__ hist /*[RADIX][tiles]*/, int tiles)
 {
+    LP_DEP_ENTER();
     __shared__ int h[RS_RADIX];
     h[threadIdx.x] = 0;
     __syncthreads();
@@ -329,6 +333,7 @@ __global__ void __launch_bounds__(RS_THREADS) rs_scatter_kernel(const uint32_t *
                                                                 int64_t n, int shift, const int *__restrict__ hist_scanned, int tiles,
                                                                 uint32_t *__restrict__ keys_out, uint32_t *__restrict__ vals_out)
 {
+    LP_DEP_ENTER();
     __shared__ int base[RS_RADIX];                    // next free output slot per digit for this tile
     __shared__ int wcount[RS_THREADS / 32][RS_RADIX]; // per-warp digit counts of the current round
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -383,10 +388,10 @@ static bool radix_sort_pairs(Exec &ex, uint32_t *keys, uint32_t *vals, int64_t n
     const int tiles = (int)ceil_div64(n, RS_TILE);
     uint32_t *ki = keys, *vi = vals, *ko = s.keys_alt, *vo = s.vals_alt;
     for (int p = 0; p < passes; ++p) {
-        rs_hist_kernel<<<tiles, RS_THREADS, 0, ex.st>>>(ki, n, 8 * p, s.hist, tiles);
+        launch_dep(rs_hist_kernel, dim3(tiles), dim3(RS_THREADS), 0, ex.st, ki, n, 8 * p, s.hist, tiles);
         ex.launches += 1;
         exclusive_scan_i32(ex, s.hist, (int64_t)RS_RADIX * tiles, s.hist, nullptr, s.scan_tmp);
-        rs_scatter_kernel<<<tiles, RS_THREADS, 0, ex.st>>>(ki, vi, n, 8 * p, s.hist, tiles, ko, vo);
+        launch_dep(rs_scatter_kernel, dim3(tiles), dim3(RS_THREADS), 0, ex.st, ki, vi, n, 8 * p, s.hist, tiles, ko, vo);
         ex.launches += 1;
         uint32_t *t;
         t = ki; ki = ko; ko = t;
@@ -403,6 +408,7 @@ static bool radix_sort_pairs(Exec &ex, uint32_t *keys, uint32_t *vals, int64_t n
 __global__ void expand_entries_kernel(const int *__restrict__ rowptr, int n_rows, const int *__restrict__ col, int64_t nnz,
                                       uint32_t *__restrict__ keys, uint32_t *__restrict__ vals, int *__restrict__ rows)
 {
+    LP_DEP_ENTER();
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= nnz) return;
     int lo = 0, hi = n_rows;  // largest r with rowptr[r] <= e
@@ -419,6 +425,7 @@ __global__ void expand_entries_kernel(const int *__restrict__ rowptr, int n_rows
 __global__ void expand_known_rows_kernel(const int *__restrict__ col, int64_t nnz, uint32_t *__restrict__ keys, uint32_t *__restrict__ vals,
                                          int *__restrict__ counts)
 {
+    LP_DEP_ENTER();
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= nnz) return;
     const int c = col[e];
@@ -429,6 +436,7 @@ __global__ void expand_known_rows_kernel(const int *__restrict__ col, int64_t nn
 
 __global__ void count_keys_kernel(const int *__restrict__ ids, int64_t m, int *__restrict__ counts)
 {
+    LP_DEP_ENTER();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < m) atomicAdd(&counts[ids[i]], 1);
 }
@@ -436,6 +444,7 @@ __global__ void count_keys_kernel(const int *__restrict__ ids, int64_t m, int *_
 __global__ void gather_rows_kernel(const uint32_t *__restrict__ sorted_vals, const int *__restrict__ rows, int64_t nnz,
                                    int *__restrict__ rowidx_t, int *__restrict__ perm)
 {
+    LP_DEP_ENTER();
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= nnz) return;
     const uint32_t e = sorted_vals[t];
@@ -467,18 +476,18 @@ static void transpose_csr(Exec &ex, const int *rowptr, int n_rows, int n_cols, c
     if (nnz > 0) {
         const unsigned blocks = (unsigned)ceil_div64(nnz, 256);
         if (rows_known) {  // the caller has the row of every entry (sampled blocks record it)
-            expand_known_rows_kernel<<<blocks, 256, 0, ex.st>>>(col, nnz, s.keys, s.vals, colptr);
+            launch_dep(expand_known_rows_kernel, dim3(blocks), dim3(256), 0, ex.st, col, nnz, s.keys, s.vals, colptr);
             ex.launches += 1;
         } else {
-            expand_entries_kernel<<<blocks, 256, 0, ex.st>>>(rowptr, n_rows, col, nnz, s.keys, s.vals, s.rows);
-            count_keys_kernel<<<blocks, 256, 0, ex.st>>>(col, nnz, colptr);
+            launch_dep(expand_entries_kernel, dim3(blocks), dim3(256), 0, ex.st, rowptr, n_rows, col, nnz, s.keys, s.vals, s.rows);
+            launch_dep(count_keys_kernel, dim3(blocks), dim3(256), 0, ex.st, col, nnz, colptr);
             ex.launches += 2;
         }
     }
     exclusive_scan_i32(ex, colptr, n_cols, colptr, colptr + n_cols, s.scan_tmp);
     if (nnz > 0) {
         const bool in_place = radix_sort_pairs(ex, s.keys, s.vals, nnz, bits_for(n_cols), s.sort);
-        gather_rows_kernel<<<(unsigned)ceil_div64(nnz, 256), 256, 0, ex.st>>>(in_place ? s.vals : s.sort.vals_alt, rows_known ? rows_known : s.rows, nnz, rowidx_t, perm);
+        launch_dep(gather_rows_kernel, dim3((unsigned)ceil_div64(nnz, 256)), dim3(256), 0, ex.st, in_place ? s.vals : s.sort.vals_alt, rows_known ? rows_known : s.rows, nnz, rowidx_t, perm);
         ex.launches += 1;
     }
 }

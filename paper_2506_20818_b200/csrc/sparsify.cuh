@@ -12,12 +12,14 @@
 
 __global__ void sp_nonisolated_kernel(const int *__restrict__ rowptr, int n, int *__restrict__ flags)
 {
+    LP_DEP_ENTER();
     const int v = blockIdx.x * blockDim.x + threadIdx.x;
     if (v < n) flags[v] = rowptr[v + 1] > rowptr[v] ? 1 : 0;
 }
 
 __global__ void sp_compact_kernel(const int *__restrict__ rowptr, const int *__restrict__ pos, int n, int *__restrict__ nz)
 {
+    LP_DEP_ENTER();
     const int v = blockIdx.x * blockDim.x + threadIdx.x;
     if (v < n && rowptr[v + 1] > rowptr[v]) nz[pos[v]] = v;
 }
@@ -26,6 +28,7 @@ __global__ void sp_compact_kernel(const int *__restrict__ rowptr, const int *__r
 __global__ void sp_draw_kernel(const int *__restrict__ rowptr, const int *__restrict__ col, const int *__restrict__ nz, uint32_t n_nz, uint2 key,
                                int64_t L, int *__restrict__ hits, int *__restrict__ err)
 {
+    LP_DEP_ENTER();
     const int64_t l = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (l >= L) return;
     const uint4 r = philox4x32_10(make_uint4((uint32_t)l, (uint32_t)((uint64_t)l >> 32), 0u, DRAW_SPARSIFY), key);
@@ -46,6 +49,7 @@ __global__ void sp_draw_kernel(const int *__restrict__ rowptr, const int *__rest
 
 __global__ void sp_keep_flags_kernel(const int *__restrict__ hits, int64_t nnz, int *__restrict__ flags)
 {
+    LP_DEP_ENTER();
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e < nnz) flags[e] = hits[e] > 0 ? 1 : 0;
 }
@@ -54,6 +58,7 @@ __global__ void sp_keep_flags_kernel(const int *__restrict__ hits, int64_t nnz, 
 __global__ void sp_emit_kernel(const int *__restrict__ rowptr, const int *__restrict__ col, const int *__restrict__ hits, const int *__restrict__ pos,
                                int n, double n_nz, double L, int64_t *__restrict__ out_ptr, int *__restrict__ out_col, float *__restrict__ out_w)
 {
+    LP_DEP_ENTER();
     const int v = blockIdx.x * blockDim.x + threadIdx.x;
     if (v > n) return;
     if (v == n) { out_ptr[n] = pos[rowptr[n]]; return; }

@@ -559,6 +559,7 @@ LP_DEVINL int padded_row_groups(int d, int threshold)
 }
 __global__ void padded_count_kernel(const int *__restrict__ rowptr, int n, int threshold, int *__restrict__ ngroups)
 {
+    LP_DEP_ENTER();
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= n) return;
     ngroups[r] = padded_row_groups(rowptr[r + 1] - rowptr[r], threshold);
@@ -567,6 +568,7 @@ __global__ void padded_count_kernel(const int *__restrict__ rowptr, int n, int t
 // first row, follows a heavy row, or when first_group crosses a multiple of SPMM_CHUNK_GROUPS between rows r - 1 and r
 __global__ void padded_chunk_count_kernel(const int *__restrict__ rowptr, const int *__restrict__ first_group, int n, int threshold, int *__restrict__ count)
 {
+    LP_DEP_ENTER();
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= n) return;
     const int d = rowptr[r + 1] - rowptr[r];
@@ -583,6 +585,7 @@ __global__ void padded_fill_kernel(const int *__restrict__ rowptr, const int *__
                                    const int *__restrict__ row_base, int *__restrict__ chunk_start, int *__restrict__ pcol, float *__restrict__ pval,
                                    int *__restrict__ grow)
 {
+    LP_DEP_ENTER();
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= n) return;
     if (r == n - 1) chunk_start[chunk_of[n]] = first_group[n];  // chunk_of[n] = number of chunks, first_group[n] = all groups

@@ -13,6 +13,7 @@ __global__ void view_count_kernel(int n, const int *__restrict__ rowptr, const i
                                   int keep_cross, int foreign_mode, const int64_t *__restrict__ sp_ptr, int *__restrict__ counts,
                                   unsigned long long *__restrict__ stats)
 {
+    LP_DEP_ENTER();
     const int v = blockIdx.x * blockDim.x + threadIdx.x;
     if (v >= n) return;
     int c = 0;
@@ -38,6 +39,7 @@ __global__ void view_fill_kernel(int n, const int *__restrict__ rowptr, const in
                                  int keep_cross, int foreign_mode, const int64_t *__restrict__ sp_ptr, const int *__restrict__ sp_col,
                                  const int *__restrict__ view_ptr, int *__restrict__ view_col)
 {
+    LP_DEP_ENTER();
     const int v = blockIdx.x * blockDim.x + threadIdx.x;
     if (v >= n) return;
     int o = view_ptr[v];
