@@ -800,6 +800,43 @@ def test_step_on_a_caller_stream_matches_default_stream(pkg):
     assert torch.equal(results[0][0], results[1][0]) and torch.equal(results[0][1], results[1][1])
 
 
+def test_profiler_times_every_nth_step_and_leaves_results_alone(pkg):
+    # per-category event timing: every step, then every 4th step of 8 (2 steps x 3 aggregation launches of a 2-layer SAGE
+    # model: two forward, one adjoint), and the timed steps give the same bits as untimed ones
+    g, X, params, pos, cfg = wl.make_config("c2_chunglu_sage2", scale=0.02)
+    u, v = pos[0][:2000].copy(), pos[1][:2000].copy()
+    ctx = make_ctx(pkg, g, X)
+    ctx.set_model("sage", cfg["dims"], prec="bf16", max_batch=len(u), max_k=1)
+    du, dv, p = t32(u), t32(v), t32(params)
+    _, nd = ctx.sample_negatives(3, 1, 1, du)
+    loss, grads = torch.zeros(1, device=DEV), torch.zeros(ctx.n_params, device=DEV)
+
+    def steps(n):
+        out = []
+        for _ in range(n):
+            ctx.train_step(p, du, dv, None, nd, 1, loss, grads)
+            out.append((loss.clone(), grads.clone()))
+        return out
+
+    plain = steps(1)[0]
+    ctx.profile_begin(["agg_fwd", "agg_bwd", "score"])
+    timed = steps(8)
+    prof = ctx.profile_end()
+    assert prof["agg_fwd"]["spans"] == 16 and prof["agg_bwd"]["spans"] == 8 and prof["score"]["spans"] == 8
+    assert prof["agg_fwd"]["ms"] > 0 and prof["agg_fwd"]["bytes"] > 0 and prof["gemm_fwd"]["spans"] == 0
+    ctx.profile_sample_every(4)
+    ctx.profile_begin(["agg_fwd", "agg_bwd"])
+    timed += steps(8)
+    prof = ctx.profile_end()
+    assert prof["agg_fwd"]["spans"] == 4 and prof["agg_bwd"]["spans"] == 2
+    ctx.profile_sample_every(1)
+    with pytest.raises(pkg.LpError):
+        ctx.profile_sample_every(0)
+    for l, gr in timed:
+        assert torch.equal(l, plain[0]) and torch.equal(gr, plain[1])
+    ctx.close()
+
+
 @pytest.mark.parametrize("arch", ["gcn", "sage"])
 def test_cached_input_aggregation_gives_identical_steps(pkg, arch):
     g, X, params, pos, cfg = wl.make_config("c3_coauthor_gcn3", scale=0.02)
