@@ -896,7 +896,9 @@ def test_mlp_predictor_step(pkg, arch, prec, fanout):
         sel = np.random.default_rng(3).choice(g.nnz, 900, replace=False)
         u, v = g.col[sel].copy(), rows[sel].copy()
     else:
-        g = wl.chung_lu(6000, 14.0, 2.1, seed=5)
+        # (the BF16 case is large enough for the transforms to run on pairs of SMs, so the top layer takes its input gradient
+        # as aggregate-then-transform behind the two-operand gradient gather)
+        g = wl.chung_lu(9001 if prec == "bf16" else 6000, 14.0, 2.1, seed=5)
         pu, pv = wl.undirected_edge_list(g)
         sel = np.random.default_rng(3).choice(len(pu), 2500, replace=False)
         u, v = pu[sel].copy(), pv[sel].copy()
