@@ -20,10 +20,13 @@ __global__ void check_ids_kernel(const int *__restrict__ ids, int64_t m, int n_i
 
 // the same for the up to four id arrays of a step in one launch (null arrays are skipped)
 __global__ void check_step_ids_kernel(const int *__restrict__ a, int64_t na, const int *__restrict__ b, int64_t nb, const int *__restrict__ c, int64_t nc,
-                                      const int *__restrict__ d, int64_t nd, int n_ids, int *__restrict__ err, int *__restrict__ zero, int64_t n_zero)
+                                      const int *__restrict__ d, int64_t nd, int n_ids, int *__restrict__ err, int *__restrict__ zero, int64_t n_zero,
+                                      int *__restrict__ plan_counts)
 {
     LP_DEP_ENTER();
-    // first kernel of a step: it also clears the incidence-list counters the scoring kernel adds into
+    // first kernel of a step: it also clears the incidence-list counters the scoring kernel adds into and the two counters of
+    // the heavy-row plan of those lists
+    if (blockIdx.x == 0 && threadIdx.x < 2 && plan_counts) plan_counts[threadIdx.x] = 0;
     for (int64_t z = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; z < n_zero; z += (int64_t)gridDim.x * blockDim.x) zero[z] = 0;
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int *p = a;
@@ -260,21 +263,25 @@ edge_score_bce_pair_kernel(const T *__restrict__ H, int ldh, int D, int n_ids, c
     }
 }
 
-// loss = inv_N * sum of partials: one block of 1024 threads, thread t adds partials t, t + 1024, ... in double
+// loss = inv_N * sum of partials by one block of THREADS threads: thread t adds partials t, t + THREADS, ... in double
 // (tens of thousands of nearly equal terms), then a fixed binary tree over the threads
-__global__ void __launch_bounds__(1024) loss_reduce_kernel(const float *__restrict__ partials, int64_t m, float inv_N, float *__restrict__ loss)
+template <int THREADS> LP_DEVINL void loss_reduce_block(const float *__restrict__ partials, int64_t m, float inv_N, float *__restrict__ loss)
 {
-    LP_DEP_ENTER();
-    __shared__ double sh[1024];
+    __shared__ double sh[THREADS];
     double s = 0.0;
-    for (int64_t i = threadIdx.x; i < m; i += 1024) s += (double)partials[i];
+    for (int64_t i = threadIdx.x; i < m; i += THREADS) s += (double)partials[i];
     sh[threadIdx.x] = s;
     __syncthreads();
-    for (int w = 512; w > 0; w >>= 1) {
+    for (int w = THREADS / 2; w > 0; w >>= 1) {
         if ((int)threadIdx.x < w) sh[threadIdx.x] += sh[threadIdx.x + w];
         __syncthreads();
     }
     if (threadIdx.x == 0) *loss = (float)(sh[0] * (double)inv_N);
+}
+__global__ void __launch_bounds__(1024) loss_reduce_kernel(const float *__restrict__ partials, int64_t m, float inv_N, float *__restrict__ loss)
+{
+    LP_DEP_ENTER();
+    loss_reduce_block<1024>(partials, m, inv_N, loss);
 }
 
 // plain scores for lp_score: one warp per edge
@@ -352,12 +359,39 @@ LP_DEVINL int claim_slot(int *cursor, int node, unsigned active, int lane)
     return base + __popc(peers & ((1u << lane) - 1u));
 }
 
-__global__ void incidence_fill_kernel(int n_ids, const int *__restrict__ idmap, const int *__restrict__ pos_src, const int *__restrict__ pos_dst,
-                                      int64_t B, const int *__restrict__ neg_src, const int *__restrict__ neg_dst, int k,
-                                      const float *__restrict__ g_pos, const float *__restrict__ g_neg, int *__restrict__ cursor,
-                                      int *__restrict__ inc_col, float *__restrict__ inc_val, int *__restrict__ inc_edge, int *__restrict__ plan_counts)
+// Work that rides along with the list fill in blocks of its own, behind the fill_blocks blocks that fill: the heavy-row plan of
+// the lists (it needs only their offsets, which the scan before this launch produced; one thread per row) and the final
+// reduction of the loss partials (one block).  plan_rows = 0 / loss = null switch a rider off.
+struct FillRiders {
+    int fill_blocks = 0;
+    const int *plan_rowptr = nullptr;
+    int plan_rows = 0;
+    HeavyPlan plan;
+    const float *loss_partials = nullptr;
+    long long n_partials = 0;
+    float inv_N = 0.f;
+    float *loss = nullptr;
+};
+static inline unsigned fill_rider_blocks(const FillRiders &x) { return (unsigned)((x.plan_rows + 255) / 256 + (x.loss ? 1 : 0)); }
+
+__global__ void __launch_bounds__(256) incidence_fill_kernel(int n_ids, const int *__restrict__ idmap, const int *__restrict__ pos_src,
+                                                             const int *__restrict__ pos_dst, int64_t B, const int *__restrict__ neg_src,
+                                                             const int *__restrict__ neg_dst, int k, const float *__restrict__ g_pos,
+                                                             const float *__restrict__ g_neg, int *__restrict__ cursor, int *__restrict__ inc_col,
+                                                             float *__restrict__ inc_val, int *__restrict__ inc_edge, int *__restrict__ plan_counts,
+                                                             const FillRiders x)
 {
     LP_DEP_ENTER();
+    if (x.fill_blocks > 0 && (int)blockIdx.x >= x.fill_blocks) {
+        const int pb = (int)blockIdx.x - x.fill_blocks, plan_blocks = (x.plan_rows + 255) / 256;
+        if (pb < plan_blocks) {
+            const int r = pb * 256 + (int)threadIdx.x;
+            if (r < x.plan_rows) heavy_plan_row(x.plan_rowptr, r, x.plan, nullptr);
+        } else if (x.loss) {
+            loss_reduce_block<256>(x.loss_partials, x.n_partials, x.inv_N, x.loss);
+        }
+        return;
+    }
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e == 0 && plan_counts) { plan_counts[0] = 0; plan_counts[1] = 0; }  // the heavy-row plan of these lists is built by the next launch
     const bool valid = e < B * (1 + k);

@@ -1372,7 +1372,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     {
         const int64_t nk = k > 0 ? B * k : 0;
         launch_dep(check_step_ids_kernel, dim3(nblk(2 * B + 2 * nk)), dim3(256), 0, st, pos_src, B, pos_dst, B, neg_dst, nk, neg_src, (k > 0 && neg_src) ? nk : 0, ctx->n, ctx->err_flag,
-                   ctx->inc_ptr, ctx->inc_cap);
+                   ctx->inc_ptr, ctx->inc_cap, ctx->plan_dyn.counts);
         ctx->ex.launches += 1;
     }
     cache_weights(ctx, params);
@@ -1394,6 +1394,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     constexpr int VN = Vec16<T>::N;
     const int chunks = D / VN;
     const float *g_pos = ctx->g_pos, *g_neg = ctx->g_neg;
+    unsigned loss_parts = 0;
     // the dot-product scoring kernel also counts the incidence-list lengths (into the zeroed offsets array)
     // (the offsets array was cleared by the first kernel of the step)
     if (ctx->mlp) {
@@ -1413,17 +1414,32 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         } else if (chunks <= 32) launch_dep(edge_score_bce_kernel<T, 1>, dim3(eblocks), dim3(EDGE_THREADS), 0, st, HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials, ctx->inc_ptr);
         else if (chunks <= 64) launch_dep(edge_score_bce_kernel<T, 2>, dim3(eblocks), dim3(EDGE_THREADS), 0, st, HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials, ctx->inc_ptr);
         else launch_dep(edge_score_bce_kernel<T, 4>, dim3(eblocks), dim3(EDGE_THREADS), 0, st, HK, D, D, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, inv_N, ctx->g_pos, ctx->g_neg, nullptr, nullptr, ctx->loss_partials, ctx->inc_ptr);
-        launch_dep(loss_reduce_kernel, dim3(1), dim3(1024), 0, st, ctx->loss_partials, lparts, inv_N, loss);
+        loss_parts = lparts;  // reduced by a block that rides along with the list fill below
     }
     pscore.reset();
-    ctx->ex.launches += 2;
+    ctx->ex.launches += ctx->mlp ? 2 : 1;
 
     // incidence lists of the scored edges, grouped by node (slots claimed with integer atomics)
     std::unique_ptr<ProfScope> pinc(new ProfScope(ctx->ex, LP_PROF_INCIDENCE, (double)E * 2.0 * 24.0));
     if (ctx->mlp) launch_dep(incidence_count_kernel, dim3(nblk(E)), dim3(256), 0, st, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, ctx->inc_ptr);
     exclusive_scan_i32_copy(ctx->ex, ctx->inc_ptr, rows_out, ctx->inc_ptr, ctx->inc_cursor, ctx->inc_ptr + rows_out, ctx->scan_tmp);
-    launch_dep(incidence_fill_kernel, dim3(nblk(E)), dim3(256), 0, st, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, g_pos, g_neg, ctx->inc_cursor, ctx->inc_col,
-               ctx->mlp ? nullptr : ctx->inc_val, ctx->mlp ? ctx->inc_edge : nullptr, ctx->plan_dyn.counts);
+    {
+        // the same launch builds the heavy-row plan of the lists (their offsets are final after the scan; the plan's counters
+        // were cleared by the first kernel of the step) and, for the dot-product predictor, reduces the loss partials
+        FillRiders x;
+        x.fill_blocks = (int)nblk(E);
+        x.plan_rowptr = ctx->inc_ptr;
+        x.plan_rows = (int)rows_out;
+        x.plan = ctx->plan_dyn;
+        if (!ctx->mlp) {
+            x.loss_partials = ctx->loss_partials;
+            x.n_partials = loss_parts;
+            x.inv_N = inv_N;
+            x.loss = loss;
+        }
+        launch_dep(incidence_fill_kernel, dim3(nblk(E) + fill_rider_blocks(x)), dim3(256), 0, st, ctx->n, idmap, pos_src, pos_dst, B, neg_src, neg_dst, k, g_pos, g_neg,
+                   ctx->inc_cursor, ctx->inc_col, ctx->mlp ? nullptr : ctx->inc_val, ctx->mlp ? ctx->inc_edge : nullptr, nullptr, x);
+    }
     ctx->ex.launches += 2;
     pinc.reset();
 
@@ -1439,7 +1455,7 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
         SpmmArgs<T> a;
         a.heavy = ctx->plan_dyn;
         a.heavy.partials = ctx->inc_partials;
-        a.heavy.counts_zeroed = true;  // by the kernel that filled the lists
+        a.heavy.plan_prebuilt = true;  // by the launch that filled the lists
 
         a.nnz = 2 * E;
         a.n_rows = rows_out;

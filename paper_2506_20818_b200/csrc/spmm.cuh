@@ -35,6 +35,7 @@ struct HeavyPlan {
     float *partials = nullptr;
     int host_rows = -1, host_items = -1;  // -1: unknown on the host (plan built on the device per launch)
     bool counts_zeroed = false;           // per-launch plans: the caller's previous kernel has already cleared `counts`
+    bool plan_prebuilt = false;           // per-launch plans: an earlier kernel of the caller has already run heavy_plan_row over the rows
     int threshold = 32;                   // rows with more entries than this are heavy (>= SPMM_HEAVY_MIN)
     int seg = 512;                        // entries per item (SPMM_SEG; SPMM_PIECE for the padded form's own plan)
     // Static structures only: every row again in padded form for spmm_padded_kernel.  A row is cut into pieces of at
@@ -611,15 +612,10 @@ __global__ void padded_fill_kernel(const int *__restrict__ rowptr, const int *__
     }
 }
 
-// one thread per row: heavy rows claim a slot and a run of items
+// one row of a heavy-row plan: a row above the threshold claims a slot and a run of items
 // (row_base, optional: first item of every heavy row, -1 for the others)
-__global__ void spmm_heavy_plan_kernel(const int *__restrict__ rowptr, int n_rows, const int *__restrict__ n_rows_dev, HeavyPlan hp,
-                                       int *__restrict__ row_base = nullptr)
+LP_DEVINL void heavy_plan_row(const int *__restrict__ rowptr, int r, const HeavyPlan &hp, int *__restrict__ row_base)
 {
-    LP_DEP_ENTER();
-    const int r = blockIdx.x * blockDim.x + threadIdx.x;
-    const int lim = n_rows_dev ? min(*n_rows_dev, n_rows) : n_rows;
-    if (r >= lim) return;
     const int d = rowptr[r + 1] - rowptr[r];
     if (d <= hp.threshold) {
         if (row_base) row_base[r] = -1;
@@ -636,6 +632,16 @@ __global__ void spmm_heavy_plan_kernel(const int *__restrict__ rowptr, int n_row
         hp.item_row[b + s] = r;
         hp.item_first[b + s] = b;
     }
+}
+// one thread per row
+__global__ void spmm_heavy_plan_kernel(const int *__restrict__ rowptr, int n_rows, const int *__restrict__ n_rows_dev, HeavyPlan hp,
+                                       int *__restrict__ row_base = nullptr)
+{
+    LP_DEP_ENTER();
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    const int lim = n_rows_dev ? min(*n_rows_dev, n_rows) : n_rows;
+    if (r >= lim) return;
+    heavy_plan_row(rowptr, r, hp, row_base);
 }
 
 // adds the items of every heavy row in item order (fixed) and applies the epilogue; one lane group per row
@@ -736,10 +742,12 @@ template <typename T, int G, int NV, int RPG, int U, int MINB, typename ACC> sta
     }
     int64_t items = a.heavy.host_items;
     if (items < 0) {  // plan unknown on the host: rebuild it on the device, size the grid by the upper bound
-        if (!a.heavy.counts_zeroed) cudaMemsetAsync(a.heavy.counts, 0, 2 * sizeof(int), ex.st);
-        launch_dep(spmm_heavy_plan_kernel, dim3((unsigned)ceil_div64(a.n_rows, 256)), dim3(256), 0, ex.st, a.rowptr, a.n_rows, a.n_rows_dev, a.heavy, nullptr);
+        if (!a.heavy.plan_prebuilt) {
+            if (!a.heavy.counts_zeroed) cudaMemsetAsync(a.heavy.counts, 0, 2 * sizeof(int), ex.st);
+            launch_dep(spmm_heavy_plan_kernel, dim3((unsigned)ceil_div64(a.n_rows, 256)), dim3(256), 0, ex.st, a.rowptr, a.n_rows, a.n_rows_dev, a.heavy, nullptr);
+            ex.launches += 1;
+        }
         items = a.nnz / SPMM_HEAVY_MIN;  // a heavy row has more than SPMM_HEAVY_MIN entries and at most deg / SPMM_HEAVY_MIN items
-        ex.launches += 1;
     }
     const int item_blocks = (int)std::min<int64_t>(items, SPMM_ITEM_BLOCKS);
     const unsigned grid = (unsigned)(light_blocks + item_blocks);
