@@ -3,6 +3,7 @@
 // the gradient with respect to H^(K) be gathered row by row (no float atomics).
 #pragma once
 #include "common.cuh"
+#include "optim.cuh"
 #include "scan_sort.cuh"
 
 constexpr int EDGE_THREADS = 256;
@@ -19,15 +20,21 @@ __global__ void check_ids_kernel(const int *__restrict__ ids, int64_t m, int n_i
 }
 
 // the same for the up to four id arrays of a step in one launch (null arrays are skipped)
+// First kernel of a step.  Blocks below id_blocks check the step's node ids and clear the incidence-list counters the scoring
+// kernel adds into and the two counters of the heavy-row plan of those lists; the blocks behind them (BF16 path) make the
+// BF16 copies of the parameter vector that the transforms read (weights_cache_element).
 __global__ void check_step_ids_kernel(const int *__restrict__ a, int64_t na, const int *__restrict__ b, int64_t nb, const int *__restrict__ c, int64_t nc,
                                       const int *__restrict__ d, int64_t nd, int n_ids, int *__restrict__ err, int *__restrict__ zero, int64_t n_zero,
-                                      int *__restrict__ plan_counts)
+                                      int *__restrict__ plan_counts, int id_blocks, const float *__restrict__ w_params, long long w_n, WeightBlocks w_blocks,
+                                      bf16 *__restrict__ w_asis, bf16 *__restrict__ w_transposed, bf16 *__restrict__ w_stacked)
 {
     LP_DEP_ENTER();
-    // first kernel of a step: it also clears the incidence-list counters the scoring kernel adds into and the two counters of
-    // the heavy-row plan of those lists
+    if ((int)blockIdx.x >= id_blocks) {
+        weights_cache_element((long long)(blockIdx.x - id_blocks) * blockDim.x + threadIdx.x, w_params, w_n, w_blocks, w_asis, w_transposed, w_stacked);
+        return;
+    }
     if (blockIdx.x == 0 && threadIdx.x < 2 && plan_counts) plan_counts[threadIdx.x] = 0;
-    for (int64_t z = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; z < n_zero; z += (int64_t)gridDim.x * blockDim.x) zero[z] = 0;
+    for (int64_t z = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; z < n_zero; z += (int64_t)id_blocks * blockDim.x) zero[z] = 0;
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int *p = a;
     if (i >= na) { i -= na; p = b; if (i >= nb) { i -= nb; p = c; if (i >= nc) { i -= nc; p = d; if (i >= nd) return; } } }

@@ -1025,10 +1025,9 @@ extern "C" lp_status lp_sample_negatives(lp_ctx *ctx, uint64_t seed, uint64_t st
 // ----------------------------------------------------------------------------------------------
 template <typename T> static T *tptr(void *p) { return (T *)p; }
 
-// BF16 path: one launch turns the call's parameter vector into the two BF16 copies the transforms read
-static void cache_weights(lp_ctx *ctx, const float *params)
+// BF16 path: the weight matrices of the flat parameter vector, as the kernels that make its BF16 copies need them
+static WeightBlocks weight_blocks(const lp_ctx *ctx)
 {
-    if (ctx->desc.prec != LP_BF16 || !ctx->w16) return;
     WeightBlocks wb{};
     for (int k = 0; k < ctx->K; ++k) {
         wb.off[wb.count] = ctx->layer[k].off_w; wb.kin[wb.count] = ctx->layer[k].Kin; wb.fo[wb.count] = ctx->layer[k].Fo;
@@ -1037,7 +1036,13 @@ static void cache_weights(lp_ctx *ctx, const float *params)
     }
     if (ctx->mlp)
         for (int j = 0; j < 2; ++j) { wb.off[wb.count] = ctx->pred[j].off_w; wb.kin[wb.count] = ctx->pred[j].Kin; wb.fo[wb.count] = ctx->pred[j].Fo; ++wb.count; }
-    launch_dep(weights_cache_kernel, dim3(nblk(ctx->n_params)), dim3(256), 0, ctx->ex.st, params, ctx->n_params, wb, ctx->w16, ctx->w16t, ctx->w16s);
+    return wb;
+}
+// one launch turns the call's parameter vector into the BF16 copies the transforms read (lp_score; a training step does it in its first kernel)
+static void cache_weights(lp_ctx *ctx, const float *params)
+{
+    if (ctx->desc.prec != LP_BF16 || !ctx->w16) return;
+    launch_dep(weights_cache_kernel, dim3(nblk(ctx->n_params)), dim3(256), 0, ctx->ex.st, params, ctx->n_params, weight_blocks(ctx), ctx->w16, ctx->w16t, ctx->w16s);
     ctx->ex.launches += 1;
 }
 
@@ -1368,14 +1373,17 @@ static lp_status train_impl(lp_ctx *ctx, const float *params, const int *pos_src
     const bool sage = ctx->desc.arch == LP_SAGE_MEAN;
     const int D = ctx->desc.dims[K];
     ctx->ex.prof.tick += 1;  // lp_profile_sample_every counts training steps
-    // bad ids are clamped by every consumer and reported through the context's error word
+    // bad ids are clamped by every consumer and reported through the context's error word; the same launch clears the step's
+    // counters and (BF16 path) makes the BF16 copies of the weights
     {
         const int64_t nk = k > 0 ? B * k : 0;
-        launch_dep(check_step_ids_kernel, dim3(nblk(2 * B + 2 * nk)), dim3(256), 0, st, pos_src, B, pos_dst, B, neg_dst, nk, neg_src, (k > 0 && neg_src) ? nk : 0, ctx->n, ctx->err_flag,
-                   ctx->inc_ptr, ctx->inc_cap, ctx->plan_dyn.counts);
+        const bool w16 = ctx->desc.prec == LP_BF16 && ctx->w16;
+        const unsigned id_blocks = nblk(2 * B + 2 * nk), w_blocks = w16 ? nblk(ctx->n_params) : 0u;
+        launch_dep(check_step_ids_kernel, dim3(id_blocks + w_blocks), dim3(256), 0, st, pos_src, B, pos_dst, B, neg_dst, nk, neg_src, (k > 0 && neg_src) ? nk : 0, ctx->n,
+                   ctx->err_flag, ctx->inc_ptr, ctx->inc_cap, ctx->plan_dyn.counts, (int)id_blocks, params, (long long)ctx->n_params, weight_blocks(ctx), ctx->w16, ctx->w16t,
+                   ctx->w16s);
         ctx->ex.launches += 1;
     }
-    cache_weights(ctx, params);
     if (ctx->sampled) {
         lp_status s = build_blocks(ctx, pos_src, pos_dst, B, neg_src, neg_dst, k, seed, step);
         if (s != LP_OK) return s;

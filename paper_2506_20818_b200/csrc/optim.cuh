@@ -70,11 +70,9 @@ struct WeightBlocks {
     long long off[8];
     int kin[8], fo[8], split[8];
 };
-__global__ void weights_cache_kernel(const float *__restrict__ params, long long n, WeightBlocks blocks, bf16 *__restrict__ asis, bf16 *__restrict__ transposed,
-                                     bf16 *__restrict__ stacked)
+LP_DEVINL void weights_cache_element(long long i, const float *__restrict__ params, long long n, const WeightBlocks &blocks, bf16 *__restrict__ asis,
+                                     bf16 *__restrict__ transposed, bf16 *__restrict__ stacked)
 {
-    LP_DEP_ENTER();
-    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     const bf16 x = __float2bfloat16_rn(params[i]);
     asis[i] = x;
@@ -94,4 +92,10 @@ __global__ void weights_cache_kernel(const float *__restrict__ params, long long
         }
     }
     transposed[dst] = x;
+}
+__global__ void weights_cache_kernel(const float *__restrict__ params, long long n, WeightBlocks blocks, bf16 *__restrict__ asis, bf16 *__restrict__ transposed,
+                                     bf16 *__restrict__ stacked)
+{
+    LP_DEP_ENTER();
+    weights_cache_element((long long)blockIdx.x * blockDim.x + threadIdx.x, params, n, blocks, asis, transposed, stacked);
 }
