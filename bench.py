@@ -39,12 +39,12 @@ K_NEG = 1
 SEED = 1234
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the aggregation launches of one step on the
-# benchmark workload, from one ncu capture of a whole step at full size (layer-1 forward 124.4 MB, layer-2 forward
-# 410.1 MB, adjoint 406.3 MB): mean per timed launch.  Valid only for the kernel source it was taken with (sha1 of
+# benchmark workload, from one ncu capture of a whole step at full size (layer-1 forward 124.1 MB, layer-2 forward
+# 409.5 MB, adjoint 406.3 MB): mean per timed launch.  Valid only for the kernel source it was taken with (sha1 of
 # csrc/spmm.cuh + csrc/common.cuh); reported as null otherwise.
-NCU_TRAFFIC = {"spmm_sha1": "21f81b0744e85bd57ea98b3430d3f96add0200c8", "bytes_per_launch": (124.4e6 + 410.1e6 + 406.3e6) / 3.0,
-               # the forward mean aggregation (F = 256, BF16) on the 1 M-node graph of the HBM-bound roofline run: 3415.1 MB read + 559.8 MB written
-               "hbm_forward_bytes_per_launch": 3415.1e6 + 559.8e6}
+NCU_TRAFFIC = {"spmm_sha1": "78f78a3c22a0f25d5b0710a2e5a8e287eb3db256", "bytes_per_launch": (124.1e6 + 409.5e6 + 406.3e6) / 3.0,
+               # the forward mean aggregation (F = 256, BF16) on the 1 M-node graph of the HBM-bound roofline run: 3414.8 MB read + 560.8 MB written
+               "hbm_forward_bytes_per_launch": 3414.8e6 + 560.8e6}
 
 
 def measured_peaks():
