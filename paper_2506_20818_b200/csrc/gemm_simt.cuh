@@ -94,14 +94,14 @@ __global__ void reduce_partials_kernel(const float *__restrict__ partials, int64
     if (i >= count) return;
     float s = 0.f;
     int z = 0;
-    for (; z + 8 <= splits; z += 8) {  // eight independent loads in flight, added in index order
-        float v[8];
+    for (; z < splits; z += 16) {  // sixteen independent loads in flight (the last batch predicated), added in index order
+        float v[16];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) v[q] = __ldg(partials + (int64_t)(z + q) * count + i);
+        for (int q = 0; q < 16; ++q) v[q] = z + q < splits ? __ldg(partials + (int64_t)(z + q) * count + i) : 0.f;
 #pragma unroll
-        for (int q = 0; q < 8; ++q) s += v[q];
+        for (int q = 0; q < 16; ++q)
+            if (z + q < splits) s += v[q];
     }
-    for (; z < splits; ++z) s += __ldg(partials + (int64_t)z * count + i);
     dst[i] = accumulate ? dst[i] + s : s;
 }
 
