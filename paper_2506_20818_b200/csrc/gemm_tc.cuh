@@ -1023,11 +1023,22 @@ static void tc_destroy(TcState &tc)
 
 // Reads the device error word.  `synced` = the stream has already been synchronised by the caller;
 // otherwise the word is only inspected when the caller asks for a synchronising check.
+// the error word of the bounded waits: requested on the stream (tc_check_enqueue), read after the caller's own synchronise
+// (tc_check_result), or both at once with a synchronise in between (tc_check)
+static bool tc_check_enqueue(TcState &tc, Exec &ex)
+{
+    return cudaMemcpyAsync(tc.host_err, tc.err_word, sizeof(int), cudaMemcpyDeviceToHost, ex.st) == cudaSuccess;
+}
+static lp_status tc_check_result(TcState &tc, Exec &ex, std::string &err);
 static lp_status tc_check(TcState &tc, Exec &ex, bool synced, std::string &err)
 {
     if (!synced) return LP_OK;
-    if (cudaMemcpyAsync(tc.host_err, tc.err_word, sizeof(int), cudaMemcpyDeviceToHost, ex.st) != cudaSuccess) return LP_OK;
+    if (!tc_check_enqueue(tc, ex)) return LP_OK;
     cudaStreamSynchronize(ex.st);
+    return tc_check_result(tc, ex, err);
+}
+static lp_status tc_check_result(TcState &tc, Exec &ex, std::string &err)
+{
     if (*tc.host_err != 0) {
         char buf[128];
         snprintf(buf, sizeof buf, "tensor-core GEMM: bounded wait %d expired (1 = stage free, 2 = operands, 3 = accumulator, 4 = operands for the column sums)", *tc.host_err);

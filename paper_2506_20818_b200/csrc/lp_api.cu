@@ -1695,15 +1695,18 @@ extern "C" lp_status lp_train_step_host(lp_ctx *ctx, float *params, const int32_
     }
     CK(cudaMemcpyAsync(loss_host, ctx->d_loss_tmp, sizeof(float), cudaMemcpyDeviceToHost, st));
     if (grads_host) CK(cudaMemcpyAsync(grads_host, ctx->d_grads_tmp, sizeof(float) * (size_t)ctx->n_params, cudaMemcpyDeviceToHost, st));
-    int bad = 0;
-    CK(cudaMemcpyAsync(&bad, ctx->err_flag, sizeof bad, cudaMemcpyDeviceToHost, st));
+    // both error words travel with the loss: one synchronise for the whole call (the words land in pinned memory)
+    int *bad = ctx->host_counts + 32;
+    *bad = 0;
+    CK(cudaMemcpyAsync(bad, ctx->err_flag, sizeof(int), cudaMemcpyDeviceToHost, st));
+    const bool tc_asked = tc_check_enqueue(ctx->tc, ctx->ex);
     CK(cudaStreamSynchronize(st));
-    if (bad) {
+    if (*bad) {
         cudaMemsetAsync(ctx->err_flag, 0, sizeof(int), st);
-        if (bad & 2) return fail(ctx, LP_ETIMEOUT, "lp_train_step_host: a bounded wait inside the scan of the step expired");
+        if (*bad & 2) return fail(ctx, LP_ETIMEOUT, "lp_train_step_host: a bounded wait inside the scan of the step expired");
         return fail(ctx, LP_EINVAL, "lp_train_step_host: a node id is outside [0, n)");
     }
-    return tc_check(ctx->tc, ctx->ex, true, ctx->err);
+    return tc_asked ? tc_check_result(ctx->tc, ctx->ex, ctx->err) : LP_OK;
 }
 
 template <typename T>
