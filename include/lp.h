@@ -314,10 +314,10 @@ enum {
     LP_PROF_AGG_FWD = 0,   /* neighbour aggregation, forward (Eq. 1 AGG)                    */
     LP_PROF_AGG_BWD = 1,   /* its adjoint over the transposed structure                     */
     LP_PROF_GEMM_FWD = 2,  /* dense transform Z = A W + b (Eq. 1 UPDATE)                    */
-    LP_PROF_GEMM_DGRAD = 3,/* dA = dZ W^T                                                   */
+    LP_PROF_GEMM_DGRAD = 3,/* dA = dZ W^T, or dH = [dZ | A^T dZ] [W_self^T ; W_neigh^T]         */
     LP_PROF_GEMM_WGRAD = 4,/* dW = A^T dZ and db                                            */
-    LP_PROF_SCORE = 5,     /* edge scores, loss, per-edge gradients (Eq. 2, Algorithm 1)    */
-    LP_PROF_INCIDENCE = 6, /* grouping the scored edges by node (integer sort)              */
+    LP_PROF_SCORE = 5,     /* edge scores, loss partials, per-edge gradients (Eq. 2, Alg. 1) */
+    LP_PROF_INCIDENCE = 6, /* grouping the scored edges by node; final loss reduction        */
     LP_PROF_SCATTER = 7,   /* dL/dH^(K) gathered per node                                   */
     LP_PROF_NEGATIVES = 8, /* negative sampling                                             */
     LP_PROF_BLOCKS = 9,    /* neighbour sampling and block construction                     */
